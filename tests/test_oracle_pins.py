@@ -1,0 +1,536 @@
+"""Pins for the CPU oracle: closed forms, library routines, brute force on tiny
+inputs and the invariants the paper fixes.  No GPU needed."""
+import math
+import os
+import re
+
+import numpy as np
+import pytest
+import torch
+
+import bs_inputs
+from oracle import blockserve_oracle as O
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+F32 = np.float32
+
+
+def tiny_model(shape=None, seed=7):
+    shape = shape or bs_inputs.ModelShape("t", 2, 32, 4, 2, 8, 48, 50, init_std=0.3)
+    w = bs_inputs.weights_to_numpy_f32(bs_inputs.make_weights(shape, seed))
+    return shape, O.model_from_weights(shape, w)
+
+
+# ----------------------------------------------------------------- formulas ---
+
+def test_block_count_golden():
+    # K_i = ceil(g_i / L), Section 2.1
+    for line in open(os.path.join(GOLDEN, "block_count.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        g, L, K = map(int, line.split())
+        r = O.ReqState(0, 5, g, 1.0, np.zeros(5 + g, np.int32), 0)
+        assert r.n_blocks(L) == K
+
+
+def test_eq1_cost_golden():
+    # Eq. 1, Section 2.4
+    for line in open(os.path.join(GOLDEN, "eq1_cost.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        L, pairs, widths, cost = [s.strip() for s in line.split(";")]
+        L = int(L)
+        pb = [tuple(map(int, m)) for m in re.findall(r"\((\d+),(\d+)\)", pairs)]
+        rs = [O.ReqState(i, p, 1024, 1.0, np.zeros(1, np.int32), b) for i, (p, b) in enumerate(pb)]
+        assert [r.width(L) for r in rs] == list(map(int, widths.split()))
+        assert O.batch_cost([r.width(L) for r in rs]) == int(cost)
+    assert O.batch_cost([]) == 0
+
+
+def test_rmsnorm_closed_form_and_library():
+    # x = c * 1  =>  y = w * c / sqrt(c^2 + eps)
+    w = np.linspace(0.5, 1.5, 16).astype(F32)
+    y = O.rmsnorm(np.full((1, 16), 3.0, F32), w, 1e-6)
+    np.testing.assert_allclose(y[0], w * 3.0 / math.sqrt(9.0 + 1e-6), rtol=1e-6)
+    x = np.random.default_rng(0).normal(size=(5, 16)).astype(F32)
+    ref = torch.nn.functional.rms_norm(torch.from_numpy(x).double(), (16,), torch.from_numpy(w).double(), 1e-6)
+    np.testing.assert_allclose(O.rmsnorm(x, w, 1e-6), ref.numpy(), rtol=1e-5, atol=1e-6)
+
+
+def test_silu_values():
+    np.testing.assert_allclose(O.silu(np.array([0.0, 1.0, -1.0], F32)),
+                               [0.0, 0.7310586, -0.26894143], rtol=1e-6, atol=1e-7)
+    x = np.linspace(-6, 6, 41).astype(F32)
+    np.testing.assert_allclose(O.silu(x), torch.nn.functional.silu(torch.from_numpy(x).double()).numpy(),
+                               rtol=1e-5, atol=1e-6)
+
+
+def test_rope_closed_form_pairing_and_norm():
+    # 2-dim head: q = (1, 0) at position m becomes (cos m, sin m) (theta_0 = 1)
+    pos = np.array([0, 1, 5, 77])
+    cos, sin = O.rope_cos_sin(pos, 2, 10000.0)
+    q = np.tile(np.array([1.0, 0.0], F32), (4, 1, 1))
+    out = O.apply_rope(q, cos, sin)
+    np.testing.assert_allclose(out[:, 0, 0], np.cos(pos), atol=1e-6)
+    np.testing.assert_allclose(out[:, 0, 1], np.sin(pos), atol=1e-6)
+    # head_dim 8: pair (j, j+4) turns by pos * theta^(-2j/8); a unit vector on dim 1 lands on dims (1, 5)
+    cos, sin = O.rope_cos_sin(np.array([3]), 8, 10000.0)
+    e1 = np.zeros((1, 1, 8), F32)
+    e1[0, 0, 1] = 1.0
+    out = O.apply_rope(e1, cos, sin)[0, 0]
+    ang = 3.0 * 10000.0 ** (-2.0 / 8.0)
+    expect = np.zeros(8)
+    expect[1], expect[5] = math.cos(ang), math.sin(ang)
+    np.testing.assert_allclose(out, expect, atol=1e-6)
+    # rotations preserve norms and <q_m, k_n> depends on m - n only
+    rng = np.random.default_rng(1)
+    qv, kv = rng.normal(size=(1, 1, 8)).astype(F32), rng.normal(size=(1, 1, 8)).astype(F32)
+    def dot(m, n):
+        cq, sq = O.rope_cos_sin(np.array([m]), 8, 10000.0)
+        ck, sk = O.rope_cos_sin(np.array([n]), 8, 10000.0)
+        return float((O.apply_rope(qv, cq, sq) * O.apply_rope(kv, ck, sk)).sum())
+    assert abs(dot(10, 3) - dot(107, 100)) < 1e-4
+    assert abs(dot(10, 3) - dot(3, 10)) > 1e-3      # direction matters
+
+
+def brute_attention(q, k, v):
+    """softmax(q k^T / sqrt(dh)) v by scalar loops in double; kv head = h // group."""
+    nq, hq, dh = q.shape
+    nk, hkv, _ = k.shape
+    out = np.zeros((nq, hq, dh))
+    for i in range(nq):
+        for h in range(hq):
+            kh = h // (hq // hkv)
+            sc = [sum(float(q[i, h, c]) * float(k[j, kh, c]) for c in range(dh)) / math.sqrt(dh)
+                  for j in range(nk)]
+            m = max(sc)
+            e = [math.exp(s - m) for s in sc]
+            z = sum(e)
+            for c in range(dh):
+                out[i, h, c] = sum(e[j] * float(v[j, kh, c]) for j in range(nk)) / z
+    return out
+
+
+def test_attention_brute_force_and_library():
+    rng = np.random.default_rng(2)
+    q = rng.normal(size=(5, 4, 8)).astype(F32)
+    k = rng.normal(size=(11, 2, 8)).astype(F32)
+    v = rng.normal(size=(11, 2, 8)).astype(F32)
+    got = O.attention(q, k, v)
+    np.testing.assert_allclose(got, brute_attention(q, k, v), rtol=1e-5, atol=1e-6)
+    # GQA == MHA with K/V heads replicated; library SDPA as a second opinion
+    kr, vr = np.repeat(k, 2, axis=1), np.repeat(v, 2, axis=1)
+    np.testing.assert_allclose(O.attention(q, kr, vr), got, rtol=1e-6, atol=1e-7)
+    t = lambda a: torch.from_numpy(a).double().permute(1, 0, 2)[None]
+    ref = torch.nn.functional.scaled_dot_product_attention(t(q), t(kr), t(vr))[0].permute(1, 0, 2).numpy()
+    np.testing.assert_allclose(got, ref, rtol=1e-5, atol=1e-6)
+    # not causal: the first query sees the last key
+    v2 = v.copy()
+    v2[-1] += 10.0
+    assert np.abs(O.attention(q, k, v2)[0] - got[0]).max() > 1e-2
+
+
+def test_confidence_special_cases():
+    V, mask_id = 50, 49
+    z = np.zeros((1, V), F32)
+    tok, conf = O.confidence(z, mask_id)
+    assert tok[0] == 0 and abs(conf[0] - 1.0 / (V - 1)) < 1e-7     # mask id excluded from the softmax
+    z[0, 17] = 100.0
+    tok, conf = O.confidence(z, mask_id)
+    assert tok[0] == 17 and abs(conf[0] - 1.0) < 1e-6
+    z[0, mask_id] = 1000.0                                          # the mask id can never win
+    tok, conf = O.confidence(z, mask_id)
+    assert tok[0] == 17 and abs(conf[0] - 1.0) < 1e-6
+    z = np.zeros((1, V), F32)
+    z[0, 30] = z[0, 12] = 5.0                                       # tie -> lowest id
+    assert O.confidence(z, mask_id)[0][0] == 12
+    rng = np.random.default_rng(3)
+    z = (rng.normal(size=(6, V)) * 4).astype(F32)
+    tok, conf = O.confidence(z, mask_id)
+    zz = torch.from_numpy(z).double()
+    zz[:, mask_id] = -float("inf")
+    ref = torch.exp(zz.max(-1).values - torch.logsumexp(zz, -1)).numpy()
+    np.testing.assert_allclose(conf, ref, rtol=1e-5)
+    assert (tok == zz.argmax(-1).numpy()).all()
+
+
+def test_commit_set_rule():
+    c = np.array([0.2, 0.95, 0.5, 0.91], F32)
+    assert O.commit_set(c.copy(), 0.9).tolist() == [False, True, False, True]
+    assert O.commit_set(c.copy(), 0.99).tolist() == [False, True, False, False]   # forced pick
+    assert O.commit_set(np.array([0.3, 0.7, 0.7], F32), 0.9).tolist() == [False, True, False]  # tie -> lowest
+    assert O.commit_set(np.array([1.0, 1.0], F32), 1.0).tolist() == [True, False]   # strict >
+
+
+# ---------------------------------------------------------- model forward ---
+
+def brute_forward(shape, w, tokens, alpha):
+    """A from-scratch forward in double precision with torch primitives of a
+    different kind (einsum on explicitly replicated heads, complex-number RoPE)."""
+    d, hq, hkv, dh = shape.d_model, shape.n_q_heads, shape.n_kv_heads, shape.head_dim
+    T = lambda a: torch.from_numpy(np.asarray(a)).double()
+    n = len(tokens)
+    x = T(w["embed"])[torch.as_tensor(tokens, dtype=torch.long)]
+    pos = torch.arange(n).double()
+    inv = shape.rope_theta ** (-torch.arange(0, dh, 2).double() / dh)
+    rot = torch.polar(torch.ones(n, dh // 2).double(), pos[:, None] * inv[None, :])   # e^{i pos theta_j}
+
+    def rope(t):    # t [n, H, dh]; complex pairing of (j, j + dh/2)
+        c = torch.complex(t[..., :dh // 2], t[..., dh // 2:]) * rot[:, None, :]
+        return torch.cat([c.real, c.imag], -1)
+
+    def norm(t, g):
+        return t * torch.rsqrt((t * t).mean(-1, keepdim=True) + shape.rms_eps) * T(g)
+
+    for l in range(shape.n_layers):
+        h = norm(x, w["norm1"][l])
+        qkv = torch.einsum("nd,od->no", h, T(w["wqkv"][l]))
+        q = rope(qkv[:, :hq * dh].reshape(n, hq, dh))
+        k = rope(qkv[:, hq * dh:(hq + hkv) * dh].reshape(n, hkv, dh))
+        v = qkv[:, (hq + hkv) * dh:].reshape(n, hkv, dh)
+        k, v = k.repeat_interleave(hq // hkv, 1), v.repeat_interleave(hq // hkv, 1)
+        pr = torch.softmax(torch.einsum("ihc,jhc->hij", q, k) / math.sqrt(dh), -1)
+        a = torch.einsum("hij,jhc->ihc", pr, v).reshape(n, hq * dh)
+        x = x + torch.einsum("nk,dk->nd", a, T(w["wo"][l]))
+        h2 = norm(x, w["norm2"][l])
+        gate = torch.einsum("nd,fd->nf", h2, T(w["w_gate"][l]))
+        up = torch.einsum("nd,fd->nf", h2, T(w["w_up"][l]))
+        x = x + torch.einsum("nf,df->nd", gate * torch.sigmoid(gate) * up, T(w["w_down"][l]))
+    return (alpha * torch.einsum("nd,vd->nv", norm(x, w["final_norm"]), T(w["lm_head"]))).numpy()
+
+
+def test_full_forward_against_independent_double_forward():
+    shape = bs_inputs.ModelShape("t", 3, 32, 4, 2, 8, 48, 50, init_std=0.3)
+    w = bs_inputs.weights_to_numpy_f32(bs_inputs.make_weights(shape, 11))
+    model = O.model_from_weights(shape, w)
+    toks = np.random.default_rng(4).integers(0, 49, size=13)
+    got = O.full_forward_logits(model, toks, 2.5)
+    ref = brute_forward(shape, w, toks, 2.5)
+    np.testing.assert_allclose(got, ref, rtol=2e-4, atol=2e-4)
+
+
+def test_position_shift_leaves_logits_unchanged():
+    # relative-distance property behind the explicit position ids of Section 2.5
+    shape, model = tiny_model()
+    toks = np.random.default_rng(5).integers(0, 49, size=9).astype(np.int32)
+    base = O.full_forward_logits(model, toks, 1.0)
+    orig = O.rope_cos_sin
+    try:
+        O.rope_cos_sin = lambda pos, dh, th: orig(pos + 37, dh, th)
+        shifted = O.full_forward_logits(model, toks, 1.0)
+    finally:
+        O.rope_cos_sin = orig
+    np.testing.assert_allclose(shifted, base, rtol=1e-3, atol=1e-4)
+
+
+def _mk_req(model, p, g, L, alpha=4.0, seed=0, start=0):
+    rng = np.random.default_rng(seed)
+    prompt = rng.integers(0, model.vocab - 1, size=p)
+    prefix = rng.integers(0, model.vocab - 1, size=start * L) if start else None
+    r = O.new_request(model, seed, prompt, g, alpha, L, start, prefix)
+    r.kv_base = 0
+    O.start_block_state(r, L)
+    return r
+
+
+@pytest.mark.parametrize("suffix_mode", [O.SUFFIX_FULL, O.SUFFIX_NONE])
+def test_refresh_step_equals_cacheless_forward(suffix_mode):
+    shape, model = tiny_model()
+    L = 4
+    r = _mk_req(model, 6, 12, L, start=1)
+    vis = r.vis(L, suffix_mode)
+    rec = O.denoise_step(model, r, L, 0.9, suffix_mode, keep_logits=True)
+    assert vis == (18 if suffix_mode == O.SUFFIX_FULL else 6 + 2 * L)
+    # the row as it was before the commit: block fully masked
+    row = r.tokens[:vis].copy()
+    row[rec.positions] = model.mask_id
+    ref = O.full_forward_logits(model, row, r.alpha)[rec.positions]
+    np.testing.assert_allclose(rec.logits, ref, rtol=1e-5, atol=1e-6)
+
+
+def test_cached_step_exact_for_one_layer_and_approximate_for_two():
+    L = 4
+    for n_layers, expect_exact in ((1, True), (2, False)):
+        shape = bs_inputs.ModelShape("t", n_layers, 32, 4, 2, 8, 48, 50, init_std=0.5)
+        w = bs_inputs.weights_to_numpy_f32(bs_inputs.make_weights(shape, 5))
+        model = O.model_from_weights(shape, w)
+        r = _mk_req(model, 5, 8, L, alpha=1.0)
+        O.denoise_step(model, r, L, 1.0)                      # refresh, commits exactly one token
+        row = r.tokens.copy()
+        rec = O.denoise_step(model, r, L, 1.0, keep_logits=True)     # cached block step
+        ref = O.full_forward_logits(model, row, r.alpha)[rec.positions]
+        err = np.abs(rec.logits - ref).max() / np.abs(ref).max()
+        if expect_exact:
+            assert err < 1e-5
+        else:
+            assert err > 1e-4          # stale prefix / suffix K,V: the dual cache is an approximation
+    # and right after the next refresh the two agree again (n_layers = 2 model from the loop)
+    while r.mask:
+        O.denoise_step(model, r, L, 1.0)
+    r.b += 1
+    O.start_block_state(r, L)
+    row = r.tokens.copy()
+    rec = O.denoise_step(model, r, L, 1.0, keep_logits=True)
+    ref = O.full_forward_logits(model, row, r.alpha)[rec.positions]
+    np.testing.assert_allclose(rec.logits, ref, rtol=1e-5, atol=1e-6)
+
+
+def test_kv_written_only_at_query_rows():
+    shape, model = tiny_model()
+    L = 4
+    r = _mk_req(model, 5, 12, L, alpha=1.0)
+    O.denoise_step(model, r, L, 1.0)
+    before = [k.copy() for k in r.K]
+    O.denoise_step(model, r, L, 1.0)
+    lo, hi = r.block_range(L)
+    for l in range(model.n_layers):
+        changed = np.abs(r.K[l] - before[l]).reshape(len(before[l]), -1).max(-1) > 0
+        assert not changed[:lo].any() and not changed[hi:].any()     # prefix and suffix stay frozen
+    assert any((np.abs(r.K[l] - before[l]) > 0).any() for l in range(1, model.n_layers))
+
+
+# ------------------------------------------------------ decoding invariants ---
+
+def run_engine(model, reqs, L, tau, beta=0, max_batch=8, cap=1 << 20, suffix=O.SUFFIX_FULL, sort=True):
+    e = O.Engine(model, L, tau, beta, max_batch, cap, suffix, sort)
+    for q in reqs:
+        e.admit(*q)
+    return e
+
+
+def test_tau_one_commits_exactly_the_top_confidence_token_per_step():
+    shape, model = tiny_model()
+    L = 4
+    r = _mk_req(model, 5, 8, L, alpha=3.0)
+    for step in range(L):
+        n_before = bin(r.mask).count("1")
+        rec = O.denoise_step(model, r, L, 1.0)
+        assert rec.committed.sum() == 1
+        assert rec.committed[int(np.argmax(rec.conf))]
+        assert bin(r.mask).count("1") == n_before - 1
+    assert r.mask == 0 and r.s == L
+
+
+def test_tau_zero_finishes_every_block_in_one_step_with_refresh_argmax():
+    shape, model = tiny_model()
+    L = 4
+    r = _mk_req(model, 5, 8, L, alpha=0.5)
+    row = r.tokens.copy()
+    rec = O.denoise_step(model, r, L, 0.0)
+    assert r.mask == 0 and rec.committed.all()
+    ref = O.full_forward_logits(model, row, r.alpha)[rec.positions]
+    ref[:, model.mask_id] = -np.inf
+    assert (r.tokens[rec.positions] == ref.argmax(-1)).all()
+
+
+@pytest.mark.parametrize("suffix_mode", [O.SUFFIX_FULL, O.SUFFIX_NONE])
+def test_lifetime_token_counts_and_step_bounds(suffix_mode):
+    shape, model = tiny_model()
+    L = 4
+    rng = np.random.default_rng(9)
+    spec = [(0, 5, 10, 0.5, 0), (1, 9, 8, 6.0, 1), (2, 3, 16, 30.0, 2), (3, 7, 4, 2.0, 0), (4, 4, 7, 9.0, 0)]
+    reqs = []
+    for rid, p, g, a, st in spec:
+        reqs.append((rid, rng.integers(0, 49, size=p), g, a, st,
+                     rng.integers(0, 49, size=st * L) if st else None))
+    e = run_engine(model, reqs, L, 0.9, max_batch=3, suffix=suffix_mode)
+    cycles_seen = {rid: 0 for rid, *_ in spec}
+    while True:
+        ev, ad, n = e.evict_refill()
+        if n == 0:
+            break
+        for r in e.sched.active:
+            cycles_seen[r.req_id] += 1
+        steps = 0
+        while not e.block_done():
+            recs = e.denoise_step()
+            assert all(rec.committed.sum() >= 1 for rec in recs)       # >= 1 commit per step
+            steps += 1
+        assert steps <= L                                               # <= L steps per block
+    for rid, p, g, a, st in spec:
+        r = e.by_id[rid]
+        K = -(-g // L)
+        assert cycles_seen[rid] == K - st                               # leaves exactly at b_i >= K_i
+        assert r.committed == g - st * L                                # exactly g_i tokens
+        assert (r.tokens != model.mask_id).all()
+    assert e.total_committed == sum(g - st * L for _, _, g, _, st in spec)
+
+
+def test_request_is_independent_of_its_batch():
+    shape, model = tiny_model()
+    L = 4
+    rng = np.random.default_rng(10)
+    reqs = [(i, rng.integers(0, 49, size=p), g, a, 0, None)
+            for i, (p, g, a) in enumerate([(5, 8, 3.0), (11, 12, 8.0), (2, 4, 1.0), (8, 8, 20.0)])]
+    together = run_engine(model, reqs, L, 0.9, max_batch=2)
+    together.run()
+    for q in reqs:
+        alone = run_engine(model, [q], L, 0.9)
+        alone.run()
+        assert (alone.tokens(q[0]) == together.tokens(q[0])).all()
+        assert alone.by_id[q[0]].steps == together.by_id[q[0]].steps
+
+
+# ------------------------------------------------------------- scheduler ---
+
+def sched_req(rid, p, g, b=0):
+    return O.ReqState(rid, p, g, 1.0, np.zeros(p + g, np.int32), b)
+
+
+def drain(s, L):
+    """Model-free run of Algorithm 1 (every block finishes, nothing else matters)."""
+    order = []
+    while True:
+        ev, ad = s.evict_refill()
+        order.append((list(ev), list(ad), [r.req_id for r in s.active]))
+        if not s.active:
+            break
+        for r in s.active:
+            r.mask = 0
+    return order
+
+
+def test_admission_invariants_and_sorted_prefix():
+    L = 32
+    rng = np.random.default_rng(12)
+    s = O.Scheduler(L, 4000, 64, 1 << 20)
+    ps = rng.integers(10, 400, size=40)
+    for i, p in enumerate(ps):
+        s.submit(sched_req(i, int(p), 64 * int(rng.integers(1, 4))))
+    sorted_ids = [r.req_id for r in s.pending]
+    assert [s.pending[i].p for i in range(40)] == sorted(ps.tolist())
+    admitted_all = []
+    while True:
+        prev = [r.req_id for r in s.active]
+        ev, ad = s.evict_refill()
+        admitted_all += ad
+        ids = [r.req_id for r in s.active]
+        survivors = [i for i in prev if i not in ev]
+        assert ids == survivors + ad                      # stable compaction, new rows appended in queue order
+        widths = [r.width(L) for r in s.active]
+        if ad:                                            # Eq. 1 holds whenever something was admitted
+            assert O.batch_cost(widths) <= 4000
+        assert len(ids) <= 64
+        if s.pending and len(ids) < 64:                   # the head was refused only because it does not fit
+            c = s.pending[0]
+            assert O.batch_cost(widths + [c.width(L)]) > 4000
+        if not ids:
+            break
+        for r in s.active:
+            r.mask = 0
+    assert admitted_all == sorted_ids                      # admitted set is always a prefix of sorted P
+    assert len(s.trace) <= sum(-(-r.g // L) for r in s.finished) + 1
+
+
+def test_unlimited_budget_admits_everything_and_R_tends_to_one():
+    L = 32
+    s = O.Scheduler(L, 0, 1000, 1 << 24)
+    for i in range(50):
+        s.submit(sched_req(i, 10 + i, 64))
+    ev, ad = s.evict_refill()
+    assert len(ad) == 50
+    # fixed cap B with a long queue keeps the batch full: R -> 1 (Eq. 2)
+    s = O.Scheduler(L, 0, 4, 1 << 24)
+    for i in range(200):
+        s.submit(sched_req(i, 10 + (i * 7) % 90, 32 * (1 + i % 3)))
+    drain(s, L)
+    assert 0.97 < s.effective_compute_ratio(4) <= 1.0
+
+
+def test_bounding_box_shrinks_when_the_widest_row_leaves():
+    # Fig. 1, example 2: evicting the widest request frees budget for more admissions
+    L = 32
+    s = O.Scheduler(L, 3 * 232, 16, 1 << 20, sort_queue=False)
+    s.submit(sched_req(0, 200, 32))        # width 232, one block
+    s.submit(sched_req(1, 20, 128))
+    s.submit(sched_req(2, 30, 128))
+    for i in range(3, 9):
+        s.submit(sched_req(i, 25, 64))
+    ev, ad = s.evict_refill()
+    assert ad == [0, 1, 2] and s.trace[-1].width == 232           # 4 * 232 > budget
+    for r in s.active:
+        r.mask = 0
+    ev, ad = s.evict_refill()
+    assert ev == [0]
+    assert s.trace[-1].width < 232 and len(s.active) > 3           # box shrank, batch grew
+    assert s.trace[-1].cost <= 3 * 232
+
+
+def test_too_wide_request_is_rejected_and_first_fit():
+    s = O.Scheduler(32, 100, 4, 1000)
+    with pytest.raises(ValueError):
+        s.submit(sched_req(0, 90, 32))
+    assert O.first_fit([], 10, 100) == 0
+    assert O.first_fit([(0, 10), (30, 10)], 20, 100) == 10
+    assert O.first_fit([(0, 10), (30, 10)], 21, 100) == 40
+    assert O.first_fit([(0, 10), (30, 10)], 61, 100) == -1
+    assert O.first_fit([(5, 10)], 5, 100) == 0
+
+
+def test_kv_slabs_never_overlap_and_survivors_keep_theirs():
+    L = 32
+    rng = np.random.default_rng(13)
+    s = O.Scheduler(L, 0, 6, 2500)
+    for i in range(30):
+        s.submit(sched_req(i, int(rng.integers(5, 300)), 32 * int(rng.integers(1, 5))))
+    base_of = {}
+    while True:
+        s.evict_refill()
+        if not s.active:
+            break
+        spans = sorted((r.kv_base, r.kv_base + r.p + r.g) for r in s.active)
+        assert all(a[1] <= b[0] for a, b in zip(spans, spans[1:])) and spans[-1][1] <= 2500
+        for r in s.active:
+            assert base_of.setdefault(r.req_id, r.kv_base) == r.kv_base
+            r.mask = 0
+    assert len(s.finished) == 30
+
+
+# -------------------------------------------------------- index builder ---
+
+def test_build_indices_hand_example():
+    L = 4
+    a = O.ReqState(0, 3, 8, 1.0, np.zeros(11, np.int32), 1, s=2, mask=0b0101, kv_base=100)   # block step
+    b = O.ReqState(1, 2, 4, 1.0, np.zeros(6, np.int32), 0, s=0, mask=0b1111, kv_base=0)      # refresh
+    c = O.ReqState(2, 5, 4, 1.0, np.zeros(9, np.int32), 0, s=3, mask=0, kv_base=50)          # block done
+    ix = O.build_indices([a, b, c], L)
+    assert ix["cu_q"].tolist() == [0, 4, 10, 10]
+    assert ix["tok_row"].tolist() == [0] * 4 + [1] * 6
+    assert ix["tok_pos"].tolist() == [7, 8, 9, 10, 0, 1, 2, 3, 4, 5]       # position 0 = first prompt token
+    assert ix["tok_kv"].tolist() == [107, 108, 109, 110, 0, 1, 2, 3, 4, 5]
+    assert ix["lm_tok"].tolist() == [0, 2, 6, 7, 8, 9]
+    assert ix["lm_row"].tolist() == [0, 0, 1, 1, 1, 1]
+    assert ix["lm_slot"].tolist() == [0, 2, 0, 1, 2, 3]
+    ix = O.build_indices([b], L, O.SUFFIX_NONE)
+    assert ix["cu_q"].tolist() == [0, 6]
+    b2 = O.ReqState(1, 2, 8, 1.0, np.zeros(10, np.int32), 0, s=0, mask=0b1111, kv_base=0)
+    assert O.build_indices([b2], L, O.SUFFIX_NONE)["cu_q"].tolist() == [0, 6]      # future blocks invisible
+    assert O.build_indices([b2], L, O.SUFFIX_FULL)["cu_q"].tolist() == [0, 10]
+
+
+def test_ragged_last_block():
+    shape, model = tiny_model()
+    L = 4
+    e = run_engine(model, [(0, np.arange(5), 6, 5.0, 0, None)], L, 0.9)
+    assert e.run() == 2
+    r = e.by_id[0]
+    assert r.committed == 6 and (r.tokens != model.mask_id).all()
+
+
+def test_workload_generators_match_the_stated_shapes():
+    w1 = bs_inputs.workload(1)
+    assert [r.p for r in w1.requests[:4]] == [17, 40, 63, 9] and [r.start_block for r in w1.requests[:4]] == [0, 1, 2, 0]
+    assert all(r.g == 96 for r in w1.requests) and w1.max_batch == 4 and len(w1.requests) == 8
+    assert all(r.prompt.max() <= 1022 for r in w1.requests)
+    w2 = bs_inputs.workload(2)
+    assert len(w2.requests) == 16 and all(64 <= r.p <= 512 and 0 <= r.start_block <= 7 for r in w2.requests)
+    assert all(len(r.gen_prefix) == r.start_block * 32 for r in w2.requests if r.start_block)
+    w3 = bs_inputs.workload(3)
+    ps = np.array([r.p for r in w3.requests])
+    assert len(ps) == 256 and ps.min() >= 32 and ps.max() <= 1024 and 190 < ps.mean() < 250 and 60 < ps.std() < 120
+    w4 = bs_inputs.workload(4)
+    assert len(w4.requests) == 128 and all(1024 <= r.p <= 2048 and r.g == 512 for r in w4.requests)
+    w5 = bs_inputs.workload(5)
+    al = np.array([r.alpha for r in w5.requests])
+    assert len(al) == 1024 and set(np.unique(al)) == {0.7, 16.0} and 0.75 < (al == 16.0).mean() < 0.85
+    assert {r.g for r in w5.requests} == {128, 256, 512}
