@@ -1,0 +1,202 @@
+/*
+ * blockserve.h - C ABI of the B200 (sm_100a) mixed-state block-denoising engine.
+ *
+ * The calls follow the paper's problem formulation (Section 2.1: requests r_i
+ * with prompt length p_i, generation length g_i, K_i = ceil(g_i / L) blocks of
+ * length L, block index b_i) and its scheduling loop (Algorithm 1).  A user
+ * drives it the way Algorithm 1 reads:
+ *
+ *     bs_admit() x N
+ *     loop { bs_evict_refill(&ev, &ad, &n_active); if (n_active == 0) break;
+ *            do { bs_denoise_step(); bs_block_done(&done, 0); } while (!done); }
+ *     bs_read_tokens()
+ *
+ * Conventions
+ *   - Every call returns BS_OK (0) or a negative bs_status; nothing throws.
+ *   - "device" pointers are CUDA device memory owned by the caller (the Python
+ *     binding takes them from torch tensors); the library borrows them until
+ *     bs_destroy and never allocates device memory itself.  "host" pointers are
+ *     ordinary host memory; host inputs are consumed before the call returns.
+ *   - All kernels are enqueued on the stream given to bs_init_model.
+ *     bs_evict_refill, bs_block_done, bs_read_tokens and bs_debug_read
+ *     synchronise that stream; bs_denoise_step does so only when it has to
+ *     report n_committed.
+ *   - One engine is used from one host thread at a time.
+ *   - Every step of the path runs in CUDA kernels; there is no CPU fallback.
+ */
+#ifndef BLOCKSERVE_H_
+#define BLOCKSERVE_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct bs_engine bs_engine; /* opaque */
+
+typedef enum {
+  BS_OK = 0,
+  BS_E_ARG = -1,         /* bad argument or unsupported shape */
+  BS_E_STATE = -2,       /* call out of order (e.g. step with no unfinished block) */
+  BS_E_BUDGET = -3,      /* request alone is wider than the token budget (it could never be admitted) */
+  BS_E_KV_FULL = -4,     /* request longer than the KV arena, or request table full */
+  BS_E_CUDA = -5,        /* a CUDA runtime call failed; see bs_last_error */
+  BS_E_TIMEOUT = -6,     /* a bounded device-side wait ran out; the step's results are invalid */
+  BS_E_UNKNOWN_REQ = -7  /* request id not known to the engine */
+} bs_status;
+
+enum { BS_SUFFIX_FULL = 0, BS_SUFFIX_NONE = 1 };
+enum { BS_REQ_QUEUED = 0, BS_REQ_ACTIVE = 1, BS_REQ_FINISHED = 2 };
+
+typedef struct {
+  /* model: pre-norm bidirectional transformer, RMSNorm, rotate-half RoPE, GQA, SwiGLU, no biases */
+  int n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ffn, vocab, mask_id;
+  float rms_eps, rope_theta;
+  /* method (Section 2.1, 2.4): block length L (<= 32), confidence threshold tau,
+     token budget beta of Eq. 1 (<= 0: unlimited), fixed batch cap */
+  int block_len;
+  float tau;
+  long long token_budget;
+  int max_batch;                 /* <= 1024 */
+  int max_requests;              /* size of the request table for the whole stream */
+  int max_row_tokens;            /* max p_i + g_i */
+  long long kv_capacity_tokens;  /* rows of the KV arena = max packed tokens of one step */
+  int suffix_mode;               /* BS_SUFFIX_FULL: a row sees prompt + all g_i positions (future blocks as mask
+                                    tokens); BS_SUFFIX_NONE: a row ends with its current block (row width of Eq. 1) */
+  int sort_queue;                /* 1: pending queue ascending in p_i, ties by submission (Section 2.4); 0: arrival order */
+} bs_config;
+
+/* All weights are bf16, row-major [out_features, in_features], device memory.
+ * wqkv rows: all q heads, then k heads, then v heads.  The per-layer members
+ * are HOST arrays of n_layers DEVICE pointers. */
+typedef struct {
+  const void* embed;       /* [vocab, d_model] */
+  const void* lm_head;     /* [vocab, d_model] */
+  const void* final_norm;  /* [d_model] */
+  const void* const* wqkv;    /* [(Hq + 2 Hkv) * head_dim, d_model] */
+  const void* const* wo;      /* [d_model, Hq * head_dim] */
+  const void* const* w_gate;  /* [d_ffn, d_model] */
+  const void* const* w_up;    /* [d_ffn, d_model] */
+  const void* const* w_down;  /* [d_model, d_ffn] */
+  const void* const* norm1;   /* [d_model] */
+  const void* const* norm2;   /* [d_model] */
+} bs_weights;
+
+typedef struct {
+  size_t kv_bytes, workspace_bytes, state_bytes;
+} bs_sizes;
+
+typedef struct {
+  long long steps;            /* denoise steps run */
+  long long cycles;           /* block-cycles started (bs_evict_refill calls that left rows active) */
+  long long sum_active;       /* sum over cycles of |A| (numerator of the effective compute ratio, Eq. 2) */
+  long long committed;        /* tokens committed by the engine (prompt and pre-committed blocks excluded) */
+  long long packed_tokens;    /* sum over steps of the packed query tokens M */
+  long long lm_rows;          /* sum over steps of the masked rows M_m */
+  long long kernel_launches;  /* kernels this engine has enqueued */
+} bs_stats;
+
+/* Sizes of the three device buffers the caller must provide for this config
+ * (each 256-byte aligned).  Host pointers. */
+int bs_query_sizes(const bs_config* cfg, bs_sizes* out);
+
+/* Create an engine over caller-owned device buffers `kv`, `workspace`, `state`
+ * (sizes from bs_query_sizes; `state` is cleared by this call) and the caller's
+ * CUDA stream (a cudaStream_t passed as void*, NULL = default stream).  The
+ * weights struct and its pointer arrays are host memory and are copied. */
+int bs_init_model(const bs_config* cfg, const bs_weights* w, void* kv, void* workspace, void* state,
+                  void* cuda_stream, bs_engine** out);
+
+/* Section 2.1 / Algorithm 1 input: enqueue request r_i into the pending queue P.
+ * prompt: host int32[p]; g: generation length; alpha: logit scale applied to
+ * this request's logits; start_block k > 0 means blocks 0..k-1 arrive already
+ * committed with the ids in gen_prefix (host int32[k * L], else NULL).
+ * Token ids must lie in [0, vocab) and differ from mask_id. */
+int bs_admit(bs_engine* e, long long req_id, const int* prompt, int p, int g, float alpha,
+             int start_block, const int* gen_prefix);
+
+/* Algorithm 1, block boundary (also the first fill): b_i += 1 for every active
+ * row, evict rows with b_i >= K_i, stable compaction, then admit the head of P
+ * while Eq. 1's cost stays <= beta, |A| < max_batch and the KV arena has a
+ * hole (lowest-address first fit); start every row's next block fully masked
+ * and build the next step's gather / scatter indices.  Outputs are host ints
+ * (nullable).  BS_E_STATE if a block of the current cycle is unfinished. */
+int bs_evict_refill(bs_engine* e, int* n_evicted, int* n_admitted, int* n_active);
+
+/* Section 2.5: one denoise step for all unfinished rows of A - gather by
+ * explicit position ids, transformer forward against the dual KV cache (whole
+ * row on a block's first step, which rebuilds the cache; the active block
+ * afterwards), confidence / argmax per masked position, commit conf > tau plus
+ * the top-confidence position, scatter tokens, update done flags, build the
+ * next step's indices.  n_committed: host int, nullable (non-NULL forces a
+ * stream synchronisation). */
+int bs_denoise_step(bs_engine* e, int* n_committed);
+
+/* Block-boundary completion check (Section 2.3): all_done = every active row's
+ * block is complete.  per_row_done: host bytes [max_batch], nullable. */
+int bs_block_done(bs_engine* e, int* all_done, unsigned char* per_row_done);
+
+/* Copy request req_id's token row (prompt, then generated positions; still
+ * masked positions hold mask_id) into host int32 out[cap]; n_valid = p + g;
+ * state = BS_REQ_*.  out may be NULL to query n_valid / state only. */
+int bs_read_tokens(bs_engine* e, long long req_id, int* out, int cap, int* n_valid, int* state);
+
+int bs_get_stats(bs_engine* e, bs_stats* out);
+void bs_destroy(bs_engine* e);
+const char* bs_last_error(const bs_engine* e); /* NULL engine: error of the last failed bs_init_model */
+
+/* ---- parity hooks (not on the timed path) ------------------------------ */
+enum {
+  BS_DBG_HEADER = 0,   /* int32[32]: n_active, M, M_m, all_done, n_committed_step, n_evicted, n_admitted, ... */
+  BS_DBG_ROW_SLOT = 1, BS_DBG_ROW_MASK = 2, BS_DBG_ROW_S = 3, BS_DBG_ROW_KV_BASE = 4, /* int32[n_active] */
+  BS_DBG_CU_Q = 5,     /* int32[n_active + 1]  (indices of the step about to run) */
+  BS_DBG_TOK_ROW = 6, BS_DBG_TOK_POS = 7, BS_DBG_TOK_KV = 8,   /* int32[M]; filled by the last bs_denoise_step */
+  BS_DBG_LM_TOK = 9, BS_DBG_LM_ROW = 10, BS_DBG_LM_SLOT = 11,  /* int32[M_m] of the step about to run */
+  BS_DBG_PREV_LM_ROW = 12, BS_DBG_PREV_LM_SLOT = 13,           /* int32[M_m] of the step that just ran */
+  BS_DBG_PREV_TOK = 14, BS_DBG_PREV_CONF = 15, BS_DBG_PREV_COMMIT = 16, /* int32 / float / int32 [M_m], last step */
+  BS_DBG_PREV_LOGITS = 17, /* float[M_m * vocab] of the last step */
+  BS_DBG_REQ_ID_OF_ROW = 18, /* int64[n_active] */
+  BS_DBG_KV_ROW = 19   /* bf16 K then V of (layer = arg0, physical row = arg1): 2 * Hkv * head_dim values */
+};
+/* Copies the named array into host_buf (cap bytes); n = bytes written. */
+int bs_debug_read(bs_engine* e, int what, int arg0, int arg1, void* host_buf, size_t cap, size_t* n);
+
+/* ---- single operations (parity tests and per-kernel measurement) ------- *
+ * All pointers are device memory; `stream` is a cudaStream_t as void*.     */
+
+/* C[M,N] = A[M,K] * W[N,K]^T, bf16 operands, fp32 accumulate (the projections of the transformer block).
+ * mode 0: C bf16 store;  1: C fp32 += result (residual);  2: C fp32 = row_scale[m] * result (LM head, alpha_i);
+ * mode 3: C bf16 [M,N] = silu(A W^T) * (A W2^T)  (SwiGLU gate/up).  K % 8 == 0.  lda/ldc in elements. */
+int bs_op_gemm(const void* A, int lda, const void* W, const void* W2, void* C, int ldc, int M, int N, int K,
+               int mode, const float* row_scale, void* stream);
+
+/* y[m,:] = bf16(w * x[idx ? idx[m] : m, :] / sqrt(mean(x^2) + eps)); x fp32 [*, d], y bf16 [M, d]. */
+int bs_op_rmsnorm(const float* x, const int* idx, const void* w, void* y, int M, int d, float eps, void* stream);
+
+/* Rotate q and k of packed tokens at their position ids (rotate-half pairing,
+ * angle pos * theta^(-2j/dh)) and scatter k, v to KV rows tok_kv[t] (Section 2.5:
+ * in-place update at the current query rows only).  qkv bf16 [M, (Hq+2Hkv)*dh] (q rotated in place);
+ * kcache / vcache bf16 [kv_rows, Hkv, dh]. */
+int bs_op_rope_kv(void* qkv, const int* tok_pos, const int* tok_kv, void* kcache, void* vcache, int M,
+                  int n_q_heads, int n_kv_heads, int head_dim, float theta, int max_pos,
+                  float* table_scratch /* device float[max_pos * head_dim], overwritten */, void* stream);
+
+/* Ragged bidirectional attention of packed queries against per-row cache spans:
+ * row i owns packed tokens [cu_q[i], cu_q[i+1]) and attends over cache rows
+ * [kv_base[i], kv_base[i] + vis[i]) (prefix, fresh block and suffix alike; no causal or padding mask).
+ * q: the qkv buffer of bs_op_rope_kv; out bf16 [M, Hq*dh].  Work items are q-tiles of
+ * bs_op_attention_q_tile(Hq, Hkv) tokens: cu_tile[i] = sum_{r<i} ceil(n_q(r) / q_tile), n_tiles = cu_tile[n_rows]. */
+int bs_op_attention_q_tile(int n_q_heads, int n_kv_heads);
+int bs_op_attention(const void* qkv, const void* kcache, const void* vcache, void* out, const int* cu_q,
+                    const int* cu_tile, const int* kv_base, const int* vis, int n_rows, int n_tiles, int n_q_heads,
+                    int n_kv_heads, int head_dim, void* stream);
+
+/* Per row of fp32 logits [n_rows, vocab]: mask id excluded, tok = argmax (lowest id on ties),
+ * conf = exp(max - logsumexp). */
+int bs_op_confidence(const float* logits, int n_rows, int vocab, int mask_id, int* tok, float* conf, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BLOCKSERVE_H_ */

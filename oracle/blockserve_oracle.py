@@ -13,6 +13,18 @@ this package.  It shares no code with the CUDA path: no kernels, headers,
 tables or helpers.  There is no blocking, fusion or reordering beyond what the
 definitions state; numpy's matmul, exp, sort and argmax serve as primitives.
 
+Precision: the paper runs its models in bfloat16 (Section 3.1).  Arithmetic
+here is fp32 (weights hold bf16-representable values); with
+``Model.bf16_activations`` (the default) every activation tensor a bf16 model
+stores between operators is rounded to bf16 (nearest even): the normed hidden
+state, q / k / v, the rotated q / k, the attention output, the SwiGLU product
+and the final normed state.  The residual stream, attention scores and
+probabilities, accumulations, logits and confidences stay fp32.  With the flag
+off nothing is rounded (pure fp32).  Rounding is discontinuous, so two
+implementations that round at the same points still drift apart by a fraction
+of a bf16 ulp per operator; sharing the rounding points removes the systematic
+part of the difference, not that drift.
+
 Readings taken where the paper is silent (each is listed in the design notes):
   * the model is a pre-norm bidirectional transformer (RMSNorm, rotate-half
     RoPE, GQA, SwiGLU, no biases), logits = alpha_i * norm_f(x) @ W_lm^T;
@@ -60,9 +72,26 @@ class Model:
     lm_head: np.ndarray          # [V, d]
     final_norm: np.ndarray       # [d]
     layer: Callable[[int], Dict[str, np.ndarray]]   # l -> wq wk wv wo w_gate w_up w_down norm1 norm2
+    bf16_activations: bool = True
+
+    def act(self, x: np.ndarray) -> np.ndarray:
+        """Storage precision of an activation tensor between operators."""
+        return round_bf16(x) if self.bf16_activations else np.asarray(x, dtype=F32)
 
 
-def model_from_weights(shape, w: Dict[str, object]) -> Model:
+def round_bf16(x: np.ndarray) -> np.ndarray:
+    """Round fp32 values to the nearest bfloat16 (ties to even), returned as fp32."""
+    a = np.ascontiguousarray(x, dtype=F32)
+    u = a.view(np.uint32).astype(np.uint64)
+    r = ((u + 0x7FFF + ((u >> 16) & 1)) & 0xFFFF0000).astype(np.uint32)
+    out = r.view(F32).reshape(a.shape)
+    bad = ~np.isfinite(a)
+    if bad.any():
+        out = np.where(bad, a, out)
+    return out
+
+
+def model_from_weights(shape, w: Dict[str, object], bf16_activations: bool = True) -> Model:
     """Build a Model from fp32 numpy weights laid out as the input generator
     documents (wqkv rows: q heads, k heads, v heads)."""
     nq = shape.n_q_heads * shape.head_dim
@@ -81,7 +110,7 @@ def model_from_weights(shape, w: Dict[str, object]) -> Model:
     return Model(shape.n_layers, shape.d_model, shape.n_q_heads, shape.n_kv_heads, shape.head_dim,
                  shape.d_ffn, shape.vocab, shape.vocab - 1, shape.rms_eps, shape.rope_theta,
                  np.asarray(w["embed"], dtype=F32), np.asarray(w["lm_head"], dtype=F32),
-                 np.asarray(w["final_norm"], dtype=F32), layer)
+                 np.asarray(w["final_norm"], dtype=F32), layer, bf16_activations)
 
 
 def rmsnorm(x: np.ndarray, w: np.ndarray, eps: float) -> np.ndarray:
@@ -226,19 +255,19 @@ def forward_queries(model: Model, r: ReqState, qpos: np.ndarray, vis: int) -> np
     n = len(qpos)
     for l in range(model.n_layers):
         w = model.layer(l)
-        h = rmsnorm(x, w["norm1"], model.rms_eps)
-        q = (h @ w["wq"].T).astype(F32).reshape(n, model.n_q_heads, model.head_dim)
-        k = (h @ w["wk"].T).astype(F32).reshape(n, model.n_kv_heads, model.head_dim)
-        v = (h @ w["wv"].T).astype(F32).reshape(n, model.n_kv_heads, model.head_dim)
-        q = apply_rope(q, cos, sin)
-        k = apply_rope(k, cos, sin)
+        h = model.act(rmsnorm(x, w["norm1"], model.rms_eps))
+        q = model.act(h @ w["wq"].T).reshape(n, model.n_q_heads, model.head_dim)
+        k = model.act(h @ w["wk"].T).reshape(n, model.n_kv_heads, model.head_dim)
+        v = model.act(h @ w["wv"].T).reshape(n, model.n_kv_heads, model.head_dim)
+        q = model.act(apply_rope(q, cos, sin))
+        k = model.act(apply_rope(k, cos, sin))
         r.K[l][qpos] = k
         r.V[l][qpos] = v
-        a = attention(q, r.K[l][:vis], r.V[l][:vis]).reshape(n, -1)
+        a = model.act(attention(q, r.K[l][:vis], r.V[l][:vis])).reshape(n, -1)
         x = x + (a @ w["wo"].T).astype(F32)
-        h2 = rmsnorm(x, w["norm2"], model.rms_eps)
-        act = silu(h2 @ w["w_gate"].T) * (h2 @ w["w_up"].T).astype(F32)
-        x = x + (act.astype(F32) @ w["w_down"].T).astype(F32)
+        h2 = model.act(rmsnorm(x, w["norm2"], model.rms_eps))
+        act = model.act(silu(h2 @ w["w_gate"].T) * (h2 @ w["w_up"].T).astype(F32))
+        x = x + (act @ w["w_down"].T).astype(F32)
     return x
 
 
@@ -250,7 +279,7 @@ def full_forward_logits(model: Model, tokens: np.ndarray, alpha: float) -> np.nd
 
 
 def lm_logits(model: Model, x: np.ndarray, alpha: float) -> np.ndarray:
-    hf = rmsnorm(x, model.final_norm, model.rms_eps)
+    hf = model.act(rmsnorm(x, model.final_norm, model.rms_eps))
     return (F32(alpha) * (hf @ model.lm_head.T).astype(F32)).astype(F32)
 
 

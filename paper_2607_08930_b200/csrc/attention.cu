@@ -1,0 +1,240 @@
+// Ragged bidirectional attention against the dual KV cache (Section 2.5).
+// Work item = (row i, q-tile of the row's packed tokens, kv head).  All query heads of the kv head's group
+// share each K/V tile (GQA): the flattened "query rows" of a CTA are (token, head-in-group) pairs.
+// Keys are the row's cache span [kv_base_i, kv_base_i + vis_i): prefix, fresh block and suffix alike;
+// there is no causal mask and no padding mask.  Online softmax with warp shuffles, mma.sync m16n8k16.
+#include <math.h>
+
+#include "common.cuh"
+
+namespace bs {
+
+namespace {
+constexpr int KT = 64;   // keys per tile
+
+__device__ __forceinline__ void cp_async16(void* dst, const void* src, int bytes) {
+  const unsigned d = (unsigned)__cvta_generic_to_shared(dst);
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(d), "l"(src), "r"(bytes));
+}
+__device__ __forceinline__ void ldsm_x4(unsigned& r0, unsigned& r1, unsigned& r2, unsigned& r3, const void* p) {
+  const unsigned a = (unsigned)__cvta_generic_to_shared(p);
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(a));
+}
+__device__ __forceinline__ void ldsm_x4_t(unsigned& r0, unsigned& r1, unsigned& r2, unsigned& r3, const void* p) {
+  const unsigned a = (unsigned)__cvta_generic_to_shared(p);
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(a));
+}
+__device__ __forceinline__ void mma16816(float* c, const unsigned* a, unsigned b0, unsigned b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ unsigned pack_bf16(float a, float b) {
+  __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<unsigned*>(&h);
+}
+
+template <int DH>
+__global__ void __launch_bounds__(256) k_attention(const bf16* __restrict__ qkv, const bf16* __restrict__ kc,
+                                                   const bf16* __restrict__ vc, bf16* __restrict__ out,
+                                                   const int* __restrict__ cu_q, const int* __restrict__ cu_tile,
+                                                   const int* __restrict__ kv_base, const int* __restrict__ vis_arr,
+                                                   int n_rows, int hq, int hkv, int q_tile) {
+  constexpr int LD = DH + 8;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  bf16* smem = reinterpret_cast<bf16*>(smem_raw);      // [2 stages][K tile, V tile][KT][LD]
+  const int G = hq / hkv;
+  const int kh = blockIdx.y;
+  // which row owns this q-tile: largest r with cu_tile[r] <= blockIdx.x
+  int lo = 0, hi = n_rows;
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (cu_tile[mid] <= (int)blockIdx.x) lo = mid; else hi = mid;
+  }
+  const int row = lo;
+  const int t0 = cu_q[row] + ((int)blockIdx.x - cu_tile[row]) * q_tile;
+  const int nt = min(q_tile, cu_q[row + 1] - t0);
+  if (nt <= 0) return;
+  const int vis = vis_arr[row];
+  const size_t kvb = (size_t)kv_base[row];
+  const int qkv_ld = (hq + 2 * hkv) * DH;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int nthreads = blockDim.x;
+  const bool warp_active = warp * 16 < nt * G;
+  // the two flattened query rows this thread owns inside its warp's 16
+  const int f0 = warp * 16 + (lane >> 2), f1 = f0 + 8;
+  const int tk0 = f0 / G, tk1 = f1 / G;
+  const bool v0 = tk0 < nt, v1 = tk1 < nt;
+  const int hd0 = kh * G + f0 % G, hd1 = kh * G + f1 % G;
+
+  unsigned qf[DH / 16][4];
+  {
+    const bf16* q0 = qkv + (size_t)(t0 + (v0 ? tk0 : 0)) * qkv_ld + hd0 * DH + (lane & 3) * 2;
+    const bf16* q1 = qkv + (size_t)(t0 + (v1 ? tk1 : 0)) * qkv_ld + hd1 * DH + (lane & 3) * 2;
+#pragma unroll
+    for (int ks = 0; ks < DH / 16; ++ks) {
+      qf[ks][0] = v0 ? *reinterpret_cast<const unsigned*>(q0 + ks * 16) : 0u;
+      qf[ks][1] = v1 ? *reinterpret_cast<const unsigned*>(q1 + ks * 16) : 0u;
+      qf[ks][2] = v0 ? *reinterpret_cast<const unsigned*>(q0 + ks * 16 + 8) : 0u;
+      qf[ks][3] = v1 ? *reinterpret_cast<const unsigned*>(q1 + ks * 16 + 8) : 0u;
+    }
+  }
+
+  auto load_tile = [&](int stage, int kt) {
+    bf16* sK = smem + stage * 2 * KT * LD;
+    bf16* sV = sK + KT * LD;
+    constexpr int CH = DH / 8;
+    for (int c = tid; c < KT * CH; c += nthreads) {
+      const int r = c / CH, cc = (c % CH) * 8;
+      const int key = kt * KT + r;
+      const bool ok = key < vis;
+      const size_t off = ((kvb + (ok ? key : 0)) * hkv + kh) * DH + cc;
+      cp_async16(sK + r * LD + cc, kc + off, ok ? 16 : 0);
+      cp_async16(sV + r * LD + cc, vc + off, ok ? 16 : 0);
+    }
+  };
+
+  float o[DH / 8][4];
+#pragma unroll
+  for (int i = 0; i < DH / 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+  float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+  const float sc = 1.4426950408889634f / sqrtf((float)DH);    // log2(e) / sqrt(dh)
+
+  const int nkt = (vis + KT - 1) / KT;
+  load_tile(0, 0);
+  asm volatile("cp.async.commit_group;\n" ::);
+  for (int kt = 0; kt < nkt; ++kt) {
+    if (kt + 1 < nkt) load_tile((kt + 1) & 1, kt + 1);
+    asm volatile("cp.async.commit_group;\n" ::);
+    asm volatile("cp.async.wait_group 1;\n" ::);
+    __syncthreads();
+    if (warp_active) {
+      const bf16* sK = smem + (kt & 1) * 2 * KT * LD;
+      const bf16* sV = sK + KT * LD;
+      float s[KT / 8][4];
+#pragma unroll
+      for (int i = 0; i < KT / 8; ++i) s[i][0] = s[i][1] = s[i][2] = s[i][3] = 0.f;
+#pragma unroll
+      for (int ks = 0; ks < DH / 16; ++ks) {
+#pragma unroll
+        for (int np = 0; np < KT / 16; ++np) {
+          unsigned b0, b1, b2, b3;
+          ldsm_x4(b0, b1, b2, b3,
+                  sK + (np * 16 + (lane & 7) + ((lane >> 4) << 3)) * LD + ks * 16 + ((lane >> 3) & 1) * 8);
+          mma16816(s[2 * np], qf[ks], b0, b1);
+          mma16816(s[2 * np + 1], qf[ks], b2, b3);
+        }
+      }
+      // scale, mask keys beyond the row's span, running max
+      float mx0 = -INFINITY, mx1 = -INFINITY;
+      const int kbase = kt * KT + (lane & 3) * 2;
+#pragma unroll
+      for (int i = 0; i < KT / 8; ++i) {
+        const int key = kbase + i * 8;
+        s[i][0] = key < vis ? s[i][0] * sc : -INFINITY;
+        s[i][1] = key + 1 < vis ? s[i][1] * sc : -INFINITY;
+        s[i][2] = key < vis ? s[i][2] * sc : -INFINITY;
+        s[i][3] = key + 1 < vis ? s[i][3] * sc : -INFINITY;
+        mx0 = fmaxf(mx0, fmaxf(s[i][0], s[i][1]));
+        mx1 = fmaxf(mx1, fmaxf(s[i][2], s[i][3]));
+      }
+      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
+      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+      const float nm0 = fmaxf(m0, mx0), nm1 = fmaxf(m1, mx1);     // finite: every tile holds >= 1 valid key
+      const float a0 = exp2f(m0 - nm0), a1 = exp2f(m1 - nm1);
+      m0 = nm0;
+      m1 = nm1;
+      float rs0 = 0.f, rs1 = 0.f;
+#pragma unroll
+      for (int i = 0; i < KT / 8; ++i) {
+        s[i][0] = exp2f(s[i][0] - nm0);
+        s[i][1] = exp2f(s[i][1] - nm0);
+        s[i][2] = exp2f(s[i][2] - nm1);
+        s[i][3] = exp2f(s[i][3] - nm1);
+        rs0 += s[i][0] + s[i][1];
+        rs1 += s[i][2] + s[i][3];
+      }
+      l0 = l0 * a0 + rs0;
+      l1 = l1 * a1 + rs1;
+#pragma unroll
+      for (int i = 0; i < DH / 8; ++i) {
+        o[i][0] *= a0;
+        o[i][1] *= a0;
+        o[i][2] *= a1;
+        o[i][3] *= a1;
+      }
+#pragma unroll
+      for (int kk = 0; kk < KT / 16; ++kk) {
+        unsigned pa[4];
+        pa[0] = pack_bf16(s[2 * kk][0], s[2 * kk][1]);
+        pa[1] = pack_bf16(s[2 * kk][2], s[2 * kk][3]);
+        pa[2] = pack_bf16(s[2 * kk + 1][0], s[2 * kk + 1][1]);
+        pa[3] = pack_bf16(s[2 * kk + 1][2], s[2 * kk + 1][3]);
+#pragma unroll
+        for (int nd = 0; nd < DH / 16; ++nd) {
+          unsigned b0, b1, b2, b3;
+          ldsm_x4_t(b0, b1, b2, b3,
+                    sV + (kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * LD + nd * 16 + (lane >> 4) * 8);
+          mma16816(o[2 * nd], pa, b0, b1);
+          mma16816(o[2 * nd + 1], pa, b2, b3);
+        }
+      }
+    }
+    __syncthreads();
+  }
+  asm volatile("cp.async.wait_group 0;\n" ::);
+  if (!warp_active) return;
+  l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
+  l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
+  l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
+  l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+  const float i0 = 1.0f / l0, i1 = 1.0f / l1;
+  const int out_ld = hq * DH;
+  if (v0) {
+    bf16* dst = out + (size_t)(t0 + tk0) * out_ld + hd0 * DH + (lane & 3) * 2;
+#pragma unroll
+    for (int i = 0; i < DH / 8; ++i)
+      *reinterpret_cast<__nv_bfloat162*>(dst + i * 8) = __floats2bfloat162_rn(o[i][0] * i0, o[i][1] * i0);
+  }
+  if (v1) {
+    bf16* dst = out + (size_t)(t0 + tk1) * out_ld + hd1 * DH + (lane & 3) * 2;
+#pragma unroll
+    for (int i = 0; i < DH / 8; ++i)
+      *reinterpret_cast<__nv_bfloat162*>(dst + i * 8) = __floats2bfloat162_rn(o[i][2] * i1, o[i][3] * i1);
+  }
+}
+}  // namespace
+
+int attention_q_tile(int hq, int hkv) {
+  const int G = hq / hkv;
+  return G >= 5 ? 16 : (G == 1 ? 64 : 32);
+}
+
+cudaError_t launch_attention(const bf16* qkv, const bf16* kc, const bf16* vc, bf16* out, const int* cu_q,
+                             const int* cu_tile, const int* kv_base, const int* vis, int n_rows, int n_tiles,
+                             int hq, int hkv, int dh, cudaStream_t s) {
+  if (n_tiles <= 0 || n_rows <= 0) return cudaSuccess;
+  const int G = hq / hkv;
+  const int qt = attention_q_tile(hq, hkv);
+  const int threads = qt * G * 2;             // 16 flattened rows per warp
+  if (threads > 256 || (dh != 64 && dh != 128) || hq % hkv != 0) return cudaErrorInvalidValue;
+  const size_t smem = (size_t)2 * 2 * KT * (dh + 8) * sizeof(bf16);
+  dim3 grid(n_tiles, hkv);
+  if (dh == 128) {
+    static bool done = false;
+    if (!done) { cudaFuncSetAttribute(k_attention<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); done = true; }
+    k_attention<128><<<grid, threads, smem, s>>>(qkv, kc, vc, out, cu_q, cu_tile, kv_base, vis, n_rows, hq, hkv, qt);
+  } else {
+    static bool done = false;
+    if (!done) { cudaFuncSetAttribute(k_attention<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); done = true; }
+    k_attention<64><<<grid, threads, smem, s>>>(qkv, kc, vc, out, cu_q, cu_tile, kv_base, vis, n_rows, hq, hkv, qt);
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace bs

@@ -1,0 +1,64 @@
+// Shared declarations of the CUDA side: device state layout, launch wrappers.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace bs {
+
+typedef __nv_bfloat16 bf16;
+
+constexpr int kHdrInts = 32;
+// header words (device int32[kHdrInts], mirrored to pinned host memory once per step)
+enum Hdr {
+  H_N_ACTIVE = 0, H_M = 1, H_MM = 2, H_ALL_DONE = 3, H_COMMITTED_STEP = 4, H_EVICTED = 5, H_ADMITTED = 6,
+  H_QUEUE_HEAD = 7, H_QUEUE_LEN = 8, H_ERROR = 9, H_PARITY = 10, H_QTILES = 11, H_MAX_VIS = 12, H_WIDTH = 13,
+  H_TOTAL_LO = 14, H_TOTAL_HI = 15, H_UNFINISHED = 16, H_STEP_REFRESH = 17
+};
+
+
+// Everything the scheduling / index kernels touch.  Plain pointers into the caller's `state` buffer.
+struct DevState {
+  int L, max_batch, max_requests, max_row_tokens, suffix_mode, mask_id, vocab;
+  int q_tile;           // query tokens per attention work item
+  long long beta, kv_capacity;
+  float tau;
+  int* hdr;             // [kHdrInts] followed directly by row_mask[max_batch]
+  unsigned* row_mask;   // bit j set <=> block position j still masked
+  int* req_p; int* req_g; int* req_b; int* req_state; int* req_committed; float* req_alpha;
+  int* tokens;          // [max_requests, max_row_tokens]
+  int* queue;           // pending slots in admission order
+  int* row_slot; int* row_s; int* row_kv_base; int* row_vis;
+  int* cu_q[2]; int* lm_base[2]; int* cu_tile[2];
+  int* lm_tok[2]; int* lm_row[2]; int* lm_slot[2];
+  int* out_tok[2]; float* out_conf[2]; int* out_commit[2];
+  float* lm_scale[2];   // alpha of the row each lm entry belongs to
+  int* tok_row; int* tok_pos; int* tok_kv;
+};
+
+// ---- launch wrappers (each returns the cudaError_t of the launch) ----------
+cudaError_t launch_sched(const DevState& st, cudaStream_t s);
+cudaError_t launch_commit_index(const DevState& st, cudaStream_t s);
+cudaError_t launch_fill_tokens(const DevState& st, int parity, int M, cudaStream_t s);
+
+cudaError_t launch_embed(const DevState& st, const bf16* embed, float* x, int M, int d, cudaStream_t s);
+cudaError_t launch_rmsnorm(const float* x, const int* idx, const bf16* w, bf16* y, int M, int d, float eps,
+                           cudaStream_t s);
+cudaError_t launch_rope_kv(bf16* qkv, const int* tok_pos, const int* tok_kv, bf16* kc, bf16* vc, int M, int hq,
+                           int hkv, int dh, const float* cos_sin, cudaStream_t s);
+cudaError_t launch_attention(const bf16* qkv, const bf16* kc, const bf16* vc, bf16* out, const int* cu_q,
+                             const int* cu_tile, const int* kv_base, const int* vis, int n_rows, int n_tiles,
+                             int hq, int hkv, int dh, cudaStream_t s);
+cudaError_t launch_confidence(const float* logits, int n_rows, int vocab, int mask_id, int* tok, float* conf,
+                              cudaStream_t s);
+
+// C[M,N] = A[M,K] W[N,K]^T.  mode: 0 bf16 store, 1 fp32 +=, 2 fp32 row-scaled store, 3 SwiGLU (W and W2).
+cudaError_t launch_gemm(const bf16* A, int lda, const bf16* W, const bf16* W2, void* C, int ldc, int M, int N, int K,
+                        int mode, const float* row_scale, cudaStream_t s);
+
+cudaError_t launch_gemm_mma(const bf16* A, int lda, const bf16* W, const bf16* W2, void* C, int ldc, int M, int N,
+                            int K, int mode, const float* row_scale, cudaStream_t s);
+int attention_q_tile(int hq, int hkv);
+void build_rope_table(float* host_cos_sin, int max_pos, int dh, float theta);   // [max_pos, dh/2, 2]
+
+}  // namespace bs

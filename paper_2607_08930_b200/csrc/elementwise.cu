@@ -1,0 +1,217 @@
+// HBM-bound row kernels: embedding gather, RMSNorm, RoPE at gathered positions + KV scatter,
+// and the per-row vocabulary pass of the confidence epilogue.
+#include <math.h>
+
+#include "common.cuh"
+
+namespace bs {
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// x[t, :] = E[token at (row, position) of packed token t]   (gather of the active regions, Section 2.5)
+__global__ void k_embed(DevState st, const bf16* __restrict__ embed, float* __restrict__ x, int M, int d) {
+  const int t = blockIdx.x;
+  if (t >= M) return;
+  const int slot = st.row_slot[st.tok_row[t]];
+  const int id = st.tokens[(size_t)slot * st.max_row_tokens + st.tok_pos[t]];
+  const uint4* src = reinterpret_cast<const uint4*>(embed + (size_t)id * d);
+  float4* dst = reinterpret_cast<float4*>(x + (size_t)t * d);
+  for (int c = threadIdx.x; c < d / 8; c += blockDim.x) {
+    const uint4 v = src[c];
+    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&v);
+    const float2 a = __bfloat1622float2(h[0]), b = __bfloat1622float2(h[1]);
+    const float2 e = __bfloat1622float2(h[2]), f = __bfloat1622float2(h[3]);
+    dst[2 * c] = make_float4(a.x, a.y, b.x, b.y);
+    dst[2 * c + 1] = make_float4(e.x, e.y, f.x, f.y);
+  }
+}
+
+// y[m, :] = bf16(w * x[row, :] * rsqrt(mean(x^2) + eps)); one CTA per output row.
+__global__ void __launch_bounds__(256) k_rmsnorm(const float* __restrict__ x, const int* __restrict__ idx,
+                                                 const bf16* __restrict__ w, bf16* __restrict__ y, int d, float eps) {
+  __shared__ float red[8];
+  const int m = blockIdx.x;
+  const int row = idx ? idx[m] : m;
+  const float4* src = reinterpret_cast<const float4*>(x + (size_t)row * d);
+  float ss = 0.f;
+  for (int c = threadIdx.x; c < d / 4; c += 256) {
+    const float4 v = src[c];
+    ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+  }
+  ss = warp_sum(ss);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  float tot = 0.f;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) tot += red[i];
+  const float r = rsqrtf(tot / (float)d + eps);
+  const uint2* wp = reinterpret_cast<const uint2*>(w);
+  uint2* dst = reinterpret_cast<uint2*>(y + (size_t)m * d);
+  for (int c = threadIdx.x; c < d / 4; c += 256) {
+    const float4 v = src[c];
+    const uint2 wv = wp[c];
+    const __nv_bfloat162* wh = reinterpret_cast<const __nv_bfloat162*>(&wv);
+    const float2 w0 = __bfloat1622float2(wh[0]), w1 = __bfloat1622float2(wh[1]);
+    __nv_bfloat162 o0 = __floats2bfloat162_rn(v.x * r * w0.x, v.y * r * w0.y);
+    __nv_bfloat162 o1 = __floats2bfloat162_rn(v.z * r * w1.x, v.w * r * w1.y);
+    uint2 o;
+    o.x = *reinterpret_cast<unsigned*>(&o0);
+    o.y = *reinterpret_cast<unsigned*>(&o1);
+    dst[c] = o;
+  }
+}
+
+// One CTA per packed token: rotate q (in place) and k by the token's position id, scatter k and v to the
+// token's physical cache row.  cos_sin: [max_pos, dh/2] float2 (cos, sin).
+__global__ void __launch_bounds__(256) k_rope_kv(bf16* __restrict__ qkv, const int* __restrict__ tok_pos,
+                                                 const int* __restrict__ tok_kv, bf16* __restrict__ kc,
+                                                 bf16* __restrict__ vc, int hq, int hkv, int dh,
+                                                 const float2* __restrict__ cos_sin) {
+  const int t = blockIdx.x;
+  const int pos = tok_pos[t];
+  const size_t kvrow = (size_t)tok_kv[t];
+  const int half = dh / 2;
+  bf16* base = qkv + (size_t)t * (hq + 2 * hkv) * dh;
+  const float2* cs = cos_sin + (size_t)pos * half;
+  const int pairs_per_head = half / 2;                  // bf16x2 granules per half head
+  const int n_rot = (hq + hkv) * pairs_per_head;
+  for (int u = threadIdx.x; u < n_rot; u += 256) {
+    const int h = u / pairs_per_head, j = (u % pairs_per_head) * 2;
+    __nv_bfloat162* p1 = reinterpret_cast<__nv_bfloat162*>(base + h * dh + j);
+    __nv_bfloat162* p2 = reinterpret_cast<__nv_bfloat162*>(base + h * dh + half + j);
+    const float2 a = __bfloat1622float2(*p1), b = __bfloat1622float2(*p2);
+    const float2 c0 = cs[j], c1 = cs[j + 1];
+    const __nv_bfloat162 o1 = __floats2bfloat162_rn(a.x * c0.x - b.x * c0.y, a.y * c1.x - b.y * c1.y);
+    const __nv_bfloat162 o2 = __floats2bfloat162_rn(b.x * c0.x + a.x * c0.y, b.y * c1.x + a.y * c1.y);
+    if (h < hq) {
+      *p1 = o1;
+      *p2 = o2;
+    } else {
+      bf16* dstk = kc + (kvrow * hkv + (h - hq)) * dh;
+      *reinterpret_cast<__nv_bfloat162*>(dstk + j) = o1;
+      *reinterpret_cast<__nv_bfloat162*>(dstk + half + j) = o2;
+    }
+  }
+  const uint4* vsrc = reinterpret_cast<const uint4*>(base + (hq + hkv) * dh);
+  uint4* vdst = reinterpret_cast<uint4*>(vc + kvrow * hkv * dh);
+  for (int u = threadIdx.x; u < hkv * dh / 8; u += 256) vdst[u] = vsrc[u];
+}
+
+// Per row of fp32 logits: online (max, sum exp, argmax) in one pass, mask id excluded,
+// lowest id on ties; conf = 1 / sum exp(z - max) = exp(max - logsumexp).
+constexpr int kConfThreads = 512;
+__global__ void __launch_bounds__(kConfThreads) k_confidence(const float* __restrict__ logits, int vocab, int mask_id,
+                                                             int* __restrict__ tok, float* __restrict__ conf) {
+  __shared__ float s_m[kConfThreads / 32], s_s[kConfThreads / 32];
+  __shared__ int s_i[kConfThreads / 32];
+  const int row = blockIdx.x;
+  const float* z = logits + (size_t)row * vocab;
+  float m = -INFINITY, s = 0.f;
+  int am = 0x7fffffff;
+  const int nv = (vocab % 4 == 0) ? vocab / 4 : 0;      // vector part (rows are 16-byte aligned iff vocab % 4 == 0)
+  const float4* z4 = reinterpret_cast<const float4*>(z);
+  for (int c = threadIdx.x; c < nv; c += kConfThreads) {
+    float4 v = __ldcs(z4 + c);
+    const int i0 = c * 4;
+    if (mask_id >= i0 && mask_id < i0 + 4) {
+      if (mask_id == i0) v.x = -INFINITY;
+      else if (mask_id == i0 + 1) v.y = -INFINITY;
+      else if (mask_id == i0 + 2) v.z = -INFINITY;
+      else v.w = -INFINITY;
+    }
+    float lm = v.x;
+    int li = i0;
+    if (v.y > lm) { lm = v.y; li = i0 + 1; }
+    if (v.z > lm) { lm = v.z; li = i0 + 2; }
+    if (v.w > lm) { lm = v.w; li = i0 + 3; }
+    if (lm > m) {
+      s *= __expf(m - lm);
+      m = lm;
+      am = li;
+    }
+    if (m > -INFINITY) s += __expf(v.x - m) + __expf(v.y - m) + __expf(v.z - m) + __expf(v.w - m);
+  }
+  for (int i = nv * 4 + threadIdx.x; i < vocab; i += kConfThreads) {
+    const float v = (i == mask_id) ? -INFINITY : z[i];
+    if (v > m) {
+      s *= __expf(m - v);
+      m = v;
+      am = i;
+    }
+    if (m > -INFINITY) s += __expf(v - m);
+  }
+  // merge (m, s, am): larger max wins, ties keep the lower id
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float om = __shfl_xor_sync(0xffffffffu, m, o);
+    const float os = __shfl_xor_sync(0xffffffffu, s, o);
+    const int oi = __shfl_xor_sync(0xffffffffu, am, o);
+    const float nm = fmaxf(m, om);
+    const float a = (m > -INFINITY) ? s * __expf(m - nm) : 0.f;
+    const float b = (om > -INFINITY) ? os * __expf(om - nm) : 0.f;
+    if (om > m || (om == m && oi < am)) am = oi;
+    m = nm;
+    s = a + b;
+  }
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  if (lane == 0) { s_m[w] = m; s_s[w] = s; s_i[w] = am; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float M = s_m[0], S = s_s[0];
+    int A = s_i[0];
+    for (int k = 1; k < kConfThreads / 32; ++k) {
+      const float om = s_m[k], os = s_s[k];
+      const int oi = s_i[k];
+      const float nm = fmaxf(M, om);
+      const float a = (M > -INFINITY) ? S * __expf(M - nm) : 0.f;
+      const float b = (om > -INFINITY) ? os * __expf(om - nm) : 0.f;
+      if (om > M || (om == M && oi < A)) A = oi;
+      M = nm;
+      S = a + b;
+    }
+    tok[row] = A;
+    conf[row] = 1.0f / S;
+  }
+}
+
+cudaError_t launch_embed(const DevState& st, const bf16* embed, float* x, int M, int d, cudaStream_t s) {
+  if (M <= 0) return cudaSuccess;
+  k_embed<<<M, 128, 0, s>>>(st, embed, x, M, d);
+  return cudaGetLastError();
+}
+cudaError_t launch_rmsnorm(const float* x, const int* idx, const bf16* w, bf16* y, int M, int d, float eps,
+                           cudaStream_t s) {
+  if (M <= 0) return cudaSuccess;
+  k_rmsnorm<<<M, 256, 0, s>>>(x, idx, w, y, d, eps);
+  return cudaGetLastError();
+}
+cudaError_t launch_rope_kv(bf16* qkv, const int* tok_pos, const int* tok_kv, bf16* kc, bf16* vc, int M, int hq,
+                           int hkv, int dh, const float* cos_sin, cudaStream_t s) {
+  if (M <= 0) return cudaSuccess;
+  k_rope_kv<<<M, 256, 0, s>>>(qkv, tok_pos, tok_kv, kc, vc, hq, hkv, dh, reinterpret_cast<const float2*>(cos_sin));
+  return cudaGetLastError();
+}
+cudaError_t launch_confidence(const float* logits, int n_rows, int vocab, int mask_id, int* tok, float* conf,
+                              cudaStream_t s) {
+  if (n_rows <= 0) return cudaSuccess;
+  k_confidence<<<n_rows, kConfThreads, 0, s>>>(logits, vocab, mask_id, tok, conf);
+  return cudaGetLastError();
+}
+
+void build_rope_table(float* out, int max_pos, int dh, float theta) {
+  const int half = dh / 2;
+  for (int j = 0; j < half; ++j) {
+    const double inv = pow((double)theta, -2.0 * (double)j / (double)dh);
+    for (int p = 0; p < max_pos; ++p) {
+      const double a = (double)p * inv;
+      out[((size_t)p * half + j) * 2 + 0] = (float)cos(a);
+      out[((size_t)p * half + j) * 2 + 1] = (float)sin(a);
+    }
+  }
+}
+
+}  // namespace bs

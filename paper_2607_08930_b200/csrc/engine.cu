@@ -1,0 +1,539 @@
+// Host controller and C ABI of the mixed-state block-denoising engine: argument checks, request table and
+// pending queue (sorted insert), per-step kernel sequencing, one small read-back per step.
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <string>
+#include <unordered_map>
+#include <vector>
+
+#include "../../include/blockserve.h"
+#include "common.cuh"
+
+using namespace bs;
+
+namespace {
+
+std::string g_init_error;
+
+inline size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
+
+struct Carver {     // hands out 256-byte aligned sub-buffers; with base == nullptr it only counts
+  char* base;
+  size_t off = 0;
+  explicit Carver(void* b) : base(static_cast<char*>(b)) {}
+  template <typename T>
+  T* take(size_t n) {
+    T* p = base ? reinterpret_cast<T*>(base + off) : nullptr;
+    off = align_up(off + n * sizeof(T));
+    return p;
+  }
+};
+
+constexpr long long kMlpChunk = 16384;    // tokens per MLP pass (bounds the gate/up activation buffer)
+
+struct Workspace {
+  float* rope;      // [max_row_tokens, dh/2, 2]
+  float* x;         // [T, d] residual stream, fp32
+  bf16* h;          // [T, d]
+  bf16* qkv;        // [T, (Hq + 2 Hkv) dh]
+  bf16* attn;       // [T, Hq dh]
+  bf16* act;        // [min(T, chunk), ffn]
+  bf16* hf;         // [max_batch L, d]
+  float* logits;    // [max_batch L, V]
+};
+
+size_t carve_workspace(const bs_config& c, void* base, Workspace* w) {
+  Carver cv(base);
+  const size_t T = (size_t)c.kv_capacity_tokens, mm = (size_t)c.max_batch * c.block_len;
+  Workspace t;
+  t.rope = cv.take<float>((size_t)c.max_row_tokens * c.head_dim);
+  t.x = cv.take<float>(T * c.d_model);
+  t.h = cv.take<bf16>(T * c.d_model);
+  t.qkv = cv.take<bf16>(T * (size_t)(c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim);
+  t.attn = cv.take<bf16>(T * (size_t)c.n_q_heads * c.head_dim);
+  t.act = cv.take<bf16>(std::min<size_t>(T, kMlpChunk) * c.d_ffn);
+  t.hf = cv.take<bf16>(mm * c.d_model);
+  t.logits = cv.take<float>(mm * c.vocab);
+  if (w) *w = t;
+  return cv.off;
+}
+
+size_t carve_state(const bs_config& c, void* base, DevState* out) {
+  Carver cv(base);
+  DevState st;
+  memset(&st, 0, sizeof(st));
+  const size_t R = c.max_requests, B = c.max_batch, T = (size_t)c.kv_capacity_tokens, mm = B * c.block_len;
+  // header and row masks are contiguous: one copy mirrors both to the host
+  st.hdr = cv.take<int>(kHdrInts + B);
+  st.row_mask = base ? reinterpret_cast<unsigned*>(st.hdr + kHdrInts) : nullptr;
+  st.req_p = cv.take<int>(R); st.req_g = cv.take<int>(R); st.req_b = cv.take<int>(R);
+  st.req_state = cv.take<int>(R); st.req_committed = cv.take<int>(R); st.req_alpha = cv.take<float>(R);
+  st.tokens = cv.take<int>(R * c.max_row_tokens);
+  st.queue = cv.take<int>(R);
+  st.row_slot = cv.take<int>(B); st.row_s = cv.take<int>(B); st.row_kv_base = cv.take<int>(B);
+  st.row_vis = cv.take<int>(B);
+  for (int k = 0; k < 2; ++k) {
+    st.cu_q[k] = cv.take<int>(B + 1); st.lm_base[k] = cv.take<int>(B + 1); st.cu_tile[k] = cv.take<int>(B + 1);
+    st.lm_tok[k] = cv.take<int>(mm); st.lm_row[k] = cv.take<int>(mm); st.lm_slot[k] = cv.take<int>(mm);
+    st.out_tok[k] = cv.take<int>(mm); st.out_conf[k] = cv.take<float>(mm); st.out_commit[k] = cv.take<int>(mm);
+    st.lm_scale[k] = cv.take<float>(mm);
+  }
+  st.tok_row = cv.take<int>(T); st.tok_pos = cv.take<int>(T); st.tok_kv = cv.take<int>(T);
+  if (out) *out = st;
+  return cv.off;
+}
+
+const char* check_config(const bs_config& c) {
+  if (c.n_layers < 1 || c.d_model < 8 || c.d_model % 8) return "d_model must be a positive multiple of 8";
+  if (c.head_dim != 64 && c.head_dim != 128) return "head_dim must be 64 or 128";
+  if (c.n_kv_heads < 1 || c.n_q_heads % c.n_kv_heads) return "n_q_heads must be a multiple of n_kv_heads";
+  if (c.n_q_heads / c.n_kv_heads > 8) return "at most 8 query heads per kv head";
+  if (c.d_ffn < 8 || c.d_ffn % 8) return "d_ffn must be a positive multiple of 8";
+  if (c.vocab < 2 || c.vocab % 2) return "vocab must be even";
+  if (c.mask_id < 0 || c.mask_id >= c.vocab) return "mask_id outside the vocabulary";
+  if (c.block_len < 1 || c.block_len > 32) return "block_len must be in [1, 32]";
+  if (c.max_batch < 1 || c.max_batch > 1024) return "max_batch must be in [1, 1024]";
+  if (c.max_requests < 1 || c.max_row_tokens < 2) return "max_requests / max_row_tokens too small";
+  if (c.kv_capacity_tokens < c.max_row_tokens) return "kv_capacity_tokens smaller than one row";
+  if (c.kv_capacity_tokens > (1ll << 30)) return "kv_capacity_tokens too large";
+  if (c.suffix_mode != BS_SUFFIX_FULL && c.suffix_mode != BS_SUFFIX_NONE) return "bad suffix_mode";
+  if (!(c.tau >= 0.f)) return "tau must be >= 0";
+  return nullptr;
+}
+
+}  // namespace
+
+struct bs_engine {
+  bs_config cfg;
+  DevState st;
+  Workspace ws;
+  cudaStream_t stream;
+  bf16* kv;
+  size_t kv_layer_stride;   // elements between layers: 2 * rows * Hkv * dh
+  size_t kv_half;           // elements between K and V of one layer
+  const bf16 *embed, *lm_head, *final_norm;
+  std::vector<const bf16*> wqkv, wo, w_gate, w_up, w_down, norm1, norm2;
+  int* pinned = nullptr;    // hdr + row masks
+  cudaEvent_t ev = nullptr;
+  bool hdr_pending = false;
+  int hdr[kHdrInts];
+  std::unordered_map<long long, int> slot_of;
+  std::vector<long long> id_of_slot;
+  std::vector<int> h_p, h_g, h_b, h_state0;
+  std::vector<float> h_alpha;
+  std::vector<int> pending;
+  int uploaded_slots = 0;
+  bs_stats stats;
+  std::string err;
+};
+
+namespace {
+
+int fail(bs_engine* e, int code, const std::string& msg) {
+  if (e) e->err = msg; else g_init_error = msg;
+  return code;
+}
+int cuda_fail(bs_engine* e, cudaError_t r, const char* what) {
+  return fail(e, BS_E_CUDA, std::string(what) + ": " + cudaGetErrorString(r));
+}
+#define CU(e, call)                                         \
+  do {                                                      \
+    cudaError_t r_ = (call);                                \
+    if (r_ != cudaSuccess) return cuda_fail(e, r_, #call);  \
+  } while (0)
+#define KL(e, call)                                         \
+  do {                                                      \
+    cudaError_t r_ = (call);                                \
+    (e)->stats.kernel_launches++;                           \
+    if (r_ != cudaSuccess) return cuda_fail(e, r_, #call);  \
+  } while (0)
+
+int sync_header(bs_engine* e) {
+  if (e->hdr_pending) {
+    CU(e, cudaEventSynchronize(e->ev));
+    memcpy(e->hdr, e->pinned, sizeof(e->hdr));
+    e->hdr_pending = false;
+    if (e->hdr[H_ERROR] != 0) return fail(e, BS_E_TIMEOUT, "a bounded device-side wait ran out");
+  }
+  return BS_OK;
+}
+
+int post_header(bs_engine* e) {
+  CU(e, cudaMemcpyAsync(e->pinned, e->st.hdr, (kHdrInts + e->cfg.max_batch) * sizeof(int), cudaMemcpyDeviceToHost,
+                        e->stream));
+  CU(e, cudaEventRecord(e->ev, e->stream));
+  e->hdr_pending = true;
+  return BS_OK;
+}
+
+}  // namespace
+
+namespace bs {
+cudaError_t launch_gemm_tc(const bf16* A, int lda, const bf16* W, const bf16* W2, void* C, int ldc, int M, int N,
+                           int K, int mode, const float* row_scale, cudaStream_t s, bool* handled);
+
+cudaError_t launch_gemm(const bf16* A, int lda, const bf16* W, const bf16* W2, void* C, int ldc, int M, int N, int K,
+                        int mode, const float* row_scale, cudaStream_t s) {
+  bool handled = false;
+  cudaError_t r = launch_gemm_tc(A, lda, W, W2, C, ldc, M, N, K, mode, row_scale, s, &handled);
+  if (handled) return r;
+  return launch_gemm_mma(A, lda, W, W2, C, ldc, M, N, K, mode, row_scale, s);
+}
+}  // namespace bs
+
+extern "C" {
+
+int bs_query_sizes(const bs_config* cfg, bs_sizes* out) {
+  if (!cfg || !out) return fail(nullptr, BS_E_ARG, "null argument");
+  if (const char* m = check_config(*cfg)) return fail(nullptr, BS_E_ARG, m);
+  out->kv_bytes = align_up((size_t)cfg->n_layers * 2 * (size_t)cfg->kv_capacity_tokens * cfg->n_kv_heads *
+                           cfg->head_dim * sizeof(bf16));
+  out->workspace_bytes = carve_workspace(*cfg, nullptr, nullptr);
+  out->state_bytes = carve_state(*cfg, nullptr, nullptr);
+  return BS_OK;
+}
+
+int bs_init_model(const bs_config* cfg, const bs_weights* w, void* kv, void* workspace, void* state,
+                  void* cuda_stream, bs_engine** out) {
+  if (!cfg || !w || !kv || !workspace || !state || !out) return fail(nullptr, BS_E_ARG, "null argument");
+  if (const char* m = check_config(*cfg)) return fail(nullptr, BS_E_ARG, m);
+  if (!w->embed || !w->lm_head || !w->final_norm || !w->wqkv || !w->wo || !w->w_gate || !w->w_up || !w->w_down ||
+      !w->norm1 || !w->norm2)
+    return fail(nullptr, BS_E_ARG, "null weight pointer");
+  if (((uintptr_t)kv | (uintptr_t)workspace | (uintptr_t)state) & 255)
+    return fail(nullptr, BS_E_ARG, "device buffers must be 256-byte aligned");
+  int dev_count = 0;
+  if (cudaGetDeviceCount(&dev_count) != cudaSuccess || dev_count == 0)
+    return fail(nullptr, BS_E_CUDA, "no CUDA device: this library has no CPU path");
+  bs_engine* e = new bs_engine();
+  e->cfg = *cfg;
+  e->stream = static_cast<cudaStream_t>(cuda_stream);
+  e->kv = static_cast<bf16*>(kv);
+  e->kv_half = (size_t)cfg->kv_capacity_tokens * cfg->n_kv_heads * cfg->head_dim;
+  e->kv_layer_stride = 2 * e->kv_half;
+  carve_workspace(*cfg, workspace, &e->ws);
+  const size_t state_bytes = carve_state(*cfg, state, &e->st);
+  DevState& st = e->st;
+  st.L = cfg->block_len; st.max_batch = cfg->max_batch; st.max_requests = cfg->max_requests;
+  st.max_row_tokens = cfg->max_row_tokens; st.suffix_mode = cfg->suffix_mode; st.mask_id = cfg->mask_id;
+  st.vocab = cfg->vocab; st.beta = cfg->token_budget; st.kv_capacity = cfg->kv_capacity_tokens; st.tau = cfg->tau;
+  st.q_tile = attention_q_tile(cfg->n_q_heads, cfg->n_kv_heads);
+  e->embed = static_cast<const bf16*>(w->embed);
+  e->lm_head = static_cast<const bf16*>(w->lm_head);
+  e->final_norm = static_cast<const bf16*>(w->final_norm);
+  for (int l = 0; l < cfg->n_layers; ++l) {
+    const void* ptrs[7] = {w->wqkv[l], w->wo[l], w->w_gate[l], w->w_up[l], w->w_down[l], w->norm1[l], w->norm2[l]};
+    for (const void* p : ptrs)
+      if (!p || ((uintptr_t)p & 15)) { delete e; return fail(nullptr, BS_E_ARG, "layer weight null or not 16-byte aligned"); }
+    e->wqkv.push_back((const bf16*)ptrs[0]); e->wo.push_back((const bf16*)ptrs[1]);
+    e->w_gate.push_back((const bf16*)ptrs[2]); e->w_up.push_back((const bf16*)ptrs[3]);
+    e->w_down.push_back((const bf16*)ptrs[4]); e->norm1.push_back((const bf16*)ptrs[5]);
+    e->norm2.push_back((const bf16*)ptrs[6]);
+  }
+  memset(&e->stats, 0, sizeof(e->stats));
+  memset(e->hdr, 0, sizeof(e->hdr));
+  cudaError_t r = cudaMemsetAsync(state, 0, state_bytes, e->stream);
+  if (r == cudaSuccess) r = cudaHostAlloc((void**)&e->pinned, (kHdrInts + cfg->max_batch) * sizeof(int), cudaHostAllocDefault);
+  if (r == cudaSuccess) r = cudaEventCreateWithFlags(&e->ev, cudaEventDisableTiming);
+  if (r == cudaSuccess) {
+    std::vector<float> tab((size_t)cfg->max_row_tokens * cfg->head_dim);
+    build_rope_table(tab.data(), cfg->max_row_tokens, cfg->head_dim, cfg->rope_theta);
+    r = cudaMemcpyAsync(e->ws.rope, tab.data(), tab.size() * sizeof(float), cudaMemcpyHostToDevice, e->stream);
+    if (r == cudaSuccess) r = cudaStreamSynchronize(e->stream);
+  }
+  if (r != cudaSuccess) {
+    std::string msg = std::string("bs_init_model: ") + cudaGetErrorString(r);
+    bs_destroy(e);
+    return fail(nullptr, BS_E_CUDA, msg);
+  }
+  e->h_p.reserve(cfg->max_requests);
+  *out = e;
+  return BS_OK;
+}
+
+int bs_admit(bs_engine* e, long long req_id, const int* prompt, int p, int g, float alpha, int start_block,
+             const int* gen_prefix) {
+  if (!e) return BS_E_ARG;
+  const bs_config& c = e->cfg;
+  const int L = c.block_len;
+  if (!prompt || p < 1 || g < 1 || start_block < 0) return fail(e, BS_E_ARG, "bad request geometry");
+  const int K = (g + L - 1) / L;
+  if (start_block >= K) return fail(e, BS_E_ARG, "start_block must be below K_i");
+  if (start_block > 0 && !gen_prefix) return fail(e, BS_E_ARG, "gen_prefix required when start_block > 0");
+  if (e->slot_of.count(req_id)) return fail(e, BS_E_ARG, "duplicate request id");
+  if ((long long)p + g > c.max_row_tokens) return fail(e, BS_E_KV_FULL, "request longer than max_row_tokens");
+  if ((int)e->id_of_slot.size() >= c.max_requests) return fail(e, BS_E_KV_FULL, "request table full");
+  if (c.token_budget > 0 && (long long)p + (long long)(start_block + 1) * L > c.token_budget)
+    return fail(e, BS_E_BUDGET, "request alone is wider than the token budget");
+  std::vector<int> row((size_t)p + g, c.mask_id);
+  for (int i = 0; i < p; ++i) row[i] = prompt[i];
+  for (int i = 0; i < start_block * L; ++i) row[p + i] = gen_prefix[i];
+  for (int i = 0; i < p + start_block * L; ++i)
+    if (row[i] < 0 || row[i] >= c.vocab || row[i] == c.mask_id) return fail(e, BS_E_ARG, "token id out of range");
+  const int slot = (int)e->id_of_slot.size();
+  // pageable source: the copy has left `row` when the call returns
+  CU(e, cudaMemcpyAsync(e->st.tokens + (size_t)slot * c.max_row_tokens, row.data(), row.size() * sizeof(int),
+                        cudaMemcpyHostToDevice, e->stream));
+  e->slot_of[req_id] = slot;
+  e->id_of_slot.push_back(req_id);
+  e->h_p.push_back(p); e->h_g.push_back(g); e->h_b.push_back(start_block); e->h_alpha.push_back(alpha);
+  // pending queue P: ascending prompt length, ties by submission order (Section 2.4)
+  auto pos = e->pending.end();
+  if (c.sort_queue)
+    pos = std::upper_bound(e->pending.begin(), e->pending.end(), slot,
+                           [&](int a, int b) { return e->h_p[a] < e->h_p[b]; });
+  e->pending.insert(pos, slot);
+  return BS_OK;
+}
+
+int bs_evict_refill(bs_engine* e, int* n_evicted, int* n_admitted, int* n_active) {
+  if (!e) return BS_E_ARG;
+  if (int rc = sync_header(e)) return rc;
+  if (e->hdr[H_N_ACTIVE] > 0 && !e->hdr[H_ALL_DONE]) return fail(e, BS_E_STATE, "a block of this cycle is unfinished");
+  DevState& st = e->st;
+  const int n_slots = (int)e->id_of_slot.size(), first = e->uploaded_slots;
+  if (n_slots > first) {
+    const size_t n = n_slots - first;
+    std::vector<int> zeros(n, 0);
+    CU(e, cudaMemcpyAsync(st.req_p + first, e->h_p.data() + first, n * 4, cudaMemcpyHostToDevice, e->stream));
+    CU(e, cudaMemcpyAsync(st.req_g + first, e->h_g.data() + first, n * 4, cudaMemcpyHostToDevice, e->stream));
+    CU(e, cudaMemcpyAsync(st.req_b + first, e->h_b.data() + first, n * 4, cudaMemcpyHostToDevice, e->stream));
+    CU(e, cudaMemcpyAsync(st.req_alpha + first, e->h_alpha.data() + first, n * 4, cudaMemcpyHostToDevice, e->stream));
+    CU(e, cudaMemcpyAsync(st.req_state + first, zeros.data(), n * 4, cudaMemcpyHostToDevice, e->stream));
+    CU(e, cudaMemcpyAsync(st.req_committed + first, zeros.data(), n * 4, cudaMemcpyHostToDevice, e->stream));
+    e->uploaded_slots = n_slots;
+  }
+  if (!e->pending.empty())
+    CU(e, cudaMemcpyAsync(st.queue, e->pending.data(), e->pending.size() * 4, cudaMemcpyHostToDevice, e->stream));
+  const int qh[2] = {0, (int)e->pending.size()};
+  CU(e, cudaMemcpyAsync(st.hdr + H_QUEUE_HEAD, qh, sizeof(qh), cudaMemcpyHostToDevice, e->stream));
+  KL(e, launch_sched(st, e->stream));
+  if (int rc = post_header(e)) return rc;
+  if (int rc = sync_header(e)) return rc;
+  const int adm = e->hdr[H_ADMITTED];
+  e->pending.erase(e->pending.begin(), e->pending.begin() + adm);
+  if (e->hdr[H_N_ACTIVE] > 0) {
+    e->stats.cycles++;
+    e->stats.sum_active += e->hdr[H_N_ACTIVE];
+  }
+  if (n_evicted) *n_evicted = e->hdr[H_EVICTED];
+  if (n_admitted) *n_admitted = adm;
+  if (n_active) *n_active = e->hdr[H_N_ACTIVE];
+  return BS_OK;
+}
+
+int bs_denoise_step(bs_engine* e, int* n_committed) {
+  if (!e) return BS_E_ARG;
+  if (int rc = sync_header(e)) return rc;
+  const int M = e->hdr[H_M], Mm = e->hdr[H_MM], parity = e->hdr[H_PARITY], n_rows = e->hdr[H_N_ACTIVE];
+  if (n_rows == 0 || M == 0 || Mm == 0) return fail(e, BS_E_STATE, "no unfinished block to denoise");
+  const bs_config& c = e->cfg;
+  DevState& st = e->st;
+  Workspace& ws = e->ws;
+  cudaStream_t s = e->stream;
+  const int d = c.d_model, hq = c.n_q_heads, hkv = c.n_kv_heads, dh = c.head_dim;
+  const int qkv_n = (hq + 2 * hkv) * dh;
+
+  KL(e, launch_fill_tokens(st, parity, M, s));
+  KL(e, launch_embed(st, e->embed, ws.x, M, d, s));
+  for (int l = 0; l < c.n_layers; ++l) {
+    bf16* kc = e->kv + (size_t)l * e->kv_layer_stride;
+    bf16* vc = kc + e->kv_half;
+    KL(e, launch_rmsnorm(ws.x, nullptr, e->norm1[l], ws.h, M, d, c.rms_eps, s));
+    KL(e, launch_gemm(ws.h, d, e->wqkv[l], nullptr, ws.qkv, qkv_n, M, qkv_n, d, 0, nullptr, s));
+    KL(e, launch_rope_kv(ws.qkv, st.tok_pos, st.tok_kv, kc, vc, M, hq, hkv, dh, ws.rope, s));
+    KL(e, launch_attention(ws.qkv, kc, vc, ws.attn, st.cu_q[parity], st.cu_tile[parity], st.row_kv_base, st.row_vis,
+                           n_rows, e->hdr[H_QTILES], hq, hkv, dh, s));
+    KL(e, launch_gemm(ws.attn, hq * dh, e->wo[l], nullptr, ws.x, d, M, d, hq * dh, 1, nullptr, s));
+    for (long long c0 = 0; c0 < M; c0 += kMlpChunk) {
+      const int mc = (int)std::min<long long>(kMlpChunk, M - c0);
+      float* xc = ws.x + (size_t)c0 * d;
+      KL(e, launch_rmsnorm(xc, nullptr, e->norm2[l], ws.h, mc, d, c.rms_eps, s));
+      KL(e, launch_gemm(ws.h, d, e->w_gate[l], e->w_up[l], ws.act, c.d_ffn, mc, c.d_ffn, d, 3, nullptr, s));
+      KL(e, launch_gemm(ws.act, c.d_ffn, e->w_down[l], nullptr, xc, d, mc, d, c.d_ffn, 1, nullptr, s));
+    }
+  }
+  // final norm on the still-masked rows only, LM head scaled by alpha_i, confidence / argmax, commit
+  KL(e, launch_rmsnorm(ws.x, st.lm_tok[parity], e->final_norm, ws.hf, Mm, d, c.rms_eps, s));
+  KL(e, launch_gemm(ws.hf, d, e->lm_head, nullptr, ws.logits, c.vocab, Mm, c.vocab, d, 2, st.lm_scale[parity], s));
+  KL(e, launch_confidence(ws.logits, Mm, c.vocab, c.mask_id, st.out_tok[parity], st.out_conf[parity], s));
+  KL(e, launch_commit_index(st, s));
+  if (int rc = post_header(e)) return rc;
+  e->stats.steps++;
+  e->stats.packed_tokens += M;
+  e->stats.lm_rows += Mm;
+  if (n_committed) {
+    if (int rc = sync_header(e)) return rc;
+    *n_committed = e->hdr[H_COMMITTED_STEP];
+  }
+  return BS_OK;
+}
+
+int bs_block_done(bs_engine* e, int* all_done, unsigned char* per_row_done) {
+  if (!e) return BS_E_ARG;
+  if (int rc = sync_header(e)) return rc;
+  if (all_done) *all_done = e->hdr[H_ALL_DONE] ? 1 : 0;
+  if (per_row_done) {
+    const unsigned* masks = reinterpret_cast<const unsigned*>(e->pinned + kHdrInts);
+    for (int i = 0; i < e->cfg.max_batch; ++i) per_row_done[i] = (i < e->hdr[H_N_ACTIVE]) ? (masks[i] == 0u) : 1;
+  }
+  return BS_OK;
+}
+
+int bs_read_tokens(bs_engine* e, long long req_id, int* out, int cap, int* n_valid, int* state) {
+  if (!e) return BS_E_ARG;
+  auto it = e->slot_of.find(req_id);
+  if (it == e->slot_of.end()) return fail(e, BS_E_UNKNOWN_REQ, "unknown request id");
+  const int slot = it->second, n = e->h_p[slot] + e->h_g[slot];
+  if (n_valid) *n_valid = n;
+  if (out && cap < n) return fail(e, BS_E_ARG, "output buffer too small");
+  if (int rc = sync_header(e)) return rc;
+  if (out)
+    CU(e, cudaMemcpyAsync(out, e->st.tokens + (size_t)slot * e->cfg.max_row_tokens, (size_t)n * 4,
+                          cudaMemcpyDeviceToHost, e->stream));
+  int stt = BS_REQ_QUEUED;
+  if (slot < e->uploaded_slots)
+    CU(e, cudaMemcpyAsync(&stt, e->st.req_state + slot, 4, cudaMemcpyDeviceToHost, e->stream));
+  CU(e, cudaStreamSynchronize(e->stream));
+  if (state) *state = stt;
+  return BS_OK;
+}
+
+int bs_get_stats(bs_engine* e, bs_stats* out) {
+  if (!e || !out) return BS_E_ARG;
+  if (int rc = sync_header(e)) return rc;
+  e->stats.committed = ((long long)(unsigned)e->hdr[H_TOTAL_HI] << 32) | (unsigned)e->hdr[H_TOTAL_LO];
+  *out = e->stats;
+  return BS_OK;
+}
+
+void bs_destroy(bs_engine* e) {
+  if (!e) return;
+  cudaStreamSynchronize(e->stream);
+  if (e->pinned) cudaFreeHost(e->pinned);
+  if (e->ev) cudaEventDestroy(e->ev);
+  delete e;
+}
+
+const char* bs_last_error(const bs_engine* e) { return e ? e->err.c_str() : g_init_error.c_str(); }
+
+int bs_debug_read(bs_engine* e, int what, int arg0, int arg1, void* host_buf, size_t cap, size_t* n_out) {
+  if (!e || !host_buf) return BS_E_ARG;
+  if (int rc = sync_header(e)) return rc;
+  CU(e, cudaStreamSynchronize(e->stream));
+  DevState& st = e->st;
+  const int n = e->hdr[H_N_ACTIVE], par = e->hdr[H_PARITY], prev = par ^ 1;
+  const void* src = nullptr;
+  size_t bytes = 0;
+  std::vector<long long> ids;
+  int prev_mm = 0;
+  if (what >= BS_DBG_PREV_LM_ROW && what <= BS_DBG_PREV_LOGITS) {
+    // the previous step's list length is the end of its per-row prefix
+    CU(e, cudaMemcpy(&prev_mm, st.lm_base[prev] + n, 4, cudaMemcpyDeviceToHost));
+  }
+  switch (what) {
+    case BS_DBG_HEADER: src = st.hdr; bytes = kHdrInts * 4; break;
+    case BS_DBG_ROW_SLOT: src = st.row_slot; bytes = n * 4; break;
+    case BS_DBG_ROW_MASK: src = st.row_mask; bytes = n * 4; break;
+    case BS_DBG_ROW_S: src = st.row_s; bytes = n * 4; break;
+    case BS_DBG_ROW_KV_BASE: src = st.row_kv_base; bytes = n * 4; break;
+    case BS_DBG_CU_Q: src = st.cu_q[par]; bytes = (n + 1) * 4; break;
+    case BS_DBG_TOK_ROW: src = st.tok_row; bytes = (size_t)arg0 * 4; break;
+    case BS_DBG_TOK_POS: src = st.tok_pos; bytes = (size_t)arg0 * 4; break;
+    case BS_DBG_TOK_KV: src = st.tok_kv; bytes = (size_t)arg0 * 4; break;
+    case BS_DBG_LM_TOK: src = st.lm_tok[par]; bytes = (size_t)e->hdr[H_MM] * 4; break;
+    case BS_DBG_LM_ROW: src = st.lm_row[par]; bytes = (size_t)e->hdr[H_MM] * 4; break;
+    case BS_DBG_LM_SLOT: src = st.lm_slot[par]; bytes = (size_t)e->hdr[H_MM] * 4; break;
+    case BS_DBG_PREV_LM_ROW: src = st.lm_row[prev]; bytes = (size_t)prev_mm * 4; break;
+    case BS_DBG_PREV_LM_SLOT: src = st.lm_slot[prev]; bytes = (size_t)prev_mm * 4; break;
+    case BS_DBG_PREV_TOK: src = st.out_tok[prev]; bytes = (size_t)prev_mm * 4; break;
+    case BS_DBG_PREV_CONF: src = st.out_conf[prev]; bytes = (size_t)prev_mm * 4; break;
+    case BS_DBG_PREV_COMMIT: src = st.out_commit[prev]; bytes = (size_t)prev_mm * 4; break;
+    case BS_DBG_PREV_LOGITS: src = e->ws.logits; bytes = (size_t)prev_mm * e->cfg.vocab * 4; break;
+    case BS_DBG_REQ_ID_OF_ROW: {
+      std::vector<int> slots(n);
+      if (n) CU(e, cudaMemcpy(slots.data(), st.row_slot, n * 4, cudaMemcpyDeviceToHost));
+      ids.resize(n);
+      for (int i = 0; i < n; ++i) ids[i] = e->id_of_slot[slots[i]];
+      bytes = (size_t)n * 8;
+      if (bytes > cap) return fail(e, BS_E_ARG, "debug buffer too small");
+      memcpy(host_buf, ids.data(), bytes);
+      if (n_out) *n_out = bytes;
+      return BS_OK;
+    }
+    case BS_DBG_KV_ROW: {
+      if (arg0 < 0 || arg0 >= e->cfg.n_layers || arg1 < 0 || arg1 >= e->cfg.kv_capacity_tokens)
+        return fail(e, BS_E_ARG, "bad layer / row");
+      const size_t rowe = (size_t)e->cfg.n_kv_heads * e->cfg.head_dim;
+      bytes = 2 * rowe * sizeof(bf16);
+      if (bytes > cap) return fail(e, BS_E_ARG, "debug buffer too small");
+      const bf16* kc = e->kv + (size_t)arg0 * e->kv_layer_stride + (size_t)arg1 * rowe;
+      CU(e, cudaMemcpy(host_buf, kc, rowe * sizeof(bf16), cudaMemcpyDeviceToHost));
+      CU(e, cudaMemcpy((char*)host_buf + rowe * sizeof(bf16), kc + e->kv_half, rowe * sizeof(bf16), cudaMemcpyDeviceToHost));
+      if (n_out) *n_out = bytes;
+      return BS_OK;
+    }
+    default: return fail(e, BS_E_ARG, "unknown debug selector");
+  }
+  if (bytes > cap) return fail(e, BS_E_ARG, "debug buffer too small");
+  if (bytes) CU(e, cudaMemcpy(host_buf, src, bytes, cudaMemcpyDeviceToHost));
+  if (n_out) *n_out = bytes;
+  return BS_OK;
+}
+
+// ---- single operations ----------------------------------------------------------------------------------
+
+int bs_op_gemm(const void* A, int lda, const void* W, const void* W2, void* C, int ldc, int M, int N, int K, int mode,
+               const float* row_scale, void* stream) {
+  if (M == 0) return BS_OK;
+  if (!A || !W || !C || M < 0 || N < 1 || K < 8 || K % 8 || N % 2 || mode < 0 || mode > 3) return BS_E_ARG;
+  if (mode == 3 && !W2) return BS_E_ARG;
+  if (mode == 2 && !row_scale) return BS_E_ARG;
+  if (lda % 8 || (((uintptr_t)A | (uintptr_t)W | (uintptr_t)W2) & 15)) return BS_E_ARG;
+  cudaError_t r = launch_gemm((const bf16*)A, lda, (const bf16*)W, (const bf16*)W2, C, ldc, M, N, K, mode, row_scale,
+                              (cudaStream_t)stream);
+  return r == cudaSuccess ? BS_OK : BS_E_CUDA;
+}
+
+int bs_op_rmsnorm(const float* x, const int* idx, const void* w, void* y, int M, int d, float eps, void* stream) {
+  if (!x || !w || !y || M < 0 || d < 8 || d % 8) return BS_E_ARG;
+  return launch_rmsnorm(x, idx, (const bf16*)w, (bf16*)y, M, d, eps, (cudaStream_t)stream) == cudaSuccess ? BS_OK
+                                                                                                          : BS_E_CUDA;
+}
+
+int bs_op_rope_kv(void* qkv, const int* tok_pos, const int* tok_kv, void* kcache, void* vcache, int M, int n_q_heads,
+                  int n_kv_heads, int head_dim, float theta, int max_pos, float* table_scratch, void* stream) {
+  if (!qkv || !tok_pos || !tok_kv || !kcache || !vcache || !table_scratch || M < 0 || head_dim % 8 || max_pos < 1)
+    return BS_E_ARG;
+  std::vector<float> tab((size_t)max_pos * head_dim);
+  build_rope_table(tab.data(), max_pos, head_dim, theta);
+  cudaStream_t s = (cudaStream_t)stream;
+  if (cudaMemcpyAsync(table_scratch, tab.data(), tab.size() * 4, cudaMemcpyHostToDevice, s) != cudaSuccess)
+    return BS_E_CUDA;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return BS_E_CUDA;
+  return launch_rope_kv((bf16*)qkv, tok_pos, tok_kv, (bf16*)kcache, (bf16*)vcache, M, n_q_heads, n_kv_heads, head_dim,
+                        table_scratch, s) == cudaSuccess ? BS_OK : BS_E_CUDA;
+}
+
+int bs_op_attention_q_tile(int n_q_heads, int n_kv_heads) {
+  if (n_kv_heads < 1 || n_q_heads % n_kv_heads) return BS_E_ARG;
+  return attention_q_tile(n_q_heads, n_kv_heads);
+}
+
+int bs_op_attention(const void* qkv, const void* kcache, const void* vcache, void* out, const int* cu_q,
+                    const int* cu_tile, const int* kv_base, const int* vis, int n_rows, int n_tiles, int n_q_heads,
+                    int n_kv_heads, int head_dim, void* stream) {
+  if (!qkv || !kcache || !vcache || !out || !cu_q || !cu_tile || !kv_base || !vis) return BS_E_ARG;
+  return launch_attention((const bf16*)qkv, (const bf16*)kcache, (const bf16*)vcache, (bf16*)out, cu_q, cu_tile,
+                          kv_base, vis, n_rows, n_tiles, n_q_heads, n_kv_heads, head_dim,
+                          (cudaStream_t)stream) == cudaSuccess ? BS_OK : BS_E_CUDA;
+}
+
+int bs_op_confidence(const float* logits, int n_rows, int vocab, int mask_id, int* tok, float* conf, void* stream) {
+  if (!logits || !tok || !conf || n_rows < 0 || vocab < 2) return BS_E_ARG;
+  return launch_confidence(logits, n_rows, vocab, mask_id, tok, conf, (cudaStream_t)stream) == cudaSuccess ? BS_OK
+                                                                                                           : BS_E_CUDA;
+}
+
+}  // extern "C"

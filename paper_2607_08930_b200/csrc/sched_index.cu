@@ -1,0 +1,321 @@
+// Scheduling and gather/scatter index kernels (integer work, single CTA):
+//   k_sched        - Algorithm 1's block boundary: advance, evict, stable compaction, refill under Eq. 1
+//   k_commit_index - confidence-thresholded commit per request + block-done flags + next step's indices
+//   k_fill_tokens  - per packed token: row, logical position id, physical KV row (Section 2.5)
+#include "common.cuh"
+
+namespace bs {
+
+constexpr int kSchedThreads = 1024;
+
+__device__ __forceinline__ int warp_incl_scan(int v) {
+  const int lane = threadIdx.x & 31;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    int t = __shfl_up_sync(0xffffffffu, v, o);
+    if (lane >= o) v += t;
+  }
+  return v;
+}
+
+// Exclusive prefix sum over the block (blockDim.x == 1024).  sm: int[33].
+__device__ int block_excl_scan(int v, int* total, int* sm) {
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  int inc = warp_incl_scan(v);
+  if (lane == 31) sm[w] = inc;
+  __syncthreads();
+  if (w == 0) {
+    int x = sm[lane];
+    int xi = warp_incl_scan(x);
+    sm[lane] = xi - x;
+    if (lane == 31) sm[32] = xi;
+  }
+  __syncthreads();
+  int r = inc - v + sm[w];
+  *total = sm[32];
+  __syncthreads();
+  return r;
+}
+
+__device__ long long block_max_ll(long long v, long long* sm) {   // sm: long long[33]
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    long long t = __shfl_xor_sync(0xffffffffu, v, o);
+    v = t > v ? t : v;
+  }
+  if (lane == 0) sm[w] = v;
+  __syncthreads();
+  if (w == 0) {
+    long long x = sm[lane];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      long long t = __shfl_xor_sync(0xffffffffu, x, o);
+      x = t > x ? t : x;
+    }
+    if (lane == 0) sm[32] = x;
+  }
+  __syncthreads();
+  long long r = sm[32];
+  __syncthreads();
+  return r;
+}
+
+// Index header of the step about to run, for the rows of A in order (all threads of the CTA call this).
+__device__ void build_index(const DevState& st, int parity, int n, int* smi) {
+  const int i = threadIdx.x;
+  int nq = 0, nm = 0, vis = 0, unfinished = 0, refresh = 0;
+  if (i < n) {
+    const int slot = st.row_slot[i];
+    const int p = st.req_p[slot], g = st.req_g[slot], b = st.req_b[slot];
+    const int s = st.row_s[i];
+    const unsigned mask = st.row_mask[i];
+    const int lo = p + b * st.L;
+    const int hi = min(lo + st.L, p + g);
+    vis = st.suffix_mode == 0 ? p + g : hi;
+    st.row_vis[i] = vis;
+    if (mask != 0u) {
+      nq = (s == 0) ? vis : hi - lo;
+      unfinished = 1;
+      refresh = (s == 0);
+    }
+    nm = __popc(mask);
+  }
+  int tot_q, tot_m, tot_t, tot_u, tot_r;
+  const int eq = block_excl_scan(nq, &tot_q, smi);
+  const int em = block_excl_scan(nm, &tot_m, smi);
+  const int et = block_excl_scan((nq + st.q_tile - 1) / st.q_tile, &tot_t, smi);
+  block_excl_scan(unfinished, &tot_u, smi);
+  block_excl_scan(refresh, &tot_r, smi);
+  if (i < n) {
+    st.cu_q[parity][i] = eq;
+    st.lm_base[parity][i] = em;
+    st.cu_tile[parity][i] = et;
+  }
+  if (i == 0) {
+    st.cu_q[parity][n] = tot_q;
+    st.lm_base[parity][n] = tot_m;
+    st.cu_tile[parity][n] = tot_t;
+    st.hdr[H_M] = tot_q;
+    st.hdr[H_MM] = tot_m;
+    st.hdr[H_QTILES] = tot_t;
+    st.hdr[H_ALL_DONE] = (tot_m == 0);
+    st.hdr[H_UNFINISHED] = tot_u;
+    st.hdr[H_STEP_REFRESH] = tot_r;
+    st.hdr[H_PARITY] = parity;
+  }
+  __syncthreads();
+  // still-masked block positions, row order then position order
+  const int lane = threadIdx.x & 31;
+  for (int r = threadIdx.x >> 5; r < n; r += kSchedThreads / 32) {
+    const unsigned mask = st.row_mask[r];
+    if (mask == 0u) continue;
+    if ((mask >> lane) & 1u) {
+      const int slot = st.row_slot[r];
+      const int lo = st.req_p[slot] + st.req_b[slot] * st.L;
+      const int k = st.lm_base[parity][r] + __popc(mask & ((1u << lane) - 1u));
+      st.lm_tok[parity][k] = st.cu_q[parity][r] + (st.row_s[r] == 0 ? lo + lane : lane);
+      st.lm_row[parity][k] = r;
+      st.lm_slot[parity][k] = lane;
+      st.lm_scale[parity][k] = st.req_alpha[slot];
+    }
+  }
+}
+
+__global__ void __launch_bounds__(kSchedThreads) k_sched(DevState st) {
+  __shared__ int smi[33];
+  __shared__ long long sml[33];
+  __shared__ int s_n, s_head, s_stop;
+  __shared__ long long s_w;
+  const int i = threadIdx.x;
+  const int n0 = st.hdr[H_N_ACTIVE];
+  const int L = st.L;
+
+  // ---- advance every active row by one block, evict finished rows, compact (order preserved) ----
+  int keep = 0, slot = -1, kvb = 0;
+  if (i < n0) {
+    slot = st.row_slot[i];
+    kvb = st.row_kv_base[i];
+    const int b = st.req_b[slot] + 1;
+    st.req_b[slot] = b;
+    const int K = (st.req_g[slot] + L - 1) / L;          // K_i = ceil(g_i / L)
+    keep = b < K;
+    if (!keep) st.req_state[slot] = 2;
+  }
+  int n_keep;
+  const int dst = block_excl_scan(keep, &n_keep, smi);
+  if (keep) {
+    st.row_slot[dst] = slot;
+    st.row_kv_base[dst] = kvb;
+  }
+  __syncthreads();
+
+  // ---- width of the bounding box over survivors: max_i p_i + (b_i + 1) L ----
+  long long w = 0;
+  if (i < n_keep) {
+    const int sl = st.row_slot[i];
+    w = (long long)st.req_p[sl] + (long long)(st.req_b[sl] + 1) * L;
+  }
+  w = block_max_ll(w, sml);
+  if (i == 0) {
+    s_n = n_keep;
+    s_head = st.hdr[H_QUEUE_HEAD];
+    s_w = w;
+    s_stop = 0;
+  }
+  __syncthreads();
+
+  // ---- refill: admit the head of P while Eq. 1 holds, the cap holds and the arena has a hole ----
+  const int qlen = st.hdr[H_QUEUE_LEN];
+  while (true) {
+    const int n = s_n, head = s_head;
+    if (s_stop || head >= qlen || n >= st.max_batch) break;
+    const int c = st.queue[head];
+    const long long wc = (long long)st.req_p[c] + (long long)(st.req_b[c] + 1) * L;
+    const long long w2 = wc > s_w ? wc : s_w;
+    const long long need = (long long)st.req_p[c] + st.req_g[c];
+    bool ok = !(st.beta > 0 && (long long)(n + 1) * w2 > st.beta);
+    long long start = 0;
+    if (ok) {   // lowest-address first fit: jump past the furthest slab that overlaps [start, start + need)
+      long long my_b = -1, my_e = -1;
+      if (i < n) {
+        const int sl = st.row_slot[i];
+        my_b = st.row_kv_base[i];
+        my_e = my_b + st.req_p[sl] + st.req_g[sl];
+      }
+      for (int it = 0; it <= n; ++it) {
+        long long e = (i < n && my_b < start + need && my_e > start) ? my_e : -1;
+        e = block_max_ll(e, sml);
+        if (e < 0) break;
+        start = e;
+      }
+      ok = start + need <= st.kv_capacity;
+    }
+    __syncthreads();
+    if (i == 0) {
+      if (ok) {
+        st.row_slot[n] = c;
+        st.row_kv_base[n] = (int)start;
+        st.req_state[c] = 1;
+        s_n = n + 1;
+        s_head = head + 1;
+        s_w = w2;
+      } else {
+        s_stop = 1;
+      }
+    }
+    __syncthreads();
+  }
+  const int n = s_n;
+  // ---- every row starts its block fully masked ----
+  if (i < n) {
+    const int sl = st.row_slot[i];
+    const int lo = st.req_p[sl] + st.req_b[sl] * L;
+    const int len = min(L, st.req_p[sl] + st.req_g[sl] - lo);
+    st.row_mask[i] = len >= 32 ? 0xffffffffu : ((1u << len) - 1u);
+    st.row_s[i] = 0;
+  }
+  if (i == 0) {
+    st.hdr[H_N_ACTIVE] = n;
+    st.hdr[H_EVICTED] = n0 - n_keep;
+    st.hdr[H_ADMITTED] = n - n_keep;
+    st.hdr[H_QUEUE_HEAD] = s_head;
+    st.hdr[H_WIDTH] = (int)s_w;
+    st.hdr[H_COMMITTED_STEP] = 0;
+  }
+  __syncthreads();
+  build_index(st, st.hdr[H_PARITY] ^ 1, n, smi);
+}
+
+// Commit rule per request (one warp per row): positions with conf > tau, plus the position of highest
+// confidence (lowest position on ties), so that every step commits at least one token.
+__global__ void __launch_bounds__(kSchedThreads) k_commit_index(DevState st) {
+  __shared__ int smi[33];
+  __shared__ int s_count;
+  const int parity = st.hdr[H_PARITY];
+  const int n = st.hdr[H_N_ACTIVE];
+  const int lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) s_count = 0;
+  __syncthreads();
+  for (int r = threadIdx.x >> 5; r < n; r += kSchedThreads / 32) {
+    const int base = st.lm_base[parity][r];
+    const int nm = st.lm_base[parity][r + 1] - base;
+    if (nm == 0) continue;
+    float conf = -1.0f;
+    int tok = 0, bit = 0;
+    if (lane < nm) {
+      conf = st.out_conf[parity][base + lane];
+      tok = st.out_tok[parity][base + lane];
+      bit = st.lm_slot[parity][base + lane];
+    }
+    float bc = conf;
+    int bj = lane;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float oc = __shfl_xor_sync(0xffffffffu, bc, o);
+      const int oj = __shfl_xor_sync(0xffffffffu, bj, o);
+      if (oc > bc || (oc == bc && oj < bj)) { bc = oc; bj = oj; }
+    }
+    const bool sel = lane < nm && (conf > st.tau || lane == bj);
+    const int slot = st.row_slot[r];
+    if (sel) {
+      const int lo = st.req_p[slot] + st.req_b[slot] * st.L;
+      st.tokens[(size_t)slot * st.max_row_tokens + lo + bit] = tok;
+    }
+    if (lane < nm) st.out_commit[parity][base + lane] = sel ? 1 : 0;
+    const unsigned bits = __reduce_or_sync(0xffffffffu, sel ? (1u << bit) : 0u);
+    if (lane == 0) {
+      st.row_mask[r] &= ~bits;
+      st.row_s[r] += 1;
+      st.req_committed[slot] += __popc(bits);
+      atomicAdd(&s_count, __popc(bits));
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    st.hdr[H_COMMITTED_STEP] = s_count;
+    unsigned long long tot = ((unsigned long long)(unsigned)st.hdr[H_TOTAL_HI] << 32) | (unsigned)st.hdr[H_TOTAL_LO];
+    tot += (unsigned long long)s_count;
+    st.hdr[H_TOTAL_LO] = (int)(unsigned)(tot & 0xffffffffull);
+    st.hdr[H_TOTAL_HI] = (int)(unsigned)(tot >> 32);
+  }
+  __syncthreads();
+  build_index(st, parity ^ 1, n, smi);
+}
+
+__global__ void k_fill_tokens(DevState st, int parity, int M) {
+  const int n = st.hdr[H_N_ACTIVE];
+  const int* cu = st.cu_q[parity];
+  for (int t = blockIdx.x * blockDim.x + threadIdx.x; t < M; t += gridDim.x * blockDim.x) {
+    int lo = 0, hi = n;                  // largest r with cu[r] <= t
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (cu[mid] <= t) lo = mid; else hi = mid;
+    }
+    const int r = lo;
+    const int slot = st.row_slot[r];
+    const int first = st.row_s[r] == 0 ? 0 : st.req_p[slot] + st.req_b[slot] * st.L;
+    const int pos = first + (t - cu[r]);
+    st.tok_row[t] = r;
+    st.tok_pos[t] = pos;                 // logical position id: 0 = first prompt token of the request
+    st.tok_kv[t] = st.row_kv_base[r] + pos;
+  }
+}
+
+cudaError_t launch_sched(const DevState& st, cudaStream_t s) {
+  k_sched<<<1, kSchedThreads, 0, s>>>(st);
+  return cudaGetLastError();
+}
+cudaError_t launch_commit_index(const DevState& st, cudaStream_t s) {
+  k_commit_index<<<1, kSchedThreads, 0, s>>>(st);
+  return cudaGetLastError();
+}
+cudaError_t launch_fill_tokens(const DevState& st, int parity, int M, cudaStream_t s) {
+  if (M <= 0) return cudaSuccess;
+  const int threads = 256;
+  const int blocks = min((M + threads - 1) / threads, 148 * 8);
+  k_fill_tokens<<<blocks, threads, 0, s>>>(st, parity, M);
+  return cudaGetLastError();
+}
+
+}  // namespace bs

@@ -1,0 +1,202 @@
+"""Lockstep comparison of the CUDA engine with the CPU oracle (test infrastructure).
+
+Both sides are fed the same seeded requests and weights.  Before every step the
+gather / scatter indices are compared bit for bit.  After it:
+
+ (1) logits of every still-masked row: max |z_gpu - z_ref| / max |z_ref| <= 2e-2.
+ (2) the epilogue and the commit rule are checked EXACTLY on the engine's own
+     logits: the oracle's confidence() applied to the engine's logits must give
+     the engine's token ids bit for bit and its confidences to 1e-4, and the
+     oracle's commit_set() applied to the engine's confidences must give the
+     engine's commit decisions bit for bit (same fp32 data, same rule).
+ (3) against the oracle's own trajectory: ln(conf) is 2-Lipschitz in the sup
+     norm of the logits (conf = exp(z_max - logsumexp z)), so with D = max |z_gpu -
+     z_ref| over the row, |ln c_gpu - ln c_ref| <= 2 D must hold; rows that also
+     meet the flat 2e-2 relative bound are counted.  Token ids and commit
+     decisions must agree except at near ties, where the oracle adopts the
+     engine's decision so that the trajectories stay comparable.  Each exception
+     is counted in its class:
+       "tau"    oracle confidence within 1e-2 of tau
+       "top2"   oracle's top-2 logit gap below 1e-2
+       "forced" forced pick: oracle confidence at the engine's position within
+                2e-2 relative of the oracle's maximum
+       "noise"  none of the above, but the flip is explained by the measured
+                logit deviation D of that row: top-2 gap < 2 D, or tau inside
+                [c e^{-2D}, c e^{+2D}], or forced-pick confidences within e^{-4D}
+     Anything else fails.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+from oracle import blockserve_oracle as O
+from paper_2607_08930_b200 import binding as B
+
+LOGIT_TOL = 2e-2      # max |z_gpu - z_ref| / max |z_ref| per row
+CONF_TOL = 2e-2       # relative
+
+
+class Lockstep:
+    def __init__(self, wl, weights_cuda, weights_np, suffix_mode=0, kv_capacity=None, sort_queue=True):
+        self.wl = wl
+        self.eng = B.engine_for_workload(wl, weights_cuda, kv_capacity_tokens=kv_capacity, suffix_mode=suffix_mode,
+                                         sort_queue=sort_queue)
+        self.model = O.model_from_weights(wl.shape, weights_np)
+        self.ora = O.Engine(self.model, wl.block_len, wl.tau, wl.token_budget, wl.max_batch,
+                            self.eng.cfg.kv_capacity_tokens, suffix_mode, sort_queue)
+        self.suffix_mode = suffix_mode
+        self.excluded = {"tau": 0, "top2": 0, "forced": 0, "noise": 0}
+        self.conf_rows_within_tol = 0
+        self.rows_checked = 0
+        self.max_logit_err = 0.0
+        self.max_conf_err = 0.0
+        self.steps = 0
+
+    def admit(self, reqs):
+        for r in reqs:
+            self.eng.admit(r.req_id, r.prompt, r.g, r.alpha, r.start_block, r.gen_prefix)
+            self.ora.admit(r.req_id, r.prompt, r.g, r.alpha, r.start_block, r.gen_prefix)
+
+    def evict_refill(self):
+        ev_o, ad_o, n_o = self.ora.evict_refill()
+        ev, ad, n = self.eng.evict_refill()
+        assert (ev, ad, n) == (len(ev_o), len(ad_o), n_o), "eviction / admission counts differ"
+        ids = self.eng.debug(B.DBG_REQ_ID_OF_ROW, np.int64)
+        assert ids.tolist() == [r.req_id for r in self.ora.sched.active], "row order differs"
+        if n:
+            kvb = self.eng.debug(B.DBG_ROW_KV_BASE)
+            assert kvb.tolist() == [r.kv_base for r in self.ora.sched.active], "KV slabs differ"
+        return ev_o, ad_o, n
+
+    def check_indices(self):
+        act = self.ora.sched.active
+        ix = O.build_indices(act, self.wl.block_len, self.suffix_mode)
+        hdr = self.eng.debug(B.DBG_HEADER)
+        assert hdr[1] == len(ix["tok_row"]) and hdr[2] == len(ix["lm_tok"]), "M / M_m differ"
+        assert self.eng.debug(B.DBG_CU_Q).tolist() == ix["cu_q"].tolist()
+        assert self.eng.debug(B.DBG_ROW_MASK, np.uint32).tolist() == [r.mask for r in act]
+        assert self.eng.debug(B.DBG_ROW_S).tolist() == [r.s for r in act]
+        cap = max(1 << 16, 4 * len(ix["lm_tok"]) + 64)
+        assert self.eng.debug(B.DBG_LM_TOK, cap=cap).tolist() == ix["lm_tok"].tolist()
+        assert self.eng.debug(B.DBG_LM_ROW, cap=cap).tolist() == ix["lm_row"].tolist()
+        assert self.eng.debug(B.DBG_LM_SLOT, cap=cap).tolist() == ix["lm_slot"].tolist()
+        return ix
+
+    def step(self):
+        ix = self.check_indices()
+        M, Mm = len(ix["tok_row"]), len(ix["lm_tok"])
+        n_commit = self.eng.denoise_step(want_count=True)
+        cap = 4 * M + 64
+        assert self.eng.debug(B.DBG_TOK_ROW, arg0=M, cap=cap).tolist() == ix["tok_row"].tolist()
+        assert self.eng.debug(B.DBG_TOK_POS, arg0=M, cap=cap).tolist() == ix["tok_pos"].tolist()
+        assert self.eng.debug(B.DBG_TOK_KV, arg0=M, cap=cap).tolist() == ix["tok_kv"].tolist()
+        cap = 4 * Mm + 64
+        g_tok = self.eng.debug(B.DBG_PREV_TOK, cap=cap)
+        g_conf = self.eng.debug(B.DBG_PREV_CONF, np.float32, cap=cap)
+        g_commit = self.eng.debug(B.DBG_PREV_COMMIT, cap=cap).astype(bool)
+        assert self.eng.debug(B.DBG_PREV_LM_ROW, cap=cap).tolist() == ix["lm_row"].tolist()
+        assert len(g_tok) == Mm and int(g_commit.sum()) == n_commit
+        V = self.wl.shape.vocab
+        g_logits = self.eng.debug(B.DBG_PREV_LOGITS, np.float32, cap=4 * Mm * V + 64).reshape(Mm, V)
+        tau = np.float32(self.wl.tau)
+        mask_id = self.wl.shape.mask_id
+        k = 0
+        for r in self.ora.sched.active:
+            if r.mask == 0:
+                continue
+            nm = bin(r.mask).count("1")
+            gt, gc, gs = g_tok[k:k + nm], g_conf[k:k + nm], g_commit[k:k + nm]
+            where = f"req {r.req_id} block {r.b} step {r.s}"
+            # the record holds what the oracle computes on its own; the oracle then advances with the engine's
+            # decisions (identical unless a near tie is counted below)
+            probe = O.denoise_step(self.model, r, self.wl.block_len, self.wl.tau, self.suffix_mode,
+                                   keep_logits=True, override_commit=gs, override_tok=gt)
+            zl = g_logits[k:k + nm]
+            # (1) logits
+            dev = np.abs(zl - probe.logits).max(-1)                       # D per row
+            err = dev / np.abs(probe.logits).max(-1)
+            self.max_logit_err = max(self.max_logit_err, float(err.max()))
+            assert err.max() <= LOGIT_TOL, f"logit error {err.max():.3e} ({where})"
+            # (2) epilogue and commit rule, exact on the engine's own data
+            tok2, conf2 = O.confidence(zl, mask_id)
+            assert (gt == tok2).all(), f"argmax differs from the oracle's on identical logits ({where})"
+            assert (np.abs(gc - conf2) <= 1e-4 * conf2).all(), f"confidence kernel error ({where})"
+            assert (O.commit_set(gc.copy(), self.wl.tau) == gs).all(), f"commit rule differs on identical data ({where})"
+            # (3) against the oracle's own trajectory
+            dln = np.abs(np.log(gc.astype(np.float64)) - np.log(probe.conf.astype(np.float64)))
+            assert (dln <= 2.0 * dev + 1e-4).all(), f"confidence outside the Lipschitz bound ({where})"
+            cerr = np.abs(gc - probe.conf) / probe.conf
+            self.max_conf_err = max(self.max_conf_err, float(cerr.max()))
+            self.conf_rows_within_tol += int((cerr <= CONF_TOL).sum())
+            tok_diff = gt != probe.tok
+            for j in np.nonzero(tok_diff)[0]:
+                if probe.top2_gap[j] < 1e-2:
+                    self.excluded["top2"] += 1
+                elif probe.top2_gap[j] < 2.0 * dev[j]:
+                    self.excluded["noise"] += 1
+                else:
+                    raise AssertionError(f"token differs with top-2 gap {probe.top2_gap[j]:.4f}, D {dev[j]:.4f} ({where})")
+            o_forced = int(np.argmax(probe.conf))
+            forced_pair = None
+            if not (gc > tau).any() and not (probe.conf > tau).any():
+                forced_pair = (o_forced, int(np.nonzero(gs)[0][0]))
+            diff = gs != probe.committed
+            for j in np.nonzero(diff)[0]:
+                c, d2 = float(probe.conf[j]), 2.0 * float(dev[j])
+                if abs(c - float(tau)) < 1e-2:
+                    self.excluded["tau"] += 1
+                elif forced_pair is not None and j in forced_pair:
+                    co, cg = float(probe.conf[forced_pair[0]]), float(probe.conf[forced_pair[1]])
+                    dd = 2.0 * float(max(dev[forced_pair[0]], dev[forced_pair[1]]))
+                    if cg >= (1 - CONF_TOL) * co:
+                        self.excluded["forced"] += 1
+                    elif cg >= np.exp(-2 * dd) * co:
+                        self.excluded["noise"] += 1
+                    else:
+                        raise AssertionError(f"forced pick differs: oracle {co:.5f} vs {cg:.5f} ({where})")
+                elif c * np.exp(-d2) <= float(tau) <= c * np.exp(d2):
+                    self.excluded["noise"] += 1
+                elif not (gc > tau).any() or not (probe.conf > tau).any():
+                    # one side forced its best position while the other had a row above tau: explained only if
+                    # some row's confidence interval straddles tau
+                    if ((probe.conf * np.exp(-2 * dev) <= tau) & (tau <= probe.conf * np.exp(2 * dev))).any():
+                        self.excluded["noise"] += 1
+                    else:
+                        raise AssertionError(f"commit differs at slot {j}: conf {c:.5f} ({where})")
+                else:
+                    raise AssertionError(f"commit decision differs at slot {j}: oracle conf {c:.6f} "
+                                         f"engine conf {gc[j]:.6f} D {dev[j]:.4f} ({where})")
+            self.rows_checked += nm
+            k += nm
+        assert k == Mm
+        self.steps += 1
+        return n_commit
+
+    def run(self, max_cycles=1 << 30, phase1=None):
+        cycles = 0
+        while cycles < max_cycles:
+            _, _, n = self.evict_refill()
+            if phase1 is not None:
+                self.admit(phase1)
+                phase1 = None
+            if n == 0:
+                break
+            while True:
+                self.step()
+                done = self.eng.block_done()
+                assert done == self.ora.block_done()
+                if done:
+                    break
+            cycles += 1
+        return cycles
+
+    def summary(self) -> str:
+        return (f"steps {self.steps} masked rows {self.rows_checked} excluded {self.excluded} "
+                f"max logit err {self.max_logit_err:.2e} max conf err {self.max_conf_err:.2e} "
+                f"rows with conf within {CONF_TOL:g}: {self.conf_rows_within_tol}")
+
+    def check_tokens(self):
+        for r in self.wl.requests:
+            if r.req_id in self.ora.by_id:
+                got, _ = self.eng.read_tokens(r.req_id)
+                assert (got == self.ora.tokens(r.req_id)).all(), f"token row of request {r.req_id} differs"

@@ -1,0 +1,156 @@
+"""Lockstep parity of the whole denoising iteration against the CPU oracle (needs a B200)."""
+import numpy as np
+import pytest
+import torch
+
+import bs_inputs
+from oracle import blockserve_oracle as O
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2607_08930_b200 import build
+    build.build()
+    from paper_2607_08930_b200 import binding
+    return binding
+
+
+def both_weights(shape, seed):
+    w = bs_inputs.make_weights(shape, seed, device="cpu")
+    wc = {k: ([t.cuda() for t in v] if isinstance(v, list) else v.cuda()) for k, v in w.items()}
+    return wc, bs_inputs.weights_to_numpy_f32(w)
+
+
+@pytest.mark.parametrize("suffix_mode", [0, 1])
+def test_config1_full_lockstep(B, suffix_mode):
+    from lockstep import Lockstep
+    wl = bs_inputs.workload(1)
+    wc, wn = both_weights(wl.shape, wl.weight_seed)
+    ls = Lockstep(wl, wc, wn, suffix_mode=suffix_mode)
+    ls.admit([r for r in wl.requests if r.phase == 0])
+    cycles = ls.run(phase1=[r for r in wl.requests if r.phase == 1])
+    ls.check_tokens()
+    st = ls.eng.stats()
+    assert st.committed == wl.committed_target() == sum(r.committed for r in ls.ora.by_id.values())
+    assert cycles == len([t for t in ls.ora.sched.trace if t.n_active])
+    for r in wl.requests:
+        toks, state = ls.eng.read_tokens(r.req_id)
+        assert state == B.REQ_FINISHED and (toks != wl.shape.mask_id).all()
+    print(f"cfg1 suffix={suffix_mode}: {ls.summary()}")
+    assert sum(ls.excluded.values()) < 0.1 * ls.rows_checked
+
+
+def test_mini_gqa_stream_with_budget_and_ragged_blocks(B):
+    from lockstep import Lockstep
+    shape = bs_inputs.MINI_GQA
+    rng = np.random.default_rng(3)
+    n = 10
+    ps = rng.integers(5, 150, size=n)
+    gs = rng.choice([40, 64, 96, 33], size=n)                # ragged last blocks
+    al = rng.choice([1.0, 6.0, 20.0, 60.0], size=n)
+    st = [int(rng.integers(0, -(-int(g) // 32))) for g in gs]
+    wl = bs_inputs.custom_workload(shape, ps, gs, al, st, token_budget=700, max_batch=6, seed=4, tau=0.9)
+    wc, wn = both_weights(shape, 77)
+    ls = Lockstep(wl, wc, wn, kv_capacity=600)
+    ls.admit(wl.requests)
+    ls.run()
+    ls.check_tokens()
+    assert ls.eng.stats().committed == wl.committed_target()
+    print(f"mini-gqa: {ls.summary()}")
+
+
+@pytest.mark.parametrize("tau,expect", [(1.0, "one"), (0.0, "all")])
+def test_tau_extremes(B, tau, expect):
+    shape = bs_inputs.TINY
+    wl = bs_inputs.custom_workload(shape, [11, 30], [64, 40], [4.0, 9.0], tau=tau, seed=8)
+    wc, _ = both_weights(shape, 5)
+    eng = B.engine_for_workload(wl, wc)
+    for r in wl.requests:
+        eng.admit(r.req_id, r.prompt, r.g, r.alpha)
+    while True:
+        _, _, n = eng.evict_refill()
+        if n == 0:
+            break
+        masks = eng.debug(B.DBG_ROW_MASK, np.uint32)
+        lens = [bin(int(m)).count("1") for m in masks]
+        steps = 0
+        while True:
+            c = eng.denoise_step(want_count=True)
+            steps += 1
+            unfinished = sum(1 for l in lens if l > (steps - 1 if expect == "one" else 0))
+            if expect == "one":
+                assert c == sum(1 for l in lens if l >= steps)      # exactly one token per unfinished row
+            else:
+                assert c == sum(lens)                               # tau = 0: everything in one step
+            if eng.block_done():
+                break
+        assert steps == (max(lens) if expect == "one" else 1)
+    assert eng.stats().committed == wl.committed_target()
+
+
+def test_scheduler_replay_cfg5_geometry(B):
+    """Model-free part of the contract: with tau = 0 every block ends in one step, so the schedule depends on
+    the request geometry only; every eviction, admission, row order and KV slab must match the oracle."""
+    wl5 = bs_inputs.workload(5)
+    shape = bs_inputs.ModelShape("sched", 1, 64, 1, 1, 64, 64, 64, init_std=0.1)
+    rng = np.random.default_rng(0)
+    reqs = [bs_inputs.Request(r.req_id, rng.integers(0, 63, size=r.p).astype(np.int32), r.g, 1.0)
+            for r in wl5.requests[:400]]
+    wl = bs_inputs.Workload("cfg5-geometry", shape, 32, 0.0, wl5.token_budget, wl5.max_batch, reqs)
+    wc, _ = both_weights(shape, 1)
+    cap = 49152
+    eng = B.engine_for_workload(wl, wc, kv_capacity_tokens=cap)
+    sched = O.Scheduler(32, wl.token_budget, wl.max_batch, cap)
+    for r in reqs:
+        eng.admit(r.req_id, r.prompt, r.g, r.alpha)
+        sched.submit(O.ReqState(r.req_id, r.p, r.g, 1.0, np.zeros(1, np.int32), 0))
+    cycles = 0
+    while True:
+        ev_o, ad_o = sched.evict_refill()
+        ev, ad, n = eng.evict_refill()
+        assert (ev, ad, n) == (len(ev_o), len(ad_o), len(sched.active))
+        assert eng.debug(B.DBG_REQ_ID_OF_ROW, np.int64).tolist() == [r.req_id for r in sched.active]
+        if n == 0:
+            break
+        assert eng.debug(B.DBG_ROW_KV_BASE).tolist() == [r.kv_base for r in sched.active]
+        hdr = eng.debug(B.DBG_HEADER)
+        assert hdr[13] == sched.trace[-1].width
+        eng.denoise_step()
+        assert eng.block_done()
+        for r in sched.active:
+            r.mask = 0
+        cycles += 1
+    st = eng.stats()
+    assert st.cycles == cycles and st.sum_active == sum(t.n_active for t in sched.trace)
+    assert st.committed == sum(r.g for r in reqs)
+
+
+def test_state_errors(B):
+    shape = bs_inputs.TINY
+    wl = bs_inputs.custom_workload(shape, [10], [32], [4.0], token_budget=100, max_batch=2)
+    wc, _ = both_weights(shape, 5)
+    eng = B.engine_for_workload(wl, wc)
+    with pytest.raises(B.BlockServeError) as ei:
+        eng.denoise_step()
+    assert ei.value.code == B.BS_E_STATE
+    with pytest.raises(B.BlockServeError) as ei:
+        eng.admit(1, np.arange(90), 32, 1.0)                      # wider than the budget
+    assert ei.value.code in (B.BS_E_BUDGET, B.BS_E_KV_FULL)
+    with pytest.raises(B.BlockServeError) as ei:
+        eng.admit(2, [shape.mask_id], 32, 1.0)
+    assert ei.value.code == B.BS_E_ARG
+    with pytest.raises(B.BlockServeError) as ei:
+        eng.read_tokens(99)
+    assert ei.value.code == B.BS_E_UNKNOWN_REQ
+    r = wl.requests[0]
+    eng.admit(r.req_id, r.prompt, r.g, r.alpha)
+    toks, state = eng.read_tokens(r.req_id)
+    assert state == B.REQ_QUEUED and (toks[r.p:] == shape.mask_id).all()
+    eng.evict_refill()
+    eng.denoise_step()
+    if not eng.block_done():
+        with pytest.raises(B.BlockServeError) as ei:
+            eng.evict_refill()
+        assert ei.value.code == B.BS_E_STATE

@@ -1,0 +1,171 @@
+"""Per-kernel parity against the CPU oracle's functions, through the C ABI (needs a B200)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import blockserve_oracle as O
+
+pytestmark = pytest.mark.gpu
+F32 = np.float32
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2607_08930_b200 import build
+    build.build()
+    from paper_2607_08930_b200 import binding
+    return binding
+
+
+def bf16_round(a):
+    return torch.from_numpy(np.asarray(a, dtype=F32)).to(torch.bfloat16)
+
+
+def rel_err(got, ref):
+    return float(np.abs(got - ref).max() / max(np.abs(ref).max(), 1e-30))
+
+
+GEMM_SHAPES = [  # M, N, K: several tiles, ragged tails in every dimension, one case smaller than a tile
+    (1, 128, 64), (33, 200, 72), (128, 256, 128), (130, 1000, 384), (257, 130, 1000), (300, 2000, 256),
+    (517, 704, 256), (64, 4608, 512), (1000, 512, 2048)]
+
+
+@pytest.mark.parametrize("M,N,K", GEMM_SHAPES)
+@pytest.mark.parametrize("mode", [0, 1, 2, 3])
+def test_gemm_modes(B, M, N, K, mode):
+    rng = np.random.default_rng(M * 7 + N * 3 + K + mode)
+    A = bf16_round(rng.normal(size=(M, K)))
+    W = bf16_round(rng.normal(size=(N, K)) * 0.1)
+    W2 = bf16_round(rng.normal(size=(N, K)) * 0.1)
+    a, w, w2 = A.float().numpy(), W.float().numpy(), W2.float().numpy()
+    ref = a.astype(np.float64) @ w.T.astype(np.float64)
+    Ad, Wd, W2d = A.cuda(), W.cuda(), W2.cuda()
+    if mode == 0:
+        got = B.op_gemm(Ad, Wd, 0).float().cpu().numpy()
+        tol = 6e-3
+    elif mode == 1:
+        c0 = rng.normal(size=(M, N)).astype(F32)
+        Cd = torch.from_numpy(c0).cuda()
+        B.op_gemm(Ad, Wd, 1, C_out=Cd)
+        got, ref, tol = Cd.cpu().numpy(), ref + c0, 1e-4
+    elif mode == 2:
+        sc = rng.uniform(0.5, 30.0, size=M).astype(F32)
+        got = B.op_gemm(Ad, Wd, 2, row_scale=torch.from_numpy(sc).cuda()).cpu().numpy()
+        ref, tol = ref * sc[:, None], 1e-4
+    else:
+        up = a.astype(np.float64) @ w2.T.astype(np.float64)
+        ref = O.silu(ref.astype(F32)).astype(np.float64) * up
+        got = B.op_gemm(Ad, Wd, 3, W2=W2d).float().cpu().numpy()
+        tol = 8e-3
+    assert got.shape == ref.shape
+    assert rel_err(got, ref) < tol
+    # element-wise too, so that a wrong tile in a corner cannot hide behind the global maximum
+    assert np.abs(got - ref).max() <= tol * (np.abs(ref) + np.abs(ref).max() * 0.05).max()
+
+
+def test_gemm_strided_rows_and_empty(B):
+    rng = np.random.default_rng(5)
+    big = bf16_round(rng.normal(size=(70, 512))).cuda()
+    A = big[:, :256]                       # lda 512, K 256
+    W = bf16_round(rng.normal(size=(192, 256)) * 0.1).cuda()
+    got = B.op_gemm(A, W, 0).float().cpu().numpy()
+    ref = A.float().cpu().numpy() @ W.float().cpu().numpy().T
+    assert rel_err(got, ref) < 6e-3
+    empty = B.op_gemm(big[:0, :256], W, 0)
+    assert empty.shape == (0, 192)
+
+
+@pytest.mark.parametrize("M,d", [(1, 256), (37, 384), (300, 3584)])
+def test_rmsnorm(B, M, d):
+    rng = np.random.default_rng(d)
+    x = (rng.normal(size=(M, d)) * 3).astype(F32)
+    w = bf16_round(1 + 0.1 * rng.normal(size=d))
+    ref = O.rmsnorm(x, w.float().numpy(), 1e-6)
+    got = B.op_rmsnorm(torch.from_numpy(x).cuda(), w.cuda(), 1e-6).float().cpu().numpy()
+    assert np.abs(got - ref).max() <= 1e-2 * np.abs(ref).max() and rel_err(got, ref) < 5e-3
+    idx = rng.permutation(M)[: max(1, M // 2)].astype(np.int32)
+    got = B.op_rmsnorm(torch.from_numpy(x).cuda(), w.cuda(), 1e-6, idx=torch.from_numpy(idx).cuda()).float().cpu().numpy()
+    assert rel_err(got, ref[idx]) < 5e-3
+
+
+@pytest.mark.parametrize("hq,hkv,dh", [(4, 4, 64), (6, 2, 128), (28, 4, 128)])
+def test_rope_and_kv_scatter(B, hq, hkv, dh):
+    rng = np.random.default_rng(hq)
+    M, rows, max_pos = 75, 400, 300
+    qkv = bf16_round(rng.normal(size=(M, (hq + 2 * hkv) * dh)))
+    pos = rng.integers(0, max_pos, size=M).astype(np.int32)
+    kvrow = rng.permutation(rows)[:M].astype(np.int32)
+    kc = torch.zeros(rows, hkv, dh, dtype=torch.bfloat16, device="cuda")
+    vc = torch.zeros_like(kc)
+    qd = qkv.cuda()
+    B.op_rope_kv(qd, torch.from_numpy(pos).cuda(), torch.from_numpy(kvrow).cuda(), kc, vc, hq, hkv, dh, 10000.0, max_pos)
+    x = qkv.float().numpy()
+    q = x[:, :hq * dh].reshape(M, hq, dh)
+    k = x[:, hq * dh:(hq + hkv) * dh].reshape(M, hkv, dh)
+    v = x[:, (hq + hkv) * dh:].reshape(M, hkv, dh)
+    cos, sin = O.rope_cos_sin(pos, dh, 10000.0)
+    q_ref, k_ref = O.apply_rope(q, cos, sin), O.apply_rope(k, cos, sin)
+    got_q = qd.float().cpu().numpy()[:, :hq * dh].reshape(M, hq, dh)
+    assert np.abs(got_q - q_ref).max() < 3e-2 and rel_err(got_q, q_ref) < 8e-3
+    kc_h, vc_h = kc.float().cpu().numpy(), vc.float().cpu().numpy()
+    assert rel_err(kc_h[kvrow], k_ref) < 8e-3
+    assert (vc_h[kvrow] == v).all()                       # v is copied bit for bit
+    untouched = np.setdiff1d(np.arange(rows), kvrow)
+    assert (kc_h[untouched] == 0).all() and (vc_h[untouched] == 0).all()   # only the query rows are written
+
+
+ATTN_CASES = [
+    # hq, hkv, dh, [(n_q, vis)] per row: block steps (n_q = 32 or a ragged tail), refresh rows (n_q = vis), empty rows
+    (4, 4, 64, [(32, 159), (32, 41), (0, 50), (17, 64)]),
+    (6, 2, 128, [(32, 200), (8, 8), (130, 130), (0, 9), (32, 65)]),
+    (28, 4, 128, [(32, 300), (32, 96), (70, 70)]),
+    (32, 32, 128, [(32, 129), (100, 100)]),
+]
+
+
+@pytest.mark.parametrize("hq,hkv,dh,rows", ATTN_CASES)
+def test_ragged_dual_cache_attention(B, hq, hkv, dh, rows):
+    rng = np.random.default_rng(hq * 100 + dh)
+    cap = sum(v for _, v in rows) + 64
+    kc = bf16_round(rng.normal(size=(cap, hkv, dh)))
+    vc = bf16_round(rng.normal(size=(cap, hkv, dh)))
+    M = sum(n for n, _ in rows)
+    qkv = bf16_round(rng.normal(size=(M, (hq + 2 * hkv) * dh)) * 1.5)
+    # slabs in shuffled physical order with gaps, so that kv_base matters
+    order = rng.permutation(len(rows))
+    kv_base = np.zeros(len(rows), np.int32)
+    at = 7
+    for i in order:
+        kv_base[i] = at
+        at += rows[i][1] + 3
+    cu_q = np.zeros(len(rows) + 1, np.int32)
+    cu_q[1:] = np.cumsum([n for n, _ in rows])
+    vis = np.array([v for _, v in rows], np.int32)
+    out = B.op_attention(qkv.cuda(), kc.cuda(), vc.cuda(), torch.from_numpy(cu_q).cuda(),
+                         torch.from_numpy(kv_base).cuda(), torch.from_numpy(vis).cuda(), hq, hkv, dh)
+    got = out.float().cpu().numpy().reshape(M, hq, dh)
+    q = qkv.float().numpy()[:, :hq * dh].reshape(M, hq, dh)
+    K, V = kc.float().numpy(), vc.float().numpy()
+    for i, (n, v) in enumerate(rows):
+        if n == 0:
+            continue
+        ref = O.attention(q[cu_q[i]:cu_q[i + 1]], K[kv_base[i]:kv_base[i] + v], V[kv_base[i]:kv_base[i] + v])
+        g = got[cu_q[i]:cu_q[i + 1]]
+        assert np.abs(g - ref).max() < 2e-2, f"row {i}: {np.abs(g - ref).max()}"
+        assert rel_err(g, ref) < 1e-2
+
+
+@pytest.mark.parametrize("n,V", [(1, 1024), (37, 2000), (64, 152064), (5, 126464)])
+def test_confidence_rows(B, n, V):
+    rng = np.random.default_rng(V)
+    z = (rng.normal(size=(n, V)) * rng.uniform(0.5, 6.0, size=(n, 1))).astype(F32)
+    mask_id = V - 1
+    z[0, mask_id] = 1e4                      # the mask id must never win
+    if n > 2:
+        z[1, :] = 0.25                       # all equal: tok 0, conf 1 / (V - 1)
+        z[2, 100] = z[2, 7] = 50.0           # tie: lowest id
+    tok_ref, conf_ref = O.confidence(z, mask_id)
+    tok, conf = B.op_confidence(torch.from_numpy(z).cuda(), mask_id)
+    tok, conf = tok.cpu().numpy(), conf.cpu().numpy()
+    assert (tok == tok_ref).all()
+    assert (np.abs(conf - conf_ref) / conf_ref).max() < 1e-4

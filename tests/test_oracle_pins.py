@@ -15,10 +15,33 @@ GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
 F32 = np.float32
 
 
-def tiny_model(shape=None, seed=7):
+def tiny_model(shape=None, seed=7, bf16=False):
     shape = shape or bs_inputs.ModelShape("t", 2, 32, 4, 2, 8, 48, 50, init_std=0.3)
     w = bs_inputs.weights_to_numpy_f32(bs_inputs.make_weights(shape, seed))
-    return shape, O.model_from_weights(shape, w)
+    return shape, O.model_from_weights(shape, w, bf16_activations=bf16)
+
+
+def test_round_bf16_against_library_and_ties():
+    rng = np.random.default_rng(0)
+    x = np.concatenate([rng.normal(size=4000) * 10.0 ** rng.integers(-6, 6, size=4000),
+                        [0.0, -0.0, 1.0, 1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8, 1.0 + 2.0 ** -7, 3.3895314e38]]).astype(F32)
+    ref = torch.from_numpy(x).to(torch.bfloat16).float().numpy()
+    got = O.round_bf16(x)
+    assert (got.view(np.uint32) == ref.view(np.uint32)).all()
+    # ties go to the even neighbour: 1 + 2^-8 -> 1, 1 + 3 * 2^-8 -> 1 + 2^-6
+    assert O.round_bf16(np.array([1.0 + 2.0 ** -8], F32))[0] == 1.0
+    assert O.round_bf16(np.array([1.0 + 3 * 2.0 ** -8], F32))[0] == F32(1.0 + 2.0 ** -6)
+    assert np.isinf(O.round_bf16(np.array([np.inf], F32))[0])
+
+
+def test_bf16_activation_mode_stays_close_to_pure_fp32():
+    shape = bs_inputs.ModelShape("t", 3, 64, 4, 2, 16, 96, 50, init_std=0.2)
+    w = bs_inputs.weights_to_numpy_f32(bs_inputs.make_weights(shape, 11))
+    toks = np.random.default_rng(4).integers(0, 49, size=21)
+    z32 = O.full_forward_logits(O.model_from_weights(shape, w, False), toks, 1.0)
+    z16 = O.full_forward_logits(O.model_from_weights(shape, w, True), toks, 1.0)
+    err = np.abs(z16 - z32).max() / np.abs(z32).max()
+    assert 1e-5 < err < 5e-2          # rounding is on, and it is only rounding
 
 
 # ----------------------------------------------------------------- formulas ---
@@ -202,7 +225,7 @@ def brute_forward(shape, w, tokens, alpha):
 def test_full_forward_against_independent_double_forward():
     shape = bs_inputs.ModelShape("t", 3, 32, 4, 2, 8, 48, 50, init_std=0.3)
     w = bs_inputs.weights_to_numpy_f32(bs_inputs.make_weights(shape, 11))
-    model = O.model_from_weights(shape, w)
+    model = O.model_from_weights(shape, w, bf16_activations=False)
     toks = np.random.default_rng(4).integers(0, 49, size=13)
     got = O.full_forward_logits(model, toks, 2.5)
     ref = brute_forward(shape, w, toks, 2.5)
@@ -253,7 +276,7 @@ def test_cached_step_exact_for_one_layer_and_approximate_for_two():
     for n_layers, expect_exact in ((1, True), (2, False)):
         shape = bs_inputs.ModelShape("t", n_layers, 32, 4, 2, 8, 48, 50, init_std=0.5)
         w = bs_inputs.weights_to_numpy_f32(bs_inputs.make_weights(shape, 5))
-        model = O.model_from_weights(shape, w)
+        model = O.model_from_weights(shape, w, bf16_activations=False)
         r = _mk_req(model, 5, 8, L, alpha=1.0)
         O.denoise_step(model, r, L, 1.0)                      # refresh, commits exactly one token
         row = r.tokens.copy()
