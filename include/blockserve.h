@@ -143,6 +143,28 @@ int bs_block_done(bs_engine* e, int* all_done, unsigned char* per_row_done);
 int bs_read_tokens(bs_engine* e, long long req_id, int* out, int cap, int* n_valid, int* state);
 
 int bs_get_stats(bs_engine* e, bs_stats* out);
+
+/* Per-kernel-family device timing (CUDA events on the engine's stream around each family's launches).
+ * Off by default; switching it on adds two event records per family per layer.  bs_get_profile fills
+ * host arrays of BS_FAM_COUNT entries (any may be NULL): milliseconds, kernel launches, algorithmic
+ * flops and algorithmic bytes accumulated since profiling was switched on (or last reset by enabling again).
+ * Algorithmic bytes: GEMMs count weights + input + output once; attention counts K and V of every
+ * unfinished row once per layer plus q and the output; the epilogue counts the logits once. */
+enum {
+  BS_FAM_INDEX = 0,      /* fill_tokens, commit + next index build, scheduler */
+  BS_FAM_EMBED_NORM = 1, /* embedding gather and RMSNorm launches */
+  BS_FAM_GEMM_QKV = 2,
+  BS_FAM_ROPE_KV = 3,
+  BS_FAM_ATTENTION = 4,
+  BS_FAM_GEMM_O = 5,
+  BS_FAM_GEMM_GATE_UP = 6,
+  BS_FAM_GEMM_DOWN = 7,
+  BS_FAM_GEMM_LM_HEAD = 8,
+  BS_FAM_CONFIDENCE = 9,
+  BS_FAM_COUNT = 10
+};
+int bs_set_profiling(bs_engine* e, int on);
+int bs_get_profile(bs_engine* e, double* ms, long long* launches, double* flops, double* bytes);
 void bs_destroy(bs_engine* e);
 const char* bs_last_error(const bs_engine* e); /* NULL engine: error of the last failed bs_init_model */
 

@@ -26,6 +26,10 @@ REQ_QUEUED, REQ_ACTIVE, REQ_FINISHED = 0, 1, 2
  DBG_PREV_CONF, DBG_PREV_COMMIT, DBG_PREV_LOGITS, DBG_REQ_ID_OF_ROW, DBG_KV_ROW) = range(20)
 
 
+FAMILIES = ("index", "embed_norm", "gemm_qkv", "rope_kv", "attention", "gemm_o", "gemm_gate_up", "gemm_down",
+            "gemm_lm_head", "confidence")
+
+
 class BsConfig(C.Structure):
     _fields_ = [("n_layers", C.c_int), ("d_model", C.c_int), ("n_q_heads", C.c_int), ("n_kv_heads", C.c_int),
                 ("head_dim", C.c_int), ("d_ffn", C.c_int), ("vocab", C.c_int), ("mask_id", C.c_int),
@@ -53,7 +57,7 @@ class BsStats(C.Structure):
 
 
 EXPORTS = ["bs_query_sizes", "bs_init_model", "bs_admit", "bs_evict_refill", "bs_denoise_step", "bs_block_done",
-           "bs_read_tokens", "bs_get_stats", "bs_destroy", "bs_last_error", "bs_debug_read", "bs_op_gemm",
+           "bs_read_tokens", "bs_get_stats", "bs_set_profiling", "bs_get_profile", "bs_destroy", "bs_last_error", "bs_debug_read", "bs_op_gemm",
            "bs_op_rmsnorm", "bs_op_rope_kv", "bs_op_attention_q_tile", "bs_op_attention", "bs_op_confidence"]
 
 _lib = None
@@ -76,6 +80,9 @@ def lib() -> C.CDLL:
         L.bs_block_done.argtypes = [vp, ip, C.POINTER(C.c_ubyte)]
         L.bs_read_tokens.argtypes = [vp, ll, ip, i, ip, ip]
         L.bs_get_stats.argtypes = [vp, C.POINTER(BsStats)]
+        L.bs_set_profiling.argtypes = [vp, i]
+        L.bs_get_profile.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(ll), C.POINTER(C.c_double),
+                                     C.POINTER(C.c_double)]
         L.bs_destroy.argtypes = [vp]
         L.bs_destroy.restype = None
         L.bs_last_error.argtypes = [vp]
@@ -208,6 +215,17 @@ class Engine:
         s = BsStats()
         self._chk(self.L.bs_get_stats(self.h, C.byref(s)))
         return s
+
+    def set_profiling(self, on: bool) -> None:
+        self._chk(self.L.bs_set_profiling(self.h, int(on)))
+
+    def profile(self) -> Dict[str, Dict[str, float]]:
+        """Per kernel family: device ms, launches, algorithmic flops and bytes since profiling was enabled."""
+        n = len(FAMILIES)
+        ms, fl, by = (C.c_double * n)(), (C.c_double * n)(), (C.c_double * n)()
+        la = (C.c_longlong * n)()
+        self._chk(self.L.bs_get_profile(self.h, ms, la, fl, by))
+        return {FAMILIES[i]: dict(ms=ms[i], launches=int(la[i]), flops=fl[i], bytes=by[i]) for i in range(n)}
 
     def debug(self, what: int, dtype=np.int32, arg0: int = 0, arg1: int = 0, cap: int = 1 << 16) -> np.ndarray:
         buf = np.empty(cap, dtype=np.uint8)

@@ -126,6 +126,16 @@ struct bs_engine {
   int uploaded_slots = 0;
   bs_stats stats;
   std::string err;
+  // per-family device timing
+  bool profiling = false;
+  std::vector<cudaEvent_t> ev_pool;
+  size_t ev_used = 0;
+  struct Span { int fam; size_t a, b; };
+  std::vector<Span> spans;
+  double prof_ms[BS_FAM_COUNT], prof_flops[BS_FAM_COUNT], prof_bytes[BS_FAM_COUNT];
+  long long prof_launches[BS_FAM_COUNT];
+  int cur_fam = -1;
+  size_t cur_a = 0;
 };
 
 namespace {
@@ -149,9 +159,47 @@ int cuda_fail(bs_engine* e, cudaError_t r, const char* what) {
     if (r_ != cudaSuccess) return cuda_fail(e, r_, #call);  \
   } while (0)
 
+void prof_collect(bs_engine* e) {     // all recorded events have completed when this runs
+  for (const bs_engine::Span& sp : e->spans) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, e->ev_pool[sp.a], e->ev_pool[sp.b]) == cudaSuccess) e->prof_ms[sp.fam] += ms;
+  }
+  e->spans.clear();
+  e->ev_used = 0;
+}
+
+cudaEvent_t prof_event(bs_engine* e, size_t* idx) {
+  if (e->ev_used == e->ev_pool.size()) {
+    cudaEvent_t ev;
+    cudaEventCreate(&ev);
+    e->ev_pool.push_back(ev);
+  }
+  *idx = e->ev_used++;
+  return e->ev_pool[*idx];
+}
+
+// Opens a timed span for `fam` (closing the one in flight); fam < 0 only closes.
+void prof_mark(bs_engine* e, int fam) {
+  if (!e->profiling) return;
+  size_t idx;
+  cudaEvent_t ev = prof_event(e, &idx);
+  cudaEventRecord(ev, e->stream);
+  if (e->cur_fam >= 0) e->spans.push_back({e->cur_fam, e->cur_a, idx});
+  e->cur_fam = fam;
+  e->cur_a = idx;
+}
+
+void prof_work(bs_engine* e, int fam, int launches, double flops, double bytes) {
+  if (!e->profiling) return;
+  e->prof_launches[fam] += launches;
+  e->prof_flops[fam] += flops;
+  e->prof_bytes[fam] += bytes;
+}
+
 int sync_header(bs_engine* e) {
   if (e->hdr_pending) {
     CU(e, cudaEventSynchronize(e->ev));
+    if (e->profiling) prof_collect(e);
     memcpy(e->hdr, e->pinned, sizeof(e->hdr));
     e->hdr_pending = false;
     if (e->hdr[H_ERROR] != 0) return fail(e, BS_E_TIMEOUT, "a bounded device-side wait ran out");
@@ -232,6 +280,7 @@ int bs_init_model(const bs_config* cfg, const bs_weights* w, void* kv, void* wor
     e->norm2.push_back((const bf16*)ptrs[6]);
   }
   memset(&e->stats, 0, sizeof(e->stats));
+  for (int i = 0; i < BS_FAM_COUNT; ++i) e->prof_ms[i] = e->prof_flops[i] = e->prof_bytes[i] = 0.0, e->prof_launches[i] = 0;
   memset(e->hdr, 0, sizeof(e->hdr));
   cudaError_t r = cudaMemsetAsync(state, 0, state_bytes, e->stream);
   if (r == cudaSuccess) r = cudaHostAlloc((void**)&e->pinned, (kHdrInts + cfg->max_batch) * sizeof(int), cudaHostAllocDefault);
@@ -335,30 +384,65 @@ int bs_denoise_step(bs_engine* e, int* n_committed) {
   const int d = c.d_model, hq = c.n_q_heads, hkv = c.n_kv_heads, dh = c.head_dim;
   const int qkv_n = (hq + 2 * hkv) * dh;
 
+  const double dM = (double)M, dd = (double)d, dq = (double)qkv_n, dhq = (double)hq * dh, df = (double)c.d_ffn;
+  const double kv_rows = (double)e->hdr[H_SUM_KV];
+  prof_mark(e, BS_FAM_INDEX);
   KL(e, launch_fill_tokens(st, parity, M, s));
+  prof_work(e, BS_FAM_INDEX, 1, 0, 12.0 * dM);
+  prof_mark(e, BS_FAM_EMBED_NORM);
   KL(e, launch_embed(st, e->embed, ws.x, M, d, s));
+  prof_work(e, BS_FAM_EMBED_NORM, 1, 0, 6.0 * dM * dd);
   for (int l = 0; l < c.n_layers; ++l) {
     bf16* kc = e->kv + (size_t)l * e->kv_layer_stride;
     bf16* vc = kc + e->kv_half;
+    prof_mark(e, BS_FAM_EMBED_NORM);
     KL(e, launch_rmsnorm(ws.x, nullptr, e->norm1[l], ws.h, M, d, c.rms_eps, s));
+    prof_work(e, BS_FAM_EMBED_NORM, 1, 0, 6.0 * dM * dd);
+    prof_mark(e, BS_FAM_GEMM_QKV);
     KL(e, launch_gemm(ws.h, d, e->wqkv[l], nullptr, ws.qkv, qkv_n, M, qkv_n, d, 0, nullptr, s));
+    prof_work(e, BS_FAM_GEMM_QKV, 1, 2.0 * dM * dq * dd, 2.0 * (dq * dd + dM * dd + dM * dq));
+    prof_mark(e, BS_FAM_ROPE_KV);
     KL(e, launch_rope_kv(ws.qkv, st.tok_pos, st.tok_kv, kc, vc, M, hq, hkv, dh, ws.rope, s));
+    prof_work(e, BS_FAM_ROPE_KV, 1, 0, 2.0 * dM * (dq + (double)(hq + 2 * hkv) * dh));
+    prof_mark(e, BS_FAM_ATTENTION);
     KL(e, launch_attention(ws.qkv, kc, vc, ws.attn, st.cu_q[parity], st.cu_tile[parity], st.row_kv_base, st.row_vis,
                            n_rows, e->hdr[H_QTILES], hq, hkv, dh, s));
+    // every query token of a row meets every cache row of that row: flops = 4 * dh * Hq * sum_rows(n_q * vis);
+    // the host knows the sums only for pure block steps and pure refresh steps, else it reports bytes alone
+    prof_work(e, BS_FAM_ATTENTION, 1, 0, 2.0 * (2.0 * kv_rows * hkv * dh + 2.0 * dM * dhq));
+    prof_mark(e, BS_FAM_GEMM_O);
     KL(e, launch_gemm(ws.attn, hq * dh, e->wo[l], nullptr, ws.x, d, M, d, hq * dh, 1, nullptr, s));
+    prof_work(e, BS_FAM_GEMM_O, 1, 2.0 * dM * dd * dhq, 2.0 * (dd * dhq + dM * dhq) + 8.0 * dM * dd);
     for (long long c0 = 0; c0 < M; c0 += kMlpChunk) {
       const int mc = (int)std::min<long long>(kMlpChunk, M - c0);
+      const double dmc = (double)mc;
       float* xc = ws.x + (size_t)c0 * d;
+      prof_mark(e, BS_FAM_EMBED_NORM);
       KL(e, launch_rmsnorm(xc, nullptr, e->norm2[l], ws.h, mc, d, c.rms_eps, s));
+      prof_work(e, BS_FAM_EMBED_NORM, 1, 0, 6.0 * dmc * dd);
+      prof_mark(e, BS_FAM_GEMM_GATE_UP);
       KL(e, launch_gemm(ws.h, d, e->w_gate[l], e->w_up[l], ws.act, c.d_ffn, mc, c.d_ffn, d, 3, nullptr, s));
+      prof_work(e, BS_FAM_GEMM_GATE_UP, 1, 4.0 * dmc * df * dd, 2.0 * (2.0 * df * dd + dmc * dd + dmc * df));
+      prof_mark(e, BS_FAM_GEMM_DOWN);
       KL(e, launch_gemm(ws.act, c.d_ffn, e->w_down[l], nullptr, xc, d, mc, d, c.d_ffn, 1, nullptr, s));
+      prof_work(e, BS_FAM_GEMM_DOWN, 1, 2.0 * dmc * dd * df, 2.0 * (dd * df + dmc * df) + 8.0 * dmc * dd);
     }
   }
   // final norm on the still-masked rows only, LM head scaled by alpha_i, confidence / argmax, commit
+  const double dMm = (double)Mm, dV = (double)c.vocab;
+  prof_mark(e, BS_FAM_EMBED_NORM);
   KL(e, launch_rmsnorm(ws.x, st.lm_tok[parity], e->final_norm, ws.hf, Mm, d, c.rms_eps, s));
+  prof_work(e, BS_FAM_EMBED_NORM, 1, 0, 6.0 * dMm * dd);
+  prof_mark(e, BS_FAM_GEMM_LM_HEAD);
   KL(e, launch_gemm(ws.hf, d, e->lm_head, nullptr, ws.logits, c.vocab, Mm, c.vocab, d, 2, st.lm_scale[parity], s));
+  prof_work(e, BS_FAM_GEMM_LM_HEAD, 1, 2.0 * dMm * dV * dd, 2.0 * (dV * dd + dMm * dd) + 4.0 * dMm * dV);
+  prof_mark(e, BS_FAM_CONFIDENCE);
   KL(e, launch_confidence(ws.logits, Mm, c.vocab, c.mask_id, st.out_tok[parity], st.out_conf[parity], s));
+  prof_work(e, BS_FAM_CONFIDENCE, 1, 0, 4.0 * dMm * dV);
+  prof_mark(e, BS_FAM_INDEX);
   KL(e, launch_commit_index(st, s));
+  prof_work(e, BS_FAM_INDEX, 1, 0, 0);
+  prof_mark(e, -1);
   if (int rc = post_header(e)) return rc;
   e->stats.steps++;
   e->stats.packed_tokens += M;
@@ -408,9 +492,35 @@ int bs_get_stats(bs_engine* e, bs_stats* out) {
   return BS_OK;
 }
 
+int bs_set_profiling(bs_engine* e, int on) {
+  if (!e) return BS_E_ARG;
+  if (int rc = sync_header(e)) return rc;
+  CU(e, cudaStreamSynchronize(e->stream));
+  e->profiling = on != 0;
+  e->spans.clear();
+  e->ev_used = 0;
+  e->cur_fam = -1;
+  if (on)
+    for (int i = 0; i < BS_FAM_COUNT; ++i) e->prof_ms[i] = e->prof_flops[i] = e->prof_bytes[i] = 0.0, e->prof_launches[i] = 0;
+  return BS_OK;
+}
+
+int bs_get_profile(bs_engine* e, double* ms, long long* launches, double* flops, double* bytes) {
+  if (!e) return BS_E_ARG;
+  if (int rc = sync_header(e)) return rc;
+  for (int i = 0; i < BS_FAM_COUNT; ++i) {
+    if (ms) ms[i] = e->prof_ms[i];
+    if (launches) launches[i] = e->prof_launches[i];
+    if (flops) flops[i] = e->prof_flops[i];
+    if (bytes) bytes[i] = e->prof_bytes[i];
+  }
+  return BS_OK;
+}
+
 void bs_destroy(bs_engine* e) {
   if (!e) return;
   cudaStreamSynchronize(e->stream);
+  for (cudaEvent_t ev : e->ev_pool) cudaEventDestroy(ev);
   if (e->pinned) cudaFreeHost(e->pinned);
   if (e->ev) cudaEventDestroy(e->ev);
   delete e;

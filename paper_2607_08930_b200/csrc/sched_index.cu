@@ -87,6 +87,8 @@ __device__ void build_index(const DevState& st, int parity, int n, int* smi) {
   const int et = block_excl_scan((nq + st.q_tile - 1) / st.q_tile, &tot_t, smi);
   block_excl_scan(unfinished, &tot_u, smi);
   block_excl_scan(refresh, &tot_r, smi);
+  int tot_kv;
+  block_excl_scan(unfinished ? vis : 0, &tot_kv, smi);
   if (i < n) {
     st.cu_q[parity][i] = eq;
     st.lm_base[parity][i] = em;
@@ -102,6 +104,7 @@ __device__ void build_index(const DevState& st, int parity, int n, int* smi) {
     st.hdr[H_ALL_DONE] = (tot_m == 0);
     st.hdr[H_UNFINISHED] = tot_u;
     st.hdr[H_STEP_REFRESH] = tot_r;
+    st.hdr[H_SUM_KV] = tot_kv;
     st.hdr[H_PARITY] = parity;
   }
   __syncthreads();
