@@ -204,6 +204,19 @@ int bs_op_rope_kv(void* qkv, const int* tok_pos, const int* tok_kv, void* kcache
                   int n_q_heads, int n_kv_heads, int head_dim, float theta, int max_pos,
                   float* table_scratch /* device float[max_pos * head_dim], overwritten */, void* stream);
 
+/* No counterpart in the paper: bs_op_rope_kv for callers that cannot allocate device memory (a host whose
+ * memory pool is fixed at start-up, a plugin whose runtime owns all allocations).  Same arguments and results
+ * as bs_op_rope_kv without the scratch buffer: the cos/sin table lives in a fixed array inside the library,
+ * BS_ROPE_STATIC_MAX_FLOATS floats (2 MiB) that every GPU loading the library holds until the process exits.
+ * Returns BS_E_ARG when max_pos * head_dim exceeds that size.  The call allocates nothing, on the device or
+ * through any library.  The first call on each device looks up the array's device address (one-time set-up,
+ * with that device current): make it before any stream capture.  All calls share the one table, which keeps
+ * the previous call's contents and is rewritten for [0, max_pos) by each call: two calls whose kernels can
+ * overlap on the GPU (different streams, no ordering between them) race on it. */
+#define BS_ROPE_STATIC_MAX_FLOATS (512 * 1024)
+int bs_op_rope_kv_static(void* qkv, const int* tok_pos, const int* tok_kv, void* kcache, void* vcache, int M,
+                         int n_q_heads, int n_kv_heads, int head_dim, float theta, int max_pos, void* stream);
+
 /* Ragged bidirectional attention of packed queries against per-row cache spans:
  * row i owns packed tokens [cu_q[i], cu_q[i+1]) and attends over cache rows
  * [kv_base[i], kv_base[i] + vis[i]) (prefix, fresh block and suffix alike; no causal or padding mask).

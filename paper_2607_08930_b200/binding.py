@@ -58,7 +58,7 @@ class BsStats(C.Structure):
 
 EXPORTS = ["bs_query_sizes", "bs_init_model", "bs_admit", "bs_evict_refill", "bs_denoise_step", "bs_block_done",
            "bs_read_tokens", "bs_get_stats", "bs_set_profiling", "bs_get_profile", "bs_destroy", "bs_last_error", "bs_debug_read", "bs_op_gemm",
-           "bs_op_rmsnorm", "bs_op_rope_kv", "bs_op_attention_q_tile", "bs_op_attention", "bs_op_confidence"]
+           "bs_op_rmsnorm", "bs_op_rope_kv", "bs_op_rope_kv_static", "bs_op_attention_q_tile", "bs_op_attention", "bs_op_confidence"]
 
 _lib = None
 
@@ -91,6 +91,7 @@ def lib() -> C.CDLL:
         L.bs_op_gemm.argtypes = [vp, i, vp, vp, vp, i, i, i, i, i, vp, vp]
         L.bs_op_rmsnorm.argtypes = [vp, vp, vp, vp, i, i, f, vp]
         L.bs_op_rope_kv.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, f, i, vp, vp]
+        L.bs_op_rope_kv_static.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, f, i, vp]
         L.bs_op_attention_q_tile.argtypes = [i, i]
         L.bs_op_attention.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, vp]
         L.bs_op_confidence.argtypes = [vp, i, i, i, vp, vp, vp]
@@ -300,6 +301,17 @@ def op_rope_kv(qkv, tok_pos, tok_kv, kcache, vcache, hq, hkv, dh, theta, max_pos
                                   vcache.data_ptr(), qkv.shape[0], hq, hkv, dh, theta, max_pos, scratch.data_ptr(),
                                   _stream()), "bs_op_rope_kv")
     torch.cuda.current_stream().synchronize()
+
+
+ROPE_STATIC_MAX_FLOATS = 512 * 1024
+
+
+def op_rope_kv_static(qkv, tok_pos, tok_kv, kcache, vcache, hq, hkv, dh, theta, max_pos) -> int:
+    """bs_op_rope_kv for callers that cannot allocate: the cos/sin table lives inside the library (at most
+    ROPE_STATIC_MAX_FLOATS = max_pos * head_dim floats).  Nothing is allocated here either: the wrapper only
+    passes the caller's pointers through.  Returns the status code (BS_E_ARG when the table would not fit)."""
+    return lib().bs_op_rope_kv_static(qkv.data_ptr(), tok_pos.data_ptr(), tok_kv.data_ptr(), kcache.data_ptr(),
+                                      vcache.data_ptr(), qkv.shape[0], hq, hkv, dh, theta, max_pos, _stream())
 
 
 def op_attention(qkv, kcache, vcache, cu_q, kv_base, vis, hq, hkv, dh) -> torch.Tensor:
