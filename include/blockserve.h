@@ -191,7 +191,9 @@ int bs_debug_read(bs_engine* e, int what, int arg0, int arg1, void* host_buf, si
  * mode 0: C bf16 store;  1: C fp32 += result (residual);  2: C fp32 = row_scale[m] * result (LM head, alpha_i);
  * mode 3: C bf16 [M,N] = silu(A W^T) * (A W2^T)  (SwiGLU gate/up).  K % 8 == 0.  lda/ldc in elements. */
 int bs_op_gemm(const void* A, int lda, const void* W, const void* W2, void* C, int ldc, int M, int N, int K,
-               int mode, const float* row_scale, void* stream);
+               int mode, const float* row_scale, float* scratch /* nullable: k-split partial sums */,
+               size_t scratch_bytes, int* error_flag /* nullable device int, set when a bounded wait runs out */,
+               void* stream);
 
 /* y[m,:] = bf16(w * x[idx ? idx[m] : m, :] / sqrt(mean(x^2) + eps)); x fp32 [*, d], y bf16 [M, d]. */
 int bs_op_rmsnorm(const float* x, const int* idx, const void* w, void* y, int M, int d, float eps, void* stream);

@@ -88,7 +88,7 @@ def lib() -> C.CDLL:
         L.bs_last_error.argtypes = [vp]
         L.bs_last_error.restype = C.c_char_p
         L.bs_debug_read.argtypes = [vp, i, i, i, vp, C.c_size_t, C.POINTER(C.c_size_t)]
-        L.bs_op_gemm.argtypes = [vp, i, vp, vp, vp, i, i, i, i, i, vp, vp]
+        L.bs_op_gemm.argtypes = [vp, i, vp, vp, vp, i, i, i, i, i, vp, vp, C.c_size_t, vp, vp]
         L.bs_op_rmsnorm.argtypes = [vp, vp, vp, vp, i, i, f, vp]
         L.bs_op_rope_kv.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, f, i, vp, vp]
         L.bs_op_rope_kv_static.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, f, i, vp]
@@ -277,13 +277,16 @@ def engine_for_workload(wl, weights, *, kv_capacity_tokens: Optional[int] = None
 # ---- single operations -------------------------------------------------------------------------------------
 
 def op_gemm(A: torch.Tensor, W: torch.Tensor, mode: int = 0, W2: Optional[torch.Tensor] = None,
-            C_out: Optional[torch.Tensor] = None, row_scale: Optional[torch.Tensor] = None) -> torch.Tensor:
+            C_out: Optional[torch.Tensor] = None, row_scale: Optional[torch.Tensor] = None,
+            scratch: Optional[torch.Tensor] = None, error_flag: Optional[torch.Tensor] = None) -> torch.Tensor:
     M, K = A.shape
     N = W.shape[0]
     if C_out is None:
         C_out = torch.empty(M, N, dtype=torch.bfloat16 if mode in (0, 3) else torch.float32, device=A.device)
     _check_op(lib().bs_op_gemm(A.data_ptr(), A.stride(0), W.data_ptr(), _ptr(W2), C_out.data_ptr(), C_out.stride(0),
-                               M, N, K, mode, _ptr(row_scale), _stream()), "bs_op_gemm")
+                               M, N, K, mode, _ptr(row_scale), _ptr(scratch),
+                               0 if scratch is None else scratch.numel() * scratch.element_size(),
+                               _ptr(error_flag), _stream()), "bs_op_gemm")
     return C_out
 
 

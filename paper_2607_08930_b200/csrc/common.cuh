@@ -53,9 +53,19 @@ cudaError_t launch_attention(const bf16* qkv, const bf16* kc, const bf16* vc, bf
 cudaError_t launch_confidence(const float* logits, int n_rows, int vocab, int mask_id, int* tok, float* conf,
                               cudaStream_t s);
 
+// Scratch a GEMM launch may use: fp32 partial sums of a k split, and the word it raises when a bounded wait runs out.
+struct GemmScratch {
+  float* partial = nullptr;
+  size_t partial_floats = 0;
+  int* error_flag = nullptr;
+};
+
 // C[M,N] = A[M,K] W[N,K]^T.  mode: 0 bf16 store, 1 fp32 +=, 2 fp32 row-scaled store, 3 SwiGLU (W and W2).
 cudaError_t launch_gemm(const bf16* A, int lda, const bf16* W, const bf16* W2, void* C, int ldc, int M, int N, int K,
-                        int mode, const float* row_scale, cudaStream_t s);
+                        int mode, const float* row_scale, const GemmScratch& scratch, cudaStream_t s);
+cudaError_t launch_gemm_tc(const bf16* A, int lda, const bf16* W, const bf16* W2, void* C, int ldc, int M, int N,
+                           int K, int mode, const float* row_scale, const GemmScratch& scratch, cudaStream_t s,
+                           bool* handled);
 
 cudaError_t launch_gemm_mma(const bf16* A, int lda, const bf16* W, const bf16* W2, void* C, int ldc, int M, int N,
                             int K, int mode, const float* row_scale, cudaStream_t s);

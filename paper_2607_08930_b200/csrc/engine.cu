@@ -41,7 +41,10 @@ struct Workspace {
   bf16* act;        // [min(T, chunk), ffn]
   bf16* hf;         // [max_batch L, d]
   float* logits;    // [max_batch L, V]
+  float* partial;   // k-split partial sums of the projection GEMMs
 };
+
+constexpr size_t kPartialFloats = 16u << 20;
 
 size_t carve_workspace(const bs_config& c, void* base, Workspace* w) {
   Carver cv(base);
@@ -55,6 +58,7 @@ size_t carve_workspace(const bs_config& c, void* base, Workspace* w) {
   t.act = cv.take<bf16>(std::min<size_t>(T, kMlpChunk) * c.d_ffn);
   t.hf = cv.take<bf16>(mm * c.d_model);
   t.logits = cv.take<float>(mm * c.vocab);
+  t.partial = cv.take<float>(kPartialFloats);
   if (w) *w = t;
   return cv.off;
 }
@@ -126,6 +130,7 @@ struct bs_engine {
   int uploaded_slots = 0;
   bs_stats stats;
   std::string err;
+  GemmScratch gemm_scratch;
   // per-family device timing
   bool profiling = false;
   std::vector<cudaEvent_t> ev_pool;
@@ -218,13 +223,10 @@ int post_header(bs_engine* e) {
 }  // namespace
 
 namespace bs {
-cudaError_t launch_gemm_tc(const bf16* A, int lda, const bf16* W, const bf16* W2, void* C, int ldc, int M, int N,
-                           int K, int mode, const float* row_scale, cudaStream_t s, bool* handled);
-
 cudaError_t launch_gemm(const bf16* A, int lda, const bf16* W, const bf16* W2, void* C, int ldc, int M, int N, int K,
-                        int mode, const float* row_scale, cudaStream_t s) {
+                        int mode, const float* row_scale, const GemmScratch& scratch, cudaStream_t s) {
   bool handled = false;
-  cudaError_t r = launch_gemm_tc(A, lda, W, W2, C, ldc, M, N, K, mode, row_scale, s, &handled);
+  cudaError_t r = launch_gemm_tc(A, lda, W, W2, C, ldc, M, N, K, mode, row_scale, scratch, s, &handled);
   if (handled) return r;
   return launch_gemm_mma(A, lda, W, W2, C, ldc, M, N, K, mode, row_scale, s);
 }
@@ -267,6 +269,9 @@ int bs_init_model(const bs_config* cfg, const bs_weights* w, void* kv, void* wor
   st.max_row_tokens = cfg->max_row_tokens; st.suffix_mode = cfg->suffix_mode; st.mask_id = cfg->mask_id;
   st.vocab = cfg->vocab; st.beta = cfg->token_budget; st.kv_capacity = cfg->kv_capacity_tokens; st.tau = cfg->tau;
   st.q_tile = attention_q_tile(cfg->n_q_heads, cfg->n_kv_heads);
+  e->gemm_scratch.partial = e->ws.partial;
+  e->gemm_scratch.partial_floats = kPartialFloats;
+  e->gemm_scratch.error_flag = st.hdr + H_ERROR;
   e->embed = static_cast<const bf16*>(w->embed);
   e->lm_head = static_cast<const bf16*>(w->lm_head);
   e->final_norm = static_cast<const bf16*>(w->final_norm);
@@ -399,7 +404,7 @@ int bs_denoise_step(bs_engine* e, int* n_committed) {
     KL(e, launch_rmsnorm(ws.x, nullptr, e->norm1[l], ws.h, M, d, c.rms_eps, s));
     prof_work(e, BS_FAM_EMBED_NORM, 1, 0, 6.0 * dM * dd);
     prof_mark(e, BS_FAM_GEMM_QKV);
-    KL(e, launch_gemm(ws.h, d, e->wqkv[l], nullptr, ws.qkv, qkv_n, M, qkv_n, d, 0, nullptr, s));
+    KL(e, launch_gemm(ws.h, d, e->wqkv[l], nullptr, ws.qkv, qkv_n, M, qkv_n, d, 0, nullptr, e->gemm_scratch, s));
     prof_work(e, BS_FAM_GEMM_QKV, 1, 2.0 * dM * dq * dd, 2.0 * (dq * dd + dM * dd + dM * dq));
     prof_mark(e, BS_FAM_ROPE_KV);
     KL(e, launch_rope_kv(ws.qkv, st.tok_pos, st.tok_kv, kc, vc, M, hq, hkv, dh, ws.rope, s));
@@ -411,7 +416,7 @@ int bs_denoise_step(bs_engine* e, int* n_committed) {
     // the host knows the sums only for pure block steps and pure refresh steps, else it reports bytes alone
     prof_work(e, BS_FAM_ATTENTION, 1, 0, 2.0 * (2.0 * kv_rows * hkv * dh + 2.0 * dM * dhq));
     prof_mark(e, BS_FAM_GEMM_O);
-    KL(e, launch_gemm(ws.attn, hq * dh, e->wo[l], nullptr, ws.x, d, M, d, hq * dh, 1, nullptr, s));
+    KL(e, launch_gemm(ws.attn, hq * dh, e->wo[l], nullptr, ws.x, d, M, d, hq * dh, 1, nullptr, e->gemm_scratch, s));
     prof_work(e, BS_FAM_GEMM_O, 1, 2.0 * dM * dd * dhq, 2.0 * (dd * dhq + dM * dhq) + 8.0 * dM * dd);
     for (long long c0 = 0; c0 < M; c0 += kMlpChunk) {
       const int mc = (int)std::min<long long>(kMlpChunk, M - c0);
@@ -421,10 +426,10 @@ int bs_denoise_step(bs_engine* e, int* n_committed) {
       KL(e, launch_rmsnorm(xc, nullptr, e->norm2[l], ws.h, mc, d, c.rms_eps, s));
       prof_work(e, BS_FAM_EMBED_NORM, 1, 0, 6.0 * dmc * dd);
       prof_mark(e, BS_FAM_GEMM_GATE_UP);
-      KL(e, launch_gemm(ws.h, d, e->w_gate[l], e->w_up[l], ws.act, c.d_ffn, mc, c.d_ffn, d, 3, nullptr, s));
+      KL(e, launch_gemm(ws.h, d, e->w_gate[l], e->w_up[l], ws.act, c.d_ffn, mc, c.d_ffn, d, 3, nullptr, e->gemm_scratch, s));
       prof_work(e, BS_FAM_GEMM_GATE_UP, 1, 4.0 * dmc * df * dd, 2.0 * (2.0 * df * dd + dmc * dd + dmc * df));
       prof_mark(e, BS_FAM_GEMM_DOWN);
-      KL(e, launch_gemm(ws.act, c.d_ffn, e->w_down[l], nullptr, xc, d, mc, d, c.d_ffn, 1, nullptr, s));
+      KL(e, launch_gemm(ws.act, c.d_ffn, e->w_down[l], nullptr, xc, d, mc, d, c.d_ffn, 1, nullptr, e->gemm_scratch, s));
       prof_work(e, BS_FAM_GEMM_DOWN, 1, 2.0 * dmc * dd * df, 2.0 * (dd * df + dmc * df) + 8.0 * dmc * dd);
     }
   }
@@ -434,7 +439,7 @@ int bs_denoise_step(bs_engine* e, int* n_committed) {
   KL(e, launch_rmsnorm(ws.x, st.lm_tok[parity], e->final_norm, ws.hf, Mm, d, c.rms_eps, s));
   prof_work(e, BS_FAM_EMBED_NORM, 1, 0, 6.0 * dMm * dd);
   prof_mark(e, BS_FAM_GEMM_LM_HEAD);
-  KL(e, launch_gemm(ws.hf, d, e->lm_head, nullptr, ws.logits, c.vocab, Mm, c.vocab, d, 2, st.lm_scale[parity], s));
+  KL(e, launch_gemm(ws.hf, d, e->lm_head, nullptr, ws.logits, c.vocab, Mm, c.vocab, d, 2, st.lm_scale[parity], e->gemm_scratch, s));
   prof_work(e, BS_FAM_GEMM_LM_HEAD, 1, 2.0 * dMm * dV * dd, 2.0 * (dV * dd + dMm * dd) + 4.0 * dMm * dV);
   prof_mark(e, BS_FAM_CONFIDENCE);
   KL(e, launch_confidence(ws.logits, Mm, c.vocab, c.mask_id, st.out_tok[parity], st.out_conf[parity], s));
@@ -595,14 +600,18 @@ int bs_debug_read(bs_engine* e, int what, int arg0, int arg1, void* host_buf, si
 // ---- single operations ----------------------------------------------------------------------------------
 
 int bs_op_gemm(const void* A, int lda, const void* W, const void* W2, void* C, int ldc, int M, int N, int K, int mode,
-               const float* row_scale, void* stream) {
+               const float* row_scale, float* scratch, size_t scratch_bytes, int* error_flag, void* stream) {
   if (M == 0) return BS_OK;
   if (!A || !W || !C || M < 0 || N < 1 || K < 8 || K % 8 || N % 2 || mode < 0 || mode > 3) return BS_E_ARG;
   if (mode == 3 && !W2) return BS_E_ARG;
   if (mode == 2 && !row_scale) return BS_E_ARG;
   if (lda % 8 || (((uintptr_t)A | (uintptr_t)W | (uintptr_t)W2) & 15)) return BS_E_ARG;
+  GemmScratch sc;
+  sc.partial = scratch;
+  sc.partial_floats = scratch ? scratch_bytes / sizeof(float) : 0;
+  sc.error_flag = error_flag;
   cudaError_t r = launch_gemm((const bf16*)A, lda, (const bf16*)W, (const bf16*)W2, C, ldc, M, N, K, mode, row_scale,
-                              (cudaStream_t)stream);
+                              sc, (cudaStream_t)stream);
   return r == cudaSuccess ? BS_OK : BS_E_CUDA;
 }
 

@@ -1,9 +1,458 @@
-// tcgen05 / TMEM GEMM fed by TMA (placeholder until the kernel lands: declines every shape).
+// Projection GEMM on the 5th-generation tensor cores: C[M,N] = A[M,K] W[N,K]^T, bf16 operands, fp32 accumulate.
+//
+// Orientation: the weight rows sit on the 128-row side of the UMMA tile and the packed tokens on its N side
+// (N = 32 .. 256), so that a block step with a few dozen tokens wastes no tensor-core rows and every CTA streams a
+// disjoint slab of the weights.  One persistent CTA per SM, warp-specialised:
+//   warp 0      TMA producer   (cp.async.bulk.tensor.2d, 128B-swizzled K-major tiles of 64 bf16, mbarrier tx counts)
+//   warp 1      MMA issuer     (tcgen05.mma cta_group::1 kind::f16, accumulators in TMEM, tcgen05.commit)
+//   warps 2..5  epilogue       (tcgen05.ld -> registers -> fused epilogue -> global), double-buffered against the
+//                              next tile's main loop through two TMEM accumulator buffers
+// Work items are (n tile, token tile, k split); split partial sums go to an fp32 scratch buffer and a small
+// kernel adds them in a fixed order and applies the epilogue (deterministic, no atomics).
+// Every wait is bounded: when one runs out the kernel raises a flag, all roles drain, TMEM is freed and the
+// host reports BS_E_TIMEOUT.
+#include <cuda.h>
+#include <cudaTypedefs.h>
+
+#include <mutex>
+#include <unordered_map>
+
 #include "common.cuh"
+
 namespace bs {
-cudaError_t launch_gemm_tc(const bf16*, int, const bf16*, const bf16*, void*, int, int, int, int, int, const float*,
-                           cudaStream_t, bool* handled) {
-  *handled = false;
-  return cudaSuccess;
+
+namespace {
+
+constexpr int BK = 64;                 // K elements per pipeline stage (128 bytes: one swizzle span)
+constexpr int TILE_N = 128;            // weight rows per tile (UMMA M)
+constexpr int kThreads = 192;
+constexpr int kSmemBudget = 200 * 1024;
+constexpr long long kWaitCycles = 4000000000ll;   // ~2 s at 2 GHz: no legitimate wait comes near it
+
+struct GemmParams {
+  int M, N, K;
+  int tn;            // tokens per tile (UMMA N)
+  int n_tiles, m_tiles, splits, kblocks;
+  int stages;
+  int mode;          // 0 bf16 store, 1 fp32 +=, 2 fp32 row-scaled store, 3 SwiGLU
+  int dual;
+  void* C;
+  int ldc;
+  const float* row_scale;
+  float* partial;    // [splits][M][N] fp32 when splits > 1
+  int* error_flag;
+};
+
+__device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(unsigned bar, unsigned count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
 }
+__device__ __forceinline__ void mbar_expect_tx(unsigned bar, unsigned bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(unsigned bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity) {
+  unsigned ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait: returns false (and raises the abort flag) if the phase does not complete in time or if
+// another role has already given up.
+__device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity, volatile int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity)) {
+    if (*abort_flag) return false;
+    if (clock64() - t0 > kWaitCycles) {
+      *abort_flag = 1;
+      return false;
+    }
+  }
+  return true;
+}
+
+__device__ __forceinline__ void tma_load_2d(unsigned dst, const CUtensorMap* map, int c0, int c1, unsigned bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
+}
+
+// K-major operand tile, rows of 128 bytes, 128B swizzle: 8-row groups are 1024 bytes apart.
+__device__ __forceinline__ unsigned long long umma_desc(unsigned smem_addr) {
+  unsigned long long d = 0;
+  d |= (unsigned long long)((smem_addr & 0x3FFFF) >> 4);        // start address
+  d |= (unsigned long long)1 << 16;                              // leading byte offset (unused for swizzled K-major)
+  d |= (unsigned long long)(1024 >> 4) << 32;                    // stride byte offset
+  d |= (unsigned long long)1 << 46;                              // descriptor version (sm_100)
+  d |= (unsigned long long)2 << 61;                              // layout: 128-byte swizzle
+  return d;
+}
+// kind::f16 instruction descriptor: fp32 accumulator, bf16 x bf16, both K-major, shape 128 x n x 16.
+__device__ __forceinline__ unsigned umma_idesc(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((unsigned)(n >> 3) << 17) | ((unsigned)(TILE_N >> 4) << 24);
+}
+__device__ __forceinline__ void umma_bf16(unsigned d_tmem, unsigned long long a, unsigned long long b, unsigned idesc,
+                                          unsigned accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(unsigned bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(unsigned taddr, float* v) {
+  unsigned r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ float silu_f(float x) { return x / (1.0f + __expf(-x)); }
+
+__global__ void __launch_bounds__(kThreads, 1)
+k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_w2,
+          const __grid_constant__ CUtensorMap map_x, const GemmParams p) {
+  extern __shared__ unsigned char smem_dyn[];
+  __shared__ __align__(8) unsigned long long bars[2 * 16 + 4];     // full[16], empty[16], tmem_full[2], tmem_empty[2]
+  __shared__ unsigned tmem_base_slot;
+  __shared__ int s_abort;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const unsigned smem0 = (smem_u32(smem_dyn) + 1023u) & ~1023u;     // 1024-byte alignment for the swizzle atoms
+  const int w_bytes = TILE_N * BK * 2;
+  const int x_bytes = p.tn * BK * 2;
+  const int stage_bytes = (p.dual ? 2 : 1) * w_bytes + x_bytes;
+  const unsigned full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[16]);
+  const unsigned tfull0 = smem_u32(&bars[32]), tempty0 = smem_u32(&bars[34]);
+
+  if (threadIdx.x == 0) {
+    s_abort = 0;
+    for (int i = 0; i < p.stages; ++i) {
+      mbar_init(full0 + 8 * i, 1);
+      mbar_init(empty0 + 8 * i, 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(tfull0 + 8 * i, 1);
+      mbar_init(tempty0 + 8 * i, 4);       // one arrival per epilogue warp
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {                          // TMEM: the whole 512 columns (one CTA per SM)
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&tmem_base_slot))
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const unsigned tmem_base = tmem_base_slot;
+  volatile int* abort_flag = &s_abort;
+
+  const int items = p.n_tiles * p.m_tiles * p.splits;
+  const int acc_cols = 256;                 // columns per accumulator buffer (dual: gate at +0, up at +128)
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int stage = 0;
+      unsigned phase = 0;
+      bool ok = true;
+      for (int it = blockIdx.x; it < items && ok; it += gridDim.x) {
+        const int split = it % p.splits;
+        const int tile = it / p.splits;
+        const int mt = tile % p.m_tiles, nt = tile / p.m_tiles;
+        const int kb0 = (int)((long long)p.kblocks * split / p.splits);
+        const int kb1 = (int)((long long)p.kblocks * (split + 1) / p.splits);
+        for (int kb = kb0; kb < kb1; ++kb) {
+          if (!mbar_wait(empty0 + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+          const unsigned sw = smem0 + stage * stage_bytes;
+          mbar_expect_tx(full0 + 8 * stage, (unsigned)stage_bytes);
+          tma_load_2d(sw, &map_w, kb * BK, nt * TILE_N, full0 + 8 * stage);
+          if (p.dual) tma_load_2d(sw + w_bytes, &map_w2, kb * BK, nt * TILE_N, full0 + 8 * stage);
+          tma_load_2d(sw + (p.dual ? 2 : 1) * w_bytes, &map_x, kb * BK, mt * p.tn, full0 + 8 * stage);
+          if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      int stage = 0;
+      unsigned phase = 0;
+      int local = 0;
+      const unsigned idesc = umma_idesc(p.tn);
+      bool ok = true;
+      for (int it = blockIdx.x; it < items && ok; it += gridDim.x, ++local) {
+        const int split = it % p.splits;
+        const int kb0 = (int)((long long)p.kblocks * split / p.splits);
+        const int kb1 = (int)((long long)p.kblocks * (split + 1) / p.splits);
+        const int acc = local & 1;
+        const unsigned acc_phase = (unsigned)(local >> 1) & 1u;
+        if (!mbar_wait(tempty0 + 8 * acc, acc_phase ^ 1u, abort_flag)) break;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const unsigned d_gate = tmem_base + acc * acc_cols;
+        const unsigned d_up = d_gate + 128;
+        for (int kb = kb0; kb < kb1; ++kb) {
+          if (!mbar_wait(full0 + 8 * stage, phase, abort_flag)) { ok = false; break; }
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const unsigned sw = smem0 + stage * stage_bytes;
+          const unsigned long long dw = umma_desc(sw);
+          const unsigned long long dx = umma_desc(sw + (p.dual ? 2 : 1) * w_bytes);
+#pragma unroll
+          for (int k = 0; k < BK / 16; ++k) {
+            const unsigned accum = (kb > kb0 || k > 0) ? 1u : 0u;
+            umma_bf16(d_gate, dw + 2 * k, dx + 2 * k, idesc, accum);     // +32 bytes per 16-element K step
+            if (p.dual) umma_bf16(d_up, umma_desc(sw + w_bytes) + 2 * k, dx + 2 * k, idesc, accum);
+          }
+          umma_commit(empty0 + 8 * stage);        // the stage is free once these MMAs have read it
+          if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+        }
+        if (ok) umma_commit(tfull0 + 8 * acc);    // accumulator complete
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue warps
+    const int q = warp & 3;                       // TMEM lane quarter this warp may read
+    int local = 0;
+    for (int it = blockIdx.x; it < items; it += gridDim.x, ++local) {
+      const int split = it % p.splits;
+      const int tile = it / p.splits;
+      const int mt = tile % p.m_tiles, nt = tile / p.m_tiles;
+      const int acc = local & 1;
+      const unsigned acc_phase = (unsigned)(local >> 1) & 1u;
+      if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag)) break;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const int n = nt * TILE_N + q * 32 + lane;
+      const bool n_ok = n < p.N;
+      const unsigned t_row = tmem_base + ((unsigned)(q * 32) << 16) + acc * acc_cols;
+      for (int c0 = 0; c0 < p.tn; c0 += 32) {
+        const int t0 = mt * p.tn + c0;
+        if (t0 >= p.M) break;                     // warp-uniform
+        float v[32];
+        tmem_ld32(t_row + c0, v);
+        if (p.splits > 1) {
+          float* dst = p.partial + ((size_t)split * p.M) * p.N;
+          if (p.dual) {
+            float u[32];
+            tmem_ld32(t_row + 128 + c0, u);
+            float* dst2 = dst + (size_t)p.splits * p.M * p.N;
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (n_ok && t0 + j < p.M) {
+                dst[(size_t)(t0 + j) * p.N + n] = v[j];
+                dst2[(size_t)(t0 + j) * p.N + n] = u[j];
+              }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (n_ok && t0 + j < p.M) dst[(size_t)(t0 + j) * p.N + n] = v[j];
+          }
+        } else if (p.mode == 0) {
+          bf16* C = reinterpret_cast<bf16*>(p.C);
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (n_ok && t0 + j < p.M) C[(size_t)(t0 + j) * p.ldc + n] = __float2bfloat16_rn(v[j]);
+        } else if (p.mode == 1) {
+          // all loads first, then the stores: interleaving them would serialise on the load latency
+          float* C = reinterpret_cast<float*>(p.C) + (size_t)t0 * p.ldc + n;
+          float c[32];
+#pragma unroll
+          for (int j = 0; j < 32; ++j) c[j] = (n_ok && t0 + j < p.M) ? C[(size_t)j * p.ldc] : 0.f;
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (n_ok && t0 + j < p.M) C[(size_t)j * p.ldc] = c[j] + v[j];
+        } else if (p.mode == 2) {
+          float* C = reinterpret_cast<float*>(p.C);
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (n_ok && t0 + j < p.M) C[(size_t)(t0 + j) * p.ldc + n] = v[j] * __ldg(p.row_scale + t0 + j);
+        } else {
+          float u[32];
+          tmem_ld32(t_row + 128 + c0, u);
+          bf16* C = reinterpret_cast<bf16*>(p.C);
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (n_ok && t0 + j < p.M) C[(size_t)(t0 + j) * p.ldc + n] = __float2bfloat16_rn(silu_f(v[j]) * u[j]);
+        }
+      }
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty0 + 8 * acc);
+    }
+  }
+
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (s_abort && threadIdx.x == 0 && p.error_flag) atomicExch(p.error_flag, 1);
+  if (warp == 1) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
+  }
+}
+
+// Adds the k-split partial sums in split order and applies the epilogue.
+__global__ void k_gemm_finish(const float* __restrict__ partial, int splits, int M, int N, int mode, void* Cv, int ldc,
+                              const float* __restrict__ row_scale) {
+  const size_t total = (size_t)M * N;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+    const int t = (int)(i / N), n = (int)(i % N);
+    float g = 0.f;
+    for (int s = 0; s < splits; ++s) g += partial[(size_t)s * total + i];
+    if (mode == 0) {
+      reinterpret_cast<bf16*>(Cv)[(size_t)t * ldc + n] = __float2bfloat16_rn(g);
+    } else if (mode == 1) {
+      reinterpret_cast<float*>(Cv)[(size_t)t * ldc + n] += g;
+    } else if (mode == 2) {
+      reinterpret_cast<float*>(Cv)[(size_t)t * ldc + n] = g * row_scale[t];
+    } else {
+      float u = 0.f;
+      for (int s = 0; s < splits; ++s) u += partial[(size_t)(splits + s) * total + i];
+      reinterpret_cast<bf16*>(Cv)[(size_t)t * ldc + n] = __float2bfloat16_rn(silu_f(g) * u);
+    }
+  }
+}
+
+// ---- host side ---------------------------------------------------------------------------------------------
+
+PFN_cuTensorMapEncodeTiled_v12000 g_encode = nullptr;
+std::mutex g_mutex;
+
+struct MapKey {
+  const void* ptr; long long rows, cols, ld; int box_rows;
+  bool operator==(const MapKey& o) const {
+    return ptr == o.ptr && rows == o.rows && cols == o.cols && ld == o.ld && box_rows == o.box_rows;
+  }
+};
+struct MapHash {
+  size_t operator()(const MapKey& k) const {
+    size_t h = std::hash<const void*>()(k.ptr);
+    h = h * 1000003u ^ std::hash<long long>()(k.rows * 131 + k.cols);
+    h = h * 1000003u ^ std::hash<long long>()(k.ld * 257 + k.box_rows);
+    return h;
+  }
+};
+std::unordered_map<MapKey, CUtensorMap, MapHash> g_maps;
+
+bool get_map(const bf16* ptr, long long rows, long long cols, long long ld, int box_rows, CUtensorMap* out) {
+  std::lock_guard<std::mutex> lock(g_mutex);
+  if (!g_encode) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn)
+      return false;
+    g_encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
+  }
+  const MapKey key{ptr, rows, cols, ld, box_rows};
+  auto it = g_maps.find(key);
+  if (it != g_maps.end()) { *out = it->second; return true; }
+  if (g_maps.size() > 8192) g_maps.clear();
+  CUtensorMap m;
+  const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)ld * sizeof(bf16)};
+  const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = g_encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<bf16*>(ptr), dims, strides, box, estr,
+                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return false;
+  g_maps.emplace(key, m);
+  *out = m;
+  return true;
+}
+
+int g_num_sms = 0;
+
+}  // namespace
+
+cudaError_t launch_gemm_tc(const bf16* A, int lda, const bf16* W, const bf16* W2, void* C, int ldc, int M, int N,
+                           int K, int mode, const float* row_scale, const GemmScratch& scratch, cudaStream_t s,
+                           bool* handled) {
+  float* const g_partial = scratch.partial;
+  const size_t g_partial_floats = scratch.partial_floats;
+  int* const g_error_flag = scratch.error_flag;
+  *handled = false;
+  if (M <= 0 || N <= 0) return cudaSuccess;
+  if (K % 8 || lda % 8 || ((uintptr_t)A & 15) || ((uintptr_t)W & 15) || (W2 && ((uintptr_t)W2 & 15)))
+    return cudaSuccess;                       // TMA needs 16-byte aligned rows: leave it to the legacy kernel
+  if (!g_num_sms) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev);
+    if (cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 1024) !=
+        cudaSuccess)
+      return cudaSuccess;
+  }
+  const int dual = mode == 3;
+  GemmParams p;
+  p.M = M; p.N = N; p.K = K; p.mode = mode; p.dual = dual; p.C = C; p.ldc = ldc; p.row_scale = row_scale;
+  p.kblocks = (K + BK - 1) / BK;
+  p.n_tiles = (N + TILE_N - 1) / TILE_N;
+  p.error_flag = g_error_flag;
+  // ---- tile shape and k split: fill the SMs, keep tensor-core tiles wide when there is work for them ----
+  const int tn_max = dual ? 128 : 256;
+  int best_tn = 32, best_s = 1;
+  double best_t = 1e30;
+  for (int tn = 32; tn <= tn_max; tn *= 2) {
+    const int m_tiles = (M + tn - 1) / tn;
+    for (int sp = 1; sp <= 8; ++sp) {
+      if (sp > 1 && (p.kblocks / sp < 4)) break;
+      if (sp > 1 && (!g_partial || (size_t)sp * (dual ? 2 : 1) * (size_t)M * N > g_partial_floats)) break;
+      const long long items = (long long)p.n_tiles * m_tiles * sp;
+      const double waves = (double)((items + g_num_sms - 1) / g_num_sms);
+      const double kslice = (double)K / sp;
+      const double mma_eff = tn >= 128 ? 1.0 : (tn == 64 ? 0.67 : 0.4);
+      const double t_mma = (dual ? 2.0 : 1.0) * TILE_N * tn * kslice / (4096.0 * mma_eff);          // clocks
+      const double t_mem = ((dual ? 2.0 : 1.0) * TILE_N + tn * 0.25) * kslice * 2.0 / 24.0;         // clocks
+      const double t_epi = 400.0 + tn * 6.0;
+      double t = waves * ((t_mma > t_mem ? t_mma : t_mem) + t_epi + 1500.0);
+      if (sp > 1) t += 2.0 * sp * (dual ? 2 : 1) * (double)M * N * 4.0 / (24.0 * g_num_sms) + 4000.0;
+      if (t < best_t) { best_t = t; best_tn = tn; best_s = sp; }
+    }
+  }
+  p.tn = best_tn;
+  p.splits = best_s;
+  p.m_tiles = (M + p.tn - 1) / p.tn;
+  p.partial = g_partial;
+  const int stage_bytes = (dual ? 2 : 1) * TILE_N * BK * 2 + p.tn * BK * 2;
+  p.stages = kSmemBudget / stage_bytes;
+  if (p.stages > 16) p.stages = 16;
+  if (p.stages < 2) return cudaSuccess;
+
+  CUtensorMap mw, mw2, mx;
+  if (!get_map(W, N, K, K, TILE_N, &mw)) return cudaSuccess;
+  if (dual) { if (!get_map(W2, N, K, K, TILE_N, &mw2)) return cudaSuccess; } else { mw2 = mw; }
+  if (!get_map(A, M, K, lda, p.tn, &mx)) return cudaSuccess;
+
+  *handled = true;
+  const long long items = (long long)p.n_tiles * p.m_tiles * p.splits;
+  const int grid = (int)(items < g_num_sms ? items : g_num_sms);
+  k_gemm_tc<<<grid, kThreads, kSmemBudget + 1024, s>>>(mw, mw2, mx, p);
+  cudaError_t r = cudaGetLastError();
+  if (r != cudaSuccess) return r;
+  if (p.splits > 1) {
+    const size_t total = (size_t)M * N;
+    const int blocks = (int)((total + 255) / 256 < (size_t)g_num_sms * 8 ? (total + 255) / 256 : (size_t)g_num_sms * 8);
+    k_gemm_finish<<<blocks, 256, 0, s>>>(g_partial, p.splits, M, N, mode, C, ldc, row_scale);
+    r = cudaGetLastError();
+  }
+  return r;
+}
+
 }  // namespace bs

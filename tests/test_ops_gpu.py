@@ -63,6 +63,41 @@ def test_gemm_modes(B, M, N, K, mode):
     assert np.abs(got - ref).max() <= tol * (np.abs(ref) + np.abs(ref).max() * 0.05).max()
 
 
+@pytest.mark.parametrize("M,N,K,mode", [(32, 512, 4096, 0), (64, 384, 2048, 1), (100, 256, 8192, 3), (96, 640, 1024, 2),
+                                          (256, 1152, 3584, 1), (40, 3584, 18944, 1)])
+def test_gemm_k_split(B, M, N, K, mode):
+    """Few output tiles and a long K: the launch splits K across CTAs and sums the partials in a fixed order."""
+    rng = np.random.default_rng(M + N + K)
+    A = bf16_round(rng.normal(size=(M, K)))
+    W = bf16_round(rng.normal(size=(N, K)) * 0.05)
+    W2 = bf16_round(rng.normal(size=(N, K)) * 0.05)
+    a, w, w2 = A.double().numpy(), W.double().numpy(), W2.double().numpy()
+    scratch = torch.empty(16 << 20, dtype=torch.float32, device="cuda")
+    flag = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ref = a @ w.T
+    kw = dict(scratch=scratch, error_flag=flag)
+    if mode == 0:
+        got, tol = B.op_gemm(A.cuda(), W.cuda(), 0, **kw).float().cpu().numpy(), 6e-3
+    elif mode == 1:
+        c0 = rng.normal(size=(M, N)).astype(F32)
+        Cd = torch.from_numpy(c0).cuda()
+        B.op_gemm(A.cuda(), W.cuda(), 1, C_out=Cd, **kw)
+        got, ref, tol = Cd.cpu().numpy(), ref + c0, 1e-4
+    elif mode == 2:
+        sc = rng.uniform(0.5, 30.0, size=M).astype(F32)
+        got = B.op_gemm(A.cuda(), W.cuda(), 2, row_scale=torch.from_numpy(sc).cuda(), **kw).cpu().numpy()
+        ref, tol = ref * sc[:, None], 1e-4
+    else:
+        ref = O.silu(ref.astype(F32)).astype(np.float64) * (a @ w2.T)
+        got, tol = B.op_gemm(A.cuda(), W.cuda(), 3, W2=W2.cuda(), **kw).float().cpu().numpy(), 8e-3
+    assert int(flag.item()) == 0
+    assert rel_err(got, ref) < tol
+    # twice the same launch gives the same bits (fixed summation order)
+    if mode == 0:
+        again = B.op_gemm(A.cuda(), W.cuda(), 0, **kw).float().cpu().numpy()
+        assert (again == got).all()
+
+
 def test_gemm_strided_rows_and_empty(B):
     rng = np.random.default_rng(5)
     big = bf16_round(rng.normal(size=(70, 512))).cuda()
