@@ -65,7 +65,18 @@ cudaError_t launch_gemm(const bf16* A, int lda, const bf16* W, const bf16* W2, v
                         int mode, const float* row_scale, const GemmScratch& scratch, cudaStream_t s);
 cudaError_t launch_gemm_tc(const bf16* A, int lda, const bf16* W, const bf16* W2, void* C, int ldc, int M, int N,
                            int K, int mode, const float* row_scale, const GemmScratch& scratch, cudaStream_t s,
-                           bool* handled);
+                           bool* handled, int* splits_out);
+// mode 4: only the k-split partial sums [splits][M][N] are written to scratch.partial; a fused finishing kernel
+// (below) adds them in split order and applies what follows the projection.
+cudaError_t launch_gemm_partial(const bf16* A, int lda, const bf16* W, int M, int N, int K, const GemmScratch& scratch,
+                                cudaStream_t s, int* splits_out);
+// q/k/v = bf16(sum of partials); RoPE on q, k at the token's position id; q -> qkv buffer, k / v -> cache rows.
+cudaError_t launch_finish_qkv_rope(const float* partial, int splits, int M, bf16* qkv, const int* tok_pos,
+                                   const int* tok_kv, bf16* kc, bf16* vc, int hq, int hkv, int dh,
+                                   const float* cos_sin, cudaStream_t s);
+// x += sum of partials; if w: h = bf16(RMSNorm(x) * w).
+cudaError_t launch_finish_residual_norm(const float* partial, int splits, int M, int d, float* x, const bf16* w,
+                                        bf16* h, float eps, cudaStream_t s);
 
 cudaError_t launch_gemm_mma(const bf16* A, int lda, const bf16* W, const bf16* W2, void* C, int ldc, int M, int N,
                             int K, int mode, const float* row_scale, cudaStream_t s);

@@ -178,6 +178,123 @@ __global__ void __launch_bounds__(kConfThreads) k_confidence(const float* __rest
   }
 }
 
+// Finishing kernel of the QKV projection on block steps: adds the k-split partial sums in split order, rounds q / k / v
+// to bf16, rotates q and k at the token's position id and scatters k, v to the token's cache row.
+__global__ void __launch_bounds__(256) k_finish_qkv_rope(const float* __restrict__ partial, int splits, int M,
+                                                         bf16* __restrict__ qkv, const int* __restrict__ tok_pos,
+                                                         const int* __restrict__ tok_kv, bf16* __restrict__ kc,
+                                                         bf16* __restrict__ vc, int hq, int hkv, int dh,
+                                                         const float2* __restrict__ cos_sin) {
+  const int t = blockIdx.x;
+  const int N = (hq + 2 * hkv) * dh, half = dh / 2;
+  const size_t slice = (size_t)M * N;
+  const float* row = partial + (size_t)t * N;
+  const int pos = tok_pos[t];
+  const size_t kvrow = (size_t)tok_kv[t];
+  const float2* cs = cos_sin + (size_t)pos * half;
+  bf16* qrow = qkv + (size_t)t * N;
+  const int pairs_per_head = half / 2;
+  const int n_rot = (hq + hkv) * pairs_per_head;
+  for (int u = threadIdx.x; u < n_rot; u += 256) {
+    const int h = u / pairs_per_head, j = (u % pairs_per_head) * 2;
+    float2 a = make_float2(0.f, 0.f), b = make_float2(0.f, 0.f);
+    for (int s = 0; s < splits; ++s) {
+      const float2 pa = *reinterpret_cast<const float2*>(row + s * slice + h * dh + j);
+      const float2 pb = *reinterpret_cast<const float2*>(row + s * slice + h * dh + half + j);
+      a.x += pa.x; a.y += pa.y; b.x += pb.x; b.y += pb.y;
+    }
+    a = __bfloat1622float2(__floats2bfloat162_rn(a.x, a.y));     // the projection's output is a bf16 tensor
+    b = __bfloat1622float2(__floats2bfloat162_rn(b.x, b.y));
+    const float2 c0 = cs[j], c1 = cs[j + 1];
+    const __nv_bfloat162 o1 = __floats2bfloat162_rn(a.x * c0.x - b.x * c0.y, a.y * c1.x - b.y * c1.y);
+    const __nv_bfloat162 o2 = __floats2bfloat162_rn(b.x * c0.x + a.x * c0.y, b.y * c1.x + a.y * c1.y);
+    bf16* dst = h < hq ? qrow + h * dh : kc + (kvrow * hkv + (h - hq)) * dh;
+    *reinterpret_cast<__nv_bfloat162*>(dst + j) = o1;
+    *reinterpret_cast<__nv_bfloat162*>(dst + half + j) = o2;
+  }
+  const int v0 = (hq + hkv) * dh;
+  bf16* vdst = vc + kvrow * hkv * dh;
+  for (int u = threadIdx.x; u < hkv * dh / 2; u += 256) {
+    float2 a = make_float2(0.f, 0.f);
+    for (int s = 0; s < splits; ++s) {
+      const float2 pa = *reinterpret_cast<const float2*>(row + s * slice + v0 + 2 * u);
+      a.x += pa.x; a.y += pa.y;
+    }
+    *reinterpret_cast<__nv_bfloat162*>(vdst + 2 * u) = __floats2bfloat162_rn(a.x, a.y);
+  }
+}
+
+// Finishing kernel of the O and down projections on block steps: x += sum of the k-split partial sums (split order),
+// then, if a gain vector is given, the RMSNorm that feeds the next projection.
+__global__ void __launch_bounds__(256) k_finish_residual_norm(const float* __restrict__ partial, int splits, int M,
+                                                              int d, float* __restrict__ x,
+                                                              const bf16* __restrict__ w, bf16* __restrict__ h,
+                                                              float eps) {
+  __shared__ float red[8];
+  const int t = blockIdx.x;
+  const size_t slice = (size_t)M * d;
+  float4* xr = reinterpret_cast<float4*>(x + (size_t)t * d);
+  const float* prow = partial + (size_t)t * d;
+  float4 vals[8];
+  float ss = 0.f;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int c = threadIdx.x + i * 256;
+    if (c < d / 4) {
+      float4 v = xr[c];
+      for (int s = 0; s < splits; ++s) {
+        const float4 pv = *reinterpret_cast<const float4*>(prow + s * slice + 4 * c);
+        v.x += pv.x; v.y += pv.y; v.z += pv.z; v.w += pv.w;
+      }
+      xr[c] = v;
+      vals[i] = v;
+      ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+    }
+  }
+  if (w == nullptr) return;
+  ss = warp_sum(ss);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  float tot = 0.f;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) tot += red[i];
+  const float r = rsqrtf(tot / (float)d + eps);
+  const uint2* wp = reinterpret_cast<const uint2*>(w);
+  uint2* dst = reinterpret_cast<uint2*>(h + (size_t)t * d);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int c = threadIdx.x + i * 256;
+    if (c < d / 4) {
+      const float4 v = vals[i];
+      const uint2 wv = wp[c];
+      const __nv_bfloat162* wh = reinterpret_cast<const __nv_bfloat162*>(&wv);
+      const float2 w0 = __bfloat1622float2(wh[0]), w1 = __bfloat1622float2(wh[1]);
+      __nv_bfloat162 o0 = __floats2bfloat162_rn(v.x * r * w0.x, v.y * r * w0.y);
+      __nv_bfloat162 o1 = __floats2bfloat162_rn(v.z * r * w1.x, v.w * r * w1.y);
+      uint2 o;
+      o.x = *reinterpret_cast<unsigned*>(&o0);
+      o.y = *reinterpret_cast<unsigned*>(&o1);
+      dst[c] = o;
+    }
+  }
+}
+
+cudaError_t launch_finish_qkv_rope(const float* partial, int splits, int M, bf16* qkv, const int* tok_pos,
+                                   const int* tok_kv, bf16* kc, bf16* vc, int hq, int hkv, int dh,
+                                   const float* cos_sin, cudaStream_t s) {
+  if (M <= 0) return cudaSuccess;
+  k_finish_qkv_rope<<<M, 256, 0, s>>>(partial, splits, M, qkv, tok_pos, tok_kv, kc, vc, hq, hkv, dh,
+                                       reinterpret_cast<const float2*>(cos_sin));
+  return cudaGetLastError();
+}
+cudaError_t launch_finish_residual_norm(const float* partial, int splits, int M, int d, float* x, const bf16* w,
+                                        bf16* h, float eps, cudaStream_t s) {
+  if (M <= 0) return cudaSuccess;
+  if (d > 8192) return cudaErrorInvalidValue;
+  k_finish_residual_norm<<<M, 256, 0, s>>>(partial, splits, M, d, x, w, h, eps);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_embed(const DevState& st, const bf16* embed, float* x, int M, int d, cudaStream_t s) {
   if (M <= 0) return cudaSuccess;
   k_embed<<<M, 128, 0, s>>>(st, embed, x, M, d);

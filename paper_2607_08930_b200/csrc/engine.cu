@@ -45,6 +45,7 @@ struct Workspace {
 };
 
 constexpr size_t kPartialFloats = 16u << 20;
+constexpr int kSmallStepTokens = 640;     // packed tokens up to which a step takes the fused block-step path
 
 size_t carve_workspace(const bs_config& c, void* base, Workspace* w) {
   Carver cv(base);
@@ -89,7 +90,8 @@ size_t carve_state(const bs_config& c, void* base, DevState* out) {
 }
 
 const char* check_config(const bs_config& c) {
-  if (c.n_layers < 1 || c.d_model < 8 || c.d_model % 8) return "d_model must be a positive multiple of 8";
+  if (c.n_layers < 1 || c.d_model < 8 || c.d_model % 8 || c.d_model > 8192)
+    return "d_model must be a positive multiple of 8, at most 8192";
   if (c.head_dim != 64 && c.head_dim != 128) return "head_dim must be 64 or 128";
   if (c.n_kv_heads < 1 || c.n_q_heads % c.n_kv_heads) return "n_q_heads must be a multiple of n_kv_heads";
   if (c.n_q_heads / c.n_kv_heads > 8) return "at most 8 query heads per kv head";
@@ -226,9 +228,17 @@ namespace bs {
 cudaError_t launch_gemm(const bf16* A, int lda, const bf16* W, const bf16* W2, void* C, int ldc, int M, int N, int K,
                         int mode, const float* row_scale, const GemmScratch& scratch, cudaStream_t s) {
   bool handled = false;
-  cudaError_t r = launch_gemm_tc(A, lda, W, W2, C, ldc, M, N, K, mode, row_scale, scratch, s, &handled);
+  cudaError_t r = launch_gemm_tc(A, lda, W, W2, C, ldc, M, N, K, mode, row_scale, scratch, s, &handled, nullptr);
   if (handled) return r;
   return launch_gemm_mma(A, lda, W, W2, C, ldc, M, N, K, mode, row_scale, s);
+}
+
+cudaError_t launch_gemm_partial(const bf16* A, int lda, const bf16* W, int M, int N, int K, const GemmScratch& scratch,
+                                cudaStream_t s, int* splits_out) {
+  bool handled = false;
+  cudaError_t r = launch_gemm_tc(A, lda, W, nullptr, nullptr, 0, M, N, K, 4, nullptr, scratch, s, &handled, splits_out);
+  if (r != cudaSuccess) return r;
+  return handled ? cudaSuccess : cudaErrorNotSupported;
 }
 }  // namespace bs
 
@@ -397,6 +407,47 @@ int bs_denoise_step(bs_engine* e, int* n_committed) {
   prof_mark(e, BS_FAM_EMBED_NORM);
   KL(e, launch_embed(st, e->embed, ws.x, M, d, s));
   prof_work(e, BS_FAM_EMBED_NORM, 1, 0, 6.0 * dM * dd);
+  // A block step (few packed tokens) runs the projections that feed a row-wise operator as k-split partial sums
+  // and lets one finishing kernel per projection add them and apply that operator (RoPE + KV scatter after QKV,
+  // residual + the next RMSNorm after O and down).  A refresh step (many tokens) uses the direct epilogues.
+  const bool small = M <= kSmallStepTokens && (size_t)M * (size_t)std::max(qkv_n, d) <= kPartialFloats;
+  if (small) {
+    prof_mark(e, BS_FAM_EMBED_NORM);
+    KL(e, launch_rmsnorm(ws.x, nullptr, e->norm1[0], ws.h, M, d, c.rms_eps, s));
+    prof_work(e, BS_FAM_EMBED_NORM, 1, 0, 6.0 * dM * dd);
+    for (int l = 0; l < c.n_layers; ++l) {
+      bf16* kc = e->kv + (size_t)l * e->kv_layer_stride;
+      bf16* vc = kc + e->kv_half;
+      int sp = 1;
+      prof_mark(e, BS_FAM_GEMM_QKV);
+      KL(e, launch_gemm_partial(ws.h, d, e->wqkv[l], M, qkv_n, d, e->gemm_scratch, s, &sp));
+      prof_work(e, BS_FAM_GEMM_QKV, 1, 2.0 * dM * dq * dd, 2.0 * (dq * dd + dM * dd) + 4.0 * sp * dM * dq);
+      prof_mark(e, BS_FAM_ROPE_KV);
+      KL(e, launch_finish_qkv_rope(ws.partial, sp, M, ws.qkv, st.tok_pos, st.tok_kv, kc, vc, hq, hkv, dh, ws.rope, s));
+      prof_work(e, BS_FAM_ROPE_KV, 1, 0, 4.0 * sp * dM * dq + 2.0 * dM * dq);
+      prof_mark(e, BS_FAM_ATTENTION);
+      KL(e, launch_attention(ws.qkv, kc, vc, ws.attn, st.cu_q[parity], st.cu_tile[parity], st.row_kv_base,
+                             st.row_vis, n_rows, e->hdr[H_QTILES], hq, hkv, dh, s));
+      prof_work(e, BS_FAM_ATTENTION, 1, 0, 2.0 * (2.0 * kv_rows * hkv * dh + 2.0 * dM * dhq));
+      prof_mark(e, BS_FAM_GEMM_O);
+      KL(e, launch_gemm_partial(ws.attn, hq * dh, e->wo[l], M, d, hq * dh, e->gemm_scratch, s, &sp));
+      prof_work(e, BS_FAM_GEMM_O, 1, 2.0 * dM * dd * dhq, 2.0 * (dd * dhq + dM * dhq) + 4.0 * sp * dM * dd);
+      prof_mark(e, BS_FAM_EMBED_NORM);
+      KL(e, launch_finish_residual_norm(ws.partial, sp, M, d, ws.x, e->norm2[l], ws.h, c.rms_eps, s));
+      prof_work(e, BS_FAM_EMBED_NORM, 1, 0, (4.0 * sp + 10.0) * dM * dd);
+      prof_mark(e, BS_FAM_GEMM_GATE_UP);
+      KL(e, launch_gemm(ws.h, d, e->w_gate[l], e->w_up[l], ws.act, c.d_ffn, M, c.d_ffn, d, 3, nullptr,
+                        e->gemm_scratch, s));
+      prof_work(e, BS_FAM_GEMM_GATE_UP, 1, 4.0 * dM * df * dd, 2.0 * (2.0 * df * dd + dM * dd + dM * df));
+      prof_mark(e, BS_FAM_GEMM_DOWN);
+      KL(e, launch_gemm_partial(ws.act, c.d_ffn, e->w_down[l], M, d, c.d_ffn, e->gemm_scratch, s, &sp));
+      prof_work(e, BS_FAM_GEMM_DOWN, 1, 2.0 * dM * dd * df, 2.0 * (dd * df + dM * df) + 4.0 * sp * dM * dd);
+      prof_mark(e, BS_FAM_EMBED_NORM);
+      const bf16* next_norm = l + 1 < c.n_layers ? e->norm1[l + 1] : nullptr;
+      KL(e, launch_finish_residual_norm(ws.partial, sp, M, d, ws.x, next_norm, ws.h, c.rms_eps, s));
+      prof_work(e, BS_FAM_EMBED_NORM, 1, 0, (4.0 * sp + 10.0) * dM * dd);
+    }
+  } else
   for (int l = 0; l < c.n_layers; ++l) {
     bf16* kc = e->kv + (size_t)l * e->kv_layer_stride;
     bf16* vc = kc + e->kv_half;

@@ -34,7 +34,7 @@ struct GemmParams {
   int tn;            // tokens per tile (UMMA N)
   int n_tiles, m_tiles, splits, kblocks;
   int stages;
-  int mode;          // 0 bf16 store, 1 fp32 +=, 2 fp32 row-scaled store, 3 SwiGLU
+  int mode;          // 0 bf16 store, 1 fp32 +=, 2 fp32 row-scaled store, 3 SwiGLU, 4 fp32 partial sums only
   int dual;
   void* C;
   int ldc;
@@ -245,9 +245,11 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
       for (int c0 = 0; c0 < p.tn; c0 += 32) {
         const int t0 = mt * p.tn + c0;
         if (t0 >= p.M) break;                     // warp-uniform
+        // columns of this chunk that hold tokens of this tile (the tile width is a multiple of 16, not of 32)
+        const int jmax = min(min(32, p.tn - c0), p.M - t0);
         float v[32];
         tmem_ld32(t_row + c0, v);
-        if (p.splits > 1) {
+        if (p.splits > 1 || p.mode == 4) {
           float* dst = p.partial + ((size_t)split * p.M) * p.N;
           if (p.dual) {
             float u[32];
@@ -255,41 +257,41 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
             float* dst2 = dst + (size_t)p.splits * p.M * p.N;
 #pragma unroll
             for (int j = 0; j < 32; ++j)
-              if (n_ok && t0 + j < p.M) {
+              if (n_ok && j < jmax) {
                 dst[(size_t)(t0 + j) * p.N + n] = v[j];
                 dst2[(size_t)(t0 + j) * p.N + n] = u[j];
               }
           } else {
 #pragma unroll
             for (int j = 0; j < 32; ++j)
-              if (n_ok && t0 + j < p.M) dst[(size_t)(t0 + j) * p.N + n] = v[j];
+              if (n_ok && j < jmax) dst[(size_t)(t0 + j) * p.N + n] = v[j];
           }
         } else if (p.mode == 0) {
           bf16* C = reinterpret_cast<bf16*>(p.C);
 #pragma unroll
           for (int j = 0; j < 32; ++j)
-            if (n_ok && t0 + j < p.M) C[(size_t)(t0 + j) * p.ldc + n] = __float2bfloat16_rn(v[j]);
+            if (n_ok && j < jmax) C[(size_t)(t0 + j) * p.ldc + n] = __float2bfloat16_rn(v[j]);
         } else if (p.mode == 1) {
           // all loads first, then the stores: interleaving them would serialise on the load latency
           float* C = reinterpret_cast<float*>(p.C) + (size_t)t0 * p.ldc + n;
           float c[32];
 #pragma unroll
-          for (int j = 0; j < 32; ++j) c[j] = (n_ok && t0 + j < p.M) ? C[(size_t)j * p.ldc] : 0.f;
+          for (int j = 0; j < 32; ++j) c[j] = (n_ok && j < jmax) ? C[(size_t)j * p.ldc] : 0.f;
 #pragma unroll
           for (int j = 0; j < 32; ++j)
-            if (n_ok && t0 + j < p.M) C[(size_t)j * p.ldc] = c[j] + v[j];
+            if (n_ok && j < jmax) C[(size_t)j * p.ldc] = c[j] + v[j];
         } else if (p.mode == 2) {
           float* C = reinterpret_cast<float*>(p.C);
 #pragma unroll
           for (int j = 0; j < 32; ++j)
-            if (n_ok && t0 + j < p.M) C[(size_t)(t0 + j) * p.ldc + n] = v[j] * __ldg(p.row_scale + t0 + j);
+            if (n_ok && j < jmax) C[(size_t)(t0 + j) * p.ldc + n] = v[j] * __ldg(p.row_scale + t0 + j);
         } else {
           float u[32];
           tmem_ld32(t_row + 128 + c0, u);
           bf16* C = reinterpret_cast<bf16*>(p.C);
 #pragma unroll
           for (int j = 0; j < 32; ++j)
-            if (n_ok && t0 + j < p.M) C[(size_t)(t0 + j) * p.ldc + n] = __float2bfloat16_rn(silu_f(v[j]) * u[j]);
+            if (n_ok && j < jmax) C[(size_t)(t0 + j) * p.ldc + n] = __float2bfloat16_rn(silu_f(v[j]) * u[j]);
         }
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -383,7 +385,7 @@ int g_num_sms = 0;
 
 cudaError_t launch_gemm_tc(const bf16* A, int lda, const bf16* W, const bf16* W2, void* C, int ldc, int M, int N,
                            int K, int mode, const float* row_scale, const GemmScratch& scratch, cudaStream_t s,
-                           bool* handled) {
+                           bool* handled, int* splits_out) {
   float* const g_partial = scratch.partial;
   const size_t g_partial_floats = scratch.partial_floats;
   int* const g_error_flag = scratch.error_flag;
@@ -405,31 +407,30 @@ cudaError_t launch_gemm_tc(const bf16* A, int lda, const bf16* W, const bf16* W2
   p.kblocks = (K + BK - 1) / BK;
   p.n_tiles = (N + TILE_N - 1) / TILE_N;
   p.error_flag = g_error_flag;
-  // ---- tile shape and k split: fill the SMs, keep tensor-core tiles wide when there is work for them ----
-  const int tn_max = dual ? 128 : 256;
-  int best_tn = 32, best_s = 1;
-  double best_t = 1e30;
-  for (int tn = 32; tn <= tn_max; tn *= 2) {
-    const int m_tiles = (M + tn - 1) / tn;
-    for (int sp = 1; sp <= 8; ++sp) {
-      if (sp > 1 && (p.kblocks / sp < 4)) break;
-      if (sp > 1 && (!g_partial || (size_t)sp * (dual ? 2 : 1) * (size_t)M * N > g_partial_floats)) break;
-      const long long items = (long long)p.n_tiles * m_tiles * sp;
-      const double waves = (double)((items + g_num_sms - 1) / g_num_sms);
-      const double kslice = (double)K / sp;
-      const double mma_eff = tn >= 128 ? 1.0 : (tn == 64 ? 0.67 : 0.4);
-      const double t_mma = (dual ? 2.0 : 1.0) * TILE_N * tn * kslice / (4096.0 * mma_eff);          // clocks
-      const double t_mem = ((dual ? 2.0 : 1.0) * TILE_N + tn * 0.25) * kslice * 2.0 / 24.0;         // clocks
-      const double t_epi = 400.0 + tn * 6.0;
-      double t = waves * ((t_mma > t_mem ? t_mma : t_mem) + t_epi + 1500.0);
-      if (sp > 1) t += 2.0 * sp * (dual ? 2 : 1) * (double)M * N * 4.0 / (24.0 * g_num_sms) + 4000.0;
-      if (t < best_t) { best_t = t; best_tn = tn; best_s = sp; }
-    }
+  // ---- token tile and k split ----
+  // Few tokens (a block step): one or two token tiles that cover M exactly (UMMA N is any multiple of 16), and a
+  // k split that spreads the weight stream over all SMs when there are fewer weight tiles than SMs.
+  // Many tokens (a refresh step): the widest tile, no split.
+  const int tn_cap = dual ? 128 : 256;
+  if (M <= 2 * tn_cap) {
+    p.m_tiles = (M + tn_cap - 1) / tn_cap;
+    p.tn = (((M + p.m_tiles - 1) / p.m_tiles) + 15) / 16 * 16;
+  } else {
+    p.tn = tn_cap;
+    p.m_tiles = (M + p.tn - 1) / p.tn;
   }
-  p.tn = best_tn;
-  p.splits = best_s;
-  p.m_tiles = (M + p.tn - 1) / p.tn;
+  p.splits = 1;
+  const long long base_items = (long long)p.n_tiles * p.m_tiles;
+  if (g_partial && base_items * 4 < (long long)g_num_sms * 3) {
+    int sp = (int)(g_num_sms / base_items);
+    if (sp > 8) sp = 8;
+    while (sp > 1 && (p.kblocks / sp < 4 || (size_t)sp * (size_t)M * N > g_partial_floats)) --sp;
+    p.splits = sp < 1 ? 1 : sp;
+  }
+  if (mode == 4 && (!g_partial || (size_t)p.splits * (size_t)M * N > g_partial_floats)) return cudaErrorInvalidValue;
+  if (dual) p.splits = 1;
   p.partial = g_partial;
+  if (splits_out) *splits_out = p.splits;
   const int stage_bytes = (dual ? 2 : 1) * TILE_N * BK * 2 + p.tn * BK * 2;
   p.stages = kSmemBudget / stage_bytes;
   if (p.stages > 16) p.stages = 16;
@@ -446,7 +447,7 @@ cudaError_t launch_gemm_tc(const bf16* A, int lda, const bf16* W, const bf16* W2
   k_gemm_tc<<<grid, kThreads, kSmemBudget + 1024, s>>>(mw, mw2, mx, p);
   cudaError_t r = cudaGetLastError();
   if (r != cudaSuccess) return r;
-  if (p.splits > 1) {
+  if (p.splits > 1 && mode != 4) {
     const size_t total = (size_t)M * N;
     const int blocks = (int)((total + 255) / 256 < (size_t)g_num_sms * 8 ? (total + 255) / 256 : (size_t)g_num_sms * 8);
     k_gemm_finish<<<blocks, 256, 0, s>>>(g_partial, p.splits, M, N, mode, C, ldc, row_scale);

@@ -27,7 +27,8 @@ def rel_err(got, ref):
 
 GEMM_SHAPES = [  # M, N, K: several tiles, ragged tails in every dimension, one case smaller than a tile
     (1, 128, 64), (33, 200, 72), (128, 256, 128), (130, 1000, 384), (257, 130, 1000), (300, 2000, 256),
-    (517, 704, 256), (64, 4608, 512), (1000, 512, 2048)]
+    (517, 704, 256), (64, 4608, 512), (1000, 512, 2048), (459, 768, 256), (459, 256, 704), (48, 384, 128),
+    (200, 640, 320)]
 
 
 @pytest.mark.parametrize("M,N,K", GEMM_SHAPES)
