@@ -226,8 +226,10 @@ int bs_op_rope_kv_static(void* qkv, const int* tok_pos, const int* tok_kv, void*
  * bs_op_attention_q_tile(Hq, Hkv) tokens: cu_tile[i] = sum_{r<i} ceil(n_q(r) / q_tile), n_tiles = cu_tile[n_rows]. */
 int bs_op_attention_q_tile(int n_q_heads, int n_kv_heads);
 int bs_op_attention(const void* qkv, const void* kcache, const void* vcache, void* out, const int* cu_q,
-                    const int* cu_tile, const int* kv_base, const int* vis, int n_rows, int n_tiles, int n_q_heads,
-                    int n_kv_heads, int head_dim, void* stream);
+                    const int* cu_tile, const int* kv_base, const int* vis, int n_rows, int n_tiles,
+                    int M /* packed tokens */, int max_vis /* largest vis[i] */, int n_q_heads, int n_kv_heads,
+                    int head_dim, float* scratch /* nullable: lets few work items split their keys over CTAs */,
+                    size_t scratch_bytes, void* stream);
 
 /* Per row of fp32 logits [n_rows, vocab]: mask id excluded, tok = argmax (lowest id on ties),
  * conf = exp(max - logsumexp). */

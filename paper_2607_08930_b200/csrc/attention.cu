@@ -4,13 +4,13 @@
 // Keys are the row's cache span [kv_base_i, kv_base_i + vis_i): prefix, fresh block and suffix alike;
 // there is no causal mask and no padding mask.  Online softmax with warp shuffles, mma.sync m16n8k16.
 #include <math.h>
+#include <stdlib.h>
 
 #include "common.cuh"
 
 namespace bs {
 
 namespace {
-constexpr int KT = 64;   // keys per tile
 
 __device__ __forceinline__ void cp_async16(void* dst, const void* src, int bytes) {
   const unsigned d = (unsigned)__cvta_generic_to_shared(dst);
@@ -36,17 +36,28 @@ __device__ __forceinline__ unsigned pack_bf16(float a, float b) {
   return *reinterpret_cast<unsigned*>(&h);
 }
 
-template <int DH>
-__global__ void __launch_bounds__(256) k_attention(const bf16* __restrict__ qkv, const bf16* __restrict__ kc,
-                                                   const bf16* __restrict__ vc, bf16* __restrict__ out,
-                                                   const int* __restrict__ cu_q, const int* __restrict__ cu_tile,
-                                                   const int* __restrict__ kv_base, const int* __restrict__ vis_arr,
-                                                   int n_rows, int hq, int hkv, int q_tile) {
+// Partial result of one KV chunk of a work item: unnormalised output (fp32) plus (running max in log2 units, sum).
+struct AttnPartial {
+  float* o;        // [chunks][M][Hq * dh]
+  float2* ml;      // [chunks][M][Hq]
+  int chunks;
+  int M;
+};
+
+template <int DH, int KT, int NSTAGE, int MINB>
+__global__ void __launch_bounds__(256, MINB) k_attention(const bf16* __restrict__ qkv, const bf16* __restrict__ kc,
+                                                         const bf16* __restrict__ vc, bf16* __restrict__ out,
+                                                         const int* __restrict__ cu_q, const int* __restrict__ cu_tile,
+                                                         const int* __restrict__ kv_base,
+                                                         const int* __restrict__ vis_arr, int n_rows, int hq, int hkv,
+                                                         int q_tile, AttnPartial part) {
   constexpr int LD = DH + 8;
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  bf16* smem = reinterpret_cast<bf16*>(smem_raw);      // [2 stages][K tile, V tile][KT][LD]
+  bf16* smem = reinterpret_cast<bf16*>(smem_raw);      // [NSTAGE][K tile, V tile][KT][LD]
   const int G = hq / hkv;
   const int kh = blockIdx.y;
+  pdl_wait();
+  pdl_trigger();
   // which row owns this q-tile: largest r with cu_tile[r] <= blockIdx.x
   int lo = 0, hi = n_rows;
   while (hi - lo > 1) {
@@ -60,6 +71,11 @@ __global__ void __launch_bounds__(256) k_attention(const bf16* __restrict__ qkv,
   const int vis = vis_arr[row];
   const size_t kvb = (size_t)kv_base[row];
   const int qkv_ld = (hq + 2 * hkv) * DH;
+  // key tiles of this CTA's chunk
+  const int nkt_all = (vis + KT - 1) / KT;
+  const int per = (nkt_all + part.chunks - 1) / part.chunks;
+  const int kt0 = (int)blockIdx.z * per;
+  const int kt1 = min(nkt_all, kt0 + per);
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int nthreads = blockDim.x;
@@ -103,16 +119,18 @@ __global__ void __launch_bounds__(256) k_attention(const bf16* __restrict__ qkv,
   float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
   const float sc = 1.4426950408889634f / sqrtf((float)DH);    // log2(e) / sqrt(dh)
 
-  const int nkt = (vis + KT - 1) / KT;
-  load_tile(0, 0);
-  asm volatile("cp.async.commit_group;\n" ::);
-  for (int kt = 0; kt < nkt; ++kt) {
-    if (kt + 1 < nkt) load_tile((kt + 1) & 1, kt + 1);
+#pragma unroll
+  for (int i = 0; i < NSTAGE - 1; ++i) {
+    if (kt0 + i < kt1) load_tile(i, kt0 + i);
     asm volatile("cp.async.commit_group;\n" ::);
-    asm volatile("cp.async.wait_group 1;\n" ::);
+  }
+  for (int kt = kt0; kt < kt1; ++kt) {
+    asm volatile("cp.async.wait_group %0;\n" ::"n"(NSTAGE - 2));
     __syncthreads();
+    if (kt + NSTAGE - 1 < kt1) load_tile((kt - kt0 + NSTAGE - 1) % NSTAGE, kt + NSTAGE - 1);
+    asm volatile("cp.async.commit_group;\n" ::);
     if (warp_active) {
-      const bf16* sK = smem + (kt & 1) * 2 * KT * LD;
+      const bf16* sK = smem + ((kt - kt0) % NSTAGE) * 2 * KT * LD;
       const bf16* sV = sK + KT * LD;
       float s[KT / 8][4];
 #pragma unroll
@@ -185,7 +203,6 @@ __global__ void __launch_bounds__(256) k_attention(const bf16* __restrict__ qkv,
         }
       }
     }
-    __syncthreads();
   }
   asm volatile("cp.async.wait_group 0;\n" ::);
   if (!warp_active) return;
@@ -193,8 +210,29 @@ __global__ void __launch_bounds__(256) k_attention(const bf16* __restrict__ qkv,
   l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
   l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
   l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
-  const float i0 = 1.0f / l0, i1 = 1.0f / l1;
   const int out_ld = hq * DH;
+  if (part.chunks > 1) {
+    // unnormalised partial of this KV chunk; the combine kernel merges the chunks
+    const size_t zoff = (size_t)blockIdx.z * part.M;
+    if (v0) {
+      float* dst = part.o + (zoff + t0 + tk0) * out_ld + hd0 * DH + (lane & 3) * 2;
+      if (l0 > 0.f) {
+#pragma unroll
+        for (int i = 0; i < DH / 8; ++i) *reinterpret_cast<float2*>(dst + i * 8) = make_float2(o[i][0], o[i][1]);
+      }
+      if ((lane & 3) == 0) part.ml[(zoff + t0 + tk0) * hq + hd0] = make_float2(m0, l0);
+    }
+    if (v1) {
+      float* dst = part.o + (zoff + t0 + tk1) * out_ld + hd1 * DH + (lane & 3) * 2;
+      if (l1 > 0.f) {
+#pragma unroll
+        for (int i = 0; i < DH / 8; ++i) *reinterpret_cast<float2*>(dst + i * 8) = make_float2(o[i][2], o[i][3]);
+      }
+      if ((lane & 3) == 0) part.ml[(zoff + t0 + tk1) * hq + hd1] = make_float2(m1, l1);
+    }
+    return;
+  }
+  const float i0 = 1.0f / l0, i1 = 1.0f / l1;
   if (v0) {
     bf16* dst = out + (size_t)(t0 + tk0) * out_ld + hd0 * DH + (lane & 3) * 2;
 #pragma unroll
@@ -208,6 +246,37 @@ __global__ void __launch_bounds__(256) k_attention(const bf16* __restrict__ qkv,
       *reinterpret_cast<__nv_bfloat162*>(dst + i * 8) = __floats2bfloat162_rn(o[i][2] * i1, o[i][3] * i1);
   }
 }
+
+// Merges the KV chunks of every (token, head): out = sum_c w_c o_c / sum_c w_c l_c with w_c = 2^(m_c - max m).
+__global__ void __launch_bounds__(256) k_attention_combine(AttnPartial part, bf16* __restrict__ out, int hq, int dh) {
+  pdl_wait();
+  pdl_trigger();
+  const int t = blockIdx.x;
+  const int out_ld = hq * dh;
+  const int pairs = out_ld / 2;
+  for (int u = threadIdx.x; u < pairs; u += 256) {
+    const int h = (2 * u) / dh;
+    float mmax = -INFINITY;
+    for (int c = 0; c < part.chunks; ++c) {
+      const float2 ml = part.ml[((size_t)c * part.M + t) * hq + h];
+      if (ml.y > 0.f) mmax = fmaxf(mmax, ml.x);
+    }
+    float2 acc = make_float2(0.f, 0.f);
+    float L = 0.f;
+    for (int c = 0; c < part.chunks; ++c) {
+      const float2 ml = part.ml[((size_t)c * part.M + t) * hq + h];
+      if (ml.y > 0.f) {
+        const float w = exp2f(ml.x - mmax);
+        const float2 ov = *reinterpret_cast<const float2*>(part.o + ((size_t)c * part.M + t) * out_ld + 2 * u);
+        acc.x += w * ov.x;
+        acc.y += w * ov.y;
+        L += w * ml.y;
+      }
+    }
+    const float inv = 1.0f / L;
+    *reinterpret_cast<__nv_bfloat162*>(out + (size_t)t * out_ld + 2 * u) = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
+  }
+}
 }  // namespace
 
 int attention_q_tile(int hq, int hkv) {
@@ -215,26 +284,79 @@ int attention_q_tile(int hq, int hkv) {
   return G >= 5 ? 16 : (G == 1 ? 64 : 32);
 }
 
+namespace {
+template <int DH, int KT, int NSTAGE, int MINB>
+cudaError_t launch_variant(dim3 grid, int threads, cudaStream_t s, const bf16* qkv, const bf16* kc, const bf16* vc,
+                           bf16* out, const int* cu_q, const int* cu_tile, const int* kv_base, const int* vis,
+                           int n_rows, int hq, int hkv, int qt, AttnPartial part) {
+  constexpr size_t smem = (size_t)NSTAGE * 2 * KT * (DH + 8) * sizeof(bf16);
+  static bool done = false;
+  if (!done) {
+    cudaFuncSetAttribute(k_attention<DH, KT, NSTAGE, MINB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    done = true;
+  }
+  return launch_pdl(k_attention<DH, KT, NSTAGE, MINB>, grid, dim3(threads), smem, s, qkv, kc, vc, out, cu_q, cu_tile,
+                    kv_base, vis, n_rows, hq, hkv, qt, part);
+}
+}  // namespace
+
 cudaError_t launch_attention(const bf16* qkv, const bf16* kc, const bf16* vc, bf16* out, const int* cu_q,
-                             const int* cu_tile, const int* kv_base, const int* vis, int n_rows, int n_tiles,
-                             int hq, int hkv, int dh, cudaStream_t s) {
+                             const int* cu_tile, const int* kv_base, const int* vis, int n_rows, int n_tiles, int M,
+                             int max_vis, int hq, int hkv, int dh, float* scratch, size_t scratch_floats,
+                             cudaStream_t s) {
   if (n_tiles <= 0 || n_rows <= 0) return cudaSuccess;
   const int G = hq / hkv;
   const int qt = attention_q_tile(hq, hkv);
   const int threads = qt * G * 2;             // 16 flattened rows per warp
   if (threads > 256 || (dh != 64 && dh != 128) || hq % hkv != 0) return cudaErrorInvalidValue;
-  const size_t smem = (size_t)2 * 2 * KT * (dh + 8) * sizeof(bf16);
-  dim3 grid(n_tiles, hkv);
-  if (dh == 128) {
-    static bool done = false;
-    if (!done) { cudaFuncSetAttribute(k_attention<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); done = true; }
-    k_attention<128><<<grid, threads, smem, s>>>(qkv, kc, vc, out, cu_q, cu_tile, kv_base, vis, n_rows, hq, hkv, qt);
-  } else {
-    static bool done = false;
-    if (!done) { cudaFuncSetAttribute(k_attention<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); done = true; }
-    k_attention<64><<<grid, threads, smem, s>>>(qkv, kc, vc, out, cu_q, cu_tile, kv_base, vis, n_rows, hq, hkv, qt);
+  // KV chunks: a block step has few (row, kv head, q tile) items, each a long serial walk over the row's keys;
+  // splitting the walk fills the SMs.  A refresh step has plenty of items already.
+  static int num_sms = 0;
+  if (!num_sms) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
   }
-  return cudaGetLastError();
+  // (measured on B200: with fewer work items than a quarter / a half of the SMs, 4 / 2 chunks shorten the
+  // serial walk enough to pay for the merge; beyond that the legacy-path MMAs are the limit and chunks only add work)
+  const long long base = (long long)n_tiles * hkv;
+  int chunks = 1;
+  if (scratch && max_vis >= 256) {
+    chunks = base * 4 <= num_sms + 12 ? 4 : (base * 2 <= num_sms ? 2 : 1);
+    while (chunks > 1 && (size_t)chunks * M * ((size_t)hq * dh + 2 * hq) > scratch_floats) chunks >>= 1;
+  }
+  if (const char* ev = getenv("BS_ATTN_CHUNKS")) {
+    const int c = atoi(ev);
+    if (c >= 1 && (c == 1 || scratch)) chunks = c;
+  }
+  int variant = 1;
+  if (const char* ev = getenv("BS_ATTN_VARIANT")) variant = atoi(ev);
+  AttnPartial part;
+  part.chunks = chunks;
+  part.M = M;
+  part.o = scratch;
+  part.ml = reinterpret_cast<float2*>(scratch + (size_t)chunks * M * hq * dh);
+  dim3 grid(n_tiles, hkv, chunks);
+  cudaError_t r;
+  if (dh == 128) {
+    if (variant == 0)
+      r = launch_variant<128, 32, 3, 2>(grid, threads, s, qkv, kc, vc, out, cu_q, cu_tile, kv_base, vis, n_rows, hq,
+                                        hkv, qt, part);
+    else if (variant == 2)
+      r = launch_variant<128, 64, 3, 1>(grid, threads, s, qkv, kc, vc, out, cu_q, cu_tile, kv_base, vis, n_rows, hq,
+                                        hkv, qt, part);
+    else
+      r = launch_variant<128, 64, 2, 1>(grid, threads, s, qkv, kc, vc, out, cu_q, cu_tile, kv_base, vis, n_rows, hq,
+                                        hkv, qt, part);
+  } else {
+    r = launch_variant<64, 64, 2, 2>(grid, threads, s, qkv, kc, vc, out, cu_q, cu_tile, kv_base, vis, n_rows, hq, hkv,
+                                     qt, part);
+  }
+  if (r != cudaSuccess) return r;
+  if (chunks > 1) {
+    r = launch_pdl(k_attention_combine, dim3(M), dim3(256), 0, s, part, out, hq, dh);
+  }
+  return r;
 }
 
 }  // namespace bs

@@ -3,10 +3,36 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <stdlib.h>
+
+#include <utility>
 
 namespace bs {
 
 typedef __nv_bfloat16 bf16;
+
+// Programmatic dependent launch: every kernel of a step is launched with the stream-serialisation attribute, calls
+// pdl_wait() before it touches global memory (the grid before it has then completed and its writes are visible) and
+// pdl_trigger() right after, so that the next kernel's launch latency and set-up overlap this kernel's run.
+// Every CTA of every kernel executes pdl_wait(): completion of a grid then implies completion of all earlier ones.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  static const bool disabled = getenv("BS_NO_PDL") != nullptr;
+  cfg.numAttrs = disabled ? 0 : 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(std::forward<Args>(args))...);
+}
 
 constexpr int kHdrInts = 32;
 // header words (device int32[kHdrInts], mirrored to pinned host memory once per step)
@@ -47,9 +73,11 @@ cudaError_t launch_rmsnorm(const float* x, const int* idx, const bf16* w, bf16* 
                            cudaStream_t s);
 cudaError_t launch_rope_kv(bf16* qkv, const int* tok_pos, const int* tok_kv, bf16* kc, bf16* vc, int M, int hq,
                            int hkv, int dh, const float* cos_sin, cudaStream_t s);
+// scratch (nullable): fp32 partial results when the keys of a work item are split over several CTAs.
 cudaError_t launch_attention(const bf16* qkv, const bf16* kc, const bf16* vc, bf16* out, const int* cu_q,
-                             const int* cu_tile, const int* kv_base, const int* vis, int n_rows, int n_tiles,
-                             int hq, int hkv, int dh, cudaStream_t s);
+                             const int* cu_tile, const int* kv_base, const int* vis, int n_rows, int n_tiles, int M,
+                             int max_vis, int hq, int hkv, int dh, float* scratch, size_t scratch_floats,
+                             cudaStream_t s);
 cudaError_t launch_confidence(const float* logits, int n_rows, int vocab, int mask_id, int* tok, float* conf,
                               cudaStream_t s);
 

@@ -14,6 +14,8 @@ __device__ __forceinline__ float warp_sum(float v) {
 
 // x[t, :] = E[token at (row, position) of packed token t]   (gather of the active regions, Section 2.5)
 __global__ void k_embed(DevState st, const bf16* __restrict__ embed, float* __restrict__ x, int M, int d) {
+  pdl_wait();
+  pdl_trigger();
   const int t = blockIdx.x;
   if (t >= M) return;
   const int slot = st.row_slot[st.tok_row[t]];
@@ -34,6 +36,8 @@ __global__ void k_embed(DevState st, const bf16* __restrict__ embed, float* __re
 __global__ void __launch_bounds__(256) k_rmsnorm(const float* __restrict__ x, const int* __restrict__ idx,
                                                  const bf16* __restrict__ w, bf16* __restrict__ y, int d, float eps) {
   __shared__ float red[8];
+  pdl_wait();
+  pdl_trigger();
   const int m = blockIdx.x;
   const int row = idx ? idx[m] : m;
   const float4* src = reinterpret_cast<const float4*>(x + (size_t)row * d);
@@ -71,6 +75,8 @@ __global__ void __launch_bounds__(256) k_rope_kv(bf16* __restrict__ qkv, const i
                                                  const int* __restrict__ tok_kv, bf16* __restrict__ kc,
                                                  bf16* __restrict__ vc, int hq, int hkv, int dh,
                                                  const float2* __restrict__ cos_sin) {
+  pdl_wait();
+  pdl_trigger();
   const int t = blockIdx.x;
   const int pos = tok_pos[t];
   const size_t kvrow = (size_t)tok_kv[t];
@@ -108,6 +114,8 @@ __global__ void __launch_bounds__(kConfThreads) k_confidence(const float* __rest
                                                              int* __restrict__ tok, float* __restrict__ conf) {
   __shared__ float s_m[kConfThreads / 32], s_s[kConfThreads / 32];
   __shared__ int s_i[kConfThreads / 32];
+  pdl_wait();
+  pdl_trigger();
   const int row = blockIdx.x;
   const float* z = logits + (size_t)row * vocab;
   float m = -INFINITY, s = 0.f;
@@ -178,59 +186,96 @@ __global__ void __launch_bounds__(kConfThreads) k_confidence(const float* __rest
   }
 }
 
+constexpr int kMaxSplits = 8;
+
 // Finishing kernel of the QKV projection on block steps: adds the k-split partial sums in split order, rounds q / k / v
 // to bf16, rotates q and k at the token's position id and scatters k, v to the token's cache row.
-__global__ void __launch_bounds__(256) k_finish_qkv_rope(const float* __restrict__ partial, int splits, int M,
+// grid (tokens, head groups of kHeadsPerBlock); all partial loads of an element are issued before they are summed.
+constexpr int kHeadsPerBlock = 4;
+__global__ void __launch_bounds__(128) k_finish_qkv_rope(const float* __restrict__ partial, int splits, int M,
                                                          bf16* __restrict__ qkv, const int* __restrict__ tok_pos,
                                                          const int* __restrict__ tok_kv, bf16* __restrict__ kc,
                                                          bf16* __restrict__ vc, int hq, int hkv, int dh,
                                                          const float2* __restrict__ cos_sin) {
+  pdl_wait();
+  pdl_trigger();
   const int t = blockIdx.x;
-  const int N = (hq + 2 * hkv) * dh, half = dh / 2;
+  const int n_heads = hq + 2 * hkv;
+  const int N = n_heads * dh, half = dh / 2;
   const size_t slice = (size_t)M * N;
   const float* row = partial + (size_t)t * N;
   const int pos = tok_pos[t];
   const size_t kvrow = (size_t)tok_kv[t];
   const float2* cs = cos_sin + (size_t)pos * half;
   bf16* qrow = qkv + (size_t)t * N;
-  const int pairs_per_head = half / 2;
-  const int n_rot = (hq + hkv) * pairs_per_head;
-  for (int u = threadIdx.x; u < n_rot; u += 256) {
-    const int h = u / pairs_per_head, j = (u % pairs_per_head) * 2;
-    float2 a = make_float2(0.f, 0.f), b = make_float2(0.f, 0.f);
-    for (int s = 0; s < splits; ++s) {
-      const float2 pa = *reinterpret_cast<const float2*>(row + s * slice + h * dh + j);
-      const float2 pb = *reinterpret_cast<const float2*>(row + s * slice + h * dh + half + j);
-      a.x += pa.x; a.y += pa.y; b.x += pb.x; b.y += pb.y;
+  const int quads_per_head = half / 4;                 // a thread rotates 4 adjacent pairs (j..j+3, j+half..)
+  const int h0 = blockIdx.y * kHeadsPerBlock;
+  for (int u = threadIdx.x; u < kHeadsPerBlock * quads_per_head; u += 128) {
+    const int h = h0 + u / quads_per_head, j = (u % quads_per_head) * 4;
+    if (h >= n_heads) break;
+    float4 pa[kMaxSplits], pb[kMaxSplits];
+#pragma unroll
+    for (int s = 0; s < kMaxSplits; ++s)
+      if (s < splits) {
+        pa[s] = *reinterpret_cast<const float4*>(row + s * slice + h * dh + j);
+        if (h < hq + hkv) pb[s] = *reinterpret_cast<const float4*>(row + s * slice + h * dh + half + j);
+      }
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+#pragma unroll
+    for (int s = 0; s < kMaxSplits; ++s)
+      if (s < splits) {
+        a.x += pa[s].x; a.y += pa[s].y; a.z += pa[s].z; a.w += pa[s].w;
+        if (h < hq + hkv) { b.x += pb[s].x; b.y += pb[s].y; b.z += pb[s].z; b.w += pb[s].w; }
+      }
+    if (h < hq + hkv) {
+      // the projection's output is a bf16 tensor: round, rotate in fp32, round again
+      const float2 a01 = __bfloat1622float2(__floats2bfloat162_rn(a.x, a.y));
+      const float2 a23 = __bfloat1622float2(__floats2bfloat162_rn(a.z, a.w));
+      const float2 b01 = __bfloat1622float2(__floats2bfloat162_rn(b.x, b.y));
+      const float2 b23 = __bfloat1622float2(__floats2bfloat162_rn(b.z, b.w));
+      const float2 c0 = cs[j], c1 = cs[j + 1], c2 = cs[j + 2], c3 = cs[j + 3];
+      __nv_bfloat162 lo01 = __floats2bfloat162_rn(a01.x * c0.x - b01.x * c0.y, a01.y * c1.x - b01.y * c1.y);
+      __nv_bfloat162 lo23 = __floats2bfloat162_rn(a23.x * c2.x - b23.x * c2.y, a23.y * c3.x - b23.y * c3.y);
+      __nv_bfloat162 hi01 = __floats2bfloat162_rn(b01.x * c0.x + a01.x * c0.y, b01.y * c1.x + a01.y * c1.y);
+      __nv_bfloat162 hi23 = __floats2bfloat162_rn(b23.x * c2.x + a23.x * c2.y, b23.y * c3.x + a23.y * c3.y);
+      bf16* dst = h < hq ? qrow + h * dh : kc + (kvrow * hkv + (h - hq)) * dh;
+      uint2 lo, hi;
+      lo.x = *reinterpret_cast<unsigned*>(&lo01); lo.y = *reinterpret_cast<unsigned*>(&lo23);
+      hi.x = *reinterpret_cast<unsigned*>(&hi01); hi.y = *reinterpret_cast<unsigned*>(&hi23);
+      *reinterpret_cast<uint2*>(dst + j) = lo;
+      *reinterpret_cast<uint2*>(dst + half + j) = hi;
+    } else {
+      // a v head: this thread owns 4 values of the first half; the second half is handled below
+      bf16* dst = vc + (kvrow * hkv + (h - hq - hkv)) * dh;
+      __nv_bfloat162 v01 = __floats2bfloat162_rn(a.x, a.y), v23 = __floats2bfloat162_rn(a.z, a.w);
+      uint2 o;
+      o.x = *reinterpret_cast<unsigned*>(&v01); o.y = *reinterpret_cast<unsigned*>(&v23);
+      *reinterpret_cast<uint2*>(dst + j) = o;
+      float4 c = make_float4(0.f, 0.f, 0.f, 0.f);
+      float4 pc[kMaxSplits];
+#pragma unroll
+      for (int s = 0; s < kMaxSplits; ++s)
+        if (s < splits) pc[s] = *reinterpret_cast<const float4*>(row + s * slice + h * dh + half + j);
+#pragma unroll
+      for (int s = 0; s < kMaxSplits; ++s)
+        if (s < splits) { c.x += pc[s].x; c.y += pc[s].y; c.z += pc[s].z; c.w += pc[s].w; }
+      v01 = __floats2bfloat162_rn(c.x, c.y);
+      v23 = __floats2bfloat162_rn(c.z, c.w);
+      o.x = *reinterpret_cast<unsigned*>(&v01); o.y = *reinterpret_cast<unsigned*>(&v23);
+      *reinterpret_cast<uint2*>(dst + half + j) = o;
     }
-    a = __bfloat1622float2(__floats2bfloat162_rn(a.x, a.y));     // the projection's output is a bf16 tensor
-    b = __bfloat1622float2(__floats2bfloat162_rn(b.x, b.y));
-    const float2 c0 = cs[j], c1 = cs[j + 1];
-    const __nv_bfloat162 o1 = __floats2bfloat162_rn(a.x * c0.x - b.x * c0.y, a.y * c1.x - b.y * c1.y);
-    const __nv_bfloat162 o2 = __floats2bfloat162_rn(b.x * c0.x + a.x * c0.y, b.y * c1.x + a.y * c1.y);
-    bf16* dst = h < hq ? qrow + h * dh : kc + (kvrow * hkv + (h - hq)) * dh;
-    *reinterpret_cast<__nv_bfloat162*>(dst + j) = o1;
-    *reinterpret_cast<__nv_bfloat162*>(dst + half + j) = o2;
-  }
-  const int v0 = (hq + hkv) * dh;
-  bf16* vdst = vc + kvrow * hkv * dh;
-  for (int u = threadIdx.x; u < hkv * dh / 2; u += 256) {
-    float2 a = make_float2(0.f, 0.f);
-    for (int s = 0; s < splits; ++s) {
-      const float2 pa = *reinterpret_cast<const float2*>(row + s * slice + v0 + 2 * u);
-      a.x += pa.x; a.y += pa.y;
-    }
-    *reinterpret_cast<__nv_bfloat162*>(vdst + 2 * u) = __floats2bfloat162_rn(a.x, a.y);
   }
 }
 
 // Finishing kernel of the O and down projections on block steps: x += sum of the k-split partial sums (split order),
-// then, if a gain vector is given, the RMSNorm that feeds the next projection.
+// then, if a gain vector is given, the RMSNorm that feeds the next projection.  One CTA per token.
 __global__ void __launch_bounds__(256) k_finish_residual_norm(const float* __restrict__ partial, int splits, int M,
                                                               int d, float* __restrict__ x,
                                                               const bf16* __restrict__ w, bf16* __restrict__ h,
                                                               float eps) {
   __shared__ float red[8];
+  pdl_wait();
+  pdl_trigger();
   const int t = blockIdx.x;
   const size_t slice = (size_t)M * d;
   float4* xr = reinterpret_cast<float4*>(x + (size_t)t * d);
@@ -242,10 +287,13 @@ __global__ void __launch_bounds__(256) k_finish_residual_norm(const float* __res
     const int c = threadIdx.x + i * 256;
     if (c < d / 4) {
       float4 v = xr[c];
-      for (int s = 0; s < splits; ++s) {
-        const float4 pv = *reinterpret_cast<const float4*>(prow + s * slice + 4 * c);
-        v.x += pv.x; v.y += pv.y; v.z += pv.z; v.w += pv.w;
-      }
+      float4 pv[kMaxSplits];
+#pragma unroll
+      for (int s = 0; s < kMaxSplits; ++s)
+        if (s < splits) pv[s] = *reinterpret_cast<const float4*>(prow + s * slice + 4 * c);
+#pragma unroll
+      for (int s = 0; s < kMaxSplits; ++s)
+        if (s < splits) { v.x += pv[s].x; v.y += pv[s].y; v.z += pv[s].z; v.w += pv[s].w; }
       xr[c] = v;
       vals[i] = v;
       ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
@@ -283,40 +331,37 @@ cudaError_t launch_finish_qkv_rope(const float* partial, int splits, int M, bf16
                                    const int* tok_kv, bf16* kc, bf16* vc, int hq, int hkv, int dh,
                                    const float* cos_sin, cudaStream_t s) {
   if (M <= 0) return cudaSuccess;
-  k_finish_qkv_rope<<<M, 256, 0, s>>>(partial, splits, M, qkv, tok_pos, tok_kv, kc, vc, hq, hkv, dh,
-                                       reinterpret_cast<const float2*>(cos_sin));
-  return cudaGetLastError();
+  if (splits > kMaxSplits || dh % 8) return cudaErrorInvalidValue;
+  dim3 grid(M, (hq + 2 * hkv + kHeadsPerBlock - 1) / kHeadsPerBlock);
+  return launch_pdl(k_finish_qkv_rope, grid, dim3(128), 0, s, partial, splits, M, qkv, tok_pos, tok_kv, kc, vc, hq, hkv,
+                    dh, reinterpret_cast<const float2*>(cos_sin));
 }
 cudaError_t launch_finish_residual_norm(const float* partial, int splits, int M, int d, float* x, const bf16* w,
                                         bf16* h, float eps, cudaStream_t s) {
   if (M <= 0) return cudaSuccess;
-  if (d > 8192) return cudaErrorInvalidValue;
-  k_finish_residual_norm<<<M, 256, 0, s>>>(partial, splits, M, d, x, w, h, eps);
-  return cudaGetLastError();
+  if (d > 8192 || splits > kMaxSplits) return cudaErrorInvalidValue;
+  return launch_pdl(k_finish_residual_norm, dim3(M), dim3(256), 0, s, partial, splits, M, d, x, w, h, eps);
 }
 
 cudaError_t launch_embed(const DevState& st, const bf16* embed, float* x, int M, int d, cudaStream_t s) {
   if (M <= 0) return cudaSuccess;
-  k_embed<<<M, 128, 0, s>>>(st, embed, x, M, d);
-  return cudaGetLastError();
+  return launch_pdl(k_embed, dim3(M), dim3(128), 0, s, st, embed, x, M, d);
 }
 cudaError_t launch_rmsnorm(const float* x, const int* idx, const bf16* w, bf16* y, int M, int d, float eps,
                            cudaStream_t s) {
   if (M <= 0) return cudaSuccess;
-  k_rmsnorm<<<M, 256, 0, s>>>(x, idx, w, y, d, eps);
-  return cudaGetLastError();
+  return launch_pdl(k_rmsnorm, dim3(M), dim3(256), 0, s, x, idx, w, y, d, eps);
 }
 cudaError_t launch_rope_kv(bf16* qkv, const int* tok_pos, const int* tok_kv, bf16* kc, bf16* vc, int M, int hq,
                            int hkv, int dh, const float* cos_sin, cudaStream_t s) {
   if (M <= 0) return cudaSuccess;
-  k_rope_kv<<<M, 256, 0, s>>>(qkv, tok_pos, tok_kv, kc, vc, hq, hkv, dh, reinterpret_cast<const float2*>(cos_sin));
-  return cudaGetLastError();
+  return launch_pdl(k_rope_kv, dim3(M), dim3(256), 0, s, qkv, tok_pos, tok_kv, kc, vc, hq, hkv, dh,
+                    reinterpret_cast<const float2*>(cos_sin));
 }
 cudaError_t launch_confidence(const float* logits, int n_rows, int vocab, int mask_id, int* tok, float* conf,
                               cudaStream_t s) {
   if (n_rows <= 0) return cudaSuccess;
-  k_confidence<<<n_rows, kConfThreads, 0, s>>>(logits, vocab, mask_id, tok, conf);
-  return cudaGetLastError();
+  return launch_pdl(k_confidence, dim3(n_rows), dim3(kConfThreads), 0, s, logits, vocab, mask_id, tok, conf);
 }
 
 void build_rope_table(float* out, int max_pos, int dh, float theta) {

@@ -38,6 +38,8 @@ __global__ void __launch_bounds__(kGemmThreads) k_gemm_mma(const bf16* __restric
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int wm = warp >> 2, wn = warp & 3;
   const int nk = (K + BK - 1) / BK;
+  pdl_wait();
+  pdl_trigger();
 
   auto load_stage = [&](int stage, int kt) {
     bf16* sA = smem + stage * kStageElems;
@@ -165,10 +167,12 @@ cudaError_t launch_gemm_mma(const bf16* A, int lda, const bf16* W, const bf16* W
   }
   if (mode == 3) {
     dim3 grid((N + 63) / 64, (M + BM - 1) / BM);
-    k_gemm_mma<true><<<grid, kGemmThreads, kSmemBytes, s>>>(A, lda, W, W2, C, ldc, M, N, K, mode, row_scale);
+    return launch_pdl(k_gemm_mma<true>, grid, dim3(kGemmThreads), kSmemBytes, s, A, lda, W, W2, C, ldc, M, N, K, mode,
+                      row_scale);
   } else {
     dim3 grid((N + 127) / 128, (M + BM - 1) / BM);
-    k_gemm_mma<false><<<grid, kGemmThreads, kSmemBytes, s>>>(A, lda, W, W2, C, ldc, M, N, K, mode, row_scale);
+    return launch_pdl(k_gemm_mma<false>, grid, dim3(kGemmThreads), kSmemBytes, s, A, lda, W, W2, C, ldc, M, N, K, mode,
+                      row_scale);
   }
   return cudaGetLastError();
 }

@@ -14,6 +14,8 @@
 #include <cuda.h>
 #include <cudaTypedefs.h>
 
+#include <stdlib.h>
+
 #include <mutex>
 #include <unordered_map>
 
@@ -34,6 +36,7 @@ struct GemmParams {
   int tn;            // tokens per tile (UMMA N)
   int n_tiles, m_tiles, splits, kblocks;
   int stages;
+  int ksub;          // 64-wide k sub-blocks per pipeline stage
   int mode;          // 0 bf16 store, 1 fp32 +=, 2 fp32 row-scaled store, 3 SwiGLU, 4 fp32 partial sums only
   int dual;
   void* C;
@@ -138,7 +141,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
   const unsigned smem0 = (smem_u32(smem_dyn) + 1023u) & ~1023u;     // 1024-byte alignment for the swizzle atoms
   const int w_bytes = TILE_N * BK * 2;
   const int x_bytes = p.tn * BK * 2;
-  const int stage_bytes = (p.dual ? 2 : 1) * w_bytes + x_bytes;
+  const int sub_bytes = (p.dual ? 2 : 1) * w_bytes + x_bytes;
+  const int stage_bytes = p.ksub * sub_bytes;
   const unsigned full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[16]);
   const unsigned tfull0 = smem_u32(&bars[32]), tempty0 = smem_u32(&bars[34]);
 
@@ -164,6 +168,9 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const unsigned tmem_base = tmem_base_slot;
   volatile int* abort_flag = &s_abort;
+  // barriers, TMEM and descriptors are set up; operands and outputs belong to earlier kernels of the stream
+  pdl_wait();
+  pdl_trigger();
 
   const int items = p.n_tiles * p.m_tiles * p.splits;
   const int acc_cols = 256;                 // columns per accumulator buffer (dual: gate at +0, up at +128)
@@ -182,11 +189,14 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
         const int kb1 = (int)((long long)p.kblocks * (split + 1) / p.splits);
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(empty0 + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
-          const unsigned sw = smem0 + stage * stage_bytes;
           mbar_expect_tx(full0 + 8 * stage, (unsigned)stage_bytes);
-          tma_load_2d(sw, &map_w, kb * BK, nt * TILE_N, full0 + 8 * stage);
-          if (p.dual) tma_load_2d(sw + w_bytes, &map_w2, kb * BK, nt * TILE_N, full0 + 8 * stage);
-          tma_load_2d(sw + (p.dual ? 2 : 1) * w_bytes, &map_x, kb * BK, mt * p.tn, full0 + 8 * stage);
+          for (int sub = 0; sub < p.ksub; ++sub) {
+            const unsigned sw = smem0 + stage * stage_bytes + sub * sub_bytes;
+            const int k0 = (kb * p.ksub + sub) * BK;       // beyond K the box is filled with zeros
+            tma_load_2d(sw, &map_w, k0, nt * TILE_N, full0 + 8 * stage);
+            if (p.dual) tma_load_2d(sw + w_bytes, &map_w2, k0, nt * TILE_N, full0 + 8 * stage);
+            tma_load_2d(sw + (p.dual ? 2 : 1) * w_bytes, &map_x, k0, mt * p.tn, full0 + 8 * stage);
+          }
           if (++stage == p.stages) { stage = 0; phase ^= 1u; }
         }
       }
@@ -212,14 +222,16 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(full0 + 8 * stage, phase, abort_flag)) { ok = false; break; }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          const unsigned sw = smem0 + stage * stage_bytes;
-          const unsigned long long dw = umma_desc(sw);
-          const unsigned long long dx = umma_desc(sw + (p.dual ? 2 : 1) * w_bytes);
+          for (int sub = 0; sub < p.ksub; ++sub) {
+            const unsigned sw = smem0 + stage * stage_bytes + sub * sub_bytes;
+            const unsigned long long dw = umma_desc(sw);
+            const unsigned long long dx = umma_desc(sw + (p.dual ? 2 : 1) * w_bytes);
 #pragma unroll
-          for (int k = 0; k < BK / 16; ++k) {
-            const unsigned accum = (kb > kb0 || k > 0) ? 1u : 0u;
-            umma_bf16(d_gate, dw + 2 * k, dx + 2 * k, idesc, accum);     // +32 bytes per 16-element K step
-            if (p.dual) umma_bf16(d_up, umma_desc(sw + w_bytes) + 2 * k, dx + 2 * k, idesc, accum);
+            for (int k = 0; k < BK / 16; ++k) {
+              const unsigned accum = (kb > kb0 || sub > 0 || k > 0) ? 1u : 0u;
+              umma_bf16(d_gate, dw + 2 * k, dx + 2 * k, idesc, accum);     // +32 bytes per 16-element K step
+              if (p.dual) umma_bf16(d_up, umma_desc(sw + w_bytes) + 2 * k, dx + 2 * k, idesc, accum);
+            }
           }
           umma_commit(empty0 + 8 * stage);        // the stage is free once these MMAs have read it
           if (++stage == p.stages) { stage = 0; phase ^= 1u; }
@@ -312,6 +324,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
 // Adds the k-split partial sums in split order and applies the epilogue.
 __global__ void k_gemm_finish(const float* __restrict__ partial, int splits, int M, int N, int mode, void* Cv, int ldc,
                               const float* __restrict__ row_scale) {
+  pdl_wait();
+  pdl_trigger();
   const size_t total = (size_t)M * N;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
     const int t = (int)(i / N), n = (int)(i % N);
@@ -404,7 +418,9 @@ cudaError_t launch_gemm_tc(const bf16* A, int lda, const bf16* W, const bf16* W2
   const int dual = mode == 3;
   GemmParams p;
   p.M = M; p.N = N; p.K = K; p.mode = mode; p.dual = dual; p.C = C; p.ldc = ldc; p.row_scale = row_scale;
-  p.kblocks = (K + BK - 1) / BK;
+  p.ksub = 1;
+  if (const char* ev = getenv("BS_GEMM_KSUB")) p.ksub = atoi(ev) == 2 ? 2 : 1;
+  p.kblocks = (K + BK * p.ksub - 1) / (BK * p.ksub);
   p.n_tiles = (N + TILE_N - 1) / TILE_N;
   p.error_flag = g_error_flag;
   // ---- token tile and k split ----
@@ -427,12 +443,17 @@ cudaError_t launch_gemm_tc(const bf16* A, int lda, const bf16* W, const bf16* W2
     while (sp > 1 && (p.kblocks / sp < 4 || (size_t)sp * (size_t)M * N > g_partial_floats)) --sp;
     p.splits = sp < 1 ? 1 : sp;
   }
+  if (const char* ev = getenv("BS_GEMM_SPLITS")) {
+    const int sp = atoi(ev);
+    if (sp >= 1 && sp <= 8 && (sp == 1 || (g_partial && (size_t)sp * (size_t)M * N <= g_partial_floats))) p.splits = sp;
+  }
   if (mode == 4 && (!g_partial || (size_t)p.splits * (size_t)M * N > g_partial_floats)) return cudaErrorInvalidValue;
   if (dual) p.splits = 1;
   p.partial = g_partial;
   if (splits_out) *splits_out = p.splits;
-  const int stage_bytes = (dual ? 2 : 1) * TILE_N * BK * 2 + p.tn * BK * 2;
+  const int stage_bytes = p.ksub * ((dual ? 2 : 1) * TILE_N * BK * 2 + p.tn * BK * 2);
   p.stages = kSmemBudget / stage_bytes;
+  if (const char* ev = getenv("BS_GEMM_STAGES")) { const int st = atoi(ev); if (st >= 2 && st < p.stages) p.stages = st; }
   if (p.stages > 16) p.stages = 16;
   if (p.stages < 2) return cudaSuccess;
 
@@ -444,14 +465,13 @@ cudaError_t launch_gemm_tc(const bf16* A, int lda, const bf16* W, const bf16* W2
   *handled = true;
   const long long items = (long long)p.n_tiles * p.m_tiles * p.splits;
   const int grid = (int)(items < g_num_sms ? items : g_num_sms);
-  k_gemm_tc<<<grid, kThreads, kSmemBudget + 1024, s>>>(mw, mw2, mx, p);
-  cudaError_t r = cudaGetLastError();
+  cudaError_t r = launch_pdl(k_gemm_tc, dim3(grid), dim3(kThreads), (size_t)kSmemBudget + 1024, s, mw, mw2, mx, p);
   if (r != cudaSuccess) return r;
   if (p.splits > 1 && mode != 4) {
     const size_t total = (size_t)M * N;
     const int blocks = (int)((total + 255) / 256 < (size_t)g_num_sms * 8 ? (total + 255) / 256 : (size_t)g_num_sms * 8);
-    k_gemm_finish<<<blocks, 256, 0, s>>>(g_partial, p.splits, M, N, mode, C, ldc, row_scale);
-    r = cudaGetLastError();
+    r = launch_pdl(k_gemm_finish, dim3(blocks), dim3(256), 0, s, (const float*)g_partial, p.splits, M, N, mode, C, ldc,
+                   row_scale);
   }
   return r;
 }

@@ -89,6 +89,8 @@ __device__ void build_index(const DevState& st, int parity, int n, int* smi) {
   block_excl_scan(refresh, &tot_r, smi);
   int tot_kv;
   block_excl_scan(unfinished ? vis : 0, &tot_kv, smi);
+  __shared__ long long sm_max[33];
+  const int max_vis = (int)block_max_ll(unfinished ? vis : 0, sm_max);
   if (i < n) {
     st.cu_q[parity][i] = eq;
     st.lm_base[parity][i] = em;
@@ -105,6 +107,7 @@ __device__ void build_index(const DevState& st, int parity, int n, int* smi) {
     st.hdr[H_UNFINISHED] = tot_u;
     st.hdr[H_STEP_REFRESH] = tot_r;
     st.hdr[H_SUM_KV] = tot_kv;
+    st.hdr[H_MAX_VIS] = max_vis;
     st.hdr[H_PARITY] = parity;
   }
   __syncthreads();
@@ -130,6 +133,8 @@ __global__ void __launch_bounds__(kSchedThreads) k_sched(DevState st) {
   __shared__ long long sml[33];
   __shared__ int s_n, s_head, s_stop;
   __shared__ long long s_w;
+  pdl_wait();
+  pdl_trigger();
   const int i = threadIdx.x;
   const int n0 = st.hdr[H_N_ACTIVE];
   const int L = st.L;
@@ -235,6 +240,8 @@ __global__ void __launch_bounds__(kSchedThreads) k_sched(DevState st) {
 __global__ void __launch_bounds__(kSchedThreads) k_commit_index(DevState st) {
   __shared__ int smi[33];
   __shared__ int s_count;
+  pdl_wait();
+  pdl_trigger();
   const int parity = st.hdr[H_PARITY];
   const int n = st.hdr[H_N_ACTIVE];
   const int lane = threadIdx.x & 31;
@@ -287,6 +294,8 @@ __global__ void __launch_bounds__(kSchedThreads) k_commit_index(DevState st) {
 }
 
 __global__ void k_fill_tokens(DevState st, int parity, int M) {
+  pdl_wait();
+  pdl_trigger();
   const int n = st.hdr[H_N_ACTIVE];
   const int* cu = st.cu_q[parity];
   for (int t = blockIdx.x * blockDim.x + threadIdx.x; t < M; t += gridDim.x * blockDim.x) {
@@ -306,19 +315,16 @@ __global__ void k_fill_tokens(DevState st, int parity, int M) {
 }
 
 cudaError_t launch_sched(const DevState& st, cudaStream_t s) {
-  k_sched<<<1, kSchedThreads, 0, s>>>(st);
-  return cudaGetLastError();
+  return launch_pdl(k_sched, dim3(1), dim3(kSchedThreads), 0, s, st);
 }
 cudaError_t launch_commit_index(const DevState& st, cudaStream_t s) {
-  k_commit_index<<<1, kSchedThreads, 0, s>>>(st);
-  return cudaGetLastError();
+  return launch_pdl(k_commit_index, dim3(1), dim3(kSchedThreads), 0, s, st);
 }
 cudaError_t launch_fill_tokens(const DevState& st, int parity, int M, cudaStream_t s) {
   if (M <= 0) return cudaSuccess;
   const int threads = 256;
   const int blocks = min((M + threads - 1) / threads, 148 * 8);
-  k_fill_tokens<<<blocks, threads, 0, s>>>(st, parity, M);
-  return cudaGetLastError();
+  return launch_pdl(k_fill_tokens, dim3(blocks), dim3(threads), 0, s, st, parity, M);
 }
 
 }  // namespace bs

@@ -22,6 +22,30 @@ SHAPES = {   # d_model, n_q_heads, n_kv_heads, head_dim, d_ffn, vocab
 }
 
 
+def _time_graph(run, reps, iters):
+    """Average device time of one launch: `reps` launches are captured into a CUDA graph and replayed, so the
+    measurement does not depend on how fast the host can issue them."""
+    for i in range(3):
+        run(i)
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            for i in range(reps):
+                run(i)
+    ts = []
+    for _ in range(iters + 1):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        ts.append(e0.elapsed_time(e1) / reps)
+    return float(np.median(ts[1:])) * 1e-3
+
+
 def _time(fn, iters, flush):
     for _ in range(3):
         fn()
@@ -64,19 +88,7 @@ def bench_gemm(args):
                 B.op_gemm(A, Ws[i % copies], mode, W2=None if W2s is None else W2s[i % copies], C_out=Cd,
                           row_scale=rs, scratch=scratch, error_flag=flag)
 
-            for i in range(3):
-                run(i)
-            ts = []
-            for _ in range(args.iters):
-                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                torch.cuda.synchronize()
-                e0.record()
-                for i in range(args.reps):
-                    run(i)
-                e1.record()
-                torch.cuda.synchronize()
-                ts.append(e0.elapsed_time(e1) / args.reps)
-            t = float(np.median(ts)) * 1e-3
+            t = _time_graph(run, args.reps, args.iters)
             fl = 2.0 * M * N * K * nw
             by = 2.0 * (N * K * nw + M * K) + Cd.numel() * Cd.element_size() * (2 if mode == 1 else 1)
             print(f"gemm {name:8s} M={M:6d} N={N:6d} K={K:6d} {t * 1e6:9.1f} us {fl / t / 1e12:8.1f} TFLOP/s "
@@ -84,18 +96,26 @@ def bench_gemm(args):
 
 
 def bench_attention(args):
+    """Back-to-back launches over rotating KV copies (together larger than L2)."""
     d, hq, hkv, dh, ffn, vocab = SHAPES[args.shape]
     rows, vis, nq = args.rows, args.vis, args.nq
     cap = rows * vis
-    kc = torch.randn(cap, hkv, dh, device="cuda").bfloat16()
-    vc = torch.randn(cap, hkv, dh, device="cuda").bfloat16()
+    copies = max(2, -(-(320 << 20) // (cap * hkv * dh * 4)))
+    kcs = [torch.randn(cap, hkv, dh, device="cuda").bfloat16() for _ in range(copies)]
+    vcs = [torch.randn(cap, hkv, dh, device="cuda").bfloat16() for _ in range(copies)]
     M = rows * nq
     qkv = torch.randn(M, (hq + 2 * hkv) * dh, device="cuda").bfloat16()
     cu_q = torch.arange(0, rows + 1, dtype=torch.int32, device="cuda") * nq
     kv_base = torch.arange(0, rows, dtype=torch.int32, device="cuda") * vis
     visd = torch.full((rows,), vis, dtype=torch.int32, device="cuda")
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
-    t = _time(lambda: B.op_attention(qkv, kc, vc, cu_q, kv_base, visd, hq, hkv, dh), args.iters, flush)
+    scratch = torch.empty(16 << 20, dtype=torch.float32, device="cuda")
+    plan = B.attention_plan(cu_q, visd, hq, hkv)
+    out = torch.empty(M, hq * dh, dtype=torch.bfloat16, device="cuda")
+    def run(i):
+        B.op_attention(qkv, kcs[i % copies], vcs[i % copies], cu_q, kv_base, visd, hq, hkv, dh, scratch=scratch,
+                       plan=plan, out=out)
+
+    t = _time_graph(run, args.reps, args.iters)
     by = 2.0 * (2.0 * rows * vis * hkv * dh + 2.0 * M * hq * dh)
     fl = 4.0 * rows * nq * vis * hq * dh
     print(f"attention {args.shape} rows={rows} n_q={nq} vis={vis} {t * 1e6:9.1f} us {fl / t / 1e12:8.1f} TFLOP/s "
@@ -123,6 +143,7 @@ def main():
     a.add_argument("--rows", type=int, default=16)
     a.add_argument("--vis", type=int, default=640)
     a.add_argument("--nq", type=int, default=32)
+    a.add_argument("--reps", type=int, default=16)
     c = sub.add_parser("confidence")
     c.add_argument("--rows", type=int, default=512)
     c.add_argument("--vocab", type=int, default=152064)

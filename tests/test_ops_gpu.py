@@ -159,8 +159,9 @@ ATTN_CASES = [
 ]
 
 
+@pytest.mark.parametrize("split_keys", [False, True])
 @pytest.mark.parametrize("hq,hkv,dh,rows", ATTN_CASES)
-def test_ragged_dual_cache_attention(B, hq, hkv, dh, rows):
+def test_ragged_dual_cache_attention(B, hq, hkv, dh, rows, split_keys):
     rng = np.random.default_rng(hq * 100 + dh)
     cap = sum(v for _, v in rows) + 64
     kc = bf16_round(rng.normal(size=(cap, hkv, dh)))
@@ -177,8 +178,10 @@ def test_ragged_dual_cache_attention(B, hq, hkv, dh, rows):
     cu_q = np.zeros(len(rows) + 1, np.int32)
     cu_q[1:] = np.cumsum([n for n, _ in rows])
     vis = np.array([v for _, v in rows], np.int32)
+    # with scratch, a launch with few work items splits each row's keys over several CTAs and merges the parts
+    scratch = torch.empty(8 << 20, dtype=torch.float32, device="cuda") if split_keys else None
     out = B.op_attention(qkv.cuda(), kc.cuda(), vc.cuda(), torch.from_numpy(cu_q).cuda(),
-                         torch.from_numpy(kv_base).cuda(), torch.from_numpy(vis).cuda(), hq, hkv, dh)
+                         torch.from_numpy(kv_base).cuda(), torch.from_numpy(vis).cuda(), hq, hkv, dh, scratch=scratch)
     got = out.float().cpu().numpy().reshape(M, hq, dh)
     q = qkv.float().numpy()[:, :hq * dh].reshape(M, hq, dh)
     K, V = kc.float().numpy(), vc.float().numpy()
