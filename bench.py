@@ -189,27 +189,31 @@ def run_ours(args):
     torch.cuda.synchronize()
 
     # ---- device-resident arm: requests admitted (copied to HBM) before the clock starts ----
-    engines = []
-    for _ in range(args.steps):
-        e = new_engine()
-        admit_all(e, pinned)
-        e.set_profiling(not args.no_profile)
-        engines.append(e)
-    torch.cuda.synchronize()
-    stream = torch.cuda.current_stream()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    def timed_jobs(profile: bool):
+        engines = []
+        for _ in range(args.steps if not profile else 1):
+            e = new_engine()
+            admit_all(e, pinned)
+            e.set_profiling(profile)
+            engines.append(e)
+        torch.cuda.synchronize()
+        stream = torch.cuda.current_stream()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier(world)
+        torch.cuda.synchronize()
+        ev0.record(stream)
+        for e in engines:
+            serve(e)
+        ev1.record(stream)
+        torch.cuda.synchronize()
+        barrier(world)
+        return engines, ev0.elapsed_time(ev1)
+
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-    barrier(world)
-    torch.cuda.synchronize()
-    ev0.record(stream)
-    for e in engines:
-        serve(e)
-    ev1.record(stream)
-    torch.cuda.synchronize()
-    barrier(world)
-    ms_total = max_over_ranks(ev0.elapsed_time(ev1), world, device)
+    engines, ms_local = timed_jobs(profile=False)
+    ms_total = max_over_ranks(ms_local, world, device)
     clocks = sampler.stop() if rank == 0 else None
     committed = sum(e.stats().committed for e in engines)
     assert committed == target * args.steps, "engine did not commit exactly g_i tokens per request"
@@ -217,15 +221,27 @@ def run_ours(args):
     steps_run = sum(e.stats().steps for e in engines)
     cycles = sum(e.stats().cycles for e in engines)
     sum_active = sum(e.stats().sum_active for e in engines)
-    prof = {}
     for e in engines:
-        for fam, v in e.profile().items():
-            acc = prof.setdefault(fam, dict(ms=0.0, launches=0, flops=0.0, bytes=0.0))
-            for k in acc:
-                acc[k] += v[k]
         e.close()
+    del engines
+    torch.cuda.empty_cache()
     total_committed = sum_over_ranks(float(committed), world, device)
     value = total_committed / (ms_total * 1e-3)
+
+    # ---- one more job with the per-family CUDA-event timers on: the roofline numbers.  The timers add two event
+    # records per kernel family per layer and keep neighbouring kernels from overlapping their launches, so this
+    # job runs a few percent slower than the timed ones; its time is reported beside them.
+    prof, prof_ms_job = {}, None
+    if not args.no_profile:
+        engines, prof_ms_job = timed_jobs(profile=True)
+        for e in engines:
+            for fam, v in e.profile().items():
+                acc = prof.setdefault(fam, dict(ms=0.0, launches=0, flops=0.0, bytes=0.0))
+                for k in acc:
+                    acc[k] += v[k]
+            e.close()
+        del engines
+        torch.cuda.empty_cache()
 
     # ---- end-to-end arm: host buffers in, host buffers out, through the C ABI ----
     e2e_engines = [new_engine() for _ in range(args.steps)]
@@ -241,6 +257,7 @@ def run_ours(args):
     e2e_s = max_over_ranks(time.perf_counter() - t0, world, device)
     for e in e2e_engines:
         e.close()
+    del e2e_engines
     e2e_value = total_committed / e2e_s
 
     if rank != 0:
@@ -263,7 +280,8 @@ def run_ours(args):
     else:
         roof = {"bound": "hbm", "achieved": gemm_by / (gemm_ms * 1e-3) / 1e9, "peak": pk["hbm_gbs"], "unit": "GB/s"}
     roof.update(frac=roof["achieved"] / roof["peak"], traffic=NCU_TRAFFIC_BYTES_PER_LAUNCH, peak_kind=pk_kind,
-                kernel="projection GEMM (all five shapes)", launches=gemm_n,
+                kernel="projection GEMM (all five shapes), from one extra job with per-family timers",
+                profiled_job_ms=prof_ms_job, launches=gemm_n,
                 avg_launch_us=1e3 * gemm_ms / max(gemm_n, 1), share_of_step=gemm_ms / max(prof_ms, 1e-9),
                 tflops=gemm_fl / (gemm_ms * 1e-3) / 1e12, gbs=gemm_by / (gemm_ms * 1e-3) / 1e9)
     families = {f: {"ms": round(v["ms"], 3), "launches": v["launches"],

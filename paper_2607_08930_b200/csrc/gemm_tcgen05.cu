@@ -168,8 +168,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const unsigned tmem_base = tmem_base_slot;
   volatile int* abort_flag = &s_abort;
-  // barriers, TMEM and descriptors are set up; operands and outputs belong to earlier kernels of the stream
-  pdl_wait();
+  // Barriers, TMEM and descriptors are set up.  Each role waits for the previous kernel of the stream only where
+  // it first touches something that kernel may have written.
   pdl_trigger();
 
   const int items = p.n_tiles * p.m_tiles * p.splits;
@@ -181,6 +181,27 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
       int stage = 0;
       unsigned phase = 0;
       bool ok = true;
+      // Weights are constants of the model: the first stages of the first item fetch their weight tiles while
+      // the previous kernel is still running; the token tiles follow once it has completed.
+      int npre = 0;
+      {
+        const int it = blockIdx.x;
+        const int split = it % p.splits;
+        const int nt = (it / p.splits) / p.m_tiles;
+        const int kb0 = (int)((long long)p.kblocks * split / p.splits);
+        const int kb1 = (int)((long long)p.kblocks * (split + 1) / p.splits);
+        npre = min(p.stages, kb1 - kb0);
+        for (int i = 0; i < npre; ++i) {
+          mbar_expect_tx(full0 + 8 * i, (unsigned)stage_bytes);
+          for (int sub = 0; sub < p.ksub; ++sub) {
+            const unsigned sw = smem0 + i * stage_bytes + sub * sub_bytes;
+            const int k0 = ((kb0 + i) * p.ksub + sub) * BK;
+            tma_load_2d(sw, &map_w, k0, nt * TILE_N, full0 + 8 * i);
+            if (p.dual) tma_load_2d(sw + w_bytes, &map_w2, k0, nt * TILE_N, full0 + 8 * i);
+          }
+        }
+      }
+      pdl_wait();
       for (int it = blockIdx.x; it < items && ok; it += gridDim.x) {
         const int split = it % p.splits;
         const int tile = it / p.splits;
@@ -188,13 +209,18 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
         const int kb0 = (int)((long long)p.kblocks * split / p.splits);
         const int kb1 = (int)((long long)p.kblocks * (split + 1) / p.splits);
         for (int kb = kb0; kb < kb1; ++kb) {
-          if (!mbar_wait(empty0 + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
-          mbar_expect_tx(full0 + 8 * stage, (unsigned)stage_bytes);
+          const bool prefetched = it == (int)blockIdx.x && kb - kb0 < npre;
+          if (!prefetched) {
+            if (!mbar_wait(empty0 + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+            mbar_expect_tx(full0 + 8 * stage, (unsigned)stage_bytes);
+          }
           for (int sub = 0; sub < p.ksub; ++sub) {
             const unsigned sw = smem0 + stage * stage_bytes + sub * sub_bytes;
             const int k0 = (kb * p.ksub + sub) * BK;       // beyond K the box is filled with zeros
-            tma_load_2d(sw, &map_w, k0, nt * TILE_N, full0 + 8 * stage);
-            if (p.dual) tma_load_2d(sw + w_bytes, &map_w2, k0, nt * TILE_N, full0 + 8 * stage);
+            if (!prefetched) {
+              tma_load_2d(sw, &map_w, k0, nt * TILE_N, full0 + 8 * stage);
+              if (p.dual) tma_load_2d(sw + w_bytes, &map_w2, k0, nt * TILE_N, full0 + 8 * stage);
+            }
             tma_load_2d(sw + (p.dual ? 2 : 1) * w_bytes, &map_x, k0, mt * p.tn, full0 + 8 * stage);
           }
           if (++stage == p.stages) { stage = 0; phase ^= 1u; }
@@ -243,6 +269,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
     // ------------------------------------------------------------------ epilogue warps
     const int q = warp & 3;                       // TMEM lane quarter this warp may read
     int local = 0;
+    pdl_wait();                                   // the output (and the residual it may add to) is shared state
     for (int it = blockIdx.x; it < items; it += gridDim.x, ++local) {
       const int split = it % p.splits;
       const int tile = it / p.splits;
@@ -418,9 +445,6 @@ cudaError_t launch_gemm_tc(const bf16* A, int lda, const bf16* W, const bf16* W2
   const int dual = mode == 3;
   GemmParams p;
   p.M = M; p.N = N; p.K = K; p.mode = mode; p.dual = dual; p.C = C; p.ldc = ldc; p.row_scale = row_scale;
-  p.ksub = 1;
-  if (const char* ev = getenv("BS_GEMM_KSUB")) p.ksub = atoi(ev) == 2 ? 2 : 1;
-  p.kblocks = (K + BK * p.ksub - 1) / (BK * p.ksub);
   p.n_tiles = (N + TILE_N - 1) / TILE_N;
   p.error_flag = g_error_flag;
   // ---- token tile and k split ----
@@ -428,13 +452,12 @@ cudaError_t launch_gemm_tc(const bf16* A, int lda, const bf16* W, const bf16* W2
   // k split that spreads the weight stream over all SMs when there are fewer weight tiles than SMs.
   // Many tokens (a refresh step): the widest tile, no split.
   const int tn_cap = dual ? 128 : 256;
-  if (M <= 2 * tn_cap) {
-    p.m_tiles = (M + tn_cap - 1) / tn_cap;
-    p.tn = (((M + p.m_tiles - 1) / p.m_tiles) + 15) / 16 * 16;
-  } else {
-    p.tn = tn_cap;
-    p.m_tiles = (M + p.tn - 1) / p.tn;
-  }
+  p.m_tiles = (M + tn_cap - 1) / tn_cap;
+  p.tn = (((M + p.m_tiles - 1) / p.m_tiles) + 15) / 16 * 16;     // tiles of equal width that cover M
+  // narrow token tiles are weight-streaming bound: 128-wide k stages halve the per-stage barrier round trips
+  p.ksub = p.tn <= 64 ? 2 : 1;
+  if (const char* ev = getenv("BS_GEMM_KSUB")) p.ksub = atoi(ev) == 2 ? 2 : 1;
+  p.kblocks = (K + BK * p.ksub - 1) / (BK * p.ksub);
   p.splits = 1;
   const long long base_items = (long long)p.n_tiles * p.m_tiles;
   if (g_partial && base_items * 4 < (long long)g_num_sms * 3) {
