@@ -1,0 +1,70 @@
+"""Parity at the benchmark's shapes (needs a B200 and ~60 GB of host memory).
+
+* shallow replicas: the Dream-7B- and LLaDA-8B-shaped models cut to 2 layers (every other dimension, the
+  vocabulary included, as in the benchmark), a few requests, full lockstep;
+* full depth: the benchmark workload itself (16 requests, 28 layers) runs on the engine in the launch
+  configuration bench.py times, while the oracle follows ONE sampled request through its block-cycle
+  (requests never interact, so the oracle can compute that request alone); every integer check still covers
+  the whole batch.
+"""
+import numpy as np
+import pytest
+import torch
+
+import bs_inputs
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2607_08930_b200 import build
+    build.build()
+    from paper_2607_08930_b200 import binding
+    return binding
+
+
+def _shallow(B, shape, ps, gs, alphas, starts, seed):
+    from lockstep import Lockstep, lazy_oracle_model
+    wl = bs_inputs.custom_workload(shape, ps, gs, alphas, starts, seed=seed, tau=0.9, max_batch=len(ps))
+    w = bs_inputs.make_weights(shape, 4242, device="cuda")
+    ls = Lockstep(wl, w, None, model=lazy_oracle_model(shape, w))
+    ls.admit(wl.requests)
+    ls.run()
+    ls.check_tokens()
+    assert ls.eng.stats().committed == wl.committed_target()
+    return ls
+
+
+def test_dream_shape_two_layers_full_lockstep(B):
+    ls = _shallow(B, bs_inputs.DREAM_7B.with_layers(2), [150, 97, 64], [64, 64, 32], [3.0, 9.0, 30.0], [0, 1, 0], 11)
+    print("dream-2L:", ls.summary())
+    assert ls.max_logit_err < 2e-2
+
+
+def test_llada_shape_two_layers_full_lockstep(B):
+    ls = _shallow(B, bs_inputs.LLADA_8B.with_layers(2), [120, 40], [64, 40], [4.0, 25.0], [0, 0], 12)
+    print("llada-2L:", ls.summary())
+    assert ls.max_logit_err < 2e-2
+
+
+def test_benchmark_workload_full_depth_sampled_request(B):
+    from lockstep import Lockstep, lazy_oracle_model
+    wl = bs_inputs.workload(2)
+    w = bs_inputs.make_weights(wl.shape, wl.weight_seed, device="cuda")
+    sample = min(wl.requests, key=lambda r: r.p + r.g)          # the shortest row keeps the oracle affordable
+    ls = Lockstep(wl, w, None, track=[sample.req_id], model=lazy_oracle_model(wl.shape, w))
+    ls.admit(wl.requests)
+    ls.evict_refill()
+    steps = 0
+    while True:
+        ls.step()
+        steps += 1
+        done = ls.eng.block_done()
+        tracked_done = ls.ora.by_id[sample.req_id].mask == 0
+        if done or (tracked_done and steps >= 3):
+            break
+    from lockstep import logit_tol
+    print(f"cfg2 full depth, request {sample.req_id} (p={sample.p}, alpha={sample.alpha:.2f}): {ls.summary()} "
+          f"(depth-28 tolerance {logit_tol(28):.3f})")
+    assert ls.rows_checked > 0 and ls.max_logit_err < logit_tol(wl.shape.n_layers)
