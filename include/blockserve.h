@@ -227,7 +227,8 @@ int bs_op_rope_kv_static(void* qkv, const int* tok_pos, const int* tok_kv, void*
 int bs_op_attention_q_tile(int n_q_heads, int n_kv_heads);
 int bs_op_attention(const void* qkv, const void* kcache, const void* vcache, void* out, const int* cu_q,
                     const int* cu_tile, const int* kv_base, const int* vis, int n_rows, int n_tiles,
-                    int M /* packed tokens */, int max_vis /* largest vis[i] */, int n_q_heads, int n_kv_heads,
+                    int M /* packed tokens */, int max_vis /* largest vis[i] */,
+                    int max_nq /* largest number of query tokens of a row; 0 = unknown */, int n_q_heads, int n_kv_heads,
                     int head_dim, float* scratch /* nullable: lets few work items split their keys over CTAs */,
                     size_t scratch_bytes, void* stream);
 

@@ -93,7 +93,7 @@ def lib() -> C.CDLL:
         L.bs_op_rope_kv.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, f, i, vp, vp]
         L.bs_op_rope_kv_static.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, f, i, vp]
         L.bs_op_attention_q_tile.argtypes = [i, i]
-        L.bs_op_attention.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, i, i, vp, C.c_size_t, vp]
+        L.bs_op_attention.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, i, i, i, vp, C.c_size_t, vp]
         L.bs_op_confidence.argtypes = [vp, i, i, i, vp, vp, vp]
         _lib = L
     return _lib
@@ -325,7 +325,8 @@ def attention_plan(cu_q: torch.Tensor, vis: torch.Tensor, hq: int, hkv: int):
     tiles = np.zeros(len(cu), dtype=np.int32)
     tiles[1:] = np.cumsum((cu[1:] - cu[:-1] + qt - 1) // qt)
     return dict(cu_tile=torch.from_numpy(tiles).to(cu_q.device), n_tiles=int(tiles[-1]),
-                max_vis=int(vis.max().item()) if len(vis) else 0)
+                max_vis=int(vis.max().item()) if len(vis) else 0,
+                max_nq=int((cu[1:] - cu[:-1]).max()) if len(cu) > 1 else 0)
 
 
 def op_attention(qkv, kcache, vcache, cu_q, kv_base, vis, hq, hkv, dh, scratch: Optional[torch.Tensor] = None,
@@ -335,7 +336,7 @@ def op_attention(qkv, kcache, vcache, cu_q, kv_base, vis, hq, hkv, dh, scratch: 
         out = torch.empty(qkv.shape[0], hq * dh, dtype=torch.bfloat16, device=qkv.device)
     _check_op(lib().bs_op_attention(qkv.data_ptr(), kcache.data_ptr(), vcache.data_ptr(), out.data_ptr(),
                                     cu_q.data_ptr(), plan["cu_tile"].data_ptr(), kv_base.data_ptr(), vis.data_ptr(),
-                                    len(cu_q) - 1, plan["n_tiles"], qkv.shape[0], plan["max_vis"],
+                                    len(cu_q) - 1, plan["n_tiles"], qkv.shape[0], plan["max_vis"], plan["max_nq"],
                                     hq, hkv, dh, _ptr(scratch),
                                     0 if scratch is None else scratch.numel() * scratch.element_size(),
                                     _stream()), "bs_op_attention")

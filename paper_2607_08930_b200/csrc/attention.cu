@@ -281,6 +281,9 @@ __global__ void __launch_bounds__(256) k_attention_combine(AttnPartial part, bf1
 
 int attention_q_tile(int hq, int hkv) {
   const int G = hq / hkv;
+  if (G == 1) {
+    if (const char* ev = getenv("BS_ATTN_QT")) return atoi(ev);
+  }
   return G >= 5 ? 16 : (G == 1 ? 64 : 32);
 }
 
@@ -302,12 +305,16 @@ cudaError_t launch_variant(dim3 grid, int threads, cudaStream_t s, const bf16* q
 
 cudaError_t launch_attention(const bf16* qkv, const bf16* kc, const bf16* vc, bf16* out, const int* cu_q,
                              const int* cu_tile, const int* kv_base, const int* vis, int n_rows, int n_tiles, int M,
-                             int max_vis, int hq, int hkv, int dh, float* scratch, size_t scratch_floats,
-                             cudaStream_t s) {
+                             int max_vis, int max_nq, int hq, int hkv, int dh, float* scratch,
+                             size_t scratch_floats, cudaStream_t s) {
   if (n_tiles <= 0 || n_rows <= 0) return cudaSuccess;
   const int G = hq / hkv;
   const int qt = attention_q_tile(hq, hkv);
-  const int threads = qt * G * 2;             // 16 flattened rows per warp
+  // 16 flattened (token, head) rows per warp; a block step has at most L <= 32 query tokens per row, so a
+  // 64-token q-tile (MHA) needs only the warps that hold tokens
+  int qt_used = qt;
+  if (max_nq > 0 && max_nq < qt) qt_used = (max_nq + 15) / 16 * 16;
+  const int threads = ((qt_used * G + 15) / 16) * 32;
   if (threads > 256 || (dh != 64 && dh != 128) || hq % hkv != 0) return cudaErrorInvalidValue;
   // KV chunks: a block step has few (row, kv head, q tile) items, each a long serial walk over the row's keys;
   // splitting the walk fills the SMs.  A refresh step has plenty of items already.

@@ -76,7 +76,7 @@ cudaError_t launch_rope_kv(bf16* qkv, const int* tok_pos, const int* tok_kv, bf1
 // scratch (nullable): fp32 partial results when the keys of a work item are split over several CTAs.
 cudaError_t launch_attention(const bf16* qkv, const bf16* kc, const bf16* vc, bf16* out, const int* cu_q,
                              const int* cu_tile, const int* kv_base, const int* vis, int n_rows, int n_tiles, int M,
-                             int max_vis, int hq, int hkv, int dh, float* scratch, size_t scratch_floats,
+                             int max_vis, int max_nq, int hq, int hkv, int dh, float* scratch, size_t scratch_floats,
                              cudaStream_t s);
 cudaError_t launch_confidence(const float* logits, int n_rows, int vocab, int mask_id, int* tok, float* conf,
                               cudaStream_t s);

@@ -410,6 +410,7 @@ int bs_denoise_step(bs_engine* e, int* n_committed) {
   // A block step (few packed tokens) runs the projections that feed a row-wise operator as k-split partial sums
   // and lets one finishing kernel per projection add them and apply that operator (RoPE + KV scatter after QKV,
   // residual + the next RMSNorm after O and down).  A refresh step (many tokens) uses the direct epilogues.
+  const int max_nq = e->hdr[H_STEP_REFRESH] > 0 ? 0 : c.block_len;    // 0: rows may bring their whole span
   const bool small = M <= kSmallStepTokens && (size_t)M * (size_t)std::max(qkv_n, d) <= kPartialFloats;
   if (small) {
     prof_mark(e, BS_FAM_EMBED_NORM);
@@ -427,8 +428,8 @@ int bs_denoise_step(bs_engine* e, int* n_committed) {
       prof_work(e, BS_FAM_ROPE_KV, 1, 0, 4.0 * sp * dM * dq + 2.0 * dM * dq);
       prof_mark(e, BS_FAM_ATTENTION);
       KL(e, launch_attention(ws.qkv, kc, vc, ws.attn, st.cu_q[parity], st.cu_tile[parity], st.row_kv_base,
-                             st.row_vis, n_rows, e->hdr[H_QTILES], M, e->hdr[H_MAX_VIS], hq, hkv, dh, ws.partial,
-                             kPartialFloats, s));
+                             st.row_vis, n_rows, e->hdr[H_QTILES], M, e->hdr[H_MAX_VIS], max_nq, hq, hkv, dh,
+                             ws.partial, kPartialFloats, s));
       prof_work(e, BS_FAM_ATTENTION, 1, 0, 2.0 * (2.0 * kv_rows * hkv * dh + 2.0 * dM * dhq));
       prof_mark(e, BS_FAM_GEMM_O);
       KL(e, launch_gemm_partial(ws.attn, hq * dh, e->wo[l], M, d, hq * dh, e->gemm_scratch, s, &sp));
@@ -463,7 +464,7 @@ int bs_denoise_step(bs_engine* e, int* n_committed) {
     prof_work(e, BS_FAM_ROPE_KV, 1, 0, 2.0 * dM * (dq + (double)(hq + 2 * hkv) * dh));
     prof_mark(e, BS_FAM_ATTENTION);
     KL(e, launch_attention(ws.qkv, kc, vc, ws.attn, st.cu_q[parity], st.cu_tile[parity], st.row_kv_base, st.row_vis,
-                           n_rows, e->hdr[H_QTILES], M, e->hdr[H_MAX_VIS], hq, hkv, dh, nullptr, 0, s));
+                           n_rows, e->hdr[H_QTILES], M, e->hdr[H_MAX_VIS], max_nq, hq, hkv, dh, nullptr, 0, s));
     // every query token of a row meets every cache row of that row: flops = 4 * dh * Hq * sum_rows(n_q * vis);
     // the host knows the sums only for pure block steps and pure refresh steps, else it reports bytes alone
     prof_work(e, BS_FAM_ATTENTION, 1, 0, 2.0 * (2.0 * kv_rows * hkv * dh + 2.0 * dM * dhq));
@@ -694,11 +695,11 @@ int bs_op_attention_q_tile(int n_q_heads, int n_kv_heads) {
 
 int bs_op_attention(const void* qkv, const void* kcache, const void* vcache, void* out, const int* cu_q,
                     const int* cu_tile, const int* kv_base, const int* vis, int n_rows, int n_tiles, int M,
-                    int max_vis, int n_q_heads, int n_kv_heads, int head_dim, float* scratch, size_t scratch_bytes,
-                    void* stream) {
+                    int max_vis, int max_nq, int n_q_heads, int n_kv_heads, int head_dim, float* scratch,
+                    size_t scratch_bytes, void* stream) {
   if (!qkv || !kcache || !vcache || !out || !cu_q || !cu_tile || !kv_base || !vis) return BS_E_ARG;
   return launch_attention((const bf16*)qkv, (const bf16*)kcache, (const bf16*)vcache, (bf16*)out, cu_q, cu_tile,
-                          kv_base, vis, n_rows, n_tiles, M, max_vis, n_q_heads, n_kv_heads, head_dim, scratch,
+                          kv_base, vis, n_rows, n_tiles, M, max_vis, max_nq, n_q_heads, n_kv_heads, head_dim, scratch,
                           scratch ? scratch_bytes / sizeof(float) : 0, (cudaStream_t)stream) == cudaSuccess
              ? BS_OK : BS_E_CUDA;
 }
