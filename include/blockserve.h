@@ -223,14 +223,17 @@ int bs_op_rope_kv_static(void* qkv, const int* tok_pos, const int* tok_kv, void*
  * row i owns packed tokens [cu_q[i], cu_q[i+1]) and attends over cache rows
  * [kv_base[i], kv_base[i] + vis[i]) (prefix, fresh block and suffix alike; no causal or padding mask).
  * q: the qkv buffer of bs_op_rope_kv; out bf16 [M, Hq*dh].  Work items are q-tiles of
- * bs_op_attention_q_tile(Hq, Hkv) tokens: cu_tile[i] = sum_{r<i} ceil(n_q(r) / q_tile), n_tiles = cu_tile[n_rows]. */
-int bs_op_attention_q_tile(int n_q_heads, int n_kv_heads);
+ * bs_op_attention_q_tile(Hq, Hkv, dh) tokens: cu_tile[i] = sum_{r<i} ceil(n_q(r) / q_tile), n_tiles = cu_tile[n_rows]. */
+int bs_op_attention_q_tile(int n_q_heads, int n_kv_heads, int head_dim);
 int bs_op_attention(const void* qkv, const void* kcache, const void* vcache, void* out, const int* cu_q,
                     const int* cu_tile, const int* kv_base, const int* vis, int n_rows, int n_tiles,
                     int M /* packed tokens */, int max_vis /* largest vis[i] */,
-                    int max_nq /* largest number of query tokens of a row; 0 = unknown */, int n_q_heads, int n_kv_heads,
-                    int head_dim, float* scratch /* nullable: lets few work items split their keys over CTAs */,
-                    size_t scratch_bytes, void* stream);
+                    int max_nq /* largest number of query tokens of a row; 0 = unknown */,
+                    long long kv_rows /* rows of kcache / vcache; every value in them must be finite */,
+                    int n_q_heads, int n_kv_heads, int head_dim,
+                    float* scratch /* nullable: lets few work items split their keys over CTAs */,
+                    size_t scratch_bytes, int* error_flag /* nullable device int, set on a wait timeout */,
+                    void* stream);
 
 /* Per row of fp32 logits [n_rows, vocab]: mask id excluded, tok = argmax (lowest id on ties),
  * conf = exp(max - logsumexp). */

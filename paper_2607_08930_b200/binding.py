@@ -92,8 +92,8 @@ def lib() -> C.CDLL:
         L.bs_op_rmsnorm.argtypes = [vp, vp, vp, vp, i, i, f, vp]
         L.bs_op_rope_kv.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, f, i, vp, vp]
         L.bs_op_rope_kv_static.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, f, i, vp]
-        L.bs_op_attention_q_tile.argtypes = [i, i]
-        L.bs_op_attention.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, i, i, i, vp, C.c_size_t, vp]
+        L.bs_op_attention_q_tile.argtypes = [i, i, i]
+        L.bs_op_attention.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, ll, i, i, i, vp, C.c_size_t, vp, vp]
         L.bs_op_confidence.argtypes = [vp, i, i, i, vp, vp, vp]
         _lib = L
     return _lib
@@ -317,10 +317,10 @@ def op_rope_kv_static(qkv, tok_pos, tok_kv, kcache, vcache, hq, hkv, dh, theta, 
                                       vcache.data_ptr(), qkv.shape[0], hq, hkv, dh, theta, max_pos, _stream())
 
 
-def attention_plan(cu_q: torch.Tensor, vis: torch.Tensor, hq: int, hkv: int):
+def attention_plan(cu_q: torch.Tensor, vis: torch.Tensor, hq: int, hkv: int, dh: int = 128):
     """Work-item prefix over rows (q-tiles) and the launch scalars of bs_op_attention; involves a device-to-host
     copy, so callers that launch repeatedly build it once."""
-    qt = lib().bs_op_attention_q_tile(hq, hkv)
+    qt = lib().bs_op_attention_q_tile(hq, hkv, dh)
     cu = cu_q.detach().cpu().numpy().astype(np.int64)
     tiles = np.zeros(len(cu), dtype=np.int32)
     tiles[1:] = np.cumsum((cu[1:] - cu[:-1] + qt - 1) // qt)
@@ -331,15 +331,15 @@ def attention_plan(cu_q: torch.Tensor, vis: torch.Tensor, hq: int, hkv: int):
 
 def op_attention(qkv, kcache, vcache, cu_q, kv_base, vis, hq, hkv, dh, scratch: Optional[torch.Tensor] = None,
                  plan=None, out: Optional[torch.Tensor] = None) -> torch.Tensor:
-    plan = plan or attention_plan(cu_q, vis, hq, hkv)
+    plan = plan or attention_plan(cu_q, vis, hq, hkv, dh)
     if out is None:
         out = torch.empty(qkv.shape[0], hq * dh, dtype=torch.bfloat16, device=qkv.device)
     _check_op(lib().bs_op_attention(qkv.data_ptr(), kcache.data_ptr(), vcache.data_ptr(), out.data_ptr(),
                                     cu_q.data_ptr(), plan["cu_tile"].data_ptr(), kv_base.data_ptr(), vis.data_ptr(),
                                     len(cu_q) - 1, plan["n_tiles"], qkv.shape[0], plan["max_vis"], plan["max_nq"],
-                                    hq, hkv, dh, _ptr(scratch),
+                                    kcache.shape[0], hq, hkv, dh, _ptr(scratch),
                                     0 if scratch is None else scratch.numel() * scratch.element_size(),
-                                    _stream()), "bs_op_attention")
+                                    None, _stream()), "bs_op_attention")
     return out
 
 

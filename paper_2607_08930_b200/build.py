@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libblockserve.so")
-SOURCES = ["engine.cu", "sched_index.cu", "elementwise.cu", "gemm_mma.cu", "gemm_tcgen05.cu", "attention.cu", "rope_static.cu"]
+SOURCES = ["engine.cu", "sched_index.cu", "elementwise.cu", "gemm_mma.cu", "gemm_tcgen05.cu", "attention.cu", "attention_tc.cu", "rope_static.cu"]
 NVCC_FLAGS = ["-std=c++17", "-O3", "-lineinfo", "-gencode", "arch=compute_100a,code=sm_100a",
               "-Xcompiler", "-fPIC", "--use_fast_math" if False else "-Xptxas", "-v"]
 

@@ -279,12 +279,22 @@ __global__ void __launch_bounds__(256) k_attention_combine(AttnPartial part, bf1
 }
 }  // namespace
 
-int attention_q_tile(int hq, int hkv) {
+int attention_tc_q_tile(int hq, int hkv);
+cudaError_t launch_attention_tc(const bf16* qkv, const bf16* kc, const bf16* vc, bf16* out, const int* cu_q,
+                                const int* cu_tile, const int* kv_base, const int* vis, int n_rows, int n_tiles,
+                                int M, long long kv_rows, int max_nq, int hq, int hkv, int dh, int* error_flag,
+                                cudaStream_t s, bool* handled);
+
+static bool use_tc_attention(int hq, int hkv, int dh) {
+  static const bool legacy = getenv("BS_ATTN_LEGACY") != nullptr;
+  return !legacy && dh == 128 && hkv > 0 && hq % hkv == 0 && hq / hkv <= 8;
+}
+
+// Query tokens per attention work item; the index kernels build their work-item prefix with it.
+int attention_q_tile(int hq, int hkv, int dh) {
+  if (use_tc_attention(hq, hkv, dh)) return attention_tc_q_tile(hq, hkv);
   const int G = hq / hkv;
-  if (G == 1) {
-    if (const char* ev = getenv("BS_ATTN_QT")) return atoi(ev);
-  }
-  return G >= 5 ? 16 : (G == 1 ? 64 : 32);
+  return G >= 5 ? 16 : (G == 1 ? 64 : 32);     // the legacy kernel's tile
 }
 
 namespace {
@@ -305,11 +315,21 @@ cudaError_t launch_variant(dim3 grid, int threads, cudaStream_t s, const bf16* q
 
 cudaError_t launch_attention(const bf16* qkv, const bf16* kc, const bf16* vc, bf16* out, const int* cu_q,
                              const int* cu_tile, const int* kv_base, const int* vis, int n_rows, int n_tiles, int M,
-                             int max_vis, int max_nq, int hq, int hkv, int dh, float* scratch,
-                             size_t scratch_floats, cudaStream_t s) {
+                             int max_vis, int max_nq, long long kv_rows, int hq, int hkv, int dh, float* scratch,
+                             size_t scratch_floats, int* error_flag, cudaStream_t s) {
   if (n_tiles <= 0 || n_rows <= 0) return cudaSuccess;
+  // Block steps of a model with one or two query heads per kv head are pure cache streaming with a few dozen
+  // query rows: several small CTAs per SM hide the load latency better than one tensor-core CTA.  Every row has
+  // at most one work item there, so the work-item prefix is the same for either kernel's q-tile.
+  const bool stream_small = max_nq > 0 && max_nq <= 32 && hq / hkv <= 2;
+  if (use_tc_attention(hq, hkv, dh) && !stream_small) {
+    bool handled = false;
+    cudaError_t r = launch_attention_tc(qkv, kc, vc, out, cu_q, cu_tile, kv_base, vis, n_rows, n_tiles, M, kv_rows,
+                                        max_nq, hq, hkv, dh, error_flag, s, &handled);
+    return handled ? r : cudaErrorNotSupported;     // the work-item prefix was built for this kernel's q-tile
+  }
   const int G = hq / hkv;
-  const int qt = attention_q_tile(hq, hkv);
+  const int qt = G >= 5 ? 16 : (G == 1 ? 64 : 32);
   // 16 flattened (token, head) rows per warp; a block step has at most L <= 32 query tokens per row, so a
   // 64-token q-tile (MHA) needs only the warps that hold tokens
   int qt_used = qt;

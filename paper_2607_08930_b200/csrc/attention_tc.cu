@@ -1,0 +1,520 @@
+// Ragged bidirectional attention against the dual KV cache on the 5th-generation tensor cores (head_dim 128).
+//
+// Work item = (row i, a span of the row's packed tokens, kv head).  Its query rows are the flattened
+// (token, head-in-group) pairs, so all query heads of a kv head share each K/V tile; they form up to two Q tiles of
+// at most 128 rows (one UMMA M tile each), and both Q tiles use every K/V tile the CTA loads.
+// Keys are the row's cache span [kv_base_i, kv_base_i + vis_i) - prefix, fresh block and suffix alike; no causal
+// or padding mask.  One CTA per SM, warp-specialised:
+//   warp 0      TMA producer: the Q tiles once (3-D boxes: 64 dims x group heads x tokens), then 64-key K and V
+//               tiles (3-D boxes over the cache [row][kv head][dim]) through a four-stage ring
+//   warp 1      MMA issuer: per Q tile S = Q K^T into one of two TMEM buffers (the next key tile's scores are
+//               computed while this tile's softmax runs), then O += P V with P read from shared memory and V as an
+//               MN-major operand straight from the cache layout
+//   warps 2..9  softmax, four warps per Q tile: thread r owns query row r (TMEM lane r), so row maxima and sums
+//               need no shuffles; p = 2^(s - m) goes to shared memory as bf16 in the 128B-swizzled K-major layout;
+//               the output accumulates in TMEM over all key tiles and is rescaled lazily (only when a row's
+//               maximum has grown by more than 2^8), the running sum follows the same scale
+// Every wait is bounded; on a timeout the flag is raised, all roles drain, TMEM is freed.
+#include <cuda.h>
+#include <cudaTypedefs.h>
+#include <math.h>
+#include <stdlib.h>
+
+#include <mutex>
+#include <unordered_map>
+
+#include "common.cuh"
+
+namespace bs {
+
+namespace {
+
+constexpr int DH = 128;
+constexpr int kThreads = 320;             // producer warp, MMA warp, 8 softmax warps
+constexpr int kHalfBytes = 128 * 128;      // 128 rows x 64 bf16: one swizzled sub-tile of Q or P
+constexpr int kQBytes = 2 * kHalfBytes;
+constexpr long long kWaitCycles = 4000000000ll;
+
+__device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(unsigned bar, unsigned count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(unsigned bar, unsigned bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(unsigned bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity) {
+  unsigned ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity, volatile int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity)) {
+    if (*abort_flag) return false;
+    if (clock64() - t0 > kWaitCycles) {
+      *abort_flag = 1;
+      return false;
+    }
+  }
+  return true;
+}
+__device__ __forceinline__ void tma_load_3d(unsigned dst, const CUtensorMap* map, int c0, int c1, int c2, unsigned bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar) : "memory");
+}
+// 128B-swizzled operand tile with rows of 128 bytes; 8-row groups are 1024 bytes apart (K-major and MN-major alike).
+__device__ __forceinline__ unsigned long long umma_desc(unsigned smem_addr) {
+  unsigned long long d = 0;
+  d |= (unsigned long long)((smem_addr & 0x3FFFF) >> 4);
+  d |= (unsigned long long)1 << 16;
+  d |= (unsigned long long)(1024 >> 4) << 32;
+  d |= (unsigned long long)1 << 46;
+  d |= (unsigned long long)2 << 61;
+  return d;
+}
+// fp32 accumulator, bf16 operands, A K-major, M = 128; B K-major (scores) or MN-major (values).
+__device__ __forceinline__ unsigned umma_idesc(int n, bool b_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn_major ? (1u << 16) : 0u) | ((unsigned)(n >> 3) << 17) |
+         ((128u >> 4) << 24);
+}
+__device__ __forceinline__ void umma_bf16(unsigned d_tmem, unsigned long long a, unsigned long long b, unsigned idesc,
+                                          unsigned accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(unsigned bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(unsigned taddr, float* v) {
+  unsigned r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+__device__ __forceinline__ void tmem_st32(unsigned taddr, const float* v) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])),
+        "r"(__float_as_uint(v[3])), "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])),
+        "r"(__float_as_uint(v[7])), "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])),
+        "r"(__float_as_uint(v[11])), "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])),
+        "r"(__float_as_uint(v[14])), "r"(__float_as_uint(v[15])), "r"(__float_as_uint(v[16])),
+        "r"(__float_as_uint(v[17])), "r"(__float_as_uint(v[18])), "r"(__float_as_uint(v[19])),
+        "r"(__float_as_uint(v[20])), "r"(__float_as_uint(v[21])), "r"(__float_as_uint(v[22])),
+        "r"(__float_as_uint(v[23])), "r"(__float_as_uint(v[24])), "r"(__float_as_uint(v[25])),
+        "r"(__float_as_uint(v[26])), "r"(__float_as_uint(v[27])), "r"(__float_as_uint(v[28])),
+        "r"(__float_as_uint(v[29])), "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31]))
+      : "memory");
+  asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// A row's output accumulator is rescaled only when its running maximum has grown by more than this (log2
+// units); until then probabilities are formed against the older maximum and stay below 2^kLazy.
+constexpr float kLazy = 8.0f;
+
+struct AttnTcParams {
+  const int* cu_q;
+  const int* cu_tile;
+  const int* kv_base;
+  const int* vis;
+  bf16* out;
+  int n_rows, hq, hkv;
+  int tq;            // tokens per Q tile (a work item holds two Q tiles)
+  int split;         // 1: one CTA per Q tile (few work items: more, shorter chains), 0: one CTA per work item
+  int* error_flag;
+};
+
+constexpr int KT = 64;                                   // keys per tile
+constexpr int kStages = 4;
+constexpr int kKvHalf = KT * 128;                        // KT rows x 64 bf16
+constexpr int kStageBytes = 4 * kKvHalf;                 // K halves, V halves
+constexpr int kPBytes = kHalfBytes;                      // 128 rows x 64 keys, per Q tile
+constexpr int kSmemBytes = 2 * kQBytes + kStages * kStageBytes + 2 * kPBytes + 1024;
+
+// Barrier slots
+enum { B_QFULL = 0, B_KVFULL = 1, B_KVEMPTY = B_KVFULL + kStages, B_SFULL = B_KVEMPTY + kStages,   // [tile][2]
+       B_SEMPTY = B_SFULL + 4, B_PFULL = B_SEMPTY + 4, B_OFULL = B_PFULL + 2, B_COUNT = B_OFULL + 2 };
+
+__global__ void __launch_bounds__(kThreads, 1)
+k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+               const __grid_constant__ CUtensorMap map_v, const AttnTcParams p) {
+  extern __shared__ unsigned char smem_dyn[];
+  __shared__ __align__(8) unsigned long long bars[B_COUNT];
+  __shared__ unsigned tmem_base_slot;
+  __shared__ int s_abort;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const unsigned smem0 = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+  const unsigned sQ = smem0;                              // [Q tile][dim half][128 rows x 128 B]
+  const unsigned sKV = sQ + 2 * kQBytes;
+  const unsigned sP = sKV + kStages * kStageBytes;        // [Q tile][128 rows x 128 B]
+  const unsigned bar0 = smem_u32(&bars[0]);
+  auto bar = [&](int i) { return bar0 + 8u * (unsigned)i; };
+
+  if (threadIdx.x == 0) {
+    s_abort = 0;
+    mbar_init(bar(B_QFULL), 1);
+    for (int i = 0; i < kStages; ++i) {
+      mbar_init(bar(B_KVFULL + i), 1);
+      mbar_init(bar(B_KVEMPTY + i), 1);
+    }
+    for (int i = 0; i < 4; ++i) {
+      mbar_init(bar(B_SFULL + i), 1);
+      mbar_init(bar(B_SEMPTY + i), 4);     // one arrival per softmax warp of the Q tile
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bar(B_PFULL + i), 4);
+      mbar_init(bar(B_OFULL + i), 1);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&tmem_base_slot))
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const unsigned tmem_base = tmem_base_slot;
+  volatile int* abort_flag = &s_abort;
+  pdl_trigger();
+  pdl_wait();       // indices, q and the cache rows of this step come from earlier kernels of the stream
+
+  // ---- which row owns this work item: largest r with cu_tile[r] <= blockIdx.x ----
+  const int G = p.hq / p.hkv;
+  const int kh = blockIdx.y;
+  int lo = 0, hi = p.n_rows;
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (p.cu_tile[mid] <= (p.split ? (int)blockIdx.x >> 1 : (int)blockIdx.x)) lo = mid; else hi = mid;
+  }
+  const int row = lo;
+  const int item = p.split ? (int)blockIdx.x >> 1 : (int)blockIdx.x;
+  const int per_cta = p.split ? p.tq : 2 * p.tq;
+  const int t0 = p.cu_q[row] + (item - p.cu_tile[row]) * 2 * p.tq + (p.split ? ((int)blockIdx.x & 1) * p.tq : 0);
+  const int nt = min(per_cta, p.cu_q[row + 1] - t0);        // query tokens of this CTA (CTA-uniform)
+  const int n_qt = nt <= 0 ? 0 : (nt > p.tq ? 2 : 1);       // Q tiles in use
+  const int vis = p.vis[row];
+  const int kvb = p.kv_base[row];
+  const int n_tiles = nt > 0 ? (vis + KT - 1) / KT : 0;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0 && n_tiles > 0) {
+      mbar_expect_tx(bar(B_QFULL), (unsigned)(n_qt * 2 * p.tq * G * 128));
+      for (int x = 0; x < n_qt; ++x) {
+        tma_load_3d(sQ + x * kQBytes, &map_q, 0, kh * G, t0 + x * p.tq, bar(B_QFULL));
+        tma_load_3d(sQ + x * kQBytes + kHalfBytes, &map_q, 64, kh * G, t0 + x * p.tq, bar(B_QFULL));
+      }
+      for (int t = 0; t < n_tiles; ++t) {
+        const int s = t % kStages;
+        if (!mbar_wait(bar(B_KVEMPTY + s), (unsigned)((t / kStages) & 1) ^ 1u, abort_flag)) break;
+        const unsigned st = sKV + s * kStageBytes;
+        mbar_expect_tx(bar(B_KVFULL + s), (unsigned)kStageBytes);
+        const int key0 = kvb + t * KT;
+        tma_load_3d(st, &map_k, 0, kh, key0, bar(B_KVFULL + s));
+        tma_load_3d(st + kKvHalf, &map_k, 64, kh, key0, bar(B_KVFULL + s));
+        tma_load_3d(st + 2 * kKvHalf, &map_v, 0, kh, key0, bar(B_KVFULL + s));
+        tma_load_3d(st + 3 * kKvHalf, &map_v, 64, kh, key0, bar(B_KVFULL + s));
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0 && n_tiles > 0) {
+      const unsigned idesc_s = umma_idesc(KT, false);
+      const unsigned idesc_o = umma_idesc(64, true);
+      bool ok = mbar_wait(bar(B_QFULL), 0, abort_flag);
+      // S = Q K^T of key tile t for every Q tile in use, into the S buffer of parity t
+      auto issue_scores = [&](int t) -> bool {
+        const int s = t % kStages, b = t & 1;
+        if (!mbar_wait(bar(B_KVFULL + s), (unsigned)(t / kStages) & 1u, abort_flag)) return false;
+        const unsigned st = sKV + s * kStageBytes;
+        for (int x = 0; x < n_qt; ++x) {
+          if (!mbar_wait(bar(B_SEMPTY + 2 * x + b), ((unsigned)(t >> 1) & 1u) ^ 1u, abort_flag)) return false;
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll
+          for (int h = 0; h < 2; ++h)
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+              umma_bf16(tmem_base + x * 256 + b * 64, umma_desc(sQ + x * kQBytes + h * kHalfBytes) + 2 * k,
+                        umma_desc(st + h * kKvHalf) + 2 * k, idesc_s, (h | k) ? 1u : 0u);
+          umma_commit(bar(B_SFULL + 2 * x + b));
+        }
+        return true;
+      };
+      if (ok) ok = issue_scores(0);
+      for (int t = 0; t < n_tiles && ok; ++t) {
+        if (t + 1 < n_tiles) ok = issue_scores(t + 1);      // next tile's scores run under this tile's softmax
+        if (!ok) break;
+        const unsigned st = sKV + (t % kStages) * kStageBytes;
+        for (int x = 0; x < n_qt && ok; ++x) {
+          if (!mbar_wait(bar(B_PFULL + x), (unsigned)t & 1u, abort_flag)) { ok = false; break; }
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll
+          for (int j = 0; j < KT / 16; ++j) {       // 16 keys per step
+            const unsigned long long da = umma_desc(sP + x * kPBytes) + 2 * j;
+#pragma unroll
+            for (int h = 0; h < 2; ++h)             // two 64-wide halves of the head dimension
+              umma_bf16(tmem_base + x * 256 + 128 + h * 64, da, umma_desc(st + (2 + h) * kKvHalf + j * 2048), idesc_o,
+                        (t | j) ? 1u : 0u);         // the output accumulates in TMEM over all key tiles
+          }
+          umma_commit(bar(B_OFULL + x));
+        }
+        if (ok) umma_commit(bar(B_KVEMPTY + (t % kStages)));
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ softmax warps: one query row per thread
+    // warps 2..5 own Q tile 0, warps 6..9 own Q tile 1; within a Q tile, warp w reads TMEM lanes 32 (w % 4) ..
+    const int x = (warp - 2) >> 2;
+    const int q = warp & 3;
+    const int r = q * 32 + lane;                        // query row of the Q tile = TMEM lane
+    const int nrows = (x == 0 ? min(nt, p.tq) : nt - p.tq) * G;      // valid rows of this Q tile
+    if (x < n_qt) {
+      const unsigned t_lane = tmem_base + ((unsigned)(q * 32) << 16) + x * 256;
+      const unsigned t_out = t_lane + 128;
+      const unsigned sPx = sP + x * kPBytes + r * 128;
+      const float sc = 1.4426950408889634f * rsqrtf((float)DH);
+      const bool warp_has_rows = q * 32 < nrows;        // warps without valid rows only keep the barriers moving
+      float m = -INFINITY, l = 0.f;                     // m: the maximum the accumulator is currently scaled by
+      bool ok = true;
+      for (int t = 0; t < n_tiles && ok; ++t) {
+        const int b = t & 1;
+        if (!mbar_wait(bar(B_SFULL + 2 * x + b), (unsigned)(t >> 1) & 1u, abort_flag)) { ok = false; break; }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        float v[KT];
+        float f = 1.0f;
+        bool rescale = false;
+        if (warp_has_rows) {
+          // scores -> probabilities in registers; this part overlaps the previous tile's P V product
+          const int key0 = t * KT;
+          tmem_ld32(t_lane + b * 64, v);
+          tmem_ld32(t_lane + b * 64 + 32, v + 32);
+          float mx = -INFINITY;
+#pragma unroll
+          for (int j = 0; j < KT; ++j) {
+            v[j] = (key0 + j < vis) ? v[j] * sc : -INFINITY;
+            mx = fmaxf(mx, v[j]);                       // finite: every tile holds a valid key
+          }
+          // lazy rescale (warp-uniform decision: TMEM loads and stores are warp-wide)
+          const bool grow = mx > m + kLazy;             // always true on the first tile (m = -inf)
+          rescale = __any_sync(0xffffffffu, grow);
+          if (grow) {
+            f = ex2(m - mx);                            // first tile: 2^-inf = 0, and the accumulator is empty
+            m = mx;
+          }
+          float rs = 0.f;
+#pragma unroll
+          for (int j = 0; j < KT; ++j) {
+            v[j] = ex2(v[j] - m);
+            rs += v[j];
+          }
+          l = l * f + rs;
+        }
+        // the previous P V product must have finished before P is overwritten or the accumulator touched
+        if (t > 0 && !mbar_wait(bar(B_OFULL + x), (unsigned)(t - 1) & 1u, abort_flag)) { ok = false; break; }
+        if (warp_has_rows) {
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          if (rescale && t > 0) {
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+              float o[32];
+              tmem_ld32(t_out + c * 32, o);
+#pragma unroll
+              for (int j = 0; j < 32; ++j) o[j] *= f;
+              tmem_st32(t_out + c * 32, o);
+            }
+          }
+          // P as bf16, rows of 128 bytes, 16-byte chunks XOR (row % 8): the 128B-swizzled K-major layout
+#pragma unroll
+          for (int g = 0; g < 8; ++g) {
+            const float* e = v + g * 8;
+            const __nv_bfloat162 p0 = __floats2bfloat162_rn(e[0], e[1]);
+            const __nv_bfloat162 p1 = __floats2bfloat162_rn(e[2], e[3]);
+            const __nv_bfloat162 p2 = __floats2bfloat162_rn(e[4], e[5]);
+            const __nv_bfloat162 p3 = __floats2bfloat162_rn(e[6], e[7]);
+            const unsigned chunk = (unsigned)g ^ (unsigned)(r & 7);
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sPx + chunk * 16),
+                         "r"(*reinterpret_cast<const unsigned*>(&p0)), "r"(*reinterpret_cast<const unsigned*>(&p1)),
+                         "r"(*reinterpret_cast<const unsigned*>(&p2)), "r"(*reinterpret_cast<const unsigned*>(&p3))
+                         : "memory");
+          }
+        }
+        // the scores buffer is free; P is visible to the tensor core (async proxy) once fenced
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive(bar(B_SEMPTY + 2 * x + b));
+          mbar_arrive(bar(B_PFULL + x));
+        }
+      }
+      if (ok && n_tiles > 0 && mbar_wait(bar(B_OFULL + x), (unsigned)(n_tiles - 1) & 1u, abort_flag) &&
+          warp_has_rows) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const int tok = r / G, hg = r % G;
+        const bool valid = r < nrows;
+        const float inv = 1.0f / l;
+        bf16* dst = p.out + (size_t)(t0 + x * p.tq + (valid ? tok : 0)) * (p.hq * DH) + (size_t)(kh * G + hg) * DH;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          float o[32];
+          tmem_ld32(t_out + c * 32, o);
+          if (valid) {
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+              uint4 w;
+              __nv_bfloat162 h0 = __floats2bfloat162_rn(o[g * 8 + 0] * inv, o[g * 8 + 1] * inv);
+              __nv_bfloat162 h1 = __floats2bfloat162_rn(o[g * 8 + 2] * inv, o[g * 8 + 3] * inv);
+              __nv_bfloat162 h2 = __floats2bfloat162_rn(o[g * 8 + 4] * inv, o[g * 8 + 5] * inv);
+              __nv_bfloat162 h3 = __floats2bfloat162_rn(o[g * 8 + 6] * inv, o[g * 8 + 7] * inv);
+              w.x = *reinterpret_cast<unsigned*>(&h0);
+              w.y = *reinterpret_cast<unsigned*>(&h1);
+              w.z = *reinterpret_cast<unsigned*>(&h2);
+              w.w = *reinterpret_cast<unsigned*>(&h3);
+              *reinterpret_cast<uint4*>(dst + c * 32 + g * 8) = w;
+            }
+          }
+        }
+      }
+    }
+  }
+
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (s_abort && threadIdx.x == 0 && p.error_flag) atomicExch(p.error_flag, 1);
+  if (warp == 1) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
+  }
+}
+
+// ---- host side ---------------------------------------------------------------------------------------------
+
+PFN_cuTensorMapEncodeTiled_v12000 g_encode = nullptr;
+std::mutex g_mutex;
+struct Key3 {
+  const void* ptr; long long d1, d2, s1, s2; int b1, b2;
+  bool operator==(const Key3& o) const {
+    return ptr == o.ptr && d1 == o.d1 && d2 == o.d2 && s1 == o.s1 && s2 == o.s2 && b1 == o.b1 && b2 == o.b2;
+  }
+};
+struct Hash3 {
+  size_t operator()(const Key3& k) const {
+    size_t h = std::hash<const void*>()(k.ptr);
+    h = h * 1000003u ^ std::hash<long long>()(k.d1 * 131 + k.d2);
+    h = h * 1000003u ^ std::hash<long long>()(k.s1 * 257 + k.s2 * 7 + k.b1 * 3 + k.b2);
+    return h;
+  }
+};
+std::unordered_map<Key3, CUtensorMap, Hash3> g_maps;
+
+// bf16 tensor [d2][d1][128] with byte strides s1 (dim 1) and s2 (dim 2); box 64 x b1 x b2, 128-byte swizzle.
+bool get_map3(const bf16* ptr, long long d1, long long d2, long long s1, long long s2, int b1, int b2, CUtensorMap* out) {
+  std::lock_guard<std::mutex> lock(g_mutex);
+  if (!g_encode) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn)
+      return false;
+    g_encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
+  }
+  const Key3 key{ptr, d1, d2, s1, s2, b1, b2};
+  auto it = g_maps.find(key);
+  if (it != g_maps.end()) { *out = it->second; return true; }
+  if (g_maps.size() > 8192) g_maps.clear();
+  CUtensorMap m;
+  const cuuint64_t dims[3] = {(cuuint64_t)DH, (cuuint64_t)d1, (cuuint64_t)d2};
+  const cuuint64_t strides[2] = {(cuuint64_t)s1, (cuuint64_t)s2};
+  const cuuint32_t box[3] = {64, (cuuint32_t)b1, (cuuint32_t)b2};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  if (g_encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<bf16*>(ptr), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return false;
+  g_maps.emplace(key, m);
+  *out = m;
+  return true;
+}
+
+}  // namespace
+
+// Tokens per Q tile: as many as fit 128 flattened (token, head-in-group) rows, in multiples of 16.
+static int tokens_per_q_tile(int hq, int hkv) {
+  const int G = hq / hkv;
+  return G == 1 ? 128 : (G == 2 ? 64 : (G <= 4 ? 32 : 16));
+}
+
+// Query tokens per work item (two Q tiles share every K/V tile a CTA loads).
+int attention_tc_q_tile(int hq, int hkv) { return 2 * tokens_per_q_tile(hq, hkv); }
+
+// Returns cudaSuccess with *handled = false when the shape is left to the legacy kernel.
+cudaError_t launch_attention_tc(const bf16* qkv, const bf16* kc, const bf16* vc, bf16* out, const int* cu_q,
+                                const int* cu_tile, const int* kv_base, const int* vis, int n_rows, int n_tiles,
+                                int M, long long kv_rows, int max_nq, int hq, int hkv, int dh, int* error_flag,
+                                cudaStream_t s, bool* handled) {
+  *handled = false;
+  (void)max_nq;
+  if (dh != DH || hq % hkv || hq / hkv > 8 || kv_rows <= 0) return cudaSuccess;
+  if (((uintptr_t)qkv | (uintptr_t)kc | (uintptr_t)vc) & 15) return cudaSuccess;
+  const int G = hq / hkv;
+  const int tq = tokens_per_q_tile(hq, hkv);
+  static bool attr_done = false;
+  if (!attr_done) {
+    if (cudaFuncSetAttribute(k_attention_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
+      return cudaSuccess;
+    attr_done = true;
+  }
+  CUtensorMap mq, mk, mv;
+  const long long qkv_heads = hq + 2 * hkv;
+  if (!get_map3(qkv, qkv_heads, M, DH * 2, qkv_heads * DH * 2, G, tq, &mq)) return cudaSuccess;
+  if (!get_map3(kc, hkv, kv_rows, DH * 2, (long long)hkv * DH * 2, 1, KT, &mk)) return cudaSuccess;
+  if (!get_map3(vc, hkv, kv_rows, DH * 2, (long long)hkv * DH * 2, 1, KT, &mv)) return cudaSuccess;
+  *handled = true;
+  AttnTcParams p;
+  p.cu_q = cu_q; p.cu_tile = cu_tile; p.kv_base = kv_base; p.vis = vis; p.out = out;
+  p.n_rows = n_rows; p.hq = hq; p.hkv = hkv; p.tq = tq; p.error_flag = error_flag;
+  static int num_sms = 0;
+  if (!num_sms) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
+  }
+  // With fewer work items than SMs each CTA is one long dependent chain over the row's key tiles: give every Q
+  // tile its own CTA.  With many work items the two Q tiles of an item share each K/V tile they load.
+  p.split = (long long)n_tiles * hkv < num_sms ? 1 : 0;
+  return launch_pdl(k_attention_tc, dim3(p.split ? 2 * n_tiles : n_tiles, hkv), dim3(kThreads), (size_t)kSmemBytes, s,
+                    mq, mk, mv, p);
+}
+
+}  // namespace bs

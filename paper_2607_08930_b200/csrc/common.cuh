@@ -76,8 +76,8 @@ cudaError_t launch_rope_kv(bf16* qkv, const int* tok_pos, const int* tok_kv, bf1
 // scratch (nullable): fp32 partial results when the keys of a work item are split over several CTAs.
 cudaError_t launch_attention(const bf16* qkv, const bf16* kc, const bf16* vc, bf16* out, const int* cu_q,
                              const int* cu_tile, const int* kv_base, const int* vis, int n_rows, int n_tiles, int M,
-                             int max_vis, int max_nq, int hq, int hkv, int dh, float* scratch, size_t scratch_floats,
-                             cudaStream_t s);
+                             int max_vis, int max_nq, long long kv_rows, int hq, int hkv, int dh, float* scratch,
+                             size_t scratch_floats, int* error_flag, cudaStream_t s);
 cudaError_t launch_confidence(const float* logits, int n_rows, int vocab, int mask_id, int* tok, float* conf,
                               cudaStream_t s);
 
@@ -108,7 +108,7 @@ cudaError_t launch_finish_residual_norm(const float* partial, int splits, int M,
 
 cudaError_t launch_gemm_mma(const bf16* A, int lda, const bf16* W, const bf16* W2, void* C, int ldc, int M, int N,
                             int K, int mode, const float* row_scale, cudaStream_t s);
-int attention_q_tile(int hq, int hkv);
+int attention_q_tile(int hq, int hkv, int dh);
 void build_rope_table(float* host_cos_sin, int max_pos, int dh, float theta);   // [max_pos, dh/2, 2]
 
 }  // namespace bs

@@ -278,7 +278,7 @@ int bs_init_model(const bs_config* cfg, const bs_weights* w, void* kv, void* wor
   st.L = cfg->block_len; st.max_batch = cfg->max_batch; st.max_requests = cfg->max_requests;
   st.max_row_tokens = cfg->max_row_tokens; st.suffix_mode = cfg->suffix_mode; st.mask_id = cfg->mask_id;
   st.vocab = cfg->vocab; st.beta = cfg->token_budget; st.kv_capacity = cfg->kv_capacity_tokens; st.tau = cfg->tau;
-  st.q_tile = attention_q_tile(cfg->n_q_heads, cfg->n_kv_heads);
+  st.q_tile = attention_q_tile(cfg->n_q_heads, cfg->n_kv_heads, cfg->head_dim);
   e->gemm_scratch.partial = e->ws.partial;
   e->gemm_scratch.partial_floats = kPartialFloats;
   e->gemm_scratch.error_flag = st.hdr + H_ERROR;
@@ -298,6 +298,10 @@ int bs_init_model(const bs_config* cfg, const bs_weights* w, void* kv, void* wor
   for (int i = 0; i < BS_FAM_COUNT; ++i) e->prof_ms[i] = e->prof_flops[i] = e->prof_bytes[i] = 0.0, e->prof_launches[i] = 0;
   memset(e->hdr, 0, sizeof(e->hdr));
   cudaError_t r = cudaMemsetAsync(state, 0, state_bytes, e->stream);
+  // cache rows are read in whole tiles: rows no request has written yet must hold finite values (they meet a
+  // probability of exactly zero, and 0 * NaN would poison the row)
+  if (r == cudaSuccess)
+    r = cudaMemsetAsync(kv, 0, (size_t)cfg->n_layers * 2 * e->kv_half * sizeof(bf16), e->stream);
   if (r == cudaSuccess) r = cudaHostAlloc((void**)&e->pinned, (kHdrInts + cfg->max_batch) * sizeof(int), cudaHostAllocDefault);
   if (r == cudaSuccess) r = cudaEventCreateWithFlags(&e->ev, cudaEventDisableTiming);
   if (r == cudaSuccess) {
@@ -428,8 +432,8 @@ int bs_denoise_step(bs_engine* e, int* n_committed) {
       prof_work(e, BS_FAM_ROPE_KV, 1, 0, 4.0 * sp * dM * dq + 2.0 * dM * dq);
       prof_mark(e, BS_FAM_ATTENTION);
       KL(e, launch_attention(ws.qkv, kc, vc, ws.attn, st.cu_q[parity], st.cu_tile[parity], st.row_kv_base,
-                             st.row_vis, n_rows, e->hdr[H_QTILES], M, e->hdr[H_MAX_VIS], max_nq, hq, hkv, dh,
-                             ws.partial, kPartialFloats, s));
+                             st.row_vis, n_rows, e->hdr[H_QTILES], M, e->hdr[H_MAX_VIS], max_nq,
+                             c.kv_capacity_tokens, hq, hkv, dh, ws.partial, kPartialFloats, st.hdr + H_ERROR, s));
       prof_work(e, BS_FAM_ATTENTION, 1, 0, 2.0 * (2.0 * kv_rows * hkv * dh + 2.0 * dM * dhq));
       prof_mark(e, BS_FAM_GEMM_O);
       KL(e, launch_gemm_partial(ws.attn, hq * dh, e->wo[l], M, d, hq * dh, e->gemm_scratch, s, &sp));
@@ -464,7 +468,8 @@ int bs_denoise_step(bs_engine* e, int* n_committed) {
     prof_work(e, BS_FAM_ROPE_KV, 1, 0, 2.0 * dM * (dq + (double)(hq + 2 * hkv) * dh));
     prof_mark(e, BS_FAM_ATTENTION);
     KL(e, launch_attention(ws.qkv, kc, vc, ws.attn, st.cu_q[parity], st.cu_tile[parity], st.row_kv_base, st.row_vis,
-                           n_rows, e->hdr[H_QTILES], M, e->hdr[H_MAX_VIS], max_nq, hq, hkv, dh, nullptr, 0, s));
+                           n_rows, e->hdr[H_QTILES], M, e->hdr[H_MAX_VIS], max_nq, c.kv_capacity_tokens, hq, hkv, dh,
+                           nullptr, 0, st.hdr + H_ERROR, s));
     // every query token of a row meets every cache row of that row: flops = 4 * dh * Hq * sum_rows(n_q * vis);
     // the host knows the sums only for pure block steps and pure refresh steps, else it reports bytes alone
     prof_work(e, BS_FAM_ATTENTION, 1, 0, 2.0 * (2.0 * kv_rows * hkv * dh + 2.0 * dM * dhq));
@@ -688,19 +693,20 @@ int bs_op_rope_kv(void* qkv, const int* tok_pos, const int* tok_kv, void* kcache
                         table_scratch, s) == cudaSuccess ? BS_OK : BS_E_CUDA;
 }
 
-int bs_op_attention_q_tile(int n_q_heads, int n_kv_heads) {
+int bs_op_attention_q_tile(int n_q_heads, int n_kv_heads, int head_dim) {
   if (n_kv_heads < 1 || n_q_heads % n_kv_heads) return BS_E_ARG;
-  return attention_q_tile(n_q_heads, n_kv_heads);
+  return attention_q_tile(n_q_heads, n_kv_heads, head_dim);
 }
 
 int bs_op_attention(const void* qkv, const void* kcache, const void* vcache, void* out, const int* cu_q,
                     const int* cu_tile, const int* kv_base, const int* vis, int n_rows, int n_tiles, int M,
-                    int max_vis, int max_nq, int n_q_heads, int n_kv_heads, int head_dim, float* scratch,
-                    size_t scratch_bytes, void* stream) {
-  if (!qkv || !kcache || !vcache || !out || !cu_q || !cu_tile || !kv_base || !vis) return BS_E_ARG;
+                    int max_vis, int max_nq, long long kv_rows, int n_q_heads, int n_kv_heads, int head_dim,
+                    float* scratch, size_t scratch_bytes, int* error_flag, void* stream) {
+  if (!qkv || !kcache || !vcache || !out || !cu_q || !cu_tile || !kv_base || !vis || kv_rows < 1) return BS_E_ARG;
   return launch_attention((const bf16*)qkv, (const bf16*)kcache, (const bf16*)vcache, (bf16*)out, cu_q, cu_tile,
-                          kv_base, vis, n_rows, n_tiles, M, max_vis, max_nq, n_q_heads, n_kv_heads, head_dim, scratch,
-                          scratch ? scratch_bytes / sizeof(float) : 0, (cudaStream_t)stream) == cudaSuccess
+                          kv_base, vis, n_rows, n_tiles, M, max_vis, max_nq, kv_rows, n_q_heads, n_kv_heads, head_dim,
+                          scratch, scratch ? scratch_bytes / sizeof(float) : 0, error_flag,
+                          (cudaStream_t)stream) == cudaSuccess
              ? BS_OK : BS_E_CUDA;
 }
 

@@ -109,7 +109,7 @@ def bench_attention(args):
     kv_base = torch.arange(0, rows, dtype=torch.int32, device="cuda") * vis
     visd = torch.full((rows,), vis, dtype=torch.int32, device="cuda")
     scratch = torch.empty(16 << 20, dtype=torch.float32, device="cuda")
-    plan = B.attention_plan(cu_q, visd, hq, hkv)
+    plan = B.attention_plan(cu_q, visd, hq, hkv, dh)
     out = torch.empty(M, hq * dh, dtype=torch.bfloat16, device="cuda")
     def run(i):
         B.op_attention(qkv, kcs[i % copies], vcs[i % copies], cu_q, kv_base, visd, hq, hkv, dh, scratch=scratch,
