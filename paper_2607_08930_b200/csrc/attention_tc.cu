@@ -72,10 +72,10 @@ __device__ __forceinline__ void tma_load_3d(unsigned dst, const CUtensorMap* map
       ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar) : "memory");
 }
 // 128B-swizzled operand tile with rows of 128 bytes; 8-row groups are 1024 bytes apart (K-major and MN-major alike).
-__device__ __forceinline__ unsigned long long umma_desc(unsigned smem_addr) {
+__device__ __forceinline__ unsigned long long umma_desc(unsigned smem_addr, unsigned lbo_bytes = 16) {
   unsigned long long d = 0;
   d |= (unsigned long long)((smem_addr & 0x3FFFF) >> 4);
-  d |= (unsigned long long)1 << 16;
+  d |= (unsigned long long)(lbo_bytes >> 4) << 16;
   d |= (unsigned long long)(1024 >> 4) << 32;
   d |= (unsigned long long)1 << 46;
   d |= (unsigned long long)2 << 61;
@@ -252,7 +252,7 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0 && n_tiles > 0) {
       const unsigned idesc_s = umma_idesc(KT, false);
-      const unsigned idesc_o = umma_idesc(64, true);
+      const unsigned idesc_o = umma_idesc(DH, true);
       bool ok = mbar_wait(bar(B_QFULL), 0, abort_flag);
       // S = Q K^T of key tile t for every Q tile in use, into the S buffer of parity t
       auto issue_scores = [&](int t) -> bool {
@@ -283,10 +283,9 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 #pragma unroll
           for (int j = 0; j < KT / 16; ++j) {       // 16 keys per step
             const unsigned long long da = umma_desc(sP + x * kPBytes) + 2 * j;
-#pragma unroll
-            for (int h = 0; h < 2; ++h)             // two 64-wide halves of the head dimension
-              umma_bf16(tmem_base + x * 256 + 128 + h * 64, da, umma_desc(st + (2 + h) * kKvHalf + j * 2048), idesc_o,
-                        (t | j) ? 1u : 0u);         // the output accumulates in TMEM over all key tiles
+            // V as an MN-major operand: its two 64-wide dim halves are kKvHalf bytes apart (leading byte offset)
+            umma_bf16(tmem_base + x * 256 + 128, da, umma_desc(st + 2 * kKvHalf + j * 2048, kKvHalf), idesc_o,
+                      (t | j) ? 1u : 0u);             // the output accumulates in TMEM over all key tiles
           }
           umma_commit(bar(B_OFULL + x));
         }
@@ -320,12 +319,24 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           const int key0 = t * KT;
           tmem_ld32(t_lane + b * 64, v);
           tmem_ld32(t_lane + b * 64 + 32, v + 32);
-          float mx = -INFINITY;
+          // eight independent chains for the row maximum and the row sum: one warp per scheduler has no other
+          // warp to hide a 64-long dependent chain behind.  The maximum is taken over the raw scores (the scale
+          // is positive) and the scale folded into the exponent's fma.
+          float mx8[8];
 #pragma unroll
-          for (int j = 0; j < KT; ++j) {
-            v[j] = (key0 + j < vis) ? v[j] * sc : -INFINITY;
-            mx = fmaxf(mx, v[j]);                       // finite: every tile holds a valid key
+          for (int i = 0; i < 8; ++i) mx8[i] = -INFINITY;
+          if (key0 + KT <= vis) {
+#pragma unroll
+            for (int j = 0; j < KT; ++j) mx8[j & 7] = fmaxf(mx8[j & 7], v[j]);
+          } else {
+#pragma unroll
+            for (int j = 0; j < KT; ++j) {
+              v[j] = (key0 + j < vis) ? v[j] : -INFINITY;
+              mx8[j & 7] = fmaxf(mx8[j & 7], v[j]);
+            }
           }
+          const float mx = sc * fmaxf(fmaxf(fmaxf(mx8[0], mx8[1]), fmaxf(mx8[2], mx8[3])),
+                                      fmaxf(fmaxf(mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])));   // finite: a valid key exists
           // lazy rescale (warp-uniform decision: TMEM loads and stores are warp-wide)
           const bool grow = mx > m + kLazy;             // always true on the first tile (m = -inf)
           rescale = __any_sync(0xffffffffu, grow);
@@ -333,13 +344,16 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             f = ex2(m - mx);                            // first tile: 2^-inf = 0, and the accumulator is empty
             m = mx;
           }
-          float rs = 0.f;
+          float rs8[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) rs8[i] = 0.f;
+          const float neg_m = -m;
 #pragma unroll
           for (int j = 0; j < KT; ++j) {
-            v[j] = ex2(v[j] - m);
-            rs += v[j];
+            v[j] = ex2(fmaf(v[j], sc, neg_m));          // 2^(-inf) = 0 for masked keys
+            rs8[j & 7] += v[j];
           }
-          l = l * f + rs;
+          l = l * f + (((rs8[0] + rs8[1]) + (rs8[2] + rs8[3])) + ((rs8[4] + rs8[5]) + (rs8[6] + rs8[7])));
         }
         // the previous P V product must have finished before P is overwritten or the accumulator touched
         if (t > 0 && !mbar_wait(bar(B_OFULL + x), (unsigned)(t - 1) & 1u, abort_flag)) { ok = false; break; }
