@@ -39,6 +39,10 @@ struct GemmParams {
   int ksub;          // 64-wide k sub-blocks per pipeline stage
   int mode;          // 0 bf16 store, 1 fp32 +=, 2 fp32 row-scaled store, 3 SwiGLU, 4 fp32 partial sums only
   int dual;
+  int wide;          // two 128-row tiles of the same weight matrix share every token tile (256 weight rows per item)
+  int rows;          // weight rows per work item: 128 or 256
+  int nbuf;          // TMEM accumulator buffers: 2, or 1 when two accumulators need more than 256 columns
+  int acc1_off;      // column offset of the second accumulator
   void* C;
   int ldc;
   const float* row_scale;
@@ -141,7 +145,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
   const unsigned smem0 = (smem_u32(smem_dyn) + 1023u) & ~1023u;     // 1024-byte alignment for the swizzle atoms
   const int w_bytes = TILE_N * BK * 2;
   const int x_bytes = p.tn * BK * 2;
-  const int sub_bytes = (p.dual ? 2 : 1) * w_bytes + x_bytes;
+  const bool two_a = p.dual || p.wide;
+  const int sub_bytes = (two_a ? 2 : 1) * w_bytes + x_bytes;
   const int stage_bytes = p.ksub * sub_bytes;
   const unsigned full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[16]);
   const unsigned tfull0 = smem_u32(&bars[32]), tempty0 = smem_u32(&bars[34]);
@@ -196,8 +201,9 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
           for (int sub = 0; sub < p.ksub; ++sub) {
             const unsigned sw = smem0 + i * stage_bytes + sub * sub_bytes;
             const int k0 = ((kb0 + i) * p.ksub + sub) * BK;
-            tma_load_2d(sw, &map_w, k0, nt * TILE_N, full0 + 8 * i);
-            if (p.dual) tma_load_2d(sw + w_bytes, &map_w2, k0, nt * TILE_N, full0 + 8 * i);
+            tma_load_2d(sw, &map_w, k0, nt * p.rows, full0 + 8 * i);
+            if (p.dual) tma_load_2d(sw + w_bytes, &map_w2, k0, nt * p.rows, full0 + 8 * i);
+            if (p.wide) tma_load_2d(sw + w_bytes, &map_w, k0, nt * p.rows + TILE_N, full0 + 8 * i);
           }
         }
       }
@@ -218,10 +224,11 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
             const unsigned sw = smem0 + stage * stage_bytes + sub * sub_bytes;
             const int k0 = (kb * p.ksub + sub) * BK;       // beyond K the box is filled with zeros
             if (!prefetched) {
-              tma_load_2d(sw, &map_w, k0, nt * TILE_N, full0 + 8 * stage);
-              if (p.dual) tma_load_2d(sw + w_bytes, &map_w2, k0, nt * TILE_N, full0 + 8 * stage);
+              tma_load_2d(sw, &map_w, k0, nt * p.rows, full0 + 8 * stage);
+              if (p.dual) tma_load_2d(sw + w_bytes, &map_w2, k0, nt * p.rows, full0 + 8 * stage);
+              if (p.wide) tma_load_2d(sw + w_bytes, &map_w, k0, nt * p.rows + TILE_N, full0 + 8 * stage);
             }
-            tma_load_2d(sw + (p.dual ? 2 : 1) * w_bytes, &map_x, k0, mt * p.tn, full0 + 8 * stage);
+            tma_load_2d(sw + (two_a ? 2 : 1) * w_bytes, &map_x, k0, mt * p.tn, full0 + 8 * stage);
           }
           if (++stage == p.stages) { stage = 0; phase ^= 1u; }
         }
@@ -239,24 +246,24 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
         const int split = it % p.splits;
         const int kb0 = (int)((long long)p.kblocks * split / p.splits);
         const int kb1 = (int)((long long)p.kblocks * (split + 1) / p.splits);
-        const int acc = local & 1;
-        const unsigned acc_phase = (unsigned)(local >> 1) & 1u;
+        const int acc = local % p.nbuf;
+        const unsigned acc_phase = (unsigned)(local / p.nbuf) & 1u;
         if (!mbar_wait(tempty0 + 8 * acc, acc_phase ^ 1u, abort_flag)) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const unsigned d_gate = tmem_base + acc * acc_cols;
-        const unsigned d_up = d_gate + 128;
+        const unsigned d_up = d_gate + p.acc1_off;
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(full0 + 8 * stage, phase, abort_flag)) { ok = false; break; }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           for (int sub = 0; sub < p.ksub; ++sub) {
             const unsigned sw = smem0 + stage * stage_bytes + sub * sub_bytes;
             const unsigned long long dw = umma_desc(sw);
-            const unsigned long long dx = umma_desc(sw + (p.dual ? 2 : 1) * w_bytes);
+            const unsigned long long dx = umma_desc(sw + (two_a ? 2 : 1) * w_bytes);
 #pragma unroll
             for (int k = 0; k < BK / 16; ++k) {
               const unsigned accum = (kb > kb0 || sub > 0 || k > 0) ? 1u : 0u;
               umma_bf16(d_gate, dw + 2 * k, dx + 2 * k, idesc, accum);     // +32 bytes per 16-element K step
-              if (p.dual) umma_bf16(d_up, umma_desc(sw + w_bytes) + 2 * k, dx + 2 * k, idesc, accum);
+              if (two_a) umma_bf16(d_up, umma_desc(sw + w_bytes) + 2 * k, dx + 2 * k, idesc, accum);
             }
           }
           umma_commit(empty0 + 8 * stage);        // the stage is free once these MMAs have read it
@@ -274,63 +281,53 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
       const int split = it % p.splits;
       const int tile = it / p.splits;
       const int mt = tile % p.m_tiles, nt = tile / p.m_tiles;
-      const int acc = local & 1;
-      const unsigned acc_phase = (unsigned)(local >> 1) & 1u;
+      const int acc = local % p.nbuf;
+      const unsigned acc_phase = (unsigned)(local / p.nbuf) & 1u;
       if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag)) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const int n = nt * TILE_N + q * 32 + lane;
-      const bool n_ok = n < p.N;
-      const unsigned t_row = tmem_base + ((unsigned)(q * 32) << 16) + acc * acc_cols;
-      for (int c0 = 0; c0 < p.tn; c0 += 32) {
-        const int t0 = mt * p.tn + c0;
-        if (t0 >= p.M) break;                     // warp-uniform
-        // columns of this chunk that hold tokens of this tile (the tile width is a multiple of 16, not of 32)
-        const int jmax = min(min(32, p.tn - c0), p.M - t0);
-        float v[32];
-        tmem_ld32(t_row + c0, v);
-        if (p.splits > 1 || p.mode == 4) {
-          float* dst = p.partial + ((size_t)split * p.M) * p.N;
-          if (p.dual) {
-            float u[32];
-            tmem_ld32(t_row + 128 + c0, u);
-            float* dst2 = dst + (size_t)p.splits * p.M * p.N;
-#pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (n_ok && j < jmax) {
-                dst[(size_t)(t0 + j) * p.N + n] = v[j];
-                dst2[(size_t)(t0 + j) * p.N + n] = u[j];
-              }
-          } else {
+      for (int a = 0; a < (p.wide ? 2 : 1); ++a) {       // a wide item holds two 128-row accumulators
+        const int n = nt * p.rows + a * TILE_N + q * 32 + lane;
+        const bool n_ok = n < p.N;
+        const unsigned t_row = tmem_base + ((unsigned)(q * 32) << 16) + acc * acc_cols + a * p.acc1_off;
+        for (int c0 = 0; c0 < p.tn; c0 += 32) {
+          const int t0 = mt * p.tn + c0;
+          if (t0 >= p.M) break;                     // warp-uniform
+          // columns of this chunk that hold tokens of this tile (the tile width is a multiple of 16, not of 32)
+          const int jmax = min(min(32, p.tn - c0), p.M - t0);
+          float v[32];
+          tmem_ld32(t_row + c0, v);
+          if (p.splits > 1 || p.mode == 4) {
+            float* dst = p.partial + ((size_t)split * p.M) * p.N;
 #pragma unroll
             for (int j = 0; j < 32; ++j)
               if (n_ok && j < jmax) dst[(size_t)(t0 + j) * p.N + n] = v[j];
+          } else if (p.mode == 0) {
+            bf16* C = reinterpret_cast<bf16*>(p.C);
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (n_ok && j < jmax) C[(size_t)(t0 + j) * p.ldc + n] = __float2bfloat16_rn(v[j]);
+          } else if (p.mode == 1) {
+            // all loads first, then the stores: interleaving them would serialise on the load latency
+            float* C = reinterpret_cast<float*>(p.C) + (size_t)t0 * p.ldc + n;
+            float c[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) c[j] = (n_ok && j < jmax) ? C[(size_t)j * p.ldc] : 0.f;
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (n_ok && j < jmax) C[(size_t)j * p.ldc] = c[j] + v[j];
+          } else if (p.mode == 2) {
+            float* C = reinterpret_cast<float*>(p.C);
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (n_ok && j < jmax) C[(size_t)(t0 + j) * p.ldc + n] = v[j] * __ldg(p.row_scale + t0 + j);
+          } else {
+            float u[32];
+            tmem_ld32(t_row + p.acc1_off + c0, u);
+            bf16* C = reinterpret_cast<bf16*>(p.C);
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (n_ok && j < jmax) C[(size_t)(t0 + j) * p.ldc + n] = __float2bfloat16_rn(silu_f(v[j]) * u[j]);
           }
-        } else if (p.mode == 0) {
-          bf16* C = reinterpret_cast<bf16*>(p.C);
-#pragma unroll
-          for (int j = 0; j < 32; ++j)
-            if (n_ok && j < jmax) C[(size_t)(t0 + j) * p.ldc + n] = __float2bfloat16_rn(v[j]);
-        } else if (p.mode == 1) {
-          // all loads first, then the stores: interleaving them would serialise on the load latency
-          float* C = reinterpret_cast<float*>(p.C) + (size_t)t0 * p.ldc + n;
-          float c[32];
-#pragma unroll
-          for (int j = 0; j < 32; ++j) c[j] = (n_ok && j < jmax) ? C[(size_t)j * p.ldc] : 0.f;
-#pragma unroll
-          for (int j = 0; j < 32; ++j)
-            if (n_ok && j < jmax) C[(size_t)j * p.ldc] = c[j] + v[j];
-        } else if (p.mode == 2) {
-          float* C = reinterpret_cast<float*>(p.C);
-#pragma unroll
-          for (int j = 0; j < 32; ++j)
-            if (n_ok && j < jmax) C[(size_t)(t0 + j) * p.ldc + n] = v[j] * __ldg(p.row_scale + t0 + j);
-        } else {
-          float u[32];
-          tmem_ld32(t_row + 128 + c0, u);
-          bf16* C = reinterpret_cast<bf16*>(p.C);
-#pragma unroll
-          for (int j = 0; j < 32; ++j)
-            if (n_ok && j < jmax) C[(size_t)(t0 + j) * p.ldc + n] = __float2bfloat16_rn(silu_f(v[j]) * u[j]);
         }
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -451,9 +448,22 @@ cudaError_t launch_gemm_tc(const bf16* A, int lda, const bf16* W, const bf16* W2
   // Few tokens (a block step): one or two token tiles that cover M exactly (UMMA N is any multiple of 16), and a
   // k split that spreads the weight stream over all SMs when there are fewer weight tiles than SMs.
   // Many tokens (a refresh step): the widest tile, no split.
-  const int tn_cap = dual ? 128 : 256;
+  // Two 128-row weight tiles per work item (gate and up, or 256 rows of one matrix) share each token tile:
+  // the same tensor-core work then needs a third fewer bytes through L2.  Their two accumulators fit TMEM
+  // twice over only up to 128 tokens; wider token tiles run single-buffered (the epilogue is then not overlapped),
+  // which pays only when the main loop is long: measured on B200, 256-row items win for K >= 8192 (the down
+  // projection: -25 % at M >= 512) and lose or tie for K = 3584.
+  static const bool wide_off = getenv("BS_GEMM_WIDE") && atoi(getenv("BS_GEMM_WIDE")) == 0;
+  p.wide = (!dual && !wide_off && M >= 128 && N >= 512 && K >= 8192) ? 1 : 0;
+  p.rows = p.wide ? 2 * TILE_N : TILE_N;
+  p.n_tiles = (N + p.rows - 1) / p.rows;
+  const bool two_a = dual || p.wide;
+  int tn_cap = 256;
+  if (dual && (wide_off || M <= 128)) tn_cap = 128;
   p.m_tiles = (M + tn_cap - 1) / tn_cap;
   p.tn = (((M + p.m_tiles - 1) / p.m_tiles) + 15) / 16 * 16;     // tiles of equal width that cover M
+  p.nbuf = (two_a && p.tn > 128) ? 1 : 2;
+  p.acc1_off = p.nbuf == 1 ? 256 : 128;
   // narrow token tiles are weight-streaming bound: 128-wide k stages halve the per-stage barrier round trips
   p.ksub = p.tn <= 64 ? 2 : 1;
   if (const char* ev = getenv("BS_GEMM_KSUB")) p.ksub = atoi(ev) == 2 ? 2 : 1;
@@ -474,7 +484,7 @@ cudaError_t launch_gemm_tc(const bf16* A, int lda, const bf16* W, const bf16* W2
   if (dual) p.splits = 1;
   p.partial = g_partial;
   if (splits_out) *splits_out = p.splits;
-  const int stage_bytes = p.ksub * ((dual ? 2 : 1) * TILE_N * BK * 2 + p.tn * BK * 2);
+  const int stage_bytes = p.ksub * ((two_a ? 2 : 1) * TILE_N * BK * 2 + p.tn * BK * 2);
   p.stages = kSmemBudget / stage_bytes;
   if (const char* ev = getenv("BS_GEMM_STAGES")) { const int st = atoi(ev); if (st >= 2 && st < p.stages) p.stages = st; }
   if (p.stages > 16) p.stages = 16;
