@@ -184,6 +184,11 @@ enum {
 /* Copies the named array into host_buf (cap bytes); n = bytes written. */
 int bs_debug_read(bs_engine* e, int what, int arg0, int arg1, void* host_buf, size_t cap, size_t* n);
 
+/* Failure-path hook: enqueues a kernel whose mbarrier wait can never be satisfied and gives up after about a
+ * millisecond, raising the engine's error word exactly as a timed-out pipeline wait would.  The next call that
+ * reads the step header returns BS_E_TIMEOUT; the CUDA context stays usable. */
+int bs_debug_inject_timeout(bs_engine* e);
+
 /* ---- single operations (parity tests and per-kernel measurement) ------- *
  * All pointers are device memory; `stream` is a cudaStream_t as void*.     */
 

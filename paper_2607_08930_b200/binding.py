@@ -57,7 +57,7 @@ class BsStats(C.Structure):
 
 
 EXPORTS = ["bs_query_sizes", "bs_init_model", "bs_admit", "bs_evict_refill", "bs_denoise_step", "bs_block_done",
-           "bs_read_tokens", "bs_get_stats", "bs_set_profiling", "bs_get_profile", "bs_destroy", "bs_last_error", "bs_debug_read", "bs_op_gemm",
+           "bs_read_tokens", "bs_get_stats", "bs_set_profiling", "bs_get_profile", "bs_destroy", "bs_last_error", "bs_debug_read", "bs_debug_inject_timeout", "bs_op_gemm",
            "bs_op_rmsnorm", "bs_op_rope_kv", "bs_op_rope_kv_static", "bs_op_attention_q_tile", "bs_op_attention", "bs_op_confidence"]
 
 _lib = None
@@ -88,6 +88,7 @@ def lib() -> C.CDLL:
         L.bs_last_error.argtypes = [vp]
         L.bs_last_error.restype = C.c_char_p
         L.bs_debug_read.argtypes = [vp, i, i, i, vp, C.c_size_t, C.POINTER(C.c_size_t)]
+        L.bs_debug_inject_timeout.argtypes = [vp]
         L.bs_op_gemm.argtypes = [vp, i, vp, vp, vp, i, i, i, i, i, vp, vp, C.c_size_t, vp, vp]
         L.bs_op_rmsnorm.argtypes = [vp, vp, vp, vp, i, i, f, vp]
         L.bs_op_rope_kv.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, f, i, vp, vp]
@@ -216,6 +217,9 @@ class Engine:
         s = BsStats()
         self._chk(self.L.bs_get_stats(self.h, C.byref(s)))
         return s
+
+    def inject_timeout(self) -> None:
+        self._chk(self.L.bs_debug_inject_timeout(self.h))
 
     def set_profiling(self, on: bool) -> None:
         self._chk(self.L.bs_set_profiling(self.h, int(on)))

@@ -655,6 +655,39 @@ int bs_debug_read(bs_engine* e, int what, int arg0, int arg1, void* host_buf, si
   return BS_OK;
 }
 
+// A wait that nothing ever satisfies, with a short limit: the same bounded-wait helper pattern the tensor-core
+// kernels use.  It runs out after about a millisecond, raises the engine's error word and returns.
+__global__ void k_wait_that_runs_out(int* error_word, long long limit_cycles) {
+  __shared__ __align__(8) unsigned long long bar;
+  const unsigned addr = (unsigned)__cvta_generic_to_shared(&bar);
+  if (threadIdx.x == 0) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(addr));
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    const long long t0 = clock64();
+    bool done = false;
+    while (!done) {
+      unsigned ok;
+      asm volatile(
+          "{\n\t.reg .pred p;\n\t"
+          "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+          "selp.u32 %0, 1, 0, p;\n\t}"
+          : "=r"(ok) : "r"(addr), "r"(0u) : "memory");
+      if (ok) done = true;
+      else if (clock64() - t0 > limit_cycles) {
+        atomicExch(error_word, 1);
+        done = true;
+      }
+    }
+  }
+}
+
+int bs_debug_inject_timeout(bs_engine* e) {
+  if (!e) return BS_E_ARG;
+  k_wait_that_runs_out<<<1, 32, 0, e->stream>>>(e->st.hdr + H_ERROR, 2000000ll);
+  e->stats.kernel_launches++;
+  return cudaGetLastError() == cudaSuccess ? BS_OK : BS_E_CUDA;
+}
+
 // ---- single operations ----------------------------------------------------------------------------------
 
 int bs_op_gemm(const void* A, int lda, const void* W, const void* W2, void* C, int ldc, int M, int N, int K, int mode,

@@ -154,3 +154,24 @@ def test_state_errors(B):
         with pytest.raises(B.BlockServeError) as ei:
             eng.evict_refill()
         assert ei.value.code == B.BS_E_STATE
+
+
+def test_bounded_wait_reports_timeout_and_keeps_the_context(B):
+    """A device-side wait that runs out raises the engine's error word; the host reports BS_E_TIMEOUT and other
+    engines on the same context keep working (no trap, no hang)."""
+    shape = bs_inputs.TINY
+    wl = bs_inputs.custom_workload(shape, [10, 12], [32, 32], [4.0, 4.0], seed=2)
+    wc, _ = both_weights(shape, 5)
+    eng = B.engine_for_workload(wl, wc)
+    for r in wl.requests:
+        eng.admit(r.req_id, r.prompt, r.g, r.alpha)
+    eng.evict_refill()
+    eng.inject_timeout()
+    with pytest.raises(B.BlockServeError) as ei:
+        eng.denoise_step(want_count=True)
+    assert ei.value.code == B.BS_E_TIMEOUT
+    other = B.engine_for_workload(wl, wc)
+    for r in wl.requests:
+        other.admit(r.req_id, r.prompt, r.g, r.alpha)
+    other.run()
+    assert other.stats().committed == wl.committed_target()
