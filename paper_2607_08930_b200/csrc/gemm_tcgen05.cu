@@ -459,7 +459,7 @@ cudaError_t launch_gemm_tc(const bf16* A, int lda, const bf16* W, const bf16* W2
   p.n_tiles = (N + p.rows - 1) / p.rows;
   const bool two_a = dual || p.wide;
   int tn_cap = 256;
-  if (dual && (wide_off || M <= 128)) tn_cap = 128;
+  if (dual && (wide_off || M <= 128 || M > 256)) tn_cap = 128;   // several token tiles: keep the epilogue overlapped
   p.m_tiles = (M + tn_cap - 1) / tn_cap;
   p.tn = (((M + p.m_tiles - 1) / p.m_tiles) + 15) / 16 * 16;     // tiles of equal width that cover M
   p.nbuf = (two_a && p.tn > 128) ? 1 : 2;

@@ -175,3 +175,22 @@ def test_bounded_wait_reports_timeout_and_keeps_the_context(B):
         other.admit(r.req_id, r.prompt, r.g, r.alpha)
     other.run()
     assert other.stats().committed == wl.committed_target()
+
+
+@pytest.mark.parametrize("L,sort_queue,max_batch", [(16, True, 3), (8, False, 1), (32, False, 2)])
+def test_other_block_lengths_queue_orders_and_batch_caps(B, L, sort_queue, max_batch):
+    """Block lengths below 32, arrival-order queue, a batch cap of one: full lockstep on the tiny model."""
+    from lockstep import Lockstep
+    shape = bs_inputs.TINY
+    rng = np.random.default_rng(L)
+    n = 5
+    ps = rng.integers(3, 70, size=n)
+    gs = [int(g) for g in rng.choice([L, 2 * L + 3, 3 * L, L + 1], size=n)]
+    al = rng.choice([2.0, 9.0, 40.0], size=n)
+    wl = bs_inputs.custom_workload(shape, ps, gs, al, L=L, token_budget=0, max_batch=max_batch, seed=L + 1, tau=0.9)
+    wc, wn = both_weights(shape, 21)
+    ls = Lockstep(wl, wc, wn, sort_queue=sort_queue)
+    ls.admit(wl.requests)
+    ls.run()
+    ls.check_tokens()
+    assert ls.eng.stats().committed == wl.committed_target()
