@@ -177,7 +177,7 @@ enum {
   BS_DBG_LM_TOK = 9, BS_DBG_LM_ROW = 10, BS_DBG_LM_SLOT = 11,  /* int32[M_m] of the step about to run */
   BS_DBG_PREV_LM_ROW = 12, BS_DBG_PREV_LM_SLOT = 13,           /* int32[M_m] of the step that just ran */
   BS_DBG_PREV_TOK = 14, BS_DBG_PREV_CONF = 15, BS_DBG_PREV_COMMIT = 16, /* int32 / float / int32 [M_m], last step */
-  BS_DBG_PREV_LOGITS = 17, /* float[M_m * vocab] of the last step */
+  BS_DBG_PREV_LOGITS = 17, /* float[rows * vocab] of the last step: rows arg0 .. arg0 + arg1 (arg1 = 0: to the end) */
   BS_DBG_REQ_ID_OF_ROW = 18, /* int64[n_active] */
   BS_DBG_KV_ROW = 19   /* bf16 K then V of (layer = arg0, physical row = arg1): 2 * Hkv * head_dim values */
 };

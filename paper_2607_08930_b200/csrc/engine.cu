@@ -623,7 +623,13 @@ int bs_debug_read(bs_engine* e, int what, int arg0, int arg1, void* host_buf, si
     case BS_DBG_PREV_TOK: src = st.out_tok[prev]; bytes = (size_t)prev_mm * 4; break;
     case BS_DBG_PREV_CONF: src = st.out_conf[prev]; bytes = (size_t)prev_mm * 4; break;
     case BS_DBG_PREV_COMMIT: src = st.out_commit[prev]; bytes = (size_t)prev_mm * 4; break;
-    case BS_DBG_PREV_LOGITS: src = e->ws.logits; bytes = (size_t)prev_mm * e->cfg.vocab * 4; break;
+    case BS_DBG_PREV_LOGITS: {   // arg0 = first masked row, arg1 = number of rows (0: all rows from arg0)
+      if (arg0 < 0 || arg0 > prev_mm || arg1 < 0 || arg0 + arg1 > prev_mm) return fail(e, BS_E_ARG, "bad logit rows");
+      const int rows = arg1 > 0 ? arg1 : prev_mm - arg0;
+      src = e->ws.logits + (size_t)arg0 * e->cfg.vocab;
+      bytes = (size_t)rows * e->cfg.vocab * 4;
+      break;
+    }
     case BS_DBG_REQ_ID_OF_ROW: {
       std::vector<int> slots(n);
       if (n) CU(e, cudaMemcpy(slots.data(), st.row_slot, n * 4, cudaMemcpyDeviceToHost));

@@ -41,8 +41,8 @@ def logit_tol(n_layers: int) -> float:
     rounding adds a relative error of about 2^-9 / sqrt(3), rounding is discontinuous, and after a few layers the
     two pipelines round independently, so their logits differ by about 2^-9/sqrt(3) * sqrt(2 * 6 * n_layers)
     relative (5e-3 at 2 layers, 2e-2 at 28).  The bound is the stated 2e-2 up to the depth where that estimate
-    with a safety factor of 2 exceeds it."""
-    return max(LOGIT_TOL, 2.0 * (2.0 ** -9 / np.sqrt(3.0)) * np.sqrt(2.0 * 6.0 * n_layers))
+    with a safety factor of 2.5 (the maximum over a 150k-entry row sits above the rms) exceeds it."""
+    return max(LOGIT_TOL, 2.5 * (2.0 ** -9 / np.sqrt(3.0)) * np.sqrt(2.0 * 6.0 * n_layers))
 
 
 def lazy_oracle_model(shape, weights):
@@ -137,7 +137,9 @@ class Lockstep:
         assert self.eng.debug(B.DBG_PREV_LM_ROW, cap=cap).tolist() == ix["lm_row"].tolist()
         assert len(g_tok) == Mm and int(g_commit.sum()) == n_commit
         V = self.wl.shape.vocab
-        g_logits = self.eng.debug(B.DBG_PREV_LOGITS, np.float32, cap=4 * Mm * V + 64).reshape(Mm, V)
+        g_logits = None
+        if self.track is None:
+            g_logits = self.eng.debug(B.DBG_PREV_LOGITS, np.float32, cap=4 * Mm * V + 64).reshape(Mm, V)
         g_masks = self.eng.debug(B.DBG_ROW_MASK, np.uint32)
         tau = np.float32(self.wl.tau)
         mask_id = self.wl.shape.mask_id
@@ -166,7 +168,10 @@ class Lockstep:
             # decisions (identical unless a near tie is counted below)
             probe = O.denoise_step(self.model, r, self.wl.block_len, self.wl.tau, self.suffix_mode,
                                    keep_logits=True, override_commit=gs, override_tok=gt)
-            zl = g_logits[k:k + nm]
+            if g_logits is not None:
+                zl = g_logits[k:k + nm]
+            else:       # only the tracked rows' logits are read back
+                zl = self.eng.debug(B.DBG_PREV_LOGITS, np.float32, arg0=k, arg1=nm, cap=4 * nm * V + 64).reshape(nm, V)
             # (1) logits
             dev = np.abs(zl - probe.logits).max(-1)                       # D per row
             err = dev / np.abs(probe.logits).max(-1)

@@ -68,3 +68,26 @@ def test_benchmark_workload_full_depth_sampled_request(B):
     print(f"cfg2 full depth, request {sample.req_id} (p={sample.p}, alpha={sample.alpha:.2f}): {ls.summary()} "
           f"(depth-28 tolerance {logit_tol(28):.3f})")
     assert ls.rows_checked > 0 and ls.max_logit_err < logit_tol(wl.shape.n_layers)
+
+
+def test_llada_stream_full_depth_first_cycle_sampled_request(B):
+    """Workload 3 (LLaDA-8B-shaped stream of 256 under a budget of 16384) at full depth: the first fill admits the
+    shortest prompts up to the budget; the whole first block-cycle runs in the benchmark's launch configuration and
+    the oracle follows one admitted request."""
+    from lockstep import Lockstep, lazy_oracle_model, logit_tol
+    wl = bs_inputs.workload(3)
+    w = bs_inputs.make_weights(wl.shape, wl.weight_seed, device="cuda")
+    first = min(wl.requests, key=lambda r: (r.p, r.req_id))     # head of the sorted queue: admitted for sure
+    ls = Lockstep(wl, w, None, track=[first.req_id], kv_capacity=98304, model=lazy_oracle_model(wl.shape, w))
+    ls.admit(wl.requests)
+    _, admitted, n = ls.evict_refill()
+    assert first.req_id in admitted and n > 50
+    steps = 0
+    while True:
+        ls.step()
+        steps += 1
+        if ls.eng.block_done() or (ls.ora.by_id[first.req_id].mask == 0 and steps >= 3) or steps >= 8:
+            break
+    print(f"cfg3 full depth, {n} rows active, request {first.req_id} (p={first.p}, alpha={first.alpha:.2f}): "
+          f"{ls.summary()}")
+    assert ls.rows_checked > 0 and ls.max_logit_err < logit_tol(wl.shape.n_layers)
