@@ -184,6 +184,22 @@ enum {
 /* Copies the named array into host_buf (cap bytes); n = bytes written. */
 int bs_debug_read(bs_engine* e, int what, int arg0, int arg1, void* host_buf, size_t cap, size_t* n);
 
+/* Dictated commit (debugging): for the active row `row` (batch order), every block position j with bit j of
+ * mask_bits set and still masked takes tokens[j] (host array indexed by block position; entries of other positions
+ * are not read) and counts as committed.  The row's step counter does not move, so a row still waiting for the
+ * refresh step of its block (Section 2.5) gets it; the index of the pending step is rebuilt.  The paper has no
+ * counterpart.  Errors: BS_E_ARG (row not active, bit beyond L, token id out of range or the mask id). */
+int bs_debug_force_commit(bs_engine* e, int row, unsigned mask_bits, const int* tokens);
+
+/* Snapshot / restore of the engine state between block cycles (host buffers).  Because the block KV cache is rebuilt
+ * from the tokens at the first step of every block (Section 2.5, refresh), the state between cycles is the token rows
+ * plus the scheduler state; the KV arena is not saved.  bs_debug_snapshot with host_buf = NULL only reports the size
+ * in *n; otherwise it writes *n <= cap bytes.  BS_E_STATE while a block cycle is unfinished.  bs_debug_restore takes
+ * a snapshot of an engine with the identical bs_config (else BS_E_ARG) and replaces requests, queue, statistics and
+ * device state; the weights and buffers stay the caller's.  A restored engine continues bit-identically. */
+int bs_debug_snapshot(bs_engine* e, void* host_buf, size_t cap, size_t* n);
+int bs_debug_restore(bs_engine* e, const void* host_buf, size_t n_bytes);
+
 /* Failure-path hook: enqueues a kernel whose mbarrier wait can never be satisfied and gives up after about a
  * millisecond, raising the engine's error word exactly as a timed-out pipeline wait would.  The next call that
  * reads the step header returns BS_E_TIMEOUT; the CUDA context stays usable. */

@@ -57,7 +57,8 @@ class BsStats(C.Structure):
 
 
 EXPORTS = ["bs_query_sizes", "bs_init_model", "bs_admit", "bs_evict_refill", "bs_denoise_step", "bs_block_done",
-           "bs_read_tokens", "bs_get_stats", "bs_set_profiling", "bs_get_profile", "bs_destroy", "bs_last_error", "bs_debug_read", "bs_debug_inject_timeout", "bs_op_gemm",
+           "bs_read_tokens", "bs_get_stats", "bs_set_profiling", "bs_get_profile", "bs_destroy", "bs_last_error", "bs_debug_read", "bs_debug_inject_timeout",
+           "bs_debug_force_commit", "bs_debug_snapshot", "bs_debug_restore", "bs_op_gemm",
            "bs_op_rmsnorm", "bs_op_rope_kv", "bs_op_rope_kv_static", "bs_op_attention_q_tile", "bs_op_attention", "bs_op_confidence"]
 
 _lib = None
@@ -89,6 +90,9 @@ def lib() -> C.CDLL:
         L.bs_last_error.restype = C.c_char_p
         L.bs_debug_read.argtypes = [vp, i, i, i, vp, C.c_size_t, C.POINTER(C.c_size_t)]
         L.bs_debug_inject_timeout.argtypes = [vp]
+        L.bs_debug_force_commit.argtypes = [vp, i, C.c_uint, vp]
+        L.bs_debug_snapshot.argtypes = [vp, vp, C.c_size_t, C.POINTER(C.c_size_t)]
+        L.bs_debug_restore.argtypes = [vp, vp, C.c_size_t]
         L.bs_op_gemm.argtypes = [vp, i, vp, vp, vp, i, i, i, i, i, vp, vp, C.c_size_t, vp, vp]
         L.bs_op_rmsnorm.argtypes = [vp, vp, vp, vp, i, i, f, vp]
         L.bs_op_rope_kv.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, f, i, vp, vp]
@@ -220,6 +224,27 @@ class Engine:
 
     def inject_timeout(self) -> None:
         self._chk(self.L.bs_debug_inject_timeout(self.h))
+
+    def force_commit(self, row: int, positions: Dict[int, int]) -> None:
+        """Commit block position -> token for the given active row (debugging aid)."""
+        toks = np.zeros(32, dtype=np.int32)
+        bits = 0
+        for j, t in positions.items():
+            toks[j] = t
+            bits |= 1 << j
+        self._chk(self.L.bs_debug_force_commit(self.h, row, bits, toks.ctypes.data))
+
+    def snapshot(self) -> np.ndarray:
+        """Engine state between block cycles as bytes (token rows + scheduler state; the KV cache is rebuilt)."""
+        n = C.c_size_t(0)
+        self._chk(self.L.bs_debug_snapshot(self.h, None, 0, C.byref(n)))
+        buf = np.empty(n.value, dtype=np.uint8)
+        self._chk(self.L.bs_debug_snapshot(self.h, buf.ctypes.data, buf.nbytes, C.byref(n)))
+        return buf[:n.value]
+
+    def restore(self, snap: np.ndarray) -> None:
+        snap = np.ascontiguousarray(snap, dtype=np.uint8)
+        self._chk(self.L.bs_debug_restore(self.h, snap.ctypes.data, snap.nbytes))
 
     def set_profiling(self, on: bool) -> None:
         self._chk(self.L.bs_set_profiling(self.h, int(on)))

@@ -67,6 +67,8 @@ struct DevState {
 cudaError_t launch_sched(const DevState& st, cudaStream_t s);
 cudaError_t launch_commit_index(const DevState& st, cudaStream_t s);
 cudaError_t launch_fill_tokens(const DevState& st, int parity, int M, cudaStream_t s);
+// tokens32[j] is read for every bit j of `bits`; positions the row has already committed are skipped.
+cudaError_t launch_force_commit(const DevState& st, int row, unsigned bits, const int* tokens32, cudaStream_t s);
 
 cudaError_t launch_embed(const DevState& st, const bf16* embed, float* x, int M, int d, cudaStream_t s);
 cudaError_t launch_rmsnorm(const float* x, const int* idx, const bf16* w, bf16* y, int M, int d, float eps,

@@ -116,6 +116,8 @@ struct bs_engine {
   Workspace ws;
   cudaStream_t stream;
   bf16* kv;
+  void* state_base = nullptr;   // the caller's state buffer, for snapshots
+  size_t state_bytes = 0;
   size_t kv_layer_stride;   // elements between layers: 2 * rows * Hkv * dh
   size_t kv_half;           // elements between K and V of one layer
   const bf16 *embed, *lm_head, *final_norm;
@@ -274,6 +276,8 @@ int bs_init_model(const bs_config* cfg, const bs_weights* w, void* kv, void* wor
   e->kv_layer_stride = 2 * e->kv_half;
   carve_workspace(*cfg, workspace, &e->ws);
   const size_t state_bytes = carve_state(*cfg, state, &e->st);
+  e->state_base = state;
+  e->state_bytes = state_bytes;
   DevState& st = e->st;
   st.L = cfg->block_len; st.max_batch = cfg->max_batch; st.max_requests = cfg->max_requests;
   st.max_row_tokens = cfg->max_row_tokens; st.suffix_mode = cfg->suffix_mode; st.mask_id = cfg->mask_id;
@@ -658,6 +662,112 @@ int bs_debug_read(bs_engine* e, int what, int arg0, int arg1, void* host_buf, si
   if (bytes > cap) return fail(e, BS_E_ARG, "debug buffer too small");
   if (bytes) CU(e, cudaMemcpy(host_buf, src, bytes, cudaMemcpyDeviceToHost));
   if (n_out) *n_out = bytes;
+  return BS_OK;
+}
+
+int bs_debug_force_commit(bs_engine* e, int row, unsigned mask_bits, const int* tokens) {
+  if (!e || !tokens) return BS_E_ARG;
+  if (int rc = sync_header(e)) return rc;
+  if (row < 0 || row >= e->hdr[H_N_ACTIVE]) return fail(e, BS_E_ARG, "row is not an active row");
+  const int L = e->cfg.block_len;
+  if (L < 32 && (mask_bits >> L) != 0u) return fail(e, BS_E_ARG, "bit beyond the block length");
+  int t32[32] = {0};
+  for (int j = 0; j < 32; ++j)
+    if ((mask_bits >> j) & 1u) {
+      if (tokens[j] < 0 || tokens[j] >= e->cfg.vocab || tokens[j] == e->cfg.mask_id)
+        return fail(e, BS_E_ARG, "token id out of range");
+      t32[j] = tokens[j];
+    }
+  KL(e, launch_force_commit(e->st, row, mask_bits, t32, e->stream));
+  return post_header(e);
+}
+
+namespace {
+struct SnapHeader {
+  unsigned long long magic;
+  unsigned long long total_bytes, state_bytes;
+  unsigned long long n_slots, n_pending, uploaded_slots;
+  bs_config cfg;
+  bs_stats stats;
+  int hdr[kHdrInts];
+};
+constexpr unsigned long long kSnapMagic = 0x31304e5353424c42ull;   // "BLBSSN01"
+size_t snapshot_bytes(const bs_engine* e) {
+  const size_t n = e->id_of_slot.size();
+  return sizeof(SnapHeader) + n * (sizeof(long long) + 3 * sizeof(int) + sizeof(float)) +
+         e->pending.size() * sizeof(int) + e->state_bytes;
+}
+}  // namespace
+
+int bs_debug_snapshot(bs_engine* e, void* host_buf, size_t cap, size_t* n_out) {
+  if (!e || !n_out) return BS_E_ARG;
+  if (int rc = sync_header(e)) return rc;
+  const size_t need = snapshot_bytes(e);
+  *n_out = need;
+  if (!host_buf) return BS_OK;                      // size query
+  if (cap < need) return fail(e, BS_E_ARG, "snapshot buffer too small");
+  // The KV cache is not saved: it is rebuilt from the tokens at the first step of every block, so the state is
+  // complete only between block cycles.
+  if (e->hdr[H_N_ACTIVE] > 0 && !e->hdr[H_ALL_DONE])
+    return fail(e, BS_E_STATE, "snapshots are taken between block cycles");
+  CU(e, cudaStreamSynchronize(e->stream));
+  char* out = static_cast<char*>(host_buf);
+  SnapHeader h;
+  memset(&h, 0, sizeof(h));
+  h.magic = kSnapMagic;
+  h.total_bytes = need;
+  h.state_bytes = e->state_bytes;
+  h.n_slots = e->id_of_slot.size();
+  h.n_pending = e->pending.size();
+  h.uploaded_slots = (unsigned long long)e->uploaded_slots;
+  h.cfg = e->cfg;
+  h.stats = e->stats;
+  memcpy(h.hdr, e->hdr, sizeof(h.hdr));
+  memcpy(out, &h, sizeof(h)); out += sizeof(h);
+  const size_t n = h.n_slots;
+  auto put = [&](const void* src, size_t bytes) { if (bytes) memcpy(out, src, bytes); out += bytes; };
+  put(e->id_of_slot.data(), n * sizeof(long long));
+  put(e->h_p.data(), n * sizeof(int));
+  put(e->h_g.data(), n * sizeof(int));
+  put(e->h_b.data(), n * sizeof(int));
+  put(e->h_alpha.data(), n * sizeof(float));
+  put(e->pending.data(), h.n_pending * sizeof(int));
+  CU(e, cudaMemcpy(out, e->state_base, e->state_bytes, cudaMemcpyDeviceToHost));
+  return BS_OK;
+}
+
+int bs_debug_restore(bs_engine* e, const void* host_buf, size_t n_bytes) {
+  if (!e || !host_buf) return BS_E_ARG;
+  if (int rc = sync_header(e)) return rc;
+  if (n_bytes < sizeof(SnapHeader)) return fail(e, BS_E_ARG, "not a snapshot");
+  const char* in = static_cast<const char*>(host_buf);
+  SnapHeader h;
+  memcpy(&h, in, sizeof(h)); in += sizeof(h);
+  if (h.magic != kSnapMagic || h.total_bytes != n_bytes) return fail(e, BS_E_ARG, "not a snapshot");
+  if (memcmp(&h.cfg, &e->cfg, sizeof(bs_config)) != 0 || h.state_bytes != e->state_bytes)
+    return fail(e, BS_E_ARG, "snapshot of an engine with another configuration");
+  const size_t n = h.n_slots;
+  if (n > (size_t)e->cfg.max_requests || h.n_pending > n || h.uploaded_slots > n ||
+      sizeof(SnapHeader) + n * (sizeof(long long) + 3 * sizeof(int) + sizeof(float)) + h.n_pending * sizeof(int) +
+              h.state_bytes != n_bytes)
+    return fail(e, BS_E_ARG, "snapshot sizes are inconsistent");
+  CU(e, cudaStreamSynchronize(e->stream));
+  auto get = [&](void* dst, size_t bytes) { if (bytes) memcpy(dst, in, bytes); in += bytes; };
+  e->id_of_slot.resize(n); e->h_p.resize(n); e->h_g.resize(n); e->h_b.resize(n); e->h_alpha.resize(n);
+  e->pending.resize(h.n_pending);
+  get(e->id_of_slot.data(), n * sizeof(long long));
+  get(e->h_p.data(), n * sizeof(int));
+  get(e->h_g.data(), n * sizeof(int));
+  get(e->h_b.data(), n * sizeof(int));
+  get(e->h_alpha.data(), n * sizeof(float));
+  get(e->pending.data(), h.n_pending * sizeof(int));
+  e->slot_of.clear();
+  for (size_t i = 0; i < n; ++i) e->slot_of[e->id_of_slot[i]] = (int)i;
+  e->uploaded_slots = (int)h.uploaded_slots;
+  e->stats = h.stats;
+  memcpy(e->hdr, h.hdr, sizeof(e->hdr));
+  e->hdr_pending = false;
+  CU(e, cudaMemcpy(e->state_base, in, e->state_bytes, cudaMemcpyHostToDevice));
   return BS_OK;
 }
 

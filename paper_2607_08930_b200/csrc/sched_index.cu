@@ -293,6 +293,34 @@ __global__ void __launch_bounds__(kSchedThreads) k_commit_index(DevState st) {
   build_index(st, parity ^ 1, n, smi);
 }
 
+// Debug aid: commits the given block positions of one active row with the given tokens, as if a step had chosen
+// them, and rebuilds the index of the pending step.  The row's step counter is left alone, so a row that has not
+// had its refresh step yet still gets one.
+struct ForcedTokens { int t[32]; };
+__global__ void __launch_bounds__(kSchedThreads) k_force_commit(DevState st, int row, unsigned bits, ForcedTokens ft) {
+  __shared__ int smi[33];
+  const int parity = st.hdr[H_PARITY];
+  const int n = st.hdr[H_N_ACTIVE];
+  if (row < n) {
+    const unsigned take = bits & st.row_mask[row];
+    const int slot = st.row_slot[row];
+    const int lo = st.req_p[slot] + st.req_b[slot] * st.L;
+    if (threadIdx.x < 32 && ((take >> threadIdx.x) & 1u))
+      st.tokens[(size_t)slot * st.max_row_tokens + lo + threadIdx.x] = ft.t[threadIdx.x];
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      st.row_mask[row] &= ~take;
+      st.req_committed[slot] += __popc(take);
+      unsigned long long tot = ((unsigned long long)(unsigned)st.hdr[H_TOTAL_HI] << 32) | (unsigned)st.hdr[H_TOTAL_LO];
+      tot += (unsigned long long)__popc(take);
+      st.hdr[H_TOTAL_LO] = (int)(unsigned)(tot & 0xffffffffull);
+      st.hdr[H_TOTAL_HI] = (int)(unsigned)(tot >> 32);
+    }
+  }
+  __syncthreads();
+  build_index(st, parity, n, smi);
+}
+
 __global__ void k_fill_tokens(DevState st, int parity, int M) {
   pdl_wait();
   pdl_trigger();
@@ -319,6 +347,12 @@ cudaError_t launch_sched(const DevState& st, cudaStream_t s) {
 }
 cudaError_t launch_commit_index(const DevState& st, cudaStream_t s) {
   return launch_pdl(k_commit_index, dim3(1), dim3(kSchedThreads), 0, s, st);
+}
+cudaError_t launch_force_commit(const DevState& st, int row, unsigned bits, const int* tokens32, cudaStream_t s) {
+  ForcedTokens ft;
+  for (int i = 0; i < 32; ++i) ft.t[i] = tokens32[i];
+  k_force_commit<<<1, kSchedThreads, 0, s>>>(st, row, bits, ft);
+  return cudaGetLastError();
 }
 cudaError_t launch_fill_tokens(const DevState& st, int parity, int M, cudaStream_t s) {
   if (M <= 0) return cudaSuccess;

@@ -194,3 +194,112 @@ def test_other_block_lengths_queue_orders_and_batch_caps(B, L, sort_queue, max_b
     ls.run()
     ls.check_tokens()
     assert ls.eng.stats().committed == wl.committed_target()
+
+
+def _drive(eng, max_cycles=1 << 30):
+    cycles = 0
+    while cycles < max_cycles:
+        _, _, n = eng.evict_refill()
+        if n == 0:
+            break
+        while True:
+            eng.denoise_step()
+            if eng.block_done():
+                break
+        cycles += 1
+    return cycles
+
+
+def test_snapshot_restore_between_cycles_continues_bit_identically(B):
+    shape = bs_inputs.MINI_GQA
+    rng = np.random.default_rng(21)
+    n = 9
+    ps = rng.integers(8, 120, size=n)
+    gs = rng.choice([64, 96, 40], size=n)
+    al = rng.choice([2.0, 10.0, 40.0], size=n)
+    wl = bs_inputs.custom_workload(shape, ps, gs, al, token_budget=600, max_batch=4, seed=9, tau=0.9)
+    wc, _ = both_weights(shape, 31)
+    eng = B.engine_for_workload(wl, wc)
+    for r in wl.requests:
+        eng.admit(r.req_id, r.prompt, r.g, r.alpha)
+    assert _drive(eng, max_cycles=2) == 2
+    snap = eng.snapshot().copy()
+    steps_at_snap = eng.stats().steps
+    _drive(eng)
+    want = {r.req_id: eng.read_tokens(r.req_id) for r in wl.requests}
+    st_want = eng.stats()
+    assert st_want.committed == wl.committed_target()
+    # same engine, rewound
+    eng.restore(snap)
+    assert eng.stats().steps == steps_at_snap
+    _drive(eng)
+    for r in wl.requests:
+        toks, state = eng.read_tokens(r.req_id)
+        assert state == want[r.req_id][1] and (toks == want[r.req_id][0]).all()
+    st = eng.stats()
+    assert (st.committed, st.steps, st.cycles, st.packed_tokens) == \
+        (st_want.committed, st_want.steps, st_want.cycles, st_want.packed_tokens)
+    # a fresh engine of the same configuration picks the run up from the bytes alone
+    eng2 = B.engine_for_workload(wl, wc)
+    eng2.restore(snap)
+    _drive(eng2)
+    for r in wl.requests:
+        toks, state = eng2.read_tokens(r.req_id)
+        assert state == want[r.req_id][1] and (toks == want[r.req_id][0]).all()
+    assert eng2.stats().committed == st_want.committed
+
+
+def test_snapshot_refused_inside_a_cycle_and_for_another_config(B):
+    shape = bs_inputs.TINY
+    wl = bs_inputs.custom_workload(shape, [12, 20], [64, 64], [3.0, 5.0], seed=2, tau=0.95)
+    wc, _ = both_weights(shape, 5)
+    eng = B.engine_for_workload(wl, wc)
+    for r in wl.requests:
+        eng.admit(r.req_id, r.prompt, r.g, r.alpha)
+    snap0 = eng.snapshot().copy()            # before the first cycle: allowed
+    eng.evict_refill()
+    eng.denoise_step()
+    assert not eng.block_done()
+    with pytest.raises(B.BlockServeError) as ei:
+        eng.snapshot()
+    assert ei.value.code == B.BS_E_STATE
+    wl2 = bs_inputs.custom_workload(shape, [12, 20], [64, 64], [3.0, 5.0], seed=2, tau=0.5)
+    eng2 = B.engine_for_workload(wl2, wc)
+    with pytest.raises(B.BlockServeError) as ei:
+        eng2.restore(snap0)
+    assert ei.value.code == B.BS_E_ARG
+    with pytest.raises(B.BlockServeError):
+        eng.restore(snap0[:100])
+
+
+def test_force_commit_then_lockstep(B):
+    """A dictated commit before the refresh step: both sides apply it, then the block runs in lockstep."""
+    from lockstep import Lockstep
+    shape = bs_inputs.TINY
+    wl = bs_inputs.custom_workload(shape, [9, 17, 30], [64, 40, 33], [4.0, 8.0, 2.0], seed=12, tau=0.9)
+    wc, wn = both_weights(shape, 6)
+    ls = Lockstep(wl, wc, wn)
+    ls.admit(wl.requests)
+    ls.evict_refill()
+    forced = {0: {0: 7, 5: 11, 31: 3}, 2: {1: 19}}
+    for row, pos in forced.items():
+        ls.eng.force_commit(row, pos)
+        r = ls.ora.sched.active[row]
+        lo, _ = r.block_range(wl.block_len)
+        for j, t in pos.items():
+            assert (r.mask >> j) & 1
+            r.tokens[lo + j] = t
+            r.mask &= ~(1 << j)
+            r.committed += 1
+    assert ls.eng.debug(B.DBG_ROW_S).tolist() == [0, 0, 0]
+    while True:
+        ls.step()
+        done = ls.eng.block_done()
+        assert done == ls.ora.block_done()
+        if done:
+            break
+    ls.run()
+    ls.check_tokens()
+    assert ls.eng.stats().committed == wl.committed_target()
+    with pytest.raises(B.BlockServeError):      # no active row is left
+        ls.eng.force_commit(0, {0: 1})
