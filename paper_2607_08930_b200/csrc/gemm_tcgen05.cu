@@ -14,6 +14,7 @@
 #include <cuda.h>
 #include <cudaTypedefs.h>
 
+#include <stdio.h>
 #include <stdlib.h>
 
 #include <mutex>
@@ -113,6 +114,44 @@ __device__ __forceinline__ void umma_bf16(unsigned d_tmem, unsigned long long a,
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(d_tmem), "l"(a), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
 }
+// The MMA issuer is one thread, and every scalar instruction it spends between two tcgen05.mma delays the next
+// one: descriptors are therefore handled as 32-bit low words (start address >> 4, plus the fixed LBO field) that
+// advance by plain adds, with the constant high word (SBO, version, swizzle) joined inside the asm block.
+constexpr unsigned kDescHi = (unsigned)(1024 >> 4) | (1u << 14) | (2u << 29);
+__device__ __forceinline__ unsigned desc_lo(unsigned smem_addr) { return ((smem_addr & 0x3FFFFu) >> 4) | (1u << 16); }
+template <int CG>
+__device__ __forceinline__ void umma_lo(unsigned d_tmem, unsigned a_lo, unsigned b_lo, unsigned idesc,
+                                        unsigned accumulate) {
+  if (CG == 1) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "mov.b64 da, {%1, %5};\n\t"
+        "mov.b64 db, {%2, %5};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kDescHi) : "memory");
+  } else {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "mov.b64 da, {%1, %5};\n\t"
+        "mov.b64 db, {%2, %5};\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kDescHi) : "memory");
+  }
+}
+// One pipeline stage: 64 k elements = four K=16 steps (descriptor low word + 2 per step) for one or two accumulators.
+template <int CG, bool TWO>
+__device__ __forceinline__ void issue_stage(unsigned d0, unsigned d1, unsigned a0_lo, unsigned a1_lo, unsigned b_lo,
+                                            unsigned idesc, unsigned first_accum) {
+  umma_lo<CG>(d0, a0_lo, b_lo, idesc, first_accum);
+  if (TWO) umma_lo<CG>(d1, a1_lo, b_lo, idesc, first_accum);
+#pragma unroll
+  for (int k = 1; k < BK / 16; ++k) {
+    umma_lo<CG>(d0, a0_lo + 2 * k, b_lo + 2 * k, idesc, 1u);
+    if (TWO) umma_lo<CG>(d1, a1_lo + 2 * k, b_lo + 2 * k, idesc, 1u);
+  }
+}
 __device__ __forceinline__ void umma_commit(unsigned bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
@@ -132,6 +171,51 @@ __device__ __forceinline__ void tmem_ld32(unsigned taddr, float* v) {
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 __device__ __forceinline__ float silu_f(float x) { return x / (1.0f + __expf(-x)); }
+
+// Epilogue of one accumulator row: this thread holds output feature n for the tn tokens of token tile mt, whose
+// fp32 sums sit in TMEM at t_row (lane already selected) in columns 0 .. tn-1.
+__device__ __forceinline__ void epilogue_row(const GemmParams& p, int split, int mt, int n, bool n_ok, unsigned t_row) {
+  for (int c0 = 0; c0 < p.tn; c0 += 32) {
+    const int t0 = mt * p.tn + c0;
+    if (t0 >= p.M) break;                     // warp-uniform
+    // columns of this chunk that hold tokens of this tile (the tile width is a multiple of 16, not of 32)
+    const int jmax = min(min(32, p.tn - c0), p.M - t0);
+    float v[32];
+    tmem_ld32(t_row + c0, v);
+    if (p.splits > 1 || p.mode == 4) {
+      float* dst = p.partial + ((size_t)split * p.M) * p.N;
+#pragma unroll
+      for (int j = 0; j < 32; ++j)
+        if (n_ok && j < jmax) dst[(size_t)(t0 + j) * p.N + n] = v[j];
+    } else if (p.mode == 0) {
+      bf16* C = reinterpret_cast<bf16*>(p.C);
+#pragma unroll
+      for (int j = 0; j < 32; ++j)
+        if (n_ok && j < jmax) C[(size_t)(t0 + j) * p.ldc + n] = __float2bfloat16_rn(v[j]);
+    } else if (p.mode == 1) {
+      // all loads first, then the stores: interleaving them would serialise on the load latency
+      float* C = reinterpret_cast<float*>(p.C) + (size_t)t0 * p.ldc + n;
+      float c[32];
+#pragma unroll
+      for (int j = 0; j < 32; ++j) c[j] = (n_ok && j < jmax) ? C[(size_t)j * p.ldc] : 0.f;
+#pragma unroll
+      for (int j = 0; j < 32; ++j)
+        if (n_ok && j < jmax) C[(size_t)j * p.ldc] = c[j] + v[j];
+    } else if (p.mode == 2) {
+      float* C = reinterpret_cast<float*>(p.C);
+#pragma unroll
+      for (int j = 0; j < 32; ++j)
+        if (n_ok && j < jmax) C[(size_t)(t0 + j) * p.ldc + n] = v[j] * __ldg(p.row_scale + t0 + j);
+    } else {
+      float u[32];
+      tmem_ld32(t_row + p.acc1_off + c0, u);
+      bf16* C = reinterpret_cast<bf16*>(p.C);
+#pragma unroll
+      for (int j = 0; j < 32; ++j)
+        if (n_ok && j < jmax) C[(size_t)(t0 + j) * p.ldc + n] = __float2bfloat16_rn(silu_f(v[j]) * u[j]);
+    }
+  }
+}
 
 __global__ void __launch_bounds__(kThreads, 1)
 k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_w2,
@@ -242,6 +326,10 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
       int local = 0;
       const unsigned idesc = umma_idesc(p.tn);
       bool ok = true;
+      const unsigned lo0 = desc_lo(smem0);
+      const unsigned stage_step = (unsigned)stage_bytes >> 4, sub_step = (unsigned)sub_bytes >> 4;
+      const unsigned w_step = (unsigned)w_bytes >> 4, x_off = (two_a ? 2u : 1u) * w_step;
+      unsigned lo_stage = lo0;
       for (int it = blockIdx.x; it < items && ok; it += gridDim.x, ++local) {
         const int split = it % p.splits;
         const int kb0 = (int)((long long)p.kblocks * split / p.splits);
@@ -252,22 +340,19 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const unsigned d_gate = tmem_base + acc * acc_cols;
         const unsigned d_up = d_gate + p.acc1_off;
+        unsigned accum = 0u;
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(full0 + 8 * stage, phase, abort_flag)) { ok = false; break; }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          for (int sub = 0; sub < p.ksub; ++sub) {
-            const unsigned sw = smem0 + stage * stage_bytes + sub * sub_bytes;
-            const unsigned long long dw = umma_desc(sw);
-            const unsigned long long dx = umma_desc(sw + (two_a ? 2 : 1) * w_bytes);
-#pragma unroll
-            for (int k = 0; k < BK / 16; ++k) {
-              const unsigned accum = (kb > kb0 || sub > 0 || k > 0) ? 1u : 0u;
-              umma_bf16(d_gate, dw + 2 * k, dx + 2 * k, idesc, accum);     // +32 bytes per 16-element K step
-              if (two_a) umma_bf16(d_up, umma_desc(sw + w_bytes) + 2 * k, dx + 2 * k, idesc, accum);
-            }
+          unsigned lo = lo_stage;
+          for (int sub = 0; sub < p.ksub; ++sub, lo += sub_step) {
+            if (two_a) issue_stage<1, true>(d_gate, d_up, lo, lo + w_step, lo + x_off, idesc, accum);
+            else issue_stage<1, false>(d_gate, d_up, lo, lo, lo + x_off, idesc, accum);
+            accum = 1u;
           }
           umma_commit(empty0 + 8 * stage);        // the stage is free once these MMAs have read it
-          if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+          lo_stage += stage_step;
+          if (++stage == p.stages) { stage = 0; phase ^= 1u; lo_stage = lo0; }
         }
         if (ok) umma_commit(tfull0 + 8 * acc);    // accumulator complete
       }
@@ -289,46 +374,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
         const int n = nt * p.rows + a * TILE_N + q * 32 + lane;
         const bool n_ok = n < p.N;
         const unsigned t_row = tmem_base + ((unsigned)(q * 32) << 16) + acc * acc_cols + a * p.acc1_off;
-        for (int c0 = 0; c0 < p.tn; c0 += 32) {
-          const int t0 = mt * p.tn + c0;
-          if (t0 >= p.M) break;                     // warp-uniform
-          // columns of this chunk that hold tokens of this tile (the tile width is a multiple of 16, not of 32)
-          const int jmax = min(min(32, p.tn - c0), p.M - t0);
-          float v[32];
-          tmem_ld32(t_row + c0, v);
-          if (p.splits > 1 || p.mode == 4) {
-            float* dst = p.partial + ((size_t)split * p.M) * p.N;
-#pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (n_ok && j < jmax) dst[(size_t)(t0 + j) * p.N + n] = v[j];
-          } else if (p.mode == 0) {
-            bf16* C = reinterpret_cast<bf16*>(p.C);
-#pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (n_ok && j < jmax) C[(size_t)(t0 + j) * p.ldc + n] = __float2bfloat16_rn(v[j]);
-          } else if (p.mode == 1) {
-            // all loads first, then the stores: interleaving them would serialise on the load latency
-            float* C = reinterpret_cast<float*>(p.C) + (size_t)t0 * p.ldc + n;
-            float c[32];
-#pragma unroll
-            for (int j = 0; j < 32; ++j) c[j] = (n_ok && j < jmax) ? C[(size_t)j * p.ldc] : 0.f;
-#pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (n_ok && j < jmax) C[(size_t)j * p.ldc] = c[j] + v[j];
-          } else if (p.mode == 2) {
-            float* C = reinterpret_cast<float*>(p.C);
-#pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (n_ok && j < jmax) C[(size_t)(t0 + j) * p.ldc + n] = v[j] * __ldg(p.row_scale + t0 + j);
-          } else {
-            float u[32];
-            tmem_ld32(t_row + p.acc1_off + c0, u);
-            bf16* C = reinterpret_cast<bf16*>(p.C);
-#pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (n_ok && j < jmax) C[(size_t)(t0 + j) * p.ldc + n] = __float2bfloat16_rn(silu_f(v[j]) * u[j]);
-          }
-        }
+        epilogue_row(p, split, mt, n, n_ok, t_row);
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
@@ -342,6 +388,229 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
   if (warp == 1) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
+  }
+}
+
+// ---- CTA-pair variant ---------------------------------------------------------------------------------------
+// Two CTAs of a cluster share every tensor-core instruction (tcgen05.mma cta_group::2, UMMA M = 256): each CTA
+// stages 128 weight rows and HALF of the token tile, and the hardware reads the other half from the partner's
+// shared memory.  A CTA therefore streams 128 + tn/2 operand rows per k step for a 128 x tn accumulator instead of
+// 128 + tn, which is what the L2-to-SM path limits at large M.  Roles per CTA are those of k_gemm_tc; the MMA issuer
+// runs in the leader CTA (cluster rank 0) only:
+//   full[s]    leader's barrier; both CTAs' TMA loads complete their bytes on it
+//   empty[s]   one per CTA, released for both by the leader's multicast tcgen05.commit
+//   tfull[a]   one per CTA, same mechanism;  tempty[a]  leader's barrier, 4 epilogue warps of each CTA arrive on it
+__device__ __forceinline__ unsigned cluster_ctarank() {
+  unsigned r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ unsigned map_to_cta(unsigned addr, unsigned rank) {
+  unsigned r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tma_load_2d_pair(unsigned dst, const CUtensorMap* map, int c0, int c1,
+                                                 unsigned bar_in_cluster) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar_in_cluster) : "memory");
+}
+__device__ __forceinline__ unsigned umma_idesc_pair(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((unsigned)(n >> 3) << 17) | ((unsigned)(256 >> 4) << 24);
+}
+__device__ __forceinline__ void umma_bf16_pair(unsigned d_tmem, unsigned long long a, unsigned long long b,
+                                               unsigned idesc, unsigned accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
+}
+// arrives on the barrier at this shared-memory offset in both CTAs of the pair
+__device__ __forceinline__ void umma_commit_pair(unsigned bar) {
+  const unsigned short mask = 3;
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"(mask) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_in_cluster(unsigned bar_in_cluster) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_in_cluster) : "memory");
+}
+__device__ __forceinline__ void store_in_cluster(unsigned addr_in_cluster, int v) {
+  asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(addr_in_cluster), "r"(v) : "memory");
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+k_gemm_pair(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_w2,
+            const __grid_constant__ CUtensorMap map_x, const GemmParams p) {
+  extern __shared__ unsigned char smem_dyn[];
+  __shared__ __align__(8) unsigned long long bars[2 * 16 + 4];     // full[16], empty[16], tmem_full[2], tmem_empty[2]
+  __shared__ unsigned tmem_base_slot;
+  __shared__ int s_abort;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const unsigned rank = cluster_ctarank();
+  const bool leader = rank == 0;
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+  const unsigned smem0 = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+  const int w_bytes = TILE_N * BK * 2;
+  const int half_tn = p.tn >> 1;                                    // token rows this CTA stages
+  const int n_w = p.dual ? 2 : 1;
+  const int stage_bytes = n_w * w_bytes + half_tn * BK * 2;
+  const unsigned full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[16]);
+  const unsigned tfull0 = smem_u32(&bars[32]), tempty0 = smem_u32(&bars[34]);
+  const unsigned full_leader0 = map_to_cta(full0, 0), tempty_leader0 = map_to_cta(tempty0, 0);
+  const unsigned peer_abort = map_to_cta(smem_u32(&s_abort), rank ^ 1u);
+
+  if (threadIdx.x == 0) {
+    s_abort = 0;
+    for (int i = 0; i < p.stages; ++i) {
+      mbar_init(full0 + 8 * i, 1);
+      mbar_init(empty0 + 8 * i, 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(tfull0 + 8 * i, 1);
+      mbar_init(tempty0 + 8 * i, 8);       // one arrival per epilogue warp of either CTA
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {                          // both CTAs of the pair allocate their 512 columns
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&tmem_base_slot))
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  cluster_sync_all();                       // the partner's barriers exist before anything signals them
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const unsigned tmem_base = tmem_base_slot;
+  volatile int* abort_flag = &s_abort;
+  pdl_trigger();
+
+  const int items = p.n_tiles * p.m_tiles * p.splits;
+  const int acc_cols = 256;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer (both CTAs)
+    if (lane == 0) {
+      int stage = 0;
+      unsigned phase = 0;
+      bool ok = true;
+      int npre = 0;
+      if (pair < items) {                   // weight tiles of the first stages: constants, fetched before the wait
+        const int it = pair;
+        const int split = it % p.splits;
+        const int nt = (it / p.splits) / p.m_tiles;
+        const int kb0 = (int)((long long)p.kblocks * split / p.splits);
+        const int kb1 = (int)((long long)p.kblocks * (split + 1) / p.splits);
+        npre = min(p.stages, kb1 - kb0);
+        const int wrow = nt * 256 + (int)rank * TILE_N;
+        for (int i = 0; i < npre; ++i) {
+          if (leader) mbar_expect_tx(full0 + 8 * i, 2u * (unsigned)stage_bytes);
+          const unsigned sw = smem0 + i * stage_bytes;
+          const int k0 = (kb0 + i) * BK;
+          tma_load_2d_pair(sw, &map_w, k0, wrow, full_leader0 + 8 * i);
+          if (p.dual) tma_load_2d_pair(sw + w_bytes, &map_w2, k0, wrow, full_leader0 + 8 * i);
+        }
+      }
+      pdl_wait();
+      for (int it = pair; it < items && ok; it += n_pairs) {
+        const int split = it % p.splits;
+        const int tile = it / p.splits;
+        const int mt = tile % p.m_tiles, nt = tile / p.m_tiles;
+        const int kb0 = (int)((long long)p.kblocks * split / p.splits);
+        const int kb1 = (int)((long long)p.kblocks * (split + 1) / p.splits);
+        const int wrow = nt * 256 + (int)rank * TILE_N;
+        const int xrow = mt * p.tn + (int)rank * half_tn;
+        for (int kb = kb0; kb < kb1; ++kb) {
+          const bool prefetched = it == pair && kb - kb0 < npre;
+          const unsigned sw = smem0 + stage * stage_bytes;
+          const int k0 = kb * BK;
+          if (!prefetched) {
+            if (!mbar_wait(empty0 + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+            if (leader) mbar_expect_tx(full0 + 8 * stage, 2u * (unsigned)stage_bytes);
+            tma_load_2d_pair(sw, &map_w, k0, wrow, full_leader0 + 8 * stage);
+            if (p.dual) tma_load_2d_pair(sw + w_bytes, &map_w2, k0, wrow, full_leader0 + 8 * stage);
+          }
+          tma_load_2d_pair(sw + n_w * w_bytes, &map_x, k0, xrow, full_leader0 + 8 * stage);
+          if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) store_in_cluster(peer_abort, 1);
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer (leader CTA only)
+    if (lane == 0 && leader) {
+      int stage = 0;
+      unsigned phase = 0;
+      int local = 0;
+      const unsigned idesc = umma_idesc_pair(p.tn);
+      bool ok = true;
+      const unsigned lo0 = desc_lo(smem0);
+      const unsigned stage_step = (unsigned)stage_bytes >> 4;
+      const unsigned w_step = (unsigned)w_bytes >> 4, x_off = (unsigned)n_w * w_step;
+      unsigned lo_stage = lo0;
+      for (int it = pair; it < items && ok; it += n_pairs, ++local) {
+        const int split = it % p.splits;
+        const int kb0 = (int)((long long)p.kblocks * split / p.splits);
+        const int kb1 = (int)((long long)p.kblocks * (split + 1) / p.splits);
+        const int acc = local % p.nbuf;
+        const unsigned acc_phase = (unsigned)(local / p.nbuf) & 1u;
+        if (!mbar_wait(tempty0 + 8 * acc, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const unsigned d_gate = tmem_base + acc * acc_cols;
+        const unsigned d_up = d_gate + p.acc1_off;
+        unsigned accum = 0u;
+        for (int kb = kb0; kb < kb1; ++kb) {
+          if (!mbar_wait(full0 + 8 * stage, phase, abort_flag)) { ok = false; break; }
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          if (p.dual) issue_stage<2, true>(d_gate, d_up, lo_stage, lo_stage + w_step, lo_stage + x_off, idesc, accum);
+          else issue_stage<2, false>(d_gate, d_up, lo_stage, lo_stage, lo_stage + x_off, idesc, accum);
+          accum = 1u;
+          umma_commit_pair(empty0 + 8 * stage);
+          lo_stage += stage_step;
+          if (++stage == p.stages) { stage = 0; phase ^= 1u; lo_stage = lo0; }
+        }
+        if (ok) umma_commit_pair(tfull0 + 8 * acc);
+      }
+      if (!ok) store_in_cluster(peer_abort, 1);
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue warps (both CTAs)
+    const int q = warp & 3;
+    int local = 0;
+    bool ok = true;
+    pdl_wait();
+    for (int it = pair; it < items; it += n_pairs, ++local) {
+      const int split = it % p.splits;
+      const int tile = it / p.splits;
+      const int mt = tile % p.m_tiles, nt = tile / p.m_tiles;
+      const int acc = local % p.nbuf;
+      const unsigned acc_phase = (unsigned)(local / p.nbuf) & 1u;
+      if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag)) { ok = false; break; }
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const int n = nt * 256 + (int)rank * TILE_N + q * 32 + lane;
+      const unsigned t_row = tmem_base + ((unsigned)(q * 32) << 16) + acc * acc_cols;
+      epilogue_row(p, split, mt, n, n < p.N, t_row);
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) mbar_arrive_in_cluster(tempty_leader0 + 8 * acc);
+    }
+    if (!ok && lane == 0) store_in_cluster(peer_abort, 1);
+  }
+
+  // Neither CTA may leave (or free its TMEM) while the partner can still read its shared memory, write its
+  // accumulators or signal its barriers.
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  cluster_sync_all();
+  if (s_abort && threadIdx.x == 0 && p.error_flag) atomicExch(p.error_flag, 1);
+  if (warp == 1) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
   }
 }
 
@@ -419,6 +688,93 @@ bool get_map(const bf16* ptr, long long rows, long long cols, long long ld, int 
 
 int g_num_sms = 0;
 
+int g_max_pairs = 0;     // clusters of two CTAs that can be resident at once
+
+// Plans and launches the CTA-pair kernel; *handled stays false when the shape is left to the single-CTA kernel.
+cudaError_t launch_gemm_pair(const bf16* A, int lda, const bf16* W, const bf16* W2, void* C, int ldc, int M, int N,
+                             int K, int mode, const float* row_scale, const GemmScratch& scratch, cudaStream_t s,
+                             bool* handled, int* splits_out) {
+  if (!g_max_pairs) {
+    if (cudaFuncSetAttribute(k_gemm_pair, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 1024) !=
+        cudaSuccess) {
+      cudaGetLastError();
+      g_max_pairs = -1;
+    } else {
+      cudaLaunchConfig_t qc = {};
+      qc.gridDim = dim3(2 * g_num_sms);
+      qc.blockDim = dim3(kThreads);
+      qc.dynamicSmemBytes = (size_t)kSmemBudget + 1024;
+      cudaLaunchAttribute qa[1];
+      qa[0].id = cudaLaunchAttributeClusterDimension;
+      qa[0].val.clusterDim.x = 2; qa[0].val.clusterDim.y = 1; qa[0].val.clusterDim.z = 1;
+      qc.attrs = qa; qc.numAttrs = 1;
+      int n = 0;
+      if (cudaOccupancyMaxActiveClusters(&n, k_gemm_pair, &qc) != cudaSuccess || n < 1) { cudaGetLastError(); n = -1; }
+      g_max_pairs = n;
+    }
+    if (getenv("BS_GEMM_DEBUG")) fprintf(stderr, "gemm pair kernel: %d resident CTA pairs\n", g_max_pairs);
+  }
+  if (g_max_pairs < 1) return cudaSuccess;
+  const int dual = mode == 3;
+  GemmParams p;
+  p.M = M; p.N = N; p.K = K; p.mode = mode; p.dual = dual; p.C = C; p.ldc = ldc; p.row_scale = row_scale;
+  p.error_flag = scratch.error_flag;
+  p.wide = 0; p.rows = 256; p.ksub = 1;
+  p.n_tiles = (N + 255) / 256;
+  const int tn_cap = dual ? 128 : 256;       // gate and up accumulators, double-buffered, fill TMEM at 128 tokens
+  p.m_tiles = (M + tn_cap - 1) / tn_cap;
+  p.tn = (((M + p.m_tiles - 1) / p.m_tiles) + 15) / 16 * 16;
+  p.nbuf = 2;
+  p.acc1_off = 128;
+  p.kblocks = (K + BK - 1) / BK;
+  const int stage_bytes = (dual ? 2 : 1) * TILE_N * BK * 2 + (p.tn / 2) * BK * 2;
+  p.stages = kSmemBudget / stage_bytes;
+  if (p.stages > 16) p.stages = 16;
+  p.splits = 1;
+  const long long base_items = (long long)p.n_tiles * p.m_tiles;
+  if (scratch.partial && !dual && base_items * 4 < (long long)g_max_pairs * 3) {
+    int sp = (int)(g_max_pairs / base_items);
+    if (sp > 8) sp = 8;
+    while (sp > 1 && (p.kblocks / sp < 4 || (size_t)sp * (size_t)M * N > scratch.partial_floats)) --sp;
+    p.splits = sp < 1 ? 1 : sp;
+  }
+  if (mode == 4 && (!scratch.partial || (size_t)p.splits * (size_t)M * N > scratch.partial_floats))
+    return cudaErrorInvalidValue;
+  p.partial = scratch.partial;
+  if (splits_out) *splits_out = p.splits;
+  CUtensorMap mw, mw2, mx;
+  if (!get_map(W, N, K, K, TILE_N, &mw)) return cudaSuccess;
+  if (dual) { if (!get_map(W2, N, K, K, TILE_N, &mw2)) return cudaSuccess; } else { mw2 = mw; }
+  if (!get_map(A, M, K, lda, p.tn / 2, &mx)) return cudaSuccess;
+  *handled = true;
+  const long long items = base_items * p.splits;
+  static const bool dbg = getenv("BS_GEMM_DEBUG") != nullptr;
+  if (dbg) fprintf(stderr, "pair gemm M=%d N=%d K=%d mode=%d tn=%d m_tiles=%d n_tiles=%d splits=%d stages=%d\n", M, N, K, mode, p.tn, p.m_tiles, p.n_tiles, p.splits, p.stages);
+  const int pairs = (int)(items < g_max_pairs ? items : g_max_pairs);
+  static const bool no_pdl = getenv("BS_NO_PDL") != nullptr;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * pairs);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = (size_t)kSmemBudget + 1024;
+  cfg.stream = s;
+  cudaLaunchAttribute attrs[2];
+  attrs[0].id = cudaLaunchAttributeClusterDimension;
+  attrs[0].val.clusterDim.x = 2; attrs[0].val.clusterDim.y = 1; attrs[0].val.clusterDim.z = 1;
+  attrs[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attrs[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attrs;
+  cfg.numAttrs = no_pdl ? 1 : 2;
+  cudaError_t r = cudaLaunchKernelEx(&cfg, k_gemm_pair, mw, mw2, mx, p);
+  if (r != cudaSuccess) return r;
+  if (p.splits > 1 && mode != 4) {
+    const size_t total = (size_t)M * N;
+    const int blocks = (int)((total + 255) / 256 < (size_t)g_num_sms * 8 ? (total + 255) / 256 : (size_t)g_num_sms * 8);
+    r = launch_pdl(k_gemm_finish, dim3(blocks), dim3(256), 0, s, (const float*)scratch.partial, p.splits, M, N, mode, C,
+                   ldc, row_scale);
+  }
+  return r;
+}
+
 }  // namespace
 
 cudaError_t launch_gemm_tc(const bf16* A, int lda, const bf16* W, const bf16* W2, void* C, int ldc, int M, int N,
@@ -438,6 +794,21 @@ cudaError_t launch_gemm_tc(const bf16* A, int lda, const bf16* W, const bf16* W2
     if (cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 1024) !=
         cudaSuccess)
       return cudaSuccess;
+  }
+  // From a few hundred packed tokens on, CTA pairs that share each token tile are faster (measured on B200: +12 to
+  // +20 % at M >= 384 for K = 3584; the long-K down projection keeps its k-split single-CTA plan below 768 tokens,
+  // where a pair grid would have too few work items).  BS_GEMM_PAIR=0 turns pairs off, a positive value sets the
+  // smallest M that uses them.
+  static const int pair_env = getenv("BS_GEMM_PAIR") ? atoi(getenv("BS_GEMM_PAIR")) : -1;
+  bool use_pair;
+  if (pair_env >= 0) use_pair = pair_env > 0 && M >= pair_env;
+  else if (mode == 2) use_pair = M >= 128;
+  else if (mode == 3) use_pair = M >= 192;
+  else if (K >= 8192) use_pair = M >= 768;
+  else use_pair = M >= 384;
+  if (use_pair) {
+    cudaError_t r = launch_gemm_pair(A, lda, W, W2, C, ldc, M, N, K, mode, row_scale, scratch, s, handled, splits_out);
+    if (*handled || r != cudaSuccess) return r;
   }
   const int dual = mode == 3;
   GemmParams p;
@@ -497,6 +868,8 @@ cudaError_t launch_gemm_tc(const bf16* A, int lda, const bf16* W, const bf16* W2
 
   *handled = true;
   const long long items = (long long)p.n_tiles * p.m_tiles * p.splits;
+  static const bool dbg = getenv("BS_GEMM_DEBUG") != nullptr;
+  if (dbg) fprintf(stderr, "gemm M=%d N=%d K=%d mode=%d tn=%d m_tiles=%d n_tiles=%d splits=%d stages=%d wide=%d nbuf=%d\n", M, N, K, mode, p.tn, p.m_tiles, p.n_tiles, p.splits, p.stages, p.wide, p.nbuf);
   const int grid = (int)(items < g_num_sms ? items : g_num_sms);
   cudaError_t r = launch_pdl(k_gemm_tc, dim3(grid), dim3(kThreads), (size_t)kSmemBudget + 1024, s, mw, mw2, mx, p);
   if (r != cudaSuccess) return r;

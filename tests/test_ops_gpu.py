@@ -65,7 +65,10 @@ def test_gemm_modes(B, M, N, K, mode):
 
 
 @pytest.mark.parametrize("M,N,K,mode", [(32, 512, 4096, 0), (64, 384, 2048, 1), (100, 256, 8192, 3), (96, 640, 1024, 2),
-                                          (256, 1152, 3584, 1), (40, 3584, 18944, 1)])
+                                          (256, 1152, 3584, 1), (40, 3584, 18944, 1),
+                                          # CTA-pair kernel with a k split (few 256-row tiles, enough tokens)
+                                          (400, 512, 4096, 0), (512, 256, 2048, 1), (800, 256, 8192, 1),
+                                          (400, 520, 4096, 2)])
 def test_gemm_k_split(B, M, N, K, mode):
     """Few output tiles and a long K: the launch splits K across CTAs and sums the partials in a fixed order."""
     rng = np.random.default_rng(M + N + K)
