@@ -173,50 +173,53 @@ __device__ __forceinline__ void tmem_ld32(unsigned taddr, float* v) {
 __device__ __forceinline__ float silu_f(float x) { return x / (1.0f + __expf(-x)); }
 
 // Epilogue of one accumulator row: this thread holds output feature n for the tn tokens of token tile mt, whose
-// fp32 sums sit in TMEM at t_row (lane already selected) in columns 0 .. tn-1.
+// fp32 sums sit in TMEM at t_row (lane already selected) in columns 0 .. tn-1.  EPI: 0 bf16 store, 1 fp32 +=,
+// 2 fp32 row-scaled store, 3 SwiGLU, 4 fp32 partial sums of a k split.  The four epilogue warps each own one
+// scheduler, so their instruction count is what an epilogue costs: one pointer and one stride per chunk, and the
+// per-token predicate only in the ragged last chunk.
+template <int EPI, bool FULL>
+__device__ __forceinline__ void epilogue_chunk(const float* v, const float* u, char* ptr, size_t stride, int jmax,
+                                               const float* scale) {
+#pragma unroll
+  for (int j = 0; j < 32; ++j) {
+    if (!FULL && j >= jmax) break;
+    char* q = ptr + (size_t)j * stride;
+    if (EPI == 0) *reinterpret_cast<bf16*>(q) = __float2bfloat16_rn(v[j]);
+    else if (EPI == 1) *reinterpret_cast<float*>(q) = u[j] + v[j];
+    else if (EPI == 2) *reinterpret_cast<float*>(q) = v[j] * __ldg(scale + j);
+    else if (EPI == 3) *reinterpret_cast<bf16*>(q) = __float2bfloat16_rn(silu_f(v[j]) * u[j]);
+    else *reinterpret_cast<float*>(q) = v[j];
+  }
+}
+template <int EPI>
 __device__ __forceinline__ void epilogue_row(const GemmParams& p, int split, int mt, int n, bool n_ok, unsigned t_row) {
+  constexpr int esize = (EPI == 0 || EPI == 3) ? 2 : 4;
+  const int ld = EPI == 4 ? p.N : p.ldc;
+  char* base = EPI == 4 ? reinterpret_cast<char*>(p.partial + ((size_t)split * p.M) * p.N)
+                        : reinterpret_cast<char*>(p.C);
+  const size_t stride = (size_t)ld * esize;
   for (int c0 = 0; c0 < p.tn; c0 += 32) {
     const int t0 = mt * p.tn + c0;
     if (t0 >= p.M) break;                     // warp-uniform
     // columns of this chunk that hold tokens of this tile (the tile width is a multiple of 16, not of 32)
     const int jmax = min(min(32, p.tn - c0), p.M - t0);
-    float v[32];
+    float v[32], u[32];
     tmem_ld32(t_row + c0, v);
-    if (p.splits > 1 || p.mode == 4) {
-      float* dst = p.partial + ((size_t)split * p.M) * p.N;
-#pragma unroll
-      for (int j = 0; j < 32; ++j)
-        if (n_ok && j < jmax) dst[(size_t)(t0 + j) * p.N + n] = v[j];
-    } else if (p.mode == 0) {
-      bf16* C = reinterpret_cast<bf16*>(p.C);
-#pragma unroll
-      for (int j = 0; j < 32; ++j)
-        if (n_ok && j < jmax) C[(size_t)(t0 + j) * p.ldc + n] = __float2bfloat16_rn(v[j]);
-    } else if (p.mode == 1) {
+    if (EPI == 3) tmem_ld32(t_row + p.acc1_off + c0, u);
+    if (!n_ok) continue;                      // the TMEM loads above are warp-collective; the stores are not
+    char* ptr = base + ((size_t)t0 * ld + n) * esize;
+    if (EPI == 1) {
       // all loads first, then the stores: interleaving them would serialise on the load latency
-      float* C = reinterpret_cast<float*>(p.C) + (size_t)t0 * p.ldc + n;
-      float c[32];
 #pragma unroll
-      for (int j = 0; j < 32; ++j) c[j] = (n_ok && j < jmax) ? C[(size_t)j * p.ldc] : 0.f;
-#pragma unroll
-      for (int j = 0; j < 32; ++j)
-        if (n_ok && j < jmax) C[(size_t)j * p.ldc] = c[j] + v[j];
-    } else if (p.mode == 2) {
-      float* C = reinterpret_cast<float*>(p.C);
-#pragma unroll
-      for (int j = 0; j < 32; ++j)
-        if (n_ok && j < jmax) C[(size_t)(t0 + j) * p.ldc + n] = v[j] * __ldg(p.row_scale + t0 + j);
-    } else {
-      float u[32];
-      tmem_ld32(t_row + p.acc1_off + c0, u);
-      bf16* C = reinterpret_cast<bf16*>(p.C);
-#pragma unroll
-      for (int j = 0; j < 32; ++j)
-        if (n_ok && j < jmax) C[(size_t)(t0 + j) * p.ldc + n] = __float2bfloat16_rn(silu_f(v[j]) * u[j]);
+      for (int j = 0; j < 32; ++j) u[j] = j < jmax ? *reinterpret_cast<const float*>(ptr + (size_t)j * stride) : 0.f;
     }
+    const float* scale = EPI == 2 ? p.row_scale + t0 : nullptr;
+    if (jmax == 32) epilogue_chunk<EPI, true>(v, u, ptr, stride, jmax, scale);
+    else epilogue_chunk<EPI, false>(v, u, ptr, stride, jmax, scale);
   }
 }
 
+template <int EPI>
 __global__ void __launch_bounds__(kThreads, 1)
 k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_w2,
           const __grid_constant__ CUtensorMap map_x, const GemmParams p) {
@@ -374,7 +377,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
         const int n = nt * p.rows + a * TILE_N + q * 32 + lane;
         const bool n_ok = n < p.N;
         const unsigned t_row = tmem_base + ((unsigned)(q * 32) << 16) + acc * acc_cols + a * p.acc1_off;
-        epilogue_row(p, split, mt, n, n_ok, t_row);
+        epilogue_row<EPI>(p, split, mt, n, n_ok, t_row);
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
@@ -443,6 +446,7 @@ __device__ __forceinline__ void store_in_cluster(unsigned addr_in_cluster, int v
   asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(addr_in_cluster), "r"(v) : "memory");
 }
 
+template <int EPI>
 __global__ void __launch_bounds__(kThreads, 1)
 k_gemm_pair(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_w2,
             const __grid_constant__ CUtensorMap map_x, const GemmParams p) {
@@ -594,7 +598,7 @@ k_gemm_pair(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const int n = nt * 256 + (int)rank * TILE_N + q * 32 + lane;
       const unsigned t_row = tmem_base + ((unsigned)(q * 32) << 16) + acc * acc_cols;
-      epilogue_row(p, split, mt, n, n < p.N, t_row);
+      epilogue_row<EPI>(p, split, mt, n, n < p.N, t_row);
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
       if (lane == 0) mbar_arrive_in_cluster(tempty_leader0 + 8 * acc);
@@ -690,13 +694,38 @@ int g_num_sms = 0;
 
 int g_max_pairs = 0;     // clusters of two CTAs that can be resident at once
 
+using GemmKernel = void (*)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const GemmParams);
+GemmKernel kernel_tc(int epi) {
+  switch (epi) {
+    case 0: return k_gemm_tc<0>;
+    case 1: return k_gemm_tc<1>;
+    case 2: return k_gemm_tc<2>;
+    case 3: return k_gemm_tc<3>;
+    default: return k_gemm_tc<4>;
+  }
+}
+GemmKernel kernel_pair(int epi) {
+  switch (epi) {
+    case 0: return k_gemm_pair<0>;
+    case 1: return k_gemm_pair<1>;
+    case 2: return k_gemm_pair<2>;
+    case 3: return k_gemm_pair<3>;
+    default: return k_gemm_pair<4>;
+  }
+}
+bool allow_big_smem(GemmKernel (*table)(int)) {
+  for (int e = 0; e < 5; ++e)
+    if (cudaFuncSetAttribute(table(e), cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 1024) != cudaSuccess)
+      return false;
+  return true;
+}
+
 // Plans and launches the CTA-pair kernel; *handled stays false when the shape is left to the single-CTA kernel.
 cudaError_t launch_gemm_pair(const bf16* A, int lda, const bf16* W, const bf16* W2, void* C, int ldc, int M, int N,
                              int K, int mode, const float* row_scale, const GemmScratch& scratch, cudaStream_t s,
                              bool* handled, int* splits_out) {
   if (!g_max_pairs) {
-    if (cudaFuncSetAttribute(k_gemm_pair, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 1024) !=
-        cudaSuccess) {
+    if (!allow_big_smem(kernel_pair)) {
       cudaGetLastError();
       g_max_pairs = -1;
     } else {
@@ -709,7 +738,7 @@ cudaError_t launch_gemm_pair(const bf16* A, int lda, const bf16* W, const bf16* 
       qa[0].val.clusterDim.x = 2; qa[0].val.clusterDim.y = 1; qa[0].val.clusterDim.z = 1;
       qc.attrs = qa; qc.numAttrs = 1;
       int n = 0;
-      if (cudaOccupancyMaxActiveClusters(&n, k_gemm_pair, &qc) != cudaSuccess || n < 1) { cudaGetLastError(); n = -1; }
+      if (cudaOccupancyMaxActiveClusters(&n, k_gemm_pair<0>, &qc) != cudaSuccess || n < 1) { cudaGetLastError(); n = -1; }
       g_max_pairs = n;
     }
     if (getenv("BS_GEMM_DEBUG")) fprintf(stderr, "gemm pair kernel: %d resident CTA pairs\n", g_max_pairs);
@@ -734,6 +763,8 @@ cudaError_t launch_gemm_pair(const bf16* A, int lda, const bf16* W, const bf16* 
   const long long base_items = (long long)p.n_tiles * p.m_tiles;
   if (scratch.partial && !dual && base_items * 4 < (long long)g_max_pairs * 3) {
     int sp = (int)(g_max_pairs / base_items);
+    static const int sp_cap = getenv("BS_GEMM_PAIR_SPLITS") ? atoi(getenv("BS_GEMM_PAIR_SPLITS")) : 8;
+    if (sp > sp_cap) sp = sp_cap;
     if (sp > 8) sp = 8;
     while (sp > 1 && (p.kblocks / sp < 4 || (size_t)sp * (size_t)M * N > scratch.partial_floats)) --sp;
     p.splits = sp < 1 ? 1 : sp;
@@ -764,7 +795,7 @@ cudaError_t launch_gemm_pair(const bf16* A, int lda, const bf16* W, const bf16* 
   attrs[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attrs;
   cfg.numAttrs = no_pdl ? 1 : 2;
-  cudaError_t r = cudaLaunchKernelEx(&cfg, k_gemm_pair, mw, mw2, mx, p);
+  cudaError_t r = cudaLaunchKernelEx(&cfg, kernel_pair((p.splits > 1 || mode == 4) ? 4 : mode), mw, mw2, mx, p);
   if (r != cudaSuccess) return r;
   if (p.splits > 1 && mode != 4) {
     const size_t total = (size_t)M * N;
@@ -791,9 +822,7 @@ cudaError_t launch_gemm_tc(const bf16* A, int lda, const bf16* W, const bf16* W2
     int dev = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev);
-    if (cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 1024) !=
-        cudaSuccess)
-      return cudaSuccess;
+    if (!allow_big_smem(kernel_tc)) return cudaSuccess;
   }
   // From a few hundred packed tokens on, CTA pairs that share each token tile are faster (measured on B200: +12 to
   // +20 % at M >= 384 for K = 3584; the long-K down projection keeps its k-split single-CTA plan below 768 tokens,
@@ -871,7 +900,8 @@ cudaError_t launch_gemm_tc(const bf16* A, int lda, const bf16* W, const bf16* W2
   static const bool dbg = getenv("BS_GEMM_DEBUG") != nullptr;
   if (dbg) fprintf(stderr, "gemm M=%d N=%d K=%d mode=%d tn=%d m_tiles=%d n_tiles=%d splits=%d stages=%d wide=%d nbuf=%d\n", M, N, K, mode, p.tn, p.m_tiles, p.n_tiles, p.splits, p.stages, p.wide, p.nbuf);
   const int grid = (int)(items < g_num_sms ? items : g_num_sms);
-  cudaError_t r = launch_pdl(k_gemm_tc, dim3(grid), dim3(kThreads), (size_t)kSmemBudget + 1024, s, mw, mw2, mx, p);
+  cudaError_t r = launch_pdl(kernel_tc((p.splits > 1 || mode == 4) ? 4 : mode), dim3(grid), dim3(kThreads),
+                             (size_t)kSmemBudget + 1024, s, mw, mw2, mx, p);
   if (r != cudaSuccess) return r;
   if (p.splits > 1 && mode != 4) {
     const size_t total = (size_t)M * N;
