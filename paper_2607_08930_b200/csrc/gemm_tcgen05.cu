@@ -750,11 +750,14 @@ cudaError_t launch_gemm_pair(const bf16* A, int lda, const bf16* W, const bf16* 
   p.error_flag = scratch.error_flag;
   p.wide = 0; p.rows = 256; p.ksub = 1;
   p.n_tiles = (N + 255) / 256;
-  const int tn_cap = dual ? 128 : 256;       // gate and up accumulators, double-buffered, fill TMEM at 128 tokens
+  // Token tiles of up to 256.  With gate and up accumulators that fills TMEM, so the SwiGLU GEMM runs
+  // single-buffered above 128 tokens (the epilogue is not overlapped with the next item's main loop), but a CTA
+  // then moves 40 % fewer bytes from L2 per flop: measured faster at every M (1330 vs 1259 TFLOP/s at M = 4096).
+  const int tn_cap = 256;
   p.m_tiles = (M + tn_cap - 1) / tn_cap;
   p.tn = (((M + p.m_tiles - 1) / p.m_tiles) + 15) / 16 * 16;
-  p.nbuf = 2;
-  p.acc1_off = 128;
+  p.nbuf = (dual && p.tn > 128) ? 1 : 2;
+  p.acc1_off = p.nbuf == 1 ? 256 : 128;
   p.kblocks = (K + BK - 1) / BK;
   const int stage_bytes = (dual ? 2 : 1) * TILE_N * BK * 2 + (p.tn / 2) * BK * 2;
   p.stages = kSmemBudget / stage_bytes;
