@@ -462,7 +462,8 @@ k_gemm_pair(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
   const unsigned smem0 = (smem_u32(smem_dyn) + 1023u) & ~1023u;
   const int w_bytes = TILE_N * BK * 2;
   const int half_tn = p.tn >> 1;                                    // token rows this CTA stages
-  const int n_w = p.dual ? 2 : 1;
+  const bool two_w = p.dual || p.wide;                              // two weight tiles share each token tile
+  const int n_w = two_w ? 2 : 1;
   const int stage_bytes = n_w * w_bytes + half_tn * BK * 2;
   const unsigned full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[16]);
   const unsigned tfull0 = smem_u32(&bars[32]), tempty0 = smem_u32(&bars[34]);
@@ -511,13 +512,14 @@ k_gemm_pair(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
         const int kb0 = (int)((long long)p.kblocks * split / p.splits);
         const int kb1 = (int)((long long)p.kblocks * (split + 1) / p.splits);
         npre = min(p.stages, kb1 - kb0);
-        const int wrow = nt * 256 + (int)rank * TILE_N;
+        const int wrow = nt * p.rows + (int)rank * TILE_N;
         for (int i = 0; i < npre; ++i) {
           if (leader) mbar_expect_tx(full0 + 8 * i, 2u * (unsigned)stage_bytes);
           const unsigned sw = smem0 + i * stage_bytes;
           const int k0 = (kb0 + i) * BK;
           tma_load_2d_pair(sw, &map_w, k0, wrow, full_leader0 + 8 * i);
           if (p.dual) tma_load_2d_pair(sw + w_bytes, &map_w2, k0, wrow, full_leader0 + 8 * i);
+          if (p.wide) tma_load_2d_pair(sw + w_bytes, &map_w, k0, wrow + 256, full_leader0 + 8 * i);
         }
       }
       pdl_wait();
@@ -527,7 +529,7 @@ k_gemm_pair(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
         const int mt = tile % p.m_tiles, nt = tile / p.m_tiles;
         const int kb0 = (int)((long long)p.kblocks * split / p.splits);
         const int kb1 = (int)((long long)p.kblocks * (split + 1) / p.splits);
-        const int wrow = nt * 256 + (int)rank * TILE_N;
+        const int wrow = nt * p.rows + (int)rank * TILE_N;
         const int xrow = mt * p.tn + (int)rank * half_tn;
         for (int kb = kb0; kb < kb1; ++kb) {
           const bool prefetched = it == pair && kb - kb0 < npre;
@@ -538,6 +540,7 @@ k_gemm_pair(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
             if (leader) mbar_expect_tx(full0 + 8 * stage, 2u * (unsigned)stage_bytes);
             tma_load_2d_pair(sw, &map_w, k0, wrow, full_leader0 + 8 * stage);
             if (p.dual) tma_load_2d_pair(sw + w_bytes, &map_w2, k0, wrow, full_leader0 + 8 * stage);
+            if (p.wide) tma_load_2d_pair(sw + w_bytes, &map_w, k0, wrow + 256, full_leader0 + 8 * stage);
           }
           tma_load_2d_pair(sw + n_w * w_bytes, &map_x, k0, xrow, full_leader0 + 8 * stage);
           if (++stage == p.stages) { stage = 0; phase ^= 1u; }
@@ -571,7 +574,7 @@ k_gemm_pair(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(full0 + 8 * stage, phase, abort_flag)) { ok = false; break; }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          if (p.dual) issue_stage<2, true>(d_gate, d_up, lo_stage, lo_stage + w_step, lo_stage + x_off, idesc, accum);
+          if (two_w) issue_stage<2, true>(d_gate, d_up, lo_stage, lo_stage + w_step, lo_stage + x_off, idesc, accum);
           else issue_stage<2, false>(d_gate, d_up, lo_stage, lo_stage, lo_stage + x_off, idesc, accum);
           accum = 1u;
           umma_commit_pair(empty0 + 8 * stage);
@@ -596,9 +599,11 @@ k_gemm_pair(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
       const unsigned acc_phase = (unsigned)(local / p.nbuf) & 1u;
       if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag)) { ok = false; break; }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const int n = nt * 256 + (int)rank * TILE_N + q * 32 + lane;
-      const unsigned t_row = tmem_base + ((unsigned)(q * 32) << 16) + acc * acc_cols;
-      epilogue_row<EPI>(p, split, mt, n, n < p.N, t_row);
+      for (int a = 0; a < (p.wide ? 2 : 1); ++a) {       // a wide item holds two 256-row accumulators
+        const int n = nt * p.rows + a * 256 + (int)rank * TILE_N + q * 32 + lane;
+        const unsigned t_row = tmem_base + ((unsigned)(q * 32) << 16) + acc * acc_cols + a * p.acc1_off;
+        epilogue_row<EPI>(p, split, mt, n, n < p.N, t_row);
+      }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
       if (lane == 0) mbar_arrive_in_cluster(tempty_leader0 + 8 * acc);
@@ -748,18 +753,24 @@ cudaError_t launch_gemm_pair(const bf16* A, int lda, const bf16* W, const bf16* 
   GemmParams p;
   p.M = M; p.N = N; p.K = K; p.mode = mode; p.dual = dual; p.C = C; p.ldc = ldc; p.row_scale = row_scale;
   p.error_flag = scratch.error_flag;
-  p.wide = 0; p.rows = 256; p.ksub = 1;
-  p.n_tiles = (N + 255) / 256;
+  // Two 256-row weight tiles per pair and work item (BS_GEMM_PAIR_WIDE=1) halve the token-tile traffic once more at
+  // the price of single-buffered accumulators.  Measured on B200 it gains nothing over 256-row items for the
+  // K = 3584 projections and 5-8 % for the down projection at 384-640 tokens only, so it is off by default.
+  static const bool pair_wide = getenv("BS_GEMM_PAIR_WIDE") && atoi(getenv("BS_GEMM_PAIR_WIDE")) > 0;
+  p.wide = (pair_wide && !dual && N >= 1024) ? 1 : 0;
+  p.rows = p.wide ? 512 : 256;
+  p.ksub = 1;
+  p.n_tiles = (N + p.rows - 1) / p.rows;
   // Token tiles of up to 256.  With gate and up accumulators that fills TMEM, so the SwiGLU GEMM runs
   // single-buffered above 128 tokens (the epilogue is not overlapped with the next item's main loop), but a CTA
   // then moves 40 % fewer bytes from L2 per flop: measured faster at every M (1330 vs 1259 TFLOP/s at M = 4096).
   const int tn_cap = 256;
   p.m_tiles = (M + tn_cap - 1) / tn_cap;
   p.tn = (((M + p.m_tiles - 1) / p.m_tiles) + 15) / 16 * 16;
-  p.nbuf = (dual && p.tn > 128) ? 1 : 2;
+  p.nbuf = ((dual || p.wide) && p.tn > 128) ? 1 : 2;
   p.acc1_off = p.nbuf == 1 ? 256 : 128;
   p.kblocks = (K + BK - 1) / BK;
-  const int stage_bytes = (dual ? 2 : 1) * TILE_N * BK * 2 + (p.tn / 2) * BK * 2;
+  const int stage_bytes = ((dual || p.wide) ? 2 : 1) * TILE_N * BK * 2 + (p.tn / 2) * BK * 2;
   p.stages = kSmemBudget / stage_bytes;
   if (p.stages > 16) p.stages = 16;
   p.splits = 1;
