@@ -179,6 +179,12 @@ def run_ours(args):
     h2d = sum(4 * (r.p + r.g) for r in wl.requests)
     d2h = h2d
 
+    t_start = time.perf_counter()
+
+    def phase(msg):          # progress on stderr (BS_BENCH_VERBOSE=1): the JSON line stays alone on stdout
+        if rank == 0 and os.environ.get("BS_BENCH_VERBOSE"):
+            print(f"[bench {time.perf_counter() - t_start:8.1f} s] {msg}", file=sys.stderr, flush=True)
+
     # ---- warm-up (whole jobs) ----
     for _ in range(args.warmup):
         e = new_engine()
@@ -186,44 +192,50 @@ def run_ours(args):
         serve(e)
         assert e.stats().committed == target
         e.close()
+        del e
+        phase("warm-up job done")
     torch.cuda.synchronize()
 
-    # ---- device-resident arm: requests admitted (copied to HBM) before the clock starts ----
-    def timed_jobs(profile: bool):
-        engines = []
-        for _ in range(args.steps if not profile else 1):
+    # ---- device-resident arm: requests admitted (copied to HBM) before the clock starts.  One engine is alive at a
+    # time (a KV arena can take 45 GB): each job is bracketed by barrier + synchronize and timed with CUDA events on
+    # the launching stream; the timed region is the sum over the K jobs.
+    def timed_jobs(n_jobs: int, profile: bool):
+        stream = torch.cuda.current_stream()
+        total_ms, stats, profs = 0.0, [], []
+        for _ in range(n_jobs):
             e = new_engine()
             admit_all(e, pinned)
             e.set_profiling(profile)
-            engines.append(e)
-        torch.cuda.synchronize()
-        stream = torch.cuda.current_stream()
-        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        barrier(world)
-        torch.cuda.synchronize()
-        ev0.record(stream)
-        for e in engines:
+            ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            barrier(world)
+            torch.cuda.synchronize()
+            ev0.record(stream)
             serve(e)
-        ev1.record(stream)
-        torch.cuda.synchronize()
-        barrier(world)
-        return engines, ev0.elapsed_time(ev1)
+            ev1.record(stream)
+            torch.cuda.synchronize()
+            barrier(world)
+            total_ms += ev0.elapsed_time(ev1)
+            stats.append(e.stats())
+            if profile:
+                profs.append(e.profile())
+            e.close()
+            del e
+        return total_ms, stats, profs
 
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-    engines, ms_local = timed_jobs(profile=False)
+    ms_local, job_stats, _ = timed_jobs(args.steps, profile=False)
+    phase(f"timed jobs done ({ms_local:.0f} ms)")
     ms_total = max_over_ranks(ms_local, world, device)
     clocks = sampler.stop() if rank == 0 else None
-    committed = sum(e.stats().committed for e in engines)
+    committed = sum(st.committed for st in job_stats)
     assert committed == target * args.steps, "engine did not commit exactly g_i tokens per request"
-    launches = sum(e.stats().kernel_launches for e in engines)
-    steps_run = sum(e.stats().steps for e in engines)
-    cycles = sum(e.stats().cycles for e in engines)
-    sum_active = sum(e.stats().sum_active for e in engines)
-    for e in engines:
-        e.close()
-    del engines
+    launches = sum(st.kernel_launches for st in job_stats)
+    steps_run = sum(st.steps for st in job_stats)
+    cycles = sum(st.cycles for st in job_stats)
+    sum_active = sum(st.sum_active for st in job_stats)
     torch.cuda.empty_cache()
     total_committed = sum_over_ranks(float(committed), world, device)
     value = total_committed / (ms_total * 1e-3)
@@ -233,31 +245,32 @@ def run_ours(args):
     # job runs a few percent slower than the timed ones; its time is reported beside them.
     prof, prof_ms_job = {}, None
     if not args.no_profile:
-        engines, prof_ms_job = timed_jobs(profile=True)
-        for e in engines:
-            for fam, v in e.profile().items():
+        prof_ms_job, _, profs = timed_jobs(1, profile=True)
+        for pr in profs:
+            for fam, v in pr.items():
                 acc = prof.setdefault(fam, dict(ms=0.0, launches=0, flops=0.0, bytes=0.0))
                 for k in acc:
                     acc[k] += v[k]
-            e.close()
-        del engines
         torch.cuda.empty_cache()
+        phase("profiled job done")
 
-    # ---- end-to-end arm: host buffers in, host buffers out, through the C ABI ----
-    e2e_engines = [new_engine() for _ in range(args.steps)]
-    torch.cuda.synchronize()
-    barrier(world)
-    t0 = time.perf_counter()
-    for e in e2e_engines:
+    # ---- end-to-end arm: host buffers in, host buffers out, through the C ABI (engine set-up is not timed) ----
+    e2e_local = 0.0
+    for _ in range(args.steps):
+        e = new_engine()
+        torch.cuda.synchronize()
+        barrier(world)
+        t0 = time.perf_counter()
         admit_all(e, pinned)
         serve(e)
         for r in wl.requests:
             toks, state = e.read_tokens(r.req_id)
-    torch.cuda.synchronize()
-    e2e_s = max_over_ranks(time.perf_counter() - t0, world, device)
-    for e in e2e_engines:
+        torch.cuda.synchronize()
+        e2e_local += time.perf_counter() - t0
         e.close()
-    del e2e_engines
+        del e
+    e2e_s = max_over_ranks(e2e_local, world, device)
+    phase("end-to-end jobs done")
     e2e_value = total_committed / e2e_s
 
     if rank != 0:

@@ -279,8 +279,9 @@ class Engine:
 
     def close(self) -> None:
         if getattr(self, "h", None):
-            self.L.bs_destroy(self.h)
+            self.L.bs_destroy(self.h)      # synchronises the engine's stream
             self.h = None
+            self.kv = self.workspace = self.state = None    # give the arenas back to the allocator
 
     def __del__(self):
         try:
