@@ -725,10 +725,8 @@ bool allow_big_smem(GemmKernel (*table)(int)) {
   return true;
 }
 
-// Plans and launches the CTA-pair kernel; *handled stays false when the shape is left to the single-CTA kernel.
-cudaError_t launch_gemm_pair(const bf16* A, int lda, const bf16* W, const bf16* W2, void* C, int ldc, int M, int N,
-                             int K, int mode, const float* row_scale, const GemmScratch& scratch, cudaStream_t s,
-                             bool* handled, int* splits_out) {
+// Resident clusters of two CTAs (once per process); < 1 when the pair kernel cannot be used.
+int ensure_pair_init() {
   if (!g_max_pairs) {
     if (!allow_big_smem(kernel_pair)) {
       cudaGetLastError();
@@ -748,6 +746,27 @@ cudaError_t launch_gemm_pair(const bf16* A, int lda, const bf16* W, const bf16* 
     }
     if (getenv("BS_GEMM_DEBUG")) fprintf(stderr, "gemm pair kernel: %d resident CTA pairs\n", g_max_pairs);
   }
+  return g_max_pairs;
+}
+
+// Fraction of the persistent grid that has work, averaged over its rounds.
+double grid_busy(long long items, int workers) {
+  const long long rounds = (items + workers - 1) / workers;
+  return rounds > 0 ? (double)items / (double)(rounds * workers) : 0.0;
+}
+int split_for(long long base_items, int workers, int kblocks, size_t out_floats, const GemmScratch& scratch, bool dual) {
+  if (dual || !scratch.partial || base_items * 4 >= (long long)workers * 3) return 1;
+  int sp = (int)(workers / base_items);
+  if (sp > 8) sp = 8;
+  while (sp > 1 && (kblocks / sp < 4 || (size_t)sp * out_floats > scratch.partial_floats)) --sp;
+  return sp < 1 ? 1 : sp;
+}
+
+// Plans and launches the CTA-pair kernel; *handled stays false when the shape is left to the single-CTA kernel.
+cudaError_t launch_gemm_pair(const bf16* A, int lda, const bf16* W, const bf16* W2, void* C, int ldc, int M, int N,
+                             int K, int mode, const float* row_scale, const GemmScratch& scratch, cudaStream_t s,
+                             bool* handled, int* splits_out) {
+  ensure_pair_init();
   if (g_max_pairs < 1) return cudaSuccess;
   const int dual = mode == 3;
   GemmParams p;
@@ -838,17 +857,26 @@ cudaError_t launch_gemm_tc(const bf16* A, int lda, const bf16* W, const bf16* W2
     cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev);
     if (!allow_big_smem(kernel_tc)) return cudaSuccess;
   }
-  // From a few hundred packed tokens on, CTA pairs that share each token tile are faster (measured on B200: +12 to
-  // +20 % at M >= 384 for K = 3584; the long-K down projection keeps its k-split single-CTA plan below 768 tokens,
-  // where a pair grid would have too few work items).  BS_GEMM_PAIR=0 turns pairs off, a positive value sets the
-  // smallest M that uses them.
+  // CTA pairs that share each token tile move fewer bytes per flop and are faster per work item (measured on B200:
+  // +8 to +20 %), but their grid has half as many workers.  From 128 tokens on, the pair plan is taken unless it
+  // would leave clearly more of its grid idle than the single-CTA plan (few 256-row tiles and no k split, or a last
+  // round that is mostly empty).  BS_GEMM_PAIR=0 turns pairs off, a positive value sets the smallest M for them.
   static const int pair_env = getenv("BS_GEMM_PAIR") ? atoi(getenv("BS_GEMM_PAIR")) : -1;
-  bool use_pair;
+  bool use_pair = false;
   if (pair_env >= 0) use_pair = pair_env > 0 && M >= pair_env;
-  else if (mode == 2) use_pair = M >= 128;
-  else if (mode == 3) use_pair = M >= 192;
-  else if (K >= 8192) use_pair = M >= 768;
-  else use_pair = M >= 384;
+  else if (M >= 128 && ensure_pair_init() > 0) {
+    const bool dual_ = mode == 3;
+    const int kb = (K + BK - 1) / BK;
+    const long long items_p = (long long)((N + 255) / 256) * ((M + 255) / 256);
+    const double busy_p =
+        grid_busy(items_p * split_for(items_p, g_max_pairs, kb, (size_t)M * N, scratch, dual_), g_max_pairs);
+    const bool wide_s = !dual_ && N >= 512 && K >= 8192;
+    const int tn_cap_s = (dual_ && (M <= 128 || M > 256)) ? 128 : 256;
+    const long long items_s = (long long)((N + (wide_s ? 255 : 127)) / (wide_s ? 256 : 128)) * ((M + tn_cap_s - 1) / tn_cap_s);
+    const double busy_s =
+        grid_busy(items_s * split_for(items_s, g_num_sms, kb, (size_t)M * N, scratch, dual_), g_num_sms);
+    use_pair = busy_p * 1.1 >= busy_s;
+  }
   if (use_pair) {
     cudaError_t r = launch_gemm_pair(A, lda, W, W2, C, ldc, M, N, K, mode, row_scale, scratch, s, handled, splits_out);
     if (*handled || r != cudaSuccess) return r;
