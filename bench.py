@@ -37,8 +37,8 @@ METRIC = "committed_tokens_per_s"
 UNIT = "tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu capture summarised
-# in profiles/gemm_tcgen05_gate_up_m256.md (gate/up GEMM at M = 256: algorithmic 283.2 MB, measured 283.4 MB)
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 283404800
+# in profiles/gemm_pair_gate_up_m256.md (gate/up GEMM at M = 256: algorithmic 283.1 MB, measured 277.9 MB)
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 277925888
 GEMM_FAMILIES = ("gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down", "gemm_lm_head")
 
 
