@@ -71,28 +71,28 @@ __device__ __forceinline__ void tma_load_3d(unsigned dst, const CUtensorMap* map
       "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
       ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar) : "memory");
 }
-// 128B-swizzled operand tile with rows of 128 bytes; 8-row groups are 1024 bytes apart (K-major and MN-major alike).
-__device__ __forceinline__ unsigned long long umma_desc(unsigned smem_addr, unsigned lbo_bytes = 16) {
-  unsigned long long d = 0;
-  d |= (unsigned long long)((smem_addr & 0x3FFFF) >> 4);
-  d |= (unsigned long long)(lbo_bytes >> 4) << 16;
-  d |= (unsigned long long)(1024 >> 4) << 32;
-  d |= (unsigned long long)1 << 46;
-  d |= (unsigned long long)2 << 61;
-  return d;
-}
 // fp32 accumulator, bf16 operands, A K-major, M = 128; B K-major (scores) or MN-major (values).
 __device__ __forceinline__ unsigned umma_idesc(int n, bool b_mn_major) {
   return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn_major ? (1u << 16) : 0u) | ((unsigned)(n >> 3) << 17) |
          ((128u >> 4) << 24);
 }
-__device__ __forceinline__ void umma_bf16(unsigned d_tmem, unsigned long long a, unsigned long long b, unsigned idesc,
-                                          unsigned accumulate) {
+// Operand tiles are 128B-swizzled with rows of 128 bytes; 8-row groups are 1024 bytes apart (K-major and MN-major
+// alike).  The MMA issuer is one thread, and every scalar instruction between two tcgen05.mma delays the next one:
+// descriptors are handled as 32-bit low words (start address >> 4 | LBO field) that advance by adds; the constant
+// high word (SBO = 1024, version, 128B swizzle) is joined inside the asm block.
+constexpr unsigned kDescHi = (unsigned)(1024 >> 4) | (1u << 14) | (2u << 29);
+__device__ __forceinline__ unsigned desc_lo(unsigned smem_addr, unsigned lbo_bytes = 16) {
+  return ((smem_addr & 0x3FFFFu) >> 4) | ((lbo_bytes >> 4) << 16);
+}
+__device__ __forceinline__ void umma_lo(unsigned d_tmem, unsigned a_lo, unsigned b_lo, unsigned idesc,
+                                        unsigned accumulate) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\t"
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(a), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
+      "mov.b64 da, {%1, %5};\n\t"
+      "mov.b64 db, {%2, %5};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kDescHi) : "memory");
 }
 __device__ __forceinline__ void umma_commit(unsigned bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -262,12 +262,13 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         for (int x = 0; x < n_qt; ++x) {
           if (!mbar_wait(bar(B_SEMPTY + 2 * x + b), ((unsigned)(t >> 1) & 1u) ^ 1u, abort_flag)) return false;
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const unsigned q_lo = desc_lo(sQ + x * kQBytes), k_lo = desc_lo(st), d_s = tmem_base + x * 256 + b * 64;
 #pragma unroll
           for (int h = 0; h < 2; ++h)
 #pragma unroll
             for (int k = 0; k < 4; ++k)
-              umma_bf16(tmem_base + x * 256 + b * 64, umma_desc(sQ + x * kQBytes + h * kHalfBytes) + 2 * k,
-                        umma_desc(st + h * kKvHalf) + 2 * k, idesc_s, (h | k) ? 1u : 0u);
+              umma_lo(d_s, q_lo + h * (kHalfBytes >> 4) + 2 * k, k_lo + h * (kKvHalf >> 4) + 2 * k, idesc_s,
+                      (h | k) ? 1u : 0u);
           umma_commit(bar(B_SFULL + 2 * x + b));
         }
         return true;
@@ -280,13 +281,12 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         for (int x = 0; x < n_qt && ok; ++x) {
           if (!mbar_wait(bar(B_PFULL + x), (unsigned)t & 1u, abort_flag)) { ok = false; break; }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          // V as an MN-major operand: its two 64-wide dim halves are kKvHalf bytes apart (leading byte offset)
+          const unsigned p_lo = desc_lo(sP + x * kPBytes), v_lo = desc_lo(st + 2 * kKvHalf, kKvHalf);
+          const unsigned d_o = tmem_base + x * 256 + 128;
 #pragma unroll
-          for (int j = 0; j < KT / 16; ++j) {       // 16 keys per step
-            const unsigned long long da = umma_desc(sP + x * kPBytes) + 2 * j;
-            // V as an MN-major operand: its two 64-wide dim halves are kKvHalf bytes apart (leading byte offset)
-            umma_bf16(tmem_base + x * 256 + 128, da, umma_desc(st + 2 * kKvHalf + j * 2048, kKvHalf), idesc_o,
-                      (t | j) ? 1u : 0u);             // the output accumulates in TMEM over all key tiles
-          }
+          for (int j = 0; j < KT / 16; ++j)         // 16 keys per step; the output accumulates over all key tiles
+            umma_lo(d_o, p_lo + 2 * j, v_lo + j * (2048 >> 4), idesc_o, (t | j) ? 1u : 0u);
           umma_commit(bar(B_OFULL + x));
         }
         if (ok) umma_commit(bar(B_KVEMPTY + (t % kStages)));
