@@ -1,0 +1,71 @@
+"""Throughput-only ablations of the serving policy on a synthetic workload (Section 4's research questions on queue
+order and block length, in the form that needs no trained weights): sorted vs submission-order queue, suffix
+visibility FULL vs NONE, block length L.  Prints one JSON line per variant and a markdown table.
+
+    python -m paper_2607_08930_b200.ablate --workload 3
+"""
+from __future__ import annotations
+
+import argparse
+import dataclasses
+import json
+import os
+import sys
+
+import torch
+
+sys.path.insert(0, os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
+import bs_inputs  # noqa: E402
+from paper_2607_08930_b200 import binding as B, build  # noqa: E402
+
+
+def run_variant(wl, weights, sort_queue: bool, suffix_mode: int):
+    eng = B.engine_for_workload(wl, weights, sort_queue=sort_queue, suffix_mode=suffix_mode)
+    for r in wl.requests:
+        eng.admit(r.req_id, r.prompt, r.g, r.alpha, r.start_block, r.gen_prefix)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    ev0.record()
+    eng.run()
+    ev1.record()
+    torch.cuda.synchronize()
+    st = eng.stats()
+    assert st.committed == wl.committed_target()
+    ms = ev0.elapsed_time(ev1)
+    out = dict(tokens_per_s=st.committed / (ms * 1e-3), job_s=ms * 1e-3, cycles=st.cycles, steps=st.steps,
+               packed_tokens=st.packed_tokens, mean_active=st.sum_active / max(st.cycles, 1),
+               effective_compute_ratio=st.sum_active / max(st.cycles, 1) / wl.max_batch)
+    eng.close()
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--workload", type=int, default=3)
+    ap.add_argument("--block-lens", type=int, nargs="+", default=[32, 16])
+    args = ap.parse_args()
+    build.build()
+    base = bs_inputs.workload(args.workload)
+    weights = bs_inputs.make_weights(base.shape, base.weight_seed, device="cuda:0")
+    rows = []
+    for L in args.block_lens:
+        if L != base.block_len and any(r.start_block for r in base.requests):
+            continue            # pre-committed start blocks are stated in units of the workload's own L
+        wl = dataclasses.replace(base, block_len=L)
+        for sort_queue in (True, False):
+            for suffix_mode in (B.SUFFIX_FULL, B.SUFFIX_NONE):
+                run_variant(wl, weights, sort_queue, suffix_mode)          # warm-up
+                res = run_variant(wl, weights, sort_queue, suffix_mode)
+                res.update(workload=wl.name, block_len=L, queue="sorted" if sort_queue else "submission order",
+                           suffix="full" if suffix_mode == B.SUFFIX_FULL else "none")
+                print(json.dumps(res), flush=True)
+                rows.append(res)
+    print("\n| L | queue | suffix | committed tokens/s | job s | cycles | steps | packed tokens | mean |A| |")
+    print("|---|---|---|---|---|---|---|---|---|")
+    for r in rows:
+        print(f"| {r['block_len']} | {r['queue']} | {r['suffix']} | {r['tokens_per_s']:.0f} | {r['job_s']:.1f} | "
+              f"{r['cycles']} | {r['steps']} | {r['packed_tokens']} | {r['mean_active']:.1f} |")
+
+
+if __name__ == "__main__":
+    main()

@@ -303,3 +303,12 @@ def test_force_commit_then_lockstep(B):
     assert ls.eng.stats().committed == wl.committed_target()
     with pytest.raises(B.BlockServeError):      # no active row is left
         ls.eng.force_commit(0, {0: 1})
+
+
+def test_policy_ablation_variants_commit_the_same_tokens_count(B):
+    """The ablation driver's variants (queue order, suffix visibility) all finish workload 1 with exactly g_i tokens."""
+    from paper_2607_08930_b200 import ablate
+    wl = bs_inputs.workload(1)
+    wc, _ = both_weights(wl.shape, wl.weight_seed)
+    res = [ablate.run_variant(wl, wc, sq, sm) for sq in (True, False) for sm in (B.SUFFIX_FULL, B.SUFFIX_NONE)]
+    assert all(r["steps"] > 0 and r["tokens_per_s"] > 0 for r in res)
