@@ -8,10 +8,11 @@
 //   warp 0      TMA producer: the Q tiles once (3-D boxes: 64 dims x group heads x tokens), then 64-key K and V
 //               tiles (3-D boxes over the cache [row][kv head][dim]) through a four-stage ring
 //   warp 1      MMA issuer: per Q tile S = Q K^T into one of two TMEM buffers (the next key tile's scores are
-//               computed while this tile's softmax runs), then O += P V with P read from shared memory and V as an
-//               MN-major operand straight from the cache layout
+//               computed while this tile's softmax runs), then O += P V with P as the A operand from tensor memory
+//               and V as an MN-major operand straight from the cache layout
 //   warps 2..9  softmax, four warps per Q tile: thread r owns query row r (TMEM lane r), so row maxima and sums
-//               need no shuffles; p = 2^(s - m) goes to shared memory as bf16 in the 128B-swizzled K-major layout;
+//               need no shuffles; p = 2^(s - m) goes back to tensor memory as bf16 pairs, into the first 32 columns
+//               of the scores buffer it came from (one tcgen05.st per row, no shared-memory round trip);
 //               the output accumulates in TMEM over all key tiles and is rescaled lazily (only when a row's
 //               maximum has grown by more than 2^8), the running sum follows the same scale
 // Every wait is bounded; on a timeout the flag is raised, all roles drain, TMEM is freed.
@@ -94,6 +95,16 @@ __device__ __forceinline__ void umma_lo(unsigned d_tmem, unsigned a_lo, unsigned
       "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t}"
       ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kDescHi) : "memory");
 }
+// A operand from tensor memory (lane = row, one 32-bit column = two adjacent bf16 of the row), B from shared memory.
+__device__ __forceinline__ void umma_ts(unsigned d_tmem, unsigned a_tmem, unsigned b_lo, unsigned idesc,
+                                        unsigned accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "mov.b64 db, {%2, %5};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kDescHi) : "memory");
+}
 __device__ __forceinline__ void umma_commit(unsigned bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
@@ -131,6 +142,18 @@ __device__ __forceinline__ void tmem_st32(unsigned taddr, const float* v) {
       : "memory");
   asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
 }
+__device__ __forceinline__ void tmem_st32_words(unsigned taddr, const unsigned* w) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]), "r"(w[8]),
+        "r"(w[9]), "r"(w[10]), "r"(w[11]), "r"(w[12]), "r"(w[13]), "r"(w[14]), "r"(w[15]), "r"(w[16]), "r"(w[17]),
+        "r"(w[18]), "r"(w[19]), "r"(w[20]), "r"(w[21]), "r"(w[22]), "r"(w[23]), "r"(w[24]), "r"(w[25]), "r"(w[26]),
+        "r"(w[27]), "r"(w[28]), "r"(w[29]), "r"(w[30]), "r"(w[31])
+      : "memory");
+  asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -157,12 +180,11 @@ constexpr int KT = 64;                                   // keys per tile
 constexpr int kStages = 4;
 constexpr int kKvHalf = KT * 128;                        // KT rows x 64 bf16
 constexpr int kStageBytes = 4 * kKvHalf;                 // K halves, V halves
-constexpr int kPBytes = kHalfBytes;                      // 128 rows x 64 keys, per Q tile
-constexpr int kSmemBytes = 2 * kQBytes + kStages * kStageBytes + 2 * kPBytes + 1024;
+constexpr int kSmemBytes = 2 * kQBytes + kStages * kStageBytes + 1024;
 
 // Barrier slots
 enum { B_QFULL = 0, B_KVFULL = 1, B_KVEMPTY = B_KVFULL + kStages, B_SFULL = B_KVEMPTY + kStages,   // [tile][2]
-       B_SEMPTY = B_SFULL + 4, B_PFULL = B_SEMPTY + 4, B_OFULL = B_PFULL + 2, B_COUNT = B_OFULL + 2 };
+       B_PFULL = B_SFULL + 4, B_OFULL = B_PFULL + 2, B_COUNT = B_OFULL + 2 };
 
 __global__ void __launch_bounds__(kThreads, 1)
 k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
@@ -176,7 +198,6 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   const unsigned smem0 = (smem_u32(smem_dyn) + 1023u) & ~1023u;
   const unsigned sQ = smem0;                              // [Q tile][dim half][128 rows x 128 B]
   const unsigned sKV = sQ + 2 * kQBytes;
-  const unsigned sP = sKV + kStages * kStageBytes;        // [Q tile][128 rows x 128 B]
   const unsigned bar0 = smem_u32(&bars[0]);
   auto bar = [&](int i) { return bar0 + 8u * (unsigned)i; };
 
@@ -189,10 +210,9 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     }
     for (int i = 0; i < 4; ++i) {
       mbar_init(bar(B_SFULL + i), 1);
-      mbar_init(bar(B_SEMPTY + i), 4);     // one arrival per softmax warp of the Q tile
     }
     for (int i = 0; i < 2; ++i) {
-      mbar_init(bar(B_PFULL + i), 4);
+      mbar_init(bar(B_PFULL + i), 4);      // one arrival per softmax warp of the Q tile
       mbar_init(bar(B_OFULL + i), 1);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -260,7 +280,9 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         if (!mbar_wait(bar(B_KVFULL + s), (unsigned)(t / kStages) & 1u, abort_flag)) return false;
         const unsigned st = sKV + s * kStageBytes;
         for (int x = 0; x < n_qt; ++x) {
-          if (!mbar_wait(bar(B_SEMPTY + 2 * x + b), ((unsigned)(t >> 1) & 1u) ^ 1u, abort_flag)) return false;
+          // Scores buffer b is free: the softmax warps finished with the scores of tile t - 2 before they published
+          // its probabilities (same columns), and the P V product that read those was issued by this thread after
+          // that and before this product; the tensor pipe runs one thread's instructions in order.
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           const unsigned q_lo = desc_lo(sQ + x * kQBytes), k_lo = desc_lo(st), d_s = tmem_base + x * 256 + b * 64;
 #pragma unroll
@@ -281,12 +303,13 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         for (int x = 0; x < n_qt && ok; ++x) {
           if (!mbar_wait(bar(B_PFULL + x), (unsigned)t & 1u, abort_flag)) { ok = false; break; }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          // V as an MN-major operand: its two 64-wide dim halves are kKvHalf bytes apart (leading byte offset)
-          const unsigned p_lo = desc_lo(sP + x * kPBytes), v_lo = desc_lo(st + 2 * kKvHalf, kKvHalf);
+          // P comes from tensor memory (the first 32 columns of the scores buffer of this tile: 64 bf16 per row);
+          // V is an MN-major operand whose two 64-wide dim halves are kKvHalf bytes apart (leading byte offset)
+          const unsigned p_tm = tmem_base + x * 256 + (t & 1) * 64, v_lo = desc_lo(st + 2 * kKvHalf, kKvHalf);
           const unsigned d_o = tmem_base + x * 256 + 128;
 #pragma unroll
           for (int j = 0; j < KT / 16; ++j)         // 16 keys per step; the output accumulates over all key tiles
-            umma_lo(d_o, p_lo + 2 * j, v_lo + j * (2048 >> 4), idesc_o, (t | j) ? 1u : 0u);
+            umma_ts(d_o, p_tm + j * 8, v_lo + j * (2048 >> 4), idesc_o, (t | j) ? 1u : 0u);
           umma_commit(bar(B_OFULL + x));
         }
         if (ok) umma_commit(bar(B_KVEMPTY + (t % kStages)));
@@ -302,7 +325,6 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     if (x < n_qt) {
       const unsigned t_lane = tmem_base + ((unsigned)(q * 32) << 16) + x * 256;
       const unsigned t_out = t_lane + 128;
-      const unsigned sPx = sP + x * kPBytes + r * 128;
       const float sc = 1.4426950408889634f * rsqrtf((float)DH);
       const bool warp_has_rows = q * 32 < nrows;        // warps without valid rows only keep the barriers moving
       float m = -INFINITY, l = 0.f;                     // m: the maximum the accumulator is currently scaled by
@@ -355,43 +377,32 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           }
           l = l * f + (((rs8[0] + rs8[1]) + (rs8[2] + rs8[3])) + ((rs8[4] + rs8[5]) + (rs8[6] + rs8[7])));
         }
-        // the previous P V product must have finished before P is overwritten or the accumulator touched
+        // the previous P V product must have finished before the accumulator is touched
         if (t > 0 && !mbar_wait(bar(B_OFULL + x), (unsigned)(t - 1) & 1u, abort_flag)) { ok = false; break; }
-        if (warp_has_rows) {
+        if (rescale && t > 0) {                     // warp-uniform
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          if (rescale && t > 0) {
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-              float o[32];
-              tmem_ld32(t_out + c * 32, o);
+          for (int c = 0; c < 4; ++c) {
+            float o[32];
+            tmem_ld32(t_out + c * 32, o);
 #pragma unroll
-              for (int j = 0; j < 32; ++j) o[j] *= f;
-              tmem_st32(t_out + c * 32, o);
-            }
-          }
-          // P as bf16, rows of 128 bytes, 16-byte chunks XOR (row % 8): the 128B-swizzled K-major layout
-#pragma unroll
-          for (int g = 0; g < 8; ++g) {
-            const float* e = v + g * 8;
-            const __nv_bfloat162 p0 = __floats2bfloat162_rn(e[0], e[1]);
-            const __nv_bfloat162 p1 = __floats2bfloat162_rn(e[2], e[3]);
-            const __nv_bfloat162 p2 = __floats2bfloat162_rn(e[4], e[5]);
-            const __nv_bfloat162 p3 = __floats2bfloat162_rn(e[6], e[7]);
-            const unsigned chunk = (unsigned)g ^ (unsigned)(r & 7);
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sPx + chunk * 16),
-                         "r"(*reinterpret_cast<const unsigned*>(&p0)), "r"(*reinterpret_cast<const unsigned*>(&p1)),
-                         "r"(*reinterpret_cast<const unsigned*>(&p2)), "r"(*reinterpret_cast<const unsigned*>(&p3))
-                         : "memory");
+            for (int j = 0; j < 32; ++j) o[j] *= f;
+            tmem_st32(t_out + c * 32, o);
           }
         }
-        // the scores buffer is free; P is visible to the tensor core (async proxy) once fenced
+        if (warp_has_rows) {
+          // P as bf16 pairs into the first 32 columns of this tile's scores buffer: the A operand of the P V product
+          unsigned w[32];
+#pragma unroll
+          for (int c = 0; c < 32; ++c) {
+            const __nv_bfloat162 pr = __floats2bfloat162_rn(v[2 * c], v[2 * c + 1]);
+            w[c] = *reinterpret_cast<const unsigned*>(&pr);
+          }
+          tmem_st32_words(t_lane + b * 64, w);
+        }
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
-        if (lane == 0) {
-          mbar_arrive(bar(B_SEMPTY + 2 * x + b));
-          mbar_arrive(bar(B_PFULL + x));
-        }
+        if (lane == 0) mbar_arrive(bar(B_PFULL + x));
       }
       if (ok && n_tiles > 0 && mbar_wait(bar(B_OFULL + x), (unsigned)(n_tiles - 1) & 1u, abort_flag) &&
           warp_has_rows) {
