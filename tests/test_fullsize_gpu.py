@@ -91,3 +91,31 @@ def test_llada_stream_full_depth_first_cycle_sampled_request(B):
     print(f"cfg3 full depth, {n} rows active, request {first.req_id} (p={first.p}, alpha={first.alpha:.2f}): "
           f"{ls.summary()}")
     assert ls.rows_checked > 0 and ls.max_logit_err < logit_tol(wl.shape.n_layers)
+
+
+@pytest.mark.parametrize("shape_name", ["dream", "llada"])
+def test_repeated_runs_are_bit_identical_at_benchmark_width(B, shape_name):
+    """Sixteen requests on a 4-layer replica of the benchmark shapes, served twice from scratch: every kernel sums in
+    a fixed order and every hand-off between roles is fenced, so the committed tokens, the step count and the packed
+    token count repeat exactly (a race in a pipeline shows up here as a difference or as BS_E_TIMEOUT)."""
+    shape = (bs_inputs.DREAM_7B if shape_name == "dream" else bs_inputs.LLADA_8B).with_layers(4)
+    rng = np.random.default_rng(5)
+    n = 16
+    ps = rng.integers(40, 700, size=n)
+    gs = rng.choice([64, 96], size=n)
+    al = rng.choice([2.0, 8.0, 30.0], size=n)
+    wl = bs_inputs.custom_workload(shape, ps, gs, al, seed=21, tau=0.9, max_batch=n)
+    w = bs_inputs.make_weights(shape, 99, device="cuda")
+    runs = []
+    for _ in range(2):
+        eng = B.engine_for_workload(wl, w)
+        for r in wl.requests:
+            eng.admit(r.req_id, r.prompt, r.g, r.alpha)
+        eng.run()
+        st = eng.stats()
+        assert st.committed == wl.committed_target()
+        runs.append(([eng.read_tokens(r.req_id)[0] for r in wl.requests], st.steps, st.packed_tokens))
+        eng.close()
+    assert runs[0][1:] == runs[1][1:]
+    for a, b in zip(runs[0][0], runs[1][0]):
+        assert (a == b).all()
