@@ -176,12 +176,23 @@ def confidence(logits: np.ndarray, mask_id: int):
     return tok, conf
 
 
-def commit_set(conf: np.ndarray, tau: float) -> np.ndarray:
+def transfer_quota(L: int, S: int, s: int) -> int:
+    """Per-step transfer quota of Section 2.5: the L masked tokens a block starts
+    with are spread uniformly over S diffusion steps, the first L mod S steps
+    taking one more.  S = L gives one token per step."""
+    if s >= S:
+        return 1
+    return L // S + (1 if s < L % S else 0)
+
+
+def commit_set(conf: np.ndarray, tau: float, quota: int = 1) -> np.ndarray:
     """Boolean mask over the still-masked positions of one block (in position
-    order): everything strictly above tau, plus the position of highest
-    confidence (lowest position on ties) so that every step commits >= 1."""
+    order): everything strictly above tau, plus the ``quota`` positions of
+    highest confidence (lower position first on ties), so that every step
+    commits at least its quota (all that is left, if fewer remain)."""
     sel = conf > F32(tau)
-    sel[int(np.argmax(conf))] = True
+    order = np.argsort(-conf, kind="stable")
+    sel[order[:max(int(quota), 1)]] = True
     return sel
 
 
@@ -298,7 +309,7 @@ class StepRecord:
 
 def denoise_step(model: Model, r: ReqState, L: int, tau: float, suffix_mode: int = SUFFIX_FULL,
                  keep_logits: bool = False, override_commit: Optional[np.ndarray] = None,
-                 override_tok: Optional[np.ndarray] = None) -> StepRecord:
+                 override_tok: Optional[np.ndarray] = None, steps_per_block: Optional[int] = None) -> StepRecord:
     """One denoise step of one active request whose block is not done.
 
     ``override_commit`` / ``override_tok`` let a lockstep comparison make the
@@ -317,7 +328,8 @@ def denoise_step(model: Model, r: ReqState, L: int, tau: float, suffix_mode: int
     z[:, model.mask_id] = -np.inf
     part = np.partition(z, -2, axis=-1)
     gap = (part[:, -1] - part[:, -2]).astype(F32)
-    sel = commit_set(conf.copy(), tau)
+    S = L if not steps_per_block else int(steps_per_block)
+    sel = commit_set(conf.copy(), tau, transfer_quota(L, S, r.s))
     rec = StepRecord(r.req_id, r.b, r.s, positions, logits if keep_logits else None,
                      tok.copy(), conf.copy(), sel.copy(), gap)
     use_sel = sel if override_commit is None else np.asarray(override_commit, dtype=bool)
@@ -474,8 +486,10 @@ def build_indices(active: Sequence[ReqState], L: int, suffix_mode: int = SUFFIX_
 
 class Engine:
     def __init__(self, model: Model, L: int, tau: float, token_budget: int, max_batch: int,
-                 kv_capacity: int, suffix_mode: int = SUFFIX_FULL, sort_queue: bool = True):
+                 kv_capacity: int, suffix_mode: int = SUFFIX_FULL, sort_queue: bool = True,
+                 steps_per_block: Optional[int] = None):
         self.model, self.L, self.tau, self.suffix_mode = model, L, tau, suffix_mode
+        self.steps_per_block = steps_per_block
         self.sched = Scheduler(L, token_budget, max_batch, kv_capacity, sort_queue)
         self.by_id: Dict[int, ReqState] = {}
         self.total_committed = 0
@@ -496,7 +510,8 @@ class Engine:
         recs = []
         for r in self.sched.active:
             if r.mask != 0:
-                rec = denoise_step(self.model, r, self.L, self.tau, self.suffix_mode, keep_logits)
+                rec = denoise_step(self.model, r, self.L, self.tau, self.suffix_mode, keep_logits,
+                                   steps_per_block=self.steps_per_block)
                 self.total_committed += int(rec.committed.sum())
                 recs.append(rec)
         self.total_steps += 1

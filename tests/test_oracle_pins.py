@@ -557,3 +557,42 @@ def test_workload_generators_match_the_stated_shapes():
     al = np.array([r.alpha for r in w5.requests])
     assert len(al) == 1024 and set(np.unique(al)) == {0.7, 16.0} and 0.75 < (al == 16.0).mean() < 0.85
     assert {r.g for r in w5.requests} == {128, 256, 512}
+
+
+def test_transfer_quota_spreads_the_block_over_the_steps():
+    """Section 2.5: the block's L masked tokens are distributed uniformly over S steps."""
+    for L in (1, 7, 16, 32):
+        for S in range(1, L + 1):
+            q = [O.transfer_quota(L, S, s) for s in range(S)]
+            assert sum(q) == L and max(q) - min(q) <= 1 and q == sorted(q, reverse=True)
+        assert [O.transfer_quota(L, L, s) for s in range(L)] == [1] * L
+    assert [O.transfer_quota(32, 5, s) for s in range(5)] == [7, 7, 6, 6, 6]
+    assert [O.transfer_quota(32, 8, s) for s in range(8)] == [4] * 8
+
+
+def test_commit_set_with_quota_is_threshold_union_top_q():
+    c = np.array([0.30, 0.95, 0.10, 0.95, 0.50, 0.20], F32)
+    # brute force: threshold set united with the q largest (lower position first among equals)
+    for tau in (0.0, 0.4, 0.9, 0.99):
+        for q in range(1, 8):
+            rank = sorted(range(len(c)), key=lambda i: (-float(c[i]), i))[:q]
+            want = [bool(c[i] > np.float32(tau)) or i in rank for i in range(len(c))]
+            assert O.commit_set(c.copy(), tau, q).tolist() == want
+    assert O.commit_set(c.copy(), 0.99, 1).tolist() == [False, True, False, False, False, False]
+    assert O.commit_set(c.copy(), 0.99, 3).tolist() == [False, True, False, True, True, False]
+
+
+def test_quota_finishes_every_block_within_S_steps():
+    """With quota q_s every block of a request is done after at most S steps, whatever the confidences."""
+    rng = np.random.default_rng(3)
+    for L, S in ((32, 8), (32, 5), (16, 16), (12, 4)):
+        for blk in (L, L - 3 if L > 3 else L):          # a full block and a ragged last block
+            mask = np.ones(blk, bool)
+            for s in range(S):
+                if not mask.any():
+                    break
+                conf = rng.uniform(0.0, 0.5, size=int(mask.sum())).astype(F32)      # never above tau
+                sel = O.commit_set(conf, 0.9, O.transfer_quota(L, S, s))
+                idx = np.nonzero(mask)[0]
+                mask[idx[sel]] = False
+            assert not mask.any()
