@@ -65,6 +65,9 @@ typedef struct {
   int suffix_mode;               /* BS_SUFFIX_FULL: a row sees prompt + all g_i positions (future blocks as mask
                                     tokens); BS_SUFFIX_NONE: a row ends with its current block (row width of Eq. 1) */
   int sort_queue;                /* 1: pending queue ascending in p_i, ties by submission (Section 2.4); 0: arrival order */
+  int steps_per_block;           /* S of Section 2.5: the block's L masked tokens are spread uniformly over S steps
+                                    (step s of a block commits the positions above tau united with its
+                                    floor(L/S) + [s < L mod S] most confident ones); 0 or L: one per step */
 } bs_config;
 
 /* All weights are bf16, row-major [out_features, in_features], device memory.

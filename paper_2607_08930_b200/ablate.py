@@ -1,6 +1,6 @@
 """Throughput-only ablations of the serving policy on a synthetic workload (Section 4's research questions on queue
 order and block length, in the form that needs no trained weights): sorted vs submission-order queue, suffix
-visibility FULL vs NONE, block length L.  Prints one JSON line per variant and a markdown table.
+visibility FULL vs NONE, block length L, and optionally the transfer quota S < L of Section 2.5.  Prints one JSON line per variant and a markdown table.
 
     python -m paper_2607_08930_b200.ablate --workload 3
 """
@@ -19,8 +19,9 @@ import bs_inputs  # noqa: E402
 from paper_2607_08930_b200 import binding as B, build  # noqa: E402
 
 
-def run_variant(wl, weights, sort_queue: bool, suffix_mode: int):
-    eng = B.engine_for_workload(wl, weights, sort_queue=sort_queue, suffix_mode=suffix_mode)
+def run_variant(wl, weights, sort_queue: bool, suffix_mode: int, steps_per_block: int = 0):
+    eng = B.engine_for_workload(wl, weights, sort_queue=sort_queue, suffix_mode=suffix_mode,
+                                steps_per_block=steps_per_block)
     for r in wl.requests:
         eng.admit(r.req_id, r.prompt, r.g, r.alpha, r.start_block, r.gen_prefix)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -43,6 +44,8 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--workload", type=int, default=3)
     ap.add_argument("--block-lens", type=int, nargs="+", default=[32, 16])
+    ap.add_argument("--steps-per-block", type=int, nargs="*", default=[],
+                    help="extra variants with a transfer quota S < L (sorted queue, full suffix)")
     args = ap.parse_args()
     build.build()
     base = bs_inputs.workload(args.workload)
@@ -60,6 +63,12 @@ def main():
                            suffix="full" if suffix_mode == B.SUFFIX_FULL else "none")
                 print(json.dumps(res), flush=True)
                 rows.append(res)
+    for S in args.steps_per_block:
+        run_variant(base, weights, True, B.SUFFIX_FULL, S)
+        res = run_variant(base, weights, True, B.SUFFIX_FULL, S)
+        res.update(workload=base.name, block_len=base.block_len, queue=f"sorted, S = {S}", suffix="full")
+        print(json.dumps(res), flush=True)
+        rows.append(res)
     print("\n| L | queue | suffix | committed tokens/s | job s | cycles | steps | packed tokens | mean |A| |")
     print("|---|---|---|---|---|---|---|---|---|")
     for r in rows:

@@ -105,6 +105,7 @@ const char* check_config(const bs_config& c) {
   if (c.kv_capacity_tokens > (1ll << 30)) return "kv_capacity_tokens too large";
   if (c.suffix_mode != BS_SUFFIX_FULL && c.suffix_mode != BS_SUFFIX_NONE) return "bad suffix_mode";
   if (!(c.tau >= 0.f)) return "tau must be >= 0";
+  if (c.steps_per_block < 0 || c.steps_per_block > c.block_len) return "steps_per_block must be in [0, block_len]";
   return nullptr;
 }
 
@@ -282,6 +283,7 @@ int bs_init_model(const bs_config* cfg, const bs_weights* w, void* kv, void* wor
   st.L = cfg->block_len; st.max_batch = cfg->max_batch; st.max_requests = cfg->max_requests;
   st.max_row_tokens = cfg->max_row_tokens; st.suffix_mode = cfg->suffix_mode; st.mask_id = cfg->mask_id;
   st.vocab = cfg->vocab; st.beta = cfg->token_budget; st.kv_capacity = cfg->kv_capacity_tokens; st.tau = cfg->tau;
+  st.S = cfg->steps_per_block > 0 ? cfg->steps_per_block : cfg->block_len;
   st.q_tile = attention_q_tile(cfg->n_q_heads, cfg->n_kv_heads, cfg->head_dim);
   e->gemm_scratch.partial = e->ws.partial;
   e->gemm_scratch.partial_floats = kPartialFloats;

@@ -235,8 +235,8 @@ __global__ void __launch_bounds__(kSchedThreads) k_sched(DevState st) {
   build_index(st, st.hdr[H_PARITY] ^ 1, n, smi);
 }
 
-// Commit rule per request (one warp per row): positions with conf > tau, plus the position of highest
-// confidence (lowest position on ties), so that every step commits at least one token.
+// Commit rule per request (one warp per row): positions with conf > tau, plus the step's quota of most confident
+// positions (lower position first on ties), so that every step commits at least its quota (one when S = L).
 __global__ void __launch_bounds__(kSchedThreads) k_commit_index(DevState st) {
   __shared__ int smi[33];
   __shared__ int s_count;
@@ -258,15 +258,23 @@ __global__ void __launch_bounds__(kSchedThreads) k_commit_index(DevState st) {
       tok = st.out_tok[parity][base + lane];
       bit = st.lm_slot[parity][base + lane];
     }
-    float bc = conf;
-    int bj = lane;
+    // transfer quota of this step (Section 2.5): the block's L masked tokens spread uniformly over S steps
+    const int s_in_block = st.row_s[r];
+    const int quota = s_in_block >= st.S ? 1 : st.L / st.S + (s_in_block < st.L % st.S ? 1 : 0);
+    bool picked = false;
+    for (int it = 0; it < quota; ++it) {          // warp-uniform trip count
+      float bc = (lane < nm && !picked) ? conf : -2.0f;
+      int bj = lane;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const float oc = __shfl_xor_sync(0xffffffffu, bc, o);
-      const int oj = __shfl_xor_sync(0xffffffffu, bj, o);
-      if (oc > bc || (oc == bc && oj < bj)) { bc = oc; bj = oj; }
+      for (int o = 16; o > 0; o >>= 1) {
+        const float oc = __shfl_xor_sync(0xffffffffu, bc, o);
+        const int oj = __shfl_xor_sync(0xffffffffu, bj, o);
+        if (oc > bc || (oc == bc && oj < bj)) { bc = oc; bj = oj; }
+      }
+      if (bc < -1.5f) break;                      // nothing left to pick (warp-uniform)
+      if (lane == bj) picked = true;
     }
-    const bool sel = lane < nm && (conf > st.tau || lane == bj);
+    const bool sel = lane < nm && (conf > st.tau || picked);
     const int slot = st.row_slot[r];
     if (sel) {
       const int lo = st.req_p[slot] + st.req_b[slot] * st.L;

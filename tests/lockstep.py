@@ -76,14 +76,18 @@ class Lockstep:
     adopts the engine's mask word after each step, since the oracle does not run their forward."""
 
     def __init__(self, wl, weights_cuda, weights_np, suffix_mode=0, kv_capacity=None, sort_queue=True, track=None,
-                 model=None):
+                 model=None, steps_per_block=0):
         self.wl = wl
         self.track = None if track is None else set(track)
+        # the near-tie classes below are written for one forced token per step; a general transfer quota is checked
+        # through the exact commit-rule and bookkeeping comparisons of untracked rows
+        assert not steps_per_block or steps_per_block == wl.block_len or self.track == set()
+        self.S = steps_per_block if steps_per_block else wl.block_len
         self.eng = B.engine_for_workload(wl, weights_cuda, kv_capacity_tokens=kv_capacity, suffix_mode=suffix_mode,
-                                         sort_queue=sort_queue)
+                                         sort_queue=sort_queue, steps_per_block=steps_per_block)
         self.model = model if model is not None else O.model_from_weights(wl.shape, weights_np)
         self.ora = O.Engine(self.model, wl.block_len, wl.tau, wl.token_budget, wl.max_batch,
-                            self.eng.cfg.kv_capacity_tokens, suffix_mode, sort_queue)
+                            self.eng.cfg.kv_capacity_tokens, suffix_mode, sort_queue, steps_per_block=steps_per_block)
         self.suffix_mode = suffix_mode
         self.excluded = {"tau": 0, "top2": 0, "forced": 0, "noise": 0}
         self.conf_rows_within_tol = 0
@@ -150,9 +154,10 @@ class Lockstep:
             nm = bin(r.mask).count("1")
             gt, gc, gs = g_tok[k:k + nm], g_conf[k:k + nm], g_commit[k:k + nm]
             where = f"req {r.req_id} block {r.b} step {r.s}"
+            quota = O.transfer_quota(self.wl.block_len, self.S, r.s)
             if self.track is not None and r.req_id not in self.track:
                 # untracked row: integer bookkeeping only; the commit rule is still checked on the engine's own data
-                assert (O.commit_set(gc.copy(), self.wl.tau) == gs).all(), f"commit rule ({where})"
+                assert (O.commit_set(gc.copy(), self.wl.tau, quota) == gs).all(), f"commit rule ({where})"
                 slots = [j for j in range(32) if (r.mask >> j) & 1]
                 new_mask = r.mask
                 for i, j in enumerate(slots):
@@ -167,7 +172,8 @@ class Lockstep:
             # the record holds what the oracle computes on its own; the oracle then advances with the engine's
             # decisions (identical unless a near tie is counted below)
             probe = O.denoise_step(self.model, r, self.wl.block_len, self.wl.tau, self.suffix_mode,
-                                   keep_logits=True, override_commit=gs, override_tok=gt)
+                                   keep_logits=True, override_commit=gs, override_tok=gt,
+                                   steps_per_block=self.S)
             if g_logits is not None:
                 zl = g_logits[k:k + nm]
             else:       # only the tracked rows' logits are read back
@@ -181,7 +187,7 @@ class Lockstep:
             tok2, conf2 = O.confidence(zl, mask_id)
             assert (gt == tok2).all(), f"argmax differs from the oracle's on identical logits ({where})"
             assert (np.abs(gc - conf2) <= 1e-4 * conf2).all(), f"confidence kernel error ({where})"
-            assert (O.commit_set(gc.copy(), self.wl.tau) == gs).all(), f"commit rule differs on identical data ({where})"
+            assert (O.commit_set(gc.copy(), self.wl.tau, quota) == gs).all(), f"commit rule differs on identical data ({where})"
             # (3) against the oracle's own trajectory
             dln = np.abs(np.log(gc.astype(np.float64)) - np.log(probe.conf.astype(np.float64)))
             assert (dln <= 2.0 * dev + 1e-4).all(), f"confidence outside the Lipschitz bound ({where})"

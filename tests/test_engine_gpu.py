@@ -312,3 +312,34 @@ def test_policy_ablation_variants_commit_the_same_tokens_count(B):
     wc, _ = both_weights(wl.shape, wl.weight_seed)
     res = [ablate.run_variant(wl, wc, sq, sm) for sq in (True, False) for sm in (B.SUFFIX_FULL, B.SUFFIX_NONE)]
     assert all(r["steps"] > 0 and r["tokens_per_s"] > 0 for r in res)
+
+
+@pytest.mark.parametrize("S", [8, 5, 1])
+def test_transfer_quota_spreads_a_block_over_S_steps(B, S):
+    """Section 2.5's per-step quota: every step commits the positions above tau united with its quota of most
+    confident ones; checked exactly on the engine's own confidences (commit flags, mask words, step counters), and
+    every block finishes within S steps."""
+    from lockstep import Lockstep
+    shape = bs_inputs.TINY
+    wl = bs_inputs.custom_workload(shape, [9, 17, 30, 5], [64, 40, 33, 96], [4.0, 8.0, 2.0, 1.0], seed=12, tau=0.95,
+                                   max_batch=3)
+    wc, wn = both_weights(shape, 6)
+    ls = Lockstep(wl, wc, wn, track=set(), steps_per_block=S)
+    ls.admit(wl.requests)
+    while True:
+        _, _, n = ls.evict_refill()
+        if n == 0:
+            break
+        steps = 0
+        while True:
+            ls.step()
+            steps += 1
+            done = ls.eng.block_done()
+            assert done == ls.ora.block_done()
+            if done:
+                break
+        assert steps <= S
+    assert ls.eng.stats().committed == wl.committed_target()
+    for r in wl.requests:
+        toks, state = ls.eng.read_tokens(r.req_id)
+        assert state == B.REQ_FINISHED and (toks != shape.mask_id).all()
