@@ -43,7 +43,7 @@ def run_variant(wl, weights, sort_queue: bool, suffix_mode: int, steps_per_block
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--workload", type=int, default=3)
-    ap.add_argument("--block-lens", type=int, nargs="+", default=[32, 16])
+    ap.add_argument("--block-lens", type=int, nargs="*", default=[32, 16])
     ap.add_argument("--steps-per-block", type=int, nargs="*", default=[],
                     help="extra variants with a transfer quota S < L (sorted queue, full suffix)")
     args = ap.parse_args()
