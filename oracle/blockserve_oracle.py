@@ -379,9 +379,10 @@ class Scheduler:
     block-boundary advance / evict / stable compaction / refill."""
 
     def __init__(self, L: int, token_budget: int, max_batch: int, kv_capacity: int,
-                 sort_queue: bool = True):
+                 sort_queue: bool = True, eos_id: Optional[int] = None):
         self.L, self.beta, self.max_batch, self.kv_capacity = L, token_budget, max_batch, kv_capacity
         self.sort_queue = sort_queue
+        self.eos_id = None if eos_id is None or eos_id < 0 else int(eos_id)
         self.pending: List[ReqState] = []
         self.active: List[ReqState] = []
         self.finished: List[ReqState] = []
@@ -404,14 +405,18 @@ class Scheduler:
 
     def evict_refill(self, first: bool = False):
         """Block boundary: b_i += 1 for every active row (not on the very first
-        fill of a row), evict rows with b_i >= K_i, keep survivors in order,
+        fill of a row), evict rows with b_i >= K_i or CheckEOS(r_i) (Algorithm 1:
+        an end-of-sequence token among the blocks generated so far; off when
+        no eos_id is configured), keep survivors in order,
         then admit the head of P while Eq. 1 stays within the budget, the batch
         cap holds and the KV arena has a hole; admitted rows are appended."""
         L = self.L
         evicted, survivors = [], []
         for r in self.active:
             r.b += 1
-            if r.b >= r.n_blocks(L):
+            done_upto = min(r.p + r.b * L, r.p + r.g)
+            has_eos = self.eos_id is not None and bool((r.tokens[r.p:done_upto] == self.eos_id).any())
+            if r.b >= r.n_blocks(L) or has_eos:
                 evicted.append(r.req_id)
                 r.kv_base = -1
                 self.finished.append(r)
@@ -487,10 +492,10 @@ def build_indices(active: Sequence[ReqState], L: int, suffix_mode: int = SUFFIX_
 class Engine:
     def __init__(self, model: Model, L: int, tau: float, token_budget: int, max_batch: int,
                  kv_capacity: int, suffix_mode: int = SUFFIX_FULL, sort_queue: bool = True,
-                 steps_per_block: Optional[int] = None):
+                 steps_per_block: Optional[int] = None, eos_id: Optional[int] = None):
         self.model, self.L, self.tau, self.suffix_mode = model, L, tau, suffix_mode
         self.steps_per_block = steps_per_block
-        self.sched = Scheduler(L, token_budget, max_batch, kv_capacity, sort_queue)
+        self.sched = Scheduler(L, token_budget, max_batch, kv_capacity, sort_queue, eos_id)
         self.by_id: Dict[int, ReqState] = {}
         self.total_committed = 0
         self.total_steps = 0

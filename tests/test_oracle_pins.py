@@ -596,3 +596,34 @@ def test_quota_finishes_every_block_within_S_steps():
                 idx = np.nonzero(mask)[0]
                 mask[idx[sel]] = False
             assert not mask.any()
+
+
+def test_check_eos_evicts_at_the_block_boundary_after_the_token_appears():
+    """Algorithm 1: a request leaves A when b_i >= K_i or CheckEOS(r_i); the check runs at block boundaries only."""
+    L, EOS = 32, 7
+    s = O.Scheduler(L, 0, 4, 1 << 20, eos_id=EOS)
+    for i in range(3):
+        s.submit(sched_req(i, 10 + i, 128))            # K_i = 4 blocks each
+    s.evict_refill()
+    assert [r.req_id for r in s.active] == [0, 1, 2]
+    # request 1 generates the end-of-sequence token in its first block, request 2 in its second
+    for r in s.active:
+        r.tokens[r.p:r.p + L] = 3
+        r.mask = 0
+    s.active[1].tokens[s.active[1].p + 5] = EOS
+    ev, ad = s.evict_refill()
+    assert ev == [1] and [r.req_id for r in s.active] == [0, 2]
+    for r in s.active:
+        r.tokens[r.p + L:r.p + 2 * L] = 3
+        r.mask = 0
+    s.active[1].tokens[s.active[1].p + 2 * L - 1] = EOS        # last position of the second block
+    ev, ad = s.evict_refill()
+    assert ev == [2] and [r.req_id for r in s.active] == [0]
+    # without an eos id nothing but b_i >= K_i evicts
+    s2 = O.Scheduler(L, 0, 4, 1 << 20)
+    s2.submit(sched_req(0, 10, 128))
+    s2.evict_refill()
+    s2.active[0].tokens[s2.active[0].p:s2.active[0].p + L] = EOS
+    s2.active[0].mask = 0
+    ev, ad = s2.evict_refill()
+    assert ev == [] and len(s2.active) == 1
