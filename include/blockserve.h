@@ -68,6 +68,9 @@ typedef struct {
   int steps_per_block;           /* S of Section 2.5: the block's L masked tokens are spread uniformly over S steps
                                     (step s of a block commits the positions above tau united with its
                                     floor(L/S) + [s < L mod S] most confident ones); 0 or L: one per step */
+  int eos_id;                    /* CheckEOS of Algorithm 1: at a block boundary a request whose finished blocks hold
+                                    this token id leaves the active set (its later positions stay masked, its state
+                                    becomes BS_REQ_FINISHED); < 0: off, every request generates exactly g_i tokens */
 } bs_config;
 
 /* All weights are bf16, row-major [out_features, in_features], device memory.

@@ -49,6 +49,7 @@ struct DevState {
   int L, max_batch, max_requests, max_row_tokens, suffix_mode, mask_id, vocab;
   int q_tile;           // query tokens per attention work item
   int S;                // diffusion steps per block (transfer quota of Section 2.5); S = L: one forced token per step
+  int eos_id;           // CheckEOS of Algorithm 1 (< 0: off)
   long long beta, kv_capacity;
   float tau;
   int* hdr;             // [kHdrInts] followed directly by row_mask[max_batch]

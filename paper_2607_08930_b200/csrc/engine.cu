@@ -106,6 +106,7 @@ const char* check_config(const bs_config& c) {
   if (c.suffix_mode != BS_SUFFIX_FULL && c.suffix_mode != BS_SUFFIX_NONE) return "bad suffix_mode";
   if (!(c.tau >= 0.f)) return "tau must be >= 0";
   if (c.steps_per_block < 0 || c.steps_per_block > c.block_len) return "steps_per_block must be in [0, block_len]";
+  if (c.eos_id >= c.vocab || c.eos_id == c.mask_id) return "eos_id must be a token id other than the mask id, or negative";
   return nullptr;
 }
 
@@ -284,6 +285,7 @@ int bs_init_model(const bs_config* cfg, const bs_weights* w, void* kv, void* wor
   st.max_row_tokens = cfg->max_row_tokens; st.suffix_mode = cfg->suffix_mode; st.mask_id = cfg->mask_id;
   st.vocab = cfg->vocab; st.beta = cfg->token_budget; st.kv_capacity = cfg->kv_capacity_tokens; st.tau = cfg->tau;
   st.S = cfg->steps_per_block > 0 ? cfg->steps_per_block : cfg->block_len;
+  st.eos_id = cfg->eos_id;
   st.q_tile = attention_q_tile(cfg->n_q_heads, cfg->n_kv_heads, cfg->head_dim);
   e->gemm_scratch.partial = e->ws.partial;
   e->gemm_scratch.partial_floats = kPartialFloats;

@@ -139,7 +139,8 @@ __global__ void __launch_bounds__(kSchedThreads) k_sched(DevState st) {
   const int n0 = st.hdr[H_N_ACTIVE];
   const int L = st.L;
 
-  // ---- advance every active row by one block, evict finished rows, compact (order preserved) ----
+  // ---- advance every active row by one block, evict finished rows (b_i >= K_i or CheckEOS), compact (order
+  // preserved) ----
   int keep = 0, slot = -1, kvb = 0;
   if (i < n0) {
     slot = st.row_slot[i];
@@ -148,6 +149,13 @@ __global__ void __launch_bounds__(kSchedThreads) k_sched(DevState st) {
     st.req_b[slot] = b;
     const int K = (st.req_g[slot] + L - 1) / L;          // K_i = ceil(g_i / L)
     keep = b < K;
+    if (keep && st.eos_id >= 0) {                        // CheckEOS over the blocks finished so far
+      const int p = st.req_p[slot];
+      const int* row = st.tokens + (size_t)slot * st.max_row_tokens;
+      const int upto = min(p + b * L, p + st.req_g[slot]);
+      for (int t = p; t < upto; ++t)
+        if (row[t] == st.eos_id) { keep = 0; break; }
+    }
     if (!keep) st.req_state[slot] = 2;
   }
   int n_keep;

@@ -343,3 +343,44 @@ def test_transfer_quota_spreads_a_block_over_S_steps(B, S):
     for r in wl.requests:
         toks, state = ls.eng.read_tokens(r.req_id)
         assert state == B.REQ_FINISHED and (toks != shape.mask_id).all()
+
+
+def test_check_eos_evicts_requests_early_in_lockstep(B):
+    """CheckEOS of Algorithm 1.  The end-of-sequence id is chosen from a first run without it (the most frequent
+    generated token), so that several requests meet it; the second run, in full lockstep, must evict them at the
+    block boundary after the token appears, on both sides alike."""
+    from collections import Counter
+    from lockstep import Lockstep
+    shape = bs_inputs.TINY
+    rng = np.random.default_rng(44)
+    n = 8
+    wl = bs_inputs.custom_workload(shape, rng.integers(5, 60, size=n), [128] * n, rng.choice([2.0, 6.0], size=n),
+                                   seed=31, tau=0.9, max_batch=4)
+    wc, wn = both_weights(shape, 8)
+    eng = B.engine_for_workload(wl, wc)
+    for r in wl.requests:
+        eng.admit(r.req_id, r.prompt, r.g, r.alpha)
+    _drive(eng)
+    gen = np.concatenate([eng.read_tokens(r.req_id)[0][r.p:r.p + 64] for r in wl.requests])
+    eos = int(Counter(gen.tolist()).most_common(1)[0][0])
+    eng.close()
+
+    ls = Lockstep(wl, wc, wn, eos_id=eos)
+    ls.admit(wl.requests)
+    ls.run()
+    ls.check_tokens()
+    early = 0
+    for r in wl.requests:
+        toks, state = ls.eng.read_tokens(r.req_id)
+        assert state == B.REQ_FINISHED
+        g = toks[r.p:]
+        if (g == shape.mask_id).any():
+            early += 1
+            first_masked = int(np.nonzero(g == shape.mask_id)[0][0])
+            assert first_masked % wl.block_len == 0                         # whole blocks only
+            assert (g[first_masked:] == shape.mask_id).all()
+            assert (g[:first_masked] == eos).any()                          # an end-of-sequence token came before
+            assert not (g[:first_masked - wl.block_len] == eos).any()       # and only in the last finished block
+    assert early >= 1
+    assert ls.eng.stats().committed < wl.committed_target()
+    assert ls.eng.stats().committed == sum(r.committed for r in ls.ora.by_id.values())
