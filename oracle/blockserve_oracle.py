@@ -379,9 +379,10 @@ class Scheduler:
     block-boundary advance / evict / stable compaction / refill."""
 
     def __init__(self, L: int, token_budget: int, max_batch: int, kv_capacity: int,
-                 sort_queue: bool = True, eos_id: Optional[int] = None):
+                 sort_queue: bool = True, eos_id: Optional[int] = None, static_groups: bool = False):
         self.L, self.beta, self.max_batch, self.kv_capacity = L, token_budget, max_batch, kv_capacity
         self.sort_queue = sort_queue
+        self.static_groups = bool(static_groups)     # comparison policy of Section 3.1: fixed groups, no refill
         self.eos_id = None if eos_id is None or eos_id < 0 else int(eos_id)
         self.pending: List[ReqState] = []
         self.active: List[ReqState] = []
@@ -424,7 +425,9 @@ class Scheduler:
                 survivors.append(r)
         self.active = survivors
         admitted = []
-        while self.pending and len(self.active) < self.max_batch:
+        # static groups: the next group starts only when every request of the current one has finished
+        refill = not (self.static_groups and self.active)
+        while refill and self.pending and len(self.active) < self.max_batch:
             c = self.pending[0]
             widths = [r.width(L) for r in self.active] + [c.width(L)]
             if self.beta > 0 and batch_cost(widths) > self.beta:
@@ -492,10 +495,10 @@ def build_indices(active: Sequence[ReqState], L: int, suffix_mode: int = SUFFIX_
 class Engine:
     def __init__(self, model: Model, L: int, tau: float, token_budget: int, max_batch: int,
                  kv_capacity: int, suffix_mode: int = SUFFIX_FULL, sort_queue: bool = True,
-                 steps_per_block: Optional[int] = None, eos_id: Optional[int] = None):
+                 steps_per_block: Optional[int] = None, eos_id: Optional[int] = None, static_groups: bool = False):
         self.model, self.L, self.tau, self.suffix_mode = model, L, tau, suffix_mode
         self.steps_per_block = steps_per_block
-        self.sched = Scheduler(L, token_budget, max_batch, kv_capacity, sort_queue, eos_id)
+        self.sched = Scheduler(L, token_budget, max_batch, kv_capacity, sort_queue, eos_id, static_groups)
         self.by_id: Dict[int, ReqState] = {}
         self.total_committed = 0
         self.total_steps = 0

@@ -627,3 +627,25 @@ def test_check_eos_evicts_at_the_block_boundary_after_the_token_appears():
     s2.active[0].mask = 0
     ev, ad = s2.evict_refill()
     assert ev == [] and len(s2.active) == 1
+
+
+def test_static_groups_admit_only_into_an_empty_batch_and_lose_to_refill_on_stragglers():
+    """The comparison policy of Section 3.1: requests run in fixed groups and the next group starts when the whole
+    group has finished.  With one long request per group its effective compute ratio (Eq. 2) collapses, while
+    block-boundary refill keeps the batch full."""
+    L, Bsz = 32, 4
+    def fill(s):
+        for i in range(40):
+            s.submit(sched_req(i, 20, 32 * (8 if i % 4 == 0 else 1)))      # every fourth request is a straggler
+    st = O.Scheduler(L, 0, Bsz, 1 << 24, sort_queue=False, static_groups=True)
+    fill(st)
+    drain(st, L)
+    for t in st.trace:                                  # admissions only into an empty batch
+        assert not t.admitted or len(t.admitted) == t.n_active
+    co = O.Scheduler(L, 0, Bsz, 1 << 24, sort_queue=False)
+    fill(co)
+    drain(co, L)
+    r_static, r_refill = st.effective_compute_ratio(Bsz), co.effective_compute_ratio(Bsz)
+    # a static group of one 8-block and three 1-block requests runs 8 cycles with 4, 1, 1, ... rows: R = 11 / 32
+    assert abs(r_static - 11.0 / 32.0) < 1e-9
+    assert r_refill > 0.9 and len(co.trace) < len(st.trace)
