@@ -71,6 +71,8 @@ typedef struct {
   int eos_id;                    /* CheckEOS of Algorithm 1: at a block boundary a request whose finished blocks hold
                                     this token id leaves the active set (its later positions stay masked, its state
                                     becomes BS_REQ_FINISHED); < 0: off, every request generates exactly g_i tokens */
+  int static_groups;             /* 1: the comparison policy of Section 3.1 (fixed groups: nothing is admitted until
+                                    every request of the current group has finished); 0: block-boundary refill */
 } bs_config;
 
 /* All weights are bf16, row-major [out_features, in_features], device memory.

@@ -19,9 +19,10 @@ import bs_inputs  # noqa: E402
 from paper_2607_08930_b200 import binding as B, build  # noqa: E402
 
 
-def run_variant(wl, weights, sort_queue: bool, suffix_mode: int, steps_per_block: int = 0):
+def run_variant(wl, weights, sort_queue: bool, suffix_mode: int, steps_per_block: int = 0,
+                static_groups: bool = False):
     eng = B.engine_for_workload(wl, weights, sort_queue=sort_queue, suffix_mode=suffix_mode,
-                                steps_per_block=steps_per_block)
+                                steps_per_block=steps_per_block, static_groups=static_groups)
     for r in wl.requests:
         eng.admit(r.req_id, r.prompt, r.g, r.alpha, r.start_block, r.gen_prefix)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -44,11 +45,16 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--workload", type=int, default=3)
     ap.add_argument("--block-lens", type=int, nargs="*", default=[32, 16])
+    ap.add_argument("--static-groups", action="store_true",
+                    help="add the comparison policy: fixed groups in submission order, no refill until a group is done")
+    ap.add_argument("--requests", type=int, default=0, help="use only the first N requests of the workload")
     ap.add_argument("--steps-per-block", type=int, nargs="*", default=[],
                     help="extra variants with a transfer quota S < L (sorted queue, full suffix)")
     args = ap.parse_args()
     build.build()
     base = bs_inputs.workload(args.workload)
+    if args.requests:
+        base = dataclasses.replace(base, requests=base.requests[:args.requests])
     weights = bs_inputs.make_weights(base.shape, base.weight_seed, device="cuda:0")
     rows = []
     for L in args.block_lens:
@@ -69,6 +75,14 @@ def main():
         res.update(workload=base.name, block_len=base.block_len, queue=f"sorted, S = {S}", suffix="full")
         print(json.dumps(res), flush=True)
         rows.append(res)
+    if args.static_groups:
+        for name, kw in (("block-boundary refill, submission order", dict(sort_queue=False)),
+                         ("static groups, submission order", dict(sort_queue=False, static_groups=True))):
+            run_variant(base, weights, suffix_mode=B.SUFFIX_FULL, **kw)
+            res = run_variant(base, weights, suffix_mode=B.SUFFIX_FULL, **kw)
+            res.update(workload=base.name, block_len=base.block_len, queue=name, suffix="full")
+            print(json.dumps(res), flush=True)
+            rows.append(res)
     print("\n| L | queue | suffix | committed tokens/s | job s | cycles | steps | packed tokens | mean |A| |")
     print("|---|---|---|---|---|---|---|---|---|")
     for r in rows:

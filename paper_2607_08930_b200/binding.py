@@ -36,7 +36,8 @@ class BsConfig(C.Structure):
                 ("rms_eps", C.c_float), ("rope_theta", C.c_float), ("block_len", C.c_int), ("tau", C.c_float),
                 ("token_budget", C.c_longlong), ("max_batch", C.c_int), ("max_requests", C.c_int),
                 ("max_row_tokens", C.c_int), ("kv_capacity_tokens", C.c_longlong), ("suffix_mode", C.c_int),
-                ("sort_queue", C.c_int), ("steps_per_block", C.c_int), ("eos_id", C.c_int)]
+                ("sort_queue", C.c_int), ("steps_per_block", C.c_int), ("eos_id", C.c_int),
+                ("static_groups", C.c_int)]
 
 
 class BsWeights(C.Structure):
@@ -125,11 +126,12 @@ def _check_op(rc: int, name: str) -> None:
 
 def make_config(shape, block_len: int, tau: float, token_budget: int, max_batch: int, max_requests: int,
                 max_row_tokens: int, kv_capacity_tokens: int, suffix_mode: int = SUFFIX_FULL,
-                sort_queue: bool = True, steps_per_block: int = 0, eos_id: int = -1) -> BsConfig:
+                sort_queue: bool = True, steps_per_block: int = 0, eos_id: int = -1,
+                static_groups: bool = False) -> BsConfig:
     return BsConfig(shape.n_layers, shape.d_model, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, shape.d_ffn,
                     shape.vocab, shape.mask_id, shape.rms_eps, shape.rope_theta, block_len, tau, token_budget,
                     max_batch, max_requests, max_row_tokens, kv_capacity_tokens, suffix_mode, int(sort_queue),
-                    int(steps_per_block), int(eos_id))
+                    int(steps_per_block), int(eos_id), int(static_groups))
 
 
 def query_sizes(cfg: BsConfig) -> BsSizes:
@@ -293,7 +295,7 @@ class Engine:
 
 def engine_for_workload(wl, weights, *, kv_capacity_tokens: Optional[int] = None, suffix_mode: int = SUFFIX_FULL,
                         sort_queue: bool = True, steps_per_block: int = 0, eos_id: int = -1,
-                        device: str = "cuda:0") -> Engine:
+                        static_groups: bool = False, device: str = "cuda:0") -> Engine:
     """Size an engine for a bs_inputs.Workload (the caller still admits the requests)."""
     mrt = wl.max_row_tokens
     if kv_capacity_tokens is None:
@@ -302,7 +304,7 @@ def engine_for_workload(wl, weights, *, kv_capacity_tokens: Optional[int] = None
         if wl.token_budget > 0:       # Eq. 1 bounds |A| * width; rows are at most width + g long
             kv_capacity_tokens = min(kv_capacity_tokens, wl.token_budget + wl.max_batch * max(r.g for r in wl.requests))
     cfg = make_config(wl.shape, wl.block_len, wl.tau, wl.token_budget, wl.max_batch, len(wl.requests), mrt,
-                      max(kv_capacity_tokens, mrt), suffix_mode, sort_queue, steps_per_block, eos_id)
+                      max(kv_capacity_tokens, mrt), suffix_mode, sort_queue, steps_per_block, eos_id, static_groups)
     return Engine(cfg, weights, device)
 
 

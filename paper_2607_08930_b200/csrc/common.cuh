@@ -50,6 +50,7 @@ struct DevState {
   int q_tile;           // query tokens per attention work item
   int S;                // diffusion steps per block (transfer quota of Section 2.5); S = L: one forced token per step
   int eos_id;           // CheckEOS of Algorithm 1 (< 0: off)
+  int static_groups;    // 1: no admission while any row of the current group is active (comparison policy)
   long long beta, kv_capacity;
   float tau;
   int* hdr;             // [kHdrInts] followed directly by row_mask[max_batch]

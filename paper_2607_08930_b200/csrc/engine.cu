@@ -286,6 +286,7 @@ int bs_init_model(const bs_config* cfg, const bs_weights* w, void* kv, void* wor
   st.vocab = cfg->vocab; st.beta = cfg->token_budget; st.kv_capacity = cfg->kv_capacity_tokens; st.tau = cfg->tau;
   st.S = cfg->steps_per_block > 0 ? cfg->steps_per_block : cfg->block_len;
   st.eos_id = cfg->eos_id;
+  st.static_groups = cfg->static_groups ? 1 : 0;
   st.q_tile = attention_q_tile(cfg->n_q_heads, cfg->n_kv_heads, cfg->head_dim);
   e->gemm_scratch.partial = e->ws.partial;
   e->gemm_scratch.partial_floats = kPartialFloats;

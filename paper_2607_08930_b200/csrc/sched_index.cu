@@ -177,7 +177,7 @@ __global__ void __launch_bounds__(kSchedThreads) k_sched(DevState st) {
     s_n = n_keep;
     s_head = st.hdr[H_QUEUE_HEAD];
     s_w = w;
-    s_stop = 0;
+    s_stop = (st.static_groups && n_keep > 0) ? 1 : 0;    // static groups refill only an empty batch
   }
   __syncthreads();
 

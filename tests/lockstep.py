@@ -76,7 +76,7 @@ class Lockstep:
     adopts the engine's mask word after each step, since the oracle does not run their forward."""
 
     def __init__(self, wl, weights_cuda, weights_np, suffix_mode=0, kv_capacity=None, sort_queue=True, track=None,
-                 model=None, steps_per_block=0, eos_id=-1):
+                 model=None, steps_per_block=0, eos_id=-1, static_groups=False):
         self.wl = wl
         self.track = None if track is None else set(track)
         # the near-tie classes below are written for one forced token per step; a general transfer quota is checked
@@ -84,11 +84,12 @@ class Lockstep:
         assert not steps_per_block or steps_per_block == wl.block_len or self.track == set()
         self.S = steps_per_block if steps_per_block else wl.block_len
         self.eng = B.engine_for_workload(wl, weights_cuda, kv_capacity_tokens=kv_capacity, suffix_mode=suffix_mode,
-                                         sort_queue=sort_queue, steps_per_block=steps_per_block, eos_id=eos_id)
+                                         sort_queue=sort_queue, steps_per_block=steps_per_block, eos_id=eos_id,
+                                         static_groups=static_groups)
         self.model = model if model is not None else O.model_from_weights(wl.shape, weights_np)
         self.ora = O.Engine(self.model, wl.block_len, wl.tau, wl.token_budget, wl.max_batch,
                             self.eng.cfg.kv_capacity_tokens, suffix_mode, sort_queue, steps_per_block=steps_per_block,
-                            eos_id=eos_id)
+                            eos_id=eos_id, static_groups=static_groups)
         self.suffix_mode = suffix_mode
         self.excluded = {"tau": 0, "top2": 0, "forced": 0, "noise": 0}
         self.conf_rows_within_tol = 0

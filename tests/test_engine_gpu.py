@@ -384,3 +384,27 @@ def test_check_eos_evicts_requests_early_in_lockstep(B):
     assert early >= 1
     assert ls.eng.stats().committed < wl.committed_target()
     assert ls.eng.stats().committed == sum(r.committed for r in ls.ora.by_id.values())
+
+
+def test_static_group_policy_in_lockstep(B):
+    """The comparison policy (fixed groups, no refill until the group has finished): admissions, evictions, row order
+    and KV slabs follow the oracle's scheduler cycle by cycle, and admissions happen only into an empty batch."""
+    from lockstep import Lockstep
+    shape = bs_inputs.TINY
+    rng = np.random.default_rng(9)
+    n = 10
+    gs = [32 * (4 if i % 3 == 0 else 1) for i in range(n)]
+    wl = bs_inputs.custom_workload(shape, rng.integers(5, 50, size=n), gs, rng.choice([2.0, 6.0], size=n), seed=3,
+                                   tau=0.9, max_batch=3)
+    wc, wn = both_weights(shape, 8)
+    ls = Lockstep(wl, wc, wn, sort_queue=False, static_groups=True, track=set())
+    ls.admit(wl.requests)
+    cycles = ls.run()
+    for t in ls.ora.sched.trace:
+        assert not t.admitted or len(t.admitted) == t.n_active
+    st = ls.eng.stats()
+    assert st.committed == wl.committed_target()
+    # refill serves the same requests in fewer cycles
+    ls2 = Lockstep(wl, wc, wn, sort_queue=False, track=set())
+    ls2.admit(wl.requests)
+    assert ls2.run() < cycles
