@@ -38,8 +38,14 @@ def test_query_sizes_and_validation(B):
     kv = wl.shape.n_layers * 2 * 4 * wl.max_row_tokens * wl.shape.n_kv_heads * wl.shape.head_dim * 2
     assert sz.kv_bytes >= kv and sz.kv_bytes < kv + 256
     assert sz.workspace_bytes > 0 and sz.state_bytes > 8 * wl.max_row_tokens * 4
+    # the policy switches do not change any buffer size
+    cfg_p = B.make_config(wl.shape, 32, 0.9, 0, 4, 8, wl.max_row_tokens, 4 * wl.max_row_tokens, steps_per_block=8,
+                          eos_id=5, static_groups=True)
+    sz_p = B.query_sizes(cfg_p)
+    assert (sz_p.kv_bytes, sz_p.workspace_bytes, sz_p.state_bytes) == (sz.kv_bytes, sz.workspace_bytes, sz.state_bytes)
     for field, bad in (("head_dim", 48), ("block_len", 64), ("max_batch", 5000), ("vocab", 1023),
-                       ("kv_capacity_tokens", 3), ("n_q_heads", 3)):
+                       ("kv_capacity_tokens", 3), ("n_q_heads", 3), ("steps_per_block", 33), ("steps_per_block", -1),
+                       ("eos_id", wl.shape.mask_id), ("eos_id", wl.shape.vocab)):
         cfg2 = B.make_config(wl.shape, 32, 0.9, 0, 4, 8, wl.max_row_tokens, 4 * wl.max_row_tokens)
         setattr(cfg2, field, bad)
         if field == "n_q_heads":
