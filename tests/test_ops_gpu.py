@@ -28,7 +28,9 @@ def rel_err(got, ref):
 GEMM_SHAPES = [  # M, N, K: several tiles, ragged tails in every dimension, one case smaller than a tile
     (1, 128, 64), (33, 200, 72), (128, 256, 128), (130, 1000, 384), (257, 130, 1000), (300, 2000, 256),
     (517, 704, 256), (64, 4608, 512), (1000, 512, 2048), (459, 768, 256), (459, 256, 704), (48, 384, 128),
-    (200, 640, 320)]
+    (200, 640, 320),
+    # more 256-row weight tiles than CTA pairs with a ragged last round: the SwiGLU plan narrows its token tiles
+    (1760, 12288, 128)]
 
 
 @pytest.mark.parametrize("M,N,K", GEMM_SHAPES)
@@ -159,6 +161,11 @@ ATTN_CASES = [
     (6, 2, 128, [(32, 200), (8, 8), (130, 130), (0, 9), (32, 65)]),
     (28, 4, 128, [(32, 300), (32, 96), (70, 70)]),
     (32, 32, 128, [(32, 129), (100, 100)]),
+    # MHA rows longer than one Q tile (two Q tiles of 128 tokens per work item, several items per row)
+    (8, 8, 128, [(300, 300), (32, 517), (129, 129)]),
+    # four and eight query heads per kv head (32 and 16 tokens per Q tile)
+    (8, 2, 128, [(70, 200), (32, 64), (33, 33)]),
+    (16, 2, 128, [(40, 130), (32, 700)]),
 ]
 
 
