@@ -8,9 +8,10 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libblockserve.so")
-SOURCES = ["engine.cu", "sched_index.cu", "elementwise.cu", "gemm_mma.cu", "gemm_tcgen05.cu", "attention.cu", "attention_tc.cu", "rope_static.cu"]
+SOURCES = ["engine.cu", "sched_index.cu", "elementwise.cu", "gemm_tcgen05.cu", "attention.cu", "attention_tc.cu",
+           "rope_static.cu"]
 NVCC_FLAGS = ["-std=c++17", "-O3", "-lineinfo", "-gencode", "arch=compute_100a,code=sm_100a",
-              "-Xcompiler", "-fPIC", "--use_fast_math" if False else "-Xptxas", "-v"]
+              "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 
 
 def _newer(a: str, b: str) -> bool:
@@ -34,7 +35,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
                 raise RuntimeError(f"nvcc failed on {src}")
         objs.append(o)
     if force or any(_newer(o, LIB) for o in objs):
-        r = subprocess.run([nvcc, "-shared", "-o", LIB, *objs, "-lcudart", "-lcuda"], capture_output=True, text=True)
+        r = subprocess.run([nvcc, "-shared", "-o", LIB, *objs, "-lcudart"], capture_output=True, text=True)
         if r.returncode != 0:
             sys.stderr.write(r.stdout + r.stderr)
             raise RuntimeError("link failed")

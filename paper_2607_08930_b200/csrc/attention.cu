@@ -6,7 +6,9 @@
 #include <math.h>
 #include <stdlib.h>
 
-#include "common.cuh"
+#include <mutex>
+
+#include "tc_common.cuh"
 
 namespace bs {
 
@@ -303,10 +305,18 @@ cudaError_t launch_variant(dim3 grid, int threads, cudaStream_t s, const bf16* q
                            bf16* out, const int* cu_q, const int* cu_tile, const int* kv_base, const int* vis,
                            int n_rows, int hq, int hkv, int qt, AttnPartial part) {
   constexpr size_t smem = (size_t)NSTAGE * 2 * KT * (DH + 8) * sizeof(bf16);
-  static bool done = false;
-  if (!done) {
-    cudaFuncSetAttribute(k_attention<DH, KT, NSTAGE, MINB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    done = true;
+  static int done_on[kMaxDevices];         // per device: the attribute belongs to the device's copy of the kernel
+  static std::mutex mu;
+  int* done = device_slot(done_on);
+  if (!done) return cudaErrorInvalidDevice;
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    if (!*done) {
+      if (cudaFuncSetAttribute(k_attention<DH, KT, NSTAGE, MINB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               (int)smem) != cudaSuccess)
+        return cudaErrorInvalidDevice;
+      *done = 1;
+    }
   }
   return launch_pdl(k_attention<DH, KT, NSTAGE, MINB>, grid, dim3(threads), smem, s, qkv, kc, vc, out, cu_q, cu_tile,
                     kv_base, vis, n_rows, hq, hkv, qt, part);
@@ -338,12 +348,17 @@ cudaError_t launch_attention(const bf16* qkv, const bf16* kc, const bf16* vc, bf
   if (threads > 256 || (dh != 64 && dh != 128) || hq % hkv != 0) return cudaErrorInvalidValue;
   // KV chunks: a block step has few (row, kv head, q tile) items, each a long serial walk over the row's keys;
   // splitting the walk fills the SMs.  A refresh step has plenty of items already.
-  static int num_sms = 0;
-  if (!num_sms) {
-    int dev = 0;
+  static int num_sms_of[kMaxDevices];
+  int* sms = device_slot(num_sms_of);
+  if (!sms) return cudaErrorInvalidDevice;
+  if (!*sms) {
+    int dev = 0, n = 0;
     cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1)
+      return cudaErrorInvalidDevice;
+    *sms = n;
   }
+  const int num_sms = *sms;
   // (measured on B200: with fewer work items than a quarter / a half of the SMs, 4 / 2 chunks shorten the
   // serial walk enough to pay for the merge; beyond that the legacy-path MMAs are the limit and chunks only add work)
   const long long base = (long long)n_tiles * hkv;
@@ -352,12 +367,10 @@ cudaError_t launch_attention(const bf16* qkv, const bf16* kc, const bf16* vc, bf
     chunks = base * 4 <= num_sms + 12 ? 4 : (base * 2 <= num_sms ? 2 : 1);
     while (chunks > 1 && (size_t)chunks * M * ((size_t)hq * dh + 2 * hq) > scratch_floats) chunks >>= 1;
   }
-  if (const char* ev = getenv("BS_ATTN_CHUNKS")) {
-    const int c = atoi(ev);
-    if (c >= 1 && (c == 1 || scratch)) chunks = c;
-  }
-  int variant = 1;
-  if (const char* ev = getenv("BS_ATTN_VARIANT")) variant = atoi(ev);
+  // measurement overrides, read once per process
+  static const int env_chunks = getenv("BS_ATTN_CHUNKS") ? atoi(getenv("BS_ATTN_CHUNKS")) : 0;
+  static const int variant = getenv("BS_ATTN_VARIANT") ? atoi(getenv("BS_ATTN_VARIANT")) : 1;
+  if (env_chunks >= 1 && (env_chunks == 1 || scratch)) chunks = env_chunks;
   AttnPartial part;
   part.chunks = chunks;
   part.M = M;

@@ -16,57 +16,25 @@
 //               the output accumulates in TMEM over all key tiles and is rescaled lazily (only when a row's
 //               maximum has grown by more than 2^8), the running sum follows the same scale
 // Every wait is bounded; on a timeout the flag is raised, all roles drain, TMEM is freed.
-#include <cuda.h>
-#include <cudaTypedefs.h>
 #include <math.h>
 #include <stdlib.h>
 
 #include <mutex>
 #include <unordered_map>
 
-#include "common.cuh"
+#include "tc_common.cuh"
 
 namespace bs {
 
 namespace {
 
+using namespace tc;
+
 constexpr int DH = 128;
 constexpr int kThreads = 320;             // producer warp, MMA warp, 8 softmax warps
 constexpr int kHalfBytes = 128 * 128;      // 128 rows x 64 bf16: one swizzled sub-tile of Q or P
 constexpr int kQBytes = 2 * kHalfBytes;
-constexpr long long kWaitCycles = 4000000000ll;
 
-__device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(unsigned bar, unsigned count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(unsigned bar, unsigned bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(unsigned bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity) {
-  unsigned ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-__device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity, volatile int* abort_flag) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const long long t0 = clock64();
-  while (!mbar_try_wait(bar, parity)) {
-    if (*abort_flag) return false;
-    if (clock64() - t0 > kWaitCycles) {
-      *abort_flag = 1;
-      return false;
-    }
-  }
-  return true;
-}
 __device__ __forceinline__ void tma_load_3d(unsigned dst, const CUtensorMap* map, int c0, int c1, int c2, unsigned bar) {
   asm volatile(
       "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
@@ -77,14 +45,7 @@ __device__ __forceinline__ unsigned umma_idesc(int n, bool b_mn_major) {
   return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn_major ? (1u << 16) : 0u) | ((unsigned)(n >> 3) << 17) |
          ((128u >> 4) << 24);
 }
-// Operand tiles are 128B-swizzled with rows of 128 bytes; 8-row groups are 1024 bytes apart (K-major and MN-major
-// alike).  The MMA issuer is one thread, and every scalar instruction between two tcgen05.mma delays the next one:
-// descriptors are handled as 32-bit low words (start address >> 4 | LBO field) that advance by adds; the constant
-// high word (SBO = 1024, version, 128B swizzle) is joined inside the asm block.
-constexpr unsigned kDescHi = (unsigned)(1024 >> 4) | (1u << 14) | (2u << 29);
-__device__ __forceinline__ unsigned desc_lo(unsigned smem_addr, unsigned lbo_bytes = 16) {
-  return ((smem_addr & 0x3FFFFu) >> 4) | ((lbo_bytes >> 4) << 16);
-}
+// tcgen05.mma from descriptor low words (see tc_common.cuh); K-major and MN-major tiles share the 1024-byte group stride.
 __device__ __forceinline__ void umma_lo(unsigned d_tmem, unsigned a_lo, unsigned b_lo, unsigned idesc,
                                         unsigned accumulate) {
   asm volatile(
@@ -104,24 +65,6 @@ __device__ __forceinline__ void umma_ts(unsigned d_tmem, unsigned a_tmem, unsign
       "mov.b64 db, {%2, %5};\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %3, p;\n\t}"
       ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kDescHi) : "memory");
-}
-__device__ __forceinline__ void umma_commit(unsigned bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tmem_ld32(unsigned taddr, float* v) {
-  unsigned r[32];
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr));
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
 __device__ __forceinline__ void tmem_st32(unsigned taddr, const float* v) {
@@ -446,7 +389,6 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 
 // ---- host side ---------------------------------------------------------------------------------------------
 
-PFN_cuTensorMapEncodeTiled_v12000 g_encode = nullptr;
 std::mutex g_mutex;
 struct Key3 {
   const void* ptr; long long d1, d2, s1, s2; int b1, b2;
@@ -466,14 +408,9 @@ std::unordered_map<Key3, CUtensorMap, Hash3> g_maps;
 
 // bf16 tensor [d2][d1][128] with byte strides s1 (dim 1) and s2 (dim 2); box 64 x b1 x b2, 128-byte swizzle.
 bool get_map3(const bf16* ptr, long long d1, long long d2, long long s1, long long s2, int b1, int b2, CUtensorMap* out) {
+  PFN_cuTensorMapEncodeTiled_v12000 encode = tensor_map_encoder();
+  if (!encode) return false;
   std::lock_guard<std::mutex> lock(g_mutex);
-  if (!g_encode) {
-    void* fn = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn)
-      return false;
-    g_encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
-  }
   const Key3 key{ptr, d1, d2, s1, s2, b1, b2};
   auto it = g_maps.find(key);
   if (it != g_maps.end()) { *out = it->second; return true; }
@@ -483,7 +420,7 @@ bool get_map3(const bf16* ptr, long long d1, long long d2, long long s1, long lo
   const cuuint64_t strides[2] = {(cuuint64_t)s1, (cuuint64_t)s2};
   const cuuint32_t box[3] = {64, (cuuint32_t)b1, (cuuint32_t)b2};
   const cuuint32_t estr[3] = {1, 1, 1};
-  if (g_encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<bf16*>(ptr), dims, strides, box, estr,
+  if (encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<bf16*>(ptr), dims, strides, box, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return false;
@@ -514,12 +451,19 @@ cudaError_t launch_attention_tc(const bf16* qkv, const bf16* kc, const bf16* vc,
   if (((uintptr_t)qkv | (uintptr_t)kc | (uintptr_t)vc) & 15) return cudaSuccess;
   const int G = hq / hkv;
   const int tq = tokens_per_q_tile(hq, hkv);
-  static bool attr_done = false;
-  if (!attr_done) {
-    if (cudaFuncSetAttribute(k_attention_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
-      return cudaSuccess;
-    attr_done = true;
+  static int num_sms_of[kMaxDevices];      // per device; non-zero once the kernel attribute is set there
+  int* sms = device_slot(num_sms_of);
+  if (!sms) return cudaErrorInvalidDevice;
+  if (!*sms) {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    int dev = 0, n = 0;
+    cudaGetDevice(&dev);
+    if (cudaFuncSetAttribute(k_attention_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess ||
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1)
+      return cudaErrorInvalidDevice;
+    *sms = n;
   }
+  const int num_sms = *sms;
   CUtensorMap mq, mk, mv;
   const long long qkv_heads = hq + 2 * hkv;
   if (!get_map3(qkv, qkv_heads, M, DH * 2, qkv_heads * DH * 2, G, tq, &mq)) return cudaSuccess;
@@ -529,12 +473,6 @@ cudaError_t launch_attention_tc(const bf16* qkv, const bf16* kc, const bf16* vc,
   AttnTcParams p;
   p.cu_q = cu_q; p.cu_tile = cu_tile; p.kv_base = kv_base; p.vis = vis; p.out = out;
   p.n_rows = n_rows; p.hq = hq; p.hkv = hkv; p.tq = tq; p.error_flag = error_flag;
-  static int num_sms = 0;
-  if (!num_sms) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
-  }
   // With fewer work items than SMs each CTA is one long dependent chain over the row's key tiles: give every Q
   // tile its own CTA.  With many work items the two Q tiles of an item share each K/V tile they load.
   p.split = (long long)n_tiles * hkv < num_sms ? 1 : 0;

@@ -98,7 +98,10 @@ cudaError_t launch_gemm(const bf16* A, int lda, const bf16* W, const bf16* W2, v
                         int mode, const float* row_scale, const GemmScratch& scratch, cudaStream_t s);
 cudaError_t launch_gemm_tc(const bf16* A, int lda, const bf16* W, const bf16* W2, void* C, int ldc, int M, int N,
                            int K, int mode, const float* row_scale, const GemmScratch& scratch, cudaStream_t s,
-                           bool* handled, int* splits_out);
+                           int* splits_out);
+// Why the last launch_gemm* of this thread returned cudaErrorNotSupported (a shape or alignment the tensor-core
+// kernels do not take; there is no other GEMM behind them).
+const char* gemm_decline_reason();
 // mode 4: only the k-split partial sums [splits][M][N] are written to scratch.partial; a fused finishing kernel
 // (below) adds them in split order and applies what follows the projection.
 cudaError_t launch_gemm_partial(const bf16* A, int lda, const bf16* W, int M, int N, int K, const GemmScratch& scratch,
@@ -111,8 +114,6 @@ cudaError_t launch_finish_qkv_rope(const float* partial, int splits, int M, bf16
 cudaError_t launch_finish_residual_norm(const float* partial, int splits, int M, int d, float* x, const bf16* w,
                                         bf16* h, float eps, cudaStream_t s);
 
-cudaError_t launch_gemm_mma(const bf16* A, int lda, const bf16* W, const bf16* W2, void* C, int ldc, int M, int N,
-                            int K, int mode, const float* row_scale, cudaStream_t s);
 int attention_q_tile(int hq, int hkv, int dh);
 void build_rope_table(float* host_cos_sin, int max_pos, int dh, float theta);   // [max_pos, dh/2, 2]
 

@@ -156,6 +156,8 @@ int fail(bs_engine* e, int code, const std::string& msg) {
   return code;
 }
 int cuda_fail(bs_engine* e, cudaError_t r, const char* what) {
+  if (r == cudaErrorNotSupported)     // a plan the kernels declined: a property of the arguments, not of the device
+    return fail(e, BS_E_ARG, std::string("unsupported shape: ") + bs::gemm_decline_reason() + " (" + what + ")");
   return fail(e, BS_E_CUDA, std::string(what) + ": " + cudaGetErrorString(r));
 }
 #define CU(e, call)                                         \
@@ -231,18 +233,12 @@ int post_header(bs_engine* e) {
 namespace bs {
 cudaError_t launch_gemm(const bf16* A, int lda, const bf16* W, const bf16* W2, void* C, int ldc, int M, int N, int K,
                         int mode, const float* row_scale, const GemmScratch& scratch, cudaStream_t s) {
-  bool handled = false;
-  cudaError_t r = launch_gemm_tc(A, lda, W, W2, C, ldc, M, N, K, mode, row_scale, scratch, s, &handled, nullptr);
-  if (handled) return r;
-  return launch_gemm_mma(A, lda, W, W2, C, ldc, M, N, K, mode, row_scale, s);
+  return launch_gemm_tc(A, lda, W, W2, C, ldc, M, N, K, mode, row_scale, scratch, s, nullptr);
 }
 
 cudaError_t launch_gemm_partial(const bf16* A, int lda, const bf16* W, int M, int N, int K, const GemmScratch& scratch,
                                 cudaStream_t s, int* splits_out) {
-  bool handled = false;
-  cudaError_t r = launch_gemm_tc(A, lda, W, nullptr, nullptr, 0, M, N, K, 4, nullptr, scratch, s, &handled, splits_out);
-  if (r != cudaSuccess) return r;
-  return handled ? cudaSuccess : cudaErrorNotSupported;
+  return launch_gemm_tc(A, lda, W, nullptr, nullptr, 0, M, N, K, 4, nullptr, scratch, s, splits_out);
 }
 }  // namespace bs
 
@@ -824,7 +820,7 @@ int bs_op_gemm(const void* A, int lda, const void* W, const void* W2, void* C, i
   sc.error_flag = error_flag;
   cudaError_t r = launch_gemm((const bf16*)A, lda, (const bf16*)W, (const bf16*)W2, C, ldc, M, N, K, mode, row_scale,
                               sc, (cudaStream_t)stream);
-  return r == cudaSuccess ? BS_OK : BS_E_CUDA;
+  return r == cudaSuccess ? BS_OK : (r == cudaErrorNotSupported ? BS_E_ARG : BS_E_CUDA);
 }
 
 int bs_op_rmsnorm(const float* x, const int* idx, const void* w, void* y, int M, int d, float eps, void* stream) {

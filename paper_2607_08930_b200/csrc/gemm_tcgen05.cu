@@ -11,26 +11,25 @@
 // kernel adds them in a fixed order and applies the epilogue (deterministic, no atomics).
 // Every wait is bounded: when one runs out the kernel raises a flag, all roles drain, TMEM is freed and the
 // host reports BS_E_TIMEOUT.
-#include <cuda.h>
-#include <cudaTypedefs.h>
-
 #include <stdio.h>
 #include <stdlib.h>
 
 #include <mutex>
+#include <string>
 #include <unordered_map>
 
-#include "common.cuh"
+#include "tc_common.cuh"
 
 namespace bs {
 
 namespace {
 
+using namespace tc;
+
 constexpr int BK = 64;                 // K elements per pipeline stage (128 bytes: one swizzle span)
 constexpr int TILE_N = 128;            // weight rows per tile (UMMA M)
 constexpr int kThreads = 192;
 constexpr int kSmemBudget = 200 * 1024;
-constexpr long long kWaitCycles = 4000000000ll;   // ~2 s at 2 GHz: no legitimate wait comes near it
 
 struct GemmParams {
   int M, N, K;
@@ -51,74 +50,17 @@ struct GemmParams {
   int* error_flag;
 };
 
-__device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(unsigned bar, unsigned count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(unsigned bar, unsigned bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(unsigned bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity) {
-  unsigned ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-// Bounded wait: returns false (and raises the abort flag) if the phase does not complete in time or if
-// another role has already given up.
-__device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity, volatile int* abort_flag) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const long long t0 = clock64();
-  while (!mbar_try_wait(bar, parity)) {
-    if (*abort_flag) return false;
-    if (clock64() - t0 > kWaitCycles) {
-      *abort_flag = 1;
-      return false;
-    }
-  }
-  return true;
-}
-
 __device__ __forceinline__ void tma_load_2d(unsigned dst, const CUtensorMap* map, int c0, int c1, unsigned bar) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
       ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
 }
 
-// K-major operand tile, rows of 128 bytes, 128B swizzle: 8-row groups are 1024 bytes apart.
-__device__ __forceinline__ unsigned long long umma_desc(unsigned smem_addr) {
-  unsigned long long d = 0;
-  d |= (unsigned long long)((smem_addr & 0x3FFFF) >> 4);        // start address
-  d |= (unsigned long long)1 << 16;                              // leading byte offset (unused for swizzled K-major)
-  d |= (unsigned long long)(1024 >> 4) << 32;                    // stride byte offset
-  d |= (unsigned long long)1 << 46;                              // descriptor version (sm_100)
-  d |= (unsigned long long)2 << 61;                              // layout: 128-byte swizzle
-  return d;
-}
 // kind::f16 instruction descriptor: fp32 accumulator, bf16 x bf16, both K-major, shape 128 x n x 16.
 __device__ __forceinline__ unsigned umma_idesc(int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((unsigned)(n >> 3) << 17) | ((unsigned)(TILE_N >> 4) << 24);
 }
-__device__ __forceinline__ void umma_bf16(unsigned d_tmem, unsigned long long a, unsigned long long b, unsigned idesc,
-                                          unsigned accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(a), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
-}
-// The MMA issuer is one thread, and every scalar instruction it spends between two tcgen05.mma delays the next
-// one: descriptors are therefore handled as 32-bit low words (start address >> 4, plus the fixed LBO field) that
-// advance by plain adds, with the constant high word (SBO, version, swizzle) joined inside the asm block.
-constexpr unsigned kDescHi = (unsigned)(1024 >> 4) | (1u << 14) | (2u << 29);
-__device__ __forceinline__ unsigned desc_lo(unsigned smem_addr) { return ((smem_addr & 0x3FFFFu) >> 4) | (1u << 16); }
+// tcgen05.mma from descriptor low words (see tc_common.cuh), for one CTA or a CTA pair.
 template <int CG>
 __device__ __forceinline__ void umma_lo(unsigned d_tmem, unsigned a_lo, unsigned b_lo, unsigned idesc,
                                         unsigned accumulate) {
@@ -151,24 +93,6 @@ __device__ __forceinline__ void issue_stage(unsigned d0, unsigned d1, unsigned a
     umma_lo<CG>(d0, a0_lo + 2 * k, b_lo + 2 * k, idesc, 1u);
     if (TWO) umma_lo<CG>(d1, a1_lo + 2 * k, b_lo + 2 * k, idesc, 1u);
   }
-}
-__device__ __forceinline__ void umma_commit(unsigned bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tmem_ld32(unsigned taddr, float* v) {
-  unsigned r[32];
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr));
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 __device__ __forceinline__ float silu_f(float x) { return x / (1.0f + __expf(-x)); }
 
@@ -425,14 +349,6 @@ __device__ __forceinline__ void tma_load_2d_pair(unsigned dst, const CUtensorMap
 __device__ __forceinline__ unsigned umma_idesc_pair(int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((unsigned)(n >> 3) << 17) | ((unsigned)(256 >> 4) << 24);
 }
-__device__ __forceinline__ void umma_bf16_pair(unsigned d_tmem, unsigned long long a, unsigned long long b,
-                                               unsigned idesc, unsigned accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(a), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
-}
 // arrives on the barrier at this shared-memory offset in both CTAs of the pair
 __device__ __forceinline__ void umma_commit_pair(unsigned bar) {
   const unsigned short mask = 3;
@@ -649,7 +565,6 @@ __global__ void k_gemm_finish(const float* __restrict__ partial, int splits, int
 
 // ---- host side ---------------------------------------------------------------------------------------------
 
-PFN_cuTensorMapEncodeTiled_v12000 g_encode = nullptr;
 std::mutex g_mutex;
 
 struct MapKey {
@@ -669,14 +584,9 @@ struct MapHash {
 std::unordered_map<MapKey, CUtensorMap, MapHash> g_maps;
 
 bool get_map(const bf16* ptr, long long rows, long long cols, long long ld, int box_rows, CUtensorMap* out) {
+  PFN_cuTensorMapEncodeTiled_v12000 encode = tensor_map_encoder();
+  if (!encode) return false;
   std::lock_guard<std::mutex> lock(g_mutex);
-  if (!g_encode) {
-    void* fn = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn)
-      return false;
-    g_encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
-  }
   const MapKey key{ptr, rows, cols, ld, box_rows};
   auto it = g_maps.find(key);
   if (it != g_maps.end()) { *out = it->second; return true; }
@@ -686,18 +596,38 @@ bool get_map(const bf16* ptr, long long rows, long long cols, long long ld, int 
   const cuuint64_t strides[1] = {(cuuint64_t)ld * sizeof(bf16)};
   const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
   const cuuint32_t estr[2] = {1, 1};
-  const CUresult r = g_encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<bf16*>(ptr), dims, strides, box, estr,
-                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  const CUresult r = encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<bf16*>(ptr), dims, strides, box, estr,
+                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return false;
   g_maps.emplace(key, m);
   *out = m;
   return true;
 }
 
-int g_num_sms = 0;
-
-int g_max_pairs = 0;     // clusters of two CTAs that can be resident at once
+// Plan overrides for measurements (environment, read once per process; the defaults are the measured best).
+struct Tuning {
+  int pair;         // BS_GEMM_PAIR: -1 automatic, 0 single-CTA kernel only, n > 0 CTA pairs from n tokens
+  int pair_wide;    // BS_GEMM_PAIR_WIDE: 512-row pair items
+  int pair_splits;  // BS_GEMM_PAIR_SPLITS: cap of the pair kernel's k split
+  int wide_off;     // BS_GEMM_WIDE=0: no 256-row items in the single-CTA kernel
+  int ksub;         // BS_GEMM_KSUB: 0 automatic, 1 or 2 k sub-blocks per stage
+  int splits;       // BS_GEMM_SPLITS: 0 automatic, 1..8
+  int stages;       // BS_GEMM_STAGES: 0 automatic
+  int debug;        // BS_GEMM_DEBUG: print every plan
+  int no_pdl;       // BS_NO_PDL
+};
+int env_int(const char* name, int dflt) {
+  const char* v = getenv(name);
+  return v ? atoi(v) : dflt;
+}
+const Tuning& tuning() {
+  static const Tuning t = {env_int("BS_GEMM_PAIR", -1), env_int("BS_GEMM_PAIR_WIDE", 0) > 0,
+                           env_int("BS_GEMM_PAIR_SPLITS", 8), getenv("BS_GEMM_WIDE") && env_int("BS_GEMM_WIDE", 1) == 0,
+                           env_int("BS_GEMM_KSUB", 0), env_int("BS_GEMM_SPLITS", 0), env_int("BS_GEMM_STAGES", 0),
+                           getenv("BS_GEMM_DEBUG") != nullptr, getenv("BS_NO_PDL") != nullptr};
+  return t;
+}
 
 using GemmKernel = void (*)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const GemmParams);
 GemmKernel kernel_tc(int epi) {
@@ -725,15 +655,33 @@ bool allow_big_smem(GemmKernel (*table)(int)) {
   return true;
 }
 
-// Resident clusters of two CTAs (once per process); < 1 when the pair kernel cannot be used.
-int ensure_pair_init() {
-  if (!g_max_pairs) {
+// One-time set-up per device: SM count, kernel attributes, resident CTA pairs.
+struct DevInfo {
+  int num_sms;      // 0: not initialised
+  int tc_ok;        // the single-CTA kernels may use their shared-memory budget
+  int max_pairs;    // 0: not queried; < 0: the pair kernel cannot be used; else resident clusters of two CTAs
+};
+DevInfo g_dev[kMaxDevices];
+
+DevInfo* dev_info() {
+  DevInfo* d = device_slot(g_dev);
+  if (!d) return nullptr;
+  std::lock_guard<std::mutex> lock(g_mutex);
+  if (!d->num_sms) {
+    int dev = 0, n = 0;
+    cudaGetDevice(&dev);
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) return nullptr;
+    d->tc_ok = allow_big_smem(kernel_tc) ? 1 : 0;
+    if (!d->tc_ok) cudaGetLastError();
+    d->num_sms = n;
+  }
+  if (!d->max_pairs) {
     if (!allow_big_smem(kernel_pair)) {
       cudaGetLastError();
-      g_max_pairs = -1;
+      d->max_pairs = -1;
     } else {
       cudaLaunchConfig_t qc = {};
-      qc.gridDim = dim3(2 * g_num_sms);
+      qc.gridDim = dim3(2 * d->num_sms);
       qc.blockDim = dim3(kThreads);
       qc.dynamicSmemBytes = (size_t)kSmemBudget + 1024;
       cudaLaunchAttribute qa[1];
@@ -742,11 +690,17 @@ int ensure_pair_init() {
       qc.attrs = qa; qc.numAttrs = 1;
       int n = 0;
       if (cudaOccupancyMaxActiveClusters(&n, k_gemm_pair<0>, &qc) != cudaSuccess || n < 1) { cudaGetLastError(); n = -1; }
-      g_max_pairs = n;
+      d->max_pairs = n;
     }
-    if (getenv("BS_GEMM_DEBUG")) fprintf(stderr, "gemm pair kernel: %d resident CTA pairs\n", g_max_pairs);
+    if (tuning().debug) fprintf(stderr, "gemm pair kernel: %d resident CTA pairs\n", d->max_pairs);
   }
-  return g_max_pairs;
+  return d;
+}
+
+thread_local std::string g_decline;     // why the last launch on this thread was refused
+cudaError_t decline(const char* why) {
+  g_decline = why;
+  return cudaErrorNotSupported;
 }
 
 // Fraction of the persistent grid that has work, averaged over its rounds.
@@ -762,12 +716,18 @@ int split_for(long long base_items, int workers, int kblocks, size_t out_floats,
   return sp < 1 ? 1 : sp;
 }
 
-// Plans and launches the CTA-pair kernel; *handled stays false when the shape is left to the single-CTA kernel.
-cudaError_t launch_gemm_pair(const bf16* A, int lda, const bf16* W, const bf16* W2, void* C, int ldc, int M, int N,
-                             int K, int mode, const float* row_scale, const GemmScratch& scratch, cudaStream_t s,
-                             bool* handled, int* splits_out) {
-  ensure_pair_init();
-  if (g_max_pairs < 1) return cudaSuccess;
+cudaError_t launch_finish(const GemmParams& p, int mode, int num_sms, cudaStream_t s) {
+  const size_t total = (size_t)p.M * p.N;
+  const size_t want = (total + 255) / 256, cap = (size_t)num_sms * 8;
+  return launch_pdl(k_gemm_finish, dim3((unsigned)(want < cap ? want : cap)), dim3(256), 0, s, (const float*)p.partial,
+                    p.splits, p.M, p.N, mode, p.C, p.ldc, p.row_scale);
+}
+
+// Plans and launches the CTA-pair kernel.
+cudaError_t launch_gemm_pair(const DevInfo& dv, const bf16* A, int lda, const bf16* W, const bf16* W2, void* C, int ldc,
+                             int M, int N, int K, int mode, const float* row_scale, const GemmScratch& scratch,
+                             cudaStream_t s, int* splits_out) {
+  const int max_pairs = dv.max_pairs;
   const int dual = mode == 3;
   GemmParams p;
   p.M = M; p.N = N; p.K = K; p.mode = mode; p.dual = dual; p.C = C; p.ldc = ldc; p.row_scale = row_scale;
@@ -775,8 +735,7 @@ cudaError_t launch_gemm_pair(const bf16* A, int lda, const bf16* W, const bf16* 
   // Two 256-row weight tiles per pair and work item (BS_GEMM_PAIR_WIDE=1) halve the token-tile traffic once more at
   // the price of single-buffered accumulators.  Measured on B200 it gains nothing over 256-row items for the
   // K = 3584 projections and 5-8 % for the down projection at 384-640 tokens only, so it is off by default.
-  static const bool pair_wide = getenv("BS_GEMM_PAIR_WIDE") && atoi(getenv("BS_GEMM_PAIR_WIDE")) > 0;
-  p.wide = (pair_wide && !dual && N >= 1024) ? 1 : 0;
+  p.wide = (tuning().pair_wide && !dual && N >= 1024) ? 1 : 0;
   p.rows = p.wide ? 512 : 256;
   p.ksub = 1;
   p.n_tiles = (N + p.rows - 1) / p.rows;
@@ -788,12 +747,12 @@ cudaError_t launch_gemm_pair(const bf16* A, int lda, const bf16* W, const bf16* 
   // The tensor-core time of a work item is linear in its token-tile width.  When the number of weight tiles does not
   // divide the grid (the LLaDA-shaped gate/up has 48 for 74 pairs), slightly narrower token tiles that fill the last
   // round of work items finish earlier; measured for the SwiGLU GEMM only (up to -3.5 %), where items are long.
-  if (dual && (long long)p.n_tiles * p.m_tiles > g_max_pairs) {
+  if (dual && (long long)p.n_tiles * p.m_tiles > max_pairs) {
     const int lo = p.m_tiles;
     long long best_cost = -1;
     for (int mt = lo; mt <= lo + lo / 2 + 1; ++mt) {
       const int tn = (((M + mt - 1) / mt) + 15) / 16 * 16;
-      const long long rounds = ((long long)p.n_tiles * mt + g_max_pairs - 1) / g_max_pairs;
+      const long long rounds = ((long long)p.n_tiles * mt + max_pairs - 1) / max_pairs;
       const long long cost = rounds * (tn + 48);            // + a fixed per-item cost (ramp, exposed epilogue)
       if (best_cost < 0 || cost < best_cost) { best_cost = cost; p.m_tiles = mt; }
     }
@@ -807,28 +766,30 @@ cudaError_t launch_gemm_pair(const bf16* A, int lda, const bf16* W, const bf16* 
   if (p.stages > 16) p.stages = 16;
   p.splits = 1;
   const long long base_items = (long long)p.n_tiles * p.m_tiles;
-  if (scratch.partial && !dual && base_items * 4 < (long long)g_max_pairs * 3) {
-    int sp = (int)(g_max_pairs / base_items);
-    static const int sp_cap = getenv("BS_GEMM_PAIR_SPLITS") ? atoi(getenv("BS_GEMM_PAIR_SPLITS")) : 8;
-    if (sp > sp_cap) sp = sp_cap;
+  if (scratch.partial && !dual && base_items * 4 < (long long)max_pairs * 3) {
+    int sp = (int)(max_pairs / base_items);
+    if (sp > tuning().pair_splits) sp = tuning().pair_splits;
     if (sp > 8) sp = 8;
     while (sp > 1 && (p.kblocks / sp < 4 || (size_t)sp * (size_t)M * N > scratch.partial_floats)) --sp;
     p.splits = sp < 1 ? 1 : sp;
   }
   if (mode == 4 && (!scratch.partial || (size_t)p.splits * (size_t)M * N > scratch.partial_floats))
-    return cudaErrorInvalidValue;
+    return decline("partial-sum scratch too small for this projection");
   p.partial = scratch.partial;
   if (splits_out) *splits_out = p.splits;
   CUtensorMap mw, mw2, mx;
-  if (!get_map(W, N, K, K, TILE_N, &mw)) return cudaSuccess;
-  if (dual) { if (!get_map(W2, N, K, K, TILE_N, &mw2)) return cudaSuccess; } else { mw2 = mw; }
-  if (!get_map(A, M, K, lda, p.tn / 2, &mx)) return cudaSuccess;
-  *handled = true;
+  if (!get_map(W, N, K, K, TILE_N, &mw)) return decline("tensor map of the weight matrix could not be encoded");
+  if (dual) {
+    if (!get_map(W2, N, K, K, TILE_N, &mw2)) return decline("tensor map of the second weight matrix could not be encoded");
+  } else {
+    mw2 = mw;
+  }
+  if (!get_map(A, M, K, lda, p.tn / 2, &mx)) return decline("tensor map of the activations could not be encoded");
   const long long items = base_items * p.splits;
-  static const bool dbg = getenv("BS_GEMM_DEBUG") != nullptr;
-  if (dbg) fprintf(stderr, "pair gemm M=%d N=%d K=%d mode=%d tn=%d m_tiles=%d n_tiles=%d splits=%d stages=%d\n", M, N, K, mode, p.tn, p.m_tiles, p.n_tiles, p.splits, p.stages);
-  const int pairs = (int)(items < g_max_pairs ? items : g_max_pairs);
-  static const bool no_pdl = getenv("BS_NO_PDL") != nullptr;
+  if (tuning().debug)
+    fprintf(stderr, "pair gemm M=%d N=%d K=%d mode=%d tn=%d m_tiles=%d n_tiles=%d splits=%d stages=%d\n", M, N, K, mode,
+            p.tn, p.m_tiles, p.n_tiles, p.splits, p.stages);
+  const int pairs = (int)(items < max_pairs ? items : max_pairs);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2 * pairs);
   cfg.blockDim = dim3(kThreads);
@@ -840,65 +801,57 @@ cudaError_t launch_gemm_pair(const bf16* A, int lda, const bf16* W, const bf16* 
   attrs[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attrs[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attrs;
-  cfg.numAttrs = no_pdl ? 1 : 2;
+  cfg.numAttrs = tuning().no_pdl ? 1 : 2;
   cudaError_t r = cudaLaunchKernelEx(&cfg, kernel_pair((p.splits > 1 || mode == 4) ? 4 : mode), mw, mw2, mx, p);
   if (r != cudaSuccess) return r;
-  if (p.splits > 1 && mode != 4) {
-    const size_t total = (size_t)M * N;
-    const int blocks = (int)((total + 255) / 256 < (size_t)g_num_sms * 8 ? (total + 255) / 256 : (size_t)g_num_sms * 8);
-    r = launch_pdl(k_gemm_finish, dim3(blocks), dim3(256), 0, s, (const float*)scratch.partial, p.splits, M, N, mode, C,
-                   ldc, row_scale);
-  }
+  if (p.splits > 1 && mode != 4) r = launch_finish(p, mode, dv.num_sms, s);
   return r;
 }
 
 }  // namespace
 
+const char* gemm_decline_reason() { return g_decline.c_str(); }
+
+// Plans and launches one projection.  A shape the tensor-core kernels cannot take is an error
+// (cudaErrorNotSupported, reason in gemm_decline_reason()): there is no second GEMM implementation behind this one.
 cudaError_t launch_gemm_tc(const bf16* A, int lda, const bf16* W, const bf16* W2, void* C, int ldc, int M, int N,
                            int K, int mode, const float* row_scale, const GemmScratch& scratch, cudaStream_t s,
-                           bool* handled, int* splits_out) {
+                           int* splits_out) {
   float* const g_partial = scratch.partial;
   const size_t g_partial_floats = scratch.partial_floats;
-  int* const g_error_flag = scratch.error_flag;
-  *handled = false;
   if (M <= 0 || N <= 0) return cudaSuccess;
   if (K % 8 || lda % 8 || ((uintptr_t)A & 15) || ((uintptr_t)W & 15) || (W2 && ((uintptr_t)W2 & 15)))
-    return cudaSuccess;                       // TMA needs 16-byte aligned rows: leave it to the legacy kernel
-  if (!g_num_sms) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev);
-    if (!allow_big_smem(kernel_tc)) return cudaSuccess;
-  }
+    return decline("operand rows must be 16-byte aligned (K and lda multiples of 8)");
+  const DevInfo* dvp = dev_info();
+  if (!dvp || !dvp->tc_ok) return decline("the device does not grant the kernels' shared-memory budget");
+  const DevInfo& dv = *dvp;
+  const int num_sms = dv.num_sms;
   // CTA pairs that share each token tile move fewer bytes per flop and are faster per work item (measured on B200:
   // +8 to +20 %), but their grid has half as many workers.  From 128 tokens on, the pair plan is taken unless it
   // would leave clearly more of its grid idle than the single-CTA plan (few 256-row tiles and no k split, or a last
-  // round that is mostly empty).  BS_GEMM_PAIR=0 turns pairs off, a positive value sets the smallest M for them.
-  static const int pair_env = getenv("BS_GEMM_PAIR") ? atoi(getenv("BS_GEMM_PAIR")) : -1;
+  // round that is mostly empty).
   bool use_pair = false;
-  if (pair_env >= 0) use_pair = pair_env > 0 && M >= pair_env;
-  else if (M >= 128 && ensure_pair_init() > 0) {
-    const bool dual_ = mode == 3;
-    const int kb = (K + BK - 1) / BK;
-    const long long items_p = (long long)((N + 255) / 256) * ((M + 255) / 256);
-    const double busy_p =
-        grid_busy(items_p * split_for(items_p, g_max_pairs, kb, (size_t)M * N, scratch, dual_), g_max_pairs);
-    const bool wide_s = !dual_ && N >= 512 && K >= 8192;
-    const int tn_cap_s = (dual_ && (M <= 128 || M > 256)) ? 128 : 256;
-    const long long items_s = (long long)((N + (wide_s ? 255 : 127)) / (wide_s ? 256 : 128)) * ((M + tn_cap_s - 1) / tn_cap_s);
-    const double busy_s =
-        grid_busy(items_s * split_for(items_s, g_num_sms, kb, (size_t)M * N, scratch, dual_), g_num_sms);
-    use_pair = busy_p * 1.1 >= busy_s;
+  if (dv.max_pairs > 0) {
+    if (tuning().pair >= 0) use_pair = tuning().pair > 0 && M >= tuning().pair;
+    else if (M >= 128) {
+      const bool dual_ = mode == 3;
+      const int kb = (K + BK - 1) / BK;
+      const long long items_p = (long long)((N + 255) / 256) * ((M + 255) / 256);
+      const double busy_p =
+          grid_busy(items_p * split_for(items_p, dv.max_pairs, kb, (size_t)M * N, scratch, dual_), dv.max_pairs);
+      const bool wide_s = !dual_ && N >= 512 && K >= 8192;
+      const int tn_cap_s = (dual_ && (M <= 128 || M > 256)) ? 128 : 256;
+      const long long items_s = (long long)((N + (wide_s ? 255 : 127)) / (wide_s ? 256 : 128)) * ((M + tn_cap_s - 1) / tn_cap_s);
+      const double busy_s = grid_busy(items_s * split_for(items_s, num_sms, kb, (size_t)M * N, scratch, dual_), num_sms);
+      use_pair = busy_p * 1.1 >= busy_s;
+    }
   }
-  if (use_pair) {
-    cudaError_t r = launch_gemm_pair(A, lda, W, W2, C, ldc, M, N, K, mode, row_scale, scratch, s, handled, splits_out);
-    if (*handled || r != cudaSuccess) return r;
-  }
+  if (use_pair) return launch_gemm_pair(dv, A, lda, W, W2, C, ldc, M, N, K, mode, row_scale, scratch, s, splits_out);
   const int dual = mode == 3;
   GemmParams p;
   p.M = M; p.N = N; p.K = K; p.mode = mode; p.dual = dual; p.C = C; p.ldc = ldc; p.row_scale = row_scale;
   p.n_tiles = (N + TILE_N - 1) / TILE_N;
-  p.error_flag = g_error_flag;
+  p.error_flag = scratch.error_flag;
   // ---- token tile and k split ----
   // Few tokens (a block step): one or two token tiles that cover M exactly (UMMA N is any multiple of 16), and a
   // k split that spreads the weight stream over all SMs when there are fewer weight tiles than SMs.
@@ -908,7 +861,7 @@ cudaError_t launch_gemm_tc(const bf16* A, int lda, const bf16* W, const bf16* W2
   // twice over only up to 128 tokens; wider token tiles run single-buffered (the epilogue is then not overlapped),
   // which pays only when the main loop is long: measured on B200, 256-row items win for K >= 8192 (the down
   // projection: -25 % at M >= 512) and lose or tie for K = 3584.
-  static const bool wide_off = getenv("BS_GEMM_WIDE") && atoi(getenv("BS_GEMM_WIDE")) == 0;
+  const bool wide_off = tuning().wide_off;
   p.wide = (!dual && !wide_off && M >= 128 && N >= 512 && K >= 8192) ? 1 : 0;
   p.rows = p.wide ? 2 * TILE_N : TILE_N;
   p.n_tiles = (N + p.rows - 1) / p.rows;
@@ -921,49 +874,47 @@ cudaError_t launch_gemm_tc(const bf16* A, int lda, const bf16* W, const bf16* W2
   p.acc1_off = p.nbuf == 1 ? 256 : 128;
   // narrow token tiles are weight-streaming bound: 128-wide k stages halve the per-stage barrier round trips
   p.ksub = p.tn <= 64 ? 2 : 1;
-  if (const char* ev = getenv("BS_GEMM_KSUB")) p.ksub = atoi(ev) == 2 ? 2 : 1;
+  if (tuning().ksub) p.ksub = tuning().ksub == 2 ? 2 : 1;
   p.kblocks = (K + BK * p.ksub - 1) / (BK * p.ksub);
   p.splits = 1;
   const long long base_items = (long long)p.n_tiles * p.m_tiles;
-  if (g_partial && base_items * 4 < (long long)g_num_sms * 3) {
-    int sp = (int)(g_num_sms / base_items);
+  if (g_partial && base_items * 4 < (long long)num_sms * 3) {
+    int sp = (int)(num_sms / base_items);
     if (sp > 8) sp = 8;
     while (sp > 1 && (p.kblocks / sp < 4 || (size_t)sp * (size_t)M * N > g_partial_floats)) --sp;
     p.splits = sp < 1 ? 1 : sp;
   }
-  if (const char* ev = getenv("BS_GEMM_SPLITS")) {
-    const int sp = atoi(ev);
+  if (const int sp = tuning().splits)
     if (sp >= 1 && sp <= 8 && (sp == 1 || (g_partial && (size_t)sp * (size_t)M * N <= g_partial_floats))) p.splits = sp;
-  }
-  if (mode == 4 && (!g_partial || (size_t)p.splits * (size_t)M * N > g_partial_floats)) return cudaErrorInvalidValue;
+  if (mode == 4 && (!g_partial || (size_t)p.splits * (size_t)M * N > g_partial_floats))
+    return decline("partial-sum scratch too small for this projection");
   if (dual) p.splits = 1;
   p.partial = g_partial;
   if (splits_out) *splits_out = p.splits;
   const int stage_bytes = p.ksub * ((two_a ? 2 : 1) * TILE_N * BK * 2 + p.tn * BK * 2);
   p.stages = kSmemBudget / stage_bytes;
-  if (const char* ev = getenv("BS_GEMM_STAGES")) { const int st = atoi(ev); if (st >= 2 && st < p.stages) p.stages = st; }
+  if (const int st = tuning().stages) { if (st >= 2 && st < p.stages) p.stages = st; }
   if (p.stages > 16) p.stages = 16;
-  if (p.stages < 2) return cudaSuccess;
+  if (p.stages < 2) return decline("operand stages do not fit shared memory");
 
   CUtensorMap mw, mw2, mx;
-  if (!get_map(W, N, K, K, TILE_N, &mw)) return cudaSuccess;
-  if (dual) { if (!get_map(W2, N, K, K, TILE_N, &mw2)) return cudaSuccess; } else { mw2 = mw; }
-  if (!get_map(A, M, K, lda, p.tn, &mx)) return cudaSuccess;
+  if (!get_map(W, N, K, K, TILE_N, &mw)) return decline("tensor map of the weight matrix could not be encoded");
+  if (dual) {
+    if (!get_map(W2, N, K, K, TILE_N, &mw2)) return decline("tensor map of the second weight matrix could not be encoded");
+  } else {
+    mw2 = mw;
+  }
+  if (!get_map(A, M, K, lda, p.tn, &mx)) return decline("tensor map of the activations could not be encoded");
 
-  *handled = true;
   const long long items = (long long)p.n_tiles * p.m_tiles * p.splits;
-  static const bool dbg = getenv("BS_GEMM_DEBUG") != nullptr;
-  if (dbg) fprintf(stderr, "gemm M=%d N=%d K=%d mode=%d tn=%d m_tiles=%d n_tiles=%d splits=%d stages=%d wide=%d nbuf=%d\n", M, N, K, mode, p.tn, p.m_tiles, p.n_tiles, p.splits, p.stages, p.wide, p.nbuf);
-  const int grid = (int)(items < g_num_sms ? items : g_num_sms);
+  if (tuning().debug)
+    fprintf(stderr, "gemm M=%d N=%d K=%d mode=%d tn=%d m_tiles=%d n_tiles=%d splits=%d stages=%d wide=%d nbuf=%d\n", M,
+            N, K, mode, p.tn, p.m_tiles, p.n_tiles, p.splits, p.stages, p.wide, p.nbuf);
+  const int grid = (int)(items < num_sms ? items : num_sms);
   cudaError_t r = launch_pdl(kernel_tc((p.splits > 1 || mode == 4) ? 4 : mode), dim3(grid), dim3(kThreads),
                              (size_t)kSmemBudget + 1024, s, mw, mw2, mx, p);
   if (r != cudaSuccess) return r;
-  if (p.splits > 1 && mode != 4) {
-    const size_t total = (size_t)M * N;
-    const int blocks = (int)((total + 255) / 256 < (size_t)g_num_sms * 8 ? (total + 255) / 256 : (size_t)g_num_sms * 8);
-    r = launch_pdl(k_gemm_finish, dim3(blocks), dim3(256), 0, s, (const float*)g_partial, p.splits, M, N, mode, C, ldc,
-                   row_scale);
-  }
+  if (p.splits > 1 && mode != 4) r = launch_finish(p, mode, num_sms, s);
   return r;
 }
 
