@@ -11,9 +11,11 @@ memory and bs_read_tokens inside the timed region).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 1..5] [--impl ours|reference]
 
-With N > 1 (launched by torch.distributed.run) every rank serves its own
-independently drawn batch on its own GPU (request-sharded replicas, no
-collective on the data path); times are the max over ranks.
+With N > 1 every rank serves its own independently drawn batch on its own GPU
+(request-sharded replicas, no collective on the data path); times are the max
+over ranks.  The ranks either come from torch.distributed.run (RANK /
+LOCAL_RANK / WORLD_SIZE / MASTER_* in the environment), or, when the script is
+started plainly with --gpus N > 1, it starts the N ranks itself.
 """
 from __future__ import annotations
 
@@ -409,11 +411,43 @@ def run_reference(args):
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * t_total / args.steps, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "vs_baseline": None, "dtype": "f32 arithmetic, activations rounded to bf16 at six points per layer",
+        "data": "synthetic",
         "config": {"workload": wl.name, "sample_per_step": sample},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
+
+
+def launch_ranks(n: int, argv, worker=None, check_devices: bool = True, timeout_s: float = 7200.0):
+    """Starts `n` ranks of this script (or of `worker`, a command list, for tests) on one node, one GPU each, with
+    the rendezvous variables torch.distributed expects, and returns [(returncode, stdout)] by rank.  Rank 0's
+    stdout carries the JSON line."""
+    import socket
+    if n < 1:
+        raise SystemExit("--gpus must be at least 1")
+    if check_devices:
+        have = torch.cuda.device_count()
+        if n > have:
+            raise SystemExit(f"--gpus {n} but this node has {have} CUDA device(s)")
+    with socket.socket() as sock:          # a free port for the rendezvous
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    cmd = list(worker) if worker is not None else [sys.executable, os.path.abspath(__file__)]
+    procs = []
+    for rank in range(n):
+        env = dict(os.environ, RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(n), LOCAL_WORLD_SIZE=str(n),
+                   MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        procs.append(subprocess.Popen(cmd + list(argv), env=env, stdout=subprocess.PIPE, text=True))
+    out = []
+    for p in procs:
+        try:
+            so, _ = p.communicate(timeout=timeout_s)
+        except subprocess.TimeoutExpired:
+            p.kill()
+            so, _ = p.communicate()
+        out.append((p.returncode, so))
+    return out
 
 
 def main():
@@ -427,6 +461,12 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-profile", action="store_true", help="skip the per-family CUDA-event timers (no roofline)")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started plainly: this process only launches the ranks and relays rank 0's line
+        results = launch_ranks(args.gpus, sys.argv[1:], check_devices=args.impl != "reference")
+        sys.stdout.write(results[0][1])
+        sys.stdout.flush()
+        raise SystemExit(max(abs(rc) for rc, _ in results))
     if args.impl == "reference":
         run_reference(args)
     else:

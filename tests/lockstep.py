@@ -1,47 +1,76 @@
 """Lockstep comparison of the CUDA engine with the CPU oracle (test infrastructure).
 
 Both sides are fed the same seeded requests and weights.  Before every step the
-gather / scatter indices are compared bit for bit.  After it:
+gather / scatter indices are compared bit for bit.  After it, for every tracked
+row, the engine's logits, token ids, confidences and commit decisions are
+compared with the oracle in BOTH of its precision modes:
 
- (1) logits of every still-masked row: max |z_gpu - z_ref| / max |z_ref| <= 2e-2.
+  "fp32"  the pure fp32 oracle: the one the stated tolerance (2e-2 max relative
+          error on logits and confidences, bf16 GPU vs fp32 oracle) is worded for;
+  "bf16"  the oracle that rounds six activation tensors per layer to bf16 where the
+          CUDA path stores them.  The oracle's trajectory follows this mode, and
+          decisions are resynchronised against it.
+
+Per mode the harness records the largest logit and confidence error and HOW MANY
+rows lie outside the flat 2e-2 bound ("met" means none); nothing is hidden behind a
+widened tolerance: the assertions that keep a test green are stated separately below.
+
+ (1) logits of every still-masked row: err = max |z_gpu - z_ref| / max |z_ref|.
+     Asserted: err <= logit_tol(n_layers) against the bf16 mode (a bound derived from
+     bf16 rounding at that depth), err <= RAW_TOL against the fp32 mode (rounding
+     only, nothing structural).  Counted against 2e-2 in both modes.
  (2) the epilogue and the commit rule are checked EXACTLY on the engine's own
      logits: the oracle's confidence() applied to the engine's logits must give
      the engine's token ids bit for bit and its confidences to 1e-4, and the
      oracle's commit_set() applied to the engine's confidences must give the
      engine's commit decisions bit for bit (same fp32 data, same rule).
- (3) against the oracle's own trajectory: ln(conf) is 2-Lipschitz in the sup
-     norm of the logits (conf = exp(z_max - logsumexp z)), so with D = max |z_gpu -
-     z_ref| over the row, |ln c_gpu - ln c_ref| <= 2 D must hold; rows that also
-     meet the flat 2e-2 relative bound are counted.  Token ids and commit
-     decisions must agree except at near ties, where the oracle adopts the
-     engine's decision so that the trajectories stay comparable.  Each exception
-     is counted in its class:
-       "tau"    oracle confidence within 1e-2 of tau
-       "top2"   oracle's top-2 logit gap below 1e-2
+ (3) confidences: ln(conf) is 2-Lipschitz in the sup norm of the logits
+     (conf = exp(z_max - logsumexp z)), so with D = max |z_gpu - z_ref| over the row
+     |ln c_gpu - ln c_ref| <= 2 D must hold (asserted, both modes); rows with
+     2 D <= 2e-2 must therefore meet the flat 2e-2 relative bound (asserted), and all
+     rows are counted against it.
+ (4) token ids and commit decisions must agree with the bf16-mode oracle except at
+     near ties, where the oracle adopts the engine's decision so that the
+     trajectories stay comparable.  Each exception is counted in its class:
+       "tau"    oracle confidence within 1e-2 of tau            } the two classes the
+       "top2"   oracle's top-2 logit gap below 1e-2             } contract allows
        "forced" forced pick: oracle confidence at the engine's position within
-                2e-2 relative of the oracle's maximum
+                2e-2 relative of the oracle's maximum (the tolerance the contract
+                grants on confidences)
        "noise"  none of the above, but the flip is explained by the measured
                 logit deviation D of that row: top-2 gap < 2 D, or tau inside
-                [c e^{-2D}, c e^{+2D}], or forced-pick confidences within e^{-4D}
-     Anything else fails.
+                [c e^{-2D}, c e^{+2D}], or forced-pick confidences within e^{-4D}.
+                D itself is bounded by (1): D <= logit_tol * max |z_ref|.
+     Anything else fails.  assert_caps() bounds every class on its own.
+     Against the fp32 mode, disagreements are counted (inside / outside the two
+     allowed classes) and reported, not resynchronised.
+ (5) check_free_run(): every tracked request is run again by the oracle ALONE,
+     without adopting anything from the engine; the engine's committed tokens must
+     equal that run's up to the block of the request's first counted exception
+     (all of them when it has none).
 """
 from __future__ import annotations
+
+import dataclasses
 
 import numpy as np
 
 from oracle import blockserve_oracle as O
 from paper_2607_08930_b200 import binding as B
 
-LOGIT_TOL = 2e-2      # max |z_gpu - z_ref| / max |z_ref| per row
-CONF_TOL = 2e-2       # relative
+LOGIT_TOL = 2e-2      # stated: max |z_gpu - z_ref| / max |z_ref| per row
+CONF_TOL = 2e-2       # stated: relative
+RAW_TOL = 8e-2        # sanity bound against the pure fp32 oracle (rounding only)
+CLASSES = ("tau", "top2", "forced", "noise")
 
 
 def logit_tol(n_layers: int) -> float:
-    """Logit tolerance for a model of this depth.  Both sides store six activation tensors per layer in bf16; each
-    rounding adds a relative error of about 2^-9 / sqrt(3), rounding is discontinuous, and after a few layers the
-    two pipelines round independently, so their logits differ by about 2^-9/sqrt(3) * sqrt(2 * 6 * n_layers)
-    relative (5e-3 at 2 layers, 2e-2 at 28).  The bound is the stated 2e-2 up to the depth where that estimate
-    with a safety factor of 2.5 (the maximum over a 150k-entry row sits above the rms) exceeds it."""
+    """Asserted logit bound against the bf16-mode oracle for a model of this depth.  Both sides store six activation
+    tensors per layer in bf16; each rounding adds a relative error of about 2^-9 / sqrt(3), rounding is discontinuous,
+    and after a few layers the two pipelines round independently, so their logits differ by about
+    2^-9/sqrt(3) * sqrt(2 * 6 * n_layers) relative (5e-3 at 2 layers, 2e-2 at 28).  The bound is the stated 2e-2 up
+    to the depth where that estimate with a safety factor of 2.5 (the maximum over a 150k-entry row sits above the
+    rms) exceeds it.  Whether the stated 2e-2 itself is met is reported separately (rows outside it are counted)."""
     return max(LOGIT_TOL, 2.5 * (2.0 ** -9 / np.sqrt(3.0)) * np.sqrt(2.0 * 6.0 * n_layers))
 
 
@@ -70,38 +99,80 @@ def lazy_oracle_model(shape, weights):
                    f32("lm_head", weights["lm_head"]), f32("final_norm", weights["final_norm"]), layer)
 
 
+@dataclasses.dataclass
+class ModeStats:
+    """What one oracle mode saw over the tracked rows."""
+    rows: int = 0
+    max_logit_err: float = 0.0
+    rows_over_logit_tol: int = 0        # rows with err > 2e-2
+    max_conf_err: float = 0.0
+    rows_over_conf_tol: int = 0         # rows with |c_gpu - c_ref| / c_ref > 2e-2
+    rows_flat_conf_bound_applies: int = 0   # rows with 2 D <= 2e-2 (the flat bound is then implied and asserted)
+    tok_diff_allowed: int = 0           # token differs, oracle top-2 gap < 1e-2
+    tok_diff_other: int = 0
+    commit_diff_allowed: int = 0        # commit differs, oracle confidence within 1e-2 of tau
+    commit_diff_other: int = 0
+
+    def met(self) -> str:
+        lz = "met" if self.rows_over_logit_tol == 0 else f"NOT met ({self.rows_over_logit_tol} rows over)"
+        cf = "met" if self.rows_over_conf_tol == 0 else f"NOT met ({self.rows_over_conf_tol} rows over)"
+        return f"logits 2e-2: {lz}; confidences 2e-2: {cf}"
+
+
 class Lockstep:
     """`track`: request ids whose floating-point results and decisions are compared (None: all).  The other rows
     are still part of every integer check (indices, row order, slabs, mask words, counts): their oracle state
-    adopts the engine's mask word after each step, since the oracle does not run their forward."""
+    adopts the engine's mask word after each step, since the oracle does not run their forward.
+    `modes`: which oracle modes are computed for tracked rows; "bf16" always is (it carries the trajectory)."""
 
     def __init__(self, wl, weights_cuda, weights_np, suffix_mode=0, kv_capacity=None, sort_queue=True, track=None,
-                 model=None, steps_per_block=0, eos_id=-1, static_groups=False):
+                 model=None, steps_per_block=0, eos_id=-1, static_groups=False, modes=("bf16", "fp32"),
+                 engine_kwargs=None):
         self.wl = wl
         self.track = None if track is None else set(track)
         # the near-tie classes below are written for one forced token per step; a general transfer quota is checked
         # through the exact commit-rule and bookkeeping comparisons of untracked rows
         assert not steps_per_block or steps_per_block == wl.block_len or self.track == set()
         self.S = steps_per_block if steps_per_block else wl.block_len
+        self.eos_id = eos_id
         self.eng = B.engine_for_workload(wl, weights_cuda, kv_capacity_tokens=kv_capacity, suffix_mode=suffix_mode,
                                          sort_queue=sort_queue, steps_per_block=steps_per_block, eos_id=eos_id,
-                                         static_groups=static_groups)
+                                         static_groups=static_groups, **(engine_kwargs or {}))
         self.model = model if model is not None else O.model_from_weights(wl.shape, weights_np)
+        assert self.model.bf16_activations
+        self.model32 = dataclasses.replace(self.model, bf16_activations=False) if "fp32" in modes else None
         self.ora = O.Engine(self.model, wl.block_len, wl.tau, wl.token_budget, wl.max_batch,
                             self.eng.cfg.kv_capacity_tokens, suffix_mode, sort_queue, steps_per_block=steps_per_block,
                             eos_id=eos_id, static_groups=static_groups)
+        self.shadow = {}                 # req_id -> the fp32-mode oracle's copy of a tracked request
         self.suffix_mode = suffix_mode
-        self.excluded = {"tau": 0, "top2": 0, "forced": 0, "noise": 0}
-        self.conf_rows_within_tol = 0
+        self.excluded = {c: 0 for c in CLASSES}
+        self.first_exception = {}        # req_id -> block index of its first counted exception
+        self.stats = {"bf16": ModeStats(), "fp32": ModeStats()}
         self.rows_checked = 0
-        self.max_logit_err = 0.0
-        self.max_conf_err = 0.0
         self.steps = 0
+        self.reqs = {}
+
+    # kept names: maxima against the bf16-mode oracle
+    @property
+    def max_logit_err(self):
+        return self.stats["bf16"].max_logit_err
+
+    @property
+    def max_conf_err(self):
+        return self.stats["bf16"].max_conf_err
+
+    def tracked(self, req_id) -> bool:
+        return self.track is None or req_id in self.track
 
     def admit(self, reqs):
         for r in reqs:
             self.eng.admit(r.req_id, r.prompt, r.g, r.alpha, r.start_block, r.gen_prefix)
             self.ora.admit(r.req_id, r.prompt, r.g, r.alpha, r.start_block, r.gen_prefix)
+            self.reqs[r.req_id] = r
+            if self.model32 is not None and self.tracked(r.req_id):
+                self.shadow[r.req_id] = O.new_request(self.model32, r.req_id, r.prompt, r.g, r.alpha,
+                                                      self.wl.block_len, r.start_block, r.gen_prefix)
 
     def evict_refill(self):
         ev_o, ad_o, n_o = self.ora.evict_refill()
@@ -112,6 +183,9 @@ class Lockstep:
         if n:
             kvb = self.eng.debug(B.DBG_ROW_KV_BASE)
             assert kvb.tolist() == [r.kv_base for r in self.ora.sched.active], "KV slabs differ"
+        for rid in ev_o:
+            if rid in self.shadow:
+                self.shadow[rid].K = self.shadow[rid].V = None
         return ev_o, ad_o, n
 
     def check_indices(self):
@@ -127,6 +201,37 @@ class Lockstep:
         assert self.eng.debug(B.DBG_LM_ROW, cap=cap).tolist() == ix["lm_row"].tolist()
         assert self.eng.debug(B.DBG_LM_SLOT, cap=cap).tolist() == ix["lm_slot"].tolist()
         return ix
+
+    def _count(self, cls, r):
+        self.excluded[cls] += 1
+        self.first_exception.setdefault(r.req_id, r.b)
+
+    def _mode_stats(self, mode, zl, gc, gt, gs, probe, where):
+        """Logit / confidence errors of the engine's rows against one oracle record; returns D per row."""
+        st = self.stats[mode]
+        dev = np.abs(zl - probe.logits).max(-1)                       # D per row
+        err = dev / np.abs(probe.logits).max(-1)
+        st.rows += len(err)
+        st.max_logit_err = max(st.max_logit_err, float(err.max()))
+        st.rows_over_logit_tol += int((err > LOGIT_TOL).sum())
+        bound = logit_tol(self.model.n_layers) if mode == "bf16" else RAW_TOL
+        assert err.max() <= bound, f"logit error {err.max():.3e} vs the {mode}-mode oracle ({where})"
+        dln = np.abs(np.log(gc.astype(np.float64)) - np.log(probe.conf.astype(np.float64)))
+        assert (dln <= 2.0 * dev + 1e-4).all(), f"confidence outside the Lipschitz bound, {mode} mode ({where})"
+        cerr = np.abs(gc - probe.conf) / probe.conf
+        st.max_conf_err = max(st.max_conf_err, float(cerr.max()))
+        st.rows_over_conf_tol += int((cerr > CONF_TOL).sum())
+        flat = 2.0 * dev <= CONF_TOL                                  # there |ln c_gpu - ln c_ref| <= 2e-2
+        st.rows_flat_conf_bound_applies += int(flat.sum())
+        assert (cerr[flat] <= np.expm1(CONF_TOL) + 1e-4).all(), f"flat confidence bound, {mode} mode ({where})"
+        tok_diff = gt != probe.tok
+        st.tok_diff_allowed += int((tok_diff & (probe.top2_gap < 1e-2)).sum())
+        st.tok_diff_other += int((tok_diff & ~(probe.top2_gap < 1e-2)).sum())
+        com_diff = gs != probe.committed
+        near_tau = np.abs(probe.conf - np.float32(self.wl.tau)) < 1e-2
+        st.commit_diff_allowed += int((com_diff & near_tau).sum())
+        st.commit_diff_other += int((com_diff & ~near_tau).sum())
+        return dev
 
     def step(self):
         ix = self.check_indices()
@@ -157,7 +262,7 @@ class Lockstep:
             gt, gc, gs = g_tok[k:k + nm], g_conf[k:k + nm], g_commit[k:k + nm]
             where = f"req {r.req_id} block {r.b} step {r.s}"
             quota = O.transfer_quota(self.wl.block_len, self.S, r.s)
-            if self.track is not None and r.req_id not in self.track:
+            if not self.tracked(r.req_id):
                 # untracked row: integer bookkeeping only; the commit rule is still checked on the engine's own data
                 assert (O.commit_set(gc.copy(), self.wl.tau, quota) == gs).all(), f"commit rule ({where})"
                 slots = [j for j in range(32) if (r.mask >> j) & 1]
@@ -171,37 +276,38 @@ class Lockstep:
                 r.s += 1
                 k += nm
                 continue
+            if g_logits is not None:
+                zl = g_logits[k:k + nm]
+            else:       # only the tracked rows' logits are read back
+                zl = self.eng.debug(B.DBG_PREV_LOGITS, np.float32, arg0=k, arg1=nm, cap=4 * nm * V + 64).reshape(nm, V)
+            # the fp32-mode oracle follows the same request state (integers and tokens are shared by construction)
+            if self.model32 is not None:
+                sh = self.shadow[r.req_id]
+                assert (sh.tokens == r.tokens).all()
+                sh.b, sh.s, sh.mask = r.b, r.s, r.mask
+                probe32 = O.denoise_step(self.model32, sh, self.wl.block_len, self.wl.tau, self.suffix_mode,
+                                         keep_logits=True, override_commit=gs, override_tok=gt,
+                                         steps_per_block=self.S)
+                self._mode_stats("fp32", zl, gc, gt, gs, probe32, where)
             # the record holds what the oracle computes on its own; the oracle then advances with the engine's
             # decisions (identical unless a near tie is counted below)
             probe = O.denoise_step(self.model, r, self.wl.block_len, self.wl.tau, self.suffix_mode,
                                    keep_logits=True, override_commit=gs, override_tok=gt,
                                    steps_per_block=self.S)
-            if g_logits is not None:
-                zl = g_logits[k:k + nm]
-            else:       # only the tracked rows' logits are read back
-                zl = self.eng.debug(B.DBG_PREV_LOGITS, np.float32, arg0=k, arg1=nm, cap=4 * nm * V + 64).reshape(nm, V)
-            # (1) logits
-            dev = np.abs(zl - probe.logits).max(-1)                       # D per row
-            err = dev / np.abs(probe.logits).max(-1)
-            self.max_logit_err = max(self.max_logit_err, float(err.max()))
-            assert err.max() <= logit_tol(self.model.n_layers), f"logit error {err.max():.3e} ({where})"
+            # (1), (3) logits and confidences
+            dev = self._mode_stats("bf16", zl, gc, gt, gs, probe, where)
             # (2) epilogue and commit rule, exact on the engine's own data
             tok2, conf2 = O.confidence(zl, mask_id)
             assert (gt == tok2).all(), f"argmax differs from the oracle's on identical logits ({where})"
             assert (np.abs(gc - conf2) <= 1e-4 * conf2).all(), f"confidence kernel error ({where})"
             assert (O.commit_set(gc.copy(), self.wl.tau, quota) == gs).all(), f"commit rule differs on identical data ({where})"
-            # (3) against the oracle's own trajectory
-            dln = np.abs(np.log(gc.astype(np.float64)) - np.log(probe.conf.astype(np.float64)))
-            assert (dln <= 2.0 * dev + 1e-4).all(), f"confidence outside the Lipschitz bound ({where})"
-            cerr = np.abs(gc - probe.conf) / probe.conf
-            self.max_conf_err = max(self.max_conf_err, float(cerr.max()))
-            self.conf_rows_within_tol += int((cerr <= CONF_TOL).sum())
+            # (4) decisions against the oracle's own trajectory
             tok_diff = gt != probe.tok
             for j in np.nonzero(tok_diff)[0]:
                 if probe.top2_gap[j] < 1e-2:
-                    self.excluded["top2"] += 1
+                    self._count("top2", r)
                 elif probe.top2_gap[j] < 2.0 * dev[j]:
-                    self.excluded["noise"] += 1
+                    self._count("noise", r)
                 else:
                     raise AssertionError(f"token differs with top-2 gap {probe.top2_gap[j]:.4f}, D {dev[j]:.4f} ({where})")
             o_forced = int(np.argmax(probe.conf))
@@ -212,23 +318,23 @@ class Lockstep:
             for j in np.nonzero(diff)[0]:
                 c, d2 = float(probe.conf[j]), 2.0 * float(dev[j])
                 if abs(c - float(tau)) < 1e-2:
-                    self.excluded["tau"] += 1
+                    self._count("tau", r)
                 elif forced_pair is not None and j in forced_pair:
                     co, cg = float(probe.conf[forced_pair[0]]), float(probe.conf[forced_pair[1]])
                     dd = 2.0 * float(max(dev[forced_pair[0]], dev[forced_pair[1]]))
                     if cg >= (1 - CONF_TOL) * co:
-                        self.excluded["forced"] += 1
+                        self._count("forced", r)
                     elif cg >= np.exp(-2 * dd) * co:
-                        self.excluded["noise"] += 1
+                        self._count("noise", r)
                     else:
                         raise AssertionError(f"forced pick differs: oracle {co:.5f} vs {cg:.5f} ({where})")
                 elif c * np.exp(-d2) <= float(tau) <= c * np.exp(d2):
-                    self.excluded["noise"] += 1
+                    self._count("noise", r)
                 elif not (gc > tau).any() or not (probe.conf > tau).any():
                     # one side forced its best position while the other had a row above tau: explained only if
                     # some row's confidence interval straddles tau
                     if ((probe.conf * np.exp(-2 * dev) <= tau) & (tau <= probe.conf * np.exp(2 * dev))).any():
-                        self.excluded["noise"] += 1
+                        self._count("noise", r)
                     else:
                         raise AssertionError(f"commit differs at slot {j}: conf {c:.5f} ({where})")
                 else:
@@ -258,15 +364,60 @@ class Lockstep:
             cycles += 1
         return cycles
 
-    def summary(self) -> str:
-        return (f"steps {self.steps} masked rows {self.rows_checked} excluded {self.excluded} "
-                f"max logit err {self.max_logit_err:.2e} max conf err {self.max_conf_err:.2e} "
-                f"rows with conf within {CONF_TOL:g}: {self.conf_rows_within_tol}")
+    # ---- reporting and end-of-run assertions ---------------------------------------------------------------
 
-    def check_tokens(self):
-        for r in self.wl.requests:
-            if self.track is not None and r.req_id not in self.track:
+    def summary(self) -> str:
+        parts = [f"steps {self.steps} masked-row decisions {self.rows_checked} exceptions {self.excluded}"]
+        for mode in ("fp32", "bf16"):
+            st = self.stats[mode]
+            if st.rows == 0:
                 continue
-            if r.req_id in self.ora.by_id:
-                got, _ = self.eng.read_tokens(r.req_id)
-                assert (got == self.ora.tokens(r.req_id)).all(), f"token row of request {r.req_id} differs"
+            parts.append(f"[{mode}-mode oracle] max logit err {st.max_logit_err:.2e} max conf err {st.max_conf_err:.2e} "
+                         f"rows within 2e-2 conf: {st.rows - st.rows_over_conf_tol}/{st.rows} "
+                         f"(flat bound implied and asserted on {st.rows_flat_conf_bound_applies}) "
+                         f"token diffs {st.tok_diff_allowed} in the top-2 class + {st.tok_diff_other} outside, "
+                         f"commit diffs {st.commit_diff_allowed} in the tau class + {st.commit_diff_other} outside; "
+                         f"{st.met()}")
+        return " | ".join(parts)
+
+    def assert_caps(self, allowed_cap=0.05, forced_cap=0.05, noise_cap=0.05, floor=3):
+        """Every exception class is bounded on its own, as a fraction of the masked-row decisions compared (with a
+        floor of a few rows for very short runs).  "tau" and "top2" are the two classes the contract allows;
+        "forced" and "noise" are this harness's additions, never folded into them."""
+        n = max(self.rows_checked, 1)
+        e = self.excluded
+        lim = lambda cap: max(floor, cap * n)
+        assert e["tau"] <= lim(allowed_cap) and e["top2"] <= lim(allowed_cap), \
+            f"too many exceptions in the allowed classes: {e} of {n}"
+        assert e["forced"] <= lim(forced_cap), f"too many forced-pick exceptions: {e} of {n}"
+        assert e["noise"] <= lim(noise_cap), (f"too many exceptions explained only by the measured logit deviation "
+                                              f"(each with D <= {logit_tol(self.model.n_layers):.3f} * max|z|): {e} of {n}")
+
+    def check_free_run(self, req_ids=None) -> dict:
+        """Token parity that can fail: the oracle runs each tracked request ALONE and free (it adopts nothing from
+        the engine; a request's trajectory does not depend on its batch).  The engine's tokens must equal that run's
+        for every block before the request's first counted exception - the whole row when it has none.  Returns how
+        many requests were compared completely / partially / not at all (exception in their first block)."""
+        L = self.wl.block_len
+        out = {"complete": 0, "partial": 0, "none": 0}
+        ids = req_ids if req_ids is not None else [rid for rid in self.ora.by_id if self.tracked(rid)]
+        for rid in ids:
+            q = self.reqs[rid]
+            r = O.new_request(self.model, rid, q.prompt, q.g, q.alpha, L, q.start_block, q.gen_prefix)
+            got, _ = self.eng.read_tokens(rid)
+            stop = self.first_exception.get(rid, r.n_blocks(L))
+            if stop <= q.start_block:
+                out["none"] += 1
+                continue
+            for b in range(q.start_block, stop):
+                r.b = b
+                O.start_block_state(r, L)
+                while r.mask:
+                    O.denoise_step(self.model, r, L, self.wl.tau, self.suffix_mode, steps_per_block=self.S)
+                lo, hi = r.block_range(L)
+                assert (got[lo:hi] == r.tokens[lo:hi]).all(), f"request {rid} block {b}: tokens differ from the free oracle run"
+                if self.eos_id >= 0 and (r.tokens[r.p:hi] == self.eos_id).any():
+                    assert (got[hi:] == self.wl.shape.mask_id).all(), f"request {rid} ran past its end-of-sequence block"
+                    break
+            out["complete" if rid not in self.first_exception else "partial"] += 1
+        return out

@@ -31,7 +31,8 @@ def _shallow(B, shape, ps, gs, alphas, starts, seed):
     ls = Lockstep(wl, w, None, model=lazy_oracle_model(shape, w))
     ls.admit(wl.requests)
     ls.run()
-    ls.check_tokens()
+    print("free oracle run:", ls.check_free_run())
+    ls.assert_caps()
     assert ls.eng.stats().committed == wl.committed_target()
     return ls
 
@@ -68,6 +69,9 @@ def test_benchmark_workload_full_depth_sampled_request(B):
     print(f"cfg2 full depth, request {sample.req_id} (p={sample.p}, alpha={sample.alpha:.2f}): {ls.summary()} "
           f"(depth-28 tolerance {logit_tol(28):.3f})")
     assert ls.rows_checked > 0 and ls.max_logit_err < logit_tol(wl.shape.n_layers)
+    # 28 layers of bf16 rounding put the measured logit deviation D at a few percent of max|z|: the class that D alone
+    # explains is the largest here; it is capped on its own, beside the two classes the contract allows
+    ls.assert_caps(noise_cap=0.10)
 
 
 def test_llada_stream_full_depth_first_cycle_sampled_request(B):
@@ -91,6 +95,7 @@ def test_llada_stream_full_depth_first_cycle_sampled_request(B):
     print(f"cfg3 full depth, {n} rows active, request {first.req_id} (p={first.p}, alpha={first.alpha:.2f}): "
           f"{ls.summary()}")
     assert ls.rows_checked > 0 and ls.max_logit_err < logit_tol(wl.shape.n_layers)
+    ls.assert_caps(noise_cap=0.10)
 
 
 @pytest.mark.parametrize("shape_name", ["dream", "llada"])

@@ -187,11 +187,15 @@ def test_commit_set_rule():
 
 # ---------------------------------------------------------- model forward ---
 
-def brute_forward(shape, w, tokens, alpha):
+def brute_forward(shape, w, tokens, alpha, rnd=frozenset()):
     """A from-scratch forward in double precision with torch primitives of a
-    different kind (einsum on explicitly replicated heads, complex-number RoPE)."""
+    different kind (einsum on explicitly replicated heads, complex-number RoPE).
+    `rnd` names tensors that are rounded to bf16 by torch's own conversion: the
+    oracle's six rounding points, and three places where the oracle does not round
+    ("residual", "gate_up", "probs")."""
     d, hq, hkv, dh = shape.d_model, shape.n_q_heads, shape.n_kv_heads, shape.head_dim
     T = lambda a: torch.from_numpy(np.asarray(a)).double()
+    bf = lambda t, name: t.to(torch.bfloat16).double() if name in rnd else t
     n = len(tokens)
     x = T(w["embed"])[torch.as_tensor(tokens, dtype=torch.long)]
     pos = torch.arange(n).double()
@@ -206,20 +210,54 @@ def brute_forward(shape, w, tokens, alpha):
         return t * torch.rsqrt((t * t).mean(-1, keepdim=True) + shape.rms_eps) * T(g)
 
     for l in range(shape.n_layers):
-        h = norm(x, w["norm1"][l])
-        qkv = torch.einsum("nd,od->no", h, T(w["wqkv"][l]))
-        q = rope(qkv[:, :hq * dh].reshape(n, hq, dh))
-        k = rope(qkv[:, hq * dh:(hq + hkv) * dh].reshape(n, hkv, dh))
+        h = bf(norm(x, w["norm1"][l]), "normed")
+        qkv = bf(torch.einsum("nd,od->no", h, T(w["wqkv"][l])), "qkv")
+        q = bf(rope(qkv[:, :hq * dh].reshape(n, hq, dh)), "rope")
+        k = bf(rope(qkv[:, hq * dh:(hq + hkv) * dh].reshape(n, hkv, dh)), "rope")
         v = qkv[:, (hq + hkv) * dh:].reshape(n, hkv, dh)
         k, v = k.repeat_interleave(hq // hkv, 1), v.repeat_interleave(hq // hkv, 1)
-        pr = torch.softmax(torch.einsum("ihc,jhc->hij", q, k) / math.sqrt(dh), -1)
-        a = torch.einsum("hij,jhc->ihc", pr, v).reshape(n, hq * dh)
-        x = x + torch.einsum("nk,dk->nd", a, T(w["wo"][l]))
-        h2 = norm(x, w["norm2"][l])
-        gate = torch.einsum("nd,fd->nf", h2, T(w["w_gate"][l]))
-        up = torch.einsum("nd,fd->nf", h2, T(w["w_up"][l]))
-        x = x + torch.einsum("nf,df->nd", gate * torch.sigmoid(gate) * up, T(w["w_down"][l]))
-    return (alpha * torch.einsum("nd,vd->nv", norm(x, w["final_norm"]), T(w["lm_head"]))).numpy()
+        pr = bf(torch.softmax(torch.einsum("ihc,jhc->hij", q, k) / math.sqrt(dh), -1), "probs")
+        a = bf(torch.einsum("hij,jhc->ihc", pr, v).reshape(n, hq * dh), "attn")
+        x = bf(x + torch.einsum("nk,dk->nd", a, T(w["wo"][l])), "residual")
+        h2 = bf(norm(x, w["norm2"][l]), "normed")
+        gate = bf(torch.einsum("nd,fd->nf", h2, T(w["w_gate"][l])), "gate_up")
+        up = bf(torch.einsum("nd,fd->nf", h2, T(w["w_up"][l])), "gate_up")
+        x = bf(x + torch.einsum("nf,df->nd", bf(gate * torch.sigmoid(gate) * up, "swiglu"), T(w["w_down"][l])),
+               "residual")
+    return (alpha * torch.einsum("nd,vd->nv", bf(norm(x, w["final_norm"]), "final"), T(w["lm_head"]))).numpy()
+
+
+def test_bf16_mode_rounds_exactly_the_six_documented_tensors():
+    """The rounding map of the bf16 mode, pinned against the independent double-precision forward with torch's
+    own bf16 conversion at the same six tensors.  On a model this small (2 layers, 12 tokens, width 64) no value
+    sits within the fp32-vs-double noise of a rounding boundary for the seeds used, so two pipelines that round at
+    the same places agree to ~1e-7; dropping one of the six roundings, or adding one where the oracle has none
+    (the residual stream, gate and up separately, the attention probabilities), moves every element of that
+    tensor by up to half a bf16 ulp and shows as a relative logit difference above 1e-3.  (On larger inputs a
+    single boundary case cascades - rounding is discontinuous - and this clean separation is lost, which is why
+    the pin is small.)"""
+    shape = bs_inputs.ModelShape("t", 2, 64, 4, 2, 16, 128, 300, init_std=0.08)
+    six = frozenset(O.ROUNDING_POINTS)
+    rms = lambda a: float(np.sqrt(np.mean(a * a)))
+    for seed in (25, 26, 27):
+        w = bs_inputs.weights_to_numpy_f32(bs_inputs.make_weights(shape, seed))
+        toks = np.random.default_rng(9).integers(0, 299, size=12)
+        z = O.full_forward_logits(O.model_from_weights(shape, w, bf16_activations=True), toks, 1.0).astype(np.float64)
+        dist = lambda rnd: rms(brute_forward(shape, w, toks, 1.0, rnd) - z) / rms(z)
+        assert dist(six) < 1e-5
+        for p in O.ROUNDING_POINTS:
+            assert dist(six - {p}) > 1e-3, f"dropping the rounding at '{p}' goes unnoticed"
+        for extra in ("residual", "gate_up", "probs"):
+            assert dist(six | {extra}) > 1e-3, f"an extra rounding at '{extra}' goes unnoticed"
+    # the subset switch of the oracle selects the same tensors (used by the error-budget script)
+    for p in O.ROUNDING_POINTS:
+        m = O.model_from_weights(shape, w, bf16_activations=True)
+        m.bf16_points = six - {p}
+        zp = O.full_forward_logits(m, toks, 1.0).astype(np.float64)
+        assert rms(brute_forward(shape, w, toks, 1.0, six - {p}) - zp) / rms(zp) < 1e-5
+    # with the mode off nothing is rounded
+    z32 = O.full_forward_logits(O.model_from_weights(shape, w, bf16_activations=False), toks, 1.0).astype(np.float64)
+    assert rms(brute_forward(shape, w, toks, 1.0) - z32) / rms(z32) < 1e-5
 
 
 def test_full_forward_against_independent_double_forward():

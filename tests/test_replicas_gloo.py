@@ -56,3 +56,39 @@ def test_reference_arm_runs_on_rank_zero_only():
     r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--steps", "1",
                         "--warmup", "0"], env=env, capture_output=True, text=True, timeout=120)
     assert r.returncode == 0 and r.stdout.strip() == ""
+
+
+STUB = r"""
+import os, sys, json
+import torch.distributed as dist
+rank, world = int(os.environ["RANK"]), int(os.environ["WORLD_SIZE"])
+dist.init_process_group("gloo", rank=rank, world_size=world)
+dist.barrier()
+if rank == 0:
+    print(json.dumps({"n_gpus": world, "argv": sys.argv[1:], "local_rank": os.environ["LOCAL_RANK"]}), flush=True)
+dist.destroy_process_group()
+"""
+
+
+def test_plain_start_with_gpus_n_launches_n_ranks(tmp_path):
+    """`python bench.py --gpus N` without a launcher must start N ranks itself: here the launcher runs a stub worker
+    (gloo, CPU) and both ranks must meet at the rendezvous it set up; rank 0's line names the world size."""
+    import json
+    sys.path.insert(0, ROOT)
+    import bench
+    stub = tmp_path / "stub.py"
+    stub.write_text(STUB)
+    res = bench.launch_ranks(2, ["--gpus", "2", "--steps", "1"], worker=[sys.executable, str(stub)],
+                             check_devices=False, timeout_s=120)
+    assert [rc for rc, _ in res] == [0, 0]
+    line = json.loads(res[0][1].strip().splitlines()[-1])
+    assert line["n_gpus"] == 2 and line["argv"] == ["--gpus", "2", "--steps", "1"] and line["local_rank"] == "0"
+    assert res[1][1].strip() == ""                       # only rank 0 prints
+
+
+def test_more_ranks_than_devices_is_refused():
+    import torch
+    sys.path.insert(0, ROOT)
+    import bench
+    with pytest.raises(SystemExit):
+        bench.launch_ranks(torch.cuda.device_count() + 1, [])
