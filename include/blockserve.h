@@ -73,6 +73,10 @@ typedef struct {
                                     becomes BS_REQ_FINISHED); < 0: off, every request generates exactly g_i tokens */
   int static_groups;             /* 1: the comparison policy of Section 3.1 (fixed groups: nothing is admitted until
                                     every request of the current group has finished); 0: block-boundary refill */
+  int keep_logits;               /* parity hook: 1 = the LM head also stores the fp32 logits [M_m, vocab] of every step
+                                    (4 * max_batch * L * vocab more workspace bytes) so that bs_debug_read can return
+                                    them; 0 = the logits never reach device memory, only the confidence partials of
+                                    the LM-head epilogue do (a twelfth of their bytes) */
 } bs_config;
 
 /* All weights are bf16, row-major [out_features, in_features], device memory.
@@ -185,7 +189,8 @@ enum {
   BS_DBG_LM_TOK = 9, BS_DBG_LM_ROW = 10, BS_DBG_LM_SLOT = 11,  /* int32[M_m] of the step about to run */
   BS_DBG_PREV_LM_ROW = 12, BS_DBG_PREV_LM_SLOT = 13,           /* int32[M_m] of the step that just ran */
   BS_DBG_PREV_TOK = 14, BS_DBG_PREV_CONF = 15, BS_DBG_PREV_COMMIT = 16, /* int32 / float / int32 [M_m], last step */
-  BS_DBG_PREV_LOGITS = 17, /* float[rows * vocab] of the last step: rows arg0 .. arg0 + arg1 (arg1 = 0: to the end) */
+  BS_DBG_PREV_LOGITS = 17, /* float[rows * vocab] of the last step: rows arg0 .. arg0 + arg1 (arg1 = 0: to the end);
+                              BS_E_STATE unless the engine was created with keep_logits */
   BS_DBG_REQ_ID_OF_ROW = 18, /* int64[n_active] */
   BS_DBG_KV_ROW = 19   /* bf16 K then V of (layer = arg0, physical row = arg1): 2 * Hkv * head_dim values */
 };
@@ -267,6 +272,17 @@ int bs_op_attention(const void* qkv, const void* kcache, const void* vcache, voi
 /* Per row of fp32 logits [n_rows, vocab]: mask id excluded, tok = argmax (lowest id on ties),
  * conf = exp(max - logsumexp). */
 int bs_op_confidence(const float* logits, int n_rows, int vocab, int mask_id, int* tok, float* conf, void* stream);
+
+/* The LM head fused with the confidence pass (the related-work description of confidence-aware parallel decoding:
+ * token = argmax, confidence = its softmax probability): logits z[m, v] = row_scale[m] * (hf[m, :] . W[v, :]) are
+ * formed in the GEMM's accumulators and reduced there, per row, to tok = argmax over v != mask_id (lowest id on ties)
+ * and conf = exp(max - logsumexp); they are written to `logits` (fp32 [M, vocab], nullable) only on request.
+ * hf bf16 [M, K] with row stride lda, W bf16 [vocab, K].  `scratch` holds the partials:
+ * bs_op_lm_head_confidence_scratch_bytes(M, vocab) bytes, 256-byte aligned. */
+size_t bs_op_lm_head_confidence_scratch_bytes(int M, int vocab);
+int bs_op_lm_head_confidence(const void* hf, int lda, const void* W, int M, int vocab, int K, const float* row_scale,
+                             int mask_id, void* scratch, size_t scratch_bytes, int* tok, float* conf,
+                             float* logits /* nullable */, int* error_flag /* nullable */, void* stream);
 
 #ifdef __cplusplus
 }

@@ -37,7 +37,7 @@ class BsConfig(C.Structure):
                 ("token_budget", C.c_longlong), ("max_batch", C.c_int), ("max_requests", C.c_int),
                 ("max_row_tokens", C.c_int), ("kv_capacity_tokens", C.c_longlong), ("suffix_mode", C.c_int),
                 ("sort_queue", C.c_int), ("steps_per_block", C.c_int), ("eos_id", C.c_int),
-                ("static_groups", C.c_int)]
+                ("static_groups", C.c_int), ("keep_logits", C.c_int)]
 
 
 class BsWeights(C.Structure):
@@ -60,7 +60,8 @@ class BsStats(C.Structure):
 EXPORTS = ["bs_query_sizes", "bs_init_model", "bs_admit", "bs_evict_refill", "bs_denoise_step", "bs_block_done",
            "bs_read_tokens", "bs_get_stats", "bs_set_profiling", "bs_get_profile", "bs_destroy", "bs_last_error", "bs_debug_read", "bs_debug_inject_timeout",
            "bs_debug_force_commit", "bs_debug_snapshot", "bs_debug_restore", "bs_op_gemm",
-           "bs_op_rmsnorm", "bs_op_rope_kv", "bs_op_rope_kv_static", "bs_op_attention_q_tile", "bs_op_attention", "bs_op_confidence"]
+           "bs_op_rmsnorm", "bs_op_rope_kv", "bs_op_rope_kv_static", "bs_op_attention_q_tile", "bs_op_attention", "bs_op_confidence",
+           "bs_op_lm_head_confidence", "bs_op_lm_head_confidence_scratch_bytes"]
 
 _lib = None
 
@@ -101,6 +102,9 @@ def lib() -> C.CDLL:
         L.bs_op_attention_q_tile.argtypes = [i, i, i]
         L.bs_op_attention.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i, i, i, i, i, ll, i, i, i, vp, C.c_size_t, vp, vp]
         L.bs_op_confidence.argtypes = [vp, i, i, i, vp, vp, vp]
+        L.bs_op_lm_head_confidence_scratch_bytes.argtypes = [i, i]
+        L.bs_op_lm_head_confidence_scratch_bytes.restype = C.c_size_t
+        L.bs_op_lm_head_confidence.argtypes = [vp, i, vp, i, i, i, vp, i, vp, C.c_size_t, vp, vp, vp, vp, vp]
         _lib = L
     return _lib
 
@@ -127,11 +131,11 @@ def _check_op(rc: int, name: str) -> None:
 def make_config(shape, block_len: int, tau: float, token_budget: int, max_batch: int, max_requests: int,
                 max_row_tokens: int, kv_capacity_tokens: int, suffix_mode: int = SUFFIX_FULL,
                 sort_queue: bool = True, steps_per_block: int = 0, eos_id: int = -1,
-                static_groups: bool = False) -> BsConfig:
+                static_groups: bool = False, keep_logits: bool = False) -> BsConfig:
     return BsConfig(shape.n_layers, shape.d_model, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, shape.d_ffn,
                     shape.vocab, shape.mask_id, shape.rms_eps, shape.rope_theta, block_len, tau, token_budget,
                     max_batch, max_requests, max_row_tokens, kv_capacity_tokens, suffix_mode, int(sort_queue),
-                    int(steps_per_block), int(eos_id), int(static_groups))
+                    int(steps_per_block), int(eos_id), int(static_groups), int(keep_logits))
 
 
 def query_sizes(cfg: BsConfig) -> BsSizes:
@@ -295,7 +299,7 @@ class Engine:
 
 def engine_for_workload(wl, weights, *, kv_capacity_tokens: Optional[int] = None, suffix_mode: int = SUFFIX_FULL,
                         sort_queue: bool = True, steps_per_block: int = 0, eos_id: int = -1,
-                        static_groups: bool = False, device: str = "cuda:0") -> Engine:
+                        static_groups: bool = False, keep_logits: bool = False, device: str = "cuda:0") -> Engine:
     """Size an engine for a bs_inputs.Workload (the caller still admits the requests)."""
     mrt = wl.max_row_tokens
     if kv_capacity_tokens is None:
@@ -304,7 +308,8 @@ def engine_for_workload(wl, weights, *, kv_capacity_tokens: Optional[int] = None
         if wl.token_budget > 0:       # Eq. 1 bounds |A| * width; rows are at most width + g long
             kv_capacity_tokens = min(kv_capacity_tokens, wl.token_budget + wl.max_batch * max(r.g for r in wl.requests))
     cfg = make_config(wl.shape, wl.block_len, wl.tau, wl.token_budget, wl.max_batch, len(wl.requests), mrt,
-                      max(kv_capacity_tokens, mrt), suffix_mode, sort_queue, steps_per_block, eos_id, static_groups)
+                      max(kv_capacity_tokens, mrt), suffix_mode, sort_queue, steps_per_block, eos_id, static_groups,
+                      keep_logits)
     return Engine(cfg, weights, device)
 
 
@@ -375,6 +380,26 @@ def op_attention(qkv, kcache, vcache, cu_q, kv_base, vis, hq, hkv, dh, scratch: 
                                     0 if scratch is None else scratch.numel() * scratch.element_size(),
                                     None, _stream()), "bs_op_attention")
     return out
+
+
+def op_lm_head_confidence(hf: torch.Tensor, W: torch.Tensor, row_scale: torch.Tensor, mask_id: int,
+                          want_logits: bool = False):
+    """LM head with the confidence pass in its epilogue: (tok int32 [M], conf fp32 [M], logits fp32 [M, V] or None)."""
+    M, K = hf.shape
+    V = W.shape[0]
+    nbytes = lib().bs_op_lm_head_confidence_scratch_bytes(M, V)
+    scratch = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=hf.device)
+    tok = torch.empty(M, dtype=torch.int32, device=hf.device)
+    conf = torch.empty(M, dtype=torch.float32, device=hf.device)
+    logits = torch.empty(M, V, dtype=torch.float32, device=hf.device) if want_logits else None
+    flag = torch.zeros(1, dtype=torch.int32, device=hf.device)
+    _check_op(lib().bs_op_lm_head_confidence(hf.data_ptr(), hf.stride(0), W.data_ptr(), M, V, K, row_scale.data_ptr(),
+                                             mask_id, scratch.data_ptr(), nbytes, tok.data_ptr(), conf.data_ptr(),
+                                             _ptr(logits), flag.data_ptr(), _stream()), "bs_op_lm_head_confidence")
+    torch.cuda.current_stream().synchronize()
+    if int(flag.item()):
+        raise BlockServeError(BS_E_TIMEOUT, "a bounded device-side wait ran out")
+    return tok, conf, logits
 
 
 def op_confidence(logits: torch.Tensor, mask_id: int):

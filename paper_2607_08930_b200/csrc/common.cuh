@@ -63,6 +63,8 @@ struct DevState {
   int* lm_tok[2]; int* lm_row[2]; int* lm_slot[2];
   int* out_tok[2]; float* out_conf[2]; int* out_commit[2];
   float* lm_scale[2];   // alpha of the row each lm entry belongs to
+  const float2* slice_ms;   // [kConfSlices][M_m]: slice partials of the fused LM-head confidence pass
+  const int* slice_am;
   int* tok_row; int* tok_pos; int* tok_kv;
 };
 
@@ -93,12 +95,31 @@ struct GemmScratch {
   int* error_flag = nullptr;
 };
 
+// Output of the LM head fused with the confidence pass (GEMM mode 5): per (group of 32 output features, token) the
+// maximum of the row-scaled outputs, the sum of exp(z - max) and the feature index of the maximum.
+struct GemmConf {
+  float2* ms;      // [ceil(N / 32)][M]
+  int* am;         // [ceil(N / 32)][M]
+  int skip;        // output feature that never takes part (the mask id), or -1
+};
+constexpr int kConfSlices = 16;      // the group partials of a token are merged in this many slices, then once more
+
 // C[M,N] = A[M,K] W[N,K]^T.  mode: 0 bf16 store, 1 fp32 +=, 2 fp32 row-scaled store, 3 SwiGLU (W and W2).
 cudaError_t launch_gemm(const bf16* A, int lda, const bf16* W, const bf16* W2, void* C, int ldc, int M, int N, int K,
                         int mode, const float* row_scale, const GemmScratch& scratch, cudaStream_t s);
 cudaError_t launch_gemm_tc(const bf16* A, int lda, const bf16* W, const bf16* W2, void* C, int ldc, int M, int N,
                            int K, int mode, const float* row_scale, const GemmScratch& scratch, cudaStream_t s,
-                           int* splits_out);
+                           int* splits_out, const GemmConf* conf = nullptr);
+// LM head fused with the confidence pass: group partials by the GEMM epilogue (logits, if not null, receives the scaled
+// fp32 outputs as well), then the partials of each token merged into kConfSlices slice partials
+// slice_ms / slice_am [kConfSlices][M] (merge_conf_slices() in conf_merge.cuh finishes the job).
+cudaError_t launch_lm_head_conf(const bf16* hf, int lda, const bf16* W, int M, int V, int K, const float* row_scale,
+                                int mask_id, const GemmConf& groups, float2* slice_ms, int* slice_am, float* logits,
+                                const GemmScratch& scratch, cudaStream_t s);
+cudaError_t launch_conf_merge(const GemmConf& groups, int M, int V, float2* slice_ms, int* slice_am, cudaStream_t s);
+// tok / conf [M] from the slice partials (stand-alone use; the engine's commit kernel does this inline).
+cudaError_t launch_conf_final(const float2* slice_ms, const int* slice_am, int M, int* tok, float* conf,
+                              cudaStream_t s);
 // Why the last launch_gemm* of this thread returned cudaErrorNotSupported (a shape or alignment the tensor-core
 // kernels do not take; there is no other GEMM behind them).
 const char* gemm_decline_reason();

@@ -2,7 +2,7 @@
 // and the per-row vocabulary pass of the confidence epilogue.
 #include <math.h>
 
-#include "common.cuh"
+#include "conf_merge.cuh"
 
 namespace bs {
 
@@ -186,6 +186,61 @@ __global__ void __launch_bounds__(kConfThreads) k_confidence(const float* __rest
   }
 }
 
+// Second stage of the fused LM-head confidence pass: the GEMM epilogue left one partial per (group of 32 vocabulary
+// entries, token).  CTA (x, y): 32 consecutive tokens (lane = token, so every load is one coalesced 256-byte row of
+// the [group][token] arrays) and slice y of the groups, its eight warps striding over the slice; one slice partial
+// per token comes out.  The commit kernel merges the kConfSlices slices.
+constexpr int kMergeWarps = 8;
+__global__ void __launch_bounds__(kMergeWarps * 32) k_conf_merge(const float2* __restrict__ group_ms,
+                                                                 const int* __restrict__ group_am, int M, int n_groups,
+                                                                 float2* __restrict__ slice_ms,
+                                                                 int* __restrict__ slice_am) {
+  __shared__ float s_m[kMergeWarps][32], s_s[kMergeWarps][32];
+  __shared__ int s_i[kMergeWarps][32];
+  pdl_wait();
+  pdl_trigger();
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const int t = blockIdx.x * 32 + lane;
+  const int per = (n_groups + kConfSlices - 1) / kConfSlices;
+  const int g0 = blockIdx.y * per, g1 = min(n_groups, g0 + per);
+  ConfPart acc = conf_empty();
+  if (t < M) {
+    int g = g0 + w;
+    for (; g + 3 * kMergeWarps < g1; g += 4 * kMergeWarps) {       // four loads in flight per thread
+      float2 ms[4];
+      int am[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const size_t at = (size_t)(g + u * kMergeWarps) * M + t;
+        ms[u] = __ldcs(group_ms + at);
+        am[u] = __ldcs(group_am + at);
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) conf_merge(acc, ms[u].x, ms[u].y, am[u]);
+    }
+    for (; g < g1; g += kMergeWarps) {
+      const size_t at = (size_t)g * M + t;
+      const float2 ms = __ldcs(group_ms + at);
+      conf_merge(acc, ms.x, ms.y, __ldcs(group_am + at));
+    }
+  }
+  s_m[w][lane] = acc.m; s_s[w][lane] = acc.s; s_i[w][lane] = acc.am;
+  __syncthreads();
+  if (w == 0 && t < M) {
+    for (int k = 1; k < kMergeWarps; ++k) conf_merge(acc, s_m[k][lane], s_s[k][lane], s_i[k][lane]);
+    slice_ms[(size_t)blockIdx.y * M + t] = make_float2(acc.m, acc.s);
+    slice_am[(size_t)blockIdx.y * M + t] = acc.am;
+  }
+}
+
+__global__ void k_conf_final(const float2* __restrict__ slice_ms, const int* __restrict__ slice_am, int M,
+                             int* __restrict__ tok, float* __restrict__ conf) {
+  pdl_wait();
+  pdl_trigger();
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t < M) merge_conf_slices(slice_ms, slice_am, M, t, tok + t, conf + t);
+}
+
 constexpr int kMaxSplits = 8;
 
 // Finishing kernel of the QKV projection on block steps: adds the k-split partial sums in split order, rounds q / k / v
@@ -362,6 +417,27 @@ cudaError_t launch_confidence(const float* logits, int n_rows, int vocab, int ma
                               cudaStream_t s) {
   if (n_rows <= 0) return cudaSuccess;
   return launch_pdl(k_confidence, dim3(n_rows), dim3(kConfThreads), 0, s, logits, vocab, mask_id, tok, conf);
+}
+
+cudaError_t launch_lm_head_conf(const bf16* hf, int lda, const bf16* W, int M, int V, int K, const float* row_scale,
+                                int mask_id, const GemmConf& groups, float2* slice_ms, int* slice_am, float* logits,
+                                const GemmScratch& scratch, cudaStream_t s) {
+  if (M <= 0) return cudaSuccess;
+  GemmConf gc = groups;
+  gc.skip = mask_id;
+  cudaError_t r = launch_gemm_tc(hf, lda, W, nullptr, logits, V, M, V, K, 5, row_scale, scratch, s, nullptr, &gc);
+  if (r != cudaSuccess) return r;
+  return launch_conf_merge(gc, M, V, slice_ms, slice_am, s);
+}
+cudaError_t launch_conf_merge(const GemmConf& groups, int M, int V, float2* slice_ms, int* slice_am, cudaStream_t s) {
+  if (M <= 0) return cudaSuccess;
+  return launch_pdl(k_conf_merge, dim3((M + 31) / 32, kConfSlices), dim3(kMergeWarps * 32), 0, s,
+                    (const float2*)groups.ms, (const int*)groups.am, M, (V + 31) / 32, slice_ms, slice_am);
+}
+cudaError_t launch_conf_final(const float2* slice_ms, const int* slice_am, int M, int* tok, float* conf,
+                              cudaStream_t s) {
+  if (M <= 0) return cudaSuccess;
+  return launch_pdl(k_conf_final, dim3((M + 127) / 128), dim3(128), 0, s, slice_ms, slice_am, M, tok, conf);
 }
 
 void build_rope_table(float* out, int max_pos, int dh, float theta) {

@@ -40,7 +40,11 @@ struct Workspace {
   bf16* attn;       // [T, Hq dh]
   bf16* act;        // [min(T, chunk), ffn]
   bf16* hf;         // [max_batch L, d]
-  float* logits;    // [max_batch L, V]
+  float* logits;    // [max_batch L, V], only with bs_config.keep_logits
+  float2* group_ms; // [ceil(V / 32)][max_batch L]: confidence partials of the LM-head epilogue
+  int* group_am;
+  float2* slice_ms; // [kConfSlices][max_batch L]
+  int* slice_am;
   float* partial;   // k-split partial sums of the projection GEMMs
 };
 
@@ -58,7 +62,12 @@ size_t carve_workspace(const bs_config& c, void* base, Workspace* w) {
   t.attn = cv.take<bf16>(T * (size_t)c.n_q_heads * c.head_dim);
   t.act = cv.take<bf16>(std::min<size_t>(T, kMlpChunk) * c.d_ffn);
   t.hf = cv.take<bf16>(mm * c.d_model);
-  t.logits = cv.take<float>(mm * c.vocab);
+  t.logits = c.keep_logits ? cv.take<float>(mm * c.vocab) : nullptr;
+  const size_t n_groups = ((size_t)c.vocab + 31) / 32;
+  t.group_ms = cv.take<float2>(n_groups * mm);
+  t.group_am = cv.take<int>(n_groups * mm);
+  t.slice_ms = cv.take<float2>((size_t)kConfSlices * mm);
+  t.slice_am = cv.take<int>((size_t)kConfSlices * mm);
   t.partial = cv.take<float>(kPartialFloats);
   if (w) *w = t;
   return cv.off;
@@ -107,6 +116,7 @@ const char* check_config(const bs_config& c) {
   if (!(c.tau >= 0.f)) return "tau must be >= 0";
   if (c.steps_per_block < 0 || c.steps_per_block > c.block_len) return "steps_per_block must be in [0, block_len]";
   if (c.eos_id >= c.vocab || c.eos_id == c.mask_id) return "eos_id must be a token id other than the mask id, or negative";
+  if (c.keep_logits != 0 && c.keep_logits != 1) return "keep_logits must be 0 or 1";
   return nullptr;
 }
 
@@ -284,6 +294,8 @@ int bs_init_model(const bs_config* cfg, const bs_weights* w, void* kv, void* wor
   st.eos_id = cfg->eos_id;
   st.static_groups = cfg->static_groups ? 1 : 0;
   st.q_tile = attention_q_tile(cfg->n_q_heads, cfg->n_kv_heads, cfg->head_dim);
+  st.slice_ms = e->ws.slice_ms;
+  st.slice_am = e->ws.slice_am;
   e->gemm_scratch.partial = e->ws.partial;
   e->gemm_scratch.partial_floats = kPartialFloats;
   e->gemm_scratch.error_flag = st.hdr + H_ERROR;
@@ -501,12 +513,18 @@ int bs_denoise_step(bs_engine* e, int* n_committed) {
   prof_mark(e, BS_FAM_EMBED_NORM);
   KL(e, launch_rmsnorm(ws.x, st.lm_tok[parity], e->final_norm, ws.hf, Mm, d, c.rms_eps, s));
   prof_work(e, BS_FAM_EMBED_NORM, 1, 0, 6.0 * dMm * dd);
+  // LM head with the confidence pass in its epilogue: per (32 vocabulary entries, row) maximum / sum of exponentials
+  // / argmax of the alpha-scaled logits, merged per row in two small stages (the second one inside the commit
+  // kernel); the fp32 logits reach HBM only when the engine was configured to keep them for the parity hooks.
   prof_mark(e, BS_FAM_GEMM_LM_HEAD);
-  KL(e, launch_gemm(ws.hf, d, e->lm_head, nullptr, ws.logits, c.vocab, Mm, c.vocab, d, 2, st.lm_scale[parity], e->gemm_scratch, s));
-  prof_work(e, BS_FAM_GEMM_LM_HEAD, 1, 2.0 * dMm * dV * dd, 2.0 * (dV * dd + dMm * dd) + 4.0 * dMm * dV);
+  GemmConf groups{ws.group_ms, ws.group_am, c.mask_id};
+  KL(e, launch_gemm_tc(ws.hf, d, e->lm_head, nullptr, ws.logits, c.vocab, Mm, c.vocab, d, 5, st.lm_scale[parity],
+                       e->gemm_scratch, s, nullptr, &groups));
+  prof_work(e, BS_FAM_GEMM_LM_HEAD, 1, 2.0 * dMm * dV * dd,
+            2.0 * (dV * dd + dMm * dd) + 12.0 * dMm * (dV / 32.0) + (ws.logits ? 4.0 * dMm * dV : 0.0));
   prof_mark(e, BS_FAM_CONFIDENCE);
-  KL(e, launch_confidence(ws.logits, Mm, c.vocab, c.mask_id, st.out_tok[parity], st.out_conf[parity], s));
-  prof_work(e, BS_FAM_CONFIDENCE, 1, 0, 4.0 * dMm * dV);
+  KL(e, launch_conf_merge(groups, Mm, c.vocab, ws.slice_ms, ws.slice_am, s));
+  prof_work(e, BS_FAM_CONFIDENCE, 1, 0, 12.0 * dMm * (dV / 32.0));
   prof_mark(e, BS_FAM_INDEX);
   KL(e, launch_commit_index(st, s));
   prof_work(e, BS_FAM_INDEX, 1, 0, 0);
@@ -629,6 +647,7 @@ int bs_debug_read(bs_engine* e, int what, int arg0, int arg1, void* host_buf, si
     case BS_DBG_PREV_CONF: src = st.out_conf[prev]; bytes = (size_t)prev_mm * 4; break;
     case BS_DBG_PREV_COMMIT: src = st.out_commit[prev]; bytes = (size_t)prev_mm * 4; break;
     case BS_DBG_PREV_LOGITS: {   // arg0 = first masked row, arg1 = number of rows (0: all rows from arg0)
+      if (!e->ws.logits) return fail(e, BS_E_STATE, "the engine was created without keep_logits");
       if (arg0 < 0 || arg0 > prev_mm || arg1 < 0 || arg0 + arg1 > prev_mm) return fail(e, BS_E_ARG, "bad logit rows");
       const int rows = arg1 > 0 ? arg1 : prev_mm - arg0;
       src = e->ws.logits + (size_t)arg0 * e->cfg.vocab;
@@ -858,6 +877,35 @@ int bs_op_attention(const void* qkv, const void* kcache, const void* vcache, voi
                           scratch, scratch ? scratch_bytes / sizeof(float) : 0, error_flag,
                           (cudaStream_t)stream) == cudaSuccess
              ? BS_OK : BS_E_CUDA;
+}
+
+size_t bs_op_lm_head_confidence_scratch_bytes(int M, int vocab) {
+  if (M < 0 || vocab < 1) return 0;
+  const size_t parts = ((size_t)vocab + 31) / 32 + kConfSlices;
+  return align_up(parts * (size_t)M * sizeof(float2)) + align_up(parts * (size_t)M * sizeof(int));
+}
+
+int bs_op_lm_head_confidence(const void* hf, int lda, const void* W, int M, int vocab, int K, const float* row_scale,
+                             int mask_id, void* scratch, size_t scratch_bytes, int* tok, float* conf, float* logits,
+                             int* error_flag, void* stream) {
+  if (M == 0) return BS_OK;
+  if (!hf || !W || !row_scale || !scratch || !tok || !conf || M < 0 || vocab < 2 || K < 8 || K % 8 || lda % 8)
+    return BS_E_ARG;
+  if ((((uintptr_t)hf | (uintptr_t)W) & 15) || ((uintptr_t)scratch & 255)) return BS_E_ARG;
+  if (scratch_bytes < bs_op_lm_head_confidence_scratch_bytes(M, vocab)) return BS_E_ARG;
+  const size_t n_groups = ((size_t)vocab + 31) / 32, parts = n_groups + kConfSlices;
+  float2* ms = static_cast<float2*>(scratch);
+  int* am = reinterpret_cast<int*>(static_cast<char*>(scratch) + align_up(parts * (size_t)M * sizeof(float2)));
+  GemmConf groups{ms, am, mask_id};
+  float2* slice_ms = ms + n_groups * (size_t)M;
+  int* slice_am = am + n_groups * (size_t)M;
+  GemmScratch sc;
+  sc.error_flag = error_flag;
+  cudaStream_t s = (cudaStream_t)stream;
+  cudaError_t r = launch_lm_head_conf((const bf16*)hf, lda, (const bf16*)W, M, vocab, K, row_scale, mask_id, groups,
+                                      slice_ms, slice_am, logits, sc, s);
+  if (r == cudaSuccess) r = launch_conf_final(slice_ms, slice_am, M, tok, conf, s);
+  return r == cudaSuccess ? BS_OK : (r == cudaErrorNotSupported ? BS_E_ARG : BS_E_CUDA);
 }
 
 int bs_op_confidence(const float* logits, int n_rows, int vocab, int mask_id, int* tok, float* conf, void* stream) {

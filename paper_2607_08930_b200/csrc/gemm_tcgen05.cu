@@ -37,7 +37,8 @@ struct GemmParams {
   int n_tiles, m_tiles, splits, kblocks;
   int stages;
   int ksub;          // 64-wide k sub-blocks per pipeline stage
-  int mode;          // 0 bf16 store, 1 fp32 +=, 2 fp32 row-scaled store, 3 SwiGLU, 4 fp32 partial sums only
+  int mode;          // 0 bf16 store, 1 fp32 +=, 2 fp32 row-scaled store, 3 SwiGLU, 4 fp32 partial sums only,
+                     // 5 row-scaled confidence partials (max, sum exp, argmax per token and 32 output features)
   int dual;
   int wide;          // two 128-row tiles of the same weight matrix share every token tile (256 weight rows per item)
   int rows;          // weight rows per work item: 128 or 256
@@ -48,6 +49,11 @@ struct GemmParams {
   const float* row_scale;
   float* partial;    // [splits][M][N] fp32 when splits > 1
   int* error_flag;
+  // mode 5: per (group of 32 output features, token) the running maximum and sum of exponentials of the row-scaled
+  // outputs and the feature index of the maximum; feature `skip` never takes part (the mask id)
+  float2* conf_ms;   // [ceil(N / 32)][M]
+  int* conf_am;      // [ceil(N / 32)][M]
+  int skip;
 };
 
 __device__ __forceinline__ void tma_load_2d(unsigned dst, const CUtensorMap* map, int c0, int c1, unsigned bar) {
@@ -140,6 +146,58 @@ __device__ __forceinline__ void epilogue_row(const GemmParams& p, int split, int
     const float* scale = EPI == 2 ? p.row_scale + t0 : nullptr;
     if (jmax == 32) epilogue_chunk<EPI, true>(v, u, ptr, stride, jmax, scale);
     else epilogue_chunk<EPI, false>(v, u, ptr, stride, jmax, scale);
+  }
+}
+
+// Epilogue of the LM head fused with the confidence pass (mode 5).  A warp holds 32 output features (vocabulary
+// entries n0 .. n0 + 31, one per lane = TMEM lane) for the tn tokens of the tile.  Per chunk of 32 tokens the
+// 32 x 32 block goes through a padded shared-memory tile, after which lane j owns token j with its 32 features:
+// it scales them by the token's row scale, and keeps their maximum, the sum of exp(z - max) and the lowest feature
+// index of the maximum - one partial per (feature group, token), a twelfth of the bytes of the logits.  When p.C
+// is set the scaled fp32 logits are stored as well (parity hooks read them; the timed path passes nullptr).
+__device__ __forceinline__ void epilogue_conf(const GemmParams& p, int mt, int n0, int lane, unsigned t_row,
+                                              float* tile /* [32][33] of this warp */) {
+  const int group = n0 >> 5;
+  const int n_valid = min(32, p.N - n0);                 // features of this group that exist (warp-uniform)
+  const int i_skip = p.skip - n0;                         // index of the excluded feature inside the group, if any
+  for (int c0 = 0; c0 < p.tn; c0 += 32) {
+    const int t0 = mt * p.tn + c0;
+    if (t0 >= p.M) break;                                 // warp-uniform
+    const int jmax = min(min(32, p.tn - c0), p.M - t0);
+    float v[32];
+    tmem_ld32(t_row + c0, v);
+    __syncwarp();                                         // the previous chunk's reads of the tile are done
+#pragma unroll
+    for (int j = 0; j < 32; ++j) tile[lane * 33 + j] = v[j];
+    __syncwarp();
+    if (lane < jmax && n_valid > 0) {
+      const int t = t0 + lane;
+      const float a = __ldg(p.row_scale + t);
+      float z[32];
+      float m = -INFINITY;
+      int am = 0;
+#pragma unroll
+      for (int i = 0; i < 32; ++i) {
+        z[i] = tile[i * 33 + lane] * a;
+        const bool use = i < n_valid && i != i_skip;
+        if (use && z[i] > m) { m = z[i]; am = i; }       // ascending index, strict: the lowest index wins ties
+      }
+      float sum = 0.f;
+      if (m > -INFINITY) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i)
+          if (i < n_valid && i != i_skip) sum += __expf(z[i] - m);
+      }
+      const size_t at = (size_t)group * p.M + t;
+      p.conf_ms[at] = make_float2(m, sum);
+      p.conf_am[at] = n0 + am;
+      if (p.C) {
+        float* dst = reinterpret_cast<float*>(p.C) + (size_t)t * p.ldc + n0;
+#pragma unroll
+        for (int i = 0; i < 32; ++i)
+          if (i < n_valid) dst[i] = z[i];
+      }
+    }
   }
 }
 
@@ -301,7 +359,12 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
         const int n = nt * p.rows + a * TILE_N + q * 32 + lane;
         const bool n_ok = n < p.N;
         const unsigned t_row = tmem_base + ((unsigned)(q * 32) << 16) + acc * acc_cols + a * p.acc1_off;
-        epilogue_row<EPI>(p, split, mt, n, n_ok, t_row);
+        if constexpr (EPI == 5) {
+          __shared__ float conf_tile[4][32 * 33];
+          epilogue_conf(p, mt, n - lane, lane, t_row, conf_tile[q]);
+        } else {
+          epilogue_row<EPI>(p, split, mt, n, n_ok, t_row);
+        }
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
@@ -518,7 +581,12 @@ k_gemm_pair(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
       for (int a = 0; a < (p.wide ? 2 : 1); ++a) {       // a wide item holds two 256-row accumulators
         const int n = nt * p.rows + a * 256 + (int)rank * TILE_N + q * 32 + lane;
         const unsigned t_row = tmem_base + ((unsigned)(q * 32) << 16) + acc * acc_cols + a * p.acc1_off;
-        epilogue_row<EPI>(p, split, mt, n, n < p.N, t_row);
+        if constexpr (EPI == 5) {
+          __shared__ float conf_tile[4][32 * 33];
+          epilogue_conf(p, mt, n - lane, lane, t_row, conf_tile[q]);
+        } else {
+          epilogue_row<EPI>(p, split, mt, n, n < p.N, t_row);
+        }
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
@@ -636,6 +704,7 @@ GemmKernel kernel_tc(int epi) {
     case 1: return k_gemm_tc<1>;
     case 2: return k_gemm_tc<2>;
     case 3: return k_gemm_tc<3>;
+    case 5: return k_gemm_tc<5>;
     default: return k_gemm_tc<4>;
   }
 }
@@ -645,11 +714,12 @@ GemmKernel kernel_pair(int epi) {
     case 1: return k_gemm_pair<1>;
     case 2: return k_gemm_pair<2>;
     case 3: return k_gemm_pair<3>;
+    case 5: return k_gemm_pair<5>;
     default: return k_gemm_pair<4>;
   }
 }
 bool allow_big_smem(GemmKernel (*table)(int)) {
-  for (int e = 0; e < 5; ++e)
+  for (int e = 0; e < 6; ++e)
     if (cudaFuncSetAttribute(table(e), cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 1024) != cudaSuccess)
       return false;
   return true;
@@ -726,12 +796,13 @@ cudaError_t launch_finish(const GemmParams& p, int mode, int num_sms, cudaStream
 // Plans and launches the CTA-pair kernel.
 cudaError_t launch_gemm_pair(const DevInfo& dv, const bf16* A, int lda, const bf16* W, const bf16* W2, void* C, int ldc,
                              int M, int N, int K, int mode, const float* row_scale, const GemmScratch& scratch,
-                             cudaStream_t s, int* splits_out) {
+                             cudaStream_t s, int* splits_out, const GemmConf* conf) {
   const int max_pairs = dv.max_pairs;
   const int dual = mode == 3;
   GemmParams p;
   p.M = M; p.N = N; p.K = K; p.mode = mode; p.dual = dual; p.C = C; p.ldc = ldc; p.row_scale = row_scale;
   p.error_flag = scratch.error_flag;
+  p.conf_ms = conf ? conf->ms : nullptr; p.conf_am = conf ? conf->am : nullptr; p.skip = conf ? conf->skip : -1;
   // Two 256-row weight tiles per pair and work item (BS_GEMM_PAIR_WIDE=1) halve the token-tile traffic once more at
   // the price of single-buffered accumulators.  Measured on B200 it gains nothing over 256-row items for the
   // K = 3584 projections and 5-8 % for the down projection at 384-640 tokens only, so it is off by default.
@@ -766,7 +837,7 @@ cudaError_t launch_gemm_pair(const DevInfo& dv, const bf16* A, int lda, const bf
   if (p.stages > 16) p.stages = 16;
   p.splits = 1;
   const long long base_items = (long long)p.n_tiles * p.m_tiles;
-  if (scratch.partial && !dual && base_items * 4 < (long long)max_pairs * 3) {
+  if (scratch.partial && !dual && mode != 5 && base_items * 4 < (long long)max_pairs * 3) {
     int sp = (int)(max_pairs / base_items);
     if (sp > tuning().pair_splits) sp = tuning().pair_splits;
     if (sp > 8) sp = 8;
@@ -816,7 +887,8 @@ const char* gemm_decline_reason() { return g_decline.c_str(); }
 // (cudaErrorNotSupported, reason in gemm_decline_reason()): there is no second GEMM implementation behind this one.
 cudaError_t launch_gemm_tc(const bf16* A, int lda, const bf16* W, const bf16* W2, void* C, int ldc, int M, int N,
                            int K, int mode, const float* row_scale, const GemmScratch& scratch, cudaStream_t s,
-                           int* splits_out) {
+                           int* splits_out, const GemmConf* conf) {
+  if (mode == 5 && (!conf || !conf->ms || !conf->am || !row_scale)) return decline("confidence partial buffers missing");
   float* const g_partial = scratch.partial;
   const size_t g_partial_floats = scratch.partial_floats;
   if (M <= 0 || N <= 0) return cudaSuccess;
@@ -834,24 +906,26 @@ cudaError_t launch_gemm_tc(const bf16* A, int lda, const bf16* W, const bf16* W2
   if (dv.max_pairs > 0) {
     if (tuning().pair >= 0) use_pair = tuning().pair > 0 && M >= tuning().pair;
     else if (M >= 128) {
-      const bool dual_ = mode == 3;
+      const bool dual_ = mode == 3 || mode == 5;      // no k split for these
       const int kb = (K + BK - 1) / BK;
       const long long items_p = (long long)((N + 255) / 256) * ((M + 255) / 256);
       const double busy_p =
           grid_busy(items_p * split_for(items_p, dv.max_pairs, kb, (size_t)M * N, scratch, dual_), dv.max_pairs);
-      const bool wide_s = !dual_ && N >= 512 && K >= 8192;
-      const int tn_cap_s = (dual_ && (M <= 128 || M > 256)) ? 128 : 256;
+      const bool wide_s = mode != 3 && N >= 512 && K >= 8192;
+      const int tn_cap_s = (mode == 3 && (M <= 128 || M > 256)) ? 128 : 256;
       const long long items_s = (long long)((N + (wide_s ? 255 : 127)) / (wide_s ? 256 : 128)) * ((M + tn_cap_s - 1) / tn_cap_s);
       const double busy_s = grid_busy(items_s * split_for(items_s, num_sms, kb, (size_t)M * N, scratch, dual_), num_sms);
       use_pair = busy_p * 1.1 >= busy_s;
     }
   }
-  if (use_pair) return launch_gemm_pair(dv, A, lda, W, W2, C, ldc, M, N, K, mode, row_scale, scratch, s, splits_out);
+  if (use_pair)
+    return launch_gemm_pair(dv, A, lda, W, W2, C, ldc, M, N, K, mode, row_scale, scratch, s, splits_out, conf);
   const int dual = mode == 3;
   GemmParams p;
   p.M = M; p.N = N; p.K = K; p.mode = mode; p.dual = dual; p.C = C; p.ldc = ldc; p.row_scale = row_scale;
   p.n_tiles = (N + TILE_N - 1) / TILE_N;
   p.error_flag = scratch.error_flag;
+  p.conf_ms = conf ? conf->ms : nullptr; p.conf_am = conf ? conf->am : nullptr; p.skip = conf ? conf->skip : -1;
   // ---- token tile and k split ----
   // Few tokens (a block step): one or two token tiles that cover M exactly (UMMA N is any multiple of 16), and a
   // k split that spreads the weight stream over all SMs when there are fewer weight tiles than SMs.
@@ -878,7 +952,7 @@ cudaError_t launch_gemm_tc(const bf16* A, int lda, const bf16* W, const bf16* W2
   p.kblocks = (K + BK * p.ksub - 1) / (BK * p.ksub);
   p.splits = 1;
   const long long base_items = (long long)p.n_tiles * p.m_tiles;
-  if (g_partial && base_items * 4 < (long long)num_sms * 3) {
+  if (g_partial && mode != 5 && base_items * 4 < (long long)num_sms * 3) {
     int sp = (int)(num_sms / base_items);
     if (sp > 8) sp = 8;
     while (sp > 1 && (p.kblocks / sp < 4 || (size_t)sp * (size_t)M * N > g_partial_floats)) --sp;
@@ -888,7 +962,7 @@ cudaError_t launch_gemm_tc(const bf16* A, int lda, const bf16* W, const bf16* W2
     if (sp >= 1 && sp <= 8 && (sp == 1 || (g_partial && (size_t)sp * (size_t)M * N <= g_partial_floats))) p.splits = sp;
   if (mode == 4 && (!g_partial || (size_t)p.splits * (size_t)M * N > g_partial_floats))
     return decline("partial-sum scratch too small for this projection");
-  if (dual) p.splits = 1;
+  if (dual || mode == 5) p.splits = 1;
   p.partial = g_partial;
   if (splits_out) *splits_out = p.splits;
   const int stage_bytes = p.ksub * ((two_a ? 2 : 1) * TILE_N * BK * 2 + p.tn * BK * 2);

@@ -2,7 +2,7 @@
 //   k_sched        - Algorithm 1's block boundary: advance, evict, stable compaction, refill under Eq. 1
 //   k_commit_index - confidence-thresholded commit per request + block-done flags + next step's indices
 //   k_fill_tokens  - per packed token: row, logical position id, physical KV row (Section 2.5)
-#include "common.cuh"
+#include "conf_merge.cuh"
 
 namespace bs {
 
@@ -262,8 +262,10 @@ __global__ void __launch_bounds__(kSchedThreads) k_commit_index(DevState st) {
     float conf = -1.0f;
     int tok = 0, bit = 0;
     if (lane < nm) {
-      conf = st.out_conf[parity][base + lane];
-      tok = st.out_tok[parity][base + lane];
+      // last stage of the confidence pass: the slice partials of this masked position -> token id and confidence
+      merge_conf_slices(st.slice_ms, st.slice_am, st.lm_base[parity][n], base + lane, &tok, &conf);
+      st.out_conf[parity][base + lane] = conf;
+      st.out_tok[parity][base + lane] = tok;
       bit = st.lm_slot[parity][base + lane];
     }
     // transfer quota of this step (Section 2.5): the block's L masked tokens spread uniformly over S steps

@@ -137,7 +137,7 @@ class Lockstep:
         self.eos_id = eos_id
         self.eng = B.engine_for_workload(wl, weights_cuda, kv_capacity_tokens=kv_capacity, suffix_mode=suffix_mode,
                                          sort_queue=sort_queue, steps_per_block=steps_per_block, eos_id=eos_id,
-                                         static_groups=static_groups, **(engine_kwargs or {}))
+                                         static_groups=static_groups, keep_logits=True, **(engine_kwargs or {}))
         self.model = model if model is not None else O.model_from_weights(wl.shape, weights_np)
         assert self.model.bf16_activations
         self.model32 = dataclasses.replace(self.model, bf16_activations=False) if "fp32" in modes else None
@@ -147,7 +147,8 @@ class Lockstep:
         self.shadow = {}                 # req_id -> the fp32-mode oracle's copy of a tracked request
         self.suffix_mode = suffix_mode
         self.excluded = {c: 0 for c in CLASSES}
-        self.first_exception = {}        # req_id -> block index of its first counted exception
+        self.first_exception = {}        # req_id -> (block, step) of its first counted exception
+        self.commit_log = {}             # req_id -> [(block, step, committed positions, their tokens)] as the engine decided
         self.stats = {"bf16": ModeStats(), "fp32": ModeStats()}
         self.rows_checked = 0
         self.steps = 0
@@ -173,6 +174,22 @@ class Lockstep:
             if self.model32 is not None and self.tracked(r.req_id):
                 self.shadow[r.req_id] = O.new_request(self.model32, r.req_id, r.prompt, r.g, r.alpha,
                                                       self.wl.block_len, r.start_block, r.gen_prefix)
+
+    def attach(self, req_ids):
+        """Starts tracking the given requests at a block boundary (between cycles).  The state there is the token
+        rows plus the scheduler's integers (every block begins with a refresh step that rebuilds the cache), so the
+        oracle takes over the engine's token rows for them - what a snapshot at this boundary holds - and follows
+        their floating-point path from the next step on.  Pass an empty list to go back to integer-only checks."""
+        self.track = set(req_ids)
+        self.shadow = {}
+        for rid in self.track:
+            r = self.ora.by_id[rid]
+            toks, _ = self.eng.read_tokens(rid)
+            r.tokens[:] = toks
+            r.K = r.V = None
+            if self.model32 is not None:
+                sh = dataclasses.replace(r, tokens=r.tokens.copy())
+                self.shadow[rid] = sh
 
     def evict_refill(self):
         ev_o, ad_o, n_o = self.ora.evict_refill()
@@ -204,7 +221,7 @@ class Lockstep:
 
     def _count(self, cls, r):
         self.excluded[cls] += 1
-        self.first_exception.setdefault(r.req_id, r.b)
+        self.first_exception.setdefault(r.req_id, (r.b, r.s - 1))     # r.s has already moved past the step
 
     def _mode_stats(self, mode, zl, gc, gt, gs, probe, where):
         """Logit / confidence errors of the engine's rows against one oracle record; returns D per row."""
@@ -294,6 +311,8 @@ class Lockstep:
             probe = O.denoise_step(self.model, r, self.wl.block_len, self.wl.tau, self.suffix_mode,
                                    keep_logits=True, override_commit=gs, override_tok=gt,
                                    steps_per_block=self.S)
+            self.commit_log.setdefault(r.req_id, []).append((probe.block, probe.step, probe.positions[gs].copy(),
+                                                             gt[gs].copy()))
             # (1), (3) logits and confidences
             dev = self._mode_stats("bf16", zl, gc, gt, gs, probe, where)
             # (2) epilogue and commit rule, exact on the engine's own data
@@ -393,31 +412,62 @@ class Lockstep:
         assert e["noise"] <= lim(noise_cap), (f"too many exceptions explained only by the measured logit deviation "
                                               f"(each with D <= {logit_tol(self.model.n_layers):.3f} * max|z|): {e} of {n}")
 
+    def dictate(self, row, positions):
+        """A dictated commit (block position -> token) for an active row, applied to the engine and to every oracle
+        state alike (debugging aid of the C ABI; not a decision of either side)."""
+        self.eng.force_commit(row, positions)
+        r = self.ora.sched.active[row]
+        lo, _ = r.block_range(self.wl.block_len)
+        for state in (r, self.shadow.get(r.req_id)):
+            if state is None:
+                continue
+            for j, t in positions.items():
+                assert (r.mask >> j) & 1 or state is not r
+                state.tokens[lo + j] = t
+        for j in positions:
+            r.mask &= ~(1 << j)
+            r.committed += 1
+        self.first_exception.setdefault(r.req_id, (r.b, -1))    # a free oracle run cannot know dictated tokens
+
     def check_free_run(self, req_ids=None) -> dict:
-        """Token parity that can fail: the oracle runs each tracked request ALONE and free (it adopts nothing from
-        the engine; a request's trajectory does not depend on its batch).  The engine's tokens must equal that run's
-        for every block before the request's first counted exception - the whole row when it has none.  Returns how
-        many requests were compared completely / partially / not at all (exception in their first block)."""
+        """Token parity that can fail: the oracle runs each tracked request ALONE and free - it adopts nothing from
+        the engine (a request's trajectory does not depend on its batch).  Step by step, up to the request's first
+        counted exception (to its end when it has none), the positions and token ids the free run commits must equal
+        what the engine committed in that step, and at the end the engine's token row must hold them.  Returns the
+        number of requests compared to their end, the number compared in part, and the steps compared."""
         L = self.wl.block_len
-        out = {"complete": 0, "partial": 0, "none": 0}
-        ids = req_ids if req_ids is not None else [rid for rid in self.ora.by_id if self.tracked(rid)]
+        out = {"complete": 0, "partial": 0, "steps": 0}
+        ids = req_ids if req_ids is not None else [rid for rid in self.commit_log]
         for rid in ids:
             q = self.reqs[rid]
             r = O.new_request(self.model, rid, q.prompt, q.g, q.alpha, L, q.start_block, q.gen_prefix)
             got, _ = self.eng.read_tokens(rid)
-            stop = self.first_exception.get(rid, r.n_blocks(L))
-            if stop <= q.start_block:
-                out["none"] += 1
-                continue
-            for b in range(q.start_block, stop):
+            stop = self.first_exception.get(rid)
+            log = iter(self.commit_log.get(rid, []))
+            finished = True
+            for b in range(q.start_block, r.n_blocks(L)):
                 r.b = b
                 O.start_block_state(r, L)
                 while r.mask:
-                    O.denoise_step(self.model, r, L, self.wl.tau, self.suffix_mode, steps_per_block=self.S)
+                    if stop is not None and (r.b, r.s) >= stop:
+                        finished = False
+                        break
+                    entry = next(log, None)
+                    if entry is None:                     # the lockstep run ended before this request did
+                        finished = False
+                        break
+                    rec = O.denoise_step(self.model, r, L, self.wl.tau, self.suffix_mode, steps_per_block=self.S)
+                    assert (entry[0], entry[1]) == (rec.block, rec.step)
+                    pos, tok = rec.positions[rec.committed], rec.tok[rec.committed]
+                    assert pos.tolist() == entry[2].tolist() and tok.tolist() == entry[3].tolist(), \
+                        f"request {rid} block {rec.block} step {rec.step}: the free oracle run commits other tokens"
+                    assert (got[pos] == tok).all(), f"request {rid}: token row differs from the free oracle run"
+                    out["steps"] += 1
+                if not finished:
+                    break
                 lo, hi = r.block_range(L)
-                assert (got[lo:hi] == r.tokens[lo:hi]).all(), f"request {rid} block {b}: tokens differ from the free oracle run"
                 if self.eos_id >= 0 and (r.tokens[r.p:hi] == self.eos_id).any():
                     assert (got[hi:] == self.wl.shape.mask_id).all(), f"request {rid} ran past its end-of-sequence block"
                     break
-            out["complete" if rid not in self.first_exception else "partial"] += 1
+            out["complete" if finished else "partial"] += 1
         return out

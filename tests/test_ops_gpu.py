@@ -218,3 +218,32 @@ def test_confidence_rows(B, n, V):
     tok, conf = tok.cpu().numpy(), conf.cpu().numpy()
     assert (tok == tok_ref).all()
     assert (np.abs(conf - conf_ref) / conf_ref).max() < 1e-4
+
+
+@pytest.mark.parametrize("M,V,K", [(1, 1024, 64), (37, 2000, 72), (130, 1026, 128), (300, 5000, 128),
+                                   (64, 152064, 256), (513, 4128, 512)])
+def test_lm_head_fused_with_the_confidence_pass(B, M, V, K):
+    """The LM-head GEMM reduces its own accumulators to (argmax, confidence) per row; the logits are stored here
+    only so that the result can be checked exactly on them: token ids bit for bit (mask id never, lowest id on ties),
+    confidences to 1e-4 against the oracle's formula, and both against the stand-alone confidence kernel."""
+    rng = np.random.default_rng(M + V + K)
+    hf = bf16_round(rng.normal(size=(M, K)))
+    W = bf16_round(rng.normal(size=(V, K)) * 0.3)
+    mask_id = V - 1
+    W[mask_id] = W[5] * 4.0 + 1.0                 # the mask id would win many rows if it took part
+    if V > 300:
+        W[300] = W[17]                            # identical columns: ties must go to the lower id
+    scale = torch.from_numpy(rng.uniform(0.3, 30.0, size=M).astype(F32))
+    tok, conf, logits = B.op_lm_head_confidence(hf.cuda(), W.cuda(), scale.cuda(), mask_id, want_logits=True)
+    tok, conf, z = tok.cpu().numpy(), conf.cpu().numpy(), logits.cpu().numpy()
+    ref = (hf.double().numpy() @ W.double().numpy().T) * scale.double().numpy()[:, None]
+    assert rel_err(z, ref) < 1e-4
+    tok_ref, conf_ref = O.confidence(z, mask_id)
+    assert (tok == tok_ref).all()
+    assert (tok != mask_id).all() and (tok != 300).all()
+    assert (np.abs(conf - conf_ref) / conf_ref).max() < 1e-4
+    tok2, conf2 = B.op_confidence(logits, mask_id)
+    assert (tok2.cpu().numpy() == tok).all() and (np.abs(conf2.cpu().numpy() - conf) / conf).max() < 1e-4
+    # without the logits store the decisions are the same
+    tok3, conf3, none = B.op_lm_head_confidence(hf.cuda(), W.cuda(), scale.cuda(), mask_id)
+    assert none is None and (tok3.cpu().numpy() == tok).all() and (conf3.cpu().numpy() == conf).all()
