@@ -40,7 +40,14 @@ Readings taken where the paper is silent (each is listed in the design notes):
   * commit rule: strictly conf > tau, plus always the masked position of
     highest confidence (lowest position on ties); argmax over the vocabulary
     takes the lowest id on ties and never the mask id;
-  * block-cycles are batch-synchronous as in Algorithm 1.
+  * block-cycles are batch-synchronous as in Algorithm 1.  ``async_advance``
+    relaxes exactly that (the straggler effect of Section 2.3: a row whose
+    block is done idles until the slowest row of the cycle is): after every
+    denoise step each row whose block is complete moves to its next block on
+    its own (or leaves), survivors keep their order, and the head of P is
+    admitted under the same Eq. 1 rule; a row's own sequence of steps - refresh
+    at the first step of each block, cached steps after it - does not change,
+    so its tokens are those of the synchronous policy bit for bit.
 
 Whole-trajectory token values for n_layers >= 2 are "parity unpinned" (the
 paper prints no worked numeric example); every component and every special
@@ -391,10 +398,14 @@ class Scheduler:
     block-boundary advance / evict / stable compaction / refill."""
 
     def __init__(self, L: int, token_budget: int, max_batch: int, kv_capacity: int,
-                 sort_queue: bool = True, eos_id: Optional[int] = None, static_groups: bool = False):
+                 sort_queue: bool = True, eos_id: Optional[int] = None, static_groups: bool = False,
+                 async_advance: bool = False):
         self.L, self.beta, self.max_batch, self.kv_capacity = L, token_budget, max_batch, kv_capacity
         self.sort_queue = sort_queue
         self.static_groups = bool(static_groups)     # comparison policy of Section 3.1: fixed groups, no refill
+        self.async_advance = bool(async_advance)     # per-row block advance after every step (Section 2.3 relaxed)
+        assert not (self.static_groups and self.async_advance)
+        self.row_steps = 0                           # sum over denoise steps of the rows that ran a forward
         self.eos_id = None if eos_id is None or eos_id < 0 else int(eos_id)
         self.pending: List[ReqState] = []
         self.active: List[ReqState] = []
@@ -416,16 +427,25 @@ class Scheduler:
         if self.sort_queue:
             self.pending.sort(key=lambda q: (q.p, q.admit_order))
 
-    def evict_refill(self, first: bool = False):
+    def evict_refill(self, first: bool = False, only_done: bool = False):
         """Block boundary: b_i += 1 for every active row (not on the very first
         fill of a row), evict rows with b_i >= K_i or CheckEOS(r_i) (Algorithm 1:
         an end-of-sequence token among the blocks generated so far; off when
         no eos_id is configured), keep survivors in order,
         then admit the head of P while Eq. 1 stays within the budget, the batch
-        cap holds and the KV arena has a hole; admitted rows are appended."""
+        cap holds and the KV arena has a hole; admitted rows are appended.
+
+        ``only_done`` (the per-row advance of ``async_advance``, called after
+        every denoise step): rows whose block is not complete stay as they are -
+        same block, same step counter, same mask word - and only rows with an
+        empty mask word advance; everything else is the same rule."""
         L = self.L
         evicted, survivors = [], []
+        started = []                      # rows that begin a block now
         for r in self.active:
+            if only_done and r.mask != 0:
+                survivors.append(r)
+                continue
             r.b += 1
             done_upto = min(r.p + r.b * L, r.p + r.g)
             has_eos = self.eos_id is not None and bool((r.tokens[r.p:done_upto] == self.eos_id).any())
@@ -435,6 +455,7 @@ class Scheduler:
                 self.finished.append(r)
             else:
                 survivors.append(r)
+                started.append(r)
         self.active = survivors
         admitted = []
         # static groups: the next group starts only when every request of the current one has finished
@@ -450,13 +471,18 @@ class Scheduler:
             c.kv_base = base
             self.pending.pop(0)
             self.active.append(c)
+            started.append(c)
             admitted.append(c.req_id)
-        for r in self.active:
+        for r in started:
             start_block_state(r, L)
         widths = [r.width(L) for r in self.active]
         self.trace.append(CycleTrace(len(self.active), max(widths) if widths else 0, batch_cost(widths),
                                      evicted, admitted, [r.req_id for r in self.active]))
         return evicted, admitted
+
+    def advance_finished(self):
+        """async_advance: the step boundary.  Rows whose block is complete advance or leave, the queue refills."""
+        return self.evict_refill(only_done=True)
 
     def effective_compute_ratio(self, nominal_batch: int) -> float:
         """Eq. 2: R = (1 / (T B)) * sum_t a_t over the cycles that ran."""
@@ -507,10 +533,13 @@ def build_indices(active: Sequence[ReqState], L: int, suffix_mode: int = SUFFIX_
 class Engine:
     def __init__(self, model: Model, L: int, tau: float, token_budget: int, max_batch: int,
                  kv_capacity: int, suffix_mode: int = SUFFIX_FULL, sort_queue: bool = True,
-                 steps_per_block: Optional[int] = None, eos_id: Optional[int] = None, static_groups: bool = False):
+                 steps_per_block: Optional[int] = None, eos_id: Optional[int] = None, static_groups: bool = False,
+                 async_advance: bool = False):
         self.model, self.L, self.tau, self.suffix_mode = model, L, tau, suffix_mode
         self.steps_per_block = steps_per_block
-        self.sched = Scheduler(L, token_budget, max_batch, kv_capacity, sort_queue, eos_id, static_groups)
+        self.async_advance = bool(async_advance)
+        self.sched = Scheduler(L, token_budget, max_batch, kv_capacity, sort_queue, eos_id, static_groups,
+                               async_advance)
         self.by_id: Dict[int, ReqState] = {}
         self.total_committed = 0
         self.total_steps = 0
@@ -526,8 +555,16 @@ class Engine:
             self.by_id[rid].K = self.by_id[rid].V = None
         return ev, ad, len(self.sched.active)
 
+    def step_boundary(self):
+        """async_advance: after a denoise step, finished rows advance or leave and the queue refills."""
+        ev, ad = self.sched.advance_finished()
+        for rid in ev:
+            self.by_id[rid].K = self.by_id[rid].V = None
+        return ev, ad, len(self.sched.active)
+
     def denoise_step(self, keep_logits: bool = False) -> List[StepRecord]:
         recs = []
+        self.sched.row_steps += sum(1 for r in self.sched.active if r.mask != 0)
         for r in self.sched.active:
             if r.mask != 0:
                 rec = denoise_step(self.model, r, self.L, self.tau, self.suffix_mode, keep_logits,
@@ -541,7 +578,8 @@ class Engine:
         return all(r.mask == 0 for r in self.sched.active)
 
     def run(self, max_cycles: int = 1 << 30) -> int:
-        """Algorithm 1 until P and A are empty; returns the number of block-cycles."""
+        """Algorithm 1 until P and A are empty; returns the number of block-cycles.  With async_advance a "cycle"
+        ends only when the active set has run empty (normally once, at the end of the stream)."""
         cycles = 0
         while cycles < max_cycles:
             _, _, n = self.evict_refill()
@@ -549,6 +587,8 @@ class Engine:
                 break
             while not self.block_done():
                 self.denoise_step()
+                if self.async_advance:
+                    self.step_boundary()
             cycles += 1
         return cycles
 

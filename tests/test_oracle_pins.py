@@ -687,3 +687,104 @@ def test_static_groups_admit_only_into_an_empty_batch_and_lose_to_refill_on_stra
     # a static group of one 8-block and three 1-block requests runs 8 cycles with 4, 1, 1, ... rows: R = 11 / 32
     assert abs(r_static - 11.0 / 32.0) < 1e-9
     assert r_refill > 0.9 and len(co.trace) < len(st.trace)
+
+
+# ------------------------------------------- asynchronous per-row block advance ---
+
+def _async_pair(model, reqs, L, tau, **kw):
+    """The same stream served by the synchronous policy of Algorithm 1 and by the per-row advance."""
+    out = []
+    for mode in (False, True):
+        e = O.Engine(model, L, tau, kw.get("beta", 0), kw.get("max_batch", 8), kw.get("cap", 1 << 20),
+                     kw.get("suffix", O.SUFFIX_FULL), True, async_advance=mode)
+        for q in reqs:
+            e.admit(*q)
+        e.run()
+        out.append(e)
+    return out
+
+
+def test_async_advance_hand_example_of_the_straggler_stall():
+    """tau = 1 makes every block take exactly its length in steps (one forced token per step), so the timeline is
+    arithmetic.  L = 32, two slots, prompts sorted r0 < r1 < r2: r0 has g = 40 (blocks of 32 and 8 steps), r1 has
+    g = 64 (32 + 32), r2 (g = 32) waits.  Synchronous cycles: 32 steps, then 32 (r0 idles for 24 of them), both rows
+    leave, then r2's 32: 96 steps.  Per-row advance: r0 leaves after step 40, r2 takes its slot and ends at 72, r1
+    ends at 64: 72 steps.  Forward passes per row are the same either way: 40 + 64 + 32."""
+    shape, model = tiny_model()
+    rng = np.random.default_rng(3)
+    reqs = [(i, rng.integers(0, 49, size=p), g, 2.0, 0, None) for i, (p, g) in enumerate([(3, 40), (5, 64), (9, 32)])]
+    sync, asyn = _async_pair(model, reqs, 32, 1.0, max_batch=2)
+    assert sync.total_steps == 96 and asyn.total_steps == 72
+    assert sync.sched.row_steps == asyn.sched.row_steps == 40 + 64 + 32
+    for q in reqs:
+        assert (sync.tokens(q[0]) == asyn.tokens(q[0])).all()
+
+
+@pytest.mark.parametrize("suffix_mode", [O.SUFFIX_FULL, O.SUFFIX_NONE])
+def test_async_advance_leaves_every_request_its_own_trajectory(suffix_mode):
+    """A row's sequence of steps (refresh at the first step of each block, cached steps after it) is the same under
+    both policies and alone, so tokens and per-request step counts agree bit for bit; only the interleaving changes,
+    and the stream needs no more steps than the synchronous cycles do."""
+    shape, model = tiny_model()
+    L = 4
+    rng = np.random.default_rng(12)
+    spec = [(5, 8, 3.0, 0), (11, 12, 8.0, 1), (2, 5, 1.0, 0), (8, 8, 20.0, 0), (6, 16, 0.7, 2), (4, 4, 30.0, 0)]
+    reqs = [(i, rng.integers(0, 49, size=p), g, a, st, rng.integers(0, 49, size=st * L) if st else None)
+            for i, (p, g, a, st) in enumerate(spec)]
+    sync, asyn = _async_pair(model, reqs, L, 0.9, max_batch=3, beta=70, suffix=suffix_mode)
+    assert asyn.total_steps <= sync.total_steps
+    assert asyn.sched.row_steps == sync.sched.row_steps == sum(r.steps for r in asyn.by_id.values())
+    for q in reqs:
+        alone = run_engine(model, [q], L, 0.9, suffix=suffix_mode)
+        alone.run()
+        for e in (sync, asyn):
+            assert (e.tokens(q[0]) == alone.tokens(q[0])).all()
+            assert e.by_id[q[0]].steps == alone.by_id[q[0]].steps
+            assert e.by_id[q[0]].committed == q[2] - q[4] * L
+
+
+def test_async_advance_scheduler_invariants():
+    """Model-free: every step boundary keeps survivors in order, appends admissions in queue order, admits only
+    within Eq. 1 and the batch cap, never moves a surviving row's KV slab, advances only rows whose block is done,
+    and leaves the mask word and step counter of the others alone."""
+    L = 32
+    rng = np.random.default_rng(5)
+    s = O.Scheduler(L, 3000, 6, 4096, async_advance=True)
+    for i in range(40):
+        s.submit(sched_req(i, int(rng.integers(5, 300)), int(rng.choice([32, 64, 40, 96]))))
+    s.evict_refill()
+    admitted_all = [r.req_id for r in s.active]
+    steps = 0
+    while s.active:
+        steps += 1
+        before = [(r.req_id, r.b, r.s, r.mask, r.kv_base) for r in s.active]
+        for r in s.active:                     # a synthetic step: each unfinished row commits 1..8 positions
+            k = int(rng.integers(1, 9))
+            for _ in range(k):
+                if r.mask:
+                    r.mask &= r.mask - 1
+            r.s += 1
+        done = {r.req_id for r in s.active if r.mask == 0}
+        mid = {r.req_id: (r.b, r.s, r.mask, r.kv_base) for r in s.active}
+        ev, ad = s.advance_finished()
+        ids = [r.req_id for r in s.active]
+        survivors = [rid for rid, *_ in before if rid not in ev]
+        assert ids == survivors + ad and set(ev) <= done
+        admitted_all += ad
+        for r in s.active:
+            if r.req_id in ad:
+                assert r.s == 0 and r.mask == (1 << min(L, r.g)) - 1
+            elif r.req_id in done:
+                b0 = mid[r.req_id][0]
+                assert r.b == b0 + 1 and r.s == 0 and r.mask != 0 and r.kv_base == mid[r.req_id][3]
+            else:
+                assert (r.b, r.s, r.mask, r.kv_base) == mid[r.req_id]
+        if ad:
+            assert O.batch_cost([r.width(L) for r in s.active]) <= 3000
+        assert len(ids) <= 6
+        slabs = sorted((r.kv_base, r.p + r.g) for r in s.active)
+        assert all(a[0] + a[1] <= b[0] for a, b in zip(slabs, slabs[1:])) and all(b + n <= 4096 for b, n in slabs)
+        assert steps < 5000
+    assert not s.pending and len(s.finished) == 40
+    order = sorted(range(40), key=lambda i: (s.finished[[r.req_id for r in s.finished].index(i)].p, i))
+    assert admitted_all == order                 # the admitted sequence is the sorted queue, front to back
