@@ -73,6 +73,13 @@ typedef struct {
                                     becomes BS_REQ_FINISHED); < 0: off, every request generates exactly g_i tokens */
   int static_groups;             /* 1: the comparison policy of Section 3.1 (fixed groups: nothing is admitted until
                                     every request of the current group has finished); 0: block-boundary refill */
+  int async_advance;             /* 1: per-row block advance - the straggler stall of Section 2.3 (a row whose block is
+                                    done idles until the slowest row of the cycle is) relaxed: every bs_denoise_step
+                                    ends with the block boundary of Algorithm 1 applied to the rows whose block is
+                                    complete (advance or evict, stable compaction, refill under Eq. 1), so a row starts
+                                    its next block in the following step.  bs_block_done then reports all_done only
+                                    when the active set is empty; bs_evict_refill is the first fill and any later fill
+                                    of an empty active set.  0: batch-synchronous block cycles (Algorithm 1) */
   int keep_logits;               /* parity hook: 1 = the LM head also stores the fp32 logits [M_m, vocab] of every step
                                     (4 * max_batch * L * vocab more workspace bytes) so that bs_debug_read can return
                                     them; 0 = the logits never reach device memory, only the confidence partials of
@@ -107,6 +114,9 @@ typedef struct {
   long long packed_tokens;    /* sum over steps of the packed query tokens M */
   long long lm_rows;          /* sum over steps of the masked rows M_m */
   long long kernel_launches;  /* kernels this engine has enqueued */
+  long long row_steps;        /* sum over steps of the rows that ran a forward (unfinished blocks) */
+  long long active_row_steps; /* sum over steps of |A|; row_steps / active_row_steps is the share of active rows
+                                 that do work in a step (1 with async_advance) */
 } bs_stats;
 
 /* Sizes of the three device buffers the caller must provide for this config

@@ -20,9 +20,10 @@ from paper_2607_08930_b200 import binding as B, build  # noqa: E402
 
 
 def run_variant(wl, weights, sort_queue: bool, suffix_mode: int, steps_per_block: int = 0,
-                static_groups: bool = False):
+                static_groups: bool = False, async_advance: bool = False, kv_capacity_tokens=None):
     eng = B.engine_for_workload(wl, weights, sort_queue=sort_queue, suffix_mode=suffix_mode,
-                                steps_per_block=steps_per_block, static_groups=static_groups)
+                                steps_per_block=steps_per_block, static_groups=static_groups,
+                                async_advance=async_advance, kv_capacity_tokens=kv_capacity_tokens)
     for r in wl.requests:
         eng.admit(r.req_id, r.prompt, r.g, r.alpha, r.start_block, r.gen_prefix)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -36,7 +37,9 @@ def run_variant(wl, weights, sort_queue: bool, suffix_mode: int, steps_per_block
     ms = ev0.elapsed_time(ev1)
     out = dict(tokens_per_s=st.committed / (ms * 1e-3), job_s=ms * 1e-3, cycles=st.cycles, steps=st.steps,
                packed_tokens=st.packed_tokens, mean_active=st.sum_active / max(st.cycles, 1),
-               effective_compute_ratio=st.sum_active / max(st.cycles, 1) / wl.max_batch)
+               effective_compute_ratio=st.sum_active / max(st.cycles, 1) / wl.max_batch,
+               mean_active_per_step=st.active_row_steps / max(st.steps, 1),
+               rows_working_per_step=st.row_steps / max(st.active_row_steps, 1))
     eng.close()
     return out
 
@@ -48,6 +51,9 @@ def main():
     ap.add_argument("--static-groups", action="store_true",
                     help="add the comparison policy: fixed groups in submission order, no refill until a group is done")
     ap.add_argument("--requests", type=int, default=0, help="use only the first N requests of the workload")
+    ap.add_argument("--async-advance", action="store_true",
+                    help="add the per-row block advance (sorted queue, full suffix) beside the synchronous cycles")
+    ap.add_argument("--kv-rows", type=int, default=0, help="rows of the KV arena (0: sized from the workload)")
     ap.add_argument("--steps-per-block", type=int, nargs="*", default=[],
                     help="extra variants with a transfer quota S < L (sorted queue, full suffix)")
     args = ap.parse_args()
@@ -75,6 +81,15 @@ def main():
         res.update(workload=base.name, block_len=base.block_len, queue=f"sorted, S = {S}", suffix="full")
         print(json.dumps(res), flush=True)
         rows.append(res)
+    if args.async_advance:
+        for name, kw in (("sorted, synchronous block cycles (Algorithm 1)", dict()),
+                         ("sorted, per-row block advance", dict(async_advance=True))):
+            kw.update(kv_capacity_tokens=args.kv_rows or None)
+            run_variant(base, weights, True, B.SUFFIX_FULL, **kw)
+            res = run_variant(base, weights, True, B.SUFFIX_FULL, **kw)
+            res.update(workload=base.name, block_len=base.block_len, queue=name, suffix="full")
+            print(json.dumps(res), flush=True)
+            rows.append(res)
     if args.static_groups:
         for name, kw in (("block-boundary refill, submission order", dict(sort_queue=False)),
                          ("static groups, submission order", dict(sort_queue=False, static_groups=True))):
@@ -83,11 +98,13 @@ def main():
             res.update(workload=base.name, block_len=base.block_len, queue=name, suffix="full")
             print(json.dumps(res), flush=True)
             rows.append(res)
-    print("\n| L | queue | suffix | committed tokens/s | job s | cycles | steps | packed tokens | mean |A| |")
-    print("|---|---|---|---|---|---|---|---|---|")
+    print("\n| L | queue | suffix | committed tokens/s | job s | cycles | steps | packed tokens | mean |A| per step | "
+          "share of active rows working |")
+    print("|---|---|---|---|---|---|---|---|---|---|")
     for r in rows:
         print(f"| {r['block_len']} | {r['queue']} | {r['suffix']} | {r['tokens_per_s']:.0f} | {r['job_s']:.1f} | "
-              f"{r['cycles']} | {r['steps']} | {r['packed_tokens']} | {r['mean_active']:.1f} |")
+              f"{r['cycles']} | {r['steps']} | {r['packed_tokens']} | {r['mean_active_per_step']:.1f} | "
+              f"{r['rows_working_per_step']:.3f} |")
 
 
 if __name__ == "__main__":

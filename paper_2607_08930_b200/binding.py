@@ -37,7 +37,7 @@ class BsConfig(C.Structure):
                 ("token_budget", C.c_longlong), ("max_batch", C.c_int), ("max_requests", C.c_int),
                 ("max_row_tokens", C.c_int), ("kv_capacity_tokens", C.c_longlong), ("suffix_mode", C.c_int),
                 ("sort_queue", C.c_int), ("steps_per_block", C.c_int), ("eos_id", C.c_int),
-                ("static_groups", C.c_int), ("keep_logits", C.c_int)]
+                ("static_groups", C.c_int), ("async_advance", C.c_int), ("keep_logits", C.c_int)]
 
 
 class BsWeights(C.Structure):
@@ -54,7 +54,7 @@ class BsSizes(C.Structure):
 class BsStats(C.Structure):
     _fields_ = [("steps", C.c_longlong), ("cycles", C.c_longlong), ("sum_active", C.c_longlong),
                 ("committed", C.c_longlong), ("packed_tokens", C.c_longlong), ("lm_rows", C.c_longlong),
-                ("kernel_launches", C.c_longlong)]
+                ("kernel_launches", C.c_longlong), ("row_steps", C.c_longlong), ("active_row_steps", C.c_longlong)]
 
 
 EXPORTS = ["bs_query_sizes", "bs_init_model", "bs_admit", "bs_evict_refill", "bs_denoise_step", "bs_block_done",
@@ -131,11 +131,11 @@ def _check_op(rc: int, name: str) -> None:
 def make_config(shape, block_len: int, tau: float, token_budget: int, max_batch: int, max_requests: int,
                 max_row_tokens: int, kv_capacity_tokens: int, suffix_mode: int = SUFFIX_FULL,
                 sort_queue: bool = True, steps_per_block: int = 0, eos_id: int = -1,
-                static_groups: bool = False, keep_logits: bool = False) -> BsConfig:
+                static_groups: bool = False, keep_logits: bool = False, async_advance: bool = False) -> BsConfig:
     return BsConfig(shape.n_layers, shape.d_model, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, shape.d_ffn,
                     shape.vocab, shape.mask_id, shape.rms_eps, shape.rope_theta, block_len, tau, token_budget,
                     max_batch, max_requests, max_row_tokens, kv_capacity_tokens, suffix_mode, int(sort_queue),
-                    int(steps_per_block), int(eos_id), int(static_groups), int(keep_logits))
+                    int(steps_per_block), int(eos_id), int(static_groups), int(async_advance), int(keep_logits))
 
 
 def query_sizes(cfg: BsConfig) -> BsSizes:
@@ -299,7 +299,8 @@ class Engine:
 
 def engine_for_workload(wl, weights, *, kv_capacity_tokens: Optional[int] = None, suffix_mode: int = SUFFIX_FULL,
                         sort_queue: bool = True, steps_per_block: int = 0, eos_id: int = -1,
-                        static_groups: bool = False, keep_logits: bool = False, device: str = "cuda:0") -> Engine:
+                        static_groups: bool = False, keep_logits: bool = False, async_advance: bool = False,
+                        device: str = "cuda:0") -> Engine:
     """Size an engine for a bs_inputs.Workload (the caller still admits the requests)."""
     mrt = wl.max_row_tokens
     if kv_capacity_tokens is None:
@@ -309,7 +310,7 @@ def engine_for_workload(wl, weights, *, kv_capacity_tokens: Optional[int] = None
             kv_capacity_tokens = min(kv_capacity_tokens, wl.token_budget + wl.max_batch * max(r.g for r in wl.requests))
     cfg = make_config(wl.shape, wl.block_len, wl.tau, wl.token_budget, wl.max_batch, len(wl.requests), mrt,
                       max(kv_capacity_tokens, mrt), suffix_mode, sort_queue, steps_per_block, eos_id, static_groups,
-                      keep_logits)
+                      keep_logits, async_advance)
     return Engine(cfg, weights, device)
 
 

@@ -51,6 +51,7 @@ struct DevState {
   int S;                // diffusion steps per block (transfer quota of Section 2.5); S = L: one forced token per step
   int eos_id;           // CheckEOS of Algorithm 1 (< 0: off)
   int static_groups;    // 1: no admission while any row of the current group is active (comparison policy)
+  int async_advance;    // 1: rows advance / leave and the queue refills after every denoise step
   long long beta, kv_capacity;
   float tau;
   int* hdr;             // [kHdrInts] followed directly by row_mask[max_batch]

@@ -117,6 +117,8 @@ const char* check_config(const bs_config& c) {
   if (c.steps_per_block < 0 || c.steps_per_block > c.block_len) return "steps_per_block must be in [0, block_len]";
   if (c.eos_id >= c.vocab || c.eos_id == c.mask_id) return "eos_id must be a token id other than the mask id, or negative";
   if (c.keep_logits != 0 && c.keep_logits != 1) return "keep_logits must be 0 or 1";
+  if (c.async_advance != 0 && c.async_advance != 1) return "async_advance must be 0 or 1";
+  if (c.async_advance && c.static_groups) return "async_advance and static_groups exclude each other";
   return nullptr;
 }
 
@@ -137,6 +139,8 @@ struct bs_engine {
   int* pinned = nullptr;    // hdr + row masks
   cudaEvent_t ev = nullptr;
   bool hdr_pending = false;
+  bool hdr_from_step = false;   // the header in flight was written by a denoise step (per-row advance: it may admit)
+  bool queue_dirty = false;     // requests were submitted since the queue was last uploaded
   int hdr[kHdrInts];
   std::unordered_map<long long, int> slot_of;
   std::vector<long long> id_of_slot;
@@ -225,16 +229,47 @@ int sync_header(bs_engine* e) {
     if (e->profiling) prof_collect(e);
     memcpy(e->hdr, e->pinned, sizeof(e->hdr));
     e->hdr_pending = false;
+    if (e->hdr_from_step && e->cfg.async_advance) {
+      // per-row advance: the step's own boundary may have admitted the head of the queue and evicted rows
+      const int adm = e->hdr[H_ADMITTED];
+      e->pending.erase(e->pending.begin(), e->pending.begin() + std::min<size_t>(adm, e->pending.size()));
+    }
+    e->hdr_from_step = false;
     if (e->hdr[H_ERROR] != 0) return fail(e, BS_E_TIMEOUT, "a bounded device-side wait ran out");
   }
   return BS_OK;
 }
 
-int post_header(bs_engine* e) {
+int post_header(bs_engine* e, bool from_step = false) {
   CU(e, cudaMemcpyAsync(e->pinned, e->st.hdr, (kHdrInts + e->cfg.max_batch) * sizeof(int), cudaMemcpyDeviceToHost,
                         e->stream));
   CU(e, cudaEventRecord(e->ev, e->stream));
   e->hdr_pending = true;
+  e->hdr_from_step = from_step;
+  return BS_OK;
+}
+
+// Request table entries of newly submitted requests and the pending queue P go to the device; the queue head restarts
+// at zero.  The header must be in sync (the device may have consumed queue entries since the last upload).
+int upload_queue(bs_engine* e) {
+  DevState& st = e->st;
+  const int n_slots = (int)e->id_of_slot.size(), first = e->uploaded_slots;
+  if (n_slots > first) {
+    const size_t n = n_slots - first;
+    std::vector<int> zeros(n, 0);
+    CU(e, cudaMemcpyAsync(st.req_p + first, e->h_p.data() + first, n * 4, cudaMemcpyHostToDevice, e->stream));
+    CU(e, cudaMemcpyAsync(st.req_g + first, e->h_g.data() + first, n * 4, cudaMemcpyHostToDevice, e->stream));
+    CU(e, cudaMemcpyAsync(st.req_b + first, e->h_b.data() + first, n * 4, cudaMemcpyHostToDevice, e->stream));
+    CU(e, cudaMemcpyAsync(st.req_alpha + first, e->h_alpha.data() + first, n * 4, cudaMemcpyHostToDevice, e->stream));
+    CU(e, cudaMemcpyAsync(st.req_state + first, zeros.data(), n * 4, cudaMemcpyHostToDevice, e->stream));
+    CU(e, cudaMemcpyAsync(st.req_committed + first, zeros.data(), n * 4, cudaMemcpyHostToDevice, e->stream));
+    e->uploaded_slots = n_slots;
+  }
+  if (!e->pending.empty())
+    CU(e, cudaMemcpyAsync(st.queue, e->pending.data(), e->pending.size() * 4, cudaMemcpyHostToDevice, e->stream));
+  const int qh[2] = {0, (int)e->pending.size()};
+  CU(e, cudaMemcpyAsync(st.hdr + H_QUEUE_HEAD, qh, sizeof(qh), cudaMemcpyHostToDevice, e->stream));
+  e->queue_dirty = false;
   return BS_OK;
 }
 
@@ -293,6 +328,7 @@ int bs_init_model(const bs_config* cfg, const bs_weights* w, void* kv, void* wor
   st.S = cfg->steps_per_block > 0 ? cfg->steps_per_block : cfg->block_len;
   st.eos_id = cfg->eos_id;
   st.static_groups = cfg->static_groups ? 1 : 0;
+  st.async_advance = cfg->async_advance ? 1 : 0;
   st.q_tile = attention_q_tile(cfg->n_q_heads, cfg->n_kv_heads, cfg->head_dim);
   st.slice_ms = e->ws.slice_ms;
   st.slice_am = e->ws.slice_am;
@@ -342,6 +378,10 @@ int bs_admit(bs_engine* e, long long req_id, const int* prompt, int p, int g, fl
   if (!e) return BS_E_ARG;
   const bs_config& c = e->cfg;
   const int L = c.block_len;
+  // per-row advance: a step in flight may still take entries off the front of the queue; account for them before
+  // the sorted insert moves positions
+  if (c.async_advance)
+    if (int rc = sync_header(e)) return rc;
   if (!prompt || p < 1 || g < 1 || start_block < 0) return fail(e, BS_E_ARG, "bad request geometry");
   const int K = (g + L - 1) / L;
   if (start_block >= K) return fail(e, BS_E_ARG, "start_block must be below K_i");
@@ -369,6 +409,7 @@ int bs_admit(bs_engine* e, long long req_id, const int* prompt, int p, int g, fl
     pos = std::upper_bound(e->pending.begin(), e->pending.end(), slot,
                            [&](int a, int b) { return e->h_p[a] < e->h_p[b]; });
   e->pending.insert(pos, slot);
+  e->queue_dirty = true;
   return BS_OK;
 }
 
@@ -377,22 +418,7 @@ int bs_evict_refill(bs_engine* e, int* n_evicted, int* n_admitted, int* n_active
   if (int rc = sync_header(e)) return rc;
   if (e->hdr[H_N_ACTIVE] > 0 && !e->hdr[H_ALL_DONE]) return fail(e, BS_E_STATE, "a block of this cycle is unfinished");
   DevState& st = e->st;
-  const int n_slots = (int)e->id_of_slot.size(), first = e->uploaded_slots;
-  if (n_slots > first) {
-    const size_t n = n_slots - first;
-    std::vector<int> zeros(n, 0);
-    CU(e, cudaMemcpyAsync(st.req_p + first, e->h_p.data() + first, n * 4, cudaMemcpyHostToDevice, e->stream));
-    CU(e, cudaMemcpyAsync(st.req_g + first, e->h_g.data() + first, n * 4, cudaMemcpyHostToDevice, e->stream));
-    CU(e, cudaMemcpyAsync(st.req_b + first, e->h_b.data() + first, n * 4, cudaMemcpyHostToDevice, e->stream));
-    CU(e, cudaMemcpyAsync(st.req_alpha + first, e->h_alpha.data() + first, n * 4, cudaMemcpyHostToDevice, e->stream));
-    CU(e, cudaMemcpyAsync(st.req_state + first, zeros.data(), n * 4, cudaMemcpyHostToDevice, e->stream));
-    CU(e, cudaMemcpyAsync(st.req_committed + first, zeros.data(), n * 4, cudaMemcpyHostToDevice, e->stream));
-    e->uploaded_slots = n_slots;
-  }
-  if (!e->pending.empty())
-    CU(e, cudaMemcpyAsync(st.queue, e->pending.data(), e->pending.size() * 4, cudaMemcpyHostToDevice, e->stream));
-  const int qh[2] = {0, (int)e->pending.size()};
-  CU(e, cudaMemcpyAsync(st.hdr + H_QUEUE_HEAD, qh, sizeof(qh), cudaMemcpyHostToDevice, e->stream));
+  if (int rc = upload_queue(e)) return rc;
   KL(e, launch_sched(st, e->stream));
   if (int rc = post_header(e)) return rc;
   if (int rc = sync_header(e)) return rc;
@@ -417,6 +443,11 @@ int bs_denoise_step(bs_engine* e, int* n_committed) {
   DevState& st = e->st;
   Workspace& ws = e->ws;
   cudaStream_t s = e->stream;
+  // per-row advance: this step's boundary admits from the queue, so requests submitted meanwhile must be on the device
+  if (c.async_advance && e->queue_dirty)
+    if (int rc = upload_queue(e)) return rc;
+  e->stats.row_steps += e->hdr[H_UNFINISHED];
+  e->stats.active_row_steps += n_rows;
   const int d = c.d_model, hq = c.n_q_heads, hkv = c.n_kv_heads, dh = c.head_dim;
   const int qkv_n = (hq + 2 * hkv) * dh;
 
@@ -529,7 +560,7 @@ int bs_denoise_step(bs_engine* e, int* n_committed) {
   KL(e, launch_commit_index(st, s));
   prof_work(e, BS_FAM_INDEX, 1, 0, 0);
   prof_mark(e, -1);
-  if (int rc = post_header(e)) return rc;
+  if (int rc = post_header(e, true)) return rc;
   e->stats.steps++;
   e->stats.packed_tokens += M;
   e->stats.lm_rows += Mm;

@@ -128,41 +128,54 @@ __device__ void build_index(const DevState& st, int parity, int n, int* smi) {
   }
 }
 
-__global__ void __launch_bounds__(kSchedThreads) k_sched(DevState st) {
+// Algorithm 1's block boundary for the rows of A (all threads of the CTA call this): advance, evict, stable
+// compaction, refill under Eq. 1, new blocks fully masked, index of the next step.
+//   only_done = false: the synchronous cycle - every active row advances by one block.
+//   only_done = true:  per-row advance (the straggler stall of Section 2.3 relaxed), run after every denoise step -
+//                      only rows whose block is complete advance or leave; the others keep their block, step counter
+//                      and mask word and merely move up when rows before them leave.
+__device__ void sched_body(const DevState& st, bool only_done) {
   __shared__ int smi[33];
   __shared__ long long sml[33];
   __shared__ int s_n, s_head, s_stop;
   __shared__ long long s_w;
-  pdl_wait();
-  pdl_trigger();
   const int i = threadIdx.x;
   const int n0 = st.hdr[H_N_ACTIVE];
   const int L = st.L;
 
-  // ---- advance every active row by one block, evict finished rows (b_i >= K_i or CheckEOS), compact (order
-  // preserved) ----
-  int keep = 0, slot = -1, kvb = 0;
+  // ---- advance, evict finished rows (b_i >= K_i or CheckEOS), compact (order preserved) ----
+  int keep = 0, slot = -1, kvb = 0, srow = 0;
+  unsigned mask = 0u;
   if (i < n0) {
     slot = st.row_slot[i];
     kvb = st.row_kv_base[i];
-    const int b = st.req_b[slot] + 1;
-    st.req_b[slot] = b;
-    const int K = (st.req_g[slot] + L - 1) / L;          // K_i = ceil(g_i / L)
-    keep = b < K;
-    if (keep && st.eos_id >= 0) {                        // CheckEOS over the blocks finished so far
-      const int p = st.req_p[slot];
-      const int* row = st.tokens + (size_t)slot * st.max_row_tokens;
-      const int upto = min(p + b * L, p + st.req_g[slot]);
-      for (int t = p; t < upto; ++t)
-        if (row[t] == st.eos_id) { keep = 0; break; }
+    mask = st.row_mask[i];
+    srow = st.row_s[i];
+    if (only_done && mask != 0u) {
+      keep = 1;                                            // mid-block: nothing changes for this row
+    } else {
+      const int b = st.req_b[slot] + 1;
+      st.req_b[slot] = b;
+      const int K = (st.req_g[slot] + L - 1) / L;          // K_i = ceil(g_i / L)
+      keep = b < K;
+      if (keep && st.eos_id >= 0) {                        // CheckEOS over the blocks finished so far
+        const int p = st.req_p[slot];
+        const int* row = st.tokens + (size_t)slot * st.max_row_tokens;
+        const int upto = min(p + b * L, p + st.req_g[slot]);
+        for (int t = p; t < upto; ++t)
+          if (row[t] == st.eos_id) { keep = 0; break; }
+      }
+      if (!keep) st.req_state[slot] = 2;
+      srow = -1;                                           // marks "starts a block now"
     }
-    if (!keep) st.req_state[slot] = 2;
   }
   int n_keep;
   const int dst = block_excl_scan(keep, &n_keep, smi);
   if (keep) {
     st.row_slot[dst] = slot;
     st.row_kv_base[dst] = kvb;
+    st.row_mask[dst] = mask;
+    st.row_s[dst] = srow;
   }
   __syncthreads();
 
@@ -212,6 +225,7 @@ __global__ void __launch_bounds__(kSchedThreads) k_sched(DevState st) {
       if (ok) {
         st.row_slot[n] = c;
         st.row_kv_base[n] = (int)start;
+        st.row_s[n] = -1;
         st.req_state[c] = 1;
         s_n = n + 1;
         s_head = head + 1;
@@ -223,8 +237,8 @@ __global__ void __launch_bounds__(kSchedThreads) k_sched(DevState st) {
     __syncthreads();
   }
   const int n = s_n;
-  // ---- every row starts its block fully masked ----
-  if (i < n) {
+  // ---- rows that start a block (advanced or admitted) begin it fully masked ----
+  if (i < n && st.row_s[i] < 0) {
     const int sl = st.row_slot[i];
     const int lo = st.req_p[sl] + st.req_b[sl] * L;
     const int len = min(L, st.req_p[sl] + st.req_g[sl] - lo);
@@ -237,10 +251,16 @@ __global__ void __launch_bounds__(kSchedThreads) k_sched(DevState st) {
     st.hdr[H_ADMITTED] = n - n_keep;
     st.hdr[H_QUEUE_HEAD] = s_head;
     st.hdr[H_WIDTH] = (int)s_w;
-    st.hdr[H_COMMITTED_STEP] = 0;
+    if (!only_done) st.hdr[H_COMMITTED_STEP] = 0;
   }
   __syncthreads();
   build_index(st, st.hdr[H_PARITY] ^ 1, n, smi);
+}
+
+__global__ void __launch_bounds__(kSchedThreads) k_sched(DevState st) {
+  pdl_wait();
+  pdl_trigger();
+  sched_body(st, false);
 }
 
 // Commit rule per request (one warp per row): positions with conf > tau, plus the step's quota of most confident
@@ -308,7 +328,8 @@ __global__ void __launch_bounds__(kSchedThreads) k_commit_index(DevState st) {
     st.hdr[H_TOTAL_HI] = (int)(unsigned)(tot >> 32);
   }
   __syncthreads();
-  build_index(st, parity ^ 1, n, smi);
+  if (st.async_advance) sched_body(st, true);     // finished rows move on or leave now, the queue refills
+  else build_index(st, parity ^ 1, n, smi);
 }
 
 // Debug aid: commits the given block positions of one active row with the given tokens, as if a step had chosen

@@ -127,7 +127,7 @@ class Lockstep:
 
     def __init__(self, wl, weights_cuda, weights_np, suffix_mode=0, kv_capacity=None, sort_queue=True, track=None,
                  model=None, steps_per_block=0, eos_id=-1, static_groups=False, modes=("bf16", "fp32"),
-                 engine_kwargs=None):
+                 async_advance=False, engine_kwargs=None):
         self.wl = wl
         self.track = None if track is None else set(track)
         # the near-tie classes below are written for one forced token per step; a general transfer quota is checked
@@ -137,13 +137,15 @@ class Lockstep:
         self.eos_id = eos_id
         self.eng = B.engine_for_workload(wl, weights_cuda, kv_capacity_tokens=kv_capacity, suffix_mode=suffix_mode,
                                          sort_queue=sort_queue, steps_per_block=steps_per_block, eos_id=eos_id,
-                                         static_groups=static_groups, keep_logits=True, **(engine_kwargs or {}))
+                                         static_groups=static_groups, keep_logits=True, async_advance=async_advance,
+                                         **(engine_kwargs or {}))
         self.model = model if model is not None else O.model_from_weights(wl.shape, weights_np)
         assert self.model.bf16_activations
         self.model32 = dataclasses.replace(self.model, bf16_activations=False) if "fp32" in modes else None
         self.ora = O.Engine(self.model, wl.block_len, wl.tau, wl.token_budget, wl.max_batch,
                             self.eng.cfg.kv_capacity_tokens, suffix_mode, sort_queue, steps_per_block=steps_per_block,
-                            eos_id=eos_id, static_groups=static_groups)
+                            eos_id=eos_id, static_groups=static_groups, async_advance=async_advance)
+        self.async_advance = async_advance
         self.shadow = {}                 # req_id -> the fp32-mode oracle's copy of a tracked request
         self.suffix_mode = suffix_mode
         self.excluded = {c: 0 for c in CLASSES}
@@ -363,6 +365,19 @@ class Lockstep:
             k += nm
         assert k == Mm
         self.steps += 1
+        if self.async_advance:
+            # per-row advance: the step ended with the block boundary for the rows whose block is complete
+            ev_o, ad_o, n_o = self.ora.step_boundary()
+            hdr = self.eng.debug(B.DBG_HEADER)
+            assert (int(hdr[5]), int(hdr[6]), int(hdr[0])) == (len(ev_o), len(ad_o), n_o), \
+                "eviction / admission counts of the step boundary differ"
+            ids = self.eng.debug(B.DBG_REQ_ID_OF_ROW, np.int64)
+            assert ids.tolist() == [r.req_id for r in self.ora.sched.active], "row order differs after the step boundary"
+            if n_o:
+                assert self.eng.debug(B.DBG_ROW_KV_BASE).tolist() == [r.kv_base for r in self.ora.sched.active]
+            for rid in ev_o:
+                if rid in self.shadow:
+                    self.shadow[rid].K = self.shadow[rid].V = None
         return n_commit
 
     def run(self, max_cycles=1 << 30, phase1=None):

@@ -407,3 +407,61 @@ def test_static_group_policy_in_lockstep(B):
     ls2 = Lockstep(wl, wc, wn, sort_queue=False, track=set())
     ls2.admit(wl.requests)
     assert ls2.run() < cycles
+
+
+@pytest.mark.parametrize("suffix_mode", [0, 1])
+def test_async_advance_config1_full_lockstep(B, suffix_mode):
+    """Per-row block advance: finished rows start their next block (a whole-row refresh) in the following step while
+    the others continue with cached block steps, so one step mixes both kinds of rows; rows leave and the queue
+    refills at any step.  Full lockstep on workload 1, and the stream needs fewer steps than the synchronous cycles."""
+    from lockstep import Lockstep
+    wl = bs_inputs.workload(1)
+    wc, wn = both_weights(wl.shape, wl.weight_seed)
+    ls = Lockstep(wl, wc, wn, suffix_mode=suffix_mode, async_advance=True)
+    ls.admit([r for r in wl.requests if r.phase == 0])
+    ls.run(phase1=[r for r in wl.requests if r.phase == 1])
+    free = ls.check_free_run()
+    st = ls.eng.stats()
+    assert st.committed == wl.committed_target() == sum(r.committed for r in ls.ora.by_id.values())
+    assert st.row_steps == st.active_row_steps == ls.ora.sched.row_steps      # every active row works in every step
+    for r in wl.requests:
+        toks, state = ls.eng.read_tokens(r.req_id)
+        assert state == B.REQ_FINISHED and (toks != wl.shape.mask_id).all()
+    sync = B.engine_for_workload(wl, wc, suffix_mode=suffix_mode)
+    for r in wl.requests:
+        sync.admit(r.req_id, r.prompt, r.g, r.alpha, r.start_block, r.gen_prefix)
+    sync.run()
+    print(f"cfg1 async suffix={suffix_mode}: {st.steps} steps (synchronous cycles: {sync.stats().steps}) "
+          f"{ls.summary()} | free oracle run: {free}")
+    assert st.steps < sync.stats().steps
+    ls.assert_caps()
+
+
+def test_async_advance_stream_with_budget_arrivals_and_ragged_blocks(B):
+    """Per-row advance on a GQA stream under an Eq. 1 budget and KV-arena pressure, with start blocks, ragged last
+    blocks, and requests submitted while the stream is running (the queue is re-sent before the next step)."""
+    from lockstep import Lockstep
+    shape = bs_inputs.MINI_GQA
+    rng = np.random.default_rng(13)
+    n = 12
+    ps = rng.integers(5, 150, size=n)
+    gs = rng.choice([40, 64, 96, 33], size=n)
+    al = rng.choice([1.0, 6.0, 20.0, 60.0], size=n)
+    st = [int(rng.integers(0, -(-int(g) // 32))) for g in gs]
+    wl = bs_inputs.custom_workload(shape, ps, gs, al, st, token_budget=700, max_batch=6, seed=14, tau=0.9)
+    wc, wn = both_weights(shape, 77)
+    ls = Lockstep(wl, wc, wn, kv_capacity=600, async_advance=True)
+    ls.admit(wl.requests[:8])
+    _, _, active = ls.evict_refill()
+    assert active > 0
+    for k in range(5):
+        ls.step()
+    ls.admit(wl.requests[8:])          # arrivals in the middle of the stream
+    while not ls.eng.block_done():
+        ls.step()
+    assert ls.ora.block_done()
+    ls.run()                           # nothing may be left: the queue drained through the step boundaries
+    assert ls.eng.stats().committed == wl.committed_target()
+    assert len(ls.ora.sched.finished) == n
+    print(f"mini-gqa async: {ls.summary()}")
+    ls.assert_caps()

@@ -154,14 +154,16 @@ def test_llada_stream_full_depth_cycle_after_the_first_refill(B):
 TOY = bs_inputs.ModelShape("toy", 1, 64, 1, 1, 64, 64, 64, init_std=0.1)
 
 
-@pytest.mark.parametrize("cfg", [1, 2, 3, 4, 5])
-def test_whole_stream_model_free_replay(B, cfg):
+@pytest.mark.parametrize("cfg,async_advance", [(1, False), (2, False), (3, False), (4, False), (5, False),
+                                               (1, True), (3, True), (5, True)])
+def test_whole_stream_model_free_replay(B, cfg, async_advance):
     """The schedule and every index array of a stream depend on the model only through which positions each step
     commits.  Here each workload's whole request stream (same prompt lengths, generation lengths, start blocks,
     alphas, budget and batch cap; token ids redrawn for the toy vocabulary) is served by the engine on a one-layer toy
     model at tau = 0.9, so rows take between one and 32 steps per block; the oracle's scheduler and index builder
     follow with the engine's mask words and must reproduce every admission, eviction, row order, KV slab, header
-    count and index array of every step, bit for bit."""
+    count and index array of every step, bit for bit.  With async_advance the boundary runs after every step (rows
+    in their refresh step and rows in cached block steps share a step; admissions at any step)."""
     from lockstep import Lockstep
     src = bs_inputs.workload(cfg)
     rng = np.random.default_rng(100 + cfg)
@@ -176,16 +178,36 @@ def test_whole_stream_model_free_replay(B, cfg):
     from oracle import blockserve_oracle as O
     model = O.model_from_weights(TOY, bs_inputs.weights_to_numpy_f32({k: ([t.cpu() for t in v] if isinstance(v, list)
                                                                           else v.cpu()) for k, v in w.items()}))
-    ls = Lockstep(wl, w, None, track=set(), kv_capacity=cap, model=model, modes=("bf16",))
+    ls = Lockstep(wl, w, None, track=set(), kv_capacity=cap, model=model, modes=("bf16",), async_advance=async_advance)
     ls.admit([r for r in reqs if r.phase == 0])
     late = [r for r in reqs if r.phase == 1]
     cycles = ls.run(phase1=late or None)
     st = ls.eng.stats()
     assert st.committed == wl.committed_target()
-    assert cycles == st.cycles == len([t for t in ls.ora.sched.trace if t.n_active])
-    assert st.sum_active == sum(t.n_active for t in ls.ora.sched.trace)
     assert len(ls.ora.sched.finished) == len(reqs)
-    steps_per_cycle = st.steps / max(cycles, 1)
-    print(f"cfg{cfg} geometry: {len(reqs)} requests, {cycles} cycles, {st.steps} steps "
-          f"({steps_per_cycle:.1f} per cycle), {st.packed_tokens} packed tokens")
-    assert 1.0 < steps_per_cycle <= 32.0
+    print(f"cfg{cfg} geometry, async_advance={async_advance}: {len(reqs)} requests, {cycles} cycles, {st.steps} steps, "
+          f"{st.packed_tokens} packed tokens, rows working per step {st.row_steps / max(st.active_row_steps, 1):.3f}")
+    if async_advance:
+        assert st.row_steps == st.active_row_steps
+    else:
+        assert cycles == st.cycles == len([t for t in ls.ora.sched.trace if t.n_active])
+        assert st.sum_active == sum(t.n_active for t in ls.ora.sched.trace)
+        assert 1.0 < st.steps / max(cycles, 1) <= 32.0
+
+
+def test_async_advance_llada_shape_two_layers(B):
+    """Per-row advance at the LLaDA-8B width (two layers, full vocabulary): steps that mix whole-row refreshes with
+    cached 32-token block steps go through the tensor-core attention and the refresh-path projections together."""
+    from lockstep import Lockstep, lazy_oracle_model
+    shape = bs_inputs.LLADA_8B.with_layers(2)
+    wl = bs_inputs.custom_workload(shape, [120, 40, 77, 200], [64, 40, 96, 64], [4.0, 25.0, 9.0, 30.0], [0, 0, 1, 0],
+                                   seed=12, tau=0.9, max_batch=3, token_budget=900)
+    w = bs_inputs.make_weights(shape, 4242, device="cuda")
+    ls = Lockstep(wl, w, None, model=lazy_oracle_model(shape, w), async_advance=True)
+    ls.admit(wl.requests)
+    ls.run()
+    st = ls.eng.stats()
+    assert st.committed == wl.committed_target() and st.row_steps == st.active_row_steps
+    print("llada-2L async:", st.steps, "steps;", ls.summary())
+    ls.assert_caps()
+    assert ls.stats["bf16"].max_logit_err < 2e-2
