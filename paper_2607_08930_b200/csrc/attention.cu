@@ -284,8 +284,9 @@ __global__ void __launch_bounds__(256) k_attention_combine(AttnPartial part, bf1
 int attention_tc_q_tile(int hq, int hkv);
 cudaError_t launch_attention_tc(const bf16* qkv, const bf16* kc, const bf16* vc, bf16* out, const int* cu_q,
                                 const int* cu_tile, const int* kv_base, const int* vis, int n_rows, int n_tiles,
-                                int M, long long kv_rows, int max_nq, int hq, int hkv, int dh, int* error_flag,
-                                cudaStream_t s, bool* handled);
+                                int M, long long kv_rows, int max_nq, int max_vis, int hq, int hkv, int dh,
+                                float* scratch, size_t scratch_floats, int* error_flag, cudaStream_t s,
+                                bool* handled);
 
 static bool use_tc_attention(int hq, int hkv, int dh) {
   static const bool legacy = getenv("BS_ATTN_LEGACY") != nullptr;
@@ -331,11 +332,13 @@ cudaError_t launch_attention(const bf16* qkv, const bf16* kc, const bf16* vc, bf
   // Block steps of a model with one or two query heads per kv head are pure cache streaming with a few dozen
   // query rows: several small CTAs per SM hide the load latency better than one tensor-core CTA.  Every row has
   // at most one work item there, so the work-item prefix is the same for either kernel's q-tile.
-  const bool stream_small = max_nq > 0 && max_nq <= 32 && hq / hkv <= 2;
+  // (BS_ATTN_STREAM, read once: 0 sends these steps to the tensor-core kernel as well, 1 is the default)
+  static const int env_stream = getenv("BS_ATTN_STREAM") ? atoi(getenv("BS_ATTN_STREAM")) : 1;
+  const bool stream_small = env_stream != 0 && max_nq > 0 && max_nq <= 32 && hq / hkv <= 2;
   if (use_tc_attention(hq, hkv, dh) && !stream_small) {
     bool handled = false;
     cudaError_t r = launch_attention_tc(qkv, kc, vc, out, cu_q, cu_tile, kv_base, vis, n_rows, n_tiles, M, kv_rows,
-                                        max_nq, hq, hkv, dh, error_flag, s, &handled);
+                                        max_nq, max_vis, hq, hkv, dh, scratch, scratch_floats, error_flag, s, &handled);
     return handled ? r : cudaErrorNotSupported;     // the work-item prefix was built for this kernel's q-tile
   }
   const int G = hq / hkv;

@@ -15,10 +15,15 @@
 //               of the scores buffer it came from (one tcgen05.st per row, no shared-memory round trip);
 //               the output accumulates in TMEM over all key tiles and is rescaled lazily (only when a row's
 //               maximum has grown by more than 2^8), the running sum follows the same scale
+// Two instantiations: NQ = 2 (a work item's two Q tiles share every K/V tile the CTA loads; one CTA per SM) for
+// steps with many work items, and NQ = 1 (one Q tile, half the tensor memory, a two-stage K/V ring: two CTAs per SM
+// hide each other's dependent chains) for steps with few.  A launch may also cut every row's keys into chunks
+// (grid z): each chunk leaves an unnormalised fp32 partial (output, scale, sum) and a small kernel merges them.
 // Every wait is bounded; on a timeout the flag is raised, all roles drain, TMEM is freed.
 #include <math.h>
 #include <stdlib.h>
 
+#include <algorithm>
 #include <mutex>
 #include <unordered_map>
 
@@ -31,7 +36,7 @@ namespace {
 using namespace tc;
 
 constexpr int DH = 128;
-constexpr int kThreads = 320;             // producer warp, MMA warp, 8 softmax warps
+__host__ __device__ constexpr int threads_for(int nq) { return 64 + 128 * nq; }     // producer warp, MMA warp, 4 softmax warps per Q tile
 constexpr int kHalfBytes = 128 * 128;      // 128 rows x 64 bf16: one swizzled sub-tile of Q or P
 constexpr int kQBytes = 2 * kHalfBytes;
 
@@ -115,23 +120,28 @@ struct AttnTcParams {
   bf16* out;
   int n_rows, hq, hkv;
   int tq;            // tokens per Q tile (a work item holds two Q tiles)
-  int split;         // 1: one CTA per Q tile (few work items: more, shorter chains), 0: one CTA per work item
+  int chunks;        // key chunks per row (grid z); > 1: partials below instead of the output
+  float* part_o;     // [chunks][M][Hq * 128] unnormalised outputs
+  float2* part_ml;   // [chunks][M][Hq] (scale in log2 units, sum); sum = 0 marks an empty chunk
+  int M;
   int* error_flag;
 };
 
 constexpr int KT = 64;                                   // keys per tile
-constexpr int kStages = 4;
 constexpr int kKvHalf = KT * 128;                        // KT rows x 64 bf16
 constexpr int kStageBytes = 4 * kKvHalf;                 // K halves, V halves
-constexpr int kSmemBytes = 2 * kQBytes + kStages * kStageBytes + 1024;
+__host__ __device__ constexpr int stages_for(int nq) { return nq == 2 ? 4 : 2; }
+__host__ __device__ constexpr int smem_for(int nq) { return nq * kQBytes + stages_for(nq) * kStageBytes + 1024; }
 
-// Barrier slots
-enum { B_QFULL = 0, B_KVFULL = 1, B_KVEMPTY = B_KVFULL + kStages, B_SFULL = B_KVEMPTY + kStages,   // [tile][2]
-       B_PFULL = B_SFULL + 4, B_OFULL = B_PFULL + 2, B_COUNT = B_OFULL + 2 };
-
-__global__ void __launch_bounds__(kThreads, 1)
+template <int NQ>
+__global__ void __launch_bounds__(threads_for(NQ), NQ == 2 ? 1 : 2)
 k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                const __grid_constant__ CUtensorMap map_v, const AttnTcParams p) {
+  constexpr int kStages = stages_for(NQ);
+  constexpr unsigned kTmemCols = NQ == 2 ? 512u : 256u;
+  // Barrier slots
+  enum { B_QFULL = 0, B_KVFULL = 1, B_KVEMPTY = B_KVFULL + kStages, B_SFULL = B_KVEMPTY + kStages,   // [tile][2]
+         B_PFULL = B_SFULL + 4, B_OFULL = B_PFULL + 2, B_COUNT = B_OFULL + 2 };
   extern __shared__ unsigned char smem_dyn[];
   __shared__ __align__(8) unsigned long long bars[B_COUNT];
   __shared__ unsigned tmem_base_slot;
@@ -140,7 +150,7 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const unsigned smem0 = (smem_u32(smem_dyn) + 1023u) & ~1023u;
   const unsigned sQ = smem0;                              // [Q tile][dim half][128 rows x 128 B]
-  const unsigned sKV = sQ + 2 * kQBytes;
+  const unsigned sKV = sQ + NQ * kQBytes;
   const unsigned bar0 = smem_u32(&bars[0]);
   auto bar = [&](int i) { return bar0 + 8u * (unsigned)i; };
 
@@ -161,8 +171,8 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&tmem_base_slot))
-                 : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(&tmem_base_slot)), "r"(kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -176,20 +186,25 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   // ---- which row owns this work item: largest r with cu_tile[r] <= blockIdx.x ----
   const int G = p.hq / p.hkv;
   const int kh = blockIdx.y;
+  constexpr bool kSplit = NQ == 1;                          // one CTA per Q tile: two CTAs share a work item
+  const int item = kSplit ? (int)blockIdx.x >> 1 : (int)blockIdx.x;
   int lo = 0, hi = p.n_rows;
   while (hi - lo > 1) {
     const int mid = (lo + hi) >> 1;
-    if (p.cu_tile[mid] <= (p.split ? (int)blockIdx.x >> 1 : (int)blockIdx.x)) lo = mid; else hi = mid;
+    if (p.cu_tile[mid] <= item) lo = mid; else hi = mid;
   }
   const int row = lo;
-  const int item = p.split ? (int)blockIdx.x >> 1 : (int)blockIdx.x;
-  const int per_cta = p.split ? p.tq : 2 * p.tq;
-  const int t0 = p.cu_q[row] + (item - p.cu_tile[row]) * 2 * p.tq + (p.split ? ((int)blockIdx.x & 1) * p.tq : 0);
+  const int per_cta = NQ * p.tq;
+  const int t0 = p.cu_q[row] + (item - p.cu_tile[row]) * 2 * p.tq + (kSplit ? ((int)blockIdx.x & 1) * p.tq : 0);
   const int nt = min(per_cta, p.cu_q[row + 1] - t0);        // query tokens of this CTA (CTA-uniform)
   const int n_qt = nt <= 0 ? 0 : (nt > p.tq ? 2 : 1);       // Q tiles in use
   const int vis = p.vis[row];
   const int kvb = p.kv_base[row];
-  const int n_tiles = nt > 0 ? (vis + KT - 1) / KT : 0;
+  // key tiles of this CTA's chunk: [kt0, kt0 + n_tiles) of the row's ceil(vis / KT)
+  const int tiles_all = (vis + KT - 1) / KT;
+  const int per_chunk = (tiles_all + p.chunks - 1) / p.chunks;
+  const int kt0 = (int)blockIdx.z * per_chunk;
+  const int n_tiles = nt > 0 ? max(0, min(tiles_all, kt0 + per_chunk) - kt0) : 0;
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -204,7 +219,7 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         if (!mbar_wait(bar(B_KVEMPTY + s), (unsigned)((t / kStages) & 1) ^ 1u, abort_flag)) break;
         const unsigned st = sKV + s * kStageBytes;
         mbar_expect_tx(bar(B_KVFULL + s), (unsigned)kStageBytes);
-        const int key0 = kvb + t * KT;
+        const int key0 = kvb + (kt0 + t) * KT;
         tma_load_3d(st, &map_k, 0, kh, key0, bar(B_KVFULL + s));
         tma_load_3d(st + kKvHalf, &map_k, 64, kh, key0, bar(B_KVFULL + s));
         tma_load_3d(st + 2 * kKvHalf, &map_v, 0, kh, key0, bar(B_KVFULL + s));
@@ -281,7 +296,7 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         bool rescale = false;
         if (warp_has_rows) {
           // scores -> probabilities in registers; this part overlaps the previous tile's P V product
-          const int key0 = t * KT;
+          const int key0 = (kt0 + t) * KT;
           tmem_ld32(t_lane + b * 64, v);
           tmem_ld32(t_lane + b * 64 + 32, v + 32);
           // eight independent chains for the row maximum and the row sum: one warp per scheduler has no other
@@ -347,18 +362,29 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         __syncwarp();
         if (lane == 0) mbar_arrive(bar(B_PFULL + x));
       }
+      if (n_tiles == 0 && p.chunks > 1 && r < nrows)      // a chunk beyond the row's keys: an empty partial
+        p.part_ml[((size_t)blockIdx.z * p.M + t0 + x * p.tq + r / G) * p.hq + kh * G + r % G] = make_float2(0.f, 0.f);
       if (ok && n_tiles > 0 && mbar_wait(bar(B_OFULL + x), (unsigned)(n_tiles - 1) & 1u, abort_flag) &&
           warp_has_rows) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const int tok = r / G, hg = r % G;
         const bool valid = r < nrows;
         const float inv = 1.0f / l;
-        bf16* dst = p.out + (size_t)(t0 + x * p.tq + (valid ? tok : 0)) * (p.hq * DH) + (size_t)(kh * G + hg) * DH;
+        const size_t out_at = (size_t)(t0 + x * p.tq + (valid ? tok : 0)) * (p.hq * DH) + (size_t)(kh * G + hg) * DH;
+        bf16* dst = p.out + out_at;
+        float* pdst = p.chunks > 1 ? p.part_o + (size_t)blockIdx.z * p.M * (p.hq * DH) + out_at : nullptr;
+        if (pdst && valid)
+          p.part_ml[((size_t)blockIdx.z * p.M + t0 + x * p.tq + tok) * p.hq + kh * G + hg] = make_float2(m, l);
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
           float o[32];
           tmem_ld32(t_out + c * 32, o);
-          if (valid) {
+          if (valid && pdst) {
+#pragma unroll
+            for (int g = 0; g < 8; ++g)
+              *reinterpret_cast<float4*>(pdst + c * 32 + g * 4) =
+                  make_float4(o[g * 4], o[g * 4 + 1], o[g * 4 + 2], o[g * 4 + 3]);
+          } else if (valid) {
 #pragma unroll
             for (int g = 0; g < 4; ++g) {
               uint4 w;
@@ -383,7 +409,42 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   if (s_abort && threadIdx.x == 0 && p.error_flag) atomicExch(p.error_flag, 1);
   if (warp == 1) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+  }
+}
+
+// Merges the key chunks of every (token, head): out = sum_c w_c o_c / sum_c w_c l_c with w_c = 2^(m_c - max m).
+__global__ void __launch_bounds__(256) k_attention_tc_combine(const float* __restrict__ part_o,
+                                                              const float2* __restrict__ part_ml, int chunks, int M,
+                                                              bf16* __restrict__ out, int hq) {
+  pdl_wait();
+  pdl_trigger();
+  const int t = blockIdx.x;
+  const int out_ld = hq * DH;
+  for (int u = threadIdx.x; u < out_ld / 4; u += 256) {
+    const int h = (4 * u) / DH;
+    float mmax = -INFINITY;
+    for (int c = 0; c < chunks; ++c) {
+      const float2 ml = part_ml[((size_t)c * M + t) * hq + h];
+      if (ml.y > 0.f) mmax = fmaxf(mmax, ml.x);
+    }
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    float L = 0.f;
+    for (int c = 0; c < chunks; ++c) {
+      const float2 ml = part_ml[((size_t)c * M + t) * hq + h];
+      if (ml.y > 0.f) {
+        const float w = exp2f(ml.x - mmax);
+        const float4 ov = *reinterpret_cast<const float4*>(part_o + ((size_t)c * M + t) * out_ld + 4 * u);
+        acc.x += w * ov.x; acc.y += w * ov.y; acc.z += w * ov.z; acc.w += w * ov.w;
+        L += w * ml.y;
+      }
+    }
+    const float inv = 1.0f / L;
+    __nv_bfloat162 a = __floats2bfloat162_rn(acc.x * inv, acc.y * inv), b = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
+    uint2 o;
+    o.x = *reinterpret_cast<unsigned*>(&a);
+    o.y = *reinterpret_cast<unsigned*>(&b);
+    *reinterpret_cast<uint2*>(out + (size_t)t * out_ld + 4 * u) = o;
   }
 }
 
@@ -440,25 +501,27 @@ static int tokens_per_q_tile(int hq, int hkv) {
 // Query tokens per work item (two Q tiles share every K/V tile a CTA loads).
 int attention_tc_q_tile(int hq, int hkv) { return 2 * tokens_per_q_tile(hq, hkv); }
 
-// Returns cudaSuccess with *handled = false when the shape is left to the legacy kernel.
+// Returns cudaSuccess with *handled = false when the shape is left to the streaming kernel.
 cudaError_t launch_attention_tc(const bf16* qkv, const bf16* kc, const bf16* vc, bf16* out, const int* cu_q,
                                 const int* cu_tile, const int* kv_base, const int* vis, int n_rows, int n_tiles,
-                                int M, long long kv_rows, int max_nq, int hq, int hkv, int dh, int* error_flag,
-                                cudaStream_t s, bool* handled) {
+                                int M, long long kv_rows, int max_nq, int max_vis, int hq, int hkv, int dh,
+                                float* scratch, size_t scratch_floats, int* error_flag, cudaStream_t s,
+                                bool* handled) {
   *handled = false;
   (void)max_nq;
   if (dh != DH || hq % hkv || hq / hkv > 8 || kv_rows <= 0) return cudaSuccess;
   if (((uintptr_t)qkv | (uintptr_t)kc | (uintptr_t)vc) & 15) return cudaSuccess;
   const int G = hq / hkv;
   const int tq = tokens_per_q_tile(hq, hkv);
-  static int num_sms_of[kMaxDevices];      // per device; non-zero once the kernel attribute is set there
+  static int num_sms_of[kMaxDevices];      // per device; non-zero once the kernel attributes are set there
   int* sms = device_slot(num_sms_of);
   if (!sms) return cudaErrorInvalidDevice;
   if (!*sms) {
     std::lock_guard<std::mutex> lock(g_mutex);
     int dev = 0, n = 0;
     cudaGetDevice(&dev);
-    if (cudaFuncSetAttribute(k_attention_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess ||
+    if (cudaFuncSetAttribute(k_attention_tc<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_for(1)) != cudaSuccess ||
+        cudaFuncSetAttribute(k_attention_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_for(2)) != cudaSuccess ||
         cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1)
       return cudaErrorInvalidDevice;
     *sms = n;
@@ -472,12 +535,36 @@ cudaError_t launch_attention_tc(const bf16* qkv, const bf16* kc, const bf16* vc,
   *handled = true;
   AttnTcParams p;
   p.cu_q = cu_q; p.cu_tile = cu_tile; p.kv_base = kv_base; p.vis = vis; p.out = out;
-  p.n_rows = n_rows; p.hq = hq; p.hkv = hkv; p.tq = tq; p.error_flag = error_flag;
-  // With fewer work items than SMs each CTA is one long dependent chain over the row's key tiles: give every Q
-  // tile its own CTA.  With many work items the two Q tiles of an item share each K/V tile they load.
-  p.split = (long long)n_tiles * hkv < num_sms ? 1 : 0;
-  return launch_pdl(k_attention_tc, dim3(p.split ? 2 * n_tiles : n_tiles, hkv), dim3(kThreads), (size_t)kSmemBytes, s,
-                    mq, mk, mv, p);
+  p.n_rows = n_rows; p.hq = hq; p.hkv = hkv; p.tq = tq; p.error_flag = error_flag; p.M = M;
+  // Few work items (a block step): each CTA is one long dependent chain over the row's key tiles.  Every Q tile gets
+  // its own small CTA, two of them share an SM, and the rows' keys are cut into chunks until about two CTAs per SM
+  // are in flight.  Many work items (a refresh step): the two Q tiles of an item share each K/V tile they load.
+  static const int env_chunks = getenv("BS_ATTN_TC_CHUNKS") ? atoi(getenv("BS_ATTN_TC_CHUNKS")) : 0;
+  static const int env_nq = getenv("BS_ATTN_TC_NQ") ? atoi(getenv("BS_ATTN_TC_NQ")) : 0;
+  const long long items = (long long)n_tiles * hkv;
+  const bool small = env_nq ? env_nq == 1 : items < 2 * (long long)num_sms;
+  int chunks = 1;
+  if (small && scratch && max_vis > 0) {
+    const long long ctas = 2 * items;
+    const int key_tiles = (max_vis + KT - 1) / KT;
+    chunks = (int)((2ll * num_sms + ctas / 2) / ctas);              // about two CTAs per SM
+    chunks = std::max(1, std::min(chunks, key_tiles / 3));          // at least three key tiles per chunk
+    while (chunks > 1 && (size_t)chunks * M * ((size_t)hq * DH + 2 * hq) > scratch_floats) --chunks;
+  }
+  if (env_chunks >= 1 && scratch && (size_t)env_chunks * M * ((size_t)hq * DH + 2 * hq) <= scratch_floats)
+    chunks = env_chunks;
+  p.chunks = chunks;
+  p.part_o = scratch;
+  p.part_ml = reinterpret_cast<float2*>(scratch + (size_t)chunks * M * hq * DH);
+  cudaError_t r;
+  if (small)
+    r = launch_pdl(k_attention_tc<1>, dim3(2 * n_tiles, hkv, chunks), dim3(threads_for(1)), (size_t)smem_for(1), s, mq,
+                   mk, mv, p);
+  else
+    r = launch_pdl(k_attention_tc<2>, dim3(n_tiles, hkv, 1), dim3(threads_for(2)), (size_t)smem_for(2), s, mq, mk, mv, p);
+  if (r != cudaSuccess || chunks == 1) return r;
+  return launch_pdl(k_attention_tc_combine, dim3(M), dim3(256), 0, s, (const float*)p.part_o,
+                    (const float2*)p.part_ml, chunks, M, out, hq);
 }
 
 }  // namespace bs

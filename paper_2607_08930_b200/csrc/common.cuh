@@ -40,7 +40,8 @@ enum Hdr {
   H_N_ACTIVE = 0, H_M = 1, H_MM = 2, H_ALL_DONE = 3, H_COMMITTED_STEP = 4, H_EVICTED = 5, H_ADMITTED = 6,
   H_QUEUE_HEAD = 7, H_QUEUE_LEN = 8, H_ERROR = 9, H_PARITY = 10, H_QTILES = 11, H_MAX_VIS = 12, H_WIDTH = 13,
   H_TOTAL_LO = 14, H_TOTAL_HI = 15, H_UNFINISHED = 16, H_STEP_REFRESH = 17,
-  H_SUM_KV = 18   // sum over unfinished rows of the cache rows they attend over
+  H_SUM_KV = 18,  // sum over unfinished rows of the cache rows they attend over
+  H_PREV_MM = 19  // masked rows of the step that just ran (its lists stay readable in the other index buffer)
 };
 
 

@@ -654,11 +654,7 @@ int bs_debug_read(bs_engine* e, int what, int arg0, int arg1, void* host_buf, si
   const void* src = nullptr;
   size_t bytes = 0;
   std::vector<long long> ids;
-  int prev_mm = 0;
-  if (what >= BS_DBG_PREV_LM_ROW && what <= BS_DBG_PREV_LOGITS) {
-    // the previous step's list length is the end of its per-row prefix
-    CU(e, cudaMemcpy(&prev_mm, st.lm_base[prev] + n, 4, cudaMemcpyDeviceToHost));
-  }
+  const int prev_mm = e->hdr[H_PREV_MM];     // length of the lists of the step that just ran
   switch (what) {
     case BS_DBG_HEADER: src = st.hdr; bytes = kHdrInts * 4; break;
     case BS_DBG_ROW_SLOT: src = st.row_slot; bytes = n * 4; break;

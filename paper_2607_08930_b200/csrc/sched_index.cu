@@ -321,6 +321,7 @@ __global__ void __launch_bounds__(kSchedThreads) k_commit_index(DevState st) {
   }
   __syncthreads();
   if (threadIdx.x == 0) {
+    st.hdr[H_PREV_MM] = st.lm_base[parity][n];
     st.hdr[H_COMMITTED_STEP] = s_count;
     unsigned long long tot = ((unsigned long long)(unsigned)st.hdr[H_TOTAL_HI] << 32) | (unsigned)st.hdr[H_TOTAL_LO];
     tot += (unsigned long long)s_count;

@@ -271,6 +271,8 @@ class Lockstep:
         if self.track is None:
             g_logits = self.eng.debug(B.DBG_PREV_LOGITS, np.float32, cap=4 * Mm * V + 64).reshape(Mm, V)
         g_masks = self.eng.debug(B.DBG_ROW_MASK, np.uint32)
+        # with the per-row advance the step has already compacted the rows: look a row's mask word up by request id
+        ids_now = self.eng.debug(B.DBG_REQ_ID_OF_ROW, np.int64).tolist() if self.async_advance else None
         tau = np.float32(self.wl.tau)
         mask_id = self.wl.shape.mask_id
         k = 0
@@ -289,7 +291,10 @@ class Lockstep:
                 for i, j in enumerate(slots):
                     if gs[i]:
                         new_mask &= ~(1 << j)
-                assert new_mask == int(g_masks[row_index]), f"mask word ({where})"
+                if ids_now is None:
+                    assert new_mask == int(g_masks[row_index]), f"mask word ({where})"
+                elif new_mask != 0:      # (a finished row has moved on or left: the next step's index check sees it)
+                    assert new_mask == int(g_masks[ids_now.index(r.req_id)]), f"mask word ({where})"
                 r.mask = new_mask
                 r.committed += int(gs.sum())
                 r.s += 1

@@ -166,6 +166,12 @@ ATTN_CASES = [
     # four and eight query heads per kv head (32 and 16 tokens per Q tile)
     (8, 2, 128, [(70, 200), (32, 64), (33, 33)]),
     (16, 2, 128, [(40, 130), (32, 700)]),
+    # long-context block steps (GQA 28 / 4): rows of 1-2.5 k keys, whose key tiles are cut into chunks over several
+    # CTAs when scratch is given, with a ragged block, an empty row and rows shorter than one chunk beside them
+    (28, 4, 128, [(32, 2304)] * 8),
+    (28, 4, 128, [(32, 1100), (32, 2560), (17, 1300), (0, 64), (32, 40)]),
+    # a refresh row beside cached block steps (steps of the per-row advance mix both)
+    (28, 4, 128, [(700, 700), (32, 900), (32, 333)]),
 ]
 
 
