@@ -163,8 +163,8 @@ def run_ours(args):
     cap = kv_capacity_for(wl)
     target = wl.committed_target()
 
-    def new_engine():
-        return B.engine_for_workload(wl, weights, kv_capacity_tokens=cap, device=str(device))
+    def new_engine(**kw):
+        return B.engine_for_workload(wl, weights, kv_capacity_tokens=cap, device=str(device), **kw)
 
     def admit_all(eng, prompts):
         for r, pr in zip(wl.requests, prompts):
@@ -201,11 +201,11 @@ def run_ours(args):
     # ---- device-resident arm: requests admitted (copied to HBM) before the clock starts.  One engine is alive at a
     # time (a KV arena can take 45 GB): each job is bracketed by barrier + synchronize and timed with CUDA events on
     # the launching stream; the timed region is the sum over the K jobs.
-    def timed_jobs(n_jobs: int, profile: bool):
+    def timed_jobs(n_jobs: int, profile: bool, **engine_kw):
         stream = torch.cuda.current_stream()
         total_ms, stats, profs = 0.0, [], []
         for _ in range(n_jobs):
-            e = new_engine()
+            e = new_engine(**engine_kw)
             admit_all(e, pinned)
             e.set_profiling(profile)
             ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -255,6 +255,14 @@ def run_ours(args):
                     acc[k] += v[k]
         torch.cuda.empty_cache()
         phase("profiled job done")
+
+    # ---- the same jobs under the per-row block advance (a policy beyond Algorithm 1's synchronous cycles; reported
+    # beside the headline, never instead of it)
+    async_ms, async_stats, _ = timed_jobs(max(1, min(args.steps, 3)), profile=False, async_advance=True)
+    async_ms = max_over_ranks(async_ms, world, device)
+    async_committed = sum_over_ranks(float(sum(st.committed for st in async_stats)), world, device)
+    assert sum(st.committed for st in async_stats) == target * len(async_stats)
+    phase("per-row advance jobs done")
 
     # ---- end-to-end arm: host buffers in, host buffers out, through the C ABI (engine set-up is not timed) ----
     e2e_local = 0.0
@@ -319,6 +327,11 @@ def run_ours(args):
                    "parallelism": "replicas only" if world > 1 else "1 gpu"},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": int(launches),
+        "per_row_advance": {"value": async_committed / (async_ms * 1e-3), "unit": UNIT,
+                            "ms_per_step": async_ms / len(async_stats),
+                            "denoise_steps_per_step": sum(st.steps for st in async_stats) / len(async_stats),
+                            "note": "bs_config.async_advance = 1: rows start their next block the step after their "
+                                    "own block completes; not part of the headline value"},
         "clocks": clocks,
         "roofline": roof,
         "families": families,

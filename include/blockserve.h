@@ -53,7 +53,7 @@ typedef struct {
   /* model: pre-norm bidirectional transformer, RMSNorm, rotate-half RoPE, GQA, SwiGLU, no biases */
   int n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ffn, vocab, mask_id;
   float rms_eps, rope_theta;
-  /* method (Section 2.1, 2.4): block length L (<= 32), confidence threshold tau,
+  /* method (Section 2.1, 2.4): block length L (<= 64), confidence threshold tau,
      token budget beta of Eq. 1 (<= 0: unlimited), fixed batch cap */
   int block_len;
   float tau;
@@ -193,7 +193,8 @@ const char* bs_last_error(const bs_engine* e); /* NULL engine: error of the last
 /* ---- parity hooks (not on the timed path) ------------------------------ */
 enum {
   BS_DBG_HEADER = 0,   /* int32[32]: n_active, M, M_m, all_done, n_committed_step, n_evicted, n_admitted, ... */
-  BS_DBG_ROW_SLOT = 1, BS_DBG_ROW_MASK = 2, BS_DBG_ROW_S = 3, BS_DBG_ROW_KV_BASE = 4, /* int32[n_active] */
+  BS_DBG_ROW_SLOT = 1, BS_DBG_ROW_S = 3, BS_DBG_ROW_KV_BASE = 4, /* int32[n_active] */
+  BS_DBG_ROW_MASK = 2, /* uint64[n_active]: bit j set = block position j still masked */
   BS_DBG_CU_Q = 5,     /* int32[n_active + 1]  (indices of the step about to run) */
   BS_DBG_TOK_ROW = 6, BS_DBG_TOK_POS = 7, BS_DBG_TOK_KV = 8,   /* int32[M]; filled by the last bs_denoise_step */
   BS_DBG_LM_TOK = 9, BS_DBG_LM_ROW = 10, BS_DBG_LM_SLOT = 11,  /* int32[M_m] of the step about to run */
@@ -208,11 +209,11 @@ enum {
 int bs_debug_read(bs_engine* e, int what, int arg0, int arg1, void* host_buf, size_t cap, size_t* n);
 
 /* Dictated commit (debugging): for the active row `row` (batch order), every block position j with bit j of
- * mask_bits set and still masked takes tokens[j] (host array indexed by block position; entries of other positions
+ * mask_bits set and still masked takes tokens[j] (host array of 64 ints indexed by block position; entries of other positions
  * are not read) and counts as committed.  The row's step counter does not move, so a row still waiting for the
  * refresh step of its block (Section 2.5) gets it; the index of the pending step is rebuilt.  The paper has no
  * counterpart.  Errors: BS_E_ARG (row not active, bit beyond L, token id out of range or the mask id). */
-int bs_debug_force_commit(bs_engine* e, int row, unsigned mask_bits, const int* tokens);
+int bs_debug_force_commit(bs_engine* e, int row, unsigned long long mask_bits, const int* tokens);
 
 /* Snapshot / restore of the engine state between block cycles (host buffers).  Because the block KV cache is rebuilt
  * from the tokens at the first step of every block (Section 2.5, refresh), the state between cycles is the token rows

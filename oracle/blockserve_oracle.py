@@ -36,7 +36,9 @@ Readings taken where the paper is silent (each is listed in the design notes):
     RoPE, GQA, SwiGLU, no biases), logits = alpha_i * norm_f(x) @ W_lm^T;
   * the cache of a request is rebuilt by a full-row forward at the first step
     of every block; later steps of the block forward only the block's tokens,
-    rewrite their K/V in place and attend over the cached prefix and suffix;
+    rewrite their K/V in place and attend over the cached prefix and suffix
+    (``refresh_at_admission_only`` is an ablation variant: only the first step
+    after admission is such a forward, the other "frozen prefix" reading);
   * commit rule: strictly conf > tau, plus always the masked position of
     highest confidence (lowest position on ties); argmax over the vocabulary
     takes the lowest id on ties and never the mask id;
@@ -235,6 +237,8 @@ class ReqState:
     committed: int = 0                 # tokens committed by the engine
     steps: int = 0
     admit_order: int = 0
+    needs_refresh: bool = True         # the block's first step forwards the whole row (rebuilds the cache)
+    refreshes: int = 0                 # whole-row forwards this request has had
 
     def n_blocks(self, L: int) -> int:
         return -(-self.g // L)         # K_i = ceil(g_i / L), Section 2.1
@@ -336,11 +340,13 @@ def denoise_step(model: Model, r: ReqState, L: int, tau: float, suffix_mode: int
     positions; they never change what the oracle *computes* and reports."""
     lo, hi = r.block_range(L)
     vis = r.vis(L, suffix_mode)
-    qpos = np.arange(0, vis) if r.s == 0 else np.arange(lo, hi)
+    refresh = r.s == 0 and r.needs_refresh
+    r.refreshes += int(refresh)
+    qpos = np.arange(0, vis) if refresh else np.arange(lo, hi)
     x = forward_queries(model, r, qpos, vis)
     slots = np.array([j for j in range(hi - lo) if (r.mask >> j) & 1], dtype=np.int64)
     positions = lo + slots
-    rows = positions if r.s == 0 else slots
+    rows = positions if refresh else slots
     logits = lm_logits(model, x[rows], r.alpha)
     tok, conf = confidence(logits, model.mask_id)
     z = np.array(logits, copy=True)
@@ -399,8 +405,11 @@ class Scheduler:
 
     def __init__(self, L: int, token_budget: int, max_batch: int, kv_capacity: int,
                  sort_queue: bool = True, eos_id: Optional[int] = None, static_groups: bool = False,
-                 async_advance: bool = False):
+                 async_advance: bool = False, refresh_at_admission_only: bool = False):
         self.L, self.beta, self.max_batch, self.kv_capacity = L, token_budget, max_batch, kv_capacity
+        # ablation variant: the cache is rebuilt once, by the first step after admission; later blocks begin with a
+        # cached block step (prefix and suffix K/V stay as earlier steps left them)
+        self.refresh_at_admission_only = bool(refresh_at_admission_only)
         self.sort_queue = sort_queue
         self.static_groups = bool(static_groups)     # comparison policy of Section 3.1: fixed groups, no refill
         self.async_advance = bool(async_advance)     # per-row block advance after every step (Section 2.3 relaxed)
@@ -456,6 +465,7 @@ class Scheduler:
             else:
                 survivors.append(r)
                 started.append(r)
+                r.needs_refresh = not self.refresh_at_admission_only
         self.active = survivors
         admitted = []
         # static groups: the next group starts only when every request of the current one has finished
@@ -472,6 +482,7 @@ class Scheduler:
             self.pending.pop(0)
             self.active.append(c)
             started.append(c)
+            c.needs_refresh = True
             admitted.append(c.req_id)
         for r in started:
             start_block_state(r, L)
@@ -505,7 +516,7 @@ def build_indices(active: Sequence[ReqState], L: int, suffix_mode: int = SUFFIX_
         lo, hi = r.block_range(L)
         if r.mask == 0:
             qpos = range(0)
-        elif r.s == 0:
+        elif r.s == 0 and r.needs_refresh:
             qpos = range(0, r.vis(L, suffix_mode))
         else:
             qpos = range(lo, hi)
@@ -534,12 +545,12 @@ class Engine:
     def __init__(self, model: Model, L: int, tau: float, token_budget: int, max_batch: int,
                  kv_capacity: int, suffix_mode: int = SUFFIX_FULL, sort_queue: bool = True,
                  steps_per_block: Optional[int] = None, eos_id: Optional[int] = None, static_groups: bool = False,
-                 async_advance: bool = False):
+                 async_advance: bool = False, refresh_at_admission_only: bool = False):
         self.model, self.L, self.tau, self.suffix_mode = model, L, tau, suffix_mode
         self.steps_per_block = steps_per_block
         self.async_advance = bool(async_advance)
         self.sched = Scheduler(L, token_budget, max_batch, kv_capacity, sort_queue, eos_id, static_groups,
-                               async_advance)
+                               async_advance, refresh_at_admission_only)
         self.by_id: Dict[int, ReqState] = {}
         self.total_committed = 0
         self.total_steps = 0

@@ -92,7 +92,7 @@ def lib() -> C.CDLL:
         L.bs_last_error.restype = C.c_char_p
         L.bs_debug_read.argtypes = [vp, i, i, i, vp, C.c_size_t, C.POINTER(C.c_size_t)]
         L.bs_debug_inject_timeout.argtypes = [vp]
-        L.bs_debug_force_commit.argtypes = [vp, i, C.c_uint, vp]
+        L.bs_debug_force_commit.argtypes = [vp, i, C.c_ulonglong, vp]
         L.bs_debug_snapshot.argtypes = [vp, vp, C.c_size_t, C.POINTER(C.c_size_t)]
         L.bs_debug_restore.argtypes = [vp, vp, C.c_size_t]
         L.bs_op_gemm.argtypes = [vp, i, vp, vp, vp, i, i, i, i, i, vp, vp, C.c_size_t, vp, vp]
@@ -234,7 +234,7 @@ class Engine:
 
     def force_commit(self, row: int, positions: Dict[int, int]) -> None:
         """Commit block position -> token for the given active row (debugging aid)."""
-        toks = np.zeros(32, dtype=np.int32)
+        toks = np.zeros(64, dtype=np.int32)
         bits = 0
         for j, t in positions.items():
             toks[j] = t
@@ -383,24 +383,32 @@ def op_attention(qkv, kcache, vcache, cu_q, kv_base, vis, hq, hkv, dh, scratch: 
     return out
 
 
+def lm_head_confidence_buffers(M: int, V: int, device) -> dict:
+    """Buffers of op_lm_head_confidence, for callers that launch repeatedly."""
+    nbytes = lib().bs_op_lm_head_confidence_scratch_bytes(M, V)
+    return dict(scratch=torch.empty(max(nbytes, 256), dtype=torch.uint8, device=device), nbytes=nbytes,
+                tok=torch.empty(M, dtype=torch.int32, device=device),
+                conf=torch.empty(M, dtype=torch.float32, device=device),
+                flag=torch.zeros(1, dtype=torch.int32, device=device))
+
+
 def op_lm_head_confidence(hf: torch.Tensor, W: torch.Tensor, row_scale: torch.Tensor, mask_id: int,
-                          want_logits: bool = False):
-    """LM head with the confidence pass in its epilogue: (tok int32 [M], conf fp32 [M], logits fp32 [M, V] or None)."""
+                          want_logits: bool = False, buffers: Optional[dict] = None):
+    """LM head with the confidence pass in its epilogue: (tok int32 [M], conf fp32 [M], logits fp32 [M, V] or None).
+    With `buffers` (from lm_head_confidence_buffers) nothing is allocated and the stream is not synchronised."""
     M, K = hf.shape
     V = W.shape[0]
-    nbytes = lib().bs_op_lm_head_confidence_scratch_bytes(M, V)
-    scratch = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=hf.device)
-    tok = torch.empty(M, dtype=torch.int32, device=hf.device)
-    conf = torch.empty(M, dtype=torch.float32, device=hf.device)
+    b = buffers or lm_head_confidence_buffers(M, V, hf.device)
     logits = torch.empty(M, V, dtype=torch.float32, device=hf.device) if want_logits else None
-    flag = torch.zeros(1, dtype=torch.int32, device=hf.device)
     _check_op(lib().bs_op_lm_head_confidence(hf.data_ptr(), hf.stride(0), W.data_ptr(), M, V, K, row_scale.data_ptr(),
-                                             mask_id, scratch.data_ptr(), nbytes, tok.data_ptr(), conf.data_ptr(),
-                                             _ptr(logits), flag.data_ptr(), _stream()), "bs_op_lm_head_confidence")
-    torch.cuda.current_stream().synchronize()
-    if int(flag.item()):
-        raise BlockServeError(BS_E_TIMEOUT, "a bounded device-side wait ran out")
-    return tok, conf, logits
+                                             mask_id, b["scratch"].data_ptr(), b["nbytes"], b["tok"].data_ptr(),
+                                             b["conf"].data_ptr(), _ptr(logits), b["flag"].data_ptr(), _stream()),
+              "bs_op_lm_head_confidence")
+    if buffers is None:
+        torch.cuda.current_stream().synchronize()
+        if int(b["flag"].item()):
+            raise BlockServeError(BS_E_TIMEOUT, "a bounded device-side wait ran out")
+    return b["tok"], b["conf"], logits
 
 
 def op_confidence(logits: torch.Tensor, mask_id: int):

@@ -15,10 +15,11 @@
 //               of the scores buffer it came from (one tcgen05.st per row, no shared-memory round trip);
 //               the output accumulates in TMEM over all key tiles and is rescaled lazily (only when a row's
 //               maximum has grown by more than 2^8), the running sum follows the same scale
-// Two instantiations: NQ = 2 (a work item's two Q tiles share every K/V tile the CTA loads; one CTA per SM) for
-// steps with many work items, and NQ = 1 (one Q tile, half the tensor memory, a two-stage K/V ring: two CTAs per SM
-// hide each other's dependent chains) for steps with few.  A launch may also cut every row's keys into chunks
-// (grid z): each chunk leaves an unnormalised fp32 partial (output, scale, sum) and a small kernel merges them.
+// Instantiations: two Q tiles per CTA (a work item's Q tiles share every K/V tile the CTA loads) for steps with many
+// work items; one Q tile per CTA (half the tensor memory) for steps with few, with a four-stage K/V ring and one
+// CTA per SM, or a two-stage ring and two CTAs per SM.  A launch with few work items may also cut every row's keys
+// into chunks (grid z): each chunk leaves an unnormalised fp32 partial (output, scale, sum) and a small kernel
+// merges them.
 // Every wait is bounded; on a timeout the flag is raised, all roles drain, TMEM is freed.
 #include <math.h>
 #include <stdlib.h>
@@ -130,14 +131,13 @@ struct AttnTcParams {
 constexpr int KT = 64;                                   // keys per tile
 constexpr int kKvHalf = KT * 128;                        // KT rows x 64 bf16
 constexpr int kStageBytes = 4 * kKvHalf;                 // K halves, V halves
-__host__ __device__ constexpr int stages_for(int nq) { return nq == 2 ? 4 : 2; }
-__host__ __device__ constexpr int smem_for(int nq) { return nq * kQBytes + stages_for(nq) * kStageBytes + 1024; }
+__host__ __device__ constexpr int smem_for(int nq, int stages) { return nq * kQBytes + stages * kStageBytes + 1024; }
 
-template <int NQ>
-__global__ void __launch_bounds__(threads_for(NQ), NQ == 2 ? 1 : 2)
+template <int NQ, int STAGES>
+__global__ void __launch_bounds__(threads_for(NQ), smem_for(NQ, STAGES) <= 112 * 1024 ? 2 : 1)
 k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                const __grid_constant__ CUtensorMap map_v, const AttnTcParams p) {
-  constexpr int kStages = stages_for(NQ);
+  constexpr int kStages = STAGES;
   constexpr unsigned kTmemCols = NQ == 2 ? 512u : 256u;
   // Barrier slots
   enum { B_QFULL = 0, B_KVFULL = 1, B_KVEMPTY = B_KVFULL + kStages, B_SFULL = B_KVEMPTY + kStages,   // [tile][2]
@@ -520,8 +520,9 @@ cudaError_t launch_attention_tc(const bf16* qkv, const bf16* kc, const bf16* vc,
     std::lock_guard<std::mutex> lock(g_mutex);
     int dev = 0, n = 0;
     cudaGetDevice(&dev);
-    if (cudaFuncSetAttribute(k_attention_tc<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_for(1)) != cudaSuccess ||
-        cudaFuncSetAttribute(k_attention_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_for(2)) != cudaSuccess ||
+    if (cudaFuncSetAttribute(k_attention_tc<1, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_for(1, 2)) != cudaSuccess ||
+        cudaFuncSetAttribute(k_attention_tc<1, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_for(1, 4)) != cudaSuccess ||
+        cudaFuncSetAttribute(k_attention_tc<2, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_for(2, 4)) != cudaSuccess ||
         cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1)
       return cudaErrorInvalidDevice;
     *sms = n;
@@ -540,28 +541,36 @@ cudaError_t launch_attention_tc(const bf16* qkv, const bf16* kc, const bf16* vc,
   // its own small CTA, two of them share an SM, and the rows' keys are cut into chunks until about two CTAs per SM
   // are in flight.  Many work items (a refresh step): the two Q tiles of an item share each K/V tile they load.
   static const int env_chunks = getenv("BS_ATTN_TC_CHUNKS") ? atoi(getenv("BS_ATTN_TC_CHUNKS")) : 0;
-  static const int env_nq = getenv("BS_ATTN_TC_NQ") ? atoi(getenv("BS_ATTN_TC_NQ")) : 0;
+  static const int env_plan = getenv("BS_ATTN_TC_PLAN") ? atoi(getenv("BS_ATTN_TC_PLAN")) : 0;   // 1, 2, 3 below
   const long long items = (long long)n_tiles * hkv;
-  const bool small = env_nq ? env_nq == 1 : items < 2 * (long long)num_sms;
+  // plan 1: two Q tiles per CTA (refresh steps); plan 2: one Q tile per CTA, four-stage ring, one CTA per SM;
+  // plan 3: one Q tile per CTA, two-stage ring, two CTAs per SM
+  int plan = items < num_sms ? 2 : 1;
+  if (env_plan >= 1 && env_plan <= 3) plan = env_plan;
   int chunks = 1;
-  if (small && scratch && max_vis > 0) {
+  if (plan != 1 && scratch && max_vis > 0) {
     const long long ctas = 2 * items;
     const int key_tiles = (max_vis + KT - 1) / KT;
-    chunks = (int)((2ll * num_sms + ctas / 2) / ctas);              // about two CTAs per SM
-    chunks = std::max(1, std::min(chunks, key_tiles / 3));          // at least three key tiles per chunk
+    chunks = (int)((plan == 3 ? 2ll : 1ll) * num_sms / ctas);        // fill the SMs (twice over for plan 3), no more
+    chunks = std::max(1, std::min(chunks, key_tiles / 6));          // at least six key tiles per chunk
     while (chunks > 1 && (size_t)chunks * M * ((size_t)hq * DH + 2 * hq) > scratch_floats) --chunks;
   }
-  if (env_chunks >= 1 && scratch && (size_t)env_chunks * M * ((size_t)hq * DH + 2 * hq) <= scratch_floats)
+  if (env_chunks >= 1 && plan != 1 && scratch &&
+      (size_t)env_chunks * M * ((size_t)hq * DH + 2 * hq) <= scratch_floats)
     chunks = env_chunks;
   p.chunks = chunks;
   p.part_o = scratch;
   p.part_ml = reinterpret_cast<float2*>(scratch + (size_t)chunks * M * hq * DH);
   cudaError_t r;
-  if (small)
-    r = launch_pdl(k_attention_tc<1>, dim3(2 * n_tiles, hkv, chunks), dim3(threads_for(1)), (size_t)smem_for(1), s, mq,
-                   mk, mv, p);
+  if (plan == 3)
+    r = launch_pdl(k_attention_tc<1, 2>, dim3(2 * n_tiles, hkv, chunks), dim3(threads_for(1)), (size_t)smem_for(1, 2),
+                   s, mq, mk, mv, p);
+  else if (plan == 2)
+    r = launch_pdl(k_attention_tc<1, 4>, dim3(2 * n_tiles, hkv, chunks), dim3(threads_for(1)), (size_t)smem_for(1, 4),
+                   s, mq, mk, mv, p);
   else
-    r = launch_pdl(k_attention_tc<2>, dim3(n_tiles, hkv, 1), dim3(threads_for(2)), (size_t)smem_for(2), s, mq, mk, mv, p);
+    r = launch_pdl(k_attention_tc<2, 4>, dim3(n_tiles, hkv, 1), dim3(threads_for(2)), (size_t)smem_for(2, 4), s, mq, mk,
+                   mv, p);
   if (r != cudaSuccess || chunks == 1) return r;
   return launch_pdl(k_attention_tc_combine, dim3(M), dim3(256), 0, s, (const float*)p.part_o,
                     (const float2*)p.part_ml, chunks, M, out, hq);

@@ -34,6 +34,8 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
   return cudaLaunchKernelEx(&cfg, kernel, KArgs(std::forward<Args>(args))...);
 }
 
+typedef unsigned long long MaskWord;      // one bit per position of a block
+constexpr int kMaxBlockLen = 64;
 constexpr int kHdrInts = 32;
 // header words (device int32[kHdrInts], mirrored to pinned host memory once per step)
 enum Hdr {
@@ -56,7 +58,7 @@ struct DevState {
   long long beta, kv_capacity;
   float tau;
   int* hdr;             // [kHdrInts] followed directly by row_mask[max_batch]
-  unsigned* row_mask;   // bit j set <=> block position j still masked
+  MaskWord* row_mask;   // bit j set <=> block position j still masked (L <= 64)
   int* req_p; int* req_g; int* req_b; int* req_state; int* req_committed; float* req_alpha;
   int* tokens;          // [max_requests, max_row_tokens]
   int* queue;           // pending slots in admission order
@@ -74,8 +76,8 @@ struct DevState {
 cudaError_t launch_sched(const DevState& st, cudaStream_t s);
 cudaError_t launch_commit_index(const DevState& st, cudaStream_t s);
 cudaError_t launch_fill_tokens(const DevState& st, int parity, int M, cudaStream_t s);
-// tokens32[j] is read for every bit j of `bits`; positions the row has already committed are skipped.
-cudaError_t launch_force_commit(const DevState& st, int row, unsigned bits, const int* tokens32, cudaStream_t s);
+// tokens[j] (kMaxBlockLen entries) is read for every bit j of `bits`; positions the row has already committed are skipped.
+cudaError_t launch_force_commit(const DevState& st, int row, MaskWord bits, const int* tokens, cudaStream_t s);
 
 cudaError_t launch_embed(const DevState& st, const bf16* embed, float* x, int M, int d, cudaStream_t s);
 cudaError_t launch_rmsnorm(const float* x, const int* idx, const bf16* w, bf16* y, int M, int d, float eps,

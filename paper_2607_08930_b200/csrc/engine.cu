@@ -79,8 +79,8 @@ size_t carve_state(const bs_config& c, void* base, DevState* out) {
   memset(&st, 0, sizeof(st));
   const size_t R = c.max_requests, B = c.max_batch, T = (size_t)c.kv_capacity_tokens, mm = B * c.block_len;
   // header and row masks are contiguous: one copy mirrors both to the host
-  st.hdr = cv.take<int>(kHdrInts + B);
-  st.row_mask = base ? reinterpret_cast<unsigned*>(st.hdr + kHdrInts) : nullptr;
+  st.hdr = cv.take<int>(kHdrInts + 2 * B);      // 64-bit mask words: two ints per row
+  st.row_mask = base ? reinterpret_cast<MaskWord*>(st.hdr + kHdrInts) : nullptr;
   st.req_p = cv.take<int>(R); st.req_g = cv.take<int>(R); st.req_b = cv.take<int>(R);
   st.req_state = cv.take<int>(R); st.req_committed = cv.take<int>(R); st.req_alpha = cv.take<float>(R);
   st.tokens = cv.take<int>(R * c.max_row_tokens);
@@ -107,7 +107,7 @@ const char* check_config(const bs_config& c) {
   if (c.d_ffn < 8 || c.d_ffn % 8) return "d_ffn must be a positive multiple of 8";
   if (c.vocab < 2 || c.vocab % 2) return "vocab must be even";
   if (c.mask_id < 0 || c.mask_id >= c.vocab) return "mask_id outside the vocabulary";
-  if (c.block_len < 1 || c.block_len > 32) return "block_len must be in [1, 32]";
+  if (c.block_len < 1 || c.block_len > kMaxBlockLen) return "block_len must be in [1, 64]";
   if (c.max_batch < 1 || c.max_batch > 1024) return "max_batch must be in [1, 1024]";
   if (c.max_requests < 1 || c.max_row_tokens < 2) return "max_requests / max_row_tokens too small";
   if (c.kv_capacity_tokens < c.max_row_tokens) return "kv_capacity_tokens smaller than one row";
@@ -241,8 +241,8 @@ int sync_header(bs_engine* e) {
 }
 
 int post_header(bs_engine* e, bool from_step = false) {
-  CU(e, cudaMemcpyAsync(e->pinned, e->st.hdr, (kHdrInts + e->cfg.max_batch) * sizeof(int), cudaMemcpyDeviceToHost,
-                        e->stream));
+  CU(e, cudaMemcpyAsync(e->pinned, e->st.hdr, (kHdrInts + 2 * e->cfg.max_batch) * sizeof(int),
+                        cudaMemcpyDeviceToHost, e->stream));
   CU(e, cudaEventRecord(e->ev, e->stream));
   e->hdr_pending = true;
   e->hdr_from_step = from_step;
@@ -355,7 +355,7 @@ int bs_init_model(const bs_config* cfg, const bs_weights* w, void* kv, void* wor
   // probability of exactly zero, and 0 * NaN would poison the row)
   if (r == cudaSuccess)
     r = cudaMemsetAsync(kv, 0, (size_t)cfg->n_layers * 2 * e->kv_half * sizeof(bf16), e->stream);
-  if (r == cudaSuccess) r = cudaHostAlloc((void**)&e->pinned, (kHdrInts + cfg->max_batch) * sizeof(int), cudaHostAllocDefault);
+  if (r == cudaSuccess) r = cudaHostAlloc((void**)&e->pinned, (kHdrInts + 2 * cfg->max_batch) * sizeof(int), cudaHostAllocDefault);
   if (r == cudaSuccess) r = cudaEventCreateWithFlags(&e->ev, cudaEventDisableTiming);
   if (r == cudaSuccess) {
     std::vector<float> tab((size_t)cfg->max_row_tokens * cfg->head_dim);
@@ -576,8 +576,8 @@ int bs_block_done(bs_engine* e, int* all_done, unsigned char* per_row_done) {
   if (int rc = sync_header(e)) return rc;
   if (all_done) *all_done = e->hdr[H_ALL_DONE] ? 1 : 0;
   if (per_row_done) {
-    const unsigned* masks = reinterpret_cast<const unsigned*>(e->pinned + kHdrInts);
-    for (int i = 0; i < e->cfg.max_batch; ++i) per_row_done[i] = (i < e->hdr[H_N_ACTIVE]) ? (masks[i] == 0u) : 1;
+    const MaskWord* masks = reinterpret_cast<const MaskWord*>(e->pinned + kHdrInts);
+    for (int i = 0; i < e->cfg.max_batch; ++i) per_row_done[i] = (i < e->hdr[H_N_ACTIVE]) ? (masks[i] == 0ull) : 1;
   }
   return BS_OK;
 }
@@ -658,7 +658,7 @@ int bs_debug_read(bs_engine* e, int what, int arg0, int arg1, void* host_buf, si
   switch (what) {
     case BS_DBG_HEADER: src = st.hdr; bytes = kHdrInts * 4; break;
     case BS_DBG_ROW_SLOT: src = st.row_slot; bytes = n * 4; break;
-    case BS_DBG_ROW_MASK: src = st.row_mask; bytes = n * 4; break;
+    case BS_DBG_ROW_MASK: src = st.row_mask; bytes = n * sizeof(MaskWord); break;
     case BS_DBG_ROW_S: src = st.row_s; bytes = n * 4; break;
     case BS_DBG_ROW_KV_BASE: src = st.row_kv_base; bytes = n * 4; break;
     case BS_DBG_CU_Q: src = st.cu_q[par]; bytes = (n + 1) * 4; break;
@@ -712,20 +712,20 @@ int bs_debug_read(bs_engine* e, int what, int arg0, int arg1, void* host_buf, si
   return BS_OK;
 }
 
-int bs_debug_force_commit(bs_engine* e, int row, unsigned mask_bits, const int* tokens) {
+int bs_debug_force_commit(bs_engine* e, int row, unsigned long long mask_bits, const int* tokens) {
   if (!e || !tokens) return BS_E_ARG;
   if (int rc = sync_header(e)) return rc;
   if (row < 0 || row >= e->hdr[H_N_ACTIVE]) return fail(e, BS_E_ARG, "row is not an active row");
   const int L = e->cfg.block_len;
-  if (L < 32 && (mask_bits >> L) != 0u) return fail(e, BS_E_ARG, "bit beyond the block length");
-  int t32[32] = {0};
-  for (int j = 0; j < 32; ++j)
-    if ((mask_bits >> j) & 1u) {
+  if (L < kMaxBlockLen && (mask_bits >> L) != 0ull) return fail(e, BS_E_ARG, "bit beyond the block length");
+  int toks[kMaxBlockLen] = {0};
+  for (int j = 0; j < kMaxBlockLen; ++j)
+    if ((mask_bits >> j) & 1ull) {
       if (tokens[j] < 0 || tokens[j] >= e->cfg.vocab || tokens[j] == e->cfg.mask_id)
         return fail(e, BS_E_ARG, "token id out of range");
-      t32[j] = tokens[j];
+      toks[j] = tokens[j];
     }
-  KL(e, launch_force_commit(e->st, row, mask_bits, t32, e->stream));
+  KL(e, launch_force_commit(e->st, row, mask_bits, toks, e->stream));
   return post_header(e);
 }
 

@@ -69,17 +69,17 @@ __device__ void build_index(const DevState& st, int parity, int n, int* smi) {
     const int slot = st.row_slot[i];
     const int p = st.req_p[slot], g = st.req_g[slot], b = st.req_b[slot];
     const int s = st.row_s[i];
-    const unsigned mask = st.row_mask[i];
+    const MaskWord mask = st.row_mask[i];
     const int lo = p + b * st.L;
     const int hi = min(lo + st.L, p + g);
     vis = st.suffix_mode == 0 ? p + g : hi;
     st.row_vis[i] = vis;
-    if (mask != 0u) {
+    if (mask != 0ull) {
       nq = (s == 0) ? vis : hi - lo;
       unfinished = 1;
       refresh = (s == 0);
     }
-    nm = __popc(mask);
+    nm = __popcll(mask);
   }
   int tot_q, tot_m, tot_t, tot_u, tot_r;
   const int eq = block_excl_scan(nq, &tot_q, smi);
@@ -114,16 +114,19 @@ __device__ void build_index(const DevState& st, int parity, int n, int* smi) {
   // still-masked block positions, row order then position order
   const int lane = threadIdx.x & 31;
   for (int r = threadIdx.x >> 5; r < n; r += kSchedThreads / 32) {
-    const unsigned mask = st.row_mask[r];
-    if (mask == 0u) continue;
-    if ((mask >> lane) & 1u) {
-      const int slot = st.row_slot[r];
-      const int lo = st.req_p[slot] + st.req_b[slot] * st.L;
-      const int k = st.lm_base[parity][r] + __popc(mask & ((1u << lane) - 1u));
-      st.lm_tok[parity][k] = st.cu_q[parity][r] + (st.row_s[r] == 0 ? lo + lane : lane);
-      st.lm_row[parity][k] = r;
-      st.lm_slot[parity][k] = lane;
-      st.lm_scale[parity][k] = st.req_alpha[slot];
+    const MaskWord mask = st.row_mask[r];
+    if (mask == 0ull) continue;
+#pragma unroll
+    for (int j = lane; j < kMaxBlockLen; j += 32) {     // a lane looks after block positions lane and lane + 32
+      if ((mask >> j) & 1ull) {
+        const int slot = st.row_slot[r];
+        const int lo = st.req_p[slot] + st.req_b[slot] * st.L;
+        const int k = st.lm_base[parity][r] + __popcll(mask & ((1ull << j) - 1ull));
+        st.lm_tok[parity][k] = st.cu_q[parity][r] + (st.row_s[r] == 0 ? lo + j : j);
+        st.lm_row[parity][k] = r;
+        st.lm_slot[parity][k] = j;
+        st.lm_scale[parity][k] = st.req_alpha[slot];
+      }
     }
   }
 }
@@ -145,13 +148,13 @@ __device__ void sched_body(const DevState& st, bool only_done) {
 
   // ---- advance, evict finished rows (b_i >= K_i or CheckEOS), compact (order preserved) ----
   int keep = 0, slot = -1, kvb = 0, srow = 0;
-  unsigned mask = 0u;
+  MaskWord mask = 0ull;
   if (i < n0) {
     slot = st.row_slot[i];
     kvb = st.row_kv_base[i];
     mask = st.row_mask[i];
     srow = st.row_s[i];
-    if (only_done && mask != 0u) {
+    if (only_done && mask != 0ull) {
       keep = 1;                                            // mid-block: nothing changes for this row
     } else {
       const int b = st.req_b[slot] + 1;
@@ -242,7 +245,7 @@ __device__ void sched_body(const DevState& st, bool only_done) {
     const int sl = st.row_slot[i];
     const int lo = st.req_p[sl] + st.req_b[sl] * L;
     const int len = min(L, st.req_p[sl] + st.req_g[sl] - lo);
-    st.row_mask[i] = len >= 32 ? 0xffffffffu : ((1u << len) - 1u);
+    st.row_mask[i] = len >= 64 ? ~0ull : ((1ull << len) - 1ull);
     st.row_s[i] = 0;
   }
   if (i == 0) {
@@ -277,24 +280,35 @@ __global__ void __launch_bounds__(kSchedThreads) k_commit_index(DevState st) {
   __syncthreads();
   for (int r = threadIdx.x >> 5; r < n; r += kSchedThreads / 32) {
     const int base = st.lm_base[parity][r];
-    const int nm = st.lm_base[parity][r + 1] - base;
+    const int nm = st.lm_base[parity][r + 1] - base;      // still-masked positions of the row: at most L <= 64
     if (nm == 0) continue;
-    float conf = -1.0f;
-    int tok = 0, bit = 0;
-    if (lane < nm) {
-      // last stage of the confidence pass: the slice partials of this masked position -> token id and confidence
-      merge_conf_slices(st.slice_ms, st.slice_am, st.lm_base[parity][n], base + lane, &tok, &conf);
-      st.out_conf[parity][base + lane] = conf;
-      st.out_tok[parity][base + lane] = tok;
-      bit = st.lm_slot[parity][base + lane];
+    // a lane looks after list entries lane and lane + 32
+    float conf[2] = {-1.0f, -1.0f};
+    int tok[2] = {0, 0}, bit[2] = {0, 0};
+    bool picked[2] = {false, false};
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const int k = lane + 32 * h;
+      if (k < nm) {
+        // last stage of the confidence pass: the slice partials of this masked position -> token id and confidence
+        merge_conf_slices(st.slice_ms, st.slice_am, st.lm_base[parity][n], base + k, &tok[h], &conf[h]);
+        st.out_conf[parity][base + k] = conf[h];
+        st.out_tok[parity][base + k] = tok[h];
+        bit[h] = st.lm_slot[parity][base + k];
+      }
     }
     // transfer quota of this step (Section 2.5): the block's L masked tokens spread uniformly over S steps
     const int s_in_block = st.row_s[r];
     const int quota = s_in_block >= st.S ? 1 : st.L / st.S + (s_in_block < st.L % st.S ? 1 : 0);
-    bool picked = false;
     for (int it = 0; it < quota; ++it) {          // warp-uniform trip count
-      float bc = (lane < nm && !picked) ? conf : -2.0f;
-      int bj = lane;
+      // this lane's better unpicked entry (the lower entry on ties), then the warp's
+      float bc = -2.0f;
+      int bj = 64;
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int k = lane + 32 * h;
+        if (k < nm && !picked[h] && conf[h] > bc) { bc = conf[h]; bj = k; }
+      }
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) {
         const float oc = __shfl_xor_sync(0xffffffffu, bc, o);
@@ -302,21 +316,29 @@ __global__ void __launch_bounds__(kSchedThreads) k_commit_index(DevState st) {
         if (oc > bc || (oc == bc && oj < bj)) { bc = oc; bj = oj; }
       }
       if (bc < -1.5f) break;                      // nothing left to pick (warp-uniform)
-      if (lane == bj) picked = true;
+      if ((bj & 31) == lane) picked[bj >> 5] = true;
     }
-    const bool sel = lane < nm && (conf > st.tau || picked);
     const int slot = st.row_slot[r];
-    if (sel) {
-      const int lo = st.req_p[slot] + st.req_b[slot] * st.L;
-      st.tokens[(size_t)slot * st.max_row_tokens + lo + bit] = tok;
+    unsigned lo_bits = 0u, hi_bits = 0u;
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const int k = lane + 32 * h;
+      const bool sel = k < nm && (conf[h] > st.tau || picked[h]);
+      if (sel) {
+        const int lo = st.req_p[slot] + st.req_b[slot] * st.L;
+        st.tokens[(size_t)slot * st.max_row_tokens + lo + bit[h]] = tok[h];
+        if (bit[h] < 32) lo_bits |= 1u << bit[h]; else hi_bits |= 1u << (bit[h] - 32);
+      }
+      if (k < nm) st.out_commit[parity][base + k] = sel ? 1 : 0;
     }
-    if (lane < nm) st.out_commit[parity][base + lane] = sel ? 1 : 0;
-    const unsigned bits = __reduce_or_sync(0xffffffffu, sel ? (1u << bit) : 0u);
+    lo_bits = __reduce_or_sync(0xffffffffu, lo_bits);
+    hi_bits = __reduce_or_sync(0xffffffffu, hi_bits);
     if (lane == 0) {
+      const MaskWord bits = ((MaskWord)hi_bits << 32) | lo_bits;
       st.row_mask[r] &= ~bits;
       st.row_s[r] += 1;
-      st.req_committed[slot] += __popc(bits);
-      atomicAdd(&s_count, __popc(bits));
+      st.req_committed[slot] += __popcll(bits);
+      atomicAdd(&s_count, __popcll(bits));
     }
   }
   __syncthreads();
@@ -336,23 +358,23 @@ __global__ void __launch_bounds__(kSchedThreads) k_commit_index(DevState st) {
 // Debug aid: commits the given block positions of one active row with the given tokens, as if a step had chosen
 // them, and rebuilds the index of the pending step.  The row's step counter is left alone, so a row that has not
 // had its refresh step yet still gets one.
-struct ForcedTokens { int t[32]; };
-__global__ void __launch_bounds__(kSchedThreads) k_force_commit(DevState st, int row, unsigned bits, ForcedTokens ft) {
+struct ForcedTokens { int t[kMaxBlockLen]; };
+__global__ void __launch_bounds__(kSchedThreads) k_force_commit(DevState st, int row, MaskWord bits, ForcedTokens ft) {
   __shared__ int smi[33];
   const int parity = st.hdr[H_PARITY];
   const int n = st.hdr[H_N_ACTIVE];
   if (row < n) {
-    const unsigned take = bits & st.row_mask[row];
+    const MaskWord take = bits & st.row_mask[row];
     const int slot = st.row_slot[row];
     const int lo = st.req_p[slot] + st.req_b[slot] * st.L;
-    if (threadIdx.x < 32 && ((take >> threadIdx.x) & 1u))
+    if (threadIdx.x < kMaxBlockLen && ((take >> threadIdx.x) & 1ull))
       st.tokens[(size_t)slot * st.max_row_tokens + lo + threadIdx.x] = ft.t[threadIdx.x];
     __syncthreads();
     if (threadIdx.x == 0) {
       st.row_mask[row] &= ~take;
-      st.req_committed[slot] += __popc(take);
+      st.req_committed[slot] += __popcll(take);
       unsigned long long tot = ((unsigned long long)(unsigned)st.hdr[H_TOTAL_HI] << 32) | (unsigned)st.hdr[H_TOTAL_LO];
-      tot += (unsigned long long)__popc(take);
+      tot += (unsigned long long)__popcll(take);
       st.hdr[H_TOTAL_LO] = (int)(unsigned)(tot & 0xffffffffull);
       st.hdr[H_TOTAL_HI] = (int)(unsigned)(tot >> 32);
     }
@@ -388,9 +410,9 @@ cudaError_t launch_sched(const DevState& st, cudaStream_t s) {
 cudaError_t launch_commit_index(const DevState& st, cudaStream_t s) {
   return launch_pdl(k_commit_index, dim3(1), dim3(kSchedThreads), 0, s, st);
 }
-cudaError_t launch_force_commit(const DevState& st, int row, unsigned bits, const int* tokens32, cudaStream_t s) {
+cudaError_t launch_force_commit(const DevState& st, int row, MaskWord bits, const int* tokens, cudaStream_t s) {
   ForcedTokens ft;
-  for (int i = 0; i < 32; ++i) ft.t[i] = tokens32[i];
+  for (int i = 0; i < kMaxBlockLen; ++i) ft.t[i] = tokens[i];
   k_force_commit<<<1, kSchedThreads, 0, s>>>(st, row, bits, ft);
   return cudaGetLastError();
 }

@@ -67,7 +67,7 @@ def bench_gemm(args):
     weights from HBM); the reported time is the average per launch, free of launch-gap artefacts."""
     d, hq, hkv, dh, ffn, vocab = SHAPES[args.shape]
     gemms = {"qkv": ((hq + 2 * hkv) * dh, d, 0), "o": (d, hq * dh, 1), "gate_up": (ffn, d, 3), "down": (d, ffn, 1),
-             "lm_head": (vocab, d, 2)}
+             "lm_head": (vocab, d, 2), "lm_head_conf": (vocab, d, 5)}
     scratch = torch.empty(16 << 20, dtype=torch.float32, device="cuda")
     flag = torch.zeros(1, dtype=torch.int32, device="cuda")
     for name, (N, K, mode) in gemms.items():
@@ -78,19 +78,29 @@ def bench_gemm(args):
         Ws = [(torch.randn(N, K, device="cuda") * 0.02).bfloat16() for _ in range(copies)]
         W2s = [(torch.randn(N, K, device="cuda") * 0.02).bfloat16() for _ in range(copies)] if mode == 3 else None
         for M in args.m:
-            if name == "lm_head" and M > 2048:
+            if name.startswith("lm_head") and M > 2048:
                 continue
             A = torch.randn(M, K, device="cuda").bfloat16()
-            Cd = torch.zeros(M, N, device="cuda", dtype=torch.bfloat16 if mode in (0, 3) else torch.float32)
-            rs = torch.ones(M, device="cuda") if mode == 2 else None
+            rs = torch.ones(M, device="cuda") if mode in (2, 5) else None
+            if mode == 5:      # the LM head with the confidence pass in its epilogue (GEMM + slice merge + final merge)
+                bufs = B.lm_head_confidence_buffers(M, N, "cuda")
+                flag = bufs["flag"]
 
-            def run(i):
-                B.op_gemm(A, Ws[i % copies], mode, W2=None if W2s is None else W2s[i % copies], C_out=Cd,
-                          row_scale=rs, scratch=scratch, error_flag=flag)
+                def run(i):
+                    B.op_lm_head_confidence(A, Ws[i % copies], rs, N - 1, buffers=bufs)
 
+                out_bytes = 2.0 * 12.0 * M * ((N + 31) // 32)       # group partials written, then read once
+            else:
+                Cd = torch.zeros(M, N, device="cuda", dtype=torch.bfloat16 if mode in (0, 3) else torch.float32)
+
+                def run(i):
+                    B.op_gemm(A, Ws[i % copies], mode, W2=None if W2s is None else W2s[i % copies], C_out=Cd,
+                              row_scale=rs, scratch=scratch, error_flag=flag)
+
+                out_bytes = Cd.numel() * Cd.element_size() * (2 if mode == 1 else 1)
             t = _time_graph(run, args.reps, args.iters)
             fl = 2.0 * M * N * K * nw
-            by = 2.0 * (N * K * nw + M * K) + Cd.numel() * Cd.element_size() * (2 if mode == 1 else 1)
+            by = 2.0 * (N * K * nw + M * K) + out_bytes
             print(f"gemm {name:8s} M={M:6d} N={N:6d} K={K:6d} {t * 1e6:9.1f} us {fl / t / 1e12:8.1f} TFLOP/s "
                   f"{by / t / 1e9:8.1f} GB/s  error_flag={int(flag.item())}")
 

@@ -213,7 +213,7 @@ class Lockstep:
         hdr = self.eng.debug(B.DBG_HEADER)
         assert hdr[1] == len(ix["tok_row"]) and hdr[2] == len(ix["lm_tok"]), "M / M_m differ"
         assert self.eng.debug(B.DBG_CU_Q).tolist() == ix["cu_q"].tolist()
-        assert self.eng.debug(B.DBG_ROW_MASK, np.uint32).tolist() == [r.mask for r in act]
+        assert self.eng.debug(B.DBG_ROW_MASK, np.uint64).tolist() == [r.mask for r in act]
         assert self.eng.debug(B.DBG_ROW_S).tolist() == [r.s for r in act]
         cap = max(1 << 16, 4 * len(ix["lm_tok"]) + 64)
         assert self.eng.debug(B.DBG_LM_TOK, cap=cap).tolist() == ix["lm_tok"].tolist()
@@ -270,7 +270,7 @@ class Lockstep:
         g_logits = None
         if self.track is None:
             g_logits = self.eng.debug(B.DBG_PREV_LOGITS, np.float32, cap=4 * Mm * V + 64).reshape(Mm, V)
-        g_masks = self.eng.debug(B.DBG_ROW_MASK, np.uint32)
+        g_masks = self.eng.debug(B.DBG_ROW_MASK, np.uint64)
         # with the per-row advance the step has already compacted the rows: look a row's mask word up by request id
         ids_now = self.eng.debug(B.DBG_REQ_ID_OF_ROW, np.int64).tolist() if self.async_advance else None
         tau = np.float32(self.wl.tau)
@@ -286,7 +286,7 @@ class Lockstep:
             if not self.tracked(r.req_id):
                 # untracked row: integer bookkeeping only; the commit rule is still checked on the engine's own data
                 assert (O.commit_set(gc.copy(), self.wl.tau, quota) == gs).all(), f"commit rule ({where})"
-                slots = [j for j in range(32) if (r.mask >> j) & 1]
+                slots = [j for j in range(64) if (r.mask >> j) & 1]
                 new_mask = r.mask
                 for i, j in enumerate(slots):
                     if gs[i]:

@@ -77,7 +77,7 @@ def test_tau_extremes(B, tau, expect):
         _, _, n = eng.evict_refill()
         if n == 0:
             break
-        masks = eng.debug(B.DBG_ROW_MASK, np.uint32)
+        masks = eng.debug(B.DBG_ROW_MASK, np.uint64)
         lens = [bin(int(m)).count("1") for m in masks]
         steps = 0
         while True:
@@ -425,7 +425,8 @@ def test_async_advance_config1_full_lockstep(B, suffix_mode):
     free = ls.check_free_run()
     st = ls.eng.stats()
     assert st.committed == wl.committed_target() == sum(r.committed for r in ls.ora.by_id.values())
-    assert st.row_steps == st.active_row_steps == ls.ora.sched.row_steps      # every active row works in every step
+    # every active row works in every step, and the rows' own step counts add up to the same number
+    assert st.row_steps == st.active_row_steps == sum(r.steps for r in ls.ora.by_id.values())
     for r in wl.requests:
         toks, state = ls.eng.read_tokens(r.req_id)
         assert state == B.REQ_FINISHED and (toks != wl.shape.mask_id).all()

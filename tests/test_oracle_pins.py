@@ -788,3 +788,64 @@ def test_async_advance_scheduler_invariants():
     assert not s.pending and len(s.finished) == 40
     order = sorted(range(40), key=lambda i: (s.finished[[r.req_id for r in s.finished].index(i)].p, i))
     assert admitted_all == order                 # the admitted sequence is the sorted queue, front to back
+
+
+# ------------------------------------------- refresh only at admission (ablation variant), block length 64 ---
+
+def test_refresh_at_admission_only_forwards_the_whole_row_once():
+    """The variant rebuilds a request's cache exactly once; a request that has a single block left at admission
+    therefore behaves exactly as under the default reading, and a multi-block request agrees with it on its first
+    block (same refresh, same cached steps) before the stale cache shows."""
+    shape, model = tiny_model()
+    L = 4
+    rng = np.random.default_rng(21)
+    spec = [(5, 4, 3.0, 0), (7, 12, 6.0, 0), (3, 8, 9.0, 1), (6, 16, 1.5, 0)]
+    reqs = [(i, rng.integers(0, 49, size=p), g, a, st, rng.integers(0, 49, size=st * L) if st else None)
+            for i, (p, g, a, st) in enumerate(spec)]
+    runs = []
+    for variant in (False, True):
+        e = O.Engine(model, L, 0.9, 0, 4, 1 << 20, refresh_at_admission_only=variant)
+        for q in reqs:
+            e.admit(*q)
+        e.run()
+        runs.append(e)
+    base, var = runs
+    for i, (p, g, a, st) in enumerate(spec):
+        K = -(-g // L)
+        assert base.by_id[i].refreshes == K - st and var.by_id[i].refreshes == 1
+        assert var.by_id[i].committed == g - st * L and (var.tokens(i) != model.mask_id).all()
+        first = slice(p + st * L, p + (st + 1) * L)
+        assert (var.tokens(i)[first] == base.tokens(i)[first]).all()
+        if K - st == 1:
+            assert (var.tokens(i) == base.tokens(i)).all() and var.by_id[i].steps == base.by_id[i].steps
+    # the index builder follows the same rule: a row in the first step of a later block brings only its block
+    e = O.Engine(model, L, 0.9, 0, 4, 1 << 20, refresh_at_admission_only=True)
+    e.admit(*reqs[1])
+    e.evict_refill()
+    assert len(O.build_indices(e.sched.active, L)["tok_pos"]) == 7 + 12
+    while not e.block_done():
+        e.denoise_step()
+    e.evict_refill()
+    ix = O.build_indices(e.sched.active, L)
+    assert ix["tok_pos"].tolist() == [11, 12, 13, 14] and ix["lm_tok"].tolist() == [0, 1, 2, 3]
+
+
+def test_block_length_64_uses_one_mask_bit_per_position():
+    """L = 64 (the largest block length of the paper's ablation): 64-bit mask words, tau = 1 gives exactly 64 steps
+    per full block, a ragged last block its own length."""
+    shape, model = tiny_model()
+    rng = np.random.default_rng(2)
+    e = O.Engine(model, 64, 1.0, 0, 2, 1 << 20)
+    e.admit(0, rng.integers(0, 49, size=5), 100, 2.0)
+    e.evict_refill()
+    r = e.sched.active[0]
+    assert r.mask == (1 << 64) - 1
+    steps = 0
+    while not e.block_done():
+        e.denoise_step()
+        steps += 1
+    assert steps == 64
+    e.evict_refill()
+    assert e.sched.active[0].mask == (1 << 36) - 1
+    ix = O.build_indices(e.sched.active, 64)
+    assert ix["lm_slot"].tolist() == list(range(36))
