@@ -48,6 +48,7 @@ typedef enum {
 
 enum { BS_SUFFIX_FULL = 0, BS_SUFFIX_NONE = 1 };
 enum { BS_REQ_QUEUED = 0, BS_REQ_ACTIVE = 1, BS_REQ_FINISHED = 2 };
+enum { BS_REFRESH_EVERY_BLOCK = 0, BS_REFRESH_AT_ADMISSION = 1 };
 
 typedef struct {
   /* model: pre-norm bidirectional transformer, RMSNorm, rotate-half RoPE, GQA, SwiGLU, no biases */
@@ -80,6 +81,12 @@ typedef struct {
                                     its next block in the following step.  bs_block_done then reports all_done only
                                     when the active set is empty; bs_evict_refill is the first fill and any later fill
                                     of an empty active set.  0: batch-synchronous block cycles (Algorithm 1) */
+  int refresh_policy;            /* when a row's prefix / suffix cache is rebuilt by a whole-row forward (Section 2.5
+                                    leaves it open: "frozen prefix cache" vs a block-wise approximate cache).
+                                    BS_REFRESH_EVERY_BLOCK (default): at the first step of every block.
+                                    BS_REFRESH_AT_ADMISSION: only at the first step after admission; later blocks
+                                    start with a cached block step and the cache keeps what earlier steps wrote
+                                    (throughput ablation; snapshots are then refused while rows are active) */
   int keep_logits;               /* parity hook: 1 = the LM head also stores the fp32 logits [M_m, vocab] of every step
                                     (4 * max_batch * L * vocab more workspace bytes) so that bs_debug_read can return
                                     them; 0 = the logits never reach device memory, only the confidence partials of

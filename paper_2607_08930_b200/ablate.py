@@ -20,10 +20,12 @@ from paper_2607_08930_b200 import binding as B, build  # noqa: E402
 
 
 def run_variant(wl, weights, sort_queue: bool, suffix_mode: int, steps_per_block: int = 0,
-                static_groups: bool = False, async_advance: bool = False, kv_capacity_tokens=None):
+                static_groups: bool = False, async_advance: bool = False, kv_capacity_tokens=None,
+                refresh_policy: int = 0):
     eng = B.engine_for_workload(wl, weights, sort_queue=sort_queue, suffix_mode=suffix_mode,
                                 steps_per_block=steps_per_block, static_groups=static_groups,
-                                async_advance=async_advance, kv_capacity_tokens=kv_capacity_tokens)
+                                async_advance=async_advance, kv_capacity_tokens=kv_capacity_tokens,
+                                refresh_policy=refresh_policy)
     for r in wl.requests:
         eng.admit(r.req_id, r.prompt, r.g, r.alpha, r.start_block, r.gen_prefix)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -52,7 +54,8 @@ def main():
                     help="add the comparison policy: fixed groups in submission order, no refill until a group is done")
     ap.add_argument("--requests", type=int, default=0, help="use only the first N requests of the workload")
     ap.add_argument("--async-advance", action="store_true",
-                    help="add the per-row block advance (sorted queue, full suffix) beside the synchronous cycles")
+                    help="add the per-row block advance and the refresh-at-admission variant (sorted queue, full "
+                         "suffix) beside the synchronous cycles")
     ap.add_argument("--kv-rows", type=int, default=0, help="rows of the KV arena (0: sized from the workload)")
     ap.add_argument("--steps-per-block", type=int, nargs="*", default=[],
                     help="extra variants with a transfer quota S < L (sorted queue, full suffix)")
@@ -83,7 +86,10 @@ def main():
         rows.append(res)
     if args.async_advance:
         for name, kw in (("sorted, synchronous block cycles (Algorithm 1)", dict()),
-                         ("sorted, per-row block advance", dict(async_advance=True))):
+                         ("sorted, per-row block advance", dict(async_advance=True)),
+                         ("sorted, cache rebuilt at admission only", dict(refresh_policy=B.REFRESH_AT_ADMISSION)),
+                         ("sorted, per-row advance + cache rebuilt at admission only",
+                          dict(async_advance=True, refresh_policy=B.REFRESH_AT_ADMISSION))):
             kw.update(kv_capacity_tokens=args.kv_rows or None)
             run_variant(base, weights, True, B.SUFFIX_FULL, **kw)
             res = run_variant(base, weights, True, B.SUFFIX_FULL, **kw)

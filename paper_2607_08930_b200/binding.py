@@ -19,6 +19,7 @@ LIB_PATH = os.path.join(_HERE, "libblockserve.so")
 BS_OK, BS_E_ARG, BS_E_STATE, BS_E_BUDGET, BS_E_KV_FULL, BS_E_CUDA, BS_E_TIMEOUT, BS_E_UNKNOWN_REQ = (
     0, -1, -2, -3, -4, -5, -6, -7)
 SUFFIX_FULL, SUFFIX_NONE = 0, 1
+REFRESH_EVERY_BLOCK, REFRESH_AT_ADMISSION = 0, 1
 REQ_QUEUED, REQ_ACTIVE, REQ_FINISHED = 0, 1, 2
 
 (DBG_HEADER, DBG_ROW_SLOT, DBG_ROW_MASK, DBG_ROW_S, DBG_ROW_KV_BASE, DBG_CU_Q, DBG_TOK_ROW, DBG_TOK_POS,
@@ -37,7 +38,8 @@ class BsConfig(C.Structure):
                 ("token_budget", C.c_longlong), ("max_batch", C.c_int), ("max_requests", C.c_int),
                 ("max_row_tokens", C.c_int), ("kv_capacity_tokens", C.c_longlong), ("suffix_mode", C.c_int),
                 ("sort_queue", C.c_int), ("steps_per_block", C.c_int), ("eos_id", C.c_int),
-                ("static_groups", C.c_int), ("async_advance", C.c_int), ("keep_logits", C.c_int)]
+                ("static_groups", C.c_int), ("async_advance", C.c_int), ("refresh_policy", C.c_int),
+                ("keep_logits", C.c_int)]
 
 
 class BsWeights(C.Structure):
@@ -131,11 +133,13 @@ def _check_op(rc: int, name: str) -> None:
 def make_config(shape, block_len: int, tau: float, token_budget: int, max_batch: int, max_requests: int,
                 max_row_tokens: int, kv_capacity_tokens: int, suffix_mode: int = SUFFIX_FULL,
                 sort_queue: bool = True, steps_per_block: int = 0, eos_id: int = -1,
-                static_groups: bool = False, keep_logits: bool = False, async_advance: bool = False) -> BsConfig:
+                static_groups: bool = False, keep_logits: bool = False, async_advance: bool = False,
+                refresh_policy: int = 0) -> BsConfig:
     return BsConfig(shape.n_layers, shape.d_model, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, shape.d_ffn,
                     shape.vocab, shape.mask_id, shape.rms_eps, shape.rope_theta, block_len, tau, token_budget,
                     max_batch, max_requests, max_row_tokens, kv_capacity_tokens, suffix_mode, int(sort_queue),
-                    int(steps_per_block), int(eos_id), int(static_groups), int(async_advance), int(keep_logits))
+                    int(steps_per_block), int(eos_id), int(static_groups), int(async_advance), int(refresh_policy),
+                    int(keep_logits))
 
 
 def query_sizes(cfg: BsConfig) -> BsSizes:
@@ -300,7 +304,7 @@ class Engine:
 def engine_for_workload(wl, weights, *, kv_capacity_tokens: Optional[int] = None, suffix_mode: int = SUFFIX_FULL,
                         sort_queue: bool = True, steps_per_block: int = 0, eos_id: int = -1,
                         static_groups: bool = False, keep_logits: bool = False, async_advance: bool = False,
-                        device: str = "cuda:0") -> Engine:
+                        refresh_policy: int = 0, device: str = "cuda:0") -> Engine:
     """Size an engine for a bs_inputs.Workload (the caller still admits the requests)."""
     mrt = wl.max_row_tokens
     if kv_capacity_tokens is None:
@@ -310,7 +314,7 @@ def engine_for_workload(wl, weights, *, kv_capacity_tokens: Optional[int] = None
             kv_capacity_tokens = min(kv_capacity_tokens, wl.token_budget + wl.max_batch * max(r.g for r in wl.requests))
     cfg = make_config(wl.shape, wl.block_len, wl.tau, wl.token_budget, wl.max_batch, len(wl.requests), mrt,
                       max(kv_capacity_tokens, mrt), suffix_mode, sort_queue, steps_per_block, eos_id, static_groups,
-                      keep_logits, async_advance)
+                      keep_logits, async_advance, refresh_policy)
     return Engine(cfg, weights, device)
 
 

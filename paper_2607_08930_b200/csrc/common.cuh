@@ -55,6 +55,7 @@ struct DevState {
   int eos_id;           // CheckEOS of Algorithm 1 (< 0: off)
   int static_groups;    // 1: no admission while any row of the current group is active (comparison policy)
   int async_advance;    // 1: rows advance / leave and the queue refills after every denoise step
+  int refresh_policy;   // 0: every block starts with a whole-row forward; 1: only the first block after admission
   long long beta, kv_capacity;
   float tau;
   int* hdr;             // [kHdrInts] followed directly by row_mask[max_batch]
@@ -63,6 +64,7 @@ struct DevState {
   int* tokens;          // [max_requests, max_row_tokens]
   int* queue;           // pending slots in admission order
   int* row_slot; int* row_s; int* row_kv_base; int* row_vis;
+  int* row_refresh;     // 1: the first step of the row's current block forwards the whole row
   int* cu_q[2]; int* lm_base[2]; int* cu_tile[2];
   int* lm_tok[2]; int* lm_row[2]; int* lm_slot[2];
   int* out_tok[2]; float* out_conf[2]; int* out_commit[2];

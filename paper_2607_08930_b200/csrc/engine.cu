@@ -87,6 +87,7 @@ size_t carve_state(const bs_config& c, void* base, DevState* out) {
   st.queue = cv.take<int>(R);
   st.row_slot = cv.take<int>(B); st.row_s = cv.take<int>(B); st.row_kv_base = cv.take<int>(B);
   st.row_vis = cv.take<int>(B);
+  st.row_refresh = cv.take<int>(B);
   for (int k = 0; k < 2; ++k) {
     st.cu_q[k] = cv.take<int>(B + 1); st.lm_base[k] = cv.take<int>(B + 1); st.cu_tile[k] = cv.take<int>(B + 1);
     st.lm_tok[k] = cv.take<int>(mm); st.lm_row[k] = cv.take<int>(mm); st.lm_slot[k] = cv.take<int>(mm);
@@ -118,6 +119,8 @@ const char* check_config(const bs_config& c) {
   if (c.eos_id >= c.vocab || c.eos_id == c.mask_id) return "eos_id must be a token id other than the mask id, or negative";
   if (c.keep_logits != 0 && c.keep_logits != 1) return "keep_logits must be 0 or 1";
   if (c.async_advance != 0 && c.async_advance != 1) return "async_advance must be 0 or 1";
+  if (c.refresh_policy != BS_REFRESH_EVERY_BLOCK && c.refresh_policy != BS_REFRESH_AT_ADMISSION)
+    return "bad refresh_policy";
   if (c.async_advance && c.static_groups) return "async_advance and static_groups exclude each other";
   return nullptr;
 }
@@ -329,6 +332,7 @@ int bs_init_model(const bs_config* cfg, const bs_weights* w, void* kv, void* wor
   st.eos_id = cfg->eos_id;
   st.static_groups = cfg->static_groups ? 1 : 0;
   st.async_advance = cfg->async_advance ? 1 : 0;
+  st.refresh_policy = cfg->refresh_policy;
   st.q_tile = attention_q_tile(cfg->n_q_heads, cfg->n_kv_heads, cfg->head_dim);
   st.slice_ms = e->ws.slice_ms;
   st.slice_am = e->ws.slice_am;
@@ -757,6 +761,8 @@ int bs_debug_snapshot(bs_engine* e, void* host_buf, size_t cap, size_t* n_out) {
   // complete only between block cycles.
   if (e->hdr[H_N_ACTIVE] > 0 && !e->hdr[H_ALL_DONE])
     return fail(e, BS_E_STATE, "snapshots are taken between block cycles");
+  if (e->cfg.refresh_policy != BS_REFRESH_EVERY_BLOCK && e->hdr[H_N_ACTIVE] > 0)
+    return fail(e, BS_E_STATE, "without a refresh at every block start the KV cache is part of the state");
   CU(e, cudaStreamSynchronize(e->stream));
   char* out = static_cast<char*>(host_buf);
   SnapHeader h;

@@ -75,9 +75,9 @@ __device__ void build_index(const DevState& st, int parity, int n, int* smi) {
     vis = st.suffix_mode == 0 ? p + g : hi;
     st.row_vis[i] = vis;
     if (mask != 0ull) {
-      nq = (s == 0) ? vis : hi - lo;
+      refresh = (s == 0 && st.row_refresh[i] != 0);
+      nq = refresh ? vis : hi - lo;
       unfinished = 1;
-      refresh = (s == 0);
     }
     nm = __popcll(mask);
   }
@@ -122,7 +122,7 @@ __device__ void build_index(const DevState& st, int parity, int n, int* smi) {
         const int slot = st.row_slot[r];
         const int lo = st.req_p[slot] + st.req_b[slot] * st.L;
         const int k = st.lm_base[parity][r] + __popcll(mask & ((1ull << j) - 1ull));
-        st.lm_tok[parity][k] = st.cu_q[parity][r] + (st.row_s[r] == 0 ? lo + j : j);
+        st.lm_tok[parity][k] = st.cu_q[parity][r] + ((st.row_s[r] == 0 && st.row_refresh[r] != 0) ? lo + j : j);
         st.lm_row[parity][k] = r;
         st.lm_slot[parity][k] = j;
         st.lm_scale[parity][k] = st.req_alpha[slot];
@@ -147,13 +147,14 @@ __device__ void sched_body(const DevState& st, bool only_done) {
   const int L = st.L;
 
   // ---- advance, evict finished rows (b_i >= K_i or CheckEOS), compact (order preserved) ----
-  int keep = 0, slot = -1, kvb = 0, srow = 0;
+  int keep = 0, slot = -1, kvb = 0, srow = 0, rfr = 0;
   MaskWord mask = 0ull;
   if (i < n0) {
     slot = st.row_slot[i];
     kvb = st.row_kv_base[i];
     mask = st.row_mask[i];
     srow = st.row_s[i];
+    rfr = st.row_refresh[i];
     if (only_done && mask != 0ull) {
       keep = 1;                                            // mid-block: nothing changes for this row
     } else {
@@ -170,6 +171,7 @@ __device__ void sched_body(const DevState& st, bool only_done) {
       }
       if (!keep) st.req_state[slot] = 2;
       srow = -1;                                           // marks "starts a block now"
+      rfr = st.refresh_policy == 0;                        // later blocks are refreshed only under the default policy
     }
   }
   int n_keep;
@@ -179,6 +181,7 @@ __device__ void sched_body(const DevState& st, bool only_done) {
     st.row_kv_base[dst] = kvb;
     st.row_mask[dst] = mask;
     st.row_s[dst] = srow;
+    st.row_refresh[dst] = rfr;
   }
   __syncthreads();
 
@@ -229,6 +232,7 @@ __device__ void sched_body(const DevState& st, bool only_done) {
         st.row_slot[n] = c;
         st.row_kv_base[n] = (int)start;
         st.row_s[n] = -1;
+        st.row_refresh[n] = 1;                             // a newly admitted row has no cache yet
         st.req_state[c] = 1;
         s_n = n + 1;
         s_head = head + 1;
@@ -396,7 +400,7 @@ __global__ void k_fill_tokens(DevState st, int parity, int M) {
     }
     const int r = lo;
     const int slot = st.row_slot[r];
-    const int first = st.row_s[r] == 0 ? 0 : st.req_p[slot] + st.req_b[slot] * st.L;
+    const int first = (st.row_s[r] == 0 && st.row_refresh[r] != 0) ? 0 : st.req_p[slot] + st.req_b[slot] * st.L;
     const int pos = first + (t - cu[r]);
     st.tok_row[t] = r;
     st.tok_pos[t] = pos;                 // logical position id: 0 = first prompt token of the request

@@ -127,7 +127,7 @@ class Lockstep:
 
     def __init__(self, wl, weights_cuda, weights_np, suffix_mode=0, kv_capacity=None, sort_queue=True, track=None,
                  model=None, steps_per_block=0, eos_id=-1, static_groups=False, modes=("bf16", "fp32"),
-                 async_advance=False, engine_kwargs=None):
+                 async_advance=False, refresh_at_admission_only=False, engine_kwargs=None):
         self.wl = wl
         self.track = None if track is None else set(track)
         # the near-tie classes below are written for one forced token per step; a general transfer quota is checked
@@ -138,14 +138,16 @@ class Lockstep:
         self.eng = B.engine_for_workload(wl, weights_cuda, kv_capacity_tokens=kv_capacity, suffix_mode=suffix_mode,
                                          sort_queue=sort_queue, steps_per_block=steps_per_block, eos_id=eos_id,
                                          static_groups=static_groups, keep_logits=True, async_advance=async_advance,
-                                         **(engine_kwargs or {}))
+                                         refresh_policy=int(refresh_at_admission_only), **(engine_kwargs or {}))
         self.model = model if model is not None else O.model_from_weights(wl.shape, weights_np)
         assert self.model.bf16_activations
         self.model32 = dataclasses.replace(self.model, bf16_activations=False) if "fp32" in modes else None
         self.ora = O.Engine(self.model, wl.block_len, wl.tau, wl.token_budget, wl.max_batch,
                             self.eng.cfg.kv_capacity_tokens, suffix_mode, sort_queue, steps_per_block=steps_per_block,
-                            eos_id=eos_id, static_groups=static_groups, async_advance=async_advance)
+                            eos_id=eos_id, static_groups=static_groups, async_advance=async_advance,
+                            refresh_at_admission_only=refresh_at_admission_only)
         self.async_advance = async_advance
+        self.refresh_only = refresh_at_admission_only
         self.shadow = {}                 # req_id -> the fp32-mode oracle's copy of a tracked request
         self.suffix_mode = suffix_mode
         self.excluded = {c: 0 for c in CLASSES}
@@ -308,7 +310,7 @@ class Lockstep:
             if self.model32 is not None:
                 sh = self.shadow[r.req_id]
                 assert (sh.tokens == r.tokens).all()
-                sh.b, sh.s, sh.mask = r.b, r.s, r.mask
+                sh.b, sh.s, sh.mask, sh.needs_refresh = r.b, r.s, r.mask, r.needs_refresh
                 probe32 = O.denoise_step(self.model32, sh, self.wl.block_len, self.wl.tau, self.suffix_mode,
                                          keep_logits=True, override_commit=gs, override_tok=gt,
                                          steps_per_block=self.S)
@@ -468,6 +470,7 @@ class Lockstep:
             for b in range(q.start_block, r.n_blocks(L)):
                 r.b = b
                 O.start_block_state(r, L)
+                r.needs_refresh = b == q.start_block or not self.refresh_only
                 while r.mask:
                     if stop is not None and (r.b, r.s) >= stop:
                         finished = False

@@ -43,7 +43,8 @@ def test_query_sizes_and_validation(B):
                           eos_id=5, static_groups=True)
     sz_p = B.query_sizes(cfg_p)
     assert (sz_p.kv_bytes, sz_p.workspace_bytes, sz_p.state_bytes) == (sz.kv_bytes, sz.workspace_bytes, sz.state_bytes)
-    for field, bad in (("head_dim", 48), ("block_len", 64), ("max_batch", 5000), ("vocab", 1023),
+    for field, bad in (("head_dim", 48), ("block_len", 65), ("max_batch", 5000), ("vocab", 1023),
+                       ("refresh_policy", 2), ("async_advance", 2), ("keep_logits", 3),
                        ("kv_capacity_tokens", 3), ("n_q_heads", 3), ("steps_per_block", 33), ("steps_per_block", -1),
                        ("eos_id", wl.shape.mask_id), ("eos_id", wl.shape.vocab)):
         cfg2 = B.make_config(wl.shape, 32, 0.9, 0, 4, 8, wl.max_row_tokens, 4 * wl.max_row_tokens)

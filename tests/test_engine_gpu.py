@@ -181,9 +181,11 @@ def test_bounded_wait_reports_timeout_and_keeps_the_context(B):
     assert other.stats().committed == wl.committed_target()
 
 
-@pytest.mark.parametrize("L,sort_queue,max_batch", [(16, True, 3), (8, False, 1), (32, False, 2)])
+@pytest.mark.parametrize("L,sort_queue,max_batch", [(16, True, 3), (8, False, 1), (32, False, 2), (64, True, 3),
+                                                    (48, False, 2)])
 def test_other_block_lengths_queue_orders_and_batch_caps(B, L, sort_queue, max_batch):
-    """Block lengths below 32, arrival-order queue, a batch cap of one: full lockstep on the tiny model."""
+    """Block lengths from 8 to 64 (mask words of up to 64 bits, two list entries per lane in the commit kernel),
+    arrival-order queue, a batch cap of one: full lockstep on the tiny model."""
     from lockstep import Lockstep
     shape = bs_inputs.TINY
     rng = np.random.default_rng(L)
@@ -468,3 +470,44 @@ def test_async_advance_stream_with_budget_arrivals_and_ragged_blocks(B):
     assert len(ls.ora.sched.finished) == n
     print(f"mini-gqa async: {ls.summary()}")
     ls.assert_caps()
+
+
+@pytest.mark.parametrize("shape_name,async_advance", [("tiny", False), ("mini", False), ("tiny", True)])
+def test_refresh_at_admission_only_in_lockstep(B, shape_name, async_advance):
+    """The ablation variant that rebuilds a row's cache only at admission: the first step of every later block is a
+    cached block step over a cache that keeps what earlier steps wrote, on both sides alike."""
+    from lockstep import Lockstep
+    shape = bs_inputs.TINY if shape_name == "tiny" else bs_inputs.MINI_GQA
+    rng = np.random.default_rng(17)
+    n = 7
+    ps = rng.integers(5, 90, size=n)
+    gs = rng.choice([96, 64, 40, 128], size=n)
+    al = rng.choice([3.0, 9.0, 30.0], size=n)
+    wl = bs_inputs.custom_workload(shape, ps, gs, al, token_budget=900, max_batch=4, seed=18, tau=0.9)
+    wc, wn = both_weights(shape, 55)
+    ls = Lockstep(wl, wc, wn, refresh_at_admission_only=True, async_advance=async_advance)
+    ls.admit(wl.requests)
+    ls.run()
+    free = ls.check_free_run()
+    st = ls.eng.stats()
+    assert st.committed == wl.committed_target()
+    assert all(r.refreshes == 1 for r in ls.ora.by_id.values())
+    # the packed-token count shows the saving: one whole-row forward per request instead of one per block
+    base = B.engine_for_workload(wl, wc, async_advance=async_advance)
+    for r in wl.requests:
+        base.admit(r.req_id, r.prompt, r.g, r.alpha)
+    base.run()
+    assert st.packed_tokens < base.stats().packed_tokens
+    print(f"refresh at admission only ({shape_name}, async={async_advance}): packed tokens {st.packed_tokens} vs "
+          f"{base.stats().packed_tokens}; {ls.summary()} | free oracle run: {free}")
+    ls.assert_caps(floor=10)
+    with pytest.raises(B.BlockServeError):
+        eng = B.engine_for_workload(wl, wc, refresh_policy=B.REFRESH_AT_ADMISSION)
+        for r in wl.requests:
+            eng.admit(r.req_id, r.prompt, r.g, r.alpha)
+        eng.evict_refill()
+        while True:
+            eng.denoise_step()
+            if eng.block_done():
+                break
+        eng.snapshot()          # rows are active and their cache is state: refused
