@@ -131,26 +131,37 @@ struct AttnTcParams {
 constexpr int KT = 64;                                   // keys per tile
 constexpr int kKvHalf = KT * 128;                        // KT rows x 64 bf16
 constexpr int kStageBytes = 4 * kKvHalf;                 // K halves, V halves
-__host__ __device__ constexpr int smem_for(int nq, int stages) { return nq * kQBytes + stages * kStageBytes + 1024; }
+__host__ __device__ constexpr int smem_for(int q_tiles, int stages) {
+  return q_tiles * kQBytes + stages * kStageBytes + 1024;
+}
 
-template <int NQ, int STAGES>
-__global__ void __launch_bounds__(threads_for(NQ), smem_for(NQ, STAGES) <= 112 * 1024 ? 2 : 1)
+// NG: softmax warp groups (each with its own scores buffers and output accumulator in tensor memory).
+//   KS = false: group x serves Q tile x of the CTA (NG Q tiles in shared memory, every K/V tile used by all of them).
+//   KS = true (NG = 2): one Q tile; the two groups are two independent streams over the row's key tiles - group x
+//        takes tiles x, x + 2, x + 4, ... with its own running maximum, sum and accumulator - and the streams are
+//        merged once at the end.  A single stream is a dependent chain per key tile (scores -> softmax -> P V ->
+//        next softmax); two of them keep the tensor pipe and the exponent unit busy through each other's waits.
+template <int NG, int STAGES, bool KS>
+__global__ void __launch_bounds__(threads_for(NG), smem_for(KS ? 1 : NG, STAGES) <= 112 * 1024 ? 2 : 1)
 k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                const __grid_constant__ CUtensorMap map_v, const AttnTcParams p) {
+  static_assert(!KS || NG == 2, "two streams need two softmax groups");
   constexpr int kStages = STAGES;
-  constexpr unsigned kTmemCols = NQ == 2 ? 512u : 256u;
+  constexpr int kQTiles = KS ? 1 : NG;                      // Q tiles of this CTA
+  constexpr unsigned kTmemCols = NG == 2 ? 512u : 256u;
   // Barrier slots
-  enum { B_QFULL = 0, B_KVFULL = 1, B_KVEMPTY = B_KVFULL + kStages, B_SFULL = B_KVEMPTY + kStages,   // [tile][2]
+  enum { B_QFULL = 0, B_KVFULL = 1, B_KVEMPTY = B_KVFULL + kStages, B_SFULL = B_KVEMPTY + kStages,   // [group][2]
          B_PFULL = B_SFULL + 4, B_OFULL = B_PFULL + 2, B_COUNT = B_OFULL + 2 };
   extern __shared__ unsigned char smem_dyn[];
   __shared__ __align__(8) unsigned long long bars[B_COUNT];
   __shared__ unsigned tmem_base_slot;
   __shared__ int s_abort;
+  __shared__ float2 s_ml[KS ? 128 : 1];                     // (scale, sum) of stream 1, per query row
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const unsigned smem0 = (smem_u32(smem_dyn) + 1023u) & ~1023u;
   const unsigned sQ = smem0;                              // [Q tile][dim half][128 rows x 128 B]
-  const unsigned sKV = sQ + NQ * kQBytes;
+  const unsigned sKV = sQ + kQTiles * kQBytes;
   const unsigned bar0 = smem_u32(&bars[0]);
   auto bar = [&](int i) { return bar0 + 8u * (unsigned)i; };
 
@@ -165,7 +176,7 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       mbar_init(bar(B_SFULL + i), 1);
     }
     for (int i = 0; i < 2; ++i) {
-      mbar_init(bar(B_PFULL + i), 4);      // one arrival per softmax warp of the Q tile
+      mbar_init(bar(B_PFULL + i), 4);      // one arrival per softmax warp of the group
       mbar_init(bar(B_OFULL + i), 1);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -183,10 +194,10 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   pdl_trigger();
   pdl_wait();       // indices, q and the cache rows of this step come from earlier kernels of the stream
 
-  // ---- which row owns this work item: largest r with cu_tile[r] <= blockIdx.x ----
+  // ---- which row owns this work item: largest r with cu_tile[r] <= item ----
   const int G = p.hq / p.hkv;
   const int kh = blockIdx.y;
-  constexpr bool kSplit = NQ == 1;                          // one CTA per Q tile: two CTAs share a work item
+  constexpr bool kSplit = kQTiles == 1;                     // one CTA per Q tile: two CTAs share a work item
   const int item = kSplit ? (int)blockIdx.x >> 1 : (int)blockIdx.x;
   int lo = 0, hi = p.n_rows;
   while (hi - lo > 1) {
@@ -194,7 +205,7 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     if (p.cu_tile[mid] <= item) lo = mid; else hi = mid;
   }
   const int row = lo;
-  const int per_cta = NQ * p.tq;
+  const int per_cta = kQTiles * p.tq;
   const int t0 = p.cu_q[row] + (item - p.cu_tile[row]) * 2 * p.tq + (kSplit ? ((int)blockIdx.x & 1) * p.tq : 0);
   const int nt = min(per_cta, p.cu_q[row + 1] - t0);        // query tokens of this CTA (CTA-uniform)
   const int n_qt = nt <= 0 ? 0 : (nt > p.tq ? 2 : 1);       // Q tiles in use
@@ -205,6 +216,7 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   const int per_chunk = (tiles_all + p.chunks - 1) / p.chunks;
   const int kt0 = (int)blockIdx.z * per_chunk;
   const int n_tiles = nt > 0 ? max(0, min(tiles_all, kt0 + per_chunk) - kt0) : 0;
+  const int n_groups = KS ? min(2, n_tiles) : n_qt;         // softmax groups with work
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -232,159 +244,223 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       const unsigned idesc_s = umma_idesc(KT, false);
       const unsigned idesc_o = umma_idesc(DH, true);
       bool ok = mbar_wait(bar(B_QFULL), 0, abort_flag);
-      // S = Q K^T of key tile t for every Q tile in use, into the S buffer of parity t
-      auto issue_scores = [&](int t) -> bool {
-        const int s = t % kStages, b = t & 1;
-        if (!mbar_wait(bar(B_KVFULL + s), (unsigned)(t / kStages) & 1u, abort_flag)) return false;
-        const unsigned st = sKV + s * kStageBytes;
-        for (int x = 0; x < n_qt; ++x) {
-          // Scores buffer b is free: the softmax warps finished with the scores of tile t - 2 before they published
-          // its probabilities (same columns), and the P V product that read those was issued by this thread after
-          // that and before this product; the tensor pipe runs one thread's instructions in order.
-          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          const unsigned q_lo = desc_lo(sQ + x * kQBytes), k_lo = desc_lo(st), d_s = tmem_base + x * 256 + b * 64;
+      // S = Q K^T of key tile t into scores buffer b of group x.
+      // The buffer is free: the softmax warps finished with the scores it held two of the group's tiles ago before
+      // they published the probabilities (same columns), and the P V product that read those was issued by this
+      // thread after that and before this product; the tensor pipe runs one thread's instructions in order.
+      auto scores = [&](unsigned st, int x, int q_tile, int b) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const unsigned q_lo = desc_lo(sQ + q_tile * kQBytes), k_lo = desc_lo(st), d_s = tmem_base + x * 256 + b * 64;
 #pragma unroll
-          for (int h = 0; h < 2; ++h)
+        for (int h = 0; h < 2; ++h)
 #pragma unroll
-            for (int k = 0; k < 4; ++k)
-              umma_lo(d_s, q_lo + h * (kHalfBytes >> 4) + 2 * k, k_lo + h * (kKvHalf >> 4) + 2 * k, idesc_s,
-                      (h | k) ? 1u : 0u);
-          umma_commit(bar(B_SFULL + 2 * x + b));
-        }
-        return true;
+          for (int k = 0; k < 4; ++k)
+            umma_lo(d_s, q_lo + h * (kHalfBytes >> 4) + 2 * k, k_lo + h * (kKvHalf >> 4) + 2 * k, idesc_s,
+                    (h | k) ? 1u : 0u);
+        umma_commit(bar(B_SFULL + 2 * x + b));
       };
-      if (ok) ok = issue_scores(0);
-      for (int t = 0; t < n_tiles && ok; ++t) {
-        if (t + 1 < n_tiles) ok = issue_scores(t + 1);      // next tile's scores run under this tile's softmax
-        if (!ok) break;
-        const unsigned st = sKV + (t % kStages) * kStageBytes;
-        for (int x = 0; x < n_qt && ok; ++x) {
-          if (!mbar_wait(bar(B_PFULL + x), (unsigned)t & 1u, abort_flag)) { ok = false; break; }
-          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          // P comes from tensor memory (the first 32 columns of the scores buffer of this tile: 64 bf16 per row);
-          // V is an MN-major operand whose two 64-wide dim halves are kKvHalf bytes apart (leading byte offset)
-          const unsigned p_tm = tmem_base + x * 256 + (t & 1) * 64, v_lo = desc_lo(st + 2 * kKvHalf, kKvHalf);
-          const unsigned d_o = tmem_base + x * 256 + 128;
+      // O_x += P V: P from tensor memory (the first 32 columns of scores buffer b of group x: 64 bf16 per row);
+      // V is an MN-major operand whose two 64-wide dim halves are kKvHalf bytes apart (leading byte offset)
+      auto pv = [&](unsigned st, int x, int b, bool first) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const unsigned p_tm = tmem_base + x * 256 + b * 64, v_lo = desc_lo(st + 2 * kKvHalf, kKvHalf);
+        const unsigned d_o = tmem_base + x * 256 + 128;
 #pragma unroll
-          for (int j = 0; j < KT / 16; ++j)         // 16 keys per step; the output accumulates over all key tiles
-            umma_ts(d_o, p_tm + j * 8, v_lo + j * (2048 >> 4), idesc_o, (t | j) ? 1u : 0u);
-          umma_commit(bar(B_OFULL + x));
+        for (int j = 0; j < KT / 16; ++j)           // 16 keys per step; the output accumulates over the group's tiles
+          umma_ts(d_o, p_tm + j * 8, v_lo + j * (2048 >> 4), idesc_o, (!first || j) ? 1u : 0u);
+        umma_commit(bar(B_OFULL + x));
+      };
+      auto stage_of = [&](int t) { return sKV + (unsigned)(t % kStages) * kStageBytes; };
+      auto wait_kv = [&](int t) { return mbar_wait(bar(B_KVFULL + t % kStages), (unsigned)(t / kStages) & 1u, abort_flag); };
+      if (KS) {
+        // key tile t belongs to stream x = t & 1 as its i-th tile, i = t >> 1; the scores of tiles t + 1 and t + 2
+        // are in flight while tile t's softmax runs
+        auto issue_scores = [&](int t) -> bool {
+          if (!wait_kv(t)) return false;
+          scores(stage_of(t), t & 1, 0, (t >> 1) & 1);
+          return true;
+        };
+        if (ok) ok = issue_scores(0);
+        if (ok && n_tiles > 1) ok = issue_scores(1);
+        for (int t = 0; t < n_tiles && ok; ++t) {
+          if (t + 2 < n_tiles) ok = issue_scores(t + 2);
+          if (!ok) break;
+          const int x = t & 1, i = t >> 1;
+          if (!mbar_wait(bar(B_PFULL + x), (unsigned)i & 1u, abort_flag)) { ok = false; break; }
+          pv(stage_of(t), x, i & 1, i == 0);
+          umma_commit(bar(B_KVEMPTY + (t % kStages)));
         }
-        if (ok) umma_commit(bar(B_KVEMPTY + (t % kStages)));
+      } else {
+        auto issue_scores = [&](int t) -> bool {
+          if (!wait_kv(t)) return false;
+          for (int x = 0; x < n_qt; ++x) scores(stage_of(t), x, x, t & 1);
+          return true;
+        };
+        if (ok) ok = issue_scores(0);
+        for (int t = 0; t < n_tiles && ok; ++t) {
+          if (t + 1 < n_tiles) ok = issue_scores(t + 1);      // next tile's scores run under this tile's softmax
+          if (!ok) break;
+          for (int x = 0; x < n_qt && ok; ++x) {
+            if (!mbar_wait(bar(B_PFULL + x), (unsigned)t & 1u, abort_flag)) { ok = false; break; }
+            pv(stage_of(t), x, t & 1, t == 0);
+          }
+          if (ok) umma_commit(bar(B_KVEMPTY + (t % kStages)));
+        }
       }
     }
-  } else {
+  } else if (nt > 0) {
     // ------------------------------------------------------------------ softmax warps: one query row per thread
-    // warps 2..5 own Q tile 0, warps 6..9 own Q tile 1; within a Q tile, warp w reads TMEM lanes 32 (w % 4) ..
+    // warps 2..5 are group 0, warps 6..9 group 1; within a group, warp w reads TMEM lanes 32 (w % 4) ..
     const int x = (warp - 2) >> 2;
     const int q = warp & 3;
     const int r = q * 32 + lane;                        // query row of the Q tile = TMEM lane
-    const int nrows = (x == 0 ? min(nt, p.tq) : nt - p.tq) * G;      // valid rows of this Q tile
-    if (x < n_qt) {
-      const unsigned t_lane = tmem_base + ((unsigned)(q * 32) << 16) + x * 256;
-      const unsigned t_out = t_lane + 128;
-      const float sc = 1.4426950408889634f * rsqrtf((float)DH);
-      const bool warp_has_rows = q * 32 < nrows;        // warps without valid rows only keep the barriers moving
-      float m = -INFINITY, l = 0.f;                     // m: the maximum the accumulator is currently scaled by
-      bool ok = true;
-      for (int t = 0; t < n_tiles && ok; ++t) {
-        const int b = t & 1;
-        if (!mbar_wait(bar(B_SFULL + 2 * x + b), (unsigned)(t >> 1) & 1u, abort_flag)) { ok = false; break; }
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        float v[KT];
-        float f = 1.0f;
-        bool rescale = false;
-        if (warp_has_rows) {
-          // scores -> probabilities in registers; this part overlaps the previous tile's P V product
-          const int key0 = (kt0 + t) * KT;
-          tmem_ld32(t_lane + b * 64, v);
-          tmem_ld32(t_lane + b * 64 + 32, v + 32);
-          // eight independent chains for the row maximum and the row sum: one warp per scheduler has no other
-          // warp to hide a 64-long dependent chain behind.  The maximum is taken over the raw scores (the scale
-          // is positive) and the scale folded into the exponent's fma.
-          float mx8[8];
+    const int q_tile = KS ? 0 : x;                      // the Q tile this group serves
+    const int nrows = (q_tile == 0 ? min(nt, p.tq) : nt - p.tq) * G;      // valid rows of that Q tile
+    const int my_tiles = x < n_groups ? (KS ? (n_tiles - x + 1) / 2 : n_tiles) : 0;
+    const unsigned t_lane = tmem_base + ((unsigned)(q * 32) << 16) + x * 256;
+    const unsigned t_out = t_lane + 128;
+    const float sc = 1.4426950408889634f * rsqrtf((float)DH);
+    const bool warp_has_rows = q * 32 < nrows;          // warps without valid rows only keep the barriers moving
+    float m = -INFINITY, l = 0.f;                       // m: the maximum the accumulator is currently scaled by
+    bool ok = true;
+    for (int i = 0; i < my_tiles && ok; ++i) {
+      const int t = KS ? 2 * i + x : i;                 // key tile inside the chunk
+      const int b = i & 1;
+      if (!mbar_wait(bar(B_SFULL + 2 * x + b), (unsigned)(i >> 1) & 1u, abort_flag)) { ok = false; break; }
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      float v[KT];
+      float f = 1.0f;
+      bool rescale = false;
+      if (warp_has_rows) {
+        // scores -> probabilities in registers; this part overlaps the group's previous P V product
+        const int key0 = (kt0 + t) * KT;
+        tmem_ld32(t_lane + b * 64, v);
+        tmem_ld32(t_lane + b * 64 + 32, v + 32);
+        // eight independent chains for the row maximum and the row sum: one warp per scheduler has no other
+        // warp to hide a 64-long dependent chain behind.  The maximum is taken over the raw scores (the scale
+        // is positive) and the scale folded into the exponent's fma.
+        float mx8[8];
 #pragma unroll
-          for (int i = 0; i < 8; ++i) mx8[i] = -INFINITY;
-          if (key0 + KT <= vis) {
+        for (int k = 0; k < 8; ++k) mx8[k] = -INFINITY;
+        if (key0 + KT <= vis) {
 #pragma unroll
-            for (int j = 0; j < KT; ++j) mx8[j & 7] = fmaxf(mx8[j & 7], v[j]);
-          } else {
-#pragma unroll
-            for (int j = 0; j < KT; ++j) {
-              v[j] = (key0 + j < vis) ? v[j] : -INFINITY;
-              mx8[j & 7] = fmaxf(mx8[j & 7], v[j]);
-            }
-          }
-          const float mx = sc * fmaxf(fmaxf(fmaxf(mx8[0], mx8[1]), fmaxf(mx8[2], mx8[3])),
-                                      fmaxf(fmaxf(mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])));   // finite: a valid key exists
-          // lazy rescale (warp-uniform decision: TMEM loads and stores are warp-wide)
-          const bool grow = mx > m + kLazy;             // always true on the first tile (m = -inf)
-          rescale = __any_sync(0xffffffffu, grow);
-          if (grow) {
-            f = ex2(m - mx);                            // first tile: 2^-inf = 0, and the accumulator is empty
-            m = mx;
-          }
-          float rs8[8];
-#pragma unroll
-          for (int i = 0; i < 8; ++i) rs8[i] = 0.f;
-          const float neg_m = -m;
+          for (int j = 0; j < KT; ++j) mx8[j & 7] = fmaxf(mx8[j & 7], v[j]);
+        } else {
 #pragma unroll
           for (int j = 0; j < KT; ++j) {
-            v[j] = ex2(fmaf(v[j], sc, neg_m));          // 2^(-inf) = 0 for masked keys
-            rs8[j & 7] += v[j];
-          }
-          l = l * f + (((rs8[0] + rs8[1]) + (rs8[2] + rs8[3])) + ((rs8[4] + rs8[5]) + (rs8[6] + rs8[7])));
-        }
-        // the previous P V product must have finished before the accumulator is touched
-        if (t > 0 && !mbar_wait(bar(B_OFULL + x), (unsigned)(t - 1) & 1u, abort_flag)) { ok = false; break; }
-        if (rescale && t > 0) {                     // warp-uniform
-          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-#pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            float o[32];
-            tmem_ld32(t_out + c * 32, o);
-#pragma unroll
-            for (int j = 0; j < 32; ++j) o[j] *= f;
-            tmem_st32(t_out + c * 32, o);
+            v[j] = (key0 + j < vis) ? v[j] : -INFINITY;
+            mx8[j & 7] = fmaxf(mx8[j & 7], v[j]);
           }
         }
-        if (warp_has_rows) {
-          // P as bf16 pairs into the first 32 columns of this tile's scores buffer: the A operand of the P V product
-          unsigned w[32];
-#pragma unroll
-          for (int c = 0; c < 32; ++c) {
-            const __nv_bfloat162 pr = __floats2bfloat162_rn(v[2 * c], v[2 * c + 1]);
-            w[c] = *reinterpret_cast<const unsigned*>(&pr);
-          }
-          tmem_st32_words(t_lane + b * 64, w);
+        const float mx = sc * fmaxf(fmaxf(fmaxf(mx8[0], mx8[1]), fmaxf(mx8[2], mx8[3])),
+                                    fmaxf(fmaxf(mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])));   // finite: a valid key exists
+        // lazy rescale (warp-uniform decision: TMEM loads and stores are warp-wide)
+        const bool grow = mx > m + kLazy;               // always true on the first tile (m = -inf)
+        rescale = __any_sync(0xffffffffu, grow);
+        if (grow) {
+          f = ex2(m - mx);                              // first tile: 2^-inf = 0, and the accumulator is empty
+          m = mx;
         }
-        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar(B_PFULL + x));
+        float rs8[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) rs8[k] = 0.f;
+        const float neg_m = -m;
+#pragma unroll
+        for (int j = 0; j < KT; ++j) {
+          v[j] = ex2(fmaf(v[j], sc, neg_m));            // 2^(-inf) = 0 for masked keys
+          rs8[j & 7] += v[j];
+        }
+        l = l * f + (((rs8[0] + rs8[1]) + (rs8[2] + rs8[3])) + ((rs8[4] + rs8[5]) + (rs8[6] + rs8[7])));
       }
-      if (n_tiles == 0 && p.chunks > 1 && r < nrows)      // a chunk beyond the row's keys: an empty partial
-        p.part_ml[((size_t)blockIdx.z * p.M + t0 + x * p.tq + r / G) * p.hq + kh * G + r % G] = make_float2(0.f, 0.f);
-      if (ok && n_tiles > 0 && mbar_wait(bar(B_OFULL + x), (unsigned)(n_tiles - 1) & 1u, abort_flag) &&
-          warp_has_rows) {
+      // the group's previous P V product must have finished before its accumulator is touched
+      if (i > 0 && !mbar_wait(bar(B_OFULL + x), (unsigned)(i - 1) & 1u, abort_flag)) { ok = false; break; }
+      if (rescale && i > 0) {                       // warp-uniform
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const int tok = r / G, hg = r % G;
-        const bool valid = r < nrows;
-        const float inv = 1.0f / l;
-        const size_t out_at = (size_t)(t0 + x * p.tq + (valid ? tok : 0)) * (p.hq * DH) + (size_t)(kh * G + hg) * DH;
-        bf16* dst = p.out + out_at;
-        float* pdst = p.chunks > 1 ? p.part_o + (size_t)blockIdx.z * p.M * (p.hq * DH) + out_at : nullptr;
-        if (pdst && valid)
-          p.part_ml[((size_t)blockIdx.z * p.M + t0 + x * p.tq + tok) * p.hq + kh * G + hg] = make_float2(m, l);
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
           float o[32];
           tmem_ld32(t_out + c * 32, o);
-          if (valid && pdst) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) o[j] *= f;
+          tmem_st32(t_out + c * 32, o);
+        }
+      }
+      if (warp_has_rows) {
+        // P as bf16 pairs into the first 32 columns of this tile's scores buffer: the A operand of the P V product
+        unsigned w[32];
+#pragma unroll
+        for (int c = 0; c < 32; ++c) {
+          const __nv_bfloat162 pr = __floats2bfloat162_rn(v[2 * c], v[2 * c + 1]);
+          w[c] = *reinterpret_cast<const unsigned*>(&pr);
+        }
+        tmem_st32_words(t_lane + b * 64, w);
+      }
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(B_PFULL + x));
+    }
+    // the group's last P V product
+    const bool have = ok && my_tiles > 0 && mbar_wait(bar(B_OFULL + x), (unsigned)(my_tiles - 1) & 1u, abort_flag);
+    if (!have) l = 0.f;                                 // no keys (or a wait ran out): this group contributes nothing
+    const int tok = r / G, hg = r % G;
+    const bool valid = r < nrows;
+    const size_t out_at = (size_t)(t0 + q_tile * p.tq + (valid ? tok : 0)) * (p.hq * DH) + (size_t)(kh * G + hg) * DH;
+    const size_t ml_at = ((size_t)blockIdx.z * p.M + t0 + q_tile * p.tq + (valid ? tok : 0)) * p.hq + kh * G + hg;
+    float w_own = 1.0f, w_other = 0.f;                  // weights of this group's and the other stream's accumulator
+    bool writer = x < n_qt;                             // KS = false: every group with a Q tile writes its own rows
+    if (KS) {
+      // merge the two streams: stream 1 publishes its (scale, sum); stream 0 reads them and both accumulators
+      if (x == 1) s_ml[r] = make_float2(m, l);
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      asm volatile("bar.sync 1, 256;" ::: "memory");    // the eight softmax warps
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      writer = x == 0;
+      if (writer) {
+        const float2 o1 = s_ml[r];
+        const float mm = fmaxf(l > 0.f ? m : -INFINITY, o1.y > 0.f ? o1.x : -INFINITY);
+        w_own = l > 0.f ? ex2(m - mm) : 0.f;
+        w_other = o1.y > 0.f ? ex2(o1.x - mm) : 0.f;
+        l = w_own * l + w_other * o1.y;
+        m = mm;
+      }
+    }
+    if (writer && warp_has_rows) {
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      if (p.chunks > 1) {
+        // unnormalised partial of this key chunk (sum 0 marks a chunk without keys); the merge kernel finishes
+        if (valid) p.part_ml[ml_at] = make_float2(l > 0.f ? m : 0.f, l);
+        float* pdst = p.part_o + (size_t)blockIdx.z * p.M * (p.hq * DH) + out_at;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          float o[32];
+          tmem_ld32(t_out + c * 32, o);        // (every lane takes part in the load; unused values are masked below)
+          if (KS) {
+            float o2[32];
+            tmem_ld32(t_out + 256 + c * 32, o2);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) o[j] = (w_own > 0.f ? w_own * o[j] : 0.f) + (w_other > 0.f ? w_other * o2[j] : 0.f);
+          }
+          if (valid && l > 0.f) {
 #pragma unroll
             for (int g = 0; g < 8; ++g)
               *reinterpret_cast<float4*>(pdst + c * 32 + g * 4) =
                   make_float4(o[g * 4], o[g * 4 + 1], o[g * 4 + 2], o[g * 4 + 3]);
-          } else if (valid) {
+          }
+        }
+      } else {
+        const float inv = 1.0f / l;
+        bf16* dst = p.out + out_at;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          float o[32];
+          tmem_ld32(t_out + c * 32, o);
+          if (KS) {
+            float o2[32];
+            tmem_ld32(t_out + 256 + c * 32, o2);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) o[j] = (w_own > 0.f ? w_own * o[j] : 0.f) + (w_other > 0.f ? w_other * o2[j] : 0.f);
+          }
+          if (valid && l > 0.f) {
 #pragma unroll
             for (int g = 0; g < 4; ++g) {
               uint4 w;
@@ -508,7 +584,6 @@ cudaError_t launch_attention_tc(const bf16* qkv, const bf16* kc, const bf16* vc,
                                 float* scratch, size_t scratch_floats, int* error_flag, cudaStream_t s,
                                 bool* handled) {
   *handled = false;
-  (void)max_nq;
   if (dh != DH || hq % hkv || hq / hkv > 8 || kv_rows <= 0) return cudaSuccess;
   if (((uintptr_t)qkv | (uintptr_t)kc | (uintptr_t)vc) & 15) return cudaSuccess;
   const int G = hq / hkv;
@@ -520,9 +595,10 @@ cudaError_t launch_attention_tc(const bf16* qkv, const bf16* kc, const bf16* vc,
     std::lock_guard<std::mutex> lock(g_mutex);
     int dev = 0, n = 0;
     cudaGetDevice(&dev);
-    if (cudaFuncSetAttribute(k_attention_tc<1, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_for(1, 2)) != cudaSuccess ||
-        cudaFuncSetAttribute(k_attention_tc<1, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_for(1, 4)) != cudaSuccess ||
-        cudaFuncSetAttribute(k_attention_tc<2, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_for(2, 4)) != cudaSuccess ||
+    if (cudaFuncSetAttribute(k_attention_tc<1, 2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_for(1, 2)) != cudaSuccess ||
+        cudaFuncSetAttribute(k_attention_tc<1, 4, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_for(1, 4)) != cudaSuccess ||
+        cudaFuncSetAttribute(k_attention_tc<2, 4, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_for(2, 4)) != cudaSuccess ||
+        cudaFuncSetAttribute(k_attention_tc<2, 4, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_for(1, 4)) != cudaSuccess ||
         cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1)
       return cudaErrorInvalidDevice;
     *sms = n;
@@ -541,20 +617,30 @@ cudaError_t launch_attention_tc(const bf16* qkv, const bf16* kc, const bf16* vc,
   // its own small CTA, two of them share an SM, and the rows' keys are cut into chunks until about two CTAs per SM
   // are in flight.  Many work items (a refresh step): the two Q tiles of an item share each K/V tile they load.
   static const int env_chunks = getenv("BS_ATTN_TC_CHUNKS") ? atoi(getenv("BS_ATTN_TC_CHUNKS")) : 0;
-  static const int env_plan = getenv("BS_ATTN_TC_PLAN") ? atoi(getenv("BS_ATTN_TC_PLAN")) : 0;   // 1, 2, 3 below
+  static const int env_plan = getenv("BS_ATTN_TC_PLAN") ? atoi(getenv("BS_ATTN_TC_PLAN")) : 0;   // 1 .. 4 below
   const long long items = (long long)n_tiles * hkv;
-  // plan 1: two Q tiles per CTA (refresh steps); plan 2: one Q tile per CTA, four-stage ring, one CTA per SM;
-  // plan 3: one Q tile per CTA, two-stage ring, two CTAs per SM
-  int plan = items < num_sms ? 2 : 1;
-  if (env_plan >= 1 && env_plan <= 3) plan = env_plan;
-  int chunks = 1;
-  if (plan != 1 && scratch && max_vis > 0) {
-    const long long ctas = 2 * items;
-    const int key_tiles = (max_vis + KT - 1) / KT;
-    chunks = (int)((plan == 3 ? 2ll : 1ll) * num_sms / ctas);        // fill the SMs (twice over for plan 3), no more
-    chunks = std::max(1, std::min(chunks, key_tiles / 6));          // at least six key tiles per chunk
-    while (chunks > 1 && (size_t)chunks * M * ((size_t)hq * DH + 2 * hq) > scratch_floats) --chunks;
+  // plan 1: two Q tiles per CTA sharing every K/V tile (refresh steps, and block steps with many rows);
+  // plan 2: one Q tile per CTA, four-stage K/V ring, optionally key chunks (block steps with few rows);
+  // plans 3 and 4 (measurement only, BS_ATTN_TC_PLAN): one Q tile per CTA with a two-stage ring and two CTAs per SM,
+  //         or with the row's key tiles in two interleaved streams merged at the end.
+  // Plan choice by a small cost model fitted to measurements on B200 (microseconds): a CTA costs a fixed ~8 (launch,
+  // tensor-memory allocation, Q load, first K/V tile, output) plus ~1.3 per 64-key tile with two Q tiles or ~0.7 with
+  // one (softmax arithmetic and the scores products bound a tile, not the dependent chain: the two-stream plan 4
+  // measured the same as plan 2); CTAs beyond one per SM run in further waves; key chunks add a merge kernel (~8).
+  const int key_tiles = max_vis > 0 ? (max_vis + KT - 1) / KT : 1;
+  const bool block_step = max_nq > 0 && max_nq <= 2 * tq;          // every row has one work item of up to two Q tiles
+  auto waves = [&](long long ctas) { return (double)((ctas + num_sms - 1) / num_sms); };
+  int plan = 1, chunks = 1;
+  if (block_step && max_vis > 0) {
+    double best = waves(items) * (8.0 + 1.3 * key_tiles);
+    const int max_chunks = scratch ? 4 : 1;
+    for (int c = 1; c <= max_chunks; ++c) {
+      if (c > 1 && ((size_t)c * M * ((size_t)hq * DH + 2 * hq) > scratch_floats || key_tiles / c < 4)) break;
+      const double cost = waves(2 * items * c) * (8.0 + 0.7 * ((key_tiles + c - 1) / c)) + (c > 1 ? 8.0 : 0.0);
+      if (cost < best) { best = cost; plan = 2; chunks = c; }
+    }
   }
+  if (env_plan >= 1 && env_plan <= 4) { plan = env_plan; if (plan == 1) chunks = 1; }
   if (env_chunks >= 1 && plan != 1 && scratch &&
       (size_t)env_chunks * M * ((size_t)hq * DH + 2 * hq) <= scratch_floats)
     chunks = env_chunks;
@@ -562,15 +648,16 @@ cudaError_t launch_attention_tc(const bf16* qkv, const bf16* kc, const bf16* vc,
   p.part_o = scratch;
   p.part_ml = reinterpret_cast<float2*>(scratch + (size_t)chunks * M * hq * DH);
   cudaError_t r;
-  if (plan == 3)
-    r = launch_pdl(k_attention_tc<1, 2>, dim3(2 * n_tiles, hkv, chunks), dim3(threads_for(1)), (size_t)smem_for(1, 2),
-                   s, mq, mk, mv, p);
+  const dim3 grid1(2 * n_tiles, hkv, chunks);
+  if (plan == 4)
+    r = launch_pdl(k_attention_tc<2, 4, true>, grid1, dim3(threads_for(2)), (size_t)smem_for(1, 4), s, mq, mk, mv, p);
+  else if (plan == 3)
+    r = launch_pdl(k_attention_tc<1, 2, false>, grid1, dim3(threads_for(1)), (size_t)smem_for(1, 2), s, mq, mk, mv, p);
   else if (plan == 2)
-    r = launch_pdl(k_attention_tc<1, 4>, dim3(2 * n_tiles, hkv, chunks), dim3(threads_for(1)), (size_t)smem_for(1, 4),
-                   s, mq, mk, mv, p);
+    r = launch_pdl(k_attention_tc<1, 4, false>, grid1, dim3(threads_for(1)), (size_t)smem_for(1, 4), s, mq, mk, mv, p);
   else
-    r = launch_pdl(k_attention_tc<2, 4>, dim3(n_tiles, hkv, 1), dim3(threads_for(2)), (size_t)smem_for(2, 4), s, mq, mk,
-                   mv, p);
+    r = launch_pdl(k_attention_tc<2, 4, false>, dim3(n_tiles, hkv, 1), dim3(threads_for(2)), (size_t)smem_for(2, 4), s,
+                   mq, mk, mv, p);
   if (r != cudaSuccess || chunks == 1) return r;
   return launch_pdl(k_attention_tc_combine, dim3(M), dim3(256), 0, s, (const float*)p.part_o,
                     (const float2*)p.part_ml, chunks, M, out, hq);
