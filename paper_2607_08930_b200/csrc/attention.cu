@@ -61,12 +61,7 @@ __global__ void __launch_bounds__(256, MINB) k_attention(const bf16* __restrict_
   pdl_wait();
   pdl_trigger();
   // which row owns this q-tile: largest r with cu_tile[r] <= blockIdx.x
-  int lo = 0, hi = n_rows;
-  while (hi - lo > 1) {
-    const int mid = (lo + hi) >> 1;
-    if (cu_tile[mid] <= (int)blockIdx.x) lo = mid; else hi = mid;
-  }
-  const int row = lo;
+  const int row = warp_find_row(cu_tile, n_rows, (int)blockIdx.x);
   const int t0 = cu_q[row] + ((int)blockIdx.x - cu_tile[row]) * q_tile;
   const int nt = min(q_tile, cu_q[row + 1] - t0);
   if (nt <= 0) return;

@@ -199,18 +199,14 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   const int kh = blockIdx.y;
   constexpr bool kSplit = kQTiles == 1;                     // one CTA per Q tile: two CTAs share a work item
   const int item = kSplit ? (int)blockIdx.x >> 1 : (int)blockIdx.x;
-  int lo = 0, hi = p.n_rows;
-  while (hi - lo > 1) {
-    const int mid = (lo + hi) >> 1;
-    if (p.cu_tile[mid] <= item) lo = mid; else hi = mid;
-  }
-  const int row = lo;
+  const int row = warp_find_row(p.cu_tile, p.n_rows, item);
   const int per_cta = kQTiles * p.tq;
-  const int t0 = p.cu_q[row] + (item - p.cu_tile[row]) * 2 * p.tq + (kSplit ? ((int)blockIdx.x & 1) * p.tq : 0);
-  const int nt = min(per_cta, p.cu_q[row + 1] - t0);        // query tokens of this CTA (CTA-uniform)
+  const int cq0 = __ldg(p.cu_q + row), cq1 = __ldg(p.cu_q + row + 1), ct0 = __ldg(p.cu_tile + row);
+  const int vis = __ldg(p.vis + row);
+  const int kvb = __ldg(p.kv_base + row);
+  const int t0 = cq0 + (item - ct0) * 2 * p.tq + (kSplit ? ((int)blockIdx.x & 1) * p.tq : 0);
+  const int nt = min(per_cta, cq1 - t0);                    // query tokens of this CTA (CTA-uniform)
   const int n_qt = nt <= 0 ? 0 : (nt > p.tq ? 2 : 1);       // Q tiles in use
-  const int vis = p.vis[row];
-  const int kvb = p.kv_base[row];
   // key tiles of this CTA's chunk: [kt0, kt0 + n_tiles) of the row's ceil(vis / KT)
   const int tiles_all = (vis + KT - 1) / KT;
   const int per_chunk = (tiles_all + p.chunks - 1) / p.chunks;
@@ -490,6 +486,7 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 }
 
 // Merges the key chunks of every (token, head): out = sum_c w_c o_c / sum_c w_c l_c with w_c = 2^(m_c - max m).
+constexpr int kMaxChunks = 4;
 __global__ void __launch_bounds__(256) k_attention_tc_combine(const float* __restrict__ part_o,
                                                               const float2* __restrict__ part_ml, int chunks, int M,
                                                               bf16* __restrict__ out, int hq) {
@@ -499,22 +496,28 @@ __global__ void __launch_bounds__(256) k_attention_tc_combine(const float* __res
   const int out_ld = hq * DH;
   for (int u = threadIdx.x; u < out_ld / 4; u += 256) {
     const int h = (4 * u) / DH;
+    // every load of this element first (independent), then the arithmetic
+    float2 ml[kMaxChunks];
+    float4 ov[kMaxChunks];
+#pragma unroll
+    for (int c = 0; c < kMaxChunks; ++c)
+      if (c < chunks) {
+        ml[c] = part_ml[((size_t)c * M + t) * hq + h];
+        ov[c] = *reinterpret_cast<const float4*>(part_o + ((size_t)c * M + t) * out_ld + 4 * u);
+      }
     float mmax = -INFINITY;
-    for (int c = 0; c < chunks; ++c) {
-      const float2 ml = part_ml[((size_t)c * M + t) * hq + h];
-      if (ml.y > 0.f) mmax = fmaxf(mmax, ml.x);
-    }
+#pragma unroll
+    for (int c = 0; c < kMaxChunks; ++c)
+      if (c < chunks && ml[c].y > 0.f) mmax = fmaxf(mmax, ml[c].x);
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     float L = 0.f;
-    for (int c = 0; c < chunks; ++c) {
-      const float2 ml = part_ml[((size_t)c * M + t) * hq + h];
-      if (ml.y > 0.f) {
-        const float w = exp2f(ml.x - mmax);
-        const float4 ov = *reinterpret_cast<const float4*>(part_o + ((size_t)c * M + t) * out_ld + 4 * u);
-        acc.x += w * ov.x; acc.y += w * ov.y; acc.z += w * ov.z; acc.w += w * ov.w;
-        L += w * ml.y;
+#pragma unroll
+    for (int c = 0; c < kMaxChunks; ++c)
+      if (c < chunks && ml[c].y > 0.f) {      // (a chunk without keys left its output slots unwritten: never used)
+        const float w = exp2f(ml[c].x - mmax);
+        acc.x += w * ov[c].x; acc.y += w * ov[c].y; acc.z += w * ov[c].z; acc.w += w * ov[c].w;
+        L += w * ml[c].y;
       }
-    }
     const float inv = 1.0f / L;
     __nv_bfloat162 a = __floats2bfloat162_rn(acc.x * inv, acc.y * inv), b = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
     uint2 o;
@@ -633,7 +636,7 @@ cudaError_t launch_attention_tc(const bf16* qkv, const bf16* kc, const bf16* vc,
   int plan = 1, chunks = 1;
   if (block_step && max_vis > 0) {
     double best = waves(items) * (8.0 + 1.3 * key_tiles);
-    const int max_chunks = scratch ? 4 : 1;
+    const int max_chunks = scratch ? kMaxChunks : 1;
     for (int c = 1; c <= max_chunks; ++c) {
       if (c > 1 && ((size_t)c * M * ((size_t)hq * DH + 2 * hq) > scratch_floats || key_tiles / c < 4)) break;
       const double cost = waves(2 * items * c) * (8.0 + 0.7 * ((key_tiles + c - 1) / c)) + (c > 1 ? 8.0 : 0.0);
@@ -641,7 +644,7 @@ cudaError_t launch_attention_tc(const bf16* qkv, const bf16* kc, const bf16* vc,
     }
   }
   if (env_plan >= 1 && env_plan <= 4) { plan = env_plan; if (plan == 1) chunks = 1; }
-  if (env_chunks >= 1 && plan != 1 && scratch &&
+  if (env_chunks >= 1 && env_chunks <= kMaxChunks && plan != 1 && scratch &&
       (size_t)env_chunks * M * ((size_t)hq * DH + 2 * hq) <= scratch_floats)
     chunks = env_chunks;
   p.chunks = chunks;

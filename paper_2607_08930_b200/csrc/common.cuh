@@ -36,6 +36,22 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
 
 typedef unsigned long long MaskWord;      // one bit per position of a block
 constexpr int kMaxBlockLen = 64;
+// Largest r in [0, n) with prefix[r] <= item, for a non-decreasing prefix with prefix[0] = 0 <= item; every lane of
+// the calling warp takes part and gets the result.  One round trip to memory per 32 rows instead of a dependent
+// load per bisection step (the callers are short kernels whose set-up time counts).
+__device__ __forceinline__ int warp_find_row(const int* __restrict__ prefix, int n, int item) {
+  const int lane = threadIdx.x & 31;
+  int below = 0;
+  for (int base = 0; base < n; base += 32) {
+    const int r = base + lane;
+    const bool le = r < n && __ldg(prefix + r) <= item;
+    const int c = __popc(__ballot_sync(0xffffffffu, le));
+    below += c;
+    if (c < 32) break;
+  }
+  return below - 1;
+}
+
 constexpr int kHdrInts = 32;
 // header words (device int32[kHdrInts], mirrored to pinned host memory once per step)
 enum Hdr {
