@@ -197,6 +197,12 @@ int bs_get_profile(bs_engine* e, double* ms, long long* launches, double* flops,
 void bs_destroy(bs_engine* e);
 const char* bs_last_error(const bs_engine* e); /* NULL engine: error of the last failed bs_init_model */
 
+/* How the library was built.  BS_BUILD_BOUNDS_CHECK: the debugging build whose gather / scatter and index kernels
+ * check every data-dependent index before use; a bad index is recorded (its access skipped) and the next call that
+ * reads the step header returns BS_E_STATE with the site in bs_last_error.  The paper has no counterpart. */
+enum { BS_BUILD_BOUNDS_CHECK = 1 };
+int bs_build_flags(void);
+
 /* ---- parity hooks (not on the timed path) ------------------------------ */
 enum {
   BS_DBG_HEADER = 0,   /* int32[32]: n_active, M, M_m, all_done, n_committed_step, n_evicted, n_admitted, ... */

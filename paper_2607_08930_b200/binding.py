@@ -14,7 +14,10 @@ import numpy as np
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libblockserve.so")
+# BS_DEBUG_LIB=1 selects the bounds-checked build (paper_2607_08930_b200.build.build(debug=True))
+DEBUG_LIB = bool(os.environ.get("BS_DEBUG_LIB"))
+LIB_PATH = os.path.join(_HERE, "libblockserve_dbg.so" if DEBUG_LIB else "libblockserve.so")
+BUILD_BOUNDS_CHECK = 1
 
 BS_OK, BS_E_ARG, BS_E_STATE, BS_E_BUDGET, BS_E_KV_FULL, BS_E_CUDA, BS_E_TIMEOUT, BS_E_UNKNOWN_REQ = (
     0, -1, -2, -3, -4, -5, -6, -7)
@@ -60,7 +63,7 @@ class BsStats(C.Structure):
 
 
 EXPORTS = ["bs_query_sizes", "bs_init_model", "bs_admit", "bs_evict_refill", "bs_denoise_step", "bs_block_done",
-           "bs_read_tokens", "bs_get_stats", "bs_set_profiling", "bs_get_profile", "bs_destroy", "bs_last_error", "bs_debug_read", "bs_debug_inject_timeout",
+           "bs_read_tokens", "bs_get_stats", "bs_set_profiling", "bs_get_profile", "bs_destroy", "bs_last_error", "bs_build_flags", "bs_debug_read", "bs_debug_inject_timeout",
            "bs_debug_force_commit", "bs_debug_snapshot", "bs_debug_restore", "bs_op_gemm",
            "bs_op_rmsnorm", "bs_op_rope_kv", "bs_op_rope_kv_static", "bs_op_attention_q_tile", "bs_op_attention", "bs_op_confidence",
            "bs_op_lm_head_confidence", "bs_op_lm_head_confidence_scratch_bytes"]
@@ -92,6 +95,7 @@ def lib() -> C.CDLL:
         L.bs_destroy.restype = None
         L.bs_last_error.argtypes = [vp]
         L.bs_last_error.restype = C.c_char_p
+        L.bs_build_flags.argtypes = []
         L.bs_debug_read.argtypes = [vp, i, i, i, vp, C.c_size_t, C.POINTER(C.c_size_t)]
         L.bs_debug_inject_timeout.argtypes = [vp]
         L.bs_debug_force_commit.argtypes = [vp, i, C.c_ulonglong, vp]

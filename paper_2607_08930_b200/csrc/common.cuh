@@ -52,6 +52,22 @@ __device__ __forceinline__ int warp_find_row(const int* __restrict__ prefix, int
   return below - 1;
 }
 
+// Bounds-checked build (-DBS_BOUNDS_CHECK, `build(debug=True)`): the data-dependent indices of the gather / scatter
+// and index kernels are checked before use; a bad one records its site (100 + site number) in the engine's error word
+// and the access is skipped, so the run continues and the host reports BS_E_STATE with the site.  The regular build
+// compiles the checks away.
+#ifdef BS_BOUNDS_CHECK
+#define BS_INDEX_OK(cond, errword, site) ((cond) ? true : (atomicMax((errword), 100 + (site)), false))
+constexpr int kBoundsCheck = 1;
+#else
+#define BS_INDEX_OK(cond, errword, site) (true)
+constexpr int kBoundsCheck = 0;
+#endif
+enum BoundsSite {
+  SITE_EMBED = 1, SITE_FILL_TOKENS = 2, SITE_ROPE_KV = 3, SITE_FINISH_QKV = 4, SITE_COMMIT = 5, SITE_INDEX = 6,
+  SITE_SCHED = 7, SITE_NORM_GATHER = 8
+};
+
 constexpr int kHdrInts = 32;
 // header words (device int32[kHdrInts], mirrored to pinned host memory once per step)
 enum Hdr {
@@ -98,10 +114,17 @@ cudaError_t launch_fill_tokens(const DevState& st, int parity, int M, cudaStream
 cudaError_t launch_force_commit(const DevState& st, int row, MaskWord bits, const int* tokens, cudaStream_t s);
 
 cudaError_t launch_embed(const DevState& st, const bf16* embed, float* x, int M, int d, cudaStream_t s);
+// `limits` (nullable): what the bounds-checked build compares gather / scatter indices with.
+struct IndexLimits {
+  int max_pos;          // rows of the RoPE table / largest position id + 1
+  long long kv_rows;    // rows of the K and V caches
+  int x_rows;           // rows of the gathered activation buffer
+  int* error_word;
+};
 cudaError_t launch_rmsnorm(const float* x, const int* idx, const bf16* w, bf16* y, int M, int d, float eps,
-                           cudaStream_t s);
+                           cudaStream_t s, const IndexLimits* limits = nullptr);
 cudaError_t launch_rope_kv(bf16* qkv, const int* tok_pos, const int* tok_kv, bf16* kc, bf16* vc, int M, int hq,
-                           int hkv, int dh, const float* cos_sin, cudaStream_t s);
+                           int hkv, int dh, const float* cos_sin, cudaStream_t s, const IndexLimits* limits = nullptr);
 // scratch (nullable): fp32 partial results when the keys of a work item are split over several CTAs.
 cudaError_t launch_attention(const bf16* qkv, const bf16* kc, const bf16* vc, bf16* out, const int* cu_q,
                              const int* cu_tile, const int* kv_base, const int* vis, int n_rows, int n_tiles, int M,
@@ -152,7 +175,7 @@ cudaError_t launch_gemm_partial(const bf16* A, int lda, const bf16* W, int M, in
 // q/k/v = bf16(sum of partials); RoPE on q, k at the token's position id; q -> qkv buffer, k / v -> cache rows.
 cudaError_t launch_finish_qkv_rope(const float* partial, int splits, int M, bf16* qkv, const int* tok_pos,
                                    const int* tok_kv, bf16* kc, bf16* vc, int hq, int hkv, int dh,
-                                   const float* cos_sin, cudaStream_t s);
+                                   const float* cos_sin, cudaStream_t s, const IndexLimits* limits = nullptr);
 // x += sum of partials; if w: h = bf16(RMSNorm(x) * w).
 cudaError_t launch_finish_residual_norm(const float* partial, int splits, int M, int d, float* x, const bf16* w,
                                         bf16* h, float eps, cudaStream_t s);

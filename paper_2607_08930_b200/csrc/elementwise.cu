@@ -18,8 +18,13 @@ __global__ void k_embed(DevState st, const bf16* __restrict__ embed, float* __re
   pdl_trigger();
   const int t = blockIdx.x;
   if (t >= M) return;
-  const int slot = st.row_slot[st.tok_row[t]];
-  const int id = st.tokens[(size_t)slot * st.max_row_tokens + st.tok_pos[t]];
+  const int trow = st.tok_row[t], tpos = st.tok_pos[t];
+  if (!BS_INDEX_OK(trow >= 0 && trow < st.max_batch && tpos >= 0 && tpos < st.max_row_tokens, st.hdr + H_ERROR, SITE_EMBED))
+    return;
+  const int slot = st.row_slot[trow];
+  if (!BS_INDEX_OK(slot >= 0 && slot < st.max_requests, st.hdr + H_ERROR, SITE_EMBED)) return;
+  const int id = st.tokens[(size_t)slot * st.max_row_tokens + tpos];
+  if (!BS_INDEX_OK(id >= 0 && id < st.vocab, st.hdr + H_ERROR, SITE_EMBED)) return;
   const uint4* src = reinterpret_cast<const uint4*>(embed + (size_t)id * d);
   float4* dst = reinterpret_cast<float4*>(x + (size_t)t * d);
   for (int c = threadIdx.x; c < d / 8; c += blockDim.x) {
@@ -34,12 +39,14 @@ __global__ void k_embed(DevState st, const bf16* __restrict__ embed, float* __re
 
 // y[m, :] = bf16(w * x[row, :] * rsqrt(mean(x^2) + eps)); one CTA per output row.
 __global__ void __launch_bounds__(256) k_rmsnorm(const float* __restrict__ x, const int* __restrict__ idx,
-                                                 const bf16* __restrict__ w, bf16* __restrict__ y, int d, float eps) {
+                                                 const bf16* __restrict__ w, bf16* __restrict__ y, int d, float eps,
+                                                 IndexLimits lim) {
   __shared__ float red[8];
   pdl_wait();
   pdl_trigger();
   const int m = blockIdx.x;
   const int row = idx ? idx[m] : m;
+  if (lim.error_word && !BS_INDEX_OK(row >= 0 && row < lim.x_rows, lim.error_word, SITE_NORM_GATHER)) return;
   const float4* src = reinterpret_cast<const float4*>(x + (size_t)row * d);
   float ss = 0.f;
   for (int c = threadIdx.x; c < d / 4; c += 256) {
@@ -74,11 +81,14 @@ __global__ void __launch_bounds__(256) k_rmsnorm(const float* __restrict__ x, co
 __global__ void __launch_bounds__(256) k_rope_kv(bf16* __restrict__ qkv, const int* __restrict__ tok_pos,
                                                  const int* __restrict__ tok_kv, bf16* __restrict__ kc,
                                                  bf16* __restrict__ vc, int hq, int hkv, int dh,
-                                                 const float2* __restrict__ cos_sin) {
+                                                 const float2* __restrict__ cos_sin, IndexLimits lim) {
   pdl_wait();
   pdl_trigger();
   const int t = blockIdx.x;
   const int pos = tok_pos[t];
+  if (lim.error_word && !BS_INDEX_OK(pos >= 0 && pos < lim.max_pos && tok_kv[t] >= 0 && tok_kv[t] < lim.kv_rows,
+                                     lim.error_word, SITE_ROPE_KV))
+    return;
   const size_t kvrow = (size_t)tok_kv[t];
   const int half = dh / 2;
   bf16* base = qkv + (size_t)t * (hq + 2 * hkv) * dh;
@@ -251,10 +261,13 @@ __global__ void __launch_bounds__(128) k_finish_qkv_rope(const float* __restrict
                                                          bf16* __restrict__ qkv, const int* __restrict__ tok_pos,
                                                          const int* __restrict__ tok_kv, bf16* __restrict__ kc,
                                                          bf16* __restrict__ vc, int hq, int hkv, int dh,
-                                                         const float2* __restrict__ cos_sin) {
+                                                         const float2* __restrict__ cos_sin, IndexLimits lim) {
   pdl_wait();
   pdl_trigger();
   const int t = blockIdx.x;
+  if (lim.error_word && !BS_INDEX_OK(tok_pos[t] >= 0 && tok_pos[t] < lim.max_pos && tok_kv[t] >= 0 &&
+                                         tok_kv[t] < lim.kv_rows, lim.error_word, SITE_FINISH_QKV))
+    return;
   const int n_heads = hq + 2 * hkv;
   const int N = n_heads * dh, half = dh / 2;
   const size_t slice = (size_t)M * N;
@@ -382,14 +395,17 @@ __global__ void __launch_bounds__(256) k_finish_residual_norm(const float* __res
   }
 }
 
+static IndexLimits limits_or_none(const IndexLimits* limits) {
+  return (limits && kBoundsCheck) ? *limits : IndexLimits{0, 0, 0, nullptr};
+}
 cudaError_t launch_finish_qkv_rope(const float* partial, int splits, int M, bf16* qkv, const int* tok_pos,
                                    const int* tok_kv, bf16* kc, bf16* vc, int hq, int hkv, int dh,
-                                   const float* cos_sin, cudaStream_t s) {
+                                   const float* cos_sin, cudaStream_t s, const IndexLimits* limits) {
   if (M <= 0) return cudaSuccess;
   if (splits > kMaxSplits || dh % 8) return cudaErrorInvalidValue;
   dim3 grid(M, (hq + 2 * hkv + kHeadsPerBlock - 1) / kHeadsPerBlock);
   return launch_pdl(k_finish_qkv_rope, grid, dim3(128), 0, s, partial, splits, M, qkv, tok_pos, tok_kv, kc, vc, hq, hkv,
-                    dh, reinterpret_cast<const float2*>(cos_sin));
+                    dh, reinterpret_cast<const float2*>(cos_sin), limits_or_none(limits));
 }
 cudaError_t launch_finish_residual_norm(const float* partial, int splits, int M, int d, float* x, const bf16* w,
                                         bf16* h, float eps, cudaStream_t s) {
@@ -403,15 +419,15 @@ cudaError_t launch_embed(const DevState& st, const bf16* embed, float* x, int M,
   return launch_pdl(k_embed, dim3(M), dim3(128), 0, s, st, embed, x, M, d);
 }
 cudaError_t launch_rmsnorm(const float* x, const int* idx, const bf16* w, bf16* y, int M, int d, float eps,
-                           cudaStream_t s) {
+                           cudaStream_t s, const IndexLimits* limits) {
   if (M <= 0) return cudaSuccess;
-  return launch_pdl(k_rmsnorm, dim3(M), dim3(256), 0, s, x, idx, w, y, d, eps);
+  return launch_pdl(k_rmsnorm, dim3(M), dim3(256), 0, s, x, idx, w, y, d, eps, limits_or_none(limits));
 }
 cudaError_t launch_rope_kv(bf16* qkv, const int* tok_pos, const int* tok_kv, bf16* kc, bf16* vc, int M, int hq,
-                           int hkv, int dh, const float* cos_sin, cudaStream_t s) {
+                           int hkv, int dh, const float* cos_sin, cudaStream_t s, const IndexLimits* limits) {
   if (M <= 0) return cudaSuccess;
   return launch_pdl(k_rope_kv, dim3(M), dim3(256), 0, s, qkv, tok_pos, tok_kv, kc, vc, hq, hkv, dh,
-                    reinterpret_cast<const float2*>(cos_sin));
+                    reinterpret_cast<const float2*>(cos_sin), limits_or_none(limits));
 }
 cudaError_t launch_confidence(const float* logits, int n_rows, int vocab, int mask_id, int* tok, float* conf,
                               cudaStream_t s) {

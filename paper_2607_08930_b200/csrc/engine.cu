@@ -238,6 +238,8 @@ int sync_header(bs_engine* e) {
       e->pending.erase(e->pending.begin(), e->pending.begin() + std::min<size_t>(adm, e->pending.size()));
     }
     e->hdr_from_step = false;
+    if (e->hdr[H_ERROR] >= 100)
+      return fail(e, BS_E_STATE, "bounds-checked build: index out of range at site " + std::to_string(e->hdr[H_ERROR] - 100));
     if (e->hdr[H_ERROR] != 0) return fail(e, BS_E_TIMEOUT, "a bounded device-side wait ran out");
   }
   return BS_OK;
@@ -454,6 +456,7 @@ int bs_denoise_step(bs_engine* e, int* n_committed) {
   e->stats.active_row_steps += n_rows;
   const int d = c.d_model, hq = c.n_q_heads, hkv = c.n_kv_heads, dh = c.head_dim;
   const int qkv_n = (hq + 2 * hkv) * dh;
+  const IndexLimits lim{c.max_row_tokens, c.kv_capacity_tokens, M, st.hdr + H_ERROR};     // read by the checked build
 
   const double dM = (double)M, dd = (double)d, dq = (double)qkv_n, dhq = (double)hq * dh, df = (double)c.d_ffn;
   const double kv_rows = (double)e->hdr[H_SUM_KV];
@@ -480,7 +483,8 @@ int bs_denoise_step(bs_engine* e, int* n_committed) {
       KL(e, launch_gemm_partial(ws.h, d, e->wqkv[l], M, qkv_n, d, e->gemm_scratch, s, &sp));
       prof_work(e, BS_FAM_GEMM_QKV, 1, 2.0 * dM * dq * dd, 2.0 * (dq * dd + dM * dd) + 4.0 * sp * dM * dq);
       prof_mark(e, BS_FAM_ROPE_KV);
-      KL(e, launch_finish_qkv_rope(ws.partial, sp, M, ws.qkv, st.tok_pos, st.tok_kv, kc, vc, hq, hkv, dh, ws.rope, s));
+      KL(e, launch_finish_qkv_rope(ws.partial, sp, M, ws.qkv, st.tok_pos, st.tok_kv, kc, vc, hq, hkv, dh, ws.rope, s,
+                                   &lim));
       prof_work(e, BS_FAM_ROPE_KV, 1, 0, 4.0 * sp * dM * dq + 2.0 * dM * dq);
       prof_mark(e, BS_FAM_ATTENTION);
       KL(e, launch_attention(ws.qkv, kc, vc, ws.attn, st.cu_q[parity], st.cu_tile[parity], st.row_kv_base,
@@ -516,7 +520,7 @@ int bs_denoise_step(bs_engine* e, int* n_committed) {
     KL(e, launch_gemm(ws.h, d, e->wqkv[l], nullptr, ws.qkv, qkv_n, M, qkv_n, d, 0, nullptr, e->gemm_scratch, s));
     prof_work(e, BS_FAM_GEMM_QKV, 1, 2.0 * dM * dq * dd, 2.0 * (dq * dd + dM * dd + dM * dq));
     prof_mark(e, BS_FAM_ROPE_KV);
-    KL(e, launch_rope_kv(ws.qkv, st.tok_pos, st.tok_kv, kc, vc, M, hq, hkv, dh, ws.rope, s));
+    KL(e, launch_rope_kv(ws.qkv, st.tok_pos, st.tok_kv, kc, vc, M, hq, hkv, dh, ws.rope, s, &lim));
     prof_work(e, BS_FAM_ROPE_KV, 1, 0, 2.0 * dM * (dq + (double)(hq + 2 * hkv) * dh));
     prof_mark(e, BS_FAM_ATTENTION);
     KL(e, launch_attention(ws.qkv, kc, vc, ws.attn, st.cu_q[parity], st.cu_tile[parity], st.row_kv_base, st.row_vis,
@@ -546,7 +550,7 @@ int bs_denoise_step(bs_engine* e, int* n_committed) {
   // final norm on the still-masked rows only, LM head scaled by alpha_i, confidence / argmax, commit
   const double dMm = (double)Mm, dV = (double)c.vocab;
   prof_mark(e, BS_FAM_EMBED_NORM);
-  KL(e, launch_rmsnorm(ws.x, st.lm_tok[parity], e->final_norm, ws.hf, Mm, d, c.rms_eps, s));
+  KL(e, launch_rmsnorm(ws.x, st.lm_tok[parity], e->final_norm, ws.hf, Mm, d, c.rms_eps, s, &lim));
   prof_work(e, BS_FAM_EMBED_NORM, 1, 0, 6.0 * dMm * dd);
   // LM head with the confidence pass in its epilogue: per (32 vocabulary entries, row) maximum / sum of exponentials
   // / argmax of the alpha-scaled logits, merged per row in two small stages (the second one inside the commit
@@ -648,6 +652,8 @@ void bs_destroy(bs_engine* e) {
 }
 
 const char* bs_last_error(const bs_engine* e) { return e ? e->err.c_str() : g_init_error.c_str(); }
+
+int bs_build_flags(void) { return kBoundsCheck ? BS_BUILD_BOUNDS_CHECK : 0; }
 
 int bs_debug_read(bs_engine* e, int what, int arg0, int arg1, void* host_buf, size_t cap, size_t* n_out) {
   if (!e || !host_buf) return BS_E_ARG;

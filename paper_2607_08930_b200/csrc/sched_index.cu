@@ -97,6 +97,8 @@ __device__ void build_index(const DevState& st, int parity, int n, int* smi) {
     st.cu_tile[parity][i] = et;
   }
   if (i == 0) {
+    (void)BS_INDEX_OK(tot_q <= st.kv_capacity && tot_m <= st.max_batch * st.L && n <= st.max_batch, st.hdr + H_ERROR,
+                      SITE_INDEX);
     st.cu_q[parity][n] = tot_q;
     st.lm_base[parity][n] = tot_m;
     st.cu_tile[parity][n] = tot_t;
@@ -122,6 +124,9 @@ __device__ void build_index(const DevState& st, int parity, int n, int* smi) {
         const int slot = st.row_slot[r];
         const int lo = st.req_p[slot] + st.req_b[slot] * st.L;
         const int k = st.lm_base[parity][r] + __popcll(mask & ((1ull << j) - 1ull));
+        if (!BS_INDEX_OK(k >= 0 && k < st.max_batch * st.L && slot >= 0 && slot < st.max_requests, st.hdr + H_ERROR,
+                         SITE_INDEX))
+          continue;
         st.lm_tok[parity][k] = st.cu_q[parity][r] + ((st.row_s[r] == 0 && st.row_refresh[r] != 0) ? lo + j : j);
         st.lm_row[parity][k] = r;
         st.lm_slot[parity][k] = j;
@@ -206,6 +211,7 @@ __device__ void sched_body(const DevState& st, bool only_done) {
     const int n = s_n, head = s_head;
     if (s_stop || head >= qlen || n >= st.max_batch) break;
     const int c = st.queue[head];
+    if (!BS_INDEX_OK(c >= 0 && c < st.max_requests, st.hdr + H_ERROR, SITE_SCHED)) break;     // (uniform: all threads read c)
     const long long wc = (long long)st.req_p[c] + (long long)(st.req_b[c] + 1) * L;
     const long long w2 = wc > s_w ? wc : s_w;
     const long long need = (long long)st.req_p[c] + st.req_g[c];
@@ -330,6 +336,9 @@ __global__ void __launch_bounds__(kSchedThreads) k_commit_index(DevState st) {
       const bool sel = k < nm && (conf[h] > st.tau || picked[h]);
       if (sel) {
         const int lo = st.req_p[slot] + st.req_b[slot] * st.L;
+        if (!BS_INDEX_OK(lo + bit[h] < st.req_p[slot] + st.req_g[slot] && lo + bit[h] < st.max_row_tokens &&
+                             tok[h] >= 0 && tok[h] < st.vocab && tok[h] != st.mask_id, st.hdr + H_ERROR, SITE_COMMIT))
+          continue;
         st.tokens[(size_t)slot * st.max_row_tokens + lo + bit[h]] = tok[h];
         if (bit[h] < 32) lo_bits |= 1u << bit[h]; else hi_bits |= 1u << (bit[h] - 32);
       }
@@ -400,8 +409,13 @@ __global__ void k_fill_tokens(DevState st, int parity, int M) {
     }
     const int r = lo;
     const int slot = st.row_slot[r];
+    if (!BS_INDEX_OK(slot >= 0 && slot < st.max_requests, st.hdr + H_ERROR, SITE_FILL_TOKENS)) continue;
     const int first = (st.row_s[r] == 0 && st.row_refresh[r] != 0) ? 0 : st.req_p[slot] + st.req_b[slot] * st.L;
     const int pos = first + (t - cu[r]);
+    if (!BS_INDEX_OK(pos >= 0 && pos < st.req_p[slot] + st.req_g[slot] && pos < st.max_row_tokens &&
+                         (long long)st.row_kv_base[r] + pos < st.kv_capacity && t < st.kv_capacity, st.hdr + H_ERROR,
+                     SITE_FILL_TOKENS))
+      continue;
     st.tok_row[t] = r;
     st.tok_pos[t] = pos;                 // logical position id: 0 = first prompt token of the request
     st.tok_kv[t] = st.row_kv_base[r] + pos;

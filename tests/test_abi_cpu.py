@@ -72,3 +72,15 @@ def test_init_fails_loudly_without_a_device(B):
     h = C.c_void_p()
     rc = B.lib().bs_init_model(C.byref(cfg), C.byref(w), 256, 256, 256, None, C.byref(h))
     assert rc == B.BS_E_CUDA and b"no CUDA device" in B.lib().bs_last_error(None)
+
+
+def test_bounds_checked_build_exports_the_same_interface():
+    """The debugging build compiles from the same sources and must export every declared symbol too."""
+    import ctypes
+    from paper_2607_08930_b200 import build, binding
+    lib = ctypes.CDLL(build.build(debug=True))
+    for name in binding.EXPORTS:
+        assert hasattr(lib, name), name
+    lib.bs_build_flags.argtypes = []
+    assert lib.bs_build_flags() == binding.BUILD_BOUNDS_CHECK
+    assert binding.lib().bs_build_flags() == (binding.BUILD_BOUNDS_CHECK if binding.DEBUG_LIB else 0)

@@ -511,3 +511,26 @@ def test_refresh_at_admission_only_in_lockstep(B, shape_name, async_advance):
             if eng.block_done():
                 break
         eng.snapshot()          # rows are active and their cache is state: refused
+
+
+def test_build_flags_name_the_loaded_library(B):
+    assert B.lib().bs_build_flags() == (B.BUILD_BOUNDS_CHECK if B.DEBUG_LIB else 0)
+
+
+def test_bounds_checked_build_runs_the_lockstep_cases_clean(B):
+    """The debugging build (-DBS_BOUNDS_CHECK: every data-dependent index of the gather / scatter and index kernels is
+    compared with its limit before use, a bad one is recorded and reported as BS_E_STATE) runs a selection of the
+    lockstep cases in a child process: no index may be flagged, and results must still match the oracle."""
+    import os
+    import subprocess
+    import sys
+    if B.DEBUG_LIB:
+        pytest.skip("already running on the bounds-checked build")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    pick = ("build_flags or config1_full_lockstep or async_advance_stream or refresh_at_admission or "
+            "mini_gqa_stream or other_block_lengths or check_eos")
+    r = subprocess.run([sys.executable, "-m", "pytest", os.path.join(root, "tests", "test_engine_gpu.py"), "-q", "-x",
+                        "-m", "gpu", "-p", "no:cacheprovider", "-k", pick], env=dict(os.environ, BS_DEBUG_LIB="1"),
+                       capture_output=True, text=True, timeout=1800)
+    assert r.returncode == 0, r.stdout[-3000:] + r.stderr[-2000:]
+    assert " passed" in r.stdout and "skipped" not in r.stdout.splitlines()[-1]
