@@ -272,7 +272,9 @@ int bs_op_rope_kv(void* qkv, const int* tok_pos, const int* tok_kv, void* kcache
  * through any library.  The first call on each device looks up the array's device address (one-time set-up,
  * with that device current): make it before any stream capture.  All calls share the one table, which keeps
  * the previous call's contents and is rewritten for [0, max_pos) by each call: two calls whose kernels can
- * overlap on the GPU (different streams, no ordering between them) race on it. */
+ * overlap on the GPU (different streams, no ordering between them) race on it.  Every tok_pos[t] must lie in
+ * [0, max_pos): the kernel does not check it, and a larger position would read entries an earlier call left
+ * (or, beyond BS_ROPE_STATIC_MAX_FLOATS / head_dim, memory outside the table). */
 #define BS_ROPE_STATIC_MAX_FLOATS (512 * 1024)
 int bs_op_rope_kv_static(void* qkv, const int* tok_pos, const int* tok_kv, void* kcache, void* vcache, int M,
                          int n_q_heads, int n_kv_heads, int head_dim, float theta, int max_pos, void* stream);

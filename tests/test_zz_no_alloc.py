@@ -22,7 +22,9 @@ def B():
 def _case(B, seed, hq, hkv, dh, theta, max_pos, M, rows):
     rng = np.random.default_rng(seed)
     qkv = torch.from_numpy(rng.normal(size=(M, (hq + 2 * hkv) * dh)).astype(np.float32)).to(torch.bfloat16).cuda()
-    pos = torch.from_numpy(rng.integers(0, max_pos, size=M).astype(np.int32)).cuda()
+    pos_h = rng.integers(0, max_pos, size=M).astype(np.int32)
+    pos_h[:2] = (max_pos - 1, 0)              # the table's last entry must be this call's own, not an earlier call's
+    pos = torch.from_numpy(pos_h).cuda()
     kvrow = torch.from_numpy(rng.permutation(rows)[:M].astype(np.int32)).cuda()
     ref_q = qkv.clone()
     ref_k = torch.zeros(rows, hkv, dh, dtype=torch.bfloat16, device="cuda")
