@@ -290,26 +290,36 @@ def run_ours(args):
         print(json.dumps({"metric": METRIC, "value": value, "unit": UNIT, "ms_per_step": ms_total / args.steps,
                           "e2e": e2e_value, "note": "per-family timers off"}))
         return
-    gemm_ms = sum(prof[f]["ms"] for f in GEMM_FAMILIES)
-    gemm_fl = sum(prof[f]["flops"] for f in GEMM_FAMILIES)
-    gemm_by = sum(prof[f]["bytes"] for f in GEMM_FAMILIES)
-    gemm_n = sum(prof[f]["launches"] for f in GEMM_FAMILIES)
     prof_ms = sum(v["ms"] for v in prof.values())
-    t_tensor = gemm_fl / (pk["bf16_tflops_sustained"] * 1e12)
-    t_hbm = gemm_by / (pk["hbm_gbs"] * 1e9)
-    if t_tensor >= t_hbm:
-        roof = {"bound": "tensor", "achieved": gemm_fl / (gemm_ms * 1e-3) / 1e12, "peak": pk["bf16_tflops_sustained"],
-                "unit": "TFLOP/s"}
-    else:
-        roof = {"bound": "hbm", "achieved": gemm_by / (gemm_ms * 1e-3) / 1e9, "peak": pk["hbm_gbs"], "unit": "GB/s"}
-    roof.update(frac=roof["achieved"] / roof["peak"], traffic=NCU_TRAFFIC_BYTES_PER_LAUNCH, peak_kind=pk_kind,
-                kernel="projection GEMM (all five shapes), from one extra job with per-family timers",
-                profiled_job_ms=prof_ms_job, launches=gemm_n,
-                avg_launch_us=1e3 * gemm_ms / max(gemm_n, 1), share_of_step=gemm_ms / max(prof_ms, 1e-9),
-                # the same work over (this kernel's share of the profiled job) x (the un-profiled job time)
-                achieved_at_timed_speed=(roof["achieved"] * gemm_ms /
-                                         max(gemm_ms / max(prof_ms, 1e-9) * ms_total / args.steps, 1e-9)),
-                tflops=gemm_fl / (gemm_ms * 1e-3) / 1e12, gbs=gemm_by / (gemm_ms * 1e-3) / 1e9)
+
+    def roof_of(fams, label):
+        """Roofline figures of a set of kernel families: algorithmic flops and bytes of their launches over the device
+        time the family timers measured for them."""
+        ms = sum(prof[f]["ms"] for f in fams)
+        fl = sum(prof[f]["flops"] for f in fams)
+        by = sum(prof[f]["bytes"] for f in fams)
+        n = sum(prof[f]["launches"] for f in fams)
+        if fl / (pk["bf16_tflops_sustained"] * 1e12) >= by / (pk["hbm_gbs"] * 1e9):
+            r = {"bound": "tensor", "achieved": fl / (ms * 1e-3) / 1e12, "peak": pk["bf16_tflops_sustained"],
+                 "unit": "TFLOP/s"}
+        else:
+            r = {"bound": "hbm", "achieved": by / (ms * 1e-3) / 1e9, "peak": pk["hbm_gbs"], "unit": "GB/s"}
+        r.update(frac=r["achieved"] / r["peak"], peak_kind=pk_kind, kernel=label, launches=n,
+                 avg_launch_us=1e3 * ms / max(n, 1), share_of_step=ms / max(prof_ms, 1e-9),
+                 # the same work over (these kernels' share of the profiled job) x (the un-profiled job time)
+                 achieved_at_timed_speed=r["achieved"] * prof_ms_job / max(ms_total / args.steps, 1e-9),
+                 tflops=fl / (ms * 1e-3) / 1e12, gbs=by / (ms * 1e-3) / 1e9)
+        return r
+
+    # the dominant kernel: the SwiGLU gate/up projection (the largest share of every workload's device time); the ncu
+    # traffic figure below is a capture of that same kernel
+    dominant = max(GEMM_FAMILIES, key=lambda f: prof[f]["ms"])
+    roof = roof_of([dominant], {"gemm_gate_up": "projection GEMM, SwiGLU gate/up (k_gemm_pair<3> / k_gemm_tc<3>)"}
+                   .get(dominant, f"projection GEMM ({dominant})") + ", from one extra job with per-family timers")
+    roof.update(traffic=NCU_TRAFFIC_BYTES_PER_LAUNCH if dominant == "gemm_gate_up" else None,
+                traffic_note="ncu DRAM bytes of one gate/up launch at M = 256 (algorithmic 283.1 MB)",
+                profiled_job_ms=prof_ms_job)
+    roof_all = roof_of(GEMM_FAMILIES, "all five projection GEMM shapes")
     families = {f: {"ms": round(v["ms"], 3), "launches": v["launches"],
                     "tflops": round(v["flops"] / max(v["ms"], 1e-9) / 1e9, 2),
                     "gbs": round(v["bytes"] / max(v["ms"], 1e-9) / 1e6, 1)} for f, v in prof.items()}
@@ -334,6 +344,7 @@ def run_ours(args):
                                     "own block completes; not part of the headline value"},
         "clocks": clocks,
         "roofline": roof,
+        "roofline_all_gemms": roof_all,
         "families": families,
     }
     if world == 1 and not args.no_cpu_baseline:

@@ -19,7 +19,7 @@ def B():
     return binding
 
 
-def _case(B, seed, hq, hkv, dh, theta, max_pos, M, rows):
+def _case(B, seed, hq, hkv, dh, theta, max_pos, M, rows, check_device_free=False):
     rng = np.random.default_rng(seed)
     qkv = torch.from_numpy(rng.normal(size=(M, (hq + 2 * hkv) * dh)).astype(np.float32)).to(torch.bfloat16).cuda()
     pos_h = rng.integers(0, max_pos, size=M).astype(np.int32)
@@ -34,10 +34,15 @@ def _case(B, seed, hq, hkv, dh, theta, max_pos, M, rows):
     got_k, got_v = torch.zeros_like(ref_k), torch.zeros_like(ref_v)
     torch.cuda.synchronize()
     before = torch.cuda.memory_allocated()
+    free_before = torch.cuda.mem_get_info()[0]
     rc = B.op_rope_kv_static(got_q, pos, kvrow, got_k, got_v, hq, hkv, dh, theta, max_pos)
     torch.cuda.synchronize()
     assert rc == B.BS_OK
     assert torch.cuda.memory_allocated() == before          # nothing was taken from torch's allocator
+    if check_device_free:
+        # nor from the device behind torch's back (a cudaMalloc inside the library would lower the free figure);
+        # checked on a call that is not the process's first, so that loading the kernels' code is not counted
+        assert torch.cuda.mem_get_info()[0] >= free_before
     for g, r in ((got_q, ref_q), (got_k, ref_k), (got_v, ref_v)):
         g, r = g.float().cpu().numpy(), r.float().cpu().numpy()
         assert np.abs(g - r).max() <= 8e-3 * max(np.abs(r).max(), 1e-30)    # tolerance of the RoPE parity test
@@ -47,7 +52,7 @@ def _case(B, seed, hq, hkv, dh, theta, max_pos, M, rows):
 def test_two_calls_in_a_row_match_the_regular_entry_point(B):
     _case(B, 1, hq=28, hkv=4, dh=128, theta=10000.0, max_pos=3000, M=333, rows=4000)
     # a different head_dim, base and table length right after: every entry read must have been rewritten
-    _case(B, 2, hq=4, hkv=4, dh=64, theta=500.0, max_pos=777, M=90, rows=900)
+    _case(B, 2, hq=4, hkv=4, dh=64, theta=500.0, max_pos=777, M=90, rows=900, check_device_free=True)
 
 
 def test_table_too_large_is_rejected(B):
