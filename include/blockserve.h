@@ -60,7 +60,8 @@ typedef struct {
   float tau;
   long long token_budget;
   int max_batch;                 /* <= 1024 */
-  int max_requests;              /* size of the request table for the whole stream */
+  int max_requests;              /* size of the request table: a lifetime cap - every bs_admit takes a slot for good
+                                    (finished requests stay readable until bs_destroy), slots are not recycled */
   int max_row_tokens;            /* max p_i + g_i */
   long long kv_capacity_tokens;  /* rows of the KV arena = max packed tokens of one step */
   int suffix_mode;               /* BS_SUFFIX_FULL: a row sees prompt + all g_i positions (future blocks as mask
@@ -189,8 +190,10 @@ enum {
   BS_FAM_GEMM_GATE_UP = 6,
   BS_FAM_GEMM_DOWN = 7,
   BS_FAM_GEMM_LM_HEAD = 8,
-  BS_FAM_CONFIDENCE = 9,
-  BS_FAM_COUNT = 10
+  BS_FAM_CONFIDENCE = 9,        /* merge of the LM-head epilogue's confidence partials */
+  BS_FAM_ATTENTION_REFRESH = 10, /* attention of steps that hold whole-row refreshes (compute-bound; BS_FAM_ATTENTION
+                                    then counts pure block steps only: cache streaming) */
+  BS_FAM_COUNT = 11
 };
 int bs_set_profiling(bs_engine* e, int on);
 int bs_get_profile(bs_engine* e, double* ms, long long* launches, double* flops, double* bytes);

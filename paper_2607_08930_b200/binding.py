@@ -31,7 +31,7 @@ REQ_QUEUED, REQ_ACTIVE, REQ_FINISHED = 0, 1, 2
 
 
 FAMILIES = ("index", "embed_norm", "gemm_qkv", "rope_kv", "attention", "gemm_o", "gemm_gate_up", "gemm_down",
-            "gemm_lm_head", "confidence")
+            "gemm_lm_head", "confidence", "attention_refresh")
 
 
 class BsConfig(C.Structure):

@@ -330,8 +330,14 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       if (warp_has_rows) {
         // scores -> probabilities in registers; this part overlaps the group's previous P V product
         const int key0 = (kt0 + t) * KT;
-        tmem_ld32(t_lane + b * 64, v);
-        tmem_ld32(t_lane + b * 64 + 32, v + 32);
+        {   // both halves of the tile's scores in flight before the one wait
+          unsigned raw[KT];
+          tmem_ld32_nowait(t_lane + b * 64, raw);
+          tmem_ld32_nowait(t_lane + b * 64 + 32, raw + 32);
+          tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < KT; ++j) v[j] = __uint_as_float(raw[j]);
+        }
         // eight independent chains for the row maximum and the row sum: one warp per scheduler has no other
         // warp to hide a 64-long dependent chain behind.  The maximum is taken over the raw scores (the scale
         // is positive) and the scale folded into the exponent's fma.

@@ -522,13 +522,14 @@ int bs_denoise_step(bs_engine* e, int* n_committed) {
     prof_mark(e, BS_FAM_ROPE_KV);
     KL(e, launch_rope_kv(ws.qkv, st.tok_pos, st.tok_kv, kc, vc, M, hq, hkv, dh, ws.rope, s, &lim));
     prof_work(e, BS_FAM_ROPE_KV, 1, 0, 2.0 * dM * (dq + (double)(hq + 2 * hkv) * dh));
-    prof_mark(e, BS_FAM_ATTENTION);
+    const int attn_fam = e->hdr[H_STEP_REFRESH] > 0 ? BS_FAM_ATTENTION_REFRESH : BS_FAM_ATTENTION;
+    prof_mark(e, attn_fam);
     KL(e, launch_attention(ws.qkv, kc, vc, ws.attn, st.cu_q[parity], st.cu_tile[parity], st.row_kv_base, st.row_vis,
                            n_rows, e->hdr[H_QTILES], M, e->hdr[H_MAX_VIS], max_nq, c.kv_capacity_tokens, hq, hkv, dh,
                            nullptr, 0, st.hdr + H_ERROR, s));
     // every query token of a row meets every cache row of that row: flops = 4 * dh * Hq * sum_rows(n_q * vis);
     // the host knows the sums only for pure block steps and pure refresh steps, else it reports bytes alone
-    prof_work(e, BS_FAM_ATTENTION, 1, 0, 2.0 * (2.0 * kv_rows * hkv * dh + 2.0 * dM * dhq));
+    prof_work(e, attn_fam, 1, 0, 2.0 * (2.0 * kv_rows * hkv * dh + 2.0 * dM * dhq));
     prof_mark(e, BS_FAM_GEMM_O);
     KL(e, launch_gemm(ws.attn, hq * dh, e->wo[l], nullptr, ws.x, d, M, d, hq * dh, 1, nullptr, e->gemm_scratch, s));
     prof_work(e, BS_FAM_GEMM_O, 1, 2.0 * dM * dd * dhq, 2.0 * (dd * dhq + dM * dhq) + 8.0 * dM * dd);

@@ -134,8 +134,16 @@ __device__ __forceinline__ void epilogue_row(const GemmParams& p, int split, int
     // columns of this chunk that hold tokens of this tile (the tile width is a multiple of 16, not of 32)
     const int jmax = min(min(32, p.tn - c0), p.M - t0);
     float v[32], u[32];
-    tmem_ld32(t_row + c0, v);
-    if (EPI == 3) tmem_ld32(t_row + p.acc1_off + c0, u);
+    if (EPI == 3) {     // gate and up: both loads in flight before the one wait
+      unsigned rv[32], ru[32];
+      tmem_ld32_nowait(t_row + c0, rv);
+      tmem_ld32_nowait(t_row + p.acc1_off + c0, ru);
+      tmem_ld_wait();
+#pragma unroll
+      for (int j = 0; j < 32; ++j) { v[j] = __uint_as_float(rv[j]); u[j] = __uint_as_float(ru[j]); }
+    } else {
+      tmem_ld32(t_row + c0, v);
+    }
     if (!n_ok) continue;                      // the TMEM loads above are warp-collective; the stores are not
     char* ptr = base + ((size_t)t0 * ld + n) * esize;
     if (EPI == 1) {
