@@ -29,6 +29,7 @@ using namespace tc;
 constexpr int BK = 64;                 // K elements per pipeline stage (128 bytes: one swizzle span)
 constexpr int TILE_N = 128;            // weight rows per tile (UMMA M)
 constexpr int kThreads = 192;
+constexpr int kPairThreads = 320;       // the pair kernel runs two groups of four epilogue warps (alternate token chunks)
 constexpr int kSmemBudget = 200 * 1024;
 
 struct GemmParams {
@@ -54,6 +55,7 @@ struct GemmParams {
   float2* conf_ms;   // [ceil(N / 32)][M]
   int* conf_am;      // [ceil(N / 32)][M]
   int skip;
+  int vec_store;     // bf16 output rows take 16-byte stores (ldc and N multiples of 8, C 16-byte aligned)
 };
 
 __device__ __forceinline__ void tma_load_2d(unsigned dst, const CUtensorMap* map, int c0, int c1, unsigned bar) {
@@ -100,7 +102,15 @@ __device__ __forceinline__ void issue_stage(unsigned d0, unsigned d1, unsigned a
     if (TWO) umma_lo<CG>(d1, a1_lo + 2 * k, b_lo + 2 * k, idesc, 1u);
   }
 }
-__device__ __forceinline__ float silu_f(float x) { return x / (1.0f + __expf(-x)); }
+// x·sigmoid(x) from the two special-function approximations (2^x, 1/x; relative error ~2^-21, far below the bf16
+// rounding that follows).  The IEEE division it replaces carries a slow-path branch per element, which kept the
+// compiler from interleaving the columns of a chunk and made the SwiGLU epilogue latency-bound.
+__device__ __forceinline__ float silu_f(float x) {
+  float e, r;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(x * -1.4426950408889634f));
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(1.0f + e));      // e = +inf (x << 0) gives r = 0
+  return x * r;
+}
 
 // Epilogue of one accumulator row: this thread holds output feature n for the tn tokens of token tile mt, whose
 // fp32 sums sit in TMEM at t_row (lane already selected) in columns 0 .. tn-1.  EPI: 0 bf16 store, 1 fp32 +=,
@@ -117,32 +127,73 @@ __device__ __forceinline__ void epilogue_chunk(const float* v, const float* u, c
     if (EPI == 0) *reinterpret_cast<bf16*>(q) = __float2bfloat16_rn(v[j]);
     else if (EPI == 1) *reinterpret_cast<float*>(q) = u[j] + v[j];
     else if (EPI == 2) *reinterpret_cast<float*>(q) = v[j] * __ldg(scale + j);
-    else if (EPI == 3) *reinterpret_cast<bf16*>(q) = __float2bfloat16_rn(silu_f(v[j]) * u[j]);
+    else if (EPI == 3) *reinterpret_cast<bf16*>(q) = __float2bfloat16_rn(v[j]);      // v already holds silu(gate)·up
     else *reinterpret_cast<float*>(q) = v[j];
   }
 }
-template <int EPI>
-__device__ __forceinline__ void epilogue_row(const GemmParams& p, int split, int mt, int n, bool n_ok, unsigned t_row) {
+// bf16 outputs (modes 0 and 3) leave through a per-warp shared-memory tile [32 tokens][32 features] when the output
+// rows allow 16-byte stores: a thread that stored one 2-byte element per token (32 store instructions per chunk, each
+// a 64-byte segment) instead writes four 16-byte vectors, eight token rows per warp instruction.  It matters for the
+// SwiGLU GEMM, whose epilogue is exposed (its two 256-column accumulators fill TMEM, so the tensor core waits for it).
+// `release` (may be empty) runs once, as soon as the item's last TMEM load of this warp has completed: the
+// accumulator is handed back to the MMA issuer before the last chunk's arithmetic and stores.  Returns whether it ran.
+template <int EPI, typename Release>
+__device__ __forceinline__ bool epilogue_row(const GemmParams& p, int split, int mt, int n, bool n_ok, unsigned t_row,
+                                             Release release, bf16* tile = nullptr, int c_first = 0, int c_step = 32) {
   constexpr int esize = (EPI == 0 || EPI == 3) ? 2 : 4;
   const int ld = EPI == 4 ? p.N : p.ldc;
   char* base = EPI == 4 ? reinterpret_cast<char*>(p.partial + ((size_t)split * p.M) * p.N)
                         : reinterpret_cast<char*>(p.C);
   const size_t stride = (size_t)ld * esize;
-  for (int c0 = 0; c0 < p.tn; c0 += 32) {
+  const int lane = threadIdx.x & 31;
+  // SwiGLU: the TMEM loads of the next chunk are issued before this chunk's stores, so that they are complete when
+  // the next iteration waits (tcgen05.wait::ld covers every outstanding load of the thread).
+  unsigned rv[EPI == 3 ? 32 : 1], ru[EPI == 3 ? 32 : 1];
+  bool released = false;
+  if (EPI == 3 && c_first < p.tn && mt * p.tn + c_first < p.M) {
+    tmem_ld32_nowait(t_row + c_first, rv);
+    tmem_ld32_nowait(t_row + p.acc1_off + c_first, ru);
+  }
+  for (int c0 = c_first; c0 < p.tn; c0 += c_step) {
     const int t0 = mt * p.tn + c0;
     if (t0 >= p.M) break;                     // warp-uniform
     // columns of this chunk that hold tokens of this tile (the tile width is a multiple of 16, not of 32)
     const int jmax = min(min(32, p.tn - c0), p.M - t0);
+    const int cn = c0 + c_step;
+    const bool more = cn < p.tn && mt * p.tn + cn < p.M;       // this warp has another chunk of the item
     float v[32], u[32];
-    if (EPI == 3) {     // gate and up: both loads in flight before the one wait
-      unsigned rv[32], ru[32];
-      tmem_ld32_nowait(t_row + c0, rv);
-      tmem_ld32_nowait(t_row + p.acc1_off + c0, ru);
+    if (EPI == 3) {
       tmem_ld_wait();
+      // all 32 products before any store, and no branch in silu_f: an epilogue warp's latency hiding is the
+      // independence of the 32 columns (and the one other warp on its scheduler)
 #pragma unroll
-      for (int j = 0; j < 32; ++j) { v[j] = __uint_as_float(rv[j]); u[j] = __uint_as_float(ru[j]); }
+      for (int j = 0; j < 32; ++j) v[j] = silu_f(__uint_as_float(rv[j])) * __uint_as_float(ru[j]);
+      if (more) {
+        tmem_ld32_nowait(t_row + cn, rv);
+        tmem_ld32_nowait(t_row + p.acc1_off + cn, ru);
+      }
     } else {
       tmem_ld32(t_row + c0, v);
+    }
+    if (!more) { release(); released = true; }
+    if ((EPI == 0 || EPI == 3) && tile != nullptr) {
+      __syncwarp();                           // the previous chunk's reads of the tile are done
+#pragma unroll
+      for (int j = 0; j < 32; ++j) tile[j * 32 + lane] = __float2bfloat16_rn(v[j]);
+      __syncwarp();
+      const int piece = lane & 3;             // eight features = 16 bytes
+      const int nb = n - lane + piece * 8;
+      if (nb < p.N) {                         // N is a multiple of 8 on this path
+        char* dst = base + ((size_t)t0 * ld + nb) * esize;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int tok = i * 8 + (lane >> 2);
+          if (tok < jmax)
+            *reinterpret_cast<uint4*>(dst + (size_t)tok * stride) =
+                *reinterpret_cast<const uint4*>(tile + tok * 32 + piece * 8);
+        }
+      }
+      continue;
     }
     if (!n_ok) continue;                      // the TMEM loads above are warp-collective; the stores are not
     char* ptr = base + ((size_t)t0 * ld + n) * esize;
@@ -155,6 +206,7 @@ __device__ __forceinline__ void epilogue_row(const GemmParams& p, int split, int
     if (jmax == 32) epilogue_chunk<EPI, true>(v, u, ptr, stride, jmax, scale);
     else epilogue_chunk<EPI, false>(v, u, ptr, stride, jmax, scale);
   }
+  return released;
 }
 
 // Epilogue of the LM head fused with the confidence pass (mode 5).  A warp holds 32 output features (vocabulary
@@ -363,20 +415,34 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
       const unsigned acc_phase = (unsigned)(local / p.nbuf) & 1u;
       if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag)) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      for (int a = 0; a < (p.wide ? 2 : 1); ++a) {       // a wide item holds two 128-row accumulators
+      bool released = false;
+      const int n_acc = p.wide ? 2 : 1;                   // a wide item holds two 128-row accumulators
+      for (int a = 0; a < n_acc; ++a) {
         const int n = nt * p.rows + a * TILE_N + q * 32 + lane;
         const bool n_ok = n < p.N;
         const unsigned t_row = tmem_base + ((unsigned)(q * 32) << 16) + acc * acc_cols + a * p.acc1_off;
+        const bool last_acc = a == n_acc - 1;
+        auto release = [&]() {
+          if (!last_acc) return;
+          asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+          __syncwarp();
+          if (lane == 0) mbar_arrive(tempty0 + 8 * acc);
+        };
         if constexpr (EPI == 5) {
           __shared__ float conf_tile[4][32 * 33];
           epilogue_conf(p, mt, n - lane, lane, t_row, conf_tile[q]);
+        } else if constexpr (EPI == 0 || EPI == 3) {
+          __shared__ __align__(16) bf16 out_tile[4][32 * 32];
+          released = epilogue_row<EPI>(p, split, mt, n, n_ok, t_row, release, p.vec_store ? out_tile[q] : nullptr) && last_acc;
         } else {
-          epilogue_row<EPI>(p, split, mt, n, n_ok, t_row);
+          released = epilogue_row<EPI>(p, split, mt, n, n_ok, t_row, release) && last_acc;
         }
       }
-      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-      __syncwarp();
-      if (lane == 0) mbar_arrive(tempty0 + 8 * acc);
+      if (!released) {
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(tempty0 + 8 * acc);
+      }
     }
   }
 
@@ -434,7 +500,7 @@ __device__ __forceinline__ void store_in_cluster(unsigned addr_in_cluster, int v
 }
 
 template <int EPI>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kPairThreads, 1)
 k_gemm_pair(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_w2,
             const __grid_constant__ CUtensorMap map_x, const GemmParams p) {
   extern __shared__ unsigned char smem_dyn[];
@@ -465,7 +531,7 @@ k_gemm_pair(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(tfull0 + 8 * i, 1);
-      mbar_init(tempty0 + 8 * i, 8);       // one arrival per epilogue warp of either CTA
+      mbar_init(tempty0 + 8 * i, 16);      // one arrival per epilogue warp of either CTA
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -574,7 +640,10 @@ k_gemm_pair(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
     }
   } else {
     // ------------------------------------------------------------------ epilogue warps (both CTAs)
+    // Warps 2-5 and 6-9: warp w reads TMEM lanes 32·(w mod 4) .. +31; the two groups take alternate 32-token chunks,
+    // which halves the time an accumulator that is not double-buffered keeps the tensor core waiting.
     const int q = warp & 3;
+    const int group = (warp - 2) >> 2;
     int local = 0;
     bool ok = true;
     pdl_wait();
@@ -586,19 +655,34 @@ k_gemm_pair(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
       const unsigned acc_phase = (unsigned)(local / p.nbuf) & 1u;
       if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag)) { ok = false; break; }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      for (int a = 0; a < (p.wide ? 2 : 1); ++a) {       // a wide item holds two 256-row accumulators
+      bool released = false;
+      const int n_acc = p.wide ? 2 : 1;                   // a wide item holds two 256-row accumulators
+      for (int a = 0; a < n_acc; ++a) {
         const int n = nt * p.rows + a * 256 + (int)rank * TILE_N + q * 32 + lane;
         const unsigned t_row = tmem_base + ((unsigned)(q * 32) << 16) + acc * acc_cols + a * p.acc1_off;
+        const bool last_acc = a == n_acc - 1;
+        auto release = [&]() {
+          if (!last_acc) return;
+          asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+          __syncwarp();
+          if (lane == 0) mbar_arrive_in_cluster(tempty_leader0 + 8 * acc);
+        };
         if constexpr (EPI == 5) {
-          __shared__ float conf_tile[4][32 * 33];
-          epilogue_conf(p, mt, n - lane, lane, t_row, conf_tile[q]);
+          __shared__ float conf_tile[4][32 * 33];         // one transposition tile per lane quarter: group 0 only
+          if (group == 0) epilogue_conf(p, mt, n - lane, lane, t_row, conf_tile[q]);
+        } else if constexpr (EPI == 0 || EPI == 3) {
+          __shared__ __align__(16) bf16 out_tile[8][32 * 32];
+          released = epilogue_row<EPI>(p, split, mt, n, n < p.N, t_row, release,
+                                       p.vec_store ? out_tile[group * 4 + q] : nullptr, group * 32, 64) && last_acc;
         } else {
-          epilogue_row<EPI>(p, split, mt, n, n < p.N, t_row);
+          released = epilogue_row<EPI>(p, split, mt, n, n < p.N, t_row, release, nullptr, group * 32, 64) && last_acc;
         }
       }
-      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-      __syncwarp();
-      if (lane == 0) mbar_arrive_in_cluster(tempty_leader0 + 8 * acc);
+      if (!released) {
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive_in_cluster(tempty_leader0 + 8 * acc);
+      }
     }
     if (!ok && lane == 0) store_in_cluster(peer_abort, 1);
   }
@@ -760,7 +844,7 @@ DevInfo* dev_info() {
     } else {
       cudaLaunchConfig_t qc = {};
       qc.gridDim = dim3(2 * d->num_sms);
-      qc.blockDim = dim3(kThreads);
+      qc.blockDim = dim3(kPairThreads);
       qc.dynamicSmemBytes = (size_t)kSmemBudget + 1024;
       cudaLaunchAttribute qa[1];
       qa[0].id = cudaLaunchAttributeClusterDimension;
@@ -811,6 +895,7 @@ cudaError_t launch_gemm_pair(const DevInfo& dv, const bf16* A, int lda, const bf
   p.M = M; p.N = N; p.K = K; p.mode = mode; p.dual = dual; p.C = C; p.ldc = ldc; p.row_scale = row_scale;
   p.error_flag = scratch.error_flag;
   p.conf_ms = conf ? conf->ms : nullptr; p.conf_am = conf ? conf->am : nullptr; p.skip = conf ? conf->skip : -1;
+  p.vec_store = (ldc % 8 == 0 && N % 8 == 0 && ((uintptr_t)C & 15) == 0) ? 1 : 0;
   // Two 256-row weight tiles per pair and work item (BS_GEMM_PAIR_WIDE=1) halve the token-tile traffic once more at
   // the price of single-buffered accumulators.  Measured on B200 it gains nothing over 256-row items for the
   // K = 3584 projections and 5-8 % for the down projection at 384-640 tokens only, so it is off by default.
@@ -843,6 +928,7 @@ cudaError_t launch_gemm_pair(const DevInfo& dv, const bf16* A, int lda, const bf
   const int stage_bytes = ((dual || p.wide) ? 2 : 1) * TILE_N * BK * 2 + (p.tn / 2) * BK * 2;
   p.stages = kSmemBudget / stage_bytes;
   if (p.stages > 16) p.stages = 16;
+  if (const int st = tuning().stages) { if (st >= 2 && st < p.stages) p.stages = st; }
   p.splits = 1;
   const long long base_items = (long long)p.n_tiles * p.m_tiles;
   if (scratch.partial && !dual && mode != 5 && base_items * 4 < (long long)max_pairs * 3) {
@@ -871,7 +957,7 @@ cudaError_t launch_gemm_pair(const DevInfo& dv, const bf16* A, int lda, const bf
   const int pairs = (int)(items < max_pairs ? items : max_pairs);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2 * pairs);
-  cfg.blockDim = dim3(kThreads);
+  cfg.blockDim = dim3(kPairThreads);
   cfg.dynamicSmemBytes = (size_t)kSmemBudget + 1024;
   cfg.stream = s;
   cudaLaunchAttribute attrs[2];
@@ -934,6 +1020,7 @@ cudaError_t launch_gemm_tc(const bf16* A, int lda, const bf16* W, const bf16* W2
   p.n_tiles = (N + TILE_N - 1) / TILE_N;
   p.error_flag = scratch.error_flag;
   p.conf_ms = conf ? conf->ms : nullptr; p.conf_am = conf ? conf->am : nullptr; p.skip = conf ? conf->skip : -1;
+  p.vec_store = (ldc % 8 == 0 && N % 8 == 0 && ((uintptr_t)C & 15) == 0) ? 1 : 0;
   // ---- token tile and k split ----
   // Few tokens (a block step): one or two token tiles that cover M exactly (UMMA N is any multiple of 16), and a
   // k split that spreads the weight stream over all SMs when there are fewer weight tiles than SMs.
