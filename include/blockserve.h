@@ -256,6 +256,12 @@ int bs_op_gemm(const void* A, int lda, const void* W, const void* W2, void* C, i
                size_t scratch_bytes, int* error_flag /* nullable device int, set when a bounded wait runs out */,
                void* stream);
 
+/* Plan query (host only, no launch): over how many CTA pairs bs_op_gemm splits the K range of every output tile of
+ * this projection INSIDE one thread-block cluster on the current device (the pairs then add their partial accumulators
+ * over distributed shared memory and the direct epilogue follows in the same kernel); 0 when the launch takes another
+ * plan.  Applies to modes 0 and 1 with a dense, 16-byte aligned C (ldc = N).  The paper has no counterpart. */
+int bs_op_gemm_cluster_splits(int M, int N, int K, int mode);
+
 /* y[m,:] = bf16(w * x[idx ? idx[m] : m, :] / sqrt(mean(x^2) + eps)); x fp32 [*, d], y bf16 [M, d]. */
 int bs_op_rmsnorm(const float* x, const int* idx, const void* w, void* y, int M, int d, float eps, void* stream);
 

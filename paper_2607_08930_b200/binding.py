@@ -64,7 +64,7 @@ class BsStats(C.Structure):
 
 EXPORTS = ["bs_query_sizes", "bs_init_model", "bs_admit", "bs_evict_refill", "bs_denoise_step", "bs_block_done",
            "bs_read_tokens", "bs_get_stats", "bs_set_profiling", "bs_get_profile", "bs_destroy", "bs_last_error", "bs_build_flags", "bs_debug_read", "bs_debug_inject_timeout",
-           "bs_debug_force_commit", "bs_debug_snapshot", "bs_debug_restore", "bs_op_gemm",
+           "bs_debug_force_commit", "bs_debug_snapshot", "bs_debug_restore", "bs_op_gemm", "bs_op_gemm_cluster_splits",
            "bs_op_rmsnorm", "bs_op_rope_kv", "bs_op_rope_kv_static", "bs_op_attention_q_tile", "bs_op_attention", "bs_op_confidence",
            "bs_op_lm_head_confidence", "bs_op_lm_head_confidence_scratch_bytes"]
 
@@ -102,6 +102,7 @@ def lib() -> C.CDLL:
         L.bs_debug_snapshot.argtypes = [vp, vp, C.c_size_t, C.POINTER(C.c_size_t)]
         L.bs_debug_restore.argtypes = [vp, vp, C.c_size_t]
         L.bs_op_gemm.argtypes = [vp, i, vp, vp, vp, i, i, i, i, i, vp, vp, C.c_size_t, vp, vp]
+        L.bs_op_gemm_cluster_splits.argtypes = [i, i, i, i]
         L.bs_op_rmsnorm.argtypes = [vp, vp, vp, vp, i, i, f, vp]
         L.bs_op_rope_kv.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, f, i, vp, vp]
         L.bs_op_rope_kv_static.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, f, i, vp]
@@ -336,6 +337,11 @@ def op_gemm(A: torch.Tensor, W: torch.Tensor, mode: int = 0, W2: Optional[torch.
                                0 if scratch is None else scratch.numel() * scratch.element_size(),
                                _ptr(error_flag), _stream()), "bs_op_gemm")
     return C_out
+
+
+def op_gemm_cluster_splits(M: int, N: int, K: int, mode: int) -> int:
+    """CTA pairs that share each output tile's K range inside one cluster for this op_gemm call (0: another plan)."""
+    return int(lib().bs_op_gemm_cluster_splits(M, N, K, mode))
 
 
 def op_rmsnorm(x: torch.Tensor, w: torch.Tensor, eps: float, idx: Optional[torch.Tensor] = None) -> torch.Tensor:

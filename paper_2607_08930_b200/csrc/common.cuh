@@ -168,6 +168,10 @@ cudaError_t launch_conf_final(const float2* slice_ms, const int* slice_am, int M
 // Why the last launch_gemm* of this thread returned cudaErrorNotSupported (a shape or alignment the tensor-core
 // kernels do not take; there is no other GEMM behind them).
 const char* gemm_decline_reason();
+// Over how many CTA pairs launch_gemm* would split the K range of each output tile of this direct projection (mode 0
+// or 1) inside one thread-block cluster, the partial accumulators being reduced over distributed shared memory;
+// 0 when the launch takes another plan.
+int gemm_cluster_splits(int M, int N, int K, int mode, int ldc, const void* C);
 // mode 4: only the k-split partial sums [splits][M][N] are written to scratch.partial; a fused finishing kernel
 // (below) adds them in split order and applies what follows the projection.
 cudaError_t launch_gemm_partial(const bf16* A, int lda, const bf16* W, int M, int N, int K, const GemmScratch& scratch,

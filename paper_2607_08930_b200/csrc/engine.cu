@@ -882,6 +882,11 @@ int bs_op_gemm(const void* A, int lda, const void* W, const void* W2, void* C, i
   return r == cudaSuccess ? BS_OK : (r == cudaErrorNotSupported ? BS_E_ARG : BS_E_CUDA);
 }
 
+int bs_op_gemm_cluster_splits(int M, int N, int K, int mode) {
+  if (M < 0 || N < 1 || K < 8) return 0;
+  return gemm_cluster_splits(M, N, K, mode, N, nullptr);
+}
+
 int bs_op_rmsnorm(const float* x, const int* idx, const void* w, void* y, int M, int d, float eps, void* stream) {
   if (!x || !w || !y || M < 0 || d < 8 || d % 8) return BS_E_ARG;
   return launch_rmsnorm(x, idx, (const bf16*)w, (bf16*)y, M, d, eps, (cudaStream_t)stream) == cudaSuccess ? BS_OK

@@ -131,6 +131,44 @@ __device__ __forceinline__ void epilogue_chunk(const float* v, const float* u, c
     else *reinterpret_cast<float*>(q) = v[j];
   }
 }
+// Stores one chunk: v[j] is the finished value of (feature n, token t0 + j), j < jmax.
+template <int EPI>
+__device__ __forceinline__ void epilogue_store(const GemmParams& p, float* v, float* u, char* base, int ld, int n,
+                                               bool n_ok, int t0, int jmax, bf16* tile) {
+  constexpr int esize = (EPI == 0 || EPI == 3) ? 2 : 4;
+  const size_t stride = (size_t)ld * esize;
+  const int lane = threadIdx.x & 31;
+  if ((EPI == 0 || EPI == 3) && tile != nullptr) {
+    __syncwarp();                             // the previous chunk's reads of the tile are done
+#pragma unroll
+    for (int j = 0; j < 32; ++j) tile[j * 32 + lane] = __float2bfloat16_rn(v[j]);
+    __syncwarp();
+    const int piece = lane & 3;               // eight features = 16 bytes
+    const int nb = n - lane + piece * 8;
+    if (nb < p.N) {                           // N is a multiple of 8 on this path
+      char* dst = base + ((size_t)t0 * ld + nb) * esize;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int tok = i * 8 + (lane >> 2);
+        if (tok < jmax)
+          *reinterpret_cast<uint4*>(dst + (size_t)tok * stride) =
+              *reinterpret_cast<const uint4*>(tile + tok * 32 + piece * 8);
+      }
+    }
+    return;
+  }
+  if (!n_ok) return;                          // (TMEM loads are warp-collective; the stores are not)
+  char* ptr = base + ((size_t)t0 * ld + n) * esize;
+  if (EPI == 1) {
+    // all loads first, then the stores: interleaving them would serialise on the load latency
+#pragma unroll
+    for (int j = 0; j < 32; ++j) u[j] = j < jmax ? *reinterpret_cast<const float*>(ptr + (size_t)j * stride) : 0.f;
+  }
+  const float* scale = EPI == 2 ? p.row_scale + t0 : nullptr;
+  if (jmax == 32) epilogue_chunk<EPI, true>(v, u, ptr, stride, jmax, scale);
+  else epilogue_chunk<EPI, false>(v, u, ptr, stride, jmax, scale);
+}
+
 // bf16 outputs (modes 0 and 3) leave through a per-warp shared-memory tile [32 tokens][32 features] when the output
 // rows allow 16-byte stores: a thread that stored one 2-byte element per token (32 store instructions per chunk, each
 // a 64-byte segment) instead writes four 16-byte vectors, eight token rows per warp instruction.  It matters for the
@@ -140,12 +178,9 @@ __device__ __forceinline__ void epilogue_chunk(const float* v, const float* u, c
 template <int EPI, typename Release>
 __device__ __forceinline__ bool epilogue_row(const GemmParams& p, int split, int mt, int n, bool n_ok, unsigned t_row,
                                              Release release, bf16* tile = nullptr, int c_first = 0, int c_step = 32) {
-  constexpr int esize = (EPI == 0 || EPI == 3) ? 2 : 4;
   const int ld = EPI == 4 ? p.N : p.ldc;
   char* base = EPI == 4 ? reinterpret_cast<char*>(p.partial + ((size_t)split * p.M) * p.N)
                         : reinterpret_cast<char*>(p.C);
-  const size_t stride = (size_t)ld * esize;
-  const int lane = threadIdx.x & 31;
   // SwiGLU: the TMEM loads of the next chunk are issued before this chunk's stores, so that they are complete when
   // the next iteration waits (tcgen05.wait::ld covers every outstanding load of the thread).
   unsigned rv[EPI == 3 ? 32 : 1], ru[EPI == 3 ? 32 : 1];
@@ -176,35 +211,7 @@ __device__ __forceinline__ bool epilogue_row(const GemmParams& p, int split, int
       tmem_ld32(t_row + c0, v);
     }
     if (!more) { release(); released = true; }
-    if ((EPI == 0 || EPI == 3) && tile != nullptr) {
-      __syncwarp();                           // the previous chunk's reads of the tile are done
-#pragma unroll
-      for (int j = 0; j < 32; ++j) tile[j * 32 + lane] = __float2bfloat16_rn(v[j]);
-      __syncwarp();
-      const int piece = lane & 3;             // eight features = 16 bytes
-      const int nb = n - lane + piece * 8;
-      if (nb < p.N) {                         // N is a multiple of 8 on this path
-        char* dst = base + ((size_t)t0 * ld + nb) * esize;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const int tok = i * 8 + (lane >> 2);
-          if (tok < jmax)
-            *reinterpret_cast<uint4*>(dst + (size_t)tok * stride) =
-                *reinterpret_cast<const uint4*>(tile + tok * 32 + piece * 8);
-        }
-      }
-      continue;
-    }
-    if (!n_ok) continue;                      // the TMEM loads above are warp-collective; the stores are not
-    char* ptr = base + ((size_t)t0 * ld + n) * esize;
-    if (EPI == 1) {
-      // all loads first, then the stores: interleaving them would serialise on the load latency
-#pragma unroll
-      for (int j = 0; j < 32; ++j) u[j] = j < jmax ? *reinterpret_cast<const float*>(ptr + (size_t)j * stride) : 0.f;
-    }
-    const float* scale = EPI == 2 ? p.row_scale + t0 : nullptr;
-    if (jmax == 32) epilogue_chunk<EPI, true>(v, u, ptr, stride, jmax, scale);
-    else epilogue_chunk<EPI, false>(v, u, ptr, stride, jmax, scale);
+    epilogue_store<EPI>(p, v, u, base, ld, n, n_ok, t0, jmax, tile);
   }
   return released;
 }
@@ -699,6 +706,204 @@ k_gemm_pair(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
   }
 }
 
+// ---- CTA-pair variant with the k split inside a cluster -----------------------------------------------------------
+// A block step has fewer output tiles than CTA pairs, so the K range of a tile is split over S pairs.  Here the S
+// pairs of a tile form ONE cluster of 2 S CTAs (pair = cluster ranks 2 s, 2 s + 1) and exchange their partial
+// accumulators through distributed shared memory instead of an fp32 round trip through L2 and a finishing kernel:
+//   1. every pair runs its K range into its own TMEM accumulator (as k_gemm_pair, one work item per cluster);
+//   2. cluster barrier: all accumulators complete, every operand ring idle;
+//   3. reduce-scatter: the 32-token chunk c of the tile is owned by split c mod S; a CTA sends every chunk it does not
+//      own to the owner with the same half of the weight rows (st.shared::cluster into the owner's idle operand ring);
+//   4. cluster barrier;
+//   5. each CTA adds, in split order, its own and the received partials of the chunks it owns and applies the direct
+//      epilogue (0: bf16 store, 1: fp32 +=).  The order is fixed, so the result is deterministic.
+// Every thread of the cluster reaches both barriers whatever happened before (a wait that ran out only marks the
+// result as failed), so no CTA can be left waiting.
+__device__ __forceinline__ void st_cluster_v4(unsigned addr_in_cluster, float a, float b, float c, float d) {
+  asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr_in_cluster), "f"(a), "f"(b), "f"(c), "f"(d)
+               : "memory");
+}
+__device__ __forceinline__ float4 ld_shared_v4(unsigned addr) {
+  float4 v;
+  asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+  return v;
+}
+
+template <int EPI>
+__global__ void __launch_bounds__(kPairThreads, 1)
+k_gemm_pair_ks(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, const GemmParams p) {
+  extern __shared__ unsigned char smem_dyn[];
+  __shared__ __align__(8) unsigned long long bars[2 * 16 + 1];     // full[16], empty[16], tmem_full
+  __shared__ unsigned tmem_base_slot;
+  __shared__ int s_abort;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int S = p.splits;
+  const unsigned rank = cluster_ctarank();
+  const int split = (int)(rank >> 1);
+  const unsigned half = rank & 1u;
+  const bool leader = half == 0;
+  const unsigned leader_rank = rank & ~1u;
+  const int tile_id = (int)blockIdx.x / (2 * S);
+  const int mt = tile_id % p.m_tiles, nt = tile_id / p.m_tiles;
+  const unsigned smem0 = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+  const int w_bytes = TILE_N * BK * 2;
+  const int half_tn = p.tn >> 1;
+  const int stage_bytes = w_bytes + half_tn * BK * 2;
+  const unsigned full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[16]), tfull = smem_u32(&bars[32]);
+  const unsigned full_leader0 = map_to_cta(full0, leader_rank);
+  const unsigned peer_abort = map_to_cta(smem_u32(&s_abort), rank ^ 1u);
+  const int kb0 = (int)((long long)p.kblocks * split / S);
+  const int kb1 = (int)((long long)p.kblocks * (split + 1) / S);
+
+  if (threadIdx.x == 0) {
+    s_abort = 0;
+    for (int i = 0; i < p.stages; ++i) {
+      mbar_init(full0 + 8 * i, 1);
+      mbar_init(empty0 + 8 * i, 1);
+    }
+    mbar_init(tfull, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], 256;" ::"r"(smem_u32(&tmem_base_slot))
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  cluster_sync_all();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const unsigned tmem_base = tmem_base_slot;
+  volatile int* abort_flag = &s_abort;
+  pdl_trigger();
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer (both CTAs of every pair)
+    if (lane == 0) {
+      const int wrow = nt * 256 + (int)half * TILE_N;
+      const int xrow = mt * p.tn + (int)half * half_tn;
+      const int npre = min(p.stages, kb1 - kb0);
+      for (int i = 0; i < npre; ++i) {      // weights are constants: fetched before the previous kernel has completed
+        if (leader) mbar_expect_tx(full0 + 8 * i, 2u * (unsigned)stage_bytes);
+        tma_load_2d_pair(smem0 + i * stage_bytes, &map_w, (kb0 + i) * BK, wrow, full_leader0 + 8 * i);
+      }
+      pdl_wait();
+      int stage = 0;
+      unsigned phase = 0;
+      bool ok = true;
+      for (int kb = kb0; kb < kb1; ++kb) {
+        const unsigned sw = smem0 + stage * stage_bytes;
+        if (kb - kb0 >= npre) {
+          if (!mbar_wait(empty0 + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+          if (leader) mbar_expect_tx(full0 + 8 * stage, 2u * (unsigned)stage_bytes);
+          tma_load_2d_pair(sw, &map_w, kb * BK, wrow, full_leader0 + 8 * stage);
+        }
+        tma_load_2d_pair(sw + w_bytes, &map_x, kb * BK, xrow, full_leader0 + 8 * stage);
+        if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+      }
+      if (!ok) store_in_cluster(peer_abort, 1);
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer (leader CTA of every pair)
+    if (lane == 0 && leader) {
+      const unsigned idesc = umma_idesc_pair(p.tn);
+      const unsigned short mask = (unsigned short)(3u << (2 * split));      // the two CTAs of this pair
+      auto commit = [&](unsigned bar) {
+        asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                     ::"r"(bar), "h"(mask) : "memory");
+      };
+      const unsigned lo0 = desc_lo(smem0);
+      const unsigned stage_step = (unsigned)stage_bytes >> 4, x_off = (unsigned)w_bytes >> 4;
+      unsigned lo_stage = lo0;
+      int stage = 0;
+      unsigned phase = 0, accum = 0u;
+      bool ok = true;
+      for (int kb = kb0; kb < kb1; ++kb) {
+        if (!mbar_wait(full0 + 8 * stage, phase, abort_flag)) { ok = false; break; }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        issue_stage<2, false>(tmem_base, tmem_base, lo_stage, lo_stage, lo_stage + x_off, idesc, accum);
+        accum = 1u;
+        commit(empty0 + 8 * stage);
+        lo_stage += stage_step;
+        if (++stage == p.stages) { stage = 0; phase ^= 1u; lo_stage = lo0; }
+      }
+      if (ok) commit(tfull);
+      else store_in_cluster(peer_abort, 1);
+    }
+  }
+
+  // ---- epilogue warps 2..9: wait for this pair's accumulator ----
+  const int q = warp & 3;                       // TMEM lane quarter of this warp
+  const int group = (warp - 2) >> 2;            // the two groups take alternate chunks
+  const bool epi = warp >= 2;
+  if (epi) {
+    pdl_wait();
+    if (!mbar_wait(tfull, 0, abort_flag) && lane == 0) store_in_cluster(peer_abort, 1);
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  cluster_sync_all();                           // every accumulator of the tile is complete, every operand ring idle
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+
+  // received partials: [sender split][owned chunk index][lane quarter][4-column group][lane][4 floats]
+  const int nch = (min(p.tn, p.M - mt * p.tn) + 31) >> 5;        // chunks of this tile that hold tokens
+  const int kmax = (((p.tn + 31) >> 5) + S - 1) / S;              // owned chunks per CTA at most
+  const unsigned t_row = tmem_base + ((unsigned)(q * 32) << 16);
+  auto slot = [&](int sender, int k) { return smem0 + (unsigned)(((sender * kmax + k) * 4 + q) * 4096 + lane * 16); };
+  if (epi) {
+    for (int c = 0; c < nch; ++c) {
+      const int owner = c % S, k = c / S;
+      if (owner == split || (k & 1) != group) continue;         // warp-uniform
+      float v[32];
+      tmem_ld32(t_row + c * 32, v);
+      const unsigned dst = map_to_cta(slot(split, k), (unsigned)(2 * owner) + half);
+#pragma unroll
+      for (int g = 0; g < 8; ++g) st_cluster_v4(dst + g * 512, v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+    }
+  }
+  cluster_sync_all();                           // the partials have arrived
+  if (epi) {
+    const int n = nt * 256 + (int)half * TILE_N + q * 32 + lane;
+    const bool n_ok = n < p.N;
+    char* base = reinterpret_cast<char*>(p.C);
+    __shared__ __align__(16) bf16 out_tile[EPI == 0 ? 8 : 1][32 * 32];
+    bf16* tile = (EPI == 0 && p.vec_store) ? out_tile[group * 4 + q] : nullptr;
+    for (int c = split; c < nch; c += S) {
+      const int k = c / S;
+      if ((k & 1) != group) continue;                           // warp-uniform
+      const int t0 = mt * p.tn + c * 32;
+      const int jmax = min(min(32, p.tn - c * 32), p.M - t0);
+      float own[32], v[32], u[32];
+      tmem_ld32(t_row + c * 32, own);
+#pragma unroll
+      for (int j = 0; j < 32; ++j) v[j] = 0.f;
+      for (int sdr = 0; sdr < S; ++sdr) {                       // split order
+        if (sdr == split) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) v[j] += own[j];
+        } else {
+          const unsigned src = slot(sdr, k);
+#pragma unroll
+          for (int g = 0; g < 8; ++g) {
+            const float4 r = ld_shared_v4(src + g * 512);
+            v[4 * g] += r.x; v[4 * g + 1] += r.y; v[4 * g + 2] += r.z; v[4 * g + 3] += r.w;
+          }
+        }
+      }
+      epilogue_store<EPI>(p, v, u, base, p.ldc, n, n_ok, t0, jmax, tile);
+    }
+  }
+
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  cluster_sync_all();                           // nobody leaves while a partner may still signal or read it
+  if (s_abort && threadIdx.x == 0 && p.error_flag) atomicExch(p.error_flag, 1);
+  if (warp == 1) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, 256;" ::"r"(tmem_base) : "memory");
+  }
+}
+
 // Adds the k-split partial sums in split order and applies the epilogue.
 __global__ void k_gemm_finish(const float* __restrict__ partial, int splits, int M, int N, int mode, void* Cv, int ldc,
                               const float* __restrict__ row_scale) {
@@ -776,6 +981,7 @@ struct Tuning {
   int stages;       // BS_GEMM_STAGES: 0 automatic
   int debug;        // BS_GEMM_DEBUG: print every plan
   int no_pdl;       // BS_NO_PDL
+  int ks;           // BS_GEMM_KS: -1 automatic, 0 never split K inside a cluster, 2 or 4 that many splits where they fit
 };
 int env_int(const char* name, int dflt) {
   const char* v = getenv(name);
@@ -785,7 +991,7 @@ const Tuning& tuning() {
   static const Tuning t = {env_int("BS_GEMM_PAIR", -1), env_int("BS_GEMM_PAIR_WIDE", 0) > 0,
                            env_int("BS_GEMM_PAIR_SPLITS", 8), getenv("BS_GEMM_WIDE") && env_int("BS_GEMM_WIDE", 1) == 0,
                            env_int("BS_GEMM_KSUB", 0), env_int("BS_GEMM_SPLITS", 0), env_int("BS_GEMM_STAGES", 0),
-                           getenv("BS_GEMM_DEBUG") != nullptr, getenv("BS_NO_PDL") != nullptr};
+                           getenv("BS_GEMM_DEBUG") != nullptr, getenv("BS_NO_PDL") != nullptr, env_int("BS_GEMM_KS", -1)};
   return t;
 }
 
@@ -822,6 +1028,7 @@ struct DevInfo {
   int num_sms;      // 0: not initialised
   int tc_ok;        // the single-CTA kernels may use their shared-memory budget
   int max_pairs;    // 0: not queried; < 0: the pair kernel cannot be used; else resident clusters of two CTAs
+  int max_ks[2];    // resident clusters of 4 and of 8 CTAs of the cluster k-split kernel (0: it cannot be used)
 };
 DevInfo g_dev[kMaxDevices];
 
@@ -854,7 +1061,30 @@ DevInfo* dev_info() {
       if (cudaOccupancyMaxActiveClusters(&n, k_gemm_pair<0>, &qc) != cudaSuccess || n < 1) { cudaGetLastError(); n = -1; }
       d->max_pairs = n;
     }
-    if (tuning().debug) fprintf(stderr, "gemm pair kernel: %d resident CTA pairs\n", d->max_pairs);
+    d->max_ks[0] = d->max_ks[1] = 0;
+    if (d->max_pairs > 0 &&
+        cudaFuncSetAttribute(k_gemm_pair_ks<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 1024) == cudaSuccess &&
+        cudaFuncSetAttribute(k_gemm_pair_ks<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 1024) == cudaSuccess) {
+      for (int i = 0; i < 2; ++i) {
+        const int cs = i == 0 ? 4 : 8;
+        cudaLaunchConfig_t qc = {};
+        qc.gridDim = dim3((unsigned)(d->num_sms / cs * cs));
+        qc.blockDim = dim3(kPairThreads);
+        qc.dynamicSmemBytes = (size_t)kSmemBudget + 1024;
+        cudaLaunchAttribute qa[1];
+        qa[0].id = cudaLaunchAttributeClusterDimension;
+        qa[0].val.clusterDim.x = (unsigned)cs; qa[0].val.clusterDim.y = 1; qa[0].val.clusterDim.z = 1;
+        qc.attrs = qa; qc.numAttrs = 1;
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, k_gemm_pair_ks<0>, &qc) != cudaSuccess || n < 1) { cudaGetLastError(); n = 0; }
+        d->max_ks[i] = n;
+      }
+    } else {
+      cudaGetLastError();
+    }
+    if (tuning().debug)
+      fprintf(stderr, "gemm pair kernel: %d resident CTA pairs; cluster k-split: %d clusters of 4, %d of 8\n", d->max_pairs,
+              d->max_ks[0], d->max_ks[1]);
   }
   return d;
 }
@@ -973,9 +1203,73 @@ cudaError_t launch_gemm_pair(const DevInfo& dv, const bf16* A, int lda, const bf
   return r;
 }
 
+// Plan of the cluster k-split kernel for a direct projection (mode 0 or 1) of a block step: how many pairs share a
+// tile's K range, or 0 when the shape is left to the other kernels.  One wave of clusters only (a cluster holds its
+// SMs until its slowest pair is done), at least 8 k blocks per pair, and at least 3/8 of the SMs busy.
+struct KsPlan { int splits, tn, m_tiles, n_tiles, kblocks; };
+KsPlan plan_ks(const DevInfo& dv, int M, int N, int K, int mode, int ldc, const void* C) {
+  KsPlan pl = {0, 0, 0, 0, 0};
+  const int want = tuning().ks;
+  if (want == 0 || (mode != 0 && mode != 1) || M < 128 || M > 1024 || N < 256) return pl;
+  if (mode == 0 && !(ldc % 8 == 0 && N % 8 == 0 && ((uintptr_t)C & 15) == 0)) return pl;
+  pl.n_tiles = (N + 255) / 256;
+  pl.m_tiles = (M + 255) / 256;
+  pl.tn = (((M + pl.m_tiles - 1) / pl.m_tiles) + 15) / 16 * 16;
+  pl.kblocks = (K + BK - 1) / BK;
+  const int tiles = pl.n_tiles * pl.m_tiles;
+  for (int i = 1; i >= 0; --i) {
+    const int sp = i == 0 ? 2 : 4;
+    if (want > 0 && want != sp) continue;
+    if (tiles > dv.max_ks[i] || pl.kblocks / sp < 8) continue;
+    if (want < 0 && tiles * 2 * sp * 8 < dv.num_sms * 3) continue;
+    pl.splits = sp;
+    break;
+  }
+  return pl;
+}
+
+cudaError_t launch_gemm_pair_ks(const KsPlan& pl, const bf16* A, int lda, const bf16* W, void* C, int ldc, int M, int N,
+                                int K, int mode, const GemmScratch& scratch, cudaStream_t s) {
+  GemmParams p = {};
+  p.M = M; p.N = N; p.K = K; p.mode = mode; p.C = C; p.ldc = ldc;
+  p.error_flag = scratch.error_flag;
+  p.skip = -1;
+  p.vec_store = (ldc % 8 == 0 && N % 8 == 0 && ((uintptr_t)C & 15) == 0) ? 1 : 0;
+  p.rows = 256; p.ksub = 1; p.nbuf = 1; p.acc1_off = 0;
+  p.n_tiles = pl.n_tiles; p.m_tiles = pl.m_tiles; p.tn = pl.tn; p.kblocks = pl.kblocks; p.splits = pl.splits;
+  const int stage_bytes = TILE_N * BK * 2 + (p.tn / 2) * BK * 2;
+  p.stages = kSmemBudget / stage_bytes;
+  if (p.stages > 16) p.stages = 16;
+  if (const int st = tuning().stages) { if (st >= 2 && st < p.stages) p.stages = st; }
+  CUtensorMap mw, mx;
+  if (!get_map(W, N, K, K, TILE_N, &mw)) return decline("tensor map of the weight matrix could not be encoded");
+  if (!get_map(A, M, K, lda, p.tn / 2, &mx)) return decline("tensor map of the activations could not be encoded");
+  if (tuning().debug)
+    fprintf(stderr, "cluster k-split gemm M=%d N=%d K=%d mode=%d tn=%d m_tiles=%d n_tiles=%d splits=%d stages=%d\n", M, N, K,
+            mode, p.tn, p.m_tiles, p.n_tiles, p.splits, p.stages);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(p.n_tiles * p.m_tiles * 2 * p.splits));
+  cfg.blockDim = dim3(kPairThreads);
+  cfg.dynamicSmemBytes = (size_t)kSmemBudget + 1024;
+  cfg.stream = s;
+  cudaLaunchAttribute attrs[2];
+  attrs[0].id = cudaLaunchAttributeClusterDimension;
+  attrs[0].val.clusterDim.x = (unsigned)(2 * p.splits); attrs[0].val.clusterDim.y = 1; attrs[0].val.clusterDim.z = 1;
+  attrs[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attrs[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attrs;
+  cfg.numAttrs = tuning().no_pdl ? 1 : 2;
+  return mode == 0 ? cudaLaunchKernelEx(&cfg, k_gemm_pair_ks<0>, mw, mx, p) : cudaLaunchKernelEx(&cfg, k_gemm_pair_ks<1>, mw, mx, p);
+}
+
 }  // namespace
 
 const char* gemm_decline_reason() { return g_decline.c_str(); }
+
+int gemm_cluster_splits(int M, int N, int K, int mode, int ldc, const void* C) {
+  const DevInfo* dv = dev_info();
+  return dv && dv->tc_ok ? plan_ks(*dv, M, N, K, mode, ldc, C).splits : 0;
+}
 
 // Plans and launches one projection.  A shape the tensor-core kernels cannot take is an error
 // (cudaErrorNotSupported, reason in gemm_decline_reason()): there is no second GEMM implementation behind this one.
@@ -992,6 +1286,13 @@ cudaError_t launch_gemm_tc(const bf16* A, int lda, const bf16* W, const bf16* W2
   if (!dvp || !dvp->tc_ok) return decline("the device does not grant the kernels' shared-memory budget");
   const DevInfo& dv = *dvp;
   const int num_sms = dv.num_sms;
+  if (mode == 0 || mode == 1) {
+    const KsPlan pl = plan_ks(dv, M, N, K, mode, ldc, C);
+    if (pl.splits > 0) {
+      if (splits_out) *splits_out = 1;
+      return launch_gemm_pair_ks(pl, A, lda, W, C, ldc, M, N, K, mode, scratch, s);
+    }
+  }
   // CTA pairs that share each token tile move fewer bytes per flop and are faster per work item (measured on B200:
   // +8 to +20 %), but their grid has half as many workers.  From 128 tokens on, the pair plan is taken unless it
   // would leave clearly more of its grid idle than the single-CTA plan (few 256-row tiles and no k split, or a last

@@ -104,6 +104,44 @@ def test_gemm_k_split(B, M, N, K, mode):
         assert (again == got).all()
 
 
+@pytest.mark.parametrize("M,N,K", [(128, 3584, 3584), (200, 4608, 3584), (256, 3584, 2048), (333, 3584, 3584),
+                                   (500, 3584, 1024), (512, 3584, 18944), (640, 1024, 4096), (1000, 512, 2048),
+                                   (144, 3592, 1024)])
+@pytest.mark.parametrize("mode", [0, 1])
+def test_gemm_k_split_inside_clusters(B, M, N, K, mode):
+    """Direct projections with few output tiles: the pairs of a tile share a cluster and add their partial accumulators
+    over distributed shared memory (ragged token tiles, a ragged weight tile, both cluster sizes, both epilogues)."""
+    assert B.op_gemm_cluster_splits(M, N, K, mode) in (2, 4), "the shape is meant to take the cluster plan"
+    rng = np.random.default_rng(M * 3 + N + K + mode)
+    A = bf16_round(rng.normal(size=(M, K)))
+    W = bf16_round(rng.normal(size=(N, K)) * 0.05)
+    ref = A.double().numpy() @ W.double().numpy().T
+    flag = torch.zeros(1, dtype=torch.int32, device="cuda")
+    if mode == 0:
+        run = lambda: B.op_gemm(A.cuda(), W.cuda(), 0, error_flag=flag).float().cpu().numpy()
+        tol = 6e-3
+    else:
+        c0 = rng.normal(size=(M, N)).astype(F32)
+        ref = ref + c0
+
+        def run():
+            Cd = torch.from_numpy(c0).cuda()
+            B.op_gemm(A.cuda(), W.cuda(), 1, C_out=Cd, error_flag=flag)
+            return Cd.cpu().numpy()
+        tol = 1e-4
+    got = run()
+    assert int(flag.item()) == 0
+    assert rel_err(got, ref) < tol
+    assert np.abs(got - ref).max() <= tol * (np.abs(ref) + np.abs(ref).max() * 0.05).max()
+    assert (run() == got).all()          # split order is fixed: the same bits every time
+
+
+def test_gemm_cluster_plan_leaves_other_shapes_alone(B):
+    for M, N, K, mode in [(64, 3584, 3584, 0), (2048, 3584, 3584, 1), (256, 3584, 3584, 3), (256, 3584, 3584, 2),
+                          (256, 128, 3584, 0), (256, 3584, 256, 0)]:
+        assert B.op_gemm_cluster_splits(M, N, K, mode) == 0
+
+
 def test_gemm_strided_rows_and_empty(B):
     rng = np.random.default_rng(5)
     big = bf16_round(rng.normal(size=(70, 512))).cuda()
