@@ -151,6 +151,19 @@ def test_llada_stream_full_depth_cycle_after_the_first_refill(B):
     ls.assert_caps(noise_cap=0.10)
 
 
+def test_long_context_stream_full_depth_first_cycle(B):
+    """Workload 4 at full depth (28 layers, rows of 1.5-2.5 k tokens under the 65536-token budget, tau = 0.95): the
+    whole batch runs in integer lockstep, the oracle follows the shortest admitted row through its refresh step and
+    the first block steps of cycle 0."""
+    wl = bs_inputs.workload(4)
+    def pick(ls):
+        return min(ls.ora.sched.active, key=lambda r: r.p + r.g).req_id
+    ls, seen = _sampled_cycles(B, wl, 98304, boundaries=(0,), pick=pick, max_steps=4)
+    print("cfg4 full depth, cycle 0:", seen, ls.summary())
+    assert seen[0]["active_rows"] > 16 and seen[0]["p"] > 1000 and ls.rows_checked > 0
+    ls.assert_caps(noise_cap=0.10)
+
+
 TOY = bs_inputs.ModelShape("toy", 1, 64, 1, 1, 64, 64, 64, init_std=0.1)
 
 
