@@ -1300,7 +1300,7 @@ cudaError_t launch_gemm_tc(const bf16* A, int lda, const bf16* W, const bf16* W2
   bool use_pair = false;
   if (dv.max_pairs > 0) {
     if (tuning().pair >= 0) use_pair = tuning().pair > 0 && M >= tuning().pair;
-    else if (M >= 128) {
+    else if (M >= ((mode == 2 || mode == 5) ? 64 : 128)) {     // the LM head (many weight tiles, no k split) gains from 64 on
       const bool dual_ = mode == 3 || mode == 5;      // no k split for these
       const int kb = (K + BK - 1) / BK;
       const long long items_p = (long long)((N + 255) / 256) * ((M + 255) / 256);
