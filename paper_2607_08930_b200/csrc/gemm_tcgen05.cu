@@ -31,6 +31,7 @@ constexpr int TILE_N = 128;            // weight rows per tile (UMMA M)
 constexpr int kThreads = 192;
 constexpr int kPairThreads = 320;       // the pair kernel runs two groups of four epilogue warps (alternate token chunks)
 constexpr int kSmemBudget = 200 * 1024;
+constexpr int kSmemBudgetConf = 176 * 1024;   // pair kernel, mode 5 on all eight epilogue warps: eight 4 KB tiles are static
 
 struct GemmParams {
   int M, N, K;
@@ -223,11 +224,12 @@ __device__ __forceinline__ bool epilogue_row(const GemmParams& p, int split, int
 // index of the maximum - one partial per (feature group, token), a twelfth of the bytes of the logits.  When p.C
 // is set the scaled fp32 logits are stored as well (parity hooks read them; the timed path passes nullptr).
 __device__ __forceinline__ void epilogue_conf(const GemmParams& p, int mt, int n0, int lane, unsigned t_row,
-                                              float* tile /* [32][33] of this warp */) {
+                                              float* tile /* [32][33] of this warp */, int c_first = 0,
+                                              int c_step = 32) {
   const int group = n0 >> 5;
   const int n_valid = min(32, p.N - n0);                 // features of this group that exist (warp-uniform)
   const int i_skip = p.skip - n0;                         // index of the excluded feature inside the group, if any
-  for (int c0 = 0; c0 < p.tn; c0 += 32) {
+  for (int c0 = c_first; c0 < p.tn; c0 += c_step) {
     const int t0 = mt * p.tn + c0;
     if (t0 >= p.M) break;                                 // warp-uniform
     const int jmax = min(min(32, p.tn - c0), p.M - t0);
@@ -677,6 +679,11 @@ k_gemm_pair(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
         if constexpr (EPI == 5) {
           __shared__ float conf_tile[4][32 * 33];         // one transposition tile per lane quarter: group 0 only
           if (group == 0) epilogue_conf(p, mt, n - lane, lane, t_row, conf_tile[q]);
+        } else if constexpr (EPI == 6) {
+          // mode 5 with token tiles wider than 128: the confidence pass of a tile would outlast the next tile's main
+          // loop on four warps, so all eight take part (eight tiles of static shared memory, a shorter operand ring)
+          __shared__ float conf_tile[8][32 * 33];
+          epilogue_conf(p, mt, n - lane, lane, t_row, conf_tile[group * 4 + q], group * 32, 64);
         } else if constexpr (EPI == 0 || EPI == 3) {
           __shared__ __align__(16) bf16 out_tile[8][32 * 32];
           released = epilogue_row<EPI>(p, split, mt, n, n < p.N, t_row, release,
@@ -1013,12 +1020,14 @@ GemmKernel kernel_pair(int epi) {
     case 2: return k_gemm_pair<2>;
     case 3: return k_gemm_pair<3>;
     case 5: return k_gemm_pair<5>;
+    case 6: return k_gemm_pair<6>;
     default: return k_gemm_pair<4>;
   }
 }
-bool allow_big_smem(GemmKernel (*table)(int)) {
-  for (int e = 0; e < 6; ++e)
-    if (cudaFuncSetAttribute(table(e), cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 1024) != cudaSuccess)
+bool allow_big_smem(GemmKernel (*table)(int), int variants) {
+  for (int e = 0; e < variants; ++e)
+    if (cudaFuncSetAttribute(table(e), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (e == 6 ? kSmemBudgetConf : kSmemBudget) + 1024) != cudaSuccess)
       return false;
   return true;
 }
@@ -1040,12 +1049,12 @@ DevInfo* dev_info() {
     int dev = 0, n = 0;
     cudaGetDevice(&dev);
     if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) return nullptr;
-    d->tc_ok = allow_big_smem(kernel_tc) ? 1 : 0;
+    d->tc_ok = allow_big_smem(kernel_tc, 6) ? 1 : 0;
     if (!d->tc_ok) cudaGetLastError();
     d->num_sms = n;
   }
   if (!d->max_pairs) {
-    if (!allow_big_smem(kernel_pair)) {
+    if (!allow_big_smem(kernel_pair, 7)) {
       cudaGetLastError();
       d->max_pairs = -1;
     } else {
@@ -1156,7 +1165,9 @@ cudaError_t launch_gemm_pair(const DevInfo& dv, const bf16* A, int lda, const bf
   p.acc1_off = p.nbuf == 1 ? 256 : 128;
   p.kblocks = (K + BK - 1) / BK;
   const int stage_bytes = ((dual || p.wide) ? 2 : 1) * TILE_N * BK * 2 + (p.tn / 2) * BK * 2;
-  p.stages = kSmemBudget / stage_bytes;
+  const bool conf8 = mode == 5 && p.tn > 128;
+  const int smem_budget = conf8 ? kSmemBudgetConf : kSmemBudget;
+  p.stages = smem_budget / stage_bytes;
   if (p.stages > 16) p.stages = 16;
   if (const int st = tuning().stages) { if (st >= 2 && st < p.stages) p.stages = st; }
   p.splits = 1;
@@ -1188,7 +1199,7 @@ cudaError_t launch_gemm_pair(const DevInfo& dv, const bf16* A, int lda, const bf
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2 * pairs);
   cfg.blockDim = dim3(kPairThreads);
-  cfg.dynamicSmemBytes = (size_t)kSmemBudget + 1024;
+  cfg.dynamicSmemBytes = (size_t)smem_budget + 1024;
   cfg.stream = s;
   cudaLaunchAttribute attrs[2];
   attrs[0].id = cudaLaunchAttributeClusterDimension;
@@ -1197,7 +1208,7 @@ cudaError_t launch_gemm_pair(const DevInfo& dv, const bf16* A, int lda, const bf
   attrs[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attrs;
   cfg.numAttrs = tuning().no_pdl ? 1 : 2;
-  cudaError_t r = cudaLaunchKernelEx(&cfg, kernel_pair((p.splits > 1 || mode == 4) ? 4 : mode), mw, mw2, mx, p);
+  cudaError_t r = cudaLaunchKernelEx(&cfg, kernel_pair((p.splits > 1 || mode == 4) ? 4 : (conf8 ? 6 : mode)), mw, mw2, mx, p);
   if (r != cudaSuccess) return r;
   if (p.splits > 1 && mode != 4) r = launch_finish(p, mode, dv.num_sms, s);
   return r;
