@@ -1135,10 +1135,15 @@ cudaError_t launch_gemm_pair(const DevInfo& dv, const bf16* A, int lda, const bf
   p.error_flag = scratch.error_flag;
   p.conf_ms = conf ? conf->ms : nullptr; p.conf_am = conf ? conf->am : nullptr; p.skip = conf ? conf->skip : -1;
   p.vec_store = (ldc % 8 == 0 && N % 8 == 0 && ((uintptr_t)C & 15) == 0) ? 1 : 0;
-  // Two 256-row weight tiles per pair and work item (BS_GEMM_PAIR_WIDE=1) halve the token-tile traffic once more at
-  // the price of single-buffered accumulators.  Measured on B200 it gains nothing over 256-row items for the
-  // K = 3584 projections and 5-8 % for the down projection at 384-640 tokens only, so it is off by default.
-  p.wide = (tuning().pair_wide && !dual && N >= 1024) ? 1 : 0;
+  // Two 256-row weight tiles per pair and work item halve the token-tile traffic once more (48 instead of 64 bytes
+  // per clock and SM from L2, the SwiGLU GEMM's figure) at the price of single-buffered accumulators; with a long K
+  // the exposed epilogue is a per cent of the item.  Measured on B200 in seconds-long loops (power-capped, the state
+  // a refresh step runs in): the down projection (K = 18944) 2-14 % faster from 2048 tokens on, and 10-15 % with token
+  // tiles narrowed to fill the last round of items (7 wide weight tiles leave 74 pairs badly divided); slower below
+  // 2048 tokens and for the K = 3584 projections (3-7 %).  BS_GEMM_PAIR_WIDE: -1 automatic, 0 never, 1 wherever it fits.
+  static const int wide_mode = env_int("BS_GEMM_PAIR_WIDE", -1);
+  static const int wide_fill = env_int("BS_GEMM_WIDE_FILL", 8);      // per-item constant of the fill cost below
+  p.wide = (!dual && mode != 5 && N >= 1024 && (wide_mode > 0 || (wide_mode < 0 && K >= 8192 && M >= 2048))) ? 1 : 0;
   p.rows = p.wide ? 512 : 256;
   p.ksub = 1;
   p.n_tiles = (N + p.rows - 1) / p.rows;
@@ -1150,13 +1155,13 @@ cudaError_t launch_gemm_pair(const DevInfo& dv, const bf16* A, int lda, const bf
   // The tensor-core time of a work item is linear in its token-tile width.  When the number of weight tiles does not
   // divide the grid (the LLaDA-shaped gate/up has 48 for 74 pairs), slightly narrower token tiles that fill the last
   // round of work items finish earlier; measured for the SwiGLU GEMM only (up to -3.5 %), where items are long.
-  if (dual && (long long)p.n_tiles * p.m_tiles > max_pairs) {
+  if ((dual || (p.wide && wide_fill)) && (long long)p.n_tiles * p.m_tiles > max_pairs) {
     const int lo = p.m_tiles;
     long long best_cost = -1;
     for (int mt = lo; mt <= lo + lo / 2 + 1; ++mt) {
       const int tn = (((M + mt - 1) / mt) + 15) / 16 * 16;
       const long long rounds = ((long long)p.n_tiles * mt + max_pairs - 1) / max_pairs;
-      const long long cost = rounds * (tn + 48);            // + a fixed per-item cost (ramp, exposed epilogue)
+      const long long cost = rounds * (tn + (dual ? 48 : wide_fill));            // + a fixed per-item cost (ramp, exposed epilogue)
       if (best_cost < 0 || cost < best_cost) { best_cost = cost; p.m_tiles = mt; }
     }
   }

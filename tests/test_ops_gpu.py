@@ -136,6 +136,34 @@ def test_gemm_k_split_inside_clusters(B, M, N, K, mode):
     assert (run() == got).all()          # split order is fixed: the same bits every time
 
 
+@pytest.mark.parametrize("M,N,K", [(2200, 1536, 8192), (2048, 1280, 8200), (4100, 1024, 8192),
+                                   (5000, 2048, 8192)])      # the last: more items than CTA pairs
+@pytest.mark.parametrize("mode", [0, 1, 2])
+def test_gemm_wide_pair_items_with_a_long_k(B, M, N, K, mode):
+    """Many tokens and a long K (the down projection of a refresh step): work items of 512 weight rows whose two
+    accumulators share every token tile, token tiles narrowed to fill the last round; ragged in every dimension
+    (a last item with 256 of its 512 weight rows, K beyond the last full k block, a partial token tile)."""
+    rng = np.random.default_rng(M + 3 * N + K + mode)
+    A = bf16_round(rng.normal(size=(M, K)))
+    W = bf16_round(rng.normal(size=(N, K)) * 0.05)
+    ref = A.double().numpy() @ W.double().numpy().T
+    flag = torch.zeros(1, dtype=torch.int32, device="cuda")
+    if mode == 0:
+        got, tol = B.op_gemm(A.cuda(), W.cuda(), 0, error_flag=flag).float().cpu().numpy(), 6e-3
+    elif mode == 1:
+        c0 = rng.normal(size=(M, N)).astype(F32)
+        Cd = torch.from_numpy(c0).cuda()
+        B.op_gemm(A.cuda(), W.cuda(), 1, C_out=Cd, error_flag=flag)
+        got, ref, tol = Cd.cpu().numpy(), ref + c0, 1e-4
+    else:
+        sc = rng.uniform(0.5, 30.0, size=M).astype(F32)
+        got = B.op_gemm(A.cuda(), W.cuda(), 2, row_scale=torch.from_numpy(sc).cuda(), error_flag=flag).cpu().numpy()
+        ref, tol = ref * sc[:, None], 1e-4
+    assert int(flag.item()) == 0
+    assert rel_err(got, ref) < tol
+    assert np.abs(got - ref).max() <= tol * (np.abs(ref) + np.abs(ref).max() * 0.05).max()
+
+
 def test_gemm_cluster_plan_leaves_other_shapes_alone(B):
     for M, N, K, mode in [(64, 3584, 3584, 0), (2048, 3584, 3584, 1), (256, 3584, 3584, 3), (256, 3584, 3584, 2),
                           (256, 128, 3584, 0), (256, 3584, 256, 0)]:
