@@ -57,12 +57,30 @@ struct GemmParams {
   int* conf_am;      // [ceil(N / 32)][M]
   int skip;
   int vec_store;     // bf16 output rows take 16-byte stores (ldc and N multiples of 8, C 16-byte aligned)
+  int mgroup;        // token tiles per group of the work-item order (0: token tile fastest over all of them)
 };
 
 __device__ __forceinline__ void tma_load_2d(unsigned dst, const CUtensorMap* map, int c0, int c1, unsigned bar) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
       ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
+}
+
+// Work-item order.  Output tiles are numbered token tile fastest, so that the CTAs of one round share a weight tile;
+// with `mgroup` > 0 the token tiles are taken in groups of that many, all weight tiles within a group before the
+// next group: the group's activations then stay in L2 while the weights stream past them (many tokens: without it
+// every weight tile re-reads the whole activation matrix, which no longer fits L2 beyond ~8 k tokens).
+__device__ __forceinline__ void tile_of(const GemmParams& p, int tile, int* mt, int* nt) {
+  if (p.mgroup <= 0) {
+    *mt = tile % p.m_tiles;
+    *nt = tile / p.m_tiles;
+    return;
+  }
+  const int per_group = p.mgroup * p.n_tiles;
+  const int g = tile / per_group, r = tile - g * per_group;
+  const int g_size = min(p.mgroup, p.m_tiles - g * p.mgroup);
+  *nt = r / g_size;
+  *mt = g * p.mgroup + r % g_size;
 }
 
 // kind::f16 instruction descriptor: fp32 accumulator, bf16 x bf16, both K-major, shape 128 x n x 16.
@@ -330,7 +348,9 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
       {
         const int it = blockIdx.x;
         const int split = it % p.splits;
-        const int nt = (it / p.splits) / p.m_tiles;
+        int mt_, nt;
+        tile_of(p, it / p.splits, &mt_, &nt);
+        (void)mt_;
         const int kb0 = (int)((long long)p.kblocks * split / p.splits);
         const int kb1 = (int)((long long)p.kblocks * (split + 1) / p.splits);
         npre = min(p.stages, kb1 - kb0);
@@ -349,7 +369,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
       for (int it = blockIdx.x; it < items && ok; it += gridDim.x) {
         const int split = it % p.splits;
         const int tile = it / p.splits;
-        const int mt = tile % p.m_tiles, nt = tile / p.m_tiles;
+        int mt, nt;
+        tile_of(p, tile, &mt, &nt);
         const int kb0 = (int)((long long)p.kblocks * split / p.splits);
         const int kb1 = (int)((long long)p.kblocks * (split + 1) / p.splits);
         for (int kb = kb0; kb < kb1; ++kb) {
@@ -419,7 +440,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
     for (int it = blockIdx.x; it < items; it += gridDim.x, ++local) {
       const int split = it % p.splits;
       const int tile = it / p.splits;
-      const int mt = tile % p.m_tiles, nt = tile / p.m_tiles;
+      int mt, nt;
+      tile_of(p, tile, &mt, &nt);
       const int acc = local % p.nbuf;
       const unsigned acc_phase = (unsigned)(local / p.nbuf) & 1u;
       if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag)) break;
@@ -570,7 +592,9 @@ k_gemm_pair(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
       if (pair < items) {                   // weight tiles of the first stages: constants, fetched before the wait
         const int it = pair;
         const int split = it % p.splits;
-        const int nt = (it / p.splits) / p.m_tiles;
+        int mt_, nt;
+        tile_of(p, it / p.splits, &mt_, &nt);
+        (void)mt_;
         const int kb0 = (int)((long long)p.kblocks * split / p.splits);
         const int kb1 = (int)((long long)p.kblocks * (split + 1) / p.splits);
         npre = min(p.stages, kb1 - kb0);
@@ -588,7 +612,8 @@ k_gemm_pair(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
       for (int it = pair; it < items && ok; it += n_pairs) {
         const int split = it % p.splits;
         const int tile = it / p.splits;
-        const int mt = tile % p.m_tiles, nt = tile / p.m_tiles;
+        int mt, nt;
+        tile_of(p, tile, &mt, &nt);
         const int kb0 = (int)((long long)p.kblocks * split / p.splits);
         const int kb1 = (int)((long long)p.kblocks * (split + 1) / p.splits);
         const int wrow = nt * p.rows + (int)rank * TILE_N;
@@ -659,7 +684,8 @@ k_gemm_pair(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
     for (int it = pair; it < items; it += n_pairs, ++local) {
       const int split = it % p.splits;
       const int tile = it / p.splits;
-      const int mt = tile % p.m_tiles, nt = tile / p.m_tiles;
+      int mt, nt;
+      tile_of(p, tile, &mt, &nt);
       const int acc = local % p.nbuf;
       const unsigned acc_phase = (unsigned)(local / p.nbuf) & 1u;
       if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag)) { ok = false; break; }
@@ -1166,6 +1192,14 @@ cudaError_t launch_gemm_pair(const DevInfo& dv, const bf16* A, int lda, const bf
     }
   }
   p.tn = (((M + p.m_tiles - 1) / p.m_tiles) + 15) / 16 * 16;
+  // Token tiles in groups once the activation matrix no longer fits L2 beside the weight stream (measured in
+  // power-capped loops: neutral or slightly slower up to ~6 k tokens of K = 3584, then QKV / O +5-8 % at 8735 tokens
+  // and +27-34 % from 16384 on, gate/up +11 % and down +9 % at 16384; group sizes 4-16 within 2 %).
+  // BS_GEMM_MGROUP: -1 automatic, 0 off, n that many token tiles per group.
+  static const int mgroup_env = env_int("BS_GEMM_MGROUP", -1);
+  int mgroup = mgroup_env;
+  if (mgroup < 0) mgroup = (size_t)M * K * sizeof(bf16) > ((size_t)56 << 20) ? (dual ? 12 : 8) : 0;
+  p.mgroup = mgroup > 0 && p.m_tiles > mgroup ? mgroup : 0;
   p.nbuf = ((dual || p.wide) && p.tn > 128) ? 1 : 2;
   p.acc1_off = p.nbuf == 1 ? 256 : 128;
   p.kblocks = (K + BK - 1) / BK;
@@ -1335,6 +1369,7 @@ cudaError_t launch_gemm_tc(const bf16* A, int lda, const bf16* W, const bf16* W2
   GemmParams p;
   p.M = M; p.N = N; p.K = K; p.mode = mode; p.dual = dual; p.C = C; p.ldc = ldc; p.row_scale = row_scale;
   p.n_tiles = (N + TILE_N - 1) / TILE_N;
+  p.mgroup = 0;
   p.error_flag = scratch.error_flag;
   p.conf_ms = conf ? conf->ms : nullptr; p.conf_am = conf ? conf->am : nullptr; p.skip = conf ? conf->skip : -1;
   p.vec_store = (ldc % 8 == 0 && N % 8 == 0 && ((uintptr_t)C & 15) == 0) ? 1 : 0;
