@@ -30,7 +30,9 @@ GEMM_SHAPES = [  # M, N, K: several tiles, ragged tails in every dimension, one 
     (517, 704, 256), (64, 4608, 512), (1000, 512, 2048), (459, 768, 256), (459, 256, 704), (48, 384, 128),
     (200, 640, 320),
     # more 256-row weight tiles than CTA pairs with a ragged last round: the SwiGLU plan narrows its token tiles
-    (1760, 12288, 128)]
+    (1760, 12288, 128),
+    # activations beyond the L2 budget: token tiles taken in groups (36 token tiles, groups of 8 or 12, ragged last group)
+    (9000, 512, 3584)]
 
 
 @pytest.mark.parametrize("M,N,K", GEMM_SHAPES)
