@@ -31,7 +31,7 @@ GEMM_SHAPES = [  # M, N, K: several tiles, ragged tails in every dimension, one 
     (200, 640, 320),
     # more 256-row weight tiles than CTA pairs with a ragged last round: the SwiGLU plan narrows its token tiles
     (1760, 12288, 128),
-    # activations beyond the L2 budget: token tiles taken in groups (36 token tiles, groups of 8 or 12, ragged last group)
+    # activations beyond the L2 budget: token tiles taken in groups (36 token tiles, groups of 8 or 16, ragged last group)
     (9000, 512, 3584)]
 
 
