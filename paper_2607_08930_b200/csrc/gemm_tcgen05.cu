@@ -1194,11 +1194,11 @@ cudaError_t launch_gemm_pair(const DevInfo& dv, const bf16* A, int lda, const bf
   p.tn = (((M + p.m_tiles - 1) / p.m_tiles) + 15) / 16 * 16;
   // Token tiles in groups once the activation matrix no longer fits L2 beside the weight stream (measured in
   // power-capped loops: neutral or slightly slower up to ~6 k tokens of K = 3584, then QKV / O +5-8 % at 8735 tokens
-  // and +27-34 % from 16384 on, gate/up +11 % and down +9 % at 16384; group sizes 4-16 within 2 %, 16 best for gate/up).
+  // and +27-34 % from 16384 on, gate/up +11 % and down +9 % at 16384; group sizes 4-16 within 2 %, 16 best for gate/up and the LM head, whose weights are the larger stream).
   // BS_GEMM_MGROUP: -1 automatic, 0 off, n that many token tiles per group.
   static const int mgroup_env = env_int("BS_GEMM_MGROUP", -1);
   int mgroup = mgroup_env;
-  if (mgroup < 0) mgroup = (size_t)M * K * sizeof(bf16) > ((size_t)56 << 20) ? (dual ? 16 : 8) : 0;
+  if (mgroup < 0) mgroup = (size_t)M * K * sizeof(bf16) > ((size_t)56 << 20) ? ((dual || N >= 32768) ? 16 : 8) : 0;
   p.mgroup = mgroup > 0 && p.m_tiles > mgroup ? mgroup : 0;
   p.nbuf = ((dual || p.wide) && p.tn > 128) ? 1 : 2;
   p.acc1_off = p.nbuf == 1 ? 256 : 128;
