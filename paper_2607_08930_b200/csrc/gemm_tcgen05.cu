@@ -1006,7 +1006,7 @@ bool get_map(const bf16* ptr, long long rows, long long cols, long long ld, int 
 // Plan overrides for measurements (environment, read once per process; the defaults are the measured best).
 struct Tuning {
   int pair;         // BS_GEMM_PAIR: -1 automatic, 0 single-CTA kernel only, n > 0 CTA pairs from n tokens
-  int pair_wide;    // BS_GEMM_PAIR_WIDE: 512-row pair items
+  int pair_wide;    // BS_GEMM_PAIR_WIDE: 512-row pair items: -1 automatic, 0 never, 1 wherever they fit
   int pair_splits;  // BS_GEMM_PAIR_SPLITS: cap of the pair kernel's k split
   int wide_off;     // BS_GEMM_WIDE=0: no 256-row items in the single-CTA kernel
   int ksub;         // BS_GEMM_KSUB: 0 automatic, 1 or 2 k sub-blocks per stage
@@ -1015,16 +1015,19 @@ struct Tuning {
   int debug;        // BS_GEMM_DEBUG: print every plan
   int no_pdl;       // BS_NO_PDL
   int ks;           // BS_GEMM_KS: -1 automatic, 0 never split K inside a cluster, 2 or 4 that many splits where they fit
+  int wide_fill;    // BS_GEMM_WIDE_FILL: per-item constant of the last-round fill cost for 512-row items (0: no fill)
+  int mgroup;       // BS_GEMM_MGROUP: token tiles per group of the work-item order: -1 automatic, 0 off
 };
 int env_int(const char* name, int dflt) {
   const char* v = getenv(name);
   return v ? atoi(v) : dflt;
 }
 const Tuning& tuning() {
-  static const Tuning t = {env_int("BS_GEMM_PAIR", -1), env_int("BS_GEMM_PAIR_WIDE", 0) > 0,
+  static const Tuning t = {env_int("BS_GEMM_PAIR", -1), env_int("BS_GEMM_PAIR_WIDE", -1),
                            env_int("BS_GEMM_PAIR_SPLITS", 8), getenv("BS_GEMM_WIDE") && env_int("BS_GEMM_WIDE", 1) == 0,
                            env_int("BS_GEMM_KSUB", 0), env_int("BS_GEMM_SPLITS", 0), env_int("BS_GEMM_STAGES", 0),
-                           getenv("BS_GEMM_DEBUG") != nullptr, getenv("BS_NO_PDL") != nullptr, env_int("BS_GEMM_KS", -1)};
+                           getenv("BS_GEMM_DEBUG") != nullptr, getenv("BS_NO_PDL") != nullptr, env_int("BS_GEMM_KS", -1),
+                           env_int("BS_GEMM_WIDE_FILL", 8), env_int("BS_GEMM_MGROUP", -1)};
   return t;
 }
 
@@ -1167,8 +1170,7 @@ cudaError_t launch_gemm_pair(const DevInfo& dv, const bf16* A, int lda, const bf
   // a refresh step runs in): the down projection (K = 18944) 2-14 % faster from 2048 tokens on, and 10-15 % with token
   // tiles narrowed to fill the last round of items (7 wide weight tiles leave 74 pairs badly divided); slower below
   // 2048 tokens and for the K = 3584 projections (3-7 %).  BS_GEMM_PAIR_WIDE: -1 automatic, 0 never, 1 wherever it fits.
-  static const int wide_mode = env_int("BS_GEMM_PAIR_WIDE", -1);
-  static const int wide_fill = env_int("BS_GEMM_WIDE_FILL", 8);      // per-item constant of the fill cost below
+  const int wide_mode = tuning().pair_wide, wide_fill = tuning().wide_fill;
   p.wide = (!dual && mode != 5 && N >= 1024 && (wide_mode > 0 || (wide_mode < 0 && K >= 8192 && M >= 2048))) ? 1 : 0;
   p.rows = p.wide ? 512 : 256;
   p.ksub = 1;
@@ -1196,8 +1198,7 @@ cudaError_t launch_gemm_pair(const DevInfo& dv, const bf16* A, int lda, const bf
   // power-capped loops: neutral or slightly slower up to ~6 k tokens of K = 3584, then QKV / O +5-8 % at 8735 tokens
   // and +27-34 % from 16384 on, gate/up +11 % and down +9 % at 16384; group sizes 4-16 within 2 %, 16 best for gate/up and the LM head, whose weights are the larger stream).
   // BS_GEMM_MGROUP: -1 automatic, 0 off, n that many token tiles per group.
-  static const int mgroup_env = env_int("BS_GEMM_MGROUP", -1);
-  int mgroup = mgroup_env;
+  int mgroup = tuning().mgroup;
   if (mgroup < 0) mgroup = (size_t)M * K * sizeof(bf16) > ((size_t)56 << 20) ? ((dual || N >= 32768) ? 16 : 8) : 0;
   p.mgroup = mgroup > 0 && p.m_tiles > mgroup ? mgroup : 0;
   p.nbuf = ((dual || p.wide) && p.tn > 128) ? 1 : 2;
