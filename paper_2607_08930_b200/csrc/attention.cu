@@ -58,15 +58,16 @@ __global__ void __launch_bounds__(256, MINB) k_attention(const bf16* __restrict_
   bf16* smem = reinterpret_cast<bf16*>(smem_raw);      // [NSTAGE][K tile, V tile][KT][LD]
   const int G = hq / hkv;
   const int kh = blockIdx.y;
-  pdl_wait();
   pdl_trigger();
-  // which row owns this q-tile: largest r with cu_tile[r] <= blockIdx.x
+  // which row owns this q-tile: largest r with cu_tile[r] <= blockIdx.x.  (The index arrays were written by the
+  // commit / scheduler kernel of the previous step: they are read before the wait for the kernel before this one.)
   const int row = warp_find_row(cu_tile, n_rows, (int)blockIdx.x);
   const int t0 = cu_q[row] + ((int)blockIdx.x - cu_tile[row]) * q_tile;
   const int nt = min(q_tile, cu_q[row + 1] - t0);
-  if (nt <= 0) return;
   const int vis = vis_arr[row];
   const size_t kvb = (size_t)kv_base[row];
+  pdl_wait();
+  if (nt <= 0) return;
   const int qkv_ld = (hq + 2 * hkv) * DH;
   // key tiles of this CTA's chunk
   const int nkt_all = (vis + KT - 1) / KT;

@@ -192,7 +192,14 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   const unsigned tmem_base = tmem_base_slot;
   volatile int* abort_flag = &s_abort;
   pdl_trigger();
-  pdl_wait();       // indices, q and the cache rows of this step come from earlier kernels of the stream
+  // The index arrays were written by the commit / scheduler kernel of the previous step, many kernels ago (the
+  // kernel before this one wrote q and the cache rows): they are read before the wait, so that the row search and
+  // its dependent loads overlap the previous kernel's tail.
+  if (threadIdx.x == 0) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_q) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_k) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_v) : "memory");
+  }
 
   // ---- which row owns this work item: largest r with cu_tile[r] <= item ----
   const int G = p.hq / p.hkv;
@@ -212,6 +219,7 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   const int per_chunk = (tiles_all + p.chunks - 1) / p.chunks;
   const int kt0 = (int)blockIdx.z * per_chunk;
   const int n_tiles = nt > 0 ? max(0, min(tiles_all, kt0 + per_chunk) - kt0) : 0;
+  pdl_wait();       // q and the cache rows of this step come from the kernel before this one
   const int n_groups = KS ? min(2, n_tiles) : n_qt;         // softmax groups with work
 
   if (warp == 0) {
