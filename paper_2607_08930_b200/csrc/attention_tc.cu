@@ -295,18 +295,25 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           umma_commit(bar(B_KVEMPTY + (t % kStages)));
         }
       } else {
-        auto issue_scores = [&](int t) -> bool {
-          if (!wait_kv(t)) return false;
-          for (int x = 0; x < n_qt; ++x) scores(stage_of(t), x, x, t & 1);
-          return true;
-        };
-        if (ok) ok = issue_scores(0);
+        // The scores run TWO tiles ahead of the P V products, one per scores buffer: S(t + 2) goes into the buffer
+        // whose probabilities P V(t) has just been issued to read (the tensor pipe runs this thread's instructions
+        // in order).  A group's softmax then finds its next scores finished when it publishes a tile, and this
+        // thread waits for probabilities only.  Traced with cycle stamps, the earlier order - S(t + 1) for both groups,
+        // then the two P V(t) - left both sides idle for a third of a tile: the scores a softmax group waited for
+        // were issued only after the other group's P V, and back-pressured issue kept this thread from looking at
+        // probabilities that had been ready for 1800 clk.
+        for (int t0s = 0; t0s < 2 && t0s < n_tiles && ok; ++t0s) {
+          ok = wait_kv(t0s);
+          for (int x = 0; x < n_qt && ok; ++x) scores(stage_of(t0s), x, x, t0s & 1);
+        }
         for (int t = 0; t < n_tiles && ok; ++t) {
-          if (t + 1 < n_tiles) ok = issue_scores(t + 1);      // next tile's scores run under this tile's softmax
-          if (!ok) break;
           for (int x = 0; x < n_qt && ok; ++x) {
             if (!mbar_wait(bar(B_PFULL + x), (unsigned)t & 1u, abort_flag)) { ok = false; break; }
             pv(stage_of(t), x, t & 1, t == 0);
+            if (t + 2 < n_tiles) {
+              if (x == 0 && !wait_kv(t + 2)) { ok = false; break; }
+              scores(stage_of(t + 2), x, x, t & 1);
+            }
           }
           if (ok) umma_commit(bar(B_KVEMPTY + (t % kStages)));
         }
