@@ -256,7 +256,9 @@ constexpr int kMaxSplits = 8;
 // Finishing kernel of the QKV projection on block steps: adds the k-split partial sums in split order, rounds q / k / v
 // to bf16, rotates q and k at the token's position id and scatters k, v to the token's cache row.
 // grid (tokens, head groups of kHeadsPerBlock); all partial loads of an element are issued before they are summed.
-constexpr int kHeadsPerBlock = 4;
+// Eight heads of 128 dims give each of the 128 threads exactly one unit of 4 rotation pairs (four heads left half of
+// the CTA idle and doubled the number of CTAs: the job measured 0.45 % slower).
+constexpr int kHeadsPerBlock = 8;
 __global__ void __launch_bounds__(128) k_finish_qkv_rope(const float* __restrict__ partial, int splits, int M,
                                                          bf16* __restrict__ qkv, const int* __restrict__ tok_pos,
                                                          const int* __restrict__ tok_kv, bf16* __restrict__ kc,
