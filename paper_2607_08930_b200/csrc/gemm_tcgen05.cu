@@ -1153,6 +1153,14 @@ cudaError_t launch_finish(const GemmParams& p, int mode, int num_sms, cudaStream
                     p.splits, p.M, p.N, mode, p.C, p.ldc, p.row_scale);
 }
 
+// The down projection of a block step with more than one token tile (k-split partial sums, K = 18944): 512-row items
+// of the pair kernel, 7 x 2 x 5 splits = 70 for 74 pairs, instead of 140 256-row items of the single-CTA kernel — a CTA
+// then loads half of each token tile (48 instead of 64 bytes per clock from L2 at the full tensor rate).
+// Measured on the Dream-7B-shaped job: +0.6 % (the steps with 288-512 packed tokens are a third of it).
+static bool pair_wide_partials(int mode, int M, int N, int K) {
+  return mode == 4 && K >= 8192 && M > 256 && N >= 1024 && tuning().pair_wide < 0;
+}
+
 // Plans and launches the CTA-pair kernel.
 cudaError_t launch_gemm_pair(const DevInfo& dv, const bf16* A, int lda, const bf16* W, const bf16* W2, void* C, int ldc,
                              int M, int N, int K, int mode, const float* row_scale, const GemmScratch& scratch,
@@ -1171,7 +1179,8 @@ cudaError_t launch_gemm_pair(const DevInfo& dv, const bf16* A, int lda, const bf
   // tiles narrowed to fill the last round of items (7 wide weight tiles leave 74 pairs badly divided); slower below
   // 2048 tokens and for the K = 3584 projections (3-7 %).  BS_GEMM_PAIR_WIDE: -1 automatic, 0 never, 1 wherever it fits.
   const int wide_mode = tuning().pair_wide, wide_fill = tuning().wide_fill;
-  p.wide = (!dual && mode != 5 && N >= 1024 && (wide_mode > 0 || (wide_mode < 0 && K >= 8192 && M >= 2048))) ? 1 : 0;
+  p.wide = (!dual && mode != 5 && N >= 1024 &&
+            (wide_mode > 0 || (wide_mode < 0 && K >= 8192 && (M >= 2048 || pair_wide_partials(mode, M, N, K))))) ? 1 : 0;
   p.rows = p.wide ? 512 : 256;
   p.ksub = 1;
   p.n_tiles = (N + p.rows - 1) / p.rows;
@@ -1354,7 +1363,8 @@ cudaError_t launch_gemm_tc(const bf16* A, int lda, const bf16* W, const bf16* W2
     else if (M >= ((mode == 2 || mode == 5) ? 64 : 128)) {     // the LM head (many weight tiles, no k split) gains from 64 on
       const bool dual_ = mode == 3 || mode == 5;      // no k split for these
       const int kb = (K + BK - 1) / BK;
-      const long long items_p = (long long)((N + 255) / 256) * ((M + 255) / 256);
+      const int rows_p = pair_wide_partials(mode, M, N, K) ? 512 : 256;
+      const long long items_p = (long long)((N + rows_p - 1) / rows_p) * ((M + 255) / 256);
       const double busy_p =
           grid_busy(items_p * split_for(items_p, dv.max_pairs, kb, (size_t)M * N, scratch, dual_), dv.max_pairs);
       const bool wide_s = mode != 3 && N >= 512 && K >= 8192;
